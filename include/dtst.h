@@ -1,0 +1,204 @@
+/*
+ * dtst.h — C ABI of the truncated spectral layer (single-GPU hot path of the
+ * Distributed Truncated Spectral Transform, DTST).
+ *
+ * The layer is  y = I( M( F(x), W ) )  with
+ *   F  forward partial DFT: only the retained modes S = S_0 x ... x S_{d-1} of a
+ *      real field are computed, one dimension at a time, by contracting with the
+ *      per-dimension basis (B_j)_{s,n} = exp(-2 pi i s (off_j + n) / N_j)
+ *      (Eq. 5, Eq. 6, Eq. 18; order of Algorithm 1 line 2);
+ *   M  per-mode complex channel mixing (Eq. 12);
+ *   I  inverse partial DFT back to the real grid (Eq. 14, B^{-1} = B^H / N),
+ *      with Hermitian doubling on the one-sided last dimension;
+ *   and the adjoint of each step for the backward pass (Section "Backward Pass").
+ *
+ * Retained set (Section "Background and Motivation"): dims 0..d-2 keep the DFT
+ * indices [0..k_j-1] followed by [N_j-k_j..N_j-1] (K_j = 2 k_j entries, ascending
+ * index); the last dim, the rfft dimension of the real input, keeps [0..k_{d-1}-1]
+ * (K_{d-1} = k_{d-1}).  M = prod K_j modes, flattened row-major.
+ *
+ * General rules for every call
+ *   - All data pointers are DEVICE pointers owned by the caller, contiguous
+ *     row-major with the last grid dimension fastest, 16-byte aligned.
+ *   - Complex values are interleaved (re, im) float pairs (float2 == complex64).
+ *   - `stream` is a cudaStream_t passed as void*; NULL means the default stream.
+ *   - Compute calls are asynchronous on `stream`, allocate nothing, and do not
+ *     synchronise.  Outputs are overwritten in full.
+ *   - Every function returns a dtst_status; nothing throws or aborts.  On error
+ *     no kernel has been launched unless the code is DTST_ERR_CUDA.
+ *   - A plan may be used from one host thread at a time.  Calls on the same
+ *     plan must be stream-ordered with respect to each other because they share
+ *     the plan's workspace.
+ */
+#ifndef DTST_H_
+#define DTST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dtst_plan dtst_plan;   /* opaque; created and destroyed by the caller */
+typedef int dtst_status;
+
+enum {
+  DTST_OK = 0,
+  DTST_ERR_INVALID_ARG = -1,     /* null/misaligned pointer, bad shape, bad option          */
+  DTST_ERR_UNSUPPORTED = -2,     /* valid request this build cannot serve                   */
+  DTST_ERR_ALLOC = -3,           /* host allocation failed                                  */
+  DTST_ERR_CUDA = -4,            /* a CUDA runtime call or launch failed                    */
+  DTST_ERR_WORKSPACE = -5,       /* workspace missing or smaller than workspace_bytes       */
+  DTST_ERR_DEVICE_TIMEOUT = -6   /* a bounded device-side wait gave up (see dtst_plan_status) */
+};
+
+#define DTST_MAX_DIMS 4
+
+/* Kernel families selectable with dtst_plan_set_kernel_path. */
+enum {
+  DTST_PATH_AUTO = 0,      /* fused streaming kernels where the shape allows, else generic */
+  DTST_PATH_GENERIC = 1    /* one generic contraction kernel per dimension                 */
+};
+
+/*
+ * Create a plan for a grid that lives entirely on the current device.
+ *   d        number of transformed dimensions, 1..DTST_MAX_DIMS
+ *   N[d]     grid extents (host array), N[d-1] contiguous in memory
+ *   kmax[d]  retained modes per dimension (host array): 1 <= k_j, 2 k_j <= N_j for
+ *            j < d-1, and k_{d-1} <= N_{d-1}/2 + 1
+ *   B, C_in, C_out  batch and channel counts (>= 1)
+ * The plan records the current CUDA device; use it with that device current.
+ * Errors: DTST_ERR_INVALID_ARG for any violated bound, DTST_ERR_ALLOC.
+ */
+dtst_status dtst_plan_create(dtst_plan** out, int d, const int64_t N[], const int32_t kmax[],
+                             int B, int C_in, int C_out);
+
+/*
+ * Create a plan for one rank's block of a distributed grid (Eq. 18): the block
+ * has extents N_local[j] and starts at global index offset[j] along each
+ * dimension; the basis carries the global phase exp(-2 pi i s (offset_j + n)/N_j).
+ * dtst_forward then yields this rank's PARTIAL spectrum (Eq. 6), which the caller
+ * sums over ranks (Eq. 7); dtst_inverse reconstructs only this rank's block.
+ * Requires 0 <= offset[j], offset[j] + N_local[j] <= N_global[j].
+ */
+dtst_status dtst_plan_create_local(dtst_plan** out, int d, const int64_t N_global[],
+                                   const int64_t N_local[], const int64_t offset[],
+                                   const int32_t kmax[], int B, int C_in, int C_out);
+
+/*
+ * Virtual shards: split the (local) grid into P slabs along dim 0, compute each
+ * slab's partial spectrum with its global phase offset and sum the P partials on
+ * the device in ascending slab order (Eq. 6-7 without a collective).  The inverse
+ * and the adjoints expand slab by slab with the same offsets.  P must divide the
+ * local extent of dim 0; P = 1 (default) turns the mode off.  Changes
+ * workspace_bytes: query it again afterwards.
+ */
+dtst_status dtst_plan_set_virtual_shards(dtst_plan* plan, int P);
+
+/* Choose the kernel family (DTST_PATH_*).  Changes workspace_bytes. */
+dtst_status dtst_plan_set_kernel_path(dtst_plan* plan, int path);
+
+/* Reports which family the plan's calls will actually run (DTST_PATH_AUTO is
+ * returned only when a fused kernel serves this shape; else DTST_PATH_GENERIC). */
+dtst_status dtst_plan_kernel_path(const dtst_plan* plan, int* path);
+
+dtst_status dtst_plan_destroy(dtst_plan* plan);
+
+/* M = number of retained modes; K[d] (host, may be NULL) = entries kept per dim. */
+dtst_status dtst_plan_num_modes(const dtst_plan* plan, int64_t* M, int64_t K[]);
+
+/* The retained DFT indices of dimension `dim`, ascending: writes K[dim] int64
+ * values to the HOST array idx.  Bit-exact contract: [0..k-1, N-k..N-1] for
+ * dim < d-1, [0..k-1] for dim = d-1. */
+dtst_status dtst_plan_mode_indices(const dtst_plan* plan, int dim, int64_t* idx);
+
+/* Scratch the compute calls need, in bytes (device memory, 256-byte aligned). */
+dtst_status dtst_plan_workspace_bytes(const dtst_plan* plan, size_t* bytes);
+
+/* Hand the plan a caller-owned device buffer of at least workspace_bytes; it must
+ * stay valid while compute calls of this plan are in flight.  The plan never
+ * frees it.  Errors: DTST_ERR_INVALID_ARG (null / not 256-byte aligned),
+ * DTST_ERR_WORKSPACE (too small). */
+dtst_status dtst_plan_set_workspace(dtst_plan* plan, void* dev_ptr, size_t bytes);
+
+/*
+ * F — forward partial DFT (Eq. 5-6, Eq. 18).
+ *   x    [B, C_in, n_0..n_{d-1}] float32 (device, read once)
+ *   Xhat [B, C_in, K_0..K_{d-1}] complex64 (device, written)
+ *   Xhat[b,c,m] = sum_n x[b,c,n] prod_j exp(-2 pi i s_j(m) (off_j + n_j) / N_j)
+ */
+dtst_status dtst_forward(dtst_plan* plan, const float* x, void* Xhat, void* stream);
+
+/*
+ * M — per-mode channel mixing (Eq. 12):
+ *   Yhat[b,o,m] = sum_i Xhat[b,i,m] * W[i,o,m]
+ *   Xhat [B, C_in, M], W [C_in, C_out, M], Yhat [B, C_out, M], all complex64.
+ * Yhat must not alias Xhat or W.
+ */
+dtst_status dtst_spectral_mul(dtst_plan* plan, const void* Xhat, const void* W, void* Yhat,
+                              void* stream);
+
+/*
+ * I — inverse partial DFT with Hermitian doubling (Eq. 14):
+ *   y[b,o,n] = (1/prod N) sum_m c(m) Re( Yhat[b,o,m] prod_j exp(+2 pi i s_j(m) (off_j+n_j)/N_j) )
+ *   c(m) = 1 if the last-dim frequency f is 0 or Nyquist (2f = N_{d-1}), else 2.
+ *   Yhat [B, C_out, M] complex64 (read), y [B, C_out, n_0..n_{d-1}] float32 (written once).
+ */
+dtst_status dtst_inverse(dtst_plan* plan, const void* Yhat, float* y, void* stream);
+
+/*
+ * B — backward pass of y = I(M(F(x), W)) for upstream gradient grad_y
+ * (Section "Backward Pass": every step is linear, so each is replaced by its adjoint):
+ *   G_Y  = (c / prod N) * F(grad_y)
+ *   G_X[b,i,m]     = sum_o G_Y[b,o,m] * conj(W[i,o,m])
+ *   grad_W[i,o,m]  = sum_b conj(Xhat_saved[b,i,m]) * G_Y[b,o,m]
+ *   grad_x[b,i,n]  = Re sum_m G_X[b,i,m] prod_j exp(+2 pi i s_j(m) (off_j+n_j)/N_j)
+ * Complex gradients follow the convention dL/dRe + i dL/dIm.
+ *   grad_y [B, C_out, n...] float32; Xhat_saved = dtst_forward's output; W as above;
+ *   grad_x [B, C_in, n...] float32 and grad_W [C_in, C_out, M] complex64 are ASSIGNED
+ *   (not accumulated); either may be NULL to skip it (not both).
+ */
+dtst_status dtst_backward(dtst_plan* plan, const float* grad_y, const void* Xhat_saved,
+                          const void* W, float* grad_x, void* grad_W, void* stream);
+
+/* Synchronises `stream` and reports the plan's device-side status word:
+ * DTST_OK, or DTST_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up
+ * (the kernel then exited normally and its output is undefined).  Clears the word. */
+dtst_status dtst_plan_status(dtst_plan* plan, void* stream);
+
+/* Number of kernel launches the plan's compute calls have issued so far. */
+dtst_status dtst_plan_launch_count(const dtst_plan* plan, int64_t* launches);
+
+/*
+ * Optional per-kernel timing for benchmarks.  When enabled, the compute calls
+ * bracket selected kernels with CUDA events on the call's stream; nothing is
+ * synchronised until the query.  `capacity` = launches recorded per kind before
+ * recording stops (events are created here, never inside a compute call);
+ * capacity 0 disables timing and frees the events.
+ * Kinds: the kernel that streams the real grid in (forward-type, used by F and by
+ * the first stage of B), the kernel that streams the real grid out (inverse-type,
+ * used by I and by the last stage of B), the mixing kernel, the mixing adjoint.
+ */
+enum {
+  DTST_KERNEL_GRID_READ = 0,
+  DTST_KERNEL_GRID_WRITE = 1,
+  DTST_KERNEL_MIX = 2,
+  DTST_KERNEL_MIX_ADJOINT = 3,
+  DTST_KERNEL_KINDS = 4
+};
+dtst_status dtst_plan_enable_kernel_timing(dtst_plan* plan, int capacity);
+
+/* Synchronises the device, then reports for `kind` the number of recorded launches and
+ * the sum of their durations in milliseconds, and resets that kind's record. */
+dtst_status dtst_plan_kernel_timing(dtst_plan* plan, int kind, int64_t* launches, double* total_ms);
+
+const char* dtst_status_string(dtst_status s);
+
+/* Library version as major*10000 + minor*100 + patch. */
+int dtst_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DTST_H_ */

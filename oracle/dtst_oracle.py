@@ -217,16 +217,21 @@ def inverse_literal(Yhat: np.ndarray, N_global, kmax) -> np.ndarray:
 # --------------------------------------------------------------------------
 # The whole layer and its backward pass (Section "Backward Pass": adjoints)
 # --------------------------------------------------------------------------
-def layer_forward(x: np.ndarray, W: np.ndarray, kmax):
-    """Returns (y, Xhat): y = I(M(F(x), W)); Xhat is what backward needs."""
-    N = x.shape[2:]
-    Xhat = forward(x, kmax)
+def layer_forward(x: np.ndarray, W: np.ndarray, kmax, N_global=None, offsets=None):
+    """Returns (y, Xhat): y = I(M(F(x), W)); Xhat is what backward needs.
+
+    With N_global/offsets, x is one rank's block: Xhat is its partial spectrum and
+    y the block of the inverse of M(Xhat) (every step is linear, Eq. 6-7).
+    """
+    n_local = x.shape[2:]
+    N = tuple(n_local) if N_global is None else tuple(N_global)
+    Xhat = forward(x, kmax, N_global=N, offsets=offsets)
     Wm = W.reshape((W.shape[0], W.shape[1]) + Xhat.shape[2:])
     Yhat = spectral_mul(Xhat, Wm)
-    return inverse(Yhat, N, kmax), Xhat
+    return inverse(Yhat, N, kmax, n_local=n_local, offsets=offsets), Xhat
 
 
-def backward(grad_y: np.ndarray, Xhat: np.ndarray, W: np.ndarray, kmax):
+def backward(grad_y: np.ndarray, Xhat: np.ndarray, W: np.ndarray, kmax, N_global=None, offsets=None):
     """Gradients of L = sum(y * grad_y) w.r.t. x and W (complex gradient = dL/dRe + i dL/dIm).
 
     G_Yhat = (c / prod N) F(grad_y)                    adjoint of the inverse
@@ -234,17 +239,19 @@ def backward(grad_y: np.ndarray, Xhat: np.ndarray, W: np.ndarray, kmax):
     G_W[i,o,m]    = sum_b conj(Xhat[b,i,m]) G_Yhat[b,o,m]
     g_x = Re sum_m G_Xhat[m] e^{+i theta_m n}           adjoint of the forward
     """
-    N = grad_y.shape[2:]
+    n_local = grad_y.shape[2:]
+    N = tuple(n_local) if N_global is None else tuple(N_global)
     B = grad_y.shape[0]
     c = hermitian_weights(N[-1], int(kmax[-1]))
-    G_Y = forward(grad_y, kmax) * c / float(math.prod(N))
+    G_Y = forward(grad_y, kmax, N_global=N, offsets=offsets) * c / float(math.prod(N))
     Ci, Co = W.shape[:2]
     Wm = W.reshape(Ci, Co, -1).astype(np.complex128)
     GYf = G_Y.reshape(B, Co, -1)
     Xf = Xhat.reshape(B, Ci, -1).astype(np.complex128)
     G_X = np.einsum("bom,iom->bim", GYf, Wm.conj())
     G_W = np.einsum("bim,bom->iom", Xf.conj(), GYf)
-    g_x = inverse(G_X.reshape((B, Ci) + G_Y.shape[2:]), N, kmax, doubling=False, normalise=False)
+    g_x = inverse(G_X.reshape((B, Ci) + G_Y.shape[2:]), N, kmax, n_local=n_local, offsets=offsets,
+                  doubling=False, normalise=False)
     return g_x, G_W.reshape(W.shape)
 
 

@@ -1,0 +1,340 @@
+"""ctypes binding of libdtst.so: argument marshalling only.
+
+Module-level functions carry the C entry points' names and take torch CUDA
+tensors where the C ABI takes device pointers.  `Plan` is a convenience wrapper
+that owns the workspace tensor and allocates outputs.  Every step of the layer
+runs in the library's CUDA kernels; there is no CPU or PyTorch fallback, and a
+missing library is a hard error.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdtst.so")
+
+DTST_OK = 0
+DTST_ERR_INVALID_ARG = -1
+DTST_ERR_UNSUPPORTED = -2
+DTST_ERR_ALLOC = -3
+DTST_ERR_CUDA = -4
+DTST_ERR_WORKSPACE = -5
+DTST_ERR_DEVICE_TIMEOUT = -6
+DTST_PATH_AUTO = 0
+DTST_PATH_GENERIC = 1
+
+# every symbol include/dtst.h declares
+EXPORTED = [
+    "dtst_plan_create", "dtst_plan_create_local", "dtst_plan_set_virtual_shards",
+    "dtst_plan_set_kernel_path", "dtst_plan_kernel_path", "dtst_plan_destroy",
+    "dtst_plan_num_modes", "dtst_plan_mode_indices", "dtst_plan_workspace_bytes",
+    "dtst_plan_set_workspace", "dtst_forward", "dtst_spectral_mul", "dtst_inverse",
+    "dtst_backward", "dtst_plan_status", "dtst_plan_launch_count", "dtst_status_string",
+    "dtst_version", "dtst_plan_enable_kernel_timing", "dtst_plan_kernel_timing",
+]
+
+
+class DtstError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libdtst.so (once).  Raises if it has not been built: no fallback exists."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2607_14394_b200.build` "
+            "(the spectral layer has no CPU or PyTorch fallback)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64p, i32p = ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int32)
+    L.dtst_plan_create.argtypes = [ctypes.POINTER(vp), i32, i64p, i32p, i32, i32, i32]
+    L.dtst_plan_create_local.argtypes = [ctypes.POINTER(vp), i32, i64p, i64p, i64p, i32p, i32, i32, i32]
+    L.dtst_plan_set_virtual_shards.argtypes = [vp, i32]
+    L.dtst_plan_set_kernel_path.argtypes = [vp, i32]
+    L.dtst_plan_kernel_path.argtypes = [vp, ctypes.POINTER(i32)]
+    L.dtst_plan_destroy.argtypes = [vp]
+    L.dtst_plan_num_modes.argtypes = [vp, i64p, i64p]
+    L.dtst_plan_mode_indices.argtypes = [vp, i32, i64p]
+    L.dtst_plan_workspace_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
+    L.dtst_plan_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+    L.dtst_forward.argtypes = [vp, vp, vp, vp]
+    L.dtst_spectral_mul.argtypes = [vp, vp, vp, vp, vp]
+    L.dtst_inverse.argtypes = [vp, vp, vp, vp]
+    L.dtst_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.dtst_plan_status.argtypes = [vp, vp]
+    L.dtst_plan_launch_count.argtypes = [vp, i64p]
+    L.dtst_plan_enable_kernel_timing.argtypes = [vp, i32]
+    L.dtst_plan_kernel_timing.argtypes = [vp, i32, i64p, ctypes.POINTER(ctypes.c_double)]
+    L.dtst_status_string.argtypes = [i32]
+    L.dtst_status_string.restype = ctypes.c_char_p
+    L.dtst_version.argtypes = []
+    for name in EXPORTED:
+        if name not in ("dtst_status_string",):
+            getattr(L, name).restype = ctypes.c_int
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().dtst_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != DTST_OK:
+        raise DtstError(status, where)
+
+
+def _i64(vals: Sequence[int]):
+    return (ctypes.c_int64 * len(vals))(*[int(v) for v in vals])
+
+
+def _i32(vals: Sequence[int]):
+    return (ctypes.c_int32 * len(vals))(*[int(v) for v in vals])
+
+
+def _ptr(t: Optional[torch.Tensor], dtype: torch.dtype, name: str) -> ctypes.c_void_p:
+    if t is None:
+        return ctypes.c_void_p(0)
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (the C ABI takes device pointers)")
+    if t.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    if isinstance(stream, torch.cuda.Stream):
+        return ctypes.c_void_p(stream.cuda_stream)
+    return ctypes.c_void_p(int(stream))
+
+
+# ------------------------------------------------------------------ C-named entry points
+def dtst_plan_create(d, N, kmax, B, C_in, C_out) -> ctypes.c_void_p:
+    h = ctypes.c_void_p(0)
+    _check(lib().dtst_plan_create(ctypes.byref(h), int(d), _i64(N), _i32(kmax), int(B), int(C_in), int(C_out)),
+           "dtst_plan_create")
+    return h
+
+
+def dtst_plan_create_local(d, N_global, N_local, offset, kmax, B, C_in, C_out) -> ctypes.c_void_p:
+    h = ctypes.c_void_p(0)
+    _check(lib().dtst_plan_create_local(ctypes.byref(h), int(d), _i64(N_global), _i64(N_local), _i64(offset),
+                                        _i32(kmax), int(B), int(C_in), int(C_out)), "dtst_plan_create_local")
+    return h
+
+
+def dtst_plan_set_virtual_shards(plan, P) -> None:
+    _check(lib().dtst_plan_set_virtual_shards(plan, int(P)), "dtst_plan_set_virtual_shards")
+
+
+def dtst_plan_set_kernel_path(plan, path) -> None:
+    _check(lib().dtst_plan_set_kernel_path(plan, int(path)), "dtst_plan_set_kernel_path")
+
+
+def dtst_plan_kernel_path(plan) -> int:
+    v = ctypes.c_int(0)
+    _check(lib().dtst_plan_kernel_path(plan, ctypes.byref(v)), "dtst_plan_kernel_path")
+    return v.value
+
+
+def dtst_plan_destroy(plan) -> None:
+    _check(lib().dtst_plan_destroy(plan), "dtst_plan_destroy")
+
+
+def dtst_plan_num_modes(plan, d):
+    M = ctypes.c_int64(0)
+    K = (ctypes.c_int64 * d)()
+    _check(lib().dtst_plan_num_modes(plan, ctypes.byref(M), K), "dtst_plan_num_modes")
+    return M.value, tuple(int(v) for v in K)
+
+
+def dtst_plan_mode_indices(plan, dim, count):
+    buf = (ctypes.c_int64 * count)()
+    _check(lib().dtst_plan_mode_indices(plan, int(dim), buf), "dtst_plan_mode_indices")
+    return [int(v) for v in buf]
+
+
+def dtst_plan_workspace_bytes(plan) -> int:
+    v = ctypes.c_size_t(0)
+    _check(lib().dtst_plan_workspace_bytes(plan, ctypes.byref(v)), "dtst_plan_workspace_bytes")
+    return int(v.value)
+
+
+def dtst_plan_set_workspace(plan, ws: torch.Tensor) -> None:
+    _check(lib().dtst_plan_set_workspace(plan, _ptr(ws, torch.uint8, "workspace"), ws.numel()),
+           "dtst_plan_set_workspace")
+
+
+def dtst_forward(plan, x, Xhat, stream=None) -> None:
+    _check(lib().dtst_forward(plan, _ptr(x, torch.float32, "x"), _ptr(Xhat, torch.complex64, "Xhat"),
+                              _stream_ptr(stream)), "dtst_forward")
+
+
+def dtst_spectral_mul(plan, Xhat, W, Yhat, stream=None) -> None:
+    _check(lib().dtst_spectral_mul(plan, _ptr(Xhat, torch.complex64, "Xhat"), _ptr(W, torch.complex64, "W"),
+                                   _ptr(Yhat, torch.complex64, "Yhat"), _stream_ptr(stream)), "dtst_spectral_mul")
+
+
+def dtst_inverse(plan, Yhat, y, stream=None) -> None:
+    _check(lib().dtst_inverse(plan, _ptr(Yhat, torch.complex64, "Yhat"), _ptr(y, torch.float32, "y"),
+                              _stream_ptr(stream)), "dtst_inverse")
+
+
+def dtst_backward(plan, grad_y, Xhat_saved, W, grad_x, grad_W, stream=None) -> None:
+    _check(lib().dtst_backward(plan, _ptr(grad_y, torch.float32, "grad_y"),
+                               _ptr(Xhat_saved, torch.complex64, "Xhat_saved"), _ptr(W, torch.complex64, "W"),
+                               _ptr(grad_x, torch.float32, "grad_x"), _ptr(grad_W, torch.complex64, "grad_W"),
+                               _stream_ptr(stream)), "dtst_backward")
+
+
+def dtst_plan_status(plan, stream=None) -> int:
+    return int(lib().dtst_plan_status(plan, _stream_ptr(stream)))
+
+
+def dtst_plan_launch_count(plan) -> int:
+    v = ctypes.c_int64(0)
+    _check(lib().dtst_plan_launch_count(plan, ctypes.byref(v)), "dtst_plan_launch_count")
+    return int(v.value)
+
+
+KERNEL_KINDS = {"grid_read": 0, "grid_write": 1, "mix": 2, "mix_adjoint": 3}
+
+
+def dtst_plan_enable_kernel_timing(plan, capacity: int) -> None:
+    _check(lib().dtst_plan_enable_kernel_timing(plan, int(capacity)), "dtst_plan_enable_kernel_timing")
+
+
+def dtst_plan_kernel_timing(plan, kind):
+    """(launches, total_ms) recorded for one kernel kind since the last query."""
+    n = ctypes.c_int64(0)
+    ms = ctypes.c_double(0.0)
+    k = KERNEL_KINDS[kind] if isinstance(kind, str) else int(kind)
+    _check(lib().dtst_plan_kernel_timing(plan, k, ctypes.byref(n), ctypes.byref(ms)), "dtst_plan_kernel_timing")
+    return int(n.value), float(ms.value)
+
+
+def dtst_version() -> int:
+    return int(lib().dtst_version())
+
+
+# ------------------------------------------------------------------ convenience wrapper
+class Plan:
+    """A truncated-spectral-layer plan plus its workspace on one CUDA device.
+
+    N: (local) grid extents, last one contiguous; kmax: retained modes per dim.
+    With N_global/offset the plan describes one rank's block (Eq. 18).
+    """
+
+    def __init__(self, N, kmax, B, C_in, C_out, N_global=None, offset=None, virtual_shards: int = 1,
+                 path: str = "auto", device=None, allocate_workspace: bool = True):
+        self.N = tuple(int(n) for n in N)
+        self.kmax = tuple(int(k) for k in kmax)
+        self.d = len(self.N)
+        self.B, self.C_in, self.C_out = int(B), int(C_in), int(C_out)
+        self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        self._h = None
+        with torch.cuda.device(self.device):
+            if N_global is None:
+                self._h = dtst_plan_create(self.d, self.N, self.kmax, B, C_in, C_out)
+            else:
+                self._h = dtst_plan_create_local(self.d, N_global, self.N, offset, self.kmax, B, C_in, C_out)
+        if path not in ("auto", "generic"):
+            raise ValueError("path must be 'auto' or 'generic'")
+        dtst_plan_set_kernel_path(self._h, DTST_PATH_AUTO if path == "auto" else DTST_PATH_GENERIC)
+        if virtual_shards != 1:
+            dtst_plan_set_virtual_shards(self._h, virtual_shards)
+        self.M, self.K = dtst_plan_num_modes(self._h, self.d)
+        self.workspace = None
+        if allocate_workspace:
+            nbytes = dtst_plan_workspace_bytes(self._h)
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            with torch.cuda.device(self.device):
+                dtst_plan_set_workspace(self._h, self.workspace)
+
+    # -- introspection
+    @property
+    def handle(self):
+        return self._h
+
+    @property
+    def kernel_path(self) -> str:
+        return "fused" if dtst_plan_kernel_path(self._h) == DTST_PATH_AUTO else "generic"
+
+    def mode_indices(self, dim: int):
+        return dtst_plan_mode_indices(self._h, dim, self.K[dim])
+
+    def workspace_bytes(self) -> int:
+        return dtst_plan_workspace_bytes(self._h)
+
+    def launch_count(self) -> int:
+        return dtst_plan_launch_count(self._h)
+
+    def status(self, stream=None) -> int:
+        return dtst_plan_status(self._h, stream)
+
+    def enable_kernel_timing(self, capacity: int) -> None:
+        dtst_plan_enable_kernel_timing(self._h, capacity)
+
+    def kernel_timing(self, kind):
+        return dtst_plan_kernel_timing(self._h, kind)
+
+    # -- compute (outputs allocated here unless given)
+    def forward(self, x, out=None, stream=None):
+        if out is None:
+            out = torch.empty((self.B, self.C_in) + self.K, dtype=torch.complex64, device=self.device)
+        dtst_forward(self._h, x, out, stream)
+        return out
+
+    def spectral_mul(self, Xhat, W, out=None, stream=None):
+        if out is None:
+            out = torch.empty((self.B, self.C_out) + self.K, dtype=torch.complex64, device=self.device)
+        dtst_spectral_mul(self._h, Xhat, W, out, stream)
+        return out
+
+    def inverse(self, Yhat, out=None, stream=None):
+        if out is None:
+            out = torch.empty((self.B, self.C_out) + self.N, dtype=torch.float32, device=self.device)
+        dtst_inverse(self._h, Yhat, out, stream)
+        return out
+
+    def backward(self, grad_y, Xhat_saved, W, grad_x=None, grad_W=None, need_grad_x=True, need_grad_W=True,
+                 stream=None):
+        if grad_x is None and need_grad_x:
+            grad_x = torch.empty((self.B, self.C_in) + self.N, dtype=torch.float32, device=self.device)
+        if grad_W is None and need_grad_W:
+            grad_W = torch.empty((self.C_in, self.C_out, self.M), dtype=torch.complex64, device=self.device)
+        dtst_backward(self._h, grad_y, Xhat_saved, W, grad_x, grad_W, stream)
+        return grad_x, grad_W
+
+    def layer(self, x, W, Xhat=None, Yhat=None, y=None, stream=None):
+        """y = I(M(F(x), W)); returns (y, Xhat)."""
+        Xhat = self.forward(x, Xhat, stream)
+        Yhat = self.spectral_mul(Xhat, W, Yhat, stream)
+        y = self.inverse(Yhat, y, stream)
+        return y, Xhat
+
+    def close(self):
+        if self._h is not None:
+            dtst_plan_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

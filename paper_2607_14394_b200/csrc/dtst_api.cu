@@ -1,0 +1,484 @@
+// C ABI of the DTST library: plan handling, argument validation and the
+// sequencing of kernels for each call.  No arithmetic of the method lives here.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "dtst_common.cuh"
+#include "dtst_fused.cuh"
+
+using namespace dtst;
+
+namespace {
+
+inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// elements of the tensor after the forward stages d-1..j have run (complex)
+long long fwd_stage_elems(const dtst_plan* p, int j, int Cn) {
+  long long n = (long long)p->B * Cn;
+  for (int i = 0; i < j; ++i) n *= p->Nl[i];
+  for (int i = j; i < p->d; ++i) n *= p->K[i];
+  return n;
+}
+
+bool mul_overflows(long long a, long long b) {
+  if (a == 0 || b == 0) return false;
+  return a > INT64_MAX / b;
+}
+
+dtst_status create_common(dtst_plan** out, int d, const int64_t* Ng, const int64_t* Nl, const int64_t* off,
+                          const int32_t* kmax, int B, int C_in, int C_out) {
+  if (out == nullptr) return DTST_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (Ng == nullptr || kmax == nullptr || d < 1 || d > kMaxDims) return DTST_ERR_INVALID_ARG;
+  if (B < 1 || C_in < 1 || C_out < 1) return DTST_ERR_INVALID_ARG;
+  long long pts_l = 1, pts_g = 1, M = 1;
+  for (int j = 0; j < d; ++j) {
+    const long long ng = Ng[j];
+    const long long nl = Nl ? Nl[j] : ng;
+    const long long o = off ? off[j] : 0;
+    if (ng < 1 || ng > (1ll << 30) || nl < 1 || o < 0 || o + nl > ng) return DTST_ERR_INVALID_ARG;
+    const long long k = kmax[j];
+    if (k < 1) return DTST_ERR_INVALID_ARG;
+    if (j < d - 1) {
+      if (2 * k > ng) return DTST_ERR_INVALID_ARG;     // the two halves of S_j must not overlap
+    } else {
+      if (k > ng / 2 + 1) return DTST_ERR_INVALID_ARG; // one-sided: at most up to Nyquist
+    }
+    const long long K = (j < d - 1) ? 2 * k : k;
+    if (mul_overflows(pts_l, nl) || mul_overflows(pts_g, ng) || mul_overflows(M, K)) return DTST_ERR_INVALID_ARG;
+    pts_l *= nl;
+    pts_g *= ng;
+    M *= K;
+  }
+  const long long cmax = C_in > C_out ? C_in : C_out;
+  if (mul_overflows(pts_l, (long long)B * cmax) || pts_l * B * cmax > (1ll << 46)) return DTST_ERR_INVALID_ARG;
+  if (mul_overflows(M, (long long)C_in * C_out) || M * C_in * C_out > (1ll << 46)) return DTST_ERR_INVALID_ARG;
+
+  dtst_plan* p = new (std::nothrow) dtst_plan;
+  if (p == nullptr) return DTST_ERR_ALLOC;
+  std::memset(p, 0, sizeof(*p));
+  p->d = d;
+  p->B = B;
+  p->C_in = C_in;
+  p->C_out = C_out;
+  for (int j = 0; j < d; ++j) {
+    p->Ng[j] = Ng[j];
+    p->Nl[j] = Nl ? Nl[j] : Ng[j];
+    p->off[j] = off ? off[j] : 0;
+    p->kmax[j] = kmax[j];
+    p->K[j] = (j < d - 1) ? 2 * kmax[j] : kmax[j];
+  }
+  p->M = M;
+  p->points_local = pts_l;
+  p->points_global = pts_g;
+  p->P = 1;
+  p->path_request = DTST_PATH_AUTO;
+  p->device = -1;
+  int dev = -1;
+  if (cudaGetDevice(&dev) == cudaSuccess) p->device = dev;
+  (void)cudaGetLastError();   // a machine without a GPU may still build plans (host logic only)
+  *out = p;
+  return DTST_OK;
+}
+
+bool use_fused(const dtst_plan* p) { return p->path_request == DTST_PATH_AUTO && fused_eligible(p); }
+
+DimOp make_op(const dtst_plan* p, int j, bool forward, int Cn) {
+  DimOp op;
+  std::memset(&op, 0, sizeof(op));
+  long long outer = (long long)p->B * Cn;
+  for (int i = 0; i < j; ++i) outer *= p->Nl[i];
+  long long inner = 1;
+  for (int i = j + 1; i < p->d; ++i) inner *= forward ? p->K[i] : p->K[i];
+  // forward: dims after j are already contracted (K); expand: dims after j are not yet expanded (K)
+  op.outer = outer;
+  op.inner = inner;
+  op.Q = forward ? (int)p->Nl[j] : p->K[j];
+  op.R = forward ? p->K[j] : (int)p->Nl[j];
+  op.N = (int)p->Ng[j];
+  op.k = p->kmax[j];
+  op.two_sided = (j < p->d - 1) ? 1 : 0;
+  op.offset = (int)p->off[j];
+  op.offset_step = 0;
+  op.forward = forward ? 1 : 0;
+  op.herm = 0;
+  op.scale = 1.0f;
+  op.slabs = 1;
+  op.in_outer_stride = (long long)op.Q * inner;
+  op.out_outer_stride = (long long)op.R * inner;
+  op.in_slab_stride = 0;
+  op.out_slab_stride = 0;
+  return op;
+}
+
+// Generic forward-type transform: real grid tensor -> [B*Cn, M] spectrum.
+// scale/herm are applied on the one-sided dimension's stage.
+dtst_status run_forward_generic(dtst_plan* p, const float* x, float2* Xhat, int Cn, float scale, bool herm,
+                                cudaStream_t st) {
+  const WsLayout L = ws_layout(p);
+  char* ws = static_cast<char*>(p->ws);
+  float2* buf[2] = {reinterpret_cast<float2*>(ws + L.bufA), reinterpret_cast<float2*>(ws + L.bufB)};
+  float2* partial = reinterpret_cast<float2*>(ws + L.partial);
+  const void* cur = x;
+  int flip = 0;
+  for (int j = p->d - 1; j >= 0; --j) {
+    DimOp op = make_op(p, j, true, Cn);
+    const bool in_real = (j == p->d - 1);
+    if (in_real) {
+      op.scale = scale;
+      op.herm = herm ? 1 : 0;
+    }
+    void* dst;
+    if (j == 0 && p->P > 1) {
+      // slab p contracts rows [p*nl, (p+1)*nl) of dim 0 with its own phase offset (Eq. 6, Eq. 18)
+      const int nl = (int)(p->Nl[0] / p->P);
+      op.slabs = p->P;
+      op.Q = nl;
+      op.offset_step = nl;
+      op.in_outer_stride = p->Nl[0] * op.inner;
+      op.in_slab_stride = (long long)nl * op.inner;
+      op.out_slab_stride = (long long)p->B * Cn * p->M;
+      dst = partial;
+    } else {
+      dst = (j == 0) ? static_cast<void*>(Xhat) : static_cast<void*>(buf[flip]);
+    }
+    {
+      KernelTimer kt(p, DTST_KERNEL_GRID_READ, st, in_real);
+      if (launch_apply_dim(op, in_real, false, cur, dst, st) != cudaSuccess) return DTST_ERR_CUDA;
+    }
+    ++p->launches;
+    cur = dst;
+    flip ^= 1;
+  }
+  if (p->P > 1) {
+    if (launch_reduce_partials(partial, Xhat, (long long)p->B * Cn * p->M, p->P, st) != cudaSuccess)
+      return DTST_ERR_CUDA;
+    ++p->launches;
+  }
+  return DTST_OK;
+}
+
+// Generic expansion: [B*Cn, M] spectrum -> real grid tensor.
+dtst_status run_inverse_generic(dtst_plan* p, const float2* Yhat, float* y, int Cn, float scale, bool herm,
+                                cudaStream_t st) {
+  const WsLayout L = ws_layout(p);
+  char* ws = static_cast<char*>(p->ws);
+  float2* buf[2] = {reinterpret_cast<float2*>(ws + L.bufA), reinterpret_cast<float2*>(ws + L.bufB)};
+  const void* cur = Yhat;
+  int flip = 0;
+  for (int j = 0; j < p->d; ++j) {
+    DimOp op = make_op(p, j, false, Cn);
+    const bool out_real = (j == p->d - 1);
+    if (out_real) {
+      op.scale = scale;
+      op.herm = herm ? 1 : 0;
+    }
+    if (j == 0 && p->P > 1) {
+      // slab p expands to rows [p*nl, (p+1)*nl) with the same offset phases; no reduction needed
+      const int nl = (int)(p->Nl[0] / p->P);
+      op.slabs = p->P;
+      op.R = nl;
+      op.offset_step = nl;
+      op.out_outer_stride = p->Nl[0] * op.inner;
+      op.out_slab_stride = (long long)nl * op.inner;
+    }
+    void* dst = out_real ? static_cast<void*>(y) : static_cast<void*>(buf[flip]);
+    {
+      KernelTimer kt(p, DTST_KERNEL_GRID_WRITE, st, out_real);
+      if (launch_apply_dim(op, false, out_real, cur, dst, st) != cudaSuccess) return DTST_ERR_CUDA;
+    }
+    ++p->launches;
+    cur = dst;
+    flip ^= 1;
+  }
+  return DTST_OK;
+}
+
+dtst_status check_ready(const dtst_plan* p) {
+  if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(p);
+  if (p->ws == nullptr || p->ws_bytes < L.total) return DTST_ERR_WORKSPACE;
+  return DTST_OK;
+}
+
+}  // namespace
+
+namespace dtst {
+
+WsLayout ws_layout(const dtst_plan* p) {
+  WsLayout L;
+  std::memset(&L, 0, sizeof(L));
+  const int Cn = p->C_in > p->C_out ? p->C_in : p->C_out;
+  long long a = 0, b = 0;
+  if (use_fused(p)) {
+    fused_workspace_elems(p, Cn, &a, &b);
+  } else {
+    // ping-pong buffers: the forward writes stage d-1 into A, d-2 into B, ...; the
+    // expansion writes stage 0 into A, 1 into B, ...  Both directions produce the same
+    // set of intermediate shapes, walked in opposite order.
+    int flip = 0;
+    for (int j = p->d - 1; j >= 1; --j) {
+      const long long n = fwd_stage_elems(p, j, Cn);
+      if (flip == 0) a = n > a ? n : a; else b = n > b ? n : b;
+      flip ^= 1;
+    }
+    flip = 0;
+    for (int j = 0; j < p->d - 1; ++j) {
+      const long long n = fwd_stage_elems(p, j + 1, Cn);
+      if (flip == 0) a = n > a ? n : a; else b = n > b ? n : b;
+      flip ^= 1;
+    }
+  }
+  L.szA = (size_t)a * sizeof(float2);
+  L.szB = (size_t)b * sizeof(float2);
+  L.szPartial = p->P > 1 ? (size_t)p->P * p->B * Cn * p->M * sizeof(float2) : 0;
+  L.szG = (size_t)p->B * Cn * p->M * sizeof(float2);
+  size_t o = 0;
+  L.status = o; o += kStatusBytes;
+  L.bufA = o; o += align256(L.szA);
+  L.bufB = o; o += align256(L.szB);
+  L.partial = o; o += align256(L.szPartial);
+  L.gy = o; o += align256(L.szG);
+  L.gx = o; o += align256(L.szG);
+  L.total = o;
+  return L;
+}
+
+}  // namespace dtst
+
+extern "C" {
+
+dtst_status dtst_plan_create(dtst_plan** out, int d, const int64_t N[], const int32_t kmax[], int B, int C_in,
+                             int C_out) {
+  return create_common(out, d, N, nullptr, nullptr, kmax, B, C_in, C_out);
+}
+
+dtst_status dtst_plan_create_local(dtst_plan** out, int d, const int64_t N_global[], const int64_t N_local[],
+                                   const int64_t offset[], const int32_t kmax[], int B, int C_in, int C_out) {
+  if (N_local == nullptr || offset == nullptr) {
+    if (out) *out = nullptr;
+    return DTST_ERR_INVALID_ARG;
+  }
+  return create_common(out, d, N_global, N_local, offset, kmax, B, C_in, C_out);
+}
+
+dtst_status dtst_plan_set_virtual_shards(dtst_plan* p, int P) {
+  if (p == nullptr || P < 1 || p->Nl[0] % P != 0) return DTST_ERR_INVALID_ARG;
+  p->P = P;
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_set_kernel_path(dtst_plan* p, int path) {
+  if (p == nullptr || (path != DTST_PATH_AUTO && path != DTST_PATH_GENERIC)) return DTST_ERR_INVALID_ARG;
+  p->path_request = path;
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_kernel_path(const dtst_plan* p, int* path) {
+  if (p == nullptr || path == nullptr) return DTST_ERR_INVALID_ARG;
+  *path = use_fused(p) ? DTST_PATH_AUTO : DTST_PATH_GENERIC;
+  return DTST_OK;
+}
+
+static void free_timing(dtst_plan* p) {
+  for (int kind = 0; kind < DTST_KERNEL_KINDS; ++kind)
+    for (int se = 0; se < 2; ++se) {
+      if (p->timing_ev[kind][se] != nullptr) {
+        for (int i = 0; i < p->timing_cap; ++i)
+          if (p->timing_ev[kind][se][i] != nullptr) cudaEventDestroy(p->timing_ev[kind][se][i]);
+        std::free(p->timing_ev[kind][se]);
+        p->timing_ev[kind][se] = nullptr;
+      }
+    }
+  p->timing_cap = 0;
+  std::memset(p->timing_n, 0, sizeof(p->timing_n));
+}
+
+dtst_status dtst_plan_enable_kernel_timing(dtst_plan* p, int capacity) {
+  if (p == nullptr || capacity < 0 || capacity > (1 << 16)) return DTST_ERR_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return DTST_ERR_CUDA;
+  free_timing(p);
+  if (capacity == 0) return DTST_OK;
+  p->timing_cap = capacity;
+  for (int kind = 0; kind < DTST_KERNEL_KINDS; ++kind)
+    for (int se = 0; se < 2; ++se) {
+      cudaEvent_t* arr = static_cast<cudaEvent_t*>(std::calloc((size_t)capacity, sizeof(cudaEvent_t)));
+      if (arr == nullptr) {
+        free_timing(p);
+        return DTST_ERR_ALLOC;
+      }
+      p->timing_ev[kind][se] = arr;
+      for (int i = 0; i < capacity; ++i)
+        if (cudaEventCreate(&arr[i]) != cudaSuccess) {
+          free_timing(p);
+          return DTST_ERR_CUDA;
+        }
+    }
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_kernel_timing(dtst_plan* p, int kind, int64_t* launches, double* total_ms) {
+  if (p == nullptr || kind < 0 || kind >= DTST_KERNEL_KINDS || launches == nullptr || total_ms == nullptr)
+    return DTST_ERR_INVALID_ARG;
+  *launches = 0;
+  *total_ms = 0.0;
+  if (p->timing_cap == 0) return DTST_OK;
+  if (cudaDeviceSynchronize() != cudaSuccess) return DTST_ERR_CUDA;
+  for (int i = 0; i < p->timing_n[kind]; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, p->timing_ev[kind][0][i], p->timing_ev[kind][1][i]) != cudaSuccess)
+      return DTST_ERR_CUDA;
+    *total_ms += ms;
+    ++*launches;
+  }
+  p->timing_n[kind] = 0;
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_destroy(dtst_plan* p) {
+  if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  free_timing(p);
+  delete p;
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_num_modes(const dtst_plan* p, int64_t* M, int64_t K[]) {
+  if (p == nullptr || M == nullptr) return DTST_ERR_INVALID_ARG;
+  *M = p->M;
+  if (K != nullptr)
+    for (int j = 0; j < p->d; ++j) K[j] = p->K[j];
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_mode_indices(const dtst_plan* p, int dim, int64_t* idx) {
+  if (p == nullptr || idx == nullptr || dim < 0 || dim >= p->d) return DTST_ERR_INVALID_ARG;
+  for (int r = 0; r < p->K[dim]; ++r)
+    idx[r] = mode_at(r, p->kmax[dim], (int)p->Ng[dim], dim < p->d - 1 ? 1 : 0);
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_workspace_bytes(const dtst_plan* p, size_t* bytes) {
+  if (p == nullptr || bytes == nullptr) return DTST_ERR_INVALID_ARG;
+  *bytes = ws_layout(p).total;
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_set_workspace(dtst_plan* p, void* dev_ptr, size_t bytes) {
+  if (p == nullptr || dev_ptr == nullptr || (reinterpret_cast<uintptr_t>(dev_ptr) & 255u) != 0)
+    return DTST_ERR_INVALID_ARG;
+  if (bytes < ws_layout(p).total) return DTST_ERR_WORKSPACE;
+  if (cudaMemset(dev_ptr, 0, kStatusBytes) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return DTST_ERR_CUDA;
+  }
+  p->ws = dev_ptr;
+  p->ws_bytes = bytes;
+  return DTST_OK;
+}
+
+dtst_status dtst_forward(dtst_plan* p, const float* x, void* Xhat, void* stream) {
+  dtst_status s = check_ready(p);
+  if (s != DTST_OK) return s;
+  if (x == nullptr || Xhat == nullptr || !aligned16(x) || !aligned16(Xhat)) return DTST_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (use_fused(p)) return fused_forward(p, x, static_cast<float2*>(Xhat), p->C_in, 1.0f, false, st);
+  return run_forward_generic(p, x, static_cast<float2*>(Xhat), p->C_in, 1.0f, false, st);
+}
+
+dtst_status dtst_spectral_mul(dtst_plan* p, const void* Xhat, const void* W, void* Yhat, void* stream) {
+  if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  if (Xhat == nullptr || W == nullptr || Yhat == nullptr || !aligned16(Xhat) || !aligned16(W) ||
+      !aligned16(Yhat) || Yhat == Xhat || Yhat == W)
+    return DTST_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  KernelTimer kt(p, DTST_KERNEL_MIX, st);
+  if (launch_mix(static_cast<const float2*>(Xhat), static_cast<const float2*>(W), static_cast<float2*>(Yhat),
+                 p->B, p->C_in, p->C_out, p->M, st, &p->launches) != cudaSuccess)
+    return DTST_ERR_CUDA;
+  return DTST_OK;
+}
+
+dtst_status dtst_inverse(dtst_plan* p, const void* Yhat, float* y, void* stream) {
+  dtst_status s = check_ready(p);
+  if (s != DTST_OK) return s;
+  if (Yhat == nullptr || y == nullptr || !aligned16(Yhat) || !aligned16(y)) return DTST_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const float scale = (float)(1.0 / (double)p->points_global);
+  if (use_fused(p)) return fused_inverse(p, static_cast<const float2*>(Yhat), y, p->C_out, scale, true, st);
+  return run_inverse_generic(p, static_cast<const float2*>(Yhat), y, p->C_out, scale, true, st);
+}
+
+dtst_status dtst_backward(dtst_plan* p, const float* grad_y, const void* Xhat_saved, const void* W,
+                          float* grad_x, void* grad_W, void* stream) {
+  dtst_status s = check_ready(p);
+  if (s != DTST_OK) return s;
+  if (grad_y == nullptr || Xhat_saved == nullptr || W == nullptr || (grad_x == nullptr && grad_W == nullptr))
+    return DTST_ERR_INVALID_ARG;
+  if (!aligned16(grad_y) || !aligned16(Xhat_saved) || !aligned16(W) || !aligned16(grad_x) || !aligned16(grad_W))
+    return DTST_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const WsLayout L = ws_layout(p);
+  char* ws = static_cast<char*>(p->ws);
+  float2* GY = reinterpret_cast<float2*>(ws + L.gy);
+  float2* GX = reinterpret_cast<float2*>(ws + L.gx);
+  const float scale = (float)(1.0 / (double)p->points_global);
+  // adjoint of I: G_Y = (c / prod N) F(grad_y)
+  s = use_fused(p) ? fused_forward(p, grad_y, GY, p->C_out, scale, true, st)
+                   : run_forward_generic(p, grad_y, GY, p->C_out, scale, true, st);
+  if (s != DTST_OK) return s;
+  // adjoint of M
+  {
+    KernelTimer kt(p, DTST_KERNEL_MIX_ADJOINT, st);
+    if (launch_mix_adjoint(GY, static_cast<const float2*>(Xhat_saved), static_cast<const float2*>(W),
+                           grad_x ? GX : nullptr, static_cast<float2*>(grad_W), p->B, p->C_in, p->C_out, p->M,
+                           st, &p->launches) != cudaSuccess)
+      return DTST_ERR_CUDA;
+  }
+  // adjoint of F: plain expansion, no doubling, no 1/prod N
+  if (grad_x != nullptr) {
+    s = use_fused(p) ? fused_inverse(p, GX, grad_x, p->C_in, 1.0f, false, st)
+                     : run_inverse_generic(p, GX, grad_x, p->C_in, 1.0f, false, st);
+    if (s != DTST_OK) return s;
+  }
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_status(dtst_plan* p, void* stream) {
+  if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return DTST_ERR_CUDA;
+  if (p->ws == nullptr) return DTST_OK;
+  int word = 0;
+  if (cudaMemcpy(&word, p->ws, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return DTST_ERR_CUDA;
+  if (word != 0) {
+    if (cudaMemset(p->ws, 0, kStatusBytes) != cudaSuccess) return DTST_ERR_CUDA;
+    return DTST_ERR_DEVICE_TIMEOUT;
+  }
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_launch_count(const dtst_plan* p, int64_t* launches) {
+  if (p == nullptr || launches == nullptr) return DTST_ERR_INVALID_ARG;
+  *launches = p->launches;
+  return DTST_OK;
+}
+
+const char* dtst_status_string(dtst_status s) {
+  switch (s) {
+    case DTST_OK: return "ok";
+    case DTST_ERR_INVALID_ARG: return "invalid argument";
+    case DTST_ERR_UNSUPPORTED: return "unsupported configuration";
+    case DTST_ERR_ALLOC: return "host allocation failed";
+    case DTST_ERR_CUDA: return "CUDA error";
+    case DTST_ERR_WORKSPACE: return "workspace missing or too small";
+    case DTST_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int dtst_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,138 @@
+// Shared declarations of the DTST CUDA library: the plan object, the description
+// of one per-dimension contraction, and the on-device basis generator.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/dtst.h"
+
+namespace dtst {
+
+constexpr int kMaxDims = DTST_MAX_DIMS;
+constexpr int kNumSMs = 148;                 // B200
+constexpr size_t kStatusBytes = 256;         // head of the workspace: device status word
+
+// One application of a (generated) complex matrix E[R x Q] along one dimension of
+// a tensor viewed as [slab][outer][Q][inner] -> [slab][outer][R][inner].
+//   forward (Eq. 18):  r = position in the retained list, q = local grid index,
+//                      E[r][q] = w * exp(-2 pi i s(r) (offset + q) / N)
+//   expand  (B^H):     r = local grid index, q = position in the retained list,
+//                      E[r][q] = w * exp(+2 pi i s(q) (offset + r) / N)
+// w = scale * (herm ? c(f) : 1) with c the Hermitian doubling weight of the
+// one-sided dimension (1 at f = 0 and Nyquist, else 2).
+struct DimOp {
+  long long outer, inner;
+  int Q, R;
+  int N;            // global extent of this dimension
+  int k;            // retained modes parameter
+  int two_sided;    // 1: list [0..k-1, N-k..N-1]; 0: [0..k-1]
+  int offset;       // global index of local element 0 (slab 0)
+  int offset_step;  // added per slab
+  int forward;      // 1: contraction grid -> modes; 0: expansion modes -> grid
+  int herm;         // apply c(f) (only meaningful on the one-sided dimension)
+  float scale;
+  int slabs;        // blockIdx.y range
+  long long in_outer_stride, out_outer_stride;   // in elements of the respective type
+  long long in_slab_stride, out_slab_stride;
+  int basis_in_smem;
+};
+
+// Retained DFT index at position pos of a dimension's list.
+__host__ __device__ inline int mode_at(int pos, int k, int N, int two_sided) {
+  return (!two_sided || pos < k) ? pos : N - 2 * k + pos;
+}
+
+// Hermitian doubling weight of one-sided frequency f.
+__host__ __device__ inline float herm_weight(int f, int N) {
+  return (f == 0 || 2 * f == N) ? 1.0f : 2.0f;
+}
+
+#ifdef __CUDACC__
+// exp(sign * 2 pi i * (s*n mod N) / N): the integer phase is reduced exactly before
+// any floating-point operation, then evaluated in double and rounded once.
+__device__ inline float2 twiddle(int s, long long n, int N, int sign) {
+  long long r = ((long long)s * n) % (long long)N;
+  double sn, cs;
+  sincospi(2.0 * (double)r / (double)N, &sn, &cs);
+  return make_float2((float)cs, (float)(sign > 0 ? sn : -sn));
+}
+
+__device__ inline float2 dimop_entry(const DimOp& p, int r, int q, int slab) {
+  const long long off = (long long)p.offset + (long long)slab * p.offset_step;
+  int pos = p.forward ? r : q;
+  long long n = off + (p.forward ? q : r);
+  int s = mode_at(pos, p.k, p.N, p.two_sided);
+  float2 e = twiddle(s, n, p.N, p.forward ? -1 : +1);
+  float w = p.scale * (p.herm ? herm_weight(s, p.N) : 1.0f);
+  e.x *= w;
+  e.y *= w;
+  return e;
+}
+#endif
+
+}  // namespace dtst
+
+// The plan: pure host-side configuration plus a caller-owned workspace pointer.
+struct dtst_plan {
+  int d;
+  int B, C_in, C_out;
+  long long Ng[dtst::kMaxDims];    // global extents
+  long long Nl[dtst::kMaxDims];    // local extents
+  long long off[dtst::kMaxDims];   // global offsets
+  int kmax[dtst::kMaxDims];
+  int K[dtst::kMaxDims];           // retained entries per dim
+  long long M;                     // prod K
+  long long points_local;          // prod Nl
+  long long points_global;         // prod Ng
+  int P;                           // virtual shards along dim 0
+  int path_request;                // DTST_PATH_*
+  int device;                      // CUDA device at creation, -1 if none
+  void* ws;
+  size_t ws_bytes;
+  long long launches;
+  // optional per-kernel event timing (benchmarks only)
+  int timing_cap;
+  int timing_n[DTST_KERNEL_KINDS];
+  cudaEvent_t* timing_ev[DTST_KERNEL_KINDS][2];
+};
+
+namespace dtst {
+
+struct WsLayout {
+  size_t status, bufA, bufB, partial, gy, gx, total;
+  size_t szA, szB, szPartial, szG;
+};
+
+bool fused_eligible(const dtst_plan* p);
+
+// Brackets one kernel launch with events when timing is enabled (no-ops otherwise).
+struct KernelTimer {
+  dtst_plan* p;
+  int kind, slot;
+  cudaStream_t st;
+  KernelTimer(dtst_plan* plan, int kind_, cudaStream_t st_, bool enabled = true)
+      : p(plan), kind(kind_), slot(-1), st(st_) {
+    if (enabled && p->timing_cap > 0 && p->timing_n[kind] < p->timing_cap) {
+      slot = p->timing_n[kind]++;
+      cudaEventRecord(p->timing_ev[kind][0][slot], st);
+    }
+  }
+  ~KernelTimer() {
+    if (slot >= 0) cudaEventRecord(p->timing_ev[kind][1][slot], st);
+  }
+};
+
+WsLayout ws_layout(const dtst_plan* p);
+
+// generic kernels (dtst_generic.cu)
+cudaError_t launch_apply_dim(const DimOp& op, bool in_real, bool out_real, const void* in, void* out,
+                             cudaStream_t st);
+cudaError_t launch_reduce_partials(const float2* partial, float2* out, long long n, int P, cudaStream_t st);
+cudaError_t launch_mix(const float2* X, const float2* W, float2* Y, int B, int Ci, int Co, long long M,
+                       cudaStream_t st, long long* launches);
+cudaError_t launch_mix_adjoint(const float2* GY, const float2* X, const float2* W, float2* GX, float2* GW,
+                               int B, int Ci, int Co, long long M, cudaStream_t st, long long* launches);
+
+}  // namespace dtst

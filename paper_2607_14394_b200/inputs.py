@@ -158,3 +158,63 @@ def make_spectrum(w: Workload, C: int, tag: int = 3) -> np.ndarray:
 
 def custom_workload(name, B, C_in, C_out, N, kmax, field="iid", seed=7, virtual_shards=1) -> Workload:
     return Workload(name, B, C_in, C_out, tuple(N), tuple(kmax), field, seed, virtual_shards)
+
+
+# --------------------------------------------------------------------------
+# Device-side generation for the large workloads (same recipe, torch RNG): a
+# channel is produced directly in GPU memory; callers that need it on the host
+# copy those very bits back, so both sides still see identical values.
+# --------------------------------------------------------------------------
+def make_field_channel_torch(w: Workload, b: int, c: int, device, tag: int = 0, rank: int = 0):
+    import torch
+
+    gen = torch.Generator(device=device)
+    gen.manual_seed(int(w.seed) * 1000003 + tag * 100003 + rank * 1009 + b * 131 + c)
+    N = tuple(w.N)
+    if w.field == "iid" or tag == 1:
+        return torch.randn(N, device=device, dtype=torch.float32, generator=gen)
+    d = len(N)
+    half = N[:-1] + (N[-1] // 2 + 1,)
+    xi = torch.randn(half + (2,), device=device, dtype=torch.float32, generator=gen)
+    k2 = torch.zeros(half, device=device, dtype=torch.float32)
+    for j in range(d):
+        if j < d - 1:
+            kj = torch.fft.fftfreq(N[j], device=device) * N[j]
+        else:
+            kj = torch.arange(half[-1], device=device, dtype=torch.float32)
+        shape = [1] * d
+        shape[j] = half[j]
+        k2 = k2 + kj.reshape(shape) ** 2
+    k2.view(-1)[0] = 1.0
+    amp = torch.rsqrt(k2)
+    amp.view(-1)[0] = 0.0
+    spec = torch.view_as_complex(xi) * amp
+    del xi, k2, amp
+    f = torch.fft.irfftn(spec, s=N, dim=tuple(range(d)))
+    del spec
+    f = f / f.std()
+    if w.field == "grf+noise":
+        f = f + 0.01 * torch.randn(N, device=device, dtype=torch.float32, generator=gen)
+    return f.contiguous()
+
+
+def make_field_torch(w: Workload, device, tag: int = 0, channels: int | None = None, rank: int = 0):
+    """x (tag 0, C_in channels) or the upstream gradient (tag 1, C_out channels, iid) on the device."""
+    import torch
+
+    C = channels if channels is not None else (w.C_in if tag == 0 else w.C_out)
+    out = torch.empty((w.B, C) + tuple(w.N), device=device, dtype=torch.float32)
+    for b in range(w.B):
+        for c in range(C):
+            out[b, c] = make_field_channel_torch(w, b, c, device, tag, rank)
+    return out
+
+
+def make_weights_torch(w: Workload, device, rank: int = 0):
+    import torch
+
+    gen = torch.Generator(device=device)
+    gen.manual_seed(int(w.seed) * 1000003 + 2 * 100003 + rank * 1009)
+    std = 1.0 / math.sqrt(w.C_in * w.C_out)
+    z = torch.randn((w.C_in, w.C_out, w.M, 2), device=device, dtype=torch.float32, generator=gen) * std
+    return torch.view_as_complex(z).contiguous()

@@ -1,0 +1,223 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64 oracle
+on the same seeded inputs.  Bar: rel-L2 <= 1e-5 over each whole output tensor
+(complex as two reals, compared in float64) and bit-exact mode-index tables."""
+import numpy as np
+import pytest
+
+from oracle import dtst_oracle as O
+from paper_2607_14394_b200 import inputs as I
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5
+
+
+def _plan(w, path="auto", P=1, **kw):
+    from paper_2607_14394_b200 import Plan
+    return Plan(w.N, w.kmax, w.B, w.C_in, w.C_out, virtual_shards=P, path=path, **kw)
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def run_layer_and_check(w, path="auto", P=1, check_backward=True, tol=TOL):
+    x = I.make_field(w)
+    W = I.make_weights(w)
+    g = I.make_upstream_grad(w)
+    plan = _plan(w, path, P)
+    lists = O.mode_index_lists(w.N, w.kmax)
+    for j in range(w.d):
+        assert plan.mode_indices(j) == lists[j].tolist()
+    xd, Wd, gd = _dev(x), _dev(W), _dev(g)
+    Xhat = plan.forward(xd)
+    Yhat = plan.spectral_mul(Xhat, Wd)
+    y = plan.inverse(Yhat)
+    torch.cuda.synchronize()
+    assert plan.status() == 0
+
+    X_ref = O.forward(x, w.kmax)
+    Wm = W.reshape((w.C_in, w.C_out) + w.K)
+    Y_ref = O.spectral_mul(X_ref, Wm)
+    y_ref = O.inverse(Y_ref, w.N, w.kmax)
+    errs = {
+        "Xhat": O.rel_l2(Xhat.cpu().numpy(), X_ref),
+        "Yhat": O.rel_l2(Yhat.cpu().numpy(), Y_ref),
+        "y": O.rel_l2(y.cpu().numpy(), y_ref),
+    }
+    if check_backward:
+        gx, gW = plan.backward(gd, Xhat, Wd)
+        torch.cuda.synchronize()
+        gx_ref, gW_ref = O.backward(g, X_ref, Wm, w.kmax)
+        errs["grad_x"] = O.rel_l2(gx.cpu().numpy(), gx_ref)
+        errs["grad_W"] = O.rel_l2(gW.cpu().numpy().reshape(gW_ref.shape), gW_ref)
+    for name, e in errs.items():
+        assert e <= tol, (w.name, path, P, name, e, errs)
+    plan.close()
+    return errs
+
+
+# ------------------------------------------------------------------ the benchmark's small configs, in full
+@pytest.mark.parametrize("path", ["auto", "generic"])
+def test_cfg1_2d(path):
+    run_layer_and_check(I.WORKLOADS["cfg1_2d_64"], path)
+
+
+@pytest.mark.parametrize("path", ["auto", "generic"])
+def test_cfg2_3d(path):
+    run_layer_and_check(I.WORKLOADS["cfg2_3d_64"], path)
+
+
+@pytest.mark.parametrize("path", ["auto", "generic"])
+def test_cfg3_4d(path):
+    run_layer_and_check(I.WORKLOADS["cfg3_4d_64"], path)
+
+
+# ------------------------------------------------------------------ edge shapes (generic path serves all of them)
+EDGE = [
+    # name, B, Ci, Co, N, kmax
+    ("d1_odd", 2, 3, 2, (7,), (4,)),
+    ("d1_nyquist", 1, 2, 2, (8,), (5,)),
+    ("d2_full_band", 1, 2, 3, (6, 8), (3, 5)),       # 2k = N and Nyquist
+    ("d2_k1", 2, 1, 1, (5, 6), (1, 1)),
+    ("d3_ragged", 1, 3, 2, (10, 6, 12), (2, 3, 3)),
+    ("d4_small", 1, 2, 2, (4, 6, 5, 8), (2, 1, 2, 3)),
+    ("big_batch", 6, 2, 3, (8, 16), (2, 4)),          # B > the mixing kernels' batch tile
+    ("tail_rows", 1, 5, 7, (12, 20, 36), (3, 5, 7)),  # nothing a multiple of a tile
+    ("wide_last", 1, 2, 2, (8, 8, 520), (2, 3, 9)),
+]
+
+
+@pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
+@pytest.mark.parametrize("path", ["auto", "generic"])
+def test_edge_shapes(case, path):
+    name, B, Ci, Co, N, k = case
+    run_layer_and_check(I.custom_workload(name, B, Ci, Co, N, k, seed=11), path)
+
+
+# ------------------------------------------------------------------ virtual shards (Eq. 6-7 on one GPU)
+@pytest.mark.parametrize("N,k,P", [((16, 8, 12), (3, 2, 4), 4), ((16, 8, 12), (3, 2, 4), 16),
+                                   ((64, 64), (8, 8), 8), ((8,), (3,), 2),
+                                   ((64, 32, 32, 16), (8, 4, 4, 4), 8)])
+@pytest.mark.parametrize("path", ["auto", "generic"])
+def test_virtual_shards_match_oracle_and_unsharded(N, k, P, path):
+    w = I.custom_workload("shards", 2, 2, 3, N, k, field="grf", seed=23)
+    run_layer_and_check(w, path, P=P)
+    x = _dev(I.make_field(w))
+    a = _plan(w, path, 1).forward(x)
+    b = _plan(w, path, P).forward(x)
+    assert O.rel_l2(b.cpu().numpy(), a.cpu().numpy()) <= TOL
+    # and the slab partial sums agree with the oracle's sharded statement
+    ref = O.forward_sharded(I.make_field(w), w.kmax, P)
+    assert O.rel_l2(b.cpu().numpy(), ref) <= TOL
+
+
+# ------------------------------------------------------------------ a rank's block with global offsets (Eq. 18)
+@pytest.mark.parametrize("path", ["auto", "generic"])
+def test_local_block_plan_gives_partial_spectrum_and_block_inverse(path):
+    from paper_2607_14394_b200 import Plan
+    Ng, k = (16, 12, 8), (3, 2, 4)
+    w = I.custom_workload("local", 1, 2, 2, Ng, k, seed=31)
+    x = I.make_field(w)
+    nl, off = (4, 6, 8), (8, 6, 0)
+    blk = np.ascontiguousarray(x[:, :, 8:12, 6:12, :])
+    plan = Plan(nl, k, 1, 2, 2, N_global=Ng, offset=off, path=path)
+    part = plan.forward(_dev(blk)).cpu().numpy()
+    ref = O.forward(blk, k, N_global=Ng, offsets=off)
+    assert O.rel_l2(part, ref) <= TOL
+    Y = (np.random.default_rng(3).standard_normal(ref.shape) + 1j * np.random.default_rng(4).standard_normal(ref.shape))
+    yb = plan.inverse(_dev(Y.astype(np.complex64))).cpu().numpy()
+    yref = O.inverse(Y.astype(np.complex64), Ng, k, n_local=nl, offsets=off)
+    assert O.rel_l2(yb, yref) <= TOL
+
+
+# ------------------------------------------------------------------ run-to-run determinism and buffer discipline
+@pytest.mark.parametrize("path", ["auto", "generic"])
+def test_bitwise_reproducible_and_no_out_of_bounds_writes(path):
+    w = I.custom_workload("repro", 2, 3, 3, (16, 12, 24), (3, 2, 5), seed=5)
+    from paper_2607_14394_b200 import binding as Bn
+    plan = _plan(w, path, P=4, allocate_workspace=False)
+    nbytes = plan.workspace_bytes()
+    guard = 4096
+    ws = torch.full((nbytes + 2 * guard,), 0xA5, dtype=torch.uint8, device="cuda")
+    Bn.dtst_plan_set_workspace(plan.handle, ws[guard:guard + nbytes])
+    x, Wd, g = _dev(I.make_field(w)), _dev(I.make_weights(w)), _dev(I.make_upstream_grad(w))
+
+    def padded(shape, dtype):
+        n = int(np.prod(shape))
+        pad = 64
+        buf = torch.full((n + 2 * pad,), float("nan"), dtype=dtype, device="cuda")
+        return buf, buf[pad:pad + n].view(shape), pad
+
+    outs = []
+    for _ in range(2):
+        Xb, X, pad = padded((w.B, w.C_in) + w.K, torch.complex64)
+        Yb, Y, _ = padded((w.B, w.C_out) + w.K, torch.complex64)
+        yb, y, _ = padded((w.B, w.C_out) + w.N, torch.float32)
+        gxb, gx, _ = padded((w.B, w.C_in) + w.N, torch.float32)
+        gWb, gW, _ = padded((w.C_in, w.C_out, w.M), torch.complex64)
+        plan.forward(x, X)
+        plan.spectral_mul(X, Wd, Y)
+        plan.inverse(Y, y)
+        plan.backward(g, X, Wd, gx, gW)
+        torch.cuda.synchronize()
+        for buf, view in ((Xb, X), (Yb, Y), (yb, y), (gxb, gx), (gWb, gW)):
+            flat = torch.view_as_real(buf) if buf.is_complex() else buf
+            assert torch.isnan(flat[:pad]).all() and torch.isnan(flat[-pad:]).all()
+            assert not torch.isnan(torch.view_as_real(view) if view.is_complex() else view).any()
+        outs.append([t.clone() for t in (X, Y, y, gx, gW)])
+    for a, b in zip(*outs):
+        assert torch.equal(torch.view_as_real(a) if a.is_complex() else a,
+                           torch.view_as_real(b) if b.is_complex() else b)
+    assert (ws[:guard] == 0xA5).all() and (ws[guard + nbytes:] == 0xA5).all()
+
+
+def test_argument_errors_on_device():
+    from paper_2607_14394_b200 import binding as Bn
+    w = I.custom_workload("err", 1, 2, 2, (8, 8), (2, 2))
+    plan = _plan(w)
+    x = torch.zeros((1, 2, 8, 8), device="cuda")
+    X = torch.zeros((1, 2, 4, 2), dtype=torch.complex64, device="cuda")
+    lib = Bn.lib()
+    import ctypes
+    st = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    assert lib.dtst_forward(plan.handle, ctypes.c_void_p(x.data_ptr() + 4), ctypes.c_void_p(X.data_ptr()), st) \
+        == Bn.DTST_ERR_INVALID_ARG
+    assert lib.dtst_spectral_mul(plan.handle, ctypes.c_void_p(X.data_ptr()), ctypes.c_void_p(X.data_ptr()),
+                                 ctypes.c_void_p(X.data_ptr()), st) == Bn.DTST_ERR_INVALID_ARG   # aliasing
+    assert lib.dtst_backward(plan.handle, ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(X.data_ptr()),
+                             ctypes.c_void_p(X.data_ptr()), None, None, st) == Bn.DTST_ERR_INVALID_ARG
+    small = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(Bn.DtstError) as e:
+        Bn.dtst_plan_set_workspace(plan.handle, small)
+    assert e.value.status == Bn.DTST_ERR_WORKSPACE
+    with pytest.raises(ValueError):
+        plan.forward(x.cpu())
+    assert plan.status() == 0
+    assert plan.launch_count() == 0
+    plan.forward(x)
+    assert plan.launch_count() > 0
+
+
+def test_adjoint_identity_on_device():
+    # <F x, Y> = <x, F^H Y> holds for the kernels themselves at a size the oracle need not touch
+    w = I.custom_workload("adj", 1, 2, 2, (32, 32, 64), (4, 6, 8), seed=77)
+    plan = _plan(w)
+    x = torch.randn((1, 2) + w.N, device="cuda", generator=torch.Generator("cuda").manual_seed(1))
+    Y = torch.randn((1, 2) + w.K, dtype=torch.complex64, device="cuda",
+                    generator=torch.Generator("cuda").manual_seed(2))
+    eye = torch.zeros((2, 2, w.M), dtype=torch.complex64, device="cuda")
+    eye[0, 0] = 1
+    eye[1, 1] = 1
+    Fx = plan.forward(x)
+    lhs = (Fx.conj() * Y).real.double().sum().item()
+    # backward with grad_y chosen so that G_X = Y is awkward; use the identity through grad_x of L = Re<F x, Y>
+    # grad_x = F^H Y is what dtst_backward's last stage computes from G_X; feed G_X through W = I and G_Y = Y
+    # by calling the expansion directly: inverse without doubling/scale is not exposed, so use linearity:
+    # <x, I(Y)> * prod(N) differs from <x, F^H Y> only by the doubling weights c(m).
+    c = torch.full((w.K[-1],), 2.0, device="cuda")
+    c[0] = 1.0
+    Yc = (Y / c).contiguous()
+    rhs = (x.double() * plan.inverse(Yc).double()).sum().item() * float(np.prod(w.N))
+    assert abs(lhs - rhs) <= 1e-5 * max(1.0, abs(lhs))

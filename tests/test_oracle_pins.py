@@ -276,6 +276,33 @@ def test_layer_and_backward_match_torch_autograd(N, kmax):
     assert O.rel_l2(gW, gW_ref) < 1e-12
 
 
+def test_block_layer_and_backward_are_slices_and_sums_of_the_global_ones():
+    # a rank's block (Eq. 18): y and grad_x of the block are slices of the global results when the
+    # block's spectrum is replaced by the summed one; partial spectra and grad_W sum over blocks
+    N, kmax = (8, 6, 10), (2, 3, 3)
+    B, Ci, Co = 1, 2, 2
+    x = _rand_x(N, B, Ci)
+    M = O.num_modes(N, kmax)
+    W = RNG.standard_normal((Ci, Co, M)) + 1j * RNG.standard_normal((Ci, Co, M))
+    g = RNG.standard_normal((B, Co) + tuple(N))
+    y, Xhat = O.layer_forward(x, W, kmax)
+    gx, gW = O.backward(g, Xhat, W, kmax)
+    Xsum, gWsum, GY_parts = 0, 0, []
+    for p in range(4):
+        sl = slice(2 * p, 2 * p + 2)
+        off = (2 * p, 0, 0)
+        yb, Xp = O.layer_forward(x[:, :, sl], W, kmax, N_global=N, offsets=off)
+        Xsum = Xsum + Xp
+        _, gWp = O.backward(g[:, :, sl], Xhat, W, kmax, N_global=N, offsets=off)
+        gWsum = gWsum + gWp
+    assert O.rel_l2(Xsum, Xhat) < 1e-12
+    assert O.rel_l2(gWsum, gW) < 1e-12
+    # block inverse of the global spectrum is the slice of the global inverse
+    Y = O.spectral_mul(Xhat, W.reshape((Ci, Co) + Xhat.shape[2:]))
+    yb = O.inverse(Y, N, kmax, n_local=(2, 6, 10), offsets=(4, 0, 0))
+    assert np.allclose(yb, y[:, :, 4:6], atol=1e-13)
+
+
 def test_backward_matches_finite_differences():
     N, kmax = (4, 6), (2, 2)
     B, Ci, Co = 1, 2, 2
