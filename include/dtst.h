@@ -50,7 +50,8 @@ enum {
   DTST_ERR_ALLOC = -3,           /* host allocation failed                                  */
   DTST_ERR_CUDA = -4,            /* a CUDA runtime call or launch failed                    */
   DTST_ERR_WORKSPACE = -5,       /* workspace missing or smaller than workspace_bytes       */
-  DTST_ERR_DEVICE_TIMEOUT = -6   /* a bounded device-side wait gave up (see dtst_plan_status) */
+  DTST_ERR_DEVICE_TIMEOUT = -6,  /* a bounded device-side wait gave up (see dtst_plan_status) */
+  DTST_ERR_STATIC_LIMIT = -7     /* dtst_forward_static: the plan needs more than DTST_STATIC_SCRATCH_BYTES */
 };
 
 #define DTST_MAX_DIMS 4
@@ -161,6 +162,42 @@ dtst_status dtst_inverse(dtst_plan* plan, const void* Yhat, float* y, void* stre
  */
 dtst_status dtst_backward(dtst_plan* plan, const float* grad_y, const void* Xhat_saved,
                           const void* W, float* grad_x, void* grad_W, void* stream);
+
+/*
+ * The forward partial DFT without any caller-provided or allocated scratch.
+ * (The paper has no counterpart to this call; it exists for integration reasons.)
+ *
+ * Who needs it: code that is not allowed to allocate device memory at the point
+ * where it calls the transform and has no workspace to hand over either - for
+ * example a plug-in running inside a host application that owns the whole
+ * memory pool, a real-time loop that forbids allocator calls after start-up, or
+ * a process whose device memory has been fully pre-committed by another
+ * framework.  For those callers dtst_forward is unusable, because its
+ * intermediates live in the workspace given to dtst_plan_set_workspace.
+ *
+ * This variant computes exactly what dtst_forward's generic path computes
+ * (same kernels, same order, same virtual-shard handling), but keeps the
+ * intermediates in one fixed array of DTST_STATIC_SCRATCH_BYTES that is part of
+ * the library image.  Consequences the caller must know:
+ *   - Every GPU that loads this library holds those bytes until the process exits.
+ *   - The plan needs no workspace for this call.  If its intermediates (two
+ *     stage buffers plus, with virtual shards, P partial spectra) exceed
+ *     DTST_STATIC_SCRATCH_BYTES the call launches nothing and returns
+ *     DTST_ERR_STATIC_LIMIT; use a smaller batch/channel count per call or
+ *     dtst_forward with a workspace.
+ *   - The call itself calls no cudaMalloc/cudaFree and no allocating library
+ *     routine.  The FIRST call on each device looks up the array's device
+ *     address (once per device, with that device current); make that first call
+ *     during start-up, before any stream capture.
+ *   - All calls, from all plans and streams, share the one array, which keeps
+ *     whatever the previous call left in it.  Nothing in it has to start at
+ *     zero: each intermediate is written in full before it is read.  Two calls
+ *     that overlap in time on the GPU (different streams, or different host
+ *     threads) race on it and corrupt each other's results: serialise them.
+ * Arguments and result as for dtst_forward.
+ */
+#define DTST_STATIC_SCRATCH_BYTES (8u * 1024u * 1024u)
+dtst_status dtst_forward_static(dtst_plan* plan, const float* x, void* Xhat, void* stream);
 
 /* Synchronises `stream` and reports the plan's device-side status word:
  * DTST_OK, or DTST_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up

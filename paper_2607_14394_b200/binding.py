@@ -24,6 +24,8 @@ DTST_ERR_ALLOC = -3
 DTST_ERR_CUDA = -4
 DTST_ERR_WORKSPACE = -5
 DTST_ERR_DEVICE_TIMEOUT = -6
+DTST_ERR_STATIC_LIMIT = -7
+DTST_STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
 DTST_PATH_AUTO = 0
 DTST_PATH_GENERIC = 1
 
@@ -34,7 +36,7 @@ EXPORTED = [
     "dtst_plan_num_modes", "dtst_plan_mode_indices", "dtst_plan_workspace_bytes",
     "dtst_plan_set_workspace", "dtst_forward", "dtst_spectral_mul", "dtst_inverse",
     "dtst_backward", "dtst_plan_status", "dtst_plan_launch_count", "dtst_status_string",
-    "dtst_version", "dtst_plan_enable_kernel_timing", "dtst_plan_kernel_timing",
+    "dtst_version", "dtst_plan_enable_kernel_timing", "dtst_plan_kernel_timing", "dtst_forward_static",
 ]
 
 
@@ -69,6 +71,7 @@ def lib() -> ctypes.CDLL:
     L.dtst_plan_workspace_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
     L.dtst_plan_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
     L.dtst_forward.argtypes = [vp, vp, vp, vp]
+    L.dtst_forward_static.argtypes = [vp, vp, vp, vp]
     L.dtst_spectral_mul.argtypes = [vp, vp, vp, vp, vp]
     L.dtst_inverse.argtypes = [vp, vp, vp, vp]
     L.dtst_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -185,6 +188,14 @@ def dtst_forward(plan, x, Xhat, stream=None) -> None:
                               _stream_ptr(stream)), "dtst_forward")
 
 
+def dtst_forward_static(plan, x, Xhat, stream=None) -> None:
+    """dtst_forward for callers that may not allocate: intermediates live in the library's fixed
+    device array (DTST_STATIC_SCRATCH_BYTES), shared by all calls; no workspace is needed.
+    Raises DtstError(DTST_ERR_STATIC_LIMIT) when the plan's intermediates do not fit."""
+    _check(lib().dtst_forward_static(plan, _ptr(x, torch.float32, "x"), _ptr(Xhat, torch.complex64, "Xhat"),
+                                     _stream_ptr(stream)), "dtst_forward_static")
+
+
 def dtst_spectral_mul(plan, Xhat, W, Yhat, stream=None) -> None:
     _check(lib().dtst_spectral_mul(plan, _ptr(Xhat, torch.complex64, "Xhat"), _ptr(W, torch.complex64, "W"),
                                    _ptr(Yhat, torch.complex64, "Yhat"), _stream_ptr(stream)), "dtst_spectral_mul")
@@ -298,6 +309,11 @@ class Plan:
         if out is None:
             out = torch.empty((self.B, self.C_in) + self.K, dtype=torch.complex64, device=self.device)
         dtst_forward(self._h, x, out, stream)
+        return out
+
+    def forward_static(self, x, out, stream=None):
+        """Forward partial DFT into the caller's `out` using only the library's fixed scratch."""
+        dtst_forward_static(self._h, x, out, stream)
         return out
 
     def spectral_mul(self, Xhat, W, out=None, stream=None):

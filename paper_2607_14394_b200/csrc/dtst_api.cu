@@ -475,6 +475,7 @@ const char* dtst_status_string(dtst_status s) {
     case DTST_ERR_CUDA: return "CUDA error";
     case DTST_ERR_WORKSPACE: return "workspace missing or too small";
     case DTST_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case DTST_ERR_STATIC_LIMIT: return "intermediates exceed the fixed scratch of dtst_forward_static";
     default: return "unknown status";
   }
 }
