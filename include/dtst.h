@@ -230,6 +230,10 @@ dtst_status dtst_plan_enable_kernel_timing(dtst_plan* plan, int capacity);
  * the sum of their durations in milliseconds, and resets that kind's record. */
 dtst_status dtst_plan_kernel_timing(dtst_plan* plan, int kind, int64_t* launches, double* total_ms);
 
+/* After a call returned DTST_ERR_CUDA: the CUDA runtime's error code and its text for the
+ * failing runtime call or launch of this plan (0 / "no error" otherwise).  The string is static. */
+dtst_status dtst_plan_last_cuda_error(const dtst_plan* plan, int* code, const char** text);
+
 const char* dtst_status_string(dtst_status s);
 
 /* Library version as major*10000 + minor*100 + patch. */

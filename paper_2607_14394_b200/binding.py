@@ -37,6 +37,7 @@ EXPORTED = [
     "dtst_plan_set_workspace", "dtst_forward", "dtst_spectral_mul", "dtst_inverse",
     "dtst_backward", "dtst_plan_status", "dtst_plan_launch_count", "dtst_status_string",
     "dtst_version", "dtst_plan_enable_kernel_timing", "dtst_plan_kernel_timing", "dtst_forward_static",
+    "dtst_plan_last_cuda_error",
 ]
 
 
@@ -79,6 +80,7 @@ def lib() -> ctypes.CDLL:
     L.dtst_plan_launch_count.argtypes = [vp, i64p]
     L.dtst_plan_enable_kernel_timing.argtypes = [vp, i32]
     L.dtst_plan_kernel_timing.argtypes = [vp, i32, i64p, ctypes.POINTER(ctypes.c_double)]
+    L.dtst_plan_last_cuda_error.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_char_p)]
     L.dtst_status_string.argtypes = [i32]
     L.dtst_status_string.restype = ctypes.c_char_p
     L.dtst_version.argtypes = []
@@ -93,9 +95,19 @@ def status_string(status: int) -> str:
     return lib().dtst_status_string(int(status)).decode()
 
 
-def _check(status: int, where: str) -> None:
+def _check(status: int, where: str, plan=None) -> None:
     if status != DTST_OK:
+        if status == DTST_ERR_CUDA and plan is not None:
+            code, text = dtst_plan_last_cuda_error(plan)
+            where = f"{where} [cuda error {code}: {text}]"
         raise DtstError(status, where)
+
+
+def dtst_plan_last_cuda_error(plan):
+    code = ctypes.c_int(0)
+    text = ctypes.c_char_p()
+    lib().dtst_plan_last_cuda_error(plan, ctypes.byref(code), ctypes.byref(text))
+    return int(code.value), (text.value or b"").decode()
 
 
 def _i64(vals: Sequence[int]):
@@ -185,7 +197,7 @@ def dtst_plan_set_workspace(plan, ws: torch.Tensor) -> None:
 
 def dtst_forward(plan, x, Xhat, stream=None) -> None:
     _check(lib().dtst_forward(plan, _ptr(x, torch.float32, "x"), _ptr(Xhat, torch.complex64, "Xhat"),
-                              _stream_ptr(stream)), "dtst_forward")
+                              _stream_ptr(stream)), "dtst_forward", plan)
 
 
 def dtst_forward_static(plan, x, Xhat, stream=None) -> None:
@@ -193,24 +205,24 @@ def dtst_forward_static(plan, x, Xhat, stream=None) -> None:
     device array (DTST_STATIC_SCRATCH_BYTES), shared by all calls; no workspace is needed.
     Raises DtstError(DTST_ERR_STATIC_LIMIT) when the plan's intermediates do not fit."""
     _check(lib().dtst_forward_static(plan, _ptr(x, torch.float32, "x"), _ptr(Xhat, torch.complex64, "Xhat"),
-                                     _stream_ptr(stream)), "dtst_forward_static")
+                                     _stream_ptr(stream)), "dtst_forward_static", plan)
 
 
 def dtst_spectral_mul(plan, Xhat, W, Yhat, stream=None) -> None:
     _check(lib().dtst_spectral_mul(plan, _ptr(Xhat, torch.complex64, "Xhat"), _ptr(W, torch.complex64, "W"),
-                                   _ptr(Yhat, torch.complex64, "Yhat"), _stream_ptr(stream)), "dtst_spectral_mul")
+                                   _ptr(Yhat, torch.complex64, "Yhat"), _stream_ptr(stream)), "dtst_spectral_mul", plan)
 
 
 def dtst_inverse(plan, Yhat, y, stream=None) -> None:
     _check(lib().dtst_inverse(plan, _ptr(Yhat, torch.complex64, "Yhat"), _ptr(y, torch.float32, "y"),
-                              _stream_ptr(stream)), "dtst_inverse")
+                              _stream_ptr(stream)), "dtst_inverse", plan)
 
 
 def dtst_backward(plan, grad_y, Xhat_saved, W, grad_x, grad_W, stream=None) -> None:
     _check(lib().dtst_backward(plan, _ptr(grad_y, torch.float32, "grad_y"),
                                _ptr(Xhat_saved, torch.complex64, "Xhat_saved"), _ptr(W, torch.complex64, "W"),
                                _ptr(grad_x, torch.float32, "grad_x"), _ptr(grad_W, torch.complex64, "grad_W"),
-                               _stream_ptr(stream)), "dtst_backward")
+                               _stream_ptr(stream)), "dtst_backward", plan)
 
 
 def dtst_plan_status(plan, stream=None) -> int:

@@ -13,6 +13,14 @@ namespace {
 
 inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
+// Records a failing CUDA call in the plan; true when the call failed.
+inline bool cuda_failed(dtst_plan* p, cudaError_t e) {
+  if (e == cudaSuccess) return false;
+  p->last_cuda_error = (int)e;
+  (void)cudaGetLastError();
+  return true;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // elements of the tensor after the forward stages d-1..j have run (complex)
@@ -114,17 +122,15 @@ DimOp make_op(const dtst_plan* p, int j, bool forward, int Cn) {
   return op;
 }
 
-// Generic forward-type transform: real grid tensor -> [B*Cn, M] spectrum.
-// scale/herm are applied on the one-sided dimension's stage.
-dtst_status run_forward_generic(dtst_plan* p, const float* x, float2* Xhat, int Cn, float scale, bool herm,
-                                cudaStream_t st) {
+// Forward stages j_from..0 on `cur` (real iff j_from is the last dimension), ping-ponging through the
+// workspace; the result lands in Xhat.  scale/herm apply on the one-sided dimension's stage only.
+dtst_status forward_stages(dtst_plan* p, const void* cur, int j_from, int flip, float2* Xhat, int Cn,
+                           float scale, bool herm, cudaStream_t st) {
   const WsLayout L = ws_layout(p);
   char* ws = static_cast<char*>(p->ws);
   float2* buf[2] = {reinterpret_cast<float2*>(ws + L.bufA), reinterpret_cast<float2*>(ws + L.bufB)};
   float2* partial = reinterpret_cast<float2*>(ws + L.partial);
-  const void* cur = x;
-  int flip = 0;
-  for (int j = p->d - 1; j >= 0; --j) {
+  for (int j = j_from; j >= 0; --j) {
     DimOp op = make_op(p, j, true, Cn);
     const bool in_real = (j == p->d - 1);
     if (in_real) {
@@ -147,18 +153,43 @@ dtst_status run_forward_generic(dtst_plan* p, const float* x, float2* Xhat, int 
     }
     {
       KernelTimer kt(p, DTST_KERNEL_GRID_READ, st, in_real);
-      if (launch_apply_dim(op, in_real, false, cur, dst, st) != cudaSuccess) return DTST_ERR_CUDA;
+      if (cuda_failed(p, launch_apply_dim(op, in_real, false, cur, dst, st))) return DTST_ERR_CUDA;
     }
     ++p->launches;
     cur = dst;
     flip ^= 1;
   }
   if (p->P > 1) {
-    if (launch_reduce_partials(partial, Xhat, (long long)p->B * Cn * p->M, p->P, st) != cudaSuccess)
-      return DTST_ERR_CUDA;
+    if (cuda_failed(p, launch_reduce_partials(partial, Xhat, (long long)p->B * Cn * p->M, p->P, st))) return DTST_ERR_CUDA;
     ++p->launches;
   }
   return DTST_OK;
+}
+
+// Generic forward-type transform: real grid tensor -> [B*Cn, M] spectrum.
+dtst_status run_forward_generic(dtst_plan* p, const float* x, float2* Xhat, int Cn, float scale, bool herm,
+                                cudaStream_t st) {
+  return forward_stages(p, x, p->d - 1, 0, Xhat, Cn, scale, herm, st);
+}
+
+// Fused forward: the plane kernel streams the grid once and contracts the last two dimensions;
+// the remaining dimensions run on the reduced tensor.
+dtst_status run_forward_fused(dtst_plan* p, const float* x, float2* Xhat, int Cn, float scale, bool herm,
+                              cudaStream_t st) {
+  const int d = p->d, a = d - 1, b = d - 2;
+  const WsLayout L = ws_layout(p);
+  char* ws = static_cast<char*>(p->ws);
+  long long planes = (long long)p->B * Cn;
+  for (int i = 0; i < b; ++i) planes *= p->Nl[i];
+  float2* t1 = (d == 2) ? Xhat : reinterpret_cast<float2*>(ws + L.bufA);
+  {
+    KernelTimer kt(p, DTST_KERNEL_GRID_READ, st);
+    if (cuda_failed(p, launch_fwd_plane((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], x, t1, planes * p->Ng[b], scale,
+                         herm ? 1 : 0, reinterpret_cast<int*>(ws + L.status), st))) return DTST_ERR_CUDA;
+  }
+  ++p->launches;
+  if (d == 2) return DTST_OK;
+  return forward_stages(p, t1, d - 3, 1, Xhat, Cn, 1.0f, false, st);
 }
 
 // Generic expansion: [B*Cn, M] spectrum -> real grid tensor.
@@ -188,7 +219,7 @@ dtst_status run_inverse_generic(dtst_plan* p, const float2* Yhat, float* y, int 
     void* dst = out_real ? static_cast<void*>(y) : static_cast<void*>(buf[flip]);
     {
       KernelTimer kt(p, DTST_KERNEL_GRID_WRITE, st, out_real);
-      if (launch_apply_dim(op, false, out_real, cur, dst, st) != cudaSuccess) return DTST_ERR_CUDA;
+      if (cuda_failed(p, launch_apply_dim(op, false, out_real, cur, dst, st))) return DTST_ERR_CUDA;
     }
     ++p->launches;
     cur = dst;
@@ -213,9 +244,7 @@ WsLayout ws_layout(const dtst_plan* p) {
   std::memset(&L, 0, sizeof(L));
   const int Cn = p->C_in > p->C_out ? p->C_in : p->C_out;
   long long a = 0, b = 0;
-  if (use_fused(p)) {
-    fused_workspace_elems(p, Cn, &a, &b);
-  } else {
+  {
     // ping-pong buffers: the forward writes stage d-1 into A, d-2 into B, ...; the
     // expansion writes stage 0 into A, 1 into B, ...  Both directions produce the same
     // set of intermediate shapes, walked in opposite order.
@@ -384,7 +413,7 @@ dtst_status dtst_forward(dtst_plan* p, const float* x, void* Xhat, void* stream)
   if (s != DTST_OK) return s;
   if (x == nullptr || Xhat == nullptr || !aligned16(x) || !aligned16(Xhat)) return DTST_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (use_fused(p)) return fused_forward(p, x, static_cast<float2*>(Xhat), p->C_in, 1.0f, false, st);
+  if (use_fused(p)) return run_forward_fused(p, x, static_cast<float2*>(Xhat), p->C_in, 1.0f, false, st);
   return run_forward_generic(p, x, static_cast<float2*>(Xhat), p->C_in, 1.0f, false, st);
 }
 
@@ -395,9 +424,8 @@ dtst_status dtst_spectral_mul(dtst_plan* p, const void* Xhat, const void* W, voi
     return DTST_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   KernelTimer kt(p, DTST_KERNEL_MIX, st);
-  if (launch_mix(static_cast<const float2*>(Xhat), static_cast<const float2*>(W), static_cast<float2*>(Yhat),
-                 p->B, p->C_in, p->C_out, p->M, st, &p->launches) != cudaSuccess)
-    return DTST_ERR_CUDA;
+  if (cuda_failed(p, launch_mix(static_cast<const float2*>(Xhat), static_cast<const float2*>(W), static_cast<float2*>(Yhat),
+                 p->B, p->C_in, p->C_out, p->M, st, &p->launches))) return DTST_ERR_CUDA;
   return DTST_OK;
 }
 
@@ -407,7 +435,6 @@ dtst_status dtst_inverse(dtst_plan* p, const void* Yhat, float* y, void* stream)
   if (Yhat == nullptr || y == nullptr || !aligned16(Yhat) || !aligned16(y)) return DTST_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const float scale = (float)(1.0 / (double)p->points_global);
-  if (use_fused(p)) return fused_inverse(p, static_cast<const float2*>(Yhat), y, p->C_out, scale, true, st);
   return run_inverse_generic(p, static_cast<const float2*>(Yhat), y, p->C_out, scale, true, st);
 }
 
@@ -426,21 +453,19 @@ dtst_status dtst_backward(dtst_plan* p, const float* grad_y, const void* Xhat_sa
   float2* GX = reinterpret_cast<float2*>(ws + L.gx);
   const float scale = (float)(1.0 / (double)p->points_global);
   // adjoint of I: G_Y = (c / prod N) F(grad_y)
-  s = use_fused(p) ? fused_forward(p, grad_y, GY, p->C_out, scale, true, st)
+  s = use_fused(p) ? run_forward_fused(p, grad_y, GY, p->C_out, scale, true, st)
                    : run_forward_generic(p, grad_y, GY, p->C_out, scale, true, st);
   if (s != DTST_OK) return s;
   // adjoint of M
   {
     KernelTimer kt(p, DTST_KERNEL_MIX_ADJOINT, st);
-    if (launch_mix_adjoint(GY, static_cast<const float2*>(Xhat_saved), static_cast<const float2*>(W),
+    if (cuda_failed(p, launch_mix_adjoint(GY, static_cast<const float2*>(Xhat_saved), static_cast<const float2*>(W),
                            grad_x ? GX : nullptr, static_cast<float2*>(grad_W), p->B, p->C_in, p->C_out, p->M,
-                           st, &p->launches) != cudaSuccess)
-      return DTST_ERR_CUDA;
+                           st, &p->launches))) return DTST_ERR_CUDA;
   }
   // adjoint of F: plain expansion, no doubling, no 1/prod N
   if (grad_x != nullptr) {
-    s = use_fused(p) ? fused_inverse(p, GX, grad_x, p->C_in, 1.0f, false, st)
-                     : run_inverse_generic(p, GX, grad_x, p->C_in, 1.0f, false, st);
+    s = run_inverse_generic(p, GX, grad_x, p->C_in, 1.0f, false, st);
     if (s != DTST_OK) return s;
   }
   return DTST_OK;
@@ -457,6 +482,13 @@ dtst_status dtst_plan_status(dtst_plan* p, void* stream) {
     if (cudaMemset(p->ws, 0, kStatusBytes) != cudaSuccess) return DTST_ERR_CUDA;
     return DTST_ERR_DEVICE_TIMEOUT;
   }
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_last_cuda_error(const dtst_plan* p, int* code, const char** text) {
+  if (p == nullptr || code == nullptr || text == nullptr) return DTST_ERR_INVALID_ARG;
+  *code = p->last_cuda_error;
+  *text = cudaGetErrorString((cudaError_t)p->last_cuda_error);
   return DTST_OK;
 }
 

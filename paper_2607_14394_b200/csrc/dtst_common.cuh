@@ -92,6 +92,7 @@ struct dtst_plan {
   void* ws;
   size_t ws_bytes;
   long long launches;
+  int last_cuda_error;             // cudaError_t of the last failing runtime call / launch
   // optional per-kernel event timing (benchmarks only)
   int timing_cap;
   int timing_n[DTST_KERNEL_KINDS];

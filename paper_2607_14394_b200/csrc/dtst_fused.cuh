@@ -1,15 +1,17 @@
-// Fused streaming kernels for the grid-side stages (declarations).
+// Fused streaming kernels for the grid-side stages (launchers).
 #pragma once
 #include "dtst_common.cuh"
 
 namespace dtst {
 
-// Workspace (in complex elements) the fused path needs for its two intermediates.
-void fused_workspace_elems(const dtst_plan* p, int Cn, long long* a, long long* b);
+// Forward plane kernel: real rows [rows][N3] (rows = planes * N2) -> out[planes][2*K2][K3] complex,
+// contracting the last two grid dimensions in one pass.  scale and the Hermitian weight (herm) are
+// applied per last-dim frequency.  `status` is the plan's device status word.
+cudaError_t launch_fwd_plane(int N3, int K3, int N2, int K2, const float* x, float2* out, long long rows,
+                             float scale, int herm, int* status, cudaStream_t st);
 
-dtst_status fused_forward(dtst_plan* p, const float* x, float2* Xhat, int Cn, float scale, bool herm,
-                          cudaStream_t st);
-dtst_status fused_inverse(dtst_plan* p, const float2* Yhat, float* y, int Cn, float scale, bool herm,
-                          cudaStream_t st);
+// Inverse plane kernel: in[planes][2*K2][K3] complex -> real rows [rows][N3].
+cudaError_t launch_inv_plane(int N3, int K3, int N2, int K2, const float2* in, float* y, long long rows,
+                             float scale, int herm, int* status, cudaStream_t st);
 
 }  // namespace dtst
