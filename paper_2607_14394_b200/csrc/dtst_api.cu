@@ -228,6 +228,55 @@ dtst_status run_inverse_generic(dtst_plan* p, const float2* Yhat, float* y, int 
   return DTST_OK;
 }
 
+// Generic expansion stages j = 0..j_to on `cur` (complex), ping-ponging through the workspace; returns
+// the buffer holding the result through *out_buf.
+dtst_status inverse_stages_complex(dtst_plan* p, const float2* cur_in, int j_to, int Cn, const float2** out_buf,
+                                   cudaStream_t st) {
+  const WsLayout L = ws_layout(p);
+  char* ws = static_cast<char*>(p->ws);
+  float2* buf[2] = {reinterpret_cast<float2*>(ws + L.bufA), reinterpret_cast<float2*>(ws + L.bufB)};
+  const void* cur = cur_in;
+  int flip = 0;
+  for (int j = 0; j <= j_to; ++j) {
+    DimOp op = make_op(p, j, false, Cn);
+    if (j == 0 && p->P > 1) {
+      const int nl = (int)(p->Nl[0] / p->P);
+      op.slabs = p->P;
+      op.R = nl;
+      op.offset_step = nl;
+      op.out_outer_stride = p->Nl[0] * op.inner;
+      op.out_slab_stride = (long long)nl * op.inner;
+    }
+    void* dst = buf[flip];
+    if (cuda_failed(p, launch_apply_dim(op, false, false, cur, dst, st))) return DTST_ERR_CUDA;
+    ++p->launches;
+    cur = dst;
+    flip ^= 1;
+  }
+  *out_buf = static_cast<const float2*>(cur);
+  return DTST_OK;
+}
+
+// Fused expansion: generic stages for dims 0..d-3 on the small tensor, then the inverse plane kernel
+// expands the last two dimensions and writes the grid once.
+dtst_status run_inverse_fused(dtst_plan* p, const float2* Yhat, float* y, int Cn, float scale, bool herm,
+                              cudaStream_t st) {
+  const int d = p->d, a = d - 1, b = d - 2;
+  const float2* src = Yhat;
+  if (d > 2) {
+    dtst_status s = inverse_stages_complex(p, Yhat, d - 3, Cn, &src, st);
+    if (s != DTST_OK) return s;
+  }
+  long long planes = (long long)p->B * Cn;
+  for (int i = 0; i < b; ++i) planes *= p->Nl[i];
+  KernelTimer kt(p, DTST_KERNEL_GRID_WRITE, st);
+  if (cuda_failed(p, launch_inv_plane((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], src, y,
+                                      planes * p->Ng[b], scale, herm ? 1 : 0, nullptr, st)))
+    return DTST_ERR_CUDA;
+  ++p->launches;
+  return DTST_OK;
+}
+
 dtst_status check_ready(const dtst_plan* p) {
   if (p == nullptr) return DTST_ERR_INVALID_ARG;
   const WsLayout L = ws_layout(p);
@@ -435,6 +484,7 @@ dtst_status dtst_inverse(dtst_plan* p, const void* Yhat, float* y, void* stream)
   if (Yhat == nullptr || y == nullptr || !aligned16(Yhat) || !aligned16(y)) return DTST_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const float scale = (float)(1.0 / (double)p->points_global);
+  if (use_fused(p)) return run_inverse_fused(p, static_cast<const float2*>(Yhat), y, p->C_out, scale, true, st);
   return run_inverse_generic(p, static_cast<const float2*>(Yhat), y, p->C_out, scale, true, st);
 }
 
@@ -465,7 +515,8 @@ dtst_status dtst_backward(dtst_plan* p, const float* grad_y, const void* Xhat_sa
   }
   // adjoint of F: plain expansion, no doubling, no 1/prod N
   if (grad_x != nullptr) {
-    s = run_inverse_generic(p, GX, grad_x, p->C_in, 1.0f, false, st);
+    s = use_fused(p) ? run_inverse_fused(p, GX, grad_x, p->C_in, 1.0f, false, st)
+                     : run_inverse_generic(p, GX, grad_x, p->C_in, 1.0f, false, st);
     if (s != DTST_OK) return s;
   }
   return DTST_OK;

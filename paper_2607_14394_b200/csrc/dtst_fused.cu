@@ -390,6 +390,253 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
 }
 
 // ---------------------------------------------------------------------------------------------
+// Inverse plane kernel: the transpose of the forward one.  in[planes][2*K2][K3] complex ->
+// real rows [planes*N2][N3].  Each warp owns a task of 128 output rows: it pre-rotates the plane's
+// modes, forms alpha_g = V'_{+g} + V'_{-g}, beta_g = i (V'_{+g} - V'_{-g}), expands them to the
+// four rows of each row quadruple (one lane per quadruple), expands every row to N3 reals with
+// the same folded basis, stages the rows in shared memory (TMA swizzle) and stores them with TMA.
+template <int N3, int K3>
+__device__ __forceinline__ void expand_row(char* stage, int box_rows, int row, const Stage1Table<N3, K3>& tab,
+                                           const float (&z)[2 * K3]) {
+  constexpr int CH = N3 / 4;
+  const uint32_t sw = (uint32_t)(row & 7);
+  char* rbase = stage + (size_t)row * 128;
+#pragma unroll
+  for (int c = 0; c < CH / 4; ++c) {
+    float a[4], b[4], cc[4], d[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int j = 4 * c + e;
+      float Ea = 0.f, Oa = 0.f, Eb = 0.f, Ob = 0.f;
+#pragma unroll
+      for (int f = 0; f < K3; ++f) {
+        if ((f & 1) == 0) {
+          Ea = fmaf(z[f], tab.cs[j][f], Ea);
+          if (f > 0) Eb = fmaf(z[K3 + f], tab.sn[j][f], Eb);
+        } else {
+          Oa = fmaf(z[f], tab.cs[j][f], Oa);
+          Ob = fmaf(z[K3 + f], tab.sn[j][f], Ob);
+        }
+      }
+      const float sa = Ea + Oa, da = Ea - Oa, sb = Eb + Ob, db = Eb - Ob;
+      a[e] = sa - sb;    // y[j]
+      d[e] = sa + sb;    // y[N3-1-j]
+      b[e] = da + db;    // y[N3/2-1-j]
+      cc[e] = da - db;   // y[N3/2+j]
+    }
+    const int c0 = c, c1 = CH / 2 - 1 - c, c2 = CH / 2 + c, c3 = CH - 1 - c;
+    *reinterpret_cast<float4*>(rbase + (size_t)(c0 / 8) * box_rows * 128 + (((uint32_t)(c0 % 8) ^ sw) << 4)) =
+        make_float4(a[0], a[1], a[2], a[3]);
+    *reinterpret_cast<float4*>(rbase + (size_t)(c1 / 8) * box_rows * 128 + (((uint32_t)(c1 % 8) ^ sw) << 4)) =
+        make_float4(b[3], b[2], b[1], b[0]);
+    *reinterpret_cast<float4*>(rbase + (size_t)(c2 / 8) * box_rows * 128 + (((uint32_t)(c2 % 8) ^ sw) << 4)) =
+        make_float4(cc[0], cc[1], cc[2], cc[3]);
+    *reinterpret_cast<float4*>(rbase + (size_t)(c3 / 8) * box_rows * 128 + (((uint32_t)(c3 % 8) ^ sw) << 4)) =
+        make_float4(d[3], d[2], d[1], d[0]);
+  }
+}
+
+template <int N3, int K3, int N2, int K2>
+struct InvCfg {
+  using P = PlaneCfg<N3, K3, N2, K2>;
+  static constexpr int ABS = P::NC + 4;                     // floats between entries
+  static constexpr int ENTRIES = 2 * K2 + 2;                // alpha_0..alpha_K2, beta_0..beta_K2 (beta_0 unused)
+  static constexpr int ABP = ENTRIES * ABS + 4;             // floats between planes (offset banks)
+  static constexpr int AB_FLOATS = ((P::G * ABP + 3) / 4) * 4;
+  static constexpr int STAGING_BYTES = kTaskRows * N3 * 4;  // 128 output rows
+  static constexpr int WARP_BYTES = STAGING_BYTES + ((AB_FLOATS * 4 + 1023) / 1024) * 1024;
+};
+
+template <int N3, int K3, int N2, int K2, int W>
+__global__ void __launch_bounds__(W * 32, 1)
+inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_constant__ Stage1Table<N3, K3> tab,
+                 const float2* __restrict__ in, long long num_tasks, float scale, int herm) {
+  using Cfg = PlaneCfg<N3, K3, N2, K2>;
+  using IC = InvCfg<N3, K3, N2, K2>;
+  constexpr int NC = Cfg::NC, QUADS = Cfg::QUADS, G = Cfg::G, LPP = Cfg::LPP;
+  constexpr int SPT = Cfg::SPT, RPS = Cfg::ROWS_PER_STAGE;
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  char* staging = reinterpret_cast<char*>(smem) + (size_t)warp * IC::WARP_BYTES;
+  float* ab = reinterpret_cast<float*>(staging + IC::STAGING_BYTES);
+  float2* rot = reinterpret_cast<float2*>(smem + (size_t)W * IC::WARP_BYTES);
+
+  if (threadIdx.x == 0) prefetch_tensormap(&out_map);
+  // conjugate rotation table: exp(-i pi (sg/N2 + f/N3)) * scale * Hermitian weight
+  for (int e = threadIdx.x; e < 2 * K2 * K3; e += blockDim.x) {
+    const int r = e / K3, f = e % K3;
+    const int sg = (r < K2) ? r : -(2 * K2 - r);
+    const long long num = (long long)sg * N3 + (long long)f * N2;
+    double sn, cs;
+    sincospi((double)num / (double)((long long)N2 * N3), &sn, &cs);
+    const float w = scale * (herm ? herm_weight(f, N3) : 1.0f);
+    rot[e] = make_float2((float)cs * w, -(float)sn * w);
+  }
+  __syncthreads();
+
+  // stage-2 role (one lane per row quadruple) and its basis values, kept in registers
+  const int pl1 = lane / QUADS, n1 = lane % QUADS;
+  float cosc[K2 + 1], sinc[K2 + 1];
+#pragma unroll
+  for (int g = 0; g <= K2; ++g) {
+    double sn, cs;
+    sincospi((double)(((long long)g * (2 * n1 + 1)) % (2 * N2)) / (double)N2, &sn, &cs);
+    cosc[g] = (float)cs;
+    sinc[g] = (float)sn;
+  }
+  // loader role: lane = (plane, mode position r)
+  const bool actl = lane < G * LPP;
+  const int pll = actl ? lane / LPP : 0, rl = lane % LPP;
+
+  const long long tstride = (long long)gridDim.x * W;
+  long long task = (long long)blockIdx.x + (long long)warp * gridDim.x;
+  float4 vin[K3 / 2];
+  if (task < num_tasks && actl) {
+    const float4* src = reinterpret_cast<const float4*>(in + ((task * G + pll) * (2 * K2) + rl) * K3);
+#pragma unroll
+    for (int i = 0; i < K3 / 2; ++i) vin[i] = __ldg(src + i);
+  }
+
+  for (; task < num_tasks; task += tstride) {
+    // ---- A. rotate this task's modes, publish V'
+    if (actl) {
+      float* dst = ab + pll * IC::ABP + rl * IC::ABS;
+      const float2* rr = rot + rl * K3;
+      float re[K3], im[K3];
+#pragma unroll
+      for (int i = 0; i < K3 / 2; ++i) {
+        const float2 r0 = rr[2 * i], r1 = rr[2 * i + 1];
+        re[2 * i] = vin[i].x * r0.x - vin[i].y * r0.y;
+        im[2 * i] = vin[i].x * r0.y + vin[i].y * r0.x;
+        re[2 * i + 1] = vin[i].z * r1.x - vin[i].w * r1.y;
+        im[2 * i + 1] = vin[i].z * r1.y + vin[i].w * r1.x;
+      }
+#pragma unroll
+      for (int i = 0; i < K3 / 4; ++i) {
+        *reinterpret_cast<float4*>(dst + 4 * i) = make_float4(re[4 * i], re[4 * i + 1], re[4 * i + 2], re[4 * i + 3]);
+        *reinterpret_cast<float4*>(dst + K3 + 4 * i) =
+            make_float4(im[4 * i], im[4 * i + 1], im[4 * i + 2], im[4 * i + 3]);
+      }
+    }
+    // prefetch the next task's modes while this one is expanded
+    {
+      const long long nt = task + tstride;
+      if (nt < num_tasks && actl) {
+        const float4* src = reinterpret_cast<const float4*>(in + ((nt * G + pll) * (2 * K2) + rl) * K3);
+#pragma unroll
+        for (int i = 0; i < K3 / 2; ++i) vin[i] = __ldg(src + i);
+      }
+    }
+    __syncwarp();
+    // ---- alpha_g = V'_{+g} + V'_{-g}, beta_g = i (V'_{+g} - V'_{-g}); lane (plane, g), g = 0..K2
+    {
+      const bool acta = lane < G * LPP && (lane % LPP) <= K2;
+      const int pla = acta ? lane / LPP : 0, g = acta ? lane % LPP : 0;
+      float vp[NC], vm[NC];
+      const float* srcp = ab + pla * IC::ABP + g * IC::ABS;
+      const float* srcm = ab + pla * IC::ABP + ((2 * K2 - g) % (2 * K2)) * IC::ABS;
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        vp[c] = (g < K2) ? srcp[c] : 0.f;
+        vm[c] = (g > 0) ? srcm[c] : 0.f;
+      }
+      __syncwarp();
+      if (acta) {
+        float* da = ab + pla * IC::ABP + g * IC::ABS;
+        float* db = ab + pla * IC::ABP + (K2 + 1 + g) * IC::ABS;
+#pragma unroll
+        for (int f = 0; f < K3; ++f) {
+          const float pr = vp[f], pi = vp[K3 + f], mr = vm[f], mi = vm[K3 + f];
+          da[f] = pr + mr;
+          da[K3 + f] = pi + mi;
+          // i * ((pr - mr) + i (pi - mi)) = -(pi - mi) + i (pr - mr)
+          db[f] = -(pi - mi);
+          db[K3 + f] = pr - mr;
+        }
+      }
+    }
+    __syncwarp();
+
+    // ---- B. expand the second dimension for this lane's row quadruple
+    float Pe[NC], Po[NC], Qe[NC], Qo[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) Pe[c] = Po[c] = Qe[c] = Qo[c] = 0.f;
+    {
+      const float* al = ab + pl1 * IC::ABP;
+      const float* be = ab + pl1 * IC::ABP + (K2 + 1) * IC::ABS;
+#pragma unroll
+      for (int g = 0; g <= K2; ++g) {
+#pragma unroll
+        for (int c4 = 0; c4 < NC / 4; ++c4) {
+          const float4 av = *reinterpret_cast<const float4*>(al + g * IC::ABS + 4 * c4);
+          if ((g & 1) == 0) {
+            Pe[4 * c4] = fmaf(cosc[g], av.x, Pe[4 * c4]);
+            Pe[4 * c4 + 1] = fmaf(cosc[g], av.y, Pe[4 * c4 + 1]);
+            Pe[4 * c4 + 2] = fmaf(cosc[g], av.z, Pe[4 * c4 + 2]);
+            Pe[4 * c4 + 3] = fmaf(cosc[g], av.w, Pe[4 * c4 + 3]);
+          } else {
+            Po[4 * c4] = fmaf(cosc[g], av.x, Po[4 * c4]);
+            Po[4 * c4 + 1] = fmaf(cosc[g], av.y, Po[4 * c4 + 1]);
+            Po[4 * c4 + 2] = fmaf(cosc[g], av.z, Po[4 * c4 + 2]);
+            Po[4 * c4 + 3] = fmaf(cosc[g], av.w, Po[4 * c4 + 3]);
+          }
+          if (g > 0) {
+            const float4 bv = *reinterpret_cast<const float4*>(be + g * IC::ABS + 4 * c4);
+            if ((g & 1) == 0) {
+              Qe[4 * c4] = fmaf(sinc[g], bv.x, Qe[4 * c4]);
+              Qe[4 * c4 + 1] = fmaf(sinc[g], bv.y, Qe[4 * c4 + 1]);
+              Qe[4 * c4 + 2] = fmaf(sinc[g], bv.z, Qe[4 * c4 + 2]);
+              Qe[4 * c4 + 3] = fmaf(sinc[g], bv.w, Qe[4 * c4 + 3]);
+            } else {
+              Qo[4 * c4] = fmaf(sinc[g], bv.x, Qo[4 * c4]);
+              Qo[4 * c4 + 1] = fmaf(sinc[g], bv.y, Qo[4 * c4 + 1]);
+              Qo[4 * c4 + 2] = fmaf(sinc[g], bv.z, Qo[4 * c4 + 2]);
+              Qo[4 * c4 + 3] = fmaf(sinc[g], bv.w, Qo[4 * c4 + 3]);
+            }
+          }
+        }
+      }
+    }
+    // the previous task's TMA stores must have finished reading the staging rows before they are rewritten
+    if (lane == 0) tma_store_wait_read<0>();
+    __syncwarp();
+
+    // ---- C/D. unfold to the four rows and expand each along the contiguous dimension
+    {
+      float z[NC];
+      const int base = pl1 * N2;
+      auto row_ptr = [&](int r) -> char* { return staging + (size_t)(r / RPS) * kStageBytes; };
+#pragma unroll
+      for (int c = 0; c < NC; ++c) z[c] = (Pe[c] + Po[c]) + (Qe[c] + Qo[c]);
+      expand_row<N3, K3>(row_ptr(base + n1), RPS, (base + n1) % RPS, tab, z);
+#pragma unroll
+      for (int c = 0; c < NC; ++c) z[c] = (Pe[c] + Po[c]) - (Qe[c] + Qo[c]);
+      expand_row<N3, K3>(row_ptr(base + N2 - 1 - n1), RPS, (base + N2 - 1 - n1) % RPS, tab, z);
+#pragma unroll
+      for (int c = 0; c < NC; ++c) z[c] = (Pe[c] - Po[c]) - (Qe[c] - Qo[c]);
+      expand_row<N3, K3>(row_ptr(base + N2 / 2 - 1 - n1), RPS, (base + N2 / 2 - 1 - n1) % RPS, tab, z);
+#pragma unroll
+      for (int c = 0; c < NC; ++c) z[c] = (Pe[c] - Po[c]) + (Qe[c] - Qo[c]);
+      expand_row<N3, K3>(row_ptr(base + N2 / 2 + n1), RPS, (base + N2 / 2 + n1) % RPS, tab, z);
+    }
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+#pragma unroll
+      for (int rb = 0; rb < SPT; ++rb)
+#pragma unroll
+        for (int h = 0; h < Cfg::BOXES; ++h)
+          tma_store_2d(&out_map, h * 32, (int)(task * kTaskRows + (long long)rb * RPS),
+                       staging + (size_t)rb * kStageBytes + (size_t)h * RPS * 128);
+      tma_store_commit();
+    }
+  }
+  if (lane == 0) tma_store_wait_all<0>();
+}
+
+// ---------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -454,9 +701,25 @@ cudaError_t launch_fwd_plane_t(const float* x, float2* out, long long rows, floa
   return cudaGetLastError();
 }
 
-struct PlaneKey {
-  int N3, K3, N2, K2;
-};
+template <int N3, int K3, int N2, int K2>
+cudaError_t launch_inv_plane_t(const float2* in, float* y, long long rows, float scale, int herm, cudaStream_t st) {
+  using IC = InvCfg<N3, K3, N2, K2>;
+  constexpr int W = (IC::WARP_BYTES * 6 + 2 * K2 * K3 * 8 + 2048 <= kSmemLimit) ? 6 : 5;
+  const size_t total = (size_t)W * IC::WARP_BYTES + (size_t)2 * K2 * K3 * 8 + 1024;
+  static_assert((size_t)W * IC::WARP_BYTES + (size_t)2 * K2 * K3 * 8 + 1024 <= kSmemLimit, "shared memory");
+  CUtensorMap map;
+  if (!make_rows_map(&map, y, rows, N3, PlaneCfg<N3, K3, N2, K2>::ROWS_PER_STAGE)) return cudaErrorNotSupported;
+  Stage1Table<N3, K3> tab;
+  fill_stage1_table(&tab);
+  auto kern = inv_plane_kernel<N3, K3, N2, K2, W>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
+  if (e != cudaSuccess) return e;
+  const long long tasks = rows / kTaskRows;
+  const long long want = (tasks + W - 1) / W;
+  const int grid = (int)(want < kNumSMs ? want : kNumSMs);
+  kern<<<grid, W * 32, total, st>>>(map, tab, in, tasks, scale, herm);
+  return cudaGetLastError();
+}
 
 }  // namespace
 
@@ -497,7 +760,11 @@ cudaError_t launch_fwd_plane(int N3, int K3, int N2, int K2, const float* x, flo
 }  // namespace dtst
 
 namespace dtst {
-cudaError_t launch_inv_plane(int, int, int, int, const float2*, float*, long long, float, int, int*, cudaStream_t) {
+cudaError_t launch_inv_plane(int N3, int K3, int N2, int K2, const float2* in, float* y, long long rows, float scale,
+                             int herm, int* /*status*/, cudaStream_t st) {
+  if (N3 == 64 && K3 == 8 && N2 == 128 && K2 == 16) return launch_inv_plane_t<64, 8, 128, 16>(in, y, rows, scale, herm, st);
+  if (N3 == 32 && K3 == 4 && N2 == 64 && K2 == 8) return launch_inv_plane_t<32, 4, 64, 8>(in, y, rows, scale, herm, st);
+  if (N3 == 64 && K3 == 8 && N2 == 64 && K2 == 8) return launch_inv_plane_t<64, 8, 64, 8>(in, y, rows, scale, herm, st);
   return cudaErrorNotSupported;
 }
 }  // namespace dtst
