@@ -379,7 +379,9 @@ def main_ours(args, w):
     # end to end through host buffers: pinned host -> device copies of x and g_y, the step,
     # device -> host reads of y, grad_x and grad_W, all inside the timed region
     e2e = None
-    if rank == 0 or world > 1:
+    if args.no_e2e:
+        e2e = {"value": None, "unit": UNIT, "skipped": "--no-e2e"}
+    elif rank == 0 or world > 1:
         try:
             e2e_steps = max(1, min(steps, args.e2e_steps))
             hx = torch.empty(x.shape, dtype=torch.float32, pin_memory=True)
@@ -477,11 +479,17 @@ def main():
     ap.add_argument("--shards", type=int, default=1, help="virtual shards along dim 0")
     ap.add_argument("--path", default="auto", choices=["auto", "generic"])
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--channels", type=int, default=0,
+                    help="override C_in = C_out (smaller cases for profiler captures; not a bench configuration)")
+    ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-torch-ref", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     from paper_2607_14394_b200 import inputs
     w = inputs.WORKLOADS[args.config]
+    if args.channels > 0:
+        w = inputs.custom_workload(f"{w.name}_c{args.channels}", w.B, args.channels, args.channels, w.N, w.kmax,
+                                   field=w.field, seed=w.seed, virtual_shards=w.virtual_shards)
     if args.impl == "reference":
         return main_reference(args, w)
     return main_ours(args, w)
