@@ -92,6 +92,15 @@ dtst_status create_common(dtst_plan** out, int d, const int64_t* Ng, const int64
   return DTST_OK;
 }
 
+// A two-sided dimension that is whole on this device, starts at global index 0 and is not cut into
+// virtual slabs can use the folded middle-dimension kernels.
+bool use_mid(const dtst_plan* p, int j) {
+  if (p->path_request != DTST_PATH_AUTO || j >= p->d - 1) return false;
+  if (p->Nl[j] != p->Ng[j] || p->off[j] != 0) return false;
+  if (j == 0 && p->P > 1) return false;
+  return mid_supported((int)p->Ng[j], p->kmax[j]);
+}
+
 bool use_fused(const dtst_plan* p) { return p->path_request == DTST_PATH_AUTO && fused_eligible(p); }
 
 DimOp make_op(const dtst_plan* p, int j, bool forward, int Cn) {
@@ -151,7 +160,11 @@ dtst_status forward_stages(dtst_plan* p, const void* cur, int j_from, int flip, 
     } else {
       dst = (j == 0) ? static_cast<void*>(Xhat) : static_cast<void*>(buf[flip]);
     }
-    {
+    if (!in_real && use_mid(p, j)) {
+      if (cuda_failed(p, launch_mid(true, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
+                                    op.outer, op.inner, op.N, 1.0f, st)))
+        return DTST_ERR_CUDA;
+    } else {
       KernelTimer kt(p, DTST_KERNEL_GRID_READ, st, in_real);
       if (cuda_failed(p, launch_apply_dim(op, in_real, false, cur, dst, st))) return DTST_ERR_CUDA;
     }
@@ -217,7 +230,11 @@ dtst_status run_inverse_generic(dtst_plan* p, const float2* Yhat, float* y, int 
       op.out_slab_stride = (long long)nl * op.inner;
     }
     void* dst = out_real ? static_cast<void*>(y) : static_cast<void*>(buf[flip]);
-    {
+    if (!out_real && use_mid(p, j)) {
+      if (cuda_failed(p, launch_mid(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
+                                    op.outer, op.inner, op.N, 1.0f, st)))
+        return DTST_ERR_CUDA;
+    } else {
       KernelTimer kt(p, DTST_KERNEL_GRID_WRITE, st, out_real);
       if (cuda_failed(p, launch_apply_dim(op, false, out_real, cur, dst, st))) return DTST_ERR_CUDA;
     }
@@ -248,7 +265,13 @@ dtst_status inverse_stages_complex(dtst_plan* p, const float2* cur_in, int j_to,
       op.out_slab_stride = (long long)nl * op.inner;
     }
     void* dst = buf[flip];
-    if (cuda_failed(p, launch_apply_dim(op, false, false, cur, dst, st))) return DTST_ERR_CUDA;
+    if (use_mid(p, j)) {
+      if (cuda_failed(p, launch_mid(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
+                                    op.outer, op.inner, op.N, 1.0f, st)))
+        return DTST_ERR_CUDA;
+    } else if (cuda_failed(p, launch_apply_dim(op, false, false, cur, dst, st))) {
+      return DTST_ERR_CUDA;
+    }
     ++p->launches;
     cur = dst;
     flip ^= 1;

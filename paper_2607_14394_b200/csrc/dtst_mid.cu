@@ -1,0 +1,265 @@
+// Contraction / expansion along a two-sided middle dimension on the already reduced
+// tensor [outer][Q][inner] (inner contiguous, complex64).
+//
+// One thread owns PT consecutive-in-memory complex positions and keeps ALL of their
+// retained-frequency sums in registers, so every input element is loaded exactly once and
+// every output written exactly once; consecutive lanes own consecutive positions, so all
+// global accesses are coalesced 8-byte-per-lane transactions.  The basis is generated on
+// the device into shared memory once per (persistent) CTA.  With the half-sample phase
+// factored out (Eq. 18 with zero offset),
+//     Z_{+-g} = e^{+-i psi_g/2} (A_g -+ i B_g),
+//     A_g = sum_{q<Q/2} (z_q + z_{Q-1-q}) cos(psi_g (q + 1/2)),
+//     B_g = sum_{q<Q/2} (z_q - z_{Q-1-q}) sin(psi_g (q + 1/2)),
+// one real-coefficient FMA pair serves both +g and -g and both mirrored inputs: a fourfold
+// cut of the multiply count against the plain complex matrix product.
+#include "dtst_common.cuh"
+
+namespace dtst {
+namespace {
+
+constexpr int kMidThreads = 128;
+
+// table[q][e]: e in [0..K] -> cos(psi_e (q+1/2)); e in [K+1..2K] -> sin(psi_{e-K} (q+1/2)); row stride TS
+template <int K>
+struct MidTab {
+  static constexpr int TS = ((2 * K + 1 + 3) / 4) * 4;
+};
+
+template <int K>
+__device__ __forceinline__ void build_mid_table(float* tab, float2* rho, int N, float scale) {
+  constexpr int TS = MidTab<K>::TS;
+  const int half = N / 2;
+  for (int e = threadIdx.x; e < half * TS; e += blockDim.x) {
+    const int q = e / TS, c = e % TS;
+    float v = 0.f;
+    if (c <= 2 * K) {
+      const int g = c <= K ? c : c - K;
+      double sn, cs;
+      // psi_g (q + 1/2) = pi g (2q+1) / N, phase reduced exactly in integers
+      sincospi((double)(((long long)g * (2 * q + 1)) % (2ll * N)) / (double)N, &sn, &cs);
+      v = c <= K ? (float)cs : (float)sn;
+    }
+    tab[e] = v;
+  }
+  for (int g = threadIdx.x; g <= K; g += blockDim.x) {
+    double sn, cs;
+    sincospi((double)g / (double)N, &sn, &cs);   // e^{i psi_g / 2}
+    rho[g] = make_float2((float)cs * scale, (float)sn * scale);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// forward: in[outer][N][inner] -> out[outer][2K][inner]
+// ------------------------------------------------------------------------------------------
+template <int K, int PT>
+__global__ void __launch_bounds__(kMidThreads) mid_contract_kernel(const float2* __restrict__ in,
+                                                                   float2* __restrict__ out, long long outer,
+                                                                   long long inner, int N, float scale) {
+  constexpr int TS = MidTab<K>::TS;
+  extern __shared__ float smem_mid[];
+  float* tab = smem_mid;
+  float2* rho = reinterpret_cast<float2*>(tab + (size_t)(N / 2) * TS);
+  build_mid_table<K>(tab, rho, N, scale);
+  __syncthreads();
+
+  const long long total = outer * inner;
+  const long long per_cta = (long long)kMidThreads * PT;
+  const long long tiles = (total + per_cta - 1) / per_cta;
+  const int half = N / 2;
+  for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    long long ibase[PT], obase[PT];
+    bool ok[PT];
+#pragma unroll
+    for (int t = 0; t < PT; ++t) {
+      const long long p = tile * per_cta + (long long)t * kMidThreads + threadIdx.x;
+      ok[t] = p < total;
+      const long long pc = ok[t] ? p : 0;
+      const long long o = pc / inner, i = pc % inner;
+      ibase[t] = o * N * inner + i;
+      obase[t] = o * (2 * K) * inner + i;
+    }
+    float2 A[PT][K + 1], B[PT][K + 1];
+#pragma unroll
+    for (int t = 0; t < PT; ++t)
+#pragma unroll
+      for (int g = 0; g <= K; ++g) A[t][g] = B[t][g] = make_float2(0.f, 0.f);
+
+#pragma unroll 2
+    for (int q = 0; q < half; ++q) {
+      float2 p[PT], m[PT];
+#pragma unroll
+      for (int t = 0; t < PT; ++t) {
+        const float2 a = __ldg(in + ibase[t] + (long long)q * inner);
+        const float2 b = __ldg(in + ibase[t] + (long long)(N - 1 - q) * inner);
+        p[t] = make_float2(a.x + b.x, a.y + b.y);
+        m[t] = make_float2(a.x - b.x, a.y - b.y);
+      }
+      const float* row = tab + q * TS;
+#pragma unroll
+      for (int g = 0; g <= K; ++g) {
+        const float c = row[g];
+#pragma unroll
+        for (int t = 0; t < PT; ++t) {
+          A[t][g].x = fmaf(p[t].x, c, A[t][g].x);
+          A[t][g].y = fmaf(p[t].y, c, A[t][g].y);
+        }
+      }
+#pragma unroll
+      for (int g = 1; g <= K; ++g) {
+        const float s = row[K + g];
+#pragma unroll
+        for (int t = 0; t < PT; ++t) {
+          B[t][g].x = fmaf(m[t].x, s, B[t][g].x);
+          B[t][g].y = fmaf(m[t].y, s, B[t][g].y);
+        }
+      }
+    }
+    // Z_{+g} = rho_g (A - iB), Z_{-g} = conj(rho_g) (A + iB); positions [0..K-1] hold +g, [K..2K-1] hold -(2K-r)
+#pragma unroll
+    for (int t = 0; t < PT; ++t) {
+      if (!ok[t]) continue;
+#pragma unroll
+      for (int g = 0; g <= K; ++g) {
+        const float2 r = rho[g];
+        const float2 a = A[t][g], b = B[t][g];
+        if (g < K) {
+          const float wr = a.x + b.y, wi = a.y - b.x;   // A - iB
+          out[obase[t] + (long long)g * inner] = make_float2(r.x * wr - r.y * wi, r.x * wi + r.y * wr);
+        }
+        if (g > 0) {
+          const float wr = a.x - b.y, wi = a.y + b.x;   // A + iB
+          out[obase[t] + (long long)(2 * K - g) * inner] = make_float2(r.x * wr + r.y * wi, r.x * wi - r.y * wr);
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// expansion: in[outer][2K][inner] -> out[outer][N][inner]   (B^H along this dimension)
+//   z_n = P_n + Q_n, z_{N-1-n} = P_n - Q_n,
+//   P_n = sum_g alpha_g cos(psi_g (n+1/2)), Q_n = sum_g beta_g sin(psi_g (n+1/2)),
+//   alpha_g = V'_{+g} + V'_{-g}, beta_g = i (V'_{+g} - V'_{-g}), V'_{+-g} = e^{-+i psi_g/2} V_{+-g}
+// ------------------------------------------------------------------------------------------
+template <int K, int PT>
+__global__ void __launch_bounds__(kMidThreads) mid_expand_kernel(const float2* __restrict__ in,
+                                                                 float2* __restrict__ out, long long outer,
+                                                                 long long inner, int N, float scale) {
+  constexpr int TS = MidTab<K>::TS;
+  extern __shared__ float smem_mid[];
+  float* tab = smem_mid;
+  float2* rho = reinterpret_cast<float2*>(tab + (size_t)(N / 2) * TS);
+  build_mid_table<K>(tab, rho, N, scale);
+  __syncthreads();
+
+  const long long total = outer * inner;
+  const long long per_cta = (long long)kMidThreads * PT;
+  const long long tiles = (total + per_cta - 1) / per_cta;
+  const int half = N / 2;
+  for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    long long ibase[PT], obase[PT];
+    bool ok[PT];
+    float2 al[PT][K + 1], be[PT][K + 1];
+#pragma unroll
+    for (int t = 0; t < PT; ++t) {
+      const long long p = tile * per_cta + (long long)t * kMidThreads + threadIdx.x;
+      ok[t] = p < total;
+      const long long pc = ok[t] ? p : 0;
+      const long long o = pc / inner, i = pc % inner;
+      ibase[t] = o * (2 * K) * inner + i;
+      obase[t] = o * N * inner + i;
+#pragma unroll
+      for (int g = 0; g <= K; ++g) {
+        const float2 r = rho[g];
+        float2 vp = make_float2(0.f, 0.f), vm = make_float2(0.f, 0.f);
+        if (g < K) {
+          const float2 v = __ldg(in + ibase[t] + (long long)g * inner);
+          vp = make_float2(v.x * r.x + v.y * r.y, v.y * r.x - v.x * r.y);   // v * conj(rho)
+        }
+        if (g > 0) {
+          const float2 v = __ldg(in + ibase[t] + (long long)(2 * K - g) * inner);
+          vm = make_float2(v.x * r.x - v.y * r.y, v.y * r.x + v.x * r.y);   // v * rho
+        }
+        al[t][g] = make_float2(vp.x + vm.x, vp.y + vm.y);
+        be[t][g] = make_float2(-(vp.y - vm.y), vp.x - vm.x);                // i (vp - vm)
+      }
+    }
+#pragma unroll 2
+    for (int n = 0; n < half; ++n) {
+      const float* row = tab + n * TS;
+      float2 P[PT], Q[PT];
+#pragma unroll
+      for (int t = 0; t < PT; ++t) P[t] = Q[t] = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int g = 0; g <= K; ++g) {
+        const float c = row[g];
+#pragma unroll
+        for (int t = 0; t < PT; ++t) {
+          P[t].x = fmaf(al[t][g].x, c, P[t].x);
+          P[t].y = fmaf(al[t][g].y, c, P[t].y);
+        }
+      }
+#pragma unroll
+      for (int g = 1; g <= K; ++g) {
+        const float s = row[K + g];
+#pragma unroll
+        for (int t = 0; t < PT; ++t) {
+          Q[t].x = fmaf(be[t][g].x, s, Q[t].x);
+          Q[t].y = fmaf(be[t][g].y, s, Q[t].y);
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < PT; ++t) {
+        if (!ok[t]) continue;
+        out[obase[t] + (long long)n * inner] = make_float2(P[t].x + Q[t].x, P[t].y + Q[t].y);
+        out[obase[t] + (long long)(N - 1 - n) * inner] = make_float2(P[t].x - Q[t].x, P[t].y - Q[t].y);
+      }
+    }
+  }
+}
+
+template <int K, int PT>
+cudaError_t launch_mid_t(bool forward, const float2* in, float2* out, long long outer, long long inner, int N,
+                         float scale, cudaStream_t st) {
+  const size_t smem = (size_t)(N / 2) * MidTab<K>::TS * 4 + (size_t)(K + 1) * 8;
+  const long long total = outer * inner;
+  const long long tiles = (total + (long long)kMidThreads * PT - 1) / ((long long)kMidThreads * PT);
+  const long long cap = (long long)kNumSMs * 3;
+  const int grid = (int)(tiles < cap ? tiles : cap);
+  cudaError_t e = cudaSuccess;
+  if (forward) {
+    if (smem > 48 * 1024)
+      e = cudaFuncSetAttribute(mid_contract_kernel<K, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    mid_contract_kernel<K, PT><<<grid, kMidThreads, smem, st>>>(in, out, outer, inner, N, scale);
+  } else {
+    if (smem > 48 * 1024)
+      e = cudaFuncSetAttribute(mid_expand_kernel<K, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    mid_expand_kernel<K, PT><<<grid, kMidThreads, smem, st>>>(in, out, outer, inner, N, scale);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool mid_supported(int N, int K) {
+  if (N % 2 != 0 || 2 * K > N) return false;
+  if (!(K == 4 || K == 8 || K == 12 || K == 16)) return false;
+  const size_t smem = (size_t)(N / 2) * (((2 * K + 1 + 3) / 4) * 4) * 4 + (size_t)(K + 1) * 8;
+  return smem <= 200 * 1024;
+}
+
+cudaError_t launch_mid(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
+                       float scale, cudaStream_t st) {
+  if (outer * inner <= 0) return cudaSuccess;
+  switch (K) {
+    case 4: return launch_mid_t<4, 2>(forward, in, out, outer, inner, N, scale, st);
+    case 8: return launch_mid_t<8, 2>(forward, in, out, outer, inner, N, scale, st);
+    case 12: return launch_mid_t<12, 2>(forward, in, out, outer, inner, N, scale, st);
+    case 16: return launch_mid_t<16, 2>(forward, in, out, outer, inner, N, scale, st);
+    default: return cudaErrorNotSupported;
+  }
+}
+
+}  // namespace dtst
