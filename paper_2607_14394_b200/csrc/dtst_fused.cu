@@ -49,17 +49,20 @@ struct PlaneCfg {
   static constexpr int G = kTaskRows / N2;                    // planes per task
   static constexpr int QUADS = N2 / 4;                        // row quadruples per plane
   static constexpr int NC = 2 * K3;                           // real columns after stage 1 (C | S)
-  static constexpr int LPP = 2 * K2;                          // stage-2 lanes per plane
-  static constexpr int CSTRIDE = NC + 4;                      // floats between parity classes
-  static constexpr int NSTRIDE = 4 * CSTRIDE + 4;             // floats between quadruples
-  static constexpr int PSTRIDE = QUADS * NSTRIDE + 16;        // floats between planes
+  static constexpr int LPP = 2 * K2;                          // output rows (modes) per plane
+  static constexpr int NKS = QUADS / 8;                       // MMA k-steps over the quadruples
+  static constexpr int MT = G * NC / 16;                      // MMA m-tiles over (plane, column)
+  static constexpr int MT2 = 2;                               // inverse: MMA m-tiles over the 32 quadruples
+  static constexpr int GT = K2 / 2;                           // frequencies per parity class
+  static constexpr int NS = 4 * NC + 8;                       // floats per combo row: 4 classes x NC, +8 pad
   static constexpr int ABS = NC + 4;                          // floats between A/B entries
   static constexpr int ABP = (2 * K2 + 1) * ABS;
-  static constexpr int COMBO_FLOATS = (G * PSTRIDE > G * ABP ? G * PSTRIDE : G * ABP);
+  static constexpr int COMBO_FLOATS = (32 * NS > G * ABP ? 32 * NS : G * ABP);
   static_assert(N3 % 32 == 0 && (N3 == 32 || N3 == 64), "N3");
   static_assert(kTaskRows % N2 == 0 && G * QUADS == 32, "one lane per row quadruple");
-  static_assert(G * LPP <= 32 && G * NC <= 32, "stage-2 lane mapping");
-  static_assert(K3 % 2 == 0 && NC % 4 == 0, "K3");
+  static_assert(G * LPP <= 32 && (G * NC) % 16 == 0, "stage-2 mapping");
+  static_assert(K3 % 2 == 0 && NC % 8 == 0 && K2 % 2 == 0 && GT <= 8 && QUADS % 8 == 0, "shape");
+  static_assert(NS % 32 == 8, "combo row stride must be 8 mod 32 words for conflict-free fragment loads");
   static_assert(SPT == 1 || SPT == 2, "SPT");
 };
 
@@ -85,6 +88,21 @@ SmemPlan smem_plan() {
 }
 
 __device__ __forceinline__ float4 lds128(const char* p) { return *reinterpret_cast<const float4*>(p); }
+
+// fp32 -> (hi, lo) TF32 pair with hi + lo = v to ~2^-22 relative (error-compensated "3xTF32")
+__device__ __forceinline__ void split_tf32(float v, uint32_t& hi, uint32_t& lo) {
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(v));
+  const float r = v - __uint_as_float(hi);
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(r));
+}
+
+// D += A(16x8, row) * B(8x8, col), TF32 inputs, fp32 accumulate
+__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 
 // One row of N3 reals -> C_f = sum u cos, S_f = sum v sin for f < K3 (half-sample phase deferred).
 template <int N3, int K3>
@@ -221,138 +239,162 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
 
     // stage-1 role: lane = (plane in task, row quadruple)
     const int pl1 = lane / QUADS, n1 = lane % QUADS;
-    // stage-2 role: lane = (plane, A_g or B_g)
+    // epilogue role: lane = (plane, mode position r)
     const bool act2 = lane < G * LPP;
     const int pl2 = act2 ? lane / LPP : 0;
     const int l2 = lane % LPP;
-    const bool isB = l2 >= K2;
-    const int g2 = isB ? l2 - K2 + 1 : l2;
-    const int cls2 = isB ? ((g2 & 1) ? 2 : 3) : ((g2 & 1) ? 1 : 0);
-    // the unpaired cosine sum A_{K2} (needed by mode -K2 only) is spread over lanes by column
-    const bool actx = lane < G * NC;
-    const int plx = actx ? lane / NC : 0, cx = lane % NC;
-    constexpr int clsx = (K2 & 1) ? 1 : 0;
+    // MMA fragment coordinates
+    const int g8 = lane >> 2, t4 = lane & 3;
 
-    float coef[QUADS], coefx[QUADS];
+    // Stage-2 basis as MMA B fragments (k = quadruple n, n = frequency slot of the parity class), split
+    // into TF32 hi/lo once.  Classes: 0 = A even (pp, cos), 1 = A odd (pd, cos), 2 = B odd (ms, sin),
+    // 3 = B even (md, sin); 4 = the unpaired A_{K2} (cos, shares the pp operand), in column 0 only.
+    uint32_t bhi[5][Cfg::NKS][2], blo[5][Cfg::NKS][2];
 #pragma unroll
-    for (int n = 0; n < QUADS; ++n) {
-      double sn, cs;
-      sincospi((double)(((long long)g2 * (2 * n + 1)) % (2 * N2)) / (double)N2, &sn, &cs);
-      coef[n] = isB ? (float)sn : (float)cs;
-      sincospi((double)(((long long)K2 * (2 * n + 1)) % (2 * N2)) / (double)N2, &sn, &cs);
-      coefx[n] = (float)cs;
-    }
+    for (int cls = 0; cls < 5; ++cls)
+#pragma unroll
+      for (int ks = 0; ks < Cfg::NKS; ++ks)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int n = 8 * ks + t4 + 4 * h;
+          int g = 0;
+          bool valid = g8 < Cfg::GT;
+          if (cls == 0) g = 2 * g8;
+          else if (cls == 1 || cls == 2) g = 2 * g8 + 1;
+          else if (cls == 3) g = 2 * g8 + 2;
+          else { g = K2; valid = (g8 == 0); }
+          double sn, cs;
+          sincospi((double)(((long long)g * (2 * n + 1)) % (2 * N2)) / (double)N2, &sn, &cs);
+          const float v = valid ? ((cls == 2 || cls == 3) ? (float)sn : (float)cs) : 0.f;
+          split_tf32(v, bhi[cls][ks][h], blo[cls][ks][h]);
+        }
 
     for (long long tl = w; tl < n_local; tl += W) {
       const long long task = first + tl * gridDim.x;
       const long long k0 = tl * SPT;
-      float ra[NC], rb[NC], rc[NC], rd[NC];
+      const int slot0 = (int)(k0 % stages), slot1 = (int)((k0 + SPT - 1) % stages);
+      constexpr bool kSplit = (SPT == 2 && N2 == 128);   // rows a, b in the first slot, c, d in the second
 
-      if constexpr (SPT == 1) {
-        const int slot = (int)(k0 % stages);
-        if (!wait_fill(fill_seq, full, slot, (uint32_t)(k0 / stages), abort_flag)) break;
-        const char* st = reinterpret_cast<const char*>(ring) + (size_t)slot * kStageBytes;
-        const int base = pl1 * N2;
-        stage1_row<N3, K3>(st, RPS, base + n1, tab, ra);
-        stage1_row<N3, K3>(st, RPS, base + N2 - 1 - n1, tab, rd);
-        stage1_row<N3, K3>(st, RPS, base + N2 / 2 - 1 - n1, tab, rb);
-        stage1_row<N3, K3>(st, RPS, base + N2 / 2 + n1, tab, rc);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[slot]);
-      } else if constexpr (N2 == 128) {
-        // rows n, 63-n live in the first slot; 64+n, 127-n in the second: release each early
-        {
-          const int slot = (int)(k0 % stages);
-          if (!wait_fill(fill_seq, full, slot, (uint32_t)(k0 / stages), abort_flag)) break;
-          const char* st = reinterpret_cast<const char*>(ring) + (size_t)slot * kStageBytes;
-          stage1_row<N3, K3>(st, RPS, n1, tab, ra);
-          stage1_row<N3, K3>(st, RPS, 63 - n1, tab, rb);
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&empty[slot]);
-        }
-        {
-          const long long k1 = k0 + 1;
-          const int slot = (int)(k1 % stages);
-          if (!wait_fill(fill_seq, full, slot, (uint32_t)(k1 / stages), abort_flag)) break;
-          const char* st = reinterpret_cast<const char*>(ring) + (size_t)slot * kStageBytes;
-          stage1_row<N3, K3>(st, RPS, n1, tab, rc);
-          stage1_row<N3, K3>(st, RPS, 63 - n1, tab, rd);
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&empty[slot]);
-        }
-      } else {
-        // two planes of 64 rows, one per slot: a lane's four rows all sit in its plane's slot
-        const int slot0 = (int)(k0 % stages), slot1 = (int)((k0 + 1) % stages);
+      // ---- stage 1: the four rows of this lane's quadruple, accumulated straight into the four
+      // parity combos  pp = a+d+b+c, pd = a+d-b-c, ms = a-d+b-c, md = a-d-b+c  (one copy of the row code)
+      float cpp[NC], cpd[NC], cms[NC], cmd[NC];
+#pragma unroll
+      for (int c = 0; c < NC; ++c) cpp[c] = cpd[c] = cms[c] = cmd[c] = 0.f;
+      if constexpr (!kSplit) {
         if (!wait_fill(fill_seq, full, slot0, (uint32_t)(k0 / stages), abort_flag)) break;
-        if (!wait_fill(fill_seq, full, slot1, (uint32_t)((k0 + 1) / stages), abort_flag)) break;
-        const char* st = reinterpret_cast<const char*>(ring) + (size_t)(pl1 ? slot1 : slot0) * kStageBytes;
-        stage1_row<N3, K3>(st, RPS, n1, tab, ra);
-        stage1_row<N3, K3>(st, RPS, N2 - 1 - n1, tab, rd);
-        stage1_row<N3, K3>(st, RPS, N2 / 2 - 1 - n1, tab, rb);
-        stage1_row<N3, K3>(st, RPS, N2 / 2 + n1, tab, rc);
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(&empty[slot0]);
+        if (SPT == 2 && !wait_fill(fill_seq, full, slot1, (uint32_t)((k0 + 1) / stages), abort_flag)) break;
+      }
+      bool alive = true;
+#pragma unroll 1
+      for (int r4 = 0; r4 < 4; ++r4) {
+        if constexpr (kSplit) {
+          if (r4 == 0) alive = wait_fill(fill_seq, full, slot0, (uint32_t)(k0 / stages), abort_flag);
+          if (r4 == 2) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[slot0]);
+            alive = wait_fill(fill_seq, full, slot1, (uint32_t)((k0 + 1) / stages), abort_flag);
+          }
+          if (!alive) break;
+        }
+        // order a, b, c, d = rows n, N2/2-1-n, N2/2+n, N2-1-n of the plane
+        const int rowq = (r4 == 0) ? n1 : (r4 == 1) ? (N2 / 2 - 1 - n1) : (r4 == 2) ? (N2 / 2 + n1) : (N2 - 1 - n1);
+        const float s1 = (r4 == 0 || r4 == 3) ? 1.f : -1.f;
+        const float s2 = (r4 <= 1) ? 1.f : -1.f;
+        const float s3 = (r4 == 0 || r4 == 2) ? 1.f : -1.f;
+        const int trow = pl1 * N2 + rowq;
+        const int sl = (trow / RPS) ? slot1 : slot0;
+        const char* st = reinterpret_cast<const char*>(ring) + (size_t)sl * kStageBytes;
+        float o[NC];
+        stage1_row<N3, K3>(st, RPS, trow % RPS, tab, o);
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+          cpp[c] += o[c];
+          cpd[c] = fmaf(s1, o[c], cpd[c]);
+          cms[c] = fmaf(s2, o[c], cms[c]);
+          cmd[c] = fmaf(s3, o[c], cmd[c]);
+        }
+      }
+      if (!alive) break;
+      __syncwarp();
+      if (lane == 0) {
+        if constexpr (kSplit) {
           mbar_arrive(&empty[slot1]);
+        } else {
+          mbar_arrive(&empty[slot0]);
+          if (SPT == 2) mbar_arrive(&empty[slot1]);
         }
       }
 
-      // fold the four rows of the quadruple (second dimension) and publish the four combos
+      // publish the combos: row (plane, n), 4 classes x NC floats, 16-byte chunks swapped pairwise on
+      // odd groups of four rows so that both these stores and the fragment loads below are conflict-free
       {
-        float* dst = combo + pl1 * Cfg::PSTRIDE + n1 * Cfg::NSTRIDE;
+        float* dst = combo + (size_t)lane * Cfg::NS;
+        const int sw = ((n1 >> 2) & 1);
 #pragma unroll
         for (int c4 = 0; c4 < NC / 4; ++c4) {
-          float pp[4], pd[4], ms[4], md[4];
+          const int cc = 4 * (c4 ^ sw);
+          *reinterpret_cast<float4*>(dst + 0 * NC + cc) = make_float4(cpp[4 * c4], cpp[4 * c4 + 1], cpp[4 * c4 + 2], cpp[4 * c4 + 3]);
+          *reinterpret_cast<float4*>(dst + 1 * NC + cc) = make_float4(cpd[4 * c4], cpd[4 * c4 + 1], cpd[4 * c4 + 2], cpd[4 * c4 + 3]);
+          *reinterpret_cast<float4*>(dst + 2 * NC + cc) = make_float4(cms[4 * c4], cms[4 * c4 + 1], cms[4 * c4 + 2], cms[4 * c4 + 3]);
+          *reinterpret_cast<float4*>(dst + 3 * NC + cc) = make_float4(cmd[4 * c4], cmd[4 * c4 + 1], cmd[4 * c4 + 2], cmd[4 * c4 + 3]);
+        }
+      }
+      __syncwarp();
+
+      // ---- stage 2 on the tensor cores (legacy warp-level MMA, TF32 with hi/lo error compensation):
+      // out[(plane, column)][frequency slot] = sum_n combo_cls[n][(plane, column)] * basis_cls[n][slot]
+      float acc[5][Cfg::MT][4];
+#pragma unroll
+      for (int cls = 0; cls < 5; ++cls)
+#pragma unroll
+        for (int mt = 0; mt < Cfg::MT; ++mt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[cls][mt][e] = 0.f;
+#pragma unroll
+      for (int cls = 0; cls < 4; ++cls)
+#pragma unroll
+        for (int ks = 0; ks < Cfg::NKS; ++ks)
+#pragma unroll
+          for (int mt = 0; mt < Cfg::MT; ++mt) {
+            uint32_t ahi[4], alo[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int m = 16 * mt + g8 + 8 * (e & 1);
+              const int n = 8 * ks + t4 + 4 * (e >> 1);
+              const int pl = m / NC, c = m % NC;
+              const float v = combo[(size_t)(pl * QUADS + n) * Cfg::NS + cls * NC + (c ^ ((e >> 1) << 2))];
+              split_tf32(v, ahi[e], alo[e]);
+            }
+            mma_tf32(acc[cls][mt], ahi, bhi[cls][ks][0], bhi[cls][ks][1]);
+            mma_tf32(acc[cls][mt], alo, bhi[cls][ks][0], bhi[cls][ks][1]);
+            mma_tf32(acc[cls][mt], ahi, blo[cls][ks][0], blo[cls][ks][1]);
+            if (cls == 0) {   // the pp operand also feeds the unpaired A_{K2}
+              mma_tf32(acc[4][mt], ahi, bhi[4][ks][0], bhi[4][ks][1]);
+              mma_tf32(acc[4][mt], alo, bhi[4][ks][0], bhi[4][ks][1]);
+              mma_tf32(acc[4][mt], ahi, blo[4][ks][0], blo[4][ks][1]);
+            }
+          }
+      __syncwarp();
+
+      // A/B sums -> shared: entry g for A_g (g <= K2), entry K2+g for B_g (g >= 1)
+#pragma unroll
+      for (int cls = 0; cls < 5; ++cls)
+#pragma unroll
+        for (int mt = 0; mt < Cfg::MT; ++mt)
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const int c = 4 * c4 + e;
-            const float p = ra[c] + rd[c], m = ra[c] - rd[c];
-            const float pq = rb[c] + rc[c], mq = rb[c] - rc[c];
-            pp[e] = p + pq;
-            pd[e] = p - pq;
-            ms[e] = m + mq;
-            md[e] = m - mq;
+            const int m = 16 * mt + g8 + 8 * (e >> 1);
+            const int gi = 2 * t4 + (e & 1);
+            const int pl = m / NC, c = m % NC;
+            int entry;
+            bool valid = gi < Cfg::GT;
+            if (cls == 0) entry = 2 * gi;
+            else if (cls == 1) entry = 2 * gi + 1;
+            else if (cls == 2) entry = K2 + 2 * gi + 1;
+            else if (cls == 3) entry = K2 + 2 * gi + 2;
+            else { entry = K2; valid = (gi == 0); }
+            if (valid) combo[pl * Cfg::ABP + entry * Cfg::ABS + c] = acc[cls][mt][e];
           }
-          *reinterpret_cast<float4*>(dst + 0 * Cfg::CSTRIDE + 4 * c4) = make_float4(pp[0], pp[1], pp[2], pp[3]);
-          *reinterpret_cast<float4*>(dst + 1 * Cfg::CSTRIDE + 4 * c4) = make_float4(pd[0], pd[1], pd[2], pd[3]);
-          *reinterpret_cast<float4*>(dst + 2 * Cfg::CSTRIDE + 4 * c4) = make_float4(ms[0], ms[1], ms[2], ms[3]);
-          *reinterpret_cast<float4*>(dst + 3 * Cfg::CSTRIDE + 4 * c4) = make_float4(md[0], md[1], md[2], md[3]);
-        }
-      }
-      __syncwarp();
-
-      // stage 2: A_g = sum_n (pp|pd)[n] cos, B_g = sum_n (md|ms)[n] sin, one lane per (g, A/B)
-      float acc[NC];
-      float accx = 0.f;
-#pragma unroll
-      for (int c = 0; c < NC; ++c) acc[c] = 0.f;
-      {
-        const float* cb = combo + pl2 * Cfg::PSTRIDE + cls2 * Cfg::CSTRIDE;
-        const float* cbx = combo + plx * Cfg::PSTRIDE + clsx * Cfg::CSTRIDE + cx;
-#pragma unroll
-        for (int n = 0; n < QUADS; ++n) {
-#pragma unroll
-          for (int c4 = 0; c4 < NC / 4; ++c4) {
-            const float4 v = *reinterpret_cast<const float4*>(cb + n * Cfg::NSTRIDE + 4 * c4);
-            acc[4 * c4 + 0] = fmaf(coef[n], v.x, acc[4 * c4 + 0]);
-            acc[4 * c4 + 1] = fmaf(coef[n], v.y, acc[4 * c4 + 1]);
-            acc[4 * c4 + 2] = fmaf(coef[n], v.z, acc[4 * c4 + 2]);
-            acc[4 * c4 + 3] = fmaf(coef[n], v.w, acc[4 * c4 + 3]);
-          }
-          accx = fmaf(coefx[n], cbx[n * Cfg::NSTRIDE], accx);
-        }
-      }
-      __syncwarp();
-
-      // A/B sums -> shared, entry g for A_g (g <= K2), entry K2+g for B_g (g >= 1)
-      if (act2) {
-        float* ab = combo + pl2 * Cfg::ABP + (isB ? K2 + g2 : g2) * Cfg::ABS;
-#pragma unroll
-        for (int c4 = 0; c4 < NC / 4; ++c4)
-          *reinterpret_cast<float4*>(ab + 4 * c4) =
-              make_float4(acc[4 * c4], acc[4 * c4 + 1], acc[4 * c4 + 2], acc[4 * c4 + 3]);
-      }
-      if (actx) combo[plx * Cfg::ABP + K2 * Cfg::ABS + cx] = accx;
       __syncwarp();
 
       // epilogue: Z_{+g} = rho (A - iB), Z_{-g} = rho (A + iB) with A = AC - i AS, B = BC - i BS
@@ -441,10 +483,12 @@ struct InvCfg {
   using P = PlaneCfg<N3, K3, N2, K2>;
   static constexpr int ABS = P::NC + 4;                     // floats between entries
   static constexpr int ENTRIES = 2 * K2 + 2;                // alpha_0..alpha_K2, beta_0..beta_K2 (beta_0 unused)
-  static constexpr int ABP = ENTRIES * ABS + 4;             // floats between planes (offset banks)
+  static constexpr int ABP = ENTRIES * ABS + 4;             // floats between planes
   static constexpr int AB_FLOATS = ((P::G * ABP + 3) / 4) * 4;
+  static constexpr int COMBO_FLOATS = 32 * P::NS;           // expanded combos, one row per quadruple
+  static constexpr int NT = P::NC / 8;                      // MMA n-tiles over the columns
   static constexpr int STAGING_BYTES = kTaskRows * N3 * 4;  // 128 output rows
-  static constexpr int WARP_BYTES = STAGING_BYTES + ((AB_FLOATS * 4 + 1023) / 1024) * 1024;
+  static constexpr int WARP_BYTES = STAGING_BYTES + (((AB_FLOATS + COMBO_FLOATS) * 4 + 1023) / 1024) * 1024;
 };
 
 template <int N3, int K3, int N2, int K2, int W>
@@ -476,16 +520,35 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
   }
   __syncthreads();
 
-  // stage-2 role (one lane per row quadruple) and its basis values, kept in registers
+  // roles: row quadruple (stage 1 / unfold), MMA fragment coordinates, mode loader
   const int pl1 = lane / QUADS, n1 = lane % QUADS;
-  float cosc[K2 + 1], sinc[K2 + 1];
+  const int g8 = lane >> 2, t4 = lane & 3;
+  float* combo = ab + IC::AB_FLOATS;
+
+  // Second-dimension basis as MMA A fragments (row = quadruple n, col = frequency slot of the parity class),
+  // TF32 hi/lo.  Classes: 0 = Pe (even g, cos), 1 = Po (odd g, cos), 2 = Qo (odd g, sin), 3 = Qe (even g, sin);
+  // index 4 = the unpaired g = K2 cosine, which adds into Pe through one extra k-step.
+  uint32_t ahi[5][Cfg::MT2][4], alo[5][Cfg::MT2][4];
 #pragma unroll
-  for (int g = 0; g <= K2; ++g) {
-    double sn, cs;
-    sincospi((double)(((long long)g * (2 * n1 + 1)) % (2 * N2)) / (double)N2, &sn, &cs);
-    cosc[g] = (float)cs;
-    sinc[g] = (float)sn;
-  }
+  for (int cls = 0; cls < 5; ++cls)
+#pragma unroll
+    for (int mt = 0; mt < Cfg::MT2; ++mt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int n = (16 * mt + g8 + 8 * (e & 1)) % QUADS;
+        const int gi = t4 + 4 * (e >> 1);
+        int g = 0;
+        bool valid = gi < Cfg::GT;
+        if (cls == 0) g = 2 * gi;
+        else if (cls == 1 || cls == 2) g = 2 * gi + 1;
+        else if (cls == 3) g = 2 * gi + 2;
+        else { g = K2; valid = (gi == 0); }
+        double sn, cs;
+        sincospi((double)(((long long)g * (2 * n + 1)) % (2 * N2)) / (double)N2, &sn, &cs);
+        const float v = valid ? ((cls == 2 || cls == 3) ? (float)sn : (float)cs) : 0.f;
+        split_tf32(v, ahi[cls][mt][e], alo[cls][mt][e]);
+      }
+
   // loader role: lane = (plane, mode position r)
   const bool actl = lane < G * LPP;
   const int pll = actl ? lane / LPP : 0, rl = lane % LPP;
@@ -500,7 +563,7 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
   }
 
   for (; task < num_tasks; task += tstride) {
-    // ---- A. rotate this task's modes, publish V'
+    // ---- rotate this task's modes, publish V'
     if (actl) {
       float* dst = ab + pll * IC::ABP + rl * IC::ABS;
       const float2* rr = rot + rl * K3;
@@ -559,73 +622,106 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
     }
     __syncwarp();
 
-    // ---- B. expand the second dimension for this lane's row quadruple
-    float Pe[NC], Po[NC], Qe[NC], Qo[NC];
+    // ---- expand the second dimension on the tensor cores (warp-level MMA, TF32 hi/lo compensated):
+    // combo_cls[quadruple n][(plane, column)] = sum_slot basis_cls[n][slot] * (alpha|beta)_cls[slot][column]
 #pragma unroll
-    for (int c = 0; c < NC; ++c) Pe[c] = Po[c] = Qe[c] = Qo[c] = 0.f;
-    {
-      const float* al = ab + pl1 * IC::ABP;
-      const float* be = ab + pl1 * IC::ABP + (K2 + 1) * IC::ABS;
+    for (int cls = 0; cls < 4; ++cls)
 #pragma unroll
-      for (int g = 0; g <= K2; ++g) {
+      for (int nt = 0; nt < IC::NT; ++nt)
 #pragma unroll
-        for (int c4 = 0; c4 < NC / 4; ++c4) {
-          const float4 av = *reinterpret_cast<const float4*>(al + g * IC::ABS + 4 * c4);
-          if ((g & 1) == 0) {
-            Pe[4 * c4] = fmaf(cosc[g], av.x, Pe[4 * c4]);
-            Pe[4 * c4 + 1] = fmaf(cosc[g], av.y, Pe[4 * c4 + 1]);
-            Pe[4 * c4 + 2] = fmaf(cosc[g], av.z, Pe[4 * c4 + 2]);
-            Pe[4 * c4 + 3] = fmaf(cosc[g], av.w, Pe[4 * c4 + 3]);
-          } else {
-            Po[4 * c4] = fmaf(cosc[g], av.x, Po[4 * c4]);
-            Po[4 * c4 + 1] = fmaf(cosc[g], av.y, Po[4 * c4 + 1]);
-            Po[4 * c4 + 2] = fmaf(cosc[g], av.z, Po[4 * c4 + 2]);
-            Po[4 * c4 + 3] = fmaf(cosc[g], av.w, Po[4 * c4 + 3]);
-          }
-          if (g > 0) {
-            const float4 bv = *reinterpret_cast<const float4*>(be + g * IC::ABS + 4 * c4);
-            if ((g & 1) == 0) {
-              Qe[4 * c4] = fmaf(sinc[g], bv.x, Qe[4 * c4]);
-              Qe[4 * c4 + 1] = fmaf(sinc[g], bv.y, Qe[4 * c4 + 1]);
-              Qe[4 * c4 + 2] = fmaf(sinc[g], bv.z, Qe[4 * c4 + 2]);
-              Qe[4 * c4 + 3] = fmaf(sinc[g], bv.w, Qe[4 * c4 + 3]);
-            } else {
-              Qo[4 * c4] = fmaf(sinc[g], bv.x, Qo[4 * c4]);
-              Qo[4 * c4 + 1] = fmaf(sinc[g], bv.y, Qo[4 * c4 + 1]);
-              Qo[4 * c4 + 2] = fmaf(sinc[g], bv.z, Qo[4 * c4 + 2]);
-              Qo[4 * c4 + 3] = fmaf(sinc[g], bv.w, Qo[4 * c4 + 3]);
+        for (int mt = 0; mt < Cfg::MT2; ++mt) {
+          const int pl = (16 * mt) / QUADS;
+          float acc[4] = {0.f, 0.f, 0.f, 0.f};
+          const int c = 8 * nt + g8;
+          {
+            uint32_t bh[2], bl[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int gi = t4 + 4 * h;
+              int entry = 0;
+              if (cls == 0) entry = 2 * gi;
+              else if (cls == 1) entry = 2 * gi + 1;
+              else if (cls == 2) entry = K2 + 1 + 2 * gi + 1;
+              else entry = K2 + 1 + 2 * gi + 2;
+              const float v = (gi < Cfg::GT) ? ab[pl * IC::ABP + entry * IC::ABS + c] : 0.f;
+              split_tf32(v, bh[h], bl[h]);
             }
+            mma_tf32(acc, ahi[cls][mt], bh[0], bh[1]);
+            mma_tf32(acc, alo[cls][mt], bh[0], bh[1]);
+            mma_tf32(acc, ahi[cls][mt], bl[0], bl[1]);
           }
+          if (cls == 0) {   // unpaired g = K2: slot 0 of an extra k-step, all other slots are zero
+            uint32_t bh[2], bl[2];
+            const float v = (t4 == 0) ? ab[pl * IC::ABP + K2 * IC::ABS + c] : 0.f;
+            split_tf32(v, bh[0], bl[0]);
+            bh[1] = 0u;
+            bl[1] = 0u;
+            mma_tf32(acc, ahi[4][mt], bh[0], bh[1]);
+            mma_tf32(acc, alo[4][mt], bh[0], bh[1]);
+            mma_tf32(acc, ahi[4][mt], bl[0], bl[1]);
+          }
+          // C fragment -> combos row (quadruple), 16-byte chunks swapped pairwise on odd groups of four rows
+          const int colp = (8 * nt + 2 * t4) ^ (((g8 >> 2) & 1) << 2);
+          float* d0 = combo + (size_t)(16 * mt + g8) * Cfg::NS + cls * NC + colp;
+          *reinterpret_cast<float2*>(d0) = make_float2(acc[0], acc[1]);
+          *reinterpret_cast<float2*>(d0 + 8 * Cfg::NS) = make_float2(acc[2], acc[3]);
         }
+    __syncwarp();
+
+    // this lane's quadruple: Pe, Po, Qo, Qe
+    float Pe[NC], Po[NC], Qo[NC], Qe[NC];
+    {
+      const float* src = combo + (size_t)lane * Cfg::NS;
+      const int sw = (n1 >> 2) & 1;
+#pragma unroll
+      for (int c4 = 0; c4 < NC / 4; ++c4) {
+        const int cc = 4 * (c4 ^ sw);
+        const float4 v0 = *reinterpret_cast<const float4*>(src + 0 * NC + cc);
+        const float4 v1 = *reinterpret_cast<const float4*>(src + 1 * NC + cc);
+        const float4 v2 = *reinterpret_cast<const float4*>(src + 2 * NC + cc);
+        const float4 v3 = *reinterpret_cast<const float4*>(src + 3 * NC + cc);
+        Pe[4 * c4] = v0.x; Pe[4 * c4 + 1] = v0.y; Pe[4 * c4 + 2] = v0.z; Pe[4 * c4 + 3] = v0.w;
+        Po[4 * c4] = v1.x; Po[4 * c4 + 1] = v1.y; Po[4 * c4 + 2] = v1.z; Po[4 * c4 + 3] = v1.w;
+        Qo[4 * c4] = v2.x; Qo[4 * c4 + 1] = v2.y; Qo[4 * c4 + 2] = v2.z; Qo[4 * c4 + 3] = v2.w;
+        Qe[4 * c4] = v3.x; Qe[4 * c4 + 1] = v3.y; Qe[4 * c4 + 2] = v3.z; Qe[4 * c4 + 3] = v3.w;
       }
     }
     // the previous task's TMA stores must have finished reading the staging rows before they are rewritten
     if (lane == 0) tma_store_wait_read<0>();
     __syncwarp();
 
-    // ---- C/D. unfold to the four rows and expand each along the contiguous dimension
-    {
+    // ---- unfold to the four rows (a: n, b: N2/2-1-n, c: N2/2+n, d: N2-1-n) and expand each along the
+    // contiguous dimension; one copy of the row code, signs select the row
+    constexpr bool kSplit = (SPT == 2 && N2 == 128);   // rows a, b fill the first staging block: store it early
+#pragma unroll 1
+    for (int r4 = 0; r4 < 4; ++r4) {
+      if constexpr (kSplit) {
+        if (r4 == 2) {
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+#pragma unroll
+            for (int h = 0; h < Cfg::BOXES; ++h)
+              tma_store_2d(&out_map, h * 32, (int)(task * kTaskRows), staging + (size_t)h * RPS * 128);
+            tma_store_commit();
+          }
+        }
+      }
+      const int rowq = (r4 == 0) ? n1 : (r4 == 1) ? (N2 / 2 - 1 - n1) : (r4 == 2) ? (N2 / 2 + n1) : (N2 - 1 - n1);
+      const float sPo = (r4 == 0 || r4 == 3) ? 1.f : -1.f;   // a, d: +Po;  b, c: -Po
+      const float sQe = (r4 == 0 || r4 == 2) ? 1.f : -1.f;   // a, c: +Qe;  b, d: -Qe
+      const float sQo = (r4 <= 1) ? 1.f : -1.f;              // a, b: +Qo;  c, d: -Qo
       float z[NC];
-      const int base = pl1 * N2;
-      auto row_ptr = [&](int r) -> char* { return staging + (size_t)(r / RPS) * kStageBytes; };
 #pragma unroll
-      for (int c = 0; c < NC; ++c) z[c] = (Pe[c] + Po[c]) + (Qe[c] + Qo[c]);
-      expand_row<N3, K3>(row_ptr(base + n1), RPS, (base + n1) % RPS, tab, z);
-#pragma unroll
-      for (int c = 0; c < NC; ++c) z[c] = (Pe[c] + Po[c]) - (Qe[c] + Qo[c]);
-      expand_row<N3, K3>(row_ptr(base + N2 - 1 - n1), RPS, (base + N2 - 1 - n1) % RPS, tab, z);
-#pragma unroll
-      for (int c = 0; c < NC; ++c) z[c] = (Pe[c] - Po[c]) - (Qe[c] - Qo[c]);
-      expand_row<N3, K3>(row_ptr(base + N2 / 2 - 1 - n1), RPS, (base + N2 / 2 - 1 - n1) % RPS, tab, z);
-#pragma unroll
-      for (int c = 0; c < NC; ++c) z[c] = (Pe[c] - Po[c]) + (Qe[c] - Qo[c]);
-      expand_row<N3, K3>(row_ptr(base + N2 / 2 + n1), RPS, (base + N2 / 2 + n1) % RPS, tab, z);
+      for (int c = 0; c < NC; ++c) z[c] = fmaf(sQo, Qo[c], fmaf(sQe, Qe[c], fmaf(sPo, Po[c], Pe[c])));
+      const int trow = pl1 * N2 + rowq;
+      expand_row<N3, K3>(staging + (size_t)(trow / RPS) * kStageBytes, RPS, trow % RPS, tab, z);
     }
     fence_proxy_async_smem();
     __syncwarp();
     if (lane == 0) {
 #pragma unroll
-      for (int rb = 0; rb < SPT; ++rb)
+      for (int rb = kSplit ? 1 : 0; rb < SPT; ++rb)
 #pragma unroll
         for (int h = 0; h < Cfg::BOXES; ++h)
           tma_store_2d(&out_map, h * 32, (int)(task * kTaskRows + (long long)rb * RPS),
