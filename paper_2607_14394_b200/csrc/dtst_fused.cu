@@ -488,7 +488,12 @@ struct InvCfg {
   static constexpr int COMBO_FLOATS = 32 * P::NS;           // expanded combos, one row per quadruple
   static constexpr int NT = P::NC / 8;                      // MMA n-tiles over the columns
   static constexpr int STAGING_BYTES = kTaskRows * N3 * 4;  // 128 output rows
-  static constexpr int WARP_BYTES = STAGING_BYTES + (((AB_FLOATS + COMBO_FLOATS) * 4 + 1023) / 1024) * 1024;
+  // With two staging blocks that are stored one after the other (rows a, b then rows c, d) the small
+  // alpha/beta and combo buffers live inside the first block: its store is issued half a task before the
+  // next task needs the space, so one bounded wait on that store group is all the aliasing costs.
+  static constexpr bool ALIAS = (P::SPT == 2 && N2 == 128) && ((AB_FLOATS + COMBO_FLOATS) * 4 <= kStageBytes);
+  static constexpr int WARP_BYTES =
+      ALIAS ? STAGING_BYTES : STAGING_BYTES + (((AB_FLOATS + COMBO_FLOATS) * 4 + 1023) / 1024) * 1024;
 };
 
 template <int N3, int K3, int N2, int K2, int W>
@@ -504,7 +509,7 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   char* staging = reinterpret_cast<char*>(smem) + (size_t)warp * IC::WARP_BYTES;
-  float* ab = reinterpret_cast<float*>(staging + IC::STAGING_BYTES);
+  float* ab = reinterpret_cast<float*>(IC::ALIAS ? staging : staging + IC::STAGING_BYTES);
   float2* rot = reinterpret_cast<float2*>(smem + (size_t)W * IC::WARP_BYTES);
 
   if (threadIdx.x == 0) prefetch_tensormap(&out_map);
@@ -563,6 +568,11 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
   }
 
   for (; task < num_tasks; task += tstride) {
+    if constexpr (IC::ALIAS) {
+      // the store of the previous task's first block (committed second to last) must have read its rows
+      if (lane == 0) tma_store_wait_read<1>();
+      __syncwarp();
+    }
     // ---- rotate this task's modes, publish V'
     if (actl) {
       float* dst = ab + pll * IC::ABP + rl * IC::ABS;
@@ -687,7 +697,10 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
       }
     }
     // the previous task's TMA stores must have finished reading the staging rows before they are rewritten
-    if (lane == 0) tma_store_wait_read<0>();
+    // (aliased layout: the first block is already free, and every lane has its combos in registers now)
+    if constexpr (!IC::ALIAS) {
+      if (lane == 0) tma_store_wait_read<0>();
+    }
     __syncwarp();
 
     // ---- unfold to the four rows (a: n, b: N2/2-1-n, c: N2/2+n, d: N2-1-n) and expand each along the
@@ -704,7 +717,10 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
             for (int h = 0; h < Cfg::BOXES; ++h)
               tma_store_2d(&out_map, h * 32, (int)(task * kTaskRows), staging + (size_t)h * RPS * 128);
             tma_store_commit();
+            // rows c, d go to the second block: the previous task's store of it must be done reading
+            if constexpr (IC::ALIAS) tma_store_wait_read<1>();
           }
+          if constexpr (IC::ALIAS) __syncwarp();
         }
       }
       const int rowq = (r4 == 0) ? n1 : (r4 == 1) ? (N2 / 2 - 1 - n1) : (r4 == 2) ? (N2 / 2 + n1) : (N2 - 1 - n1);
@@ -800,7 +816,8 @@ cudaError_t launch_fwd_plane_t(const float* x, float2* out, long long rows, floa
 template <int N3, int K3, int N2, int K2>
 cudaError_t launch_inv_plane_t(const float2* in, float* y, long long rows, float scale, int herm, cudaStream_t st) {
   using IC = InvCfg<N3, K3, N2, K2>;
-  constexpr int W = (IC::WARP_BYTES * 6 + 2 * K2 * K3 * 8 + 2048 <= kSmemLimit) ? 6 : 5;
+  constexpr int W = (IC::WARP_BYTES * 7 + 2 * K2 * K3 * 8 + 1024 <= kSmemLimit) ? 7
+                    : (IC::WARP_BYTES * 6 + 2 * K2 * K3 * 8 + 1024 <= kSmemLimit) ? 6 : 5;
   const size_t total = (size_t)W * IC::WARP_BYTES + (size_t)2 * K2 * K3 * 8 + 1024;
   static_assert((size_t)W * IC::WARP_BYTES + (size_t)2 * K2 * K3 * 8 + 1024 <= kSmemLimit, "shared memory");
   CUtensorMap map;

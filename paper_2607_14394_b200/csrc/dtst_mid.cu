@@ -51,7 +51,7 @@ __device__ __forceinline__ void build_mid_table(float* tab, float2* rho, int N, 
 // ------------------------------------------------------------------------------------------
 // forward: in[outer][N][inner] -> out[outer][2K][inner]
 // ------------------------------------------------------------------------------------------
-template <int K, int PT>
+template <int K, int PT, bool VEC>
 __global__ void __launch_bounds__(kMidThreads) mid_contract_kernel(const float2* __restrict__ in,
                                                                    float2* __restrict__ out, long long outer,
                                                                    long long inner, int N, float scale) {
@@ -67,11 +67,14 @@ __global__ void __launch_bounds__(kMidThreads) mid_contract_kernel(const float2*
   const long long tiles = (total + per_cta - 1) / per_cta;
   const int half = N / 2;
   for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    // VEC: the PT = 2 positions of a thread are adjacent in memory (one 16-byte access); otherwise they
+    // are kMidThreads apart (inner odd, 8-byte accesses)
     long long ibase[PT], obase[PT];
     bool ok[PT];
 #pragma unroll
     for (int t = 0; t < PT; ++t) {
-      const long long p = tile * per_cta + (long long)t * kMidThreads + threadIdx.x;
+      const long long p = VEC ? tile * per_cta + (long long)threadIdx.x * PT + t
+                              : tile * per_cta + (long long)t * kMidThreads + threadIdx.x;
       ok[t] = p < total;
       const long long pc = ok[t] ? p : 0;
       const long long o = pc / inner, i = pc % inner;
@@ -84,15 +87,25 @@ __global__ void __launch_bounds__(kMidThreads) mid_contract_kernel(const float2*
 #pragma unroll
       for (int g = 0; g <= K; ++g) A[t][g] = B[t][g] = make_float2(0.f, 0.f);
 
-#pragma unroll 2
+#pragma unroll 4
     for (int q = 0; q < half; ++q) {
       float2 p[PT], m[PT];
+      if constexpr (VEC) {
+        static_assert(!VEC || PT == 2, "vector path handles two adjacent positions");
+        const float4 a = __ldg(reinterpret_cast<const float4*>(in + ibase[0] + (long long)q * inner));
+        const float4 b = __ldg(reinterpret_cast<const float4*>(in + ibase[0] + (long long)(N - 1 - q) * inner));
+        p[0] = make_float2(a.x + b.x, a.y + b.y);
+        m[0] = make_float2(a.x - b.x, a.y - b.y);
+        p[PT - 1] = make_float2(a.z + b.z, a.w + b.w);
+        m[PT - 1] = make_float2(a.z - b.z, a.w - b.w);
+      } else {
 #pragma unroll
-      for (int t = 0; t < PT; ++t) {
-        const float2 a = __ldg(in + ibase[t] + (long long)q * inner);
-        const float2 b = __ldg(in + ibase[t] + (long long)(N - 1 - q) * inner);
-        p[t] = make_float2(a.x + b.x, a.y + b.y);
-        m[t] = make_float2(a.x - b.x, a.y - b.y);
+        for (int t = 0; t < PT; ++t) {
+          const float2 a = __ldg(in + ibase[t] + (long long)q * inner);
+          const float2 b = __ldg(in + ibase[t] + (long long)(N - 1 - q) * inner);
+          p[t] = make_float2(a.x + b.x, a.y + b.y);
+          m[t] = make_float2(a.x - b.x, a.y - b.y);
+        }
       }
       const float* row = tab + q * TS;
 #pragma unroll
@@ -116,19 +129,32 @@ __global__ void __launch_bounds__(kMidThreads) mid_contract_kernel(const float2*
     }
     // Z_{+g} = rho_g (A - iB), Z_{-g} = conj(rho_g) (A + iB); positions [0..K-1] hold +g, [K..2K-1] hold -(2K-r)
 #pragma unroll
-    for (int t = 0; t < PT; ++t) {
-      if (!ok[t]) continue;
+    for (int g = 0; g <= K; ++g) {
+      const float2 r = rho[g];
+      float2 zp[PT], zm[PT];
 #pragma unroll
-      for (int g = 0; g <= K; ++g) {
-        const float2 r = rho[g];
+      for (int t = 0; t < PT; ++t) {
         const float2 a = A[t][g], b = B[t][g];
-        if (g < K) {
-          const float wr = a.x + b.y, wi = a.y - b.x;   // A - iB
-          out[obase[t] + (long long)g * inner] = make_float2(r.x * wr - r.y * wi, r.x * wi + r.y * wr);
+        const float pr = a.x + b.y, pi = a.y - b.x;   // A - iB
+        const float mr = a.x - b.y, mi = a.y + b.x;   // A + iB
+        zp[t] = make_float2(r.x * pr - r.y * pi, r.x * pi + r.y * pr);
+        zm[t] = make_float2(r.x * mr + r.y * mi, r.x * mi - r.y * mr);
+      }
+      if constexpr (VEC) {
+        if (ok[0]) {
+          if (g < K)
+            *reinterpret_cast<float4*>(out + obase[0] + (long long)g * inner) =
+                make_float4(zp[0].x, zp[0].y, zp[PT - 1].x, zp[PT - 1].y);
+          if (g > 0)
+            *reinterpret_cast<float4*>(out + obase[0] + (long long)(2 * K - g) * inner) =
+                make_float4(zm[0].x, zm[0].y, zm[PT - 1].x, zm[PT - 1].y);
         }
-        if (g > 0) {
-          const float wr = a.x - b.y, wi = a.y + b.x;   // A + iB
-          out[obase[t] + (long long)(2 * K - g) * inner] = make_float2(r.x * wr + r.y * wi, r.x * wi - r.y * wr);
+      } else {
+#pragma unroll
+        for (int t = 0; t < PT; ++t) {
+          if (!ok[t]) continue;
+          if (g < K) out[obase[t] + (long long)g * inner] = zp[t];
+          if (g > 0) out[obase[t] + (long long)(2 * K - g) * inner] = zm[t];
         }
       }
     }
@@ -141,7 +167,7 @@ __global__ void __launch_bounds__(kMidThreads) mid_contract_kernel(const float2*
 //   P_n = sum_g alpha_g cos(psi_g (n+1/2)), Q_n = sum_g beta_g sin(psi_g (n+1/2)),
 //   alpha_g = V'_{+g} + V'_{-g}, beta_g = i (V'_{+g} - V'_{-g}), V'_{+-g} = e^{-+i psi_g/2} V_{+-g}
 // ------------------------------------------------------------------------------------------
-template <int K, int PT>
+template <int K, int PT, bool VEC>
 __global__ void __launch_bounds__(kMidThreads) mid_expand_kernel(const float2* __restrict__ in,
                                                                  float2* __restrict__ out, long long outer,
                                                                  long long inner, int N, float scale) {
@@ -162,26 +188,45 @@ __global__ void __launch_bounds__(kMidThreads) mid_expand_kernel(const float2* _
     float2 al[PT][K + 1], be[PT][K + 1];
 #pragma unroll
     for (int t = 0; t < PT; ++t) {
-      const long long p = tile * per_cta + (long long)t * kMidThreads + threadIdx.x;
+      const long long p = VEC ? tile * per_cta + (long long)threadIdx.x * PT + t
+                              : tile * per_cta + (long long)t * kMidThreads + threadIdx.x;
       ok[t] = p < total;
       const long long pc = ok[t] ? p : 0;
       const long long o = pc / inner, i = pc % inner;
       ibase[t] = o * (2 * K) * inner + i;
       obase[t] = o * N * inner + i;
+    }
 #pragma unroll
-      for (int g = 0; g <= K; ++g) {
-        const float2 r = rho[g];
-        float2 vp = make_float2(0.f, 0.f), vm = make_float2(0.f, 0.f);
+    for (int g = 0; g <= K; ++g) {
+      const float2 r = rho[g];
+      float2 vpl[PT], vmi[PT];
+#pragma unroll
+      for (int t = 0; t < PT; ++t) vpl[t] = vmi[t] = make_float2(0.f, 0.f);
+      if constexpr (VEC) {
         if (g < K) {
-          const float2 v = __ldg(in + ibase[t] + (long long)g * inner);
-          vp = make_float2(v.x * r.x + v.y * r.y, v.y * r.x - v.x * r.y);   // v * conj(rho)
+          const float4 v = __ldg(reinterpret_cast<const float4*>(in + ibase[0] + (long long)g * inner));
+          vpl[0] = make_float2(v.x, v.y);
+          vpl[PT - 1] = make_float2(v.z, v.w);
         }
         if (g > 0) {
-          const float2 v = __ldg(in + ibase[t] + (long long)(2 * K - g) * inner);
-          vm = make_float2(v.x * r.x - v.y * r.y, v.y * r.x + v.x * r.y);   // v * rho
+          const float4 v = __ldg(reinterpret_cast<const float4*>(in + ibase[0] + (long long)(2 * K - g) * inner));
+          vmi[0] = make_float2(v.x, v.y);
+          vmi[PT - 1] = make_float2(v.z, v.w);
         }
+      } else {
+#pragma unroll
+        for (int t = 0; t < PT; ++t) {
+          if (g < K) vpl[t] = __ldg(in + ibase[t] + (long long)g * inner);
+          if (g > 0) vmi[t] = __ldg(in + ibase[t] + (long long)(2 * K - g) * inner);
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < PT; ++t) {
+        const float2 v = vpl[t], u = vmi[t];
+        const float2 vp = make_float2(v.x * r.x + v.y * r.y, v.y * r.x - v.x * r.y);   // v * conj(rho)
+        const float2 vm = make_float2(u.x * r.x - u.y * r.y, u.y * r.x + u.x * r.y);   // u * rho
         al[t][g] = make_float2(vp.x + vm.x, vp.y + vm.y);
-        be[t][g] = make_float2(-(vp.y - vm.y), vp.x - vm.x);                // i (vp - vm)
+        be[t][g] = make_float2(-(vp.y - vm.y), vp.x - vm.x);                           // i (vp - vm)
       }
     }
 #pragma unroll 2
@@ -208,17 +253,26 @@ __global__ void __launch_bounds__(kMidThreads) mid_expand_kernel(const float2* _
           Q[t].y = fmaf(be[t][g].y, s, Q[t].y);
         }
       }
+      if constexpr (VEC) {
+        if (ok[0]) {
+          *reinterpret_cast<float4*>(out + obase[0] + (long long)n * inner) =
+              make_float4(P[0].x + Q[0].x, P[0].y + Q[0].y, P[PT - 1].x + Q[PT - 1].x, P[PT - 1].y + Q[PT - 1].y);
+          *reinterpret_cast<float4*>(out + obase[0] + (long long)(N - 1 - n) * inner) =
+              make_float4(P[0].x - Q[0].x, P[0].y - Q[0].y, P[PT - 1].x - Q[PT - 1].x, P[PT - 1].y - Q[PT - 1].y);
+        }
+      } else {
 #pragma unroll
-      for (int t = 0; t < PT; ++t) {
-        if (!ok[t]) continue;
-        out[obase[t] + (long long)n * inner] = make_float2(P[t].x + Q[t].x, P[t].y + Q[t].y);
-        out[obase[t] + (long long)(N - 1 - n) * inner] = make_float2(P[t].x - Q[t].x, P[t].y - Q[t].y);
+        for (int t = 0; t < PT; ++t) {
+          if (!ok[t]) continue;
+          out[obase[t] + (long long)n * inner] = make_float2(P[t].x + Q[t].x, P[t].y + Q[t].y);
+          out[obase[t] + (long long)(N - 1 - n) * inner] = make_float2(P[t].x - Q[t].x, P[t].y - Q[t].y);
+        }
       }
     }
   }
 }
 
-template <int K, int PT>
+template <int K, int PT, bool VEC>
 cudaError_t launch_mid_t(bool forward, const float2* in, float2* out, long long outer, long long inner, int N,
                          float scale, cudaStream_t st) {
   const size_t smem = (size_t)(N / 2) * MidTab<K>::TS * 4 + (size_t)(K + 1) * 8;
@@ -229,14 +283,14 @@ cudaError_t launch_mid_t(bool forward, const float2* in, float2* out, long long 
   cudaError_t e = cudaSuccess;
   if (forward) {
     if (smem > 48 * 1024)
-      e = cudaFuncSetAttribute(mid_contract_kernel<K, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      e = cudaFuncSetAttribute(mid_contract_kernel<K, PT, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    mid_contract_kernel<K, PT><<<grid, kMidThreads, smem, st>>>(in, out, outer, inner, N, scale);
+    mid_contract_kernel<K, PT, VEC><<<grid, kMidThreads, smem, st>>>(in, out, outer, inner, N, scale);
   } else {
     if (smem > 48 * 1024)
-      e = cudaFuncSetAttribute(mid_expand_kernel<K, PT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      e = cudaFuncSetAttribute(mid_expand_kernel<K, PT, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    mid_expand_kernel<K, PT><<<grid, kMidThreads, smem, st>>>(in, out, outer, inner, N, scale);
+    mid_expand_kernel<K, PT, VEC><<<grid, kMidThreads, smem, st>>>(in, out, outer, inner, N, scale);
   }
   return cudaGetLastError();
 }
@@ -253,13 +307,21 @@ bool mid_supported(int N, int K) {
 cudaError_t launch_mid(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
                        float scale, cudaStream_t st) {
   if (outer * inner <= 0) return cudaSuccess;
+  // two adjacent positions per thread need an even inner extent (then every pair is 16-byte aligned and
+  // never straddles two outer slices) and 16-byte aligned tensors
+  const bool vec = (inner % 2 == 0) && ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
+#define DTST_MID_CASE(KK)                                                                          \
+  case KK:                                                                                         \
+    return vec ? launch_mid_t<KK, 2, true>(forward, in, out, outer, inner, N, scale, st)           \
+               : launch_mid_t<KK, 2, false>(forward, in, out, outer, inner, N, scale, st);
   switch (K) {
-    case 4: return launch_mid_t<4, 2>(forward, in, out, outer, inner, N, scale, st);
-    case 8: return launch_mid_t<8, 2>(forward, in, out, outer, inner, N, scale, st);
-    case 12: return launch_mid_t<12, 2>(forward, in, out, outer, inner, N, scale, st);
-    case 16: return launch_mid_t<16, 2>(forward, in, out, outer, inner, N, scale, st);
+    DTST_MID_CASE(4)
+    DTST_MID_CASE(8)
+    DTST_MID_CASE(12)
+    DTST_MID_CASE(16)
     default: return cudaErrorNotSupported;
   }
+#undef DTST_MID_CASE
 }
 
 }  // namespace dtst
