@@ -12,6 +12,8 @@
 //     B_g = sum_{q<Q/2} (z_q - z_{Q-1-q}) sin(psi_g (q + 1/2)),
 // one real-coefficient FMA pair serves both +g and -g and both mirrored inputs: a fourfold
 // cut of the multiply count against the plain complex matrix product.
+#include <type_traits>
+
 #include "dtst_common.cuh"
 
 namespace dtst {
@@ -87,43 +89,83 @@ __global__ void __launch_bounds__(kMidThreads) mid_contract_kernel(const float2*
 #pragma unroll
       for (int g = 0; g <= K; ++g) A[t][g] = B[t][g] = make_float2(0.f, 0.f);
 
-#pragma unroll 4
-    for (int q = 0; q < half; ++q) {
-      float2 p[PT], m[PT];
-      if constexpr (VEC) {
-        static_assert(!VEC || PT == 2, "vector path handles two adjacent positions");
-        const float4 a = __ldg(reinterpret_cast<const float4*>(in + ibase[0] + (long long)q * inner));
-        const float4 b = __ldg(reinterpret_cast<const float4*>(in + ibase[0] + (long long)(N - 1 - q) * inner));
-        p[0] = make_float2(a.x + b.x, a.y + b.y);
-        m[0] = make_float2(a.x - b.x, a.y - b.y);
-        p[PT - 1] = make_float2(a.z + b.z, a.w + b.w);
-        m[PT - 1] = make_float2(a.z - b.z, a.w - b.w);
-      } else {
+    // Software pipeline over blocks of U mirrored row pairs: the loads of block b+1 are in flight while
+    // block b is accumulated (a plain unrolled loop leaves only a couple of loads outstanding per warp,
+    // which makes this stage latency-bound), and rows a few blocks ahead are pulled into L2.
+    constexpr int U = 4;
+    constexpr int NV = VEC ? 1 : PT;
+    using Vec = typename std::conditional<VEC, float4, float2>::type;
+    Vec nxa[U][NV], nxb[U][NV];
+    auto issue = [&](int q0) {
 #pragma unroll
-        for (int t = 0; t < PT; ++t) {
-          const float2 a = __ldg(in + ibase[t] + (long long)q * inner);
-          const float2 b = __ldg(in + ibase[t] + (long long)(N - 1 - q) * inner);
-          p[t] = make_float2(a.x + b.x, a.y + b.y);
-          m[t] = make_float2(a.x - b.x, a.y - b.y);
+      for (int u = 0; u < U; ++u) {
+        const int q = q0 + u;
+        if (q < half) {
+#pragma unroll
+          for (int t = 0; t < NV; ++t) {
+            nxa[u][t] = __ldg(reinterpret_cast<const Vec*>(in + ibase[t] + (long long)q * inner));
+            nxb[u][t] = __ldg(reinterpret_cast<const Vec*>(in + ibase[t] + (long long)(N - 1 - q) * inner));
+          }
         }
       }
-      const float* row = tab + q * TS;
+    };
+    issue(0);
+    for (int q0 = 0; q0 < half; q0 += U) {
+      Vec cua[U][NV], cub[U][NV];
 #pragma unroll
-      for (int g = 0; g <= K; ++g) {
-        const float c = row[g];
+      for (int u = 0; u < U; ++u)
 #pragma unroll
-        for (int t = 0; t < PT; ++t) {
-          A[t][g].x = fmaf(p[t].x, c, A[t][g].x);
-          A[t][g].y = fmaf(p[t].y, c, A[t][g].y);
+        for (int t = 0; t < NV; ++t) {
+          cua[u][t] = nxa[u][t];
+          cub[u][t] = nxb[u][t];
         }
+      issue(q0 + U);
+      if (q0 + 4 * U < half) {
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+          for (int t = 0; t < NV; ++t) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(in + ibase[t] + (long long)(q0 + 4 * U + u) * inner));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(in + ibase[t] + (long long)(N - 1 - q0 - 4 * U - u) * inner));
+          }
       }
 #pragma unroll
-      for (int g = 1; g <= K; ++g) {
-        const float s = row[K + g];
+      for (int u = 0; u < U; ++u) {
+        const int q = q0 + u;
+        if (q >= half) break;
+        float2 p[PT], m[PT];
+        if constexpr (VEC) {
+          const float4 a = cua[u][0], b = cub[u][0];
+          p[0] = make_float2(a.x + b.x, a.y + b.y);
+          m[0] = make_float2(a.x - b.x, a.y - b.y);
+          p[PT - 1] = make_float2(a.z + b.z, a.w + b.w);
+          m[PT - 1] = make_float2(a.z - b.z, a.w - b.w);
+        } else {
 #pragma unroll
-        for (int t = 0; t < PT; ++t) {
-          B[t][g].x = fmaf(m[t].x, s, B[t][g].x);
-          B[t][g].y = fmaf(m[t].y, s, B[t][g].y);
+          for (int t = 0; t < PT; ++t) {
+            const float2 a = cua[u][t], b = cub[u][t];
+            p[t] = make_float2(a.x + b.x, a.y + b.y);
+            m[t] = make_float2(a.x - b.x, a.y - b.y);
+          }
+        }
+        const float* row = tab + q * TS;
+#pragma unroll
+        for (int g = 0; g <= K; ++g) {
+          const float c = row[g];
+#pragma unroll
+          for (int t = 0; t < PT; ++t) {
+            A[t][g].x = fmaf(p[t].x, c, A[t][g].x);
+            A[t][g].y = fmaf(p[t].y, c, A[t][g].y);
+          }
+        }
+#pragma unroll
+        for (int g = 1; g <= K; ++g) {
+          const float s = row[K + g];
+#pragma unroll
+          for (int t = 0; t < PT; ++t) {
+            B[t][g].x = fmaf(m[t].x, s, B[t][g].x);
+            B[t][g].y = fmaf(m[t].y, s, B[t][g].y);
+          }
         }
       }
     }
@@ -278,21 +320,21 @@ cudaError_t launch_mid_t(bool forward, const float2* in, float2* out, long long 
   const size_t smem = (size_t)(N / 2) * MidTab<K>::TS * 4 + (size_t)(K + 1) * 8;
   const long long total = outer * inner;
   const long long tiles = (total + (long long)kMidThreads * PT - 1) / ((long long)kMidThreads * PT);
-  const long long cap = (long long)kNumSMs * 3;
-  const int grid = (int)(tiles < cap ? tiles : cap);
-  cudaError_t e = cudaSuccess;
-  if (forward) {
-    if (smem > 48 * 1024)
-      e = cudaFuncSetAttribute(mid_contract_kernel<K, PT, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  // persistent CTAs: exactly as many as are resident at once, so that no CTA starts late
+  auto launch = [&](auto kern) -> cudaError_t {
+    cudaError_t e = cudaSuccess;
+    if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    mid_contract_kernel<K, PT, VEC><<<grid, kMidThreads, smem, st>>>(in, out, outer, inner, N, scale);
-  } else {
-    if (smem > 48 * 1024)
-      e = cudaFuncSetAttribute(mid_expand_kernel<K, PT, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kMidThreads, smem);
     if (e != cudaSuccess) return e;
-    mid_expand_kernel<K, PT, VEC><<<grid, kMidThreads, smem, st>>>(in, out, outer, inner, N, scale);
-  }
-  return cudaGetLastError();
+    if (per_sm < 1) per_sm = 1;
+    const long long cap = (long long)kNumSMs * per_sm;
+    const int grid = (int)(tiles < cap ? tiles : cap);
+    kern<<<grid, kMidThreads, smem, st>>>(in, out, outer, inner, N, scale);
+    return cudaGetLastError();
+  };
+  return forward ? launch(mid_contract_kernel<K, PT, VEC>) : launch(mid_expand_kernel<K, PT, VEC>);
 }
 
 }  // namespace
