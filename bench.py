@@ -63,7 +63,7 @@ class ClockSampler:
             self.fh = open(self.path, "w")
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=self.fh, stderr=subprocess.DEVNULL)
+                 "-lms", "20"], stdout=self.fh, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -102,6 +102,18 @@ class ClockSampler:
         except Exception:
             pass
         return out
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu launch list of this
+# very command at full size; the summary with the command line is profiles/launch_list_cfg5_4d_128.md.
+NCU_TRAFFIC = {
+    "cfg5_4d_128": {"grid_read": 8590074368 + 533445632, "grid_write": 537079040 + 8526035968,
+                    "mix": 661641216 + 28915456, "mix_adjoint": 998619136 + 537102592},
+}
+
+
+def measured_traffic(workload: str, kind: str):
+    return NCU_TRAFFIC.get(workload, {}).get(kind)
 
 
 def algorithmic_bytes(w):
@@ -170,9 +182,10 @@ def time_oracle(w, steps, warmup, budget=1.7e7):
     sample_ptch = w.B * (w.points // w.N[0]) * n0 * cs
     # equivalent whole-layer grid points per second at the workload's channel count
     value = sample_ptch / max(w.C_in, w.C_out) / dt / 1e9
-    sample = (f"float64 numpy oracle, fwd+bwd, {cs} of {w.C_in} channels (in and out), first {n0} of {w.N[0]} "
-              f"planes along dim 0 (slab with global phase offset); value = sample point-channels / "
-              f"{max(w.C_in, w.C_out)} channels / time")
+    grid_part = (f"the whole grid" if n0 == w.N[0] else
+                 f"first {n0} of {w.N[0]} planes along dim 0 (a slab, with its global phase offset)")
+    sample = (f"float64 numpy oracle, fwd+bwd, {cs} of {w.C_in} channels (in and out), {grid_part}; "
+              f"value = sample point-channels / {max(w.C_in, w.C_out)} channels / time")
     return value, dt, {"kind": "oracle", "cores": int(min(threads, len(os.sched_getaffinity(0)))),
                        "host_cores": len(os.sched_getaffinity(0)), "sample": sample,
                        "seconds_per_sample_step": dt}
@@ -267,17 +280,14 @@ def main_ours(args, w):
     import torch
     import torch.distributed as dist
     from paper_2607_14394_b200 import Plan, inputs
+    from paper_2607_14394_b200 import dist as D
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local_rank = D.env_world()
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the spectral layer has no CPU path")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
+    D.init_process_group("nccl", dev)
 
     steps, warmup = max(1, args.steps), max(3, args.warmup)
     P = args.shards
@@ -342,13 +352,11 @@ def main_ours(args, w):
     kt = {k: plan.kernel_timing(k) for k in ("grid_read", "grid_write", "mix", "mix_adjoint")}
     plan.enable_kernel_timing(0)
 
-    if world > 1:
-        t = torch.tensor([ms_step] + ph, dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step, ph = float(t[0]), [float(v) for v in t[1:]]
+    red = D.max_over_ranks([ms_step] + ph, device=dev)
+    ms_step, ph = red[0], red[1:]
 
     pts_per_step = world * w.B * w.points
-    value = pts_per_step / (ms_step * 1e-3) / 1e9
+    value = D.whole_job_throughput(w.B * w.points, ms_step, world) / 1e9
     fwd_ms = ph[0] + ph[1] + ph[2]
     ab = algorithmic_bytes(w)
     peak, peak_src = measured_peaks()
@@ -373,7 +381,7 @@ def main_ours(args, w):
     if dom:
         a = kinds[dom]["achieved_gbs"]
         roofline = {"bound": "hbm", "kernel": dom, "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
-                    "frac_of_nominal_8TBs": a / 8000.0, "traffic": None, "peak_source": peak_src,
+                    "frac_of_nominal_8TBs": a / 8000.0, "traffic": measured_traffic(w.name, dom), "peak_source": peak_src,
                     "avg_launch_ms": kinds[dom]["avg_ms"]}
 
     # end to end through host buffers: pinned host -> device copies of x and g_y, the step,
@@ -411,10 +419,7 @@ def main_ours(args, w):
             torch.cuda.synchronize()
             barrier()
             ms_e = a0.elapsed_time(a1) / e2e_steps
-            if world > 1:
-                t = torch.tensor([ms_e], dtype=torch.float64, device=dev)
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                ms_e = float(t[0])
+            ms_e = D.max_over_ranks([ms_e], device=dev)[0]
             e2e = {"value": pts_per_step / (ms_e * 1e-3) / 1e9, "unit": UNIT,
                    "h2d_bytes_per_step": int(hx.numel() * 4 + hg.numel() * 4),
                    "d2h_bytes_per_step": int(hy.numel() * 4 + hgx.numel() * 4 + hgW.numel() * 8),

@@ -1,0 +1,134 @@
+"""Parity at the benchmark's full sizes (the two large configurations), in the launch
+configuration bench.py times.  The oracle cannot afford every channel of an 8.6 GB tensor,
+so each output is checked on whole channels the oracle CAN compute (a channel of the layer's
+grid-side stages is independent of the others), on single modes by the literal un-factored
+sum of Eq. 5, and on sampled grid points by the literal sum of Eq. 14.  Inputs are seeded,
+generated on the device, and the very same bits are copied to the host for the oracle."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import dtst_oracle as O
+from paper_2607_14394_b200 import inputs as I
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5
+
+
+def _lists(w):
+    return O.mode_index_lists(w.N, w.kmax)
+
+
+def _literal_points(Y_c, w, points, doubling=True, normalise=True):
+    """y[n] at the given grid points for one channel, by the un-factored sum over all modes (Eq. 14)."""
+    lists = _lists(w)
+    c = O.hermitian_weights(w.N[-1], w.kmax[-1]) if doubling else np.ones(w.kmax[-1])
+    out = []
+    for n in points:
+        ph = np.ones((), dtype=np.complex128)
+        for j in range(w.d):
+            r = np.mod(lists[j] * int(n[j]), w.N[j]).astype(np.float64)
+            f = np.exp(2j * np.pi * r / w.N[j])
+            shape = [1] * w.d
+            shape[j] = len(lists[j])
+            ph = ph * f.reshape(shape)
+        v = np.sum(c * np.real(Y_c.astype(np.complex128) * ph))
+        out.append(v / math.prod(w.N) if normalise else v)
+    return np.array(out)
+
+
+def _check_layer_fullsize(w, P_list, check_channels, rng_seed):
+    from paper_2607_14394_b200 import Plan
+    dev = torch.device("cuda")
+    rng = np.random.default_rng(rng_seed)
+    x = I.make_field_torch(w, dev, tag=0)
+    W = I.make_weights_torch(w, dev)
+    plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out)
+    assert plan.kernel_path in ("fused", "generic")
+    lists = _lists(w)
+    for j in range(w.d):
+        assert plan.mode_indices(j) == lists[j].tolist()
+
+    # ---- F: whole channels against the separable oracle, single modes against the literal sum
+    Xhat = plan.forward(x)
+    torch.cuda.synchronize()
+    assert plan.status() == 0
+    x_host = {c: x[0, c].cpu().numpy() for c in check_channels}
+    X_ref = {c: O.forward(x_host[c][None, None], w.kmax)[0, 0] for c in check_channels}
+    for c in check_channels:
+        assert O.rel_l2(Xhat[0, c].cpu().numpy(), X_ref[c]) <= TOL
+    c0 = check_channels[0]
+    for _ in range(3):
+        pos = tuple(int(rng.integers(0, len(s))) for s in lists)
+        v = O.forward_one_mode(x_host[c0], w.N, [lists[j][pos[j]] for j in range(w.d)])
+        got = complex(Xhat[(0, c0) + pos].item())
+        assert abs(got - v) <= 1e-5 * np.sqrt(np.mean(np.abs(X_ref[c0]) ** 2)) + 1e-5 * abs(v)
+
+    # ---- V: virtual shards against the unsharded device result and the oracle
+    for P in P_list:
+        planP = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out, virtual_shards=P)
+        XP = planP.forward(x)
+        torch.cuda.synchronize()
+        a = torch.view_as_real(XP).double()
+        b = torch.view_as_real(Xhat).double()
+        assert float((a - b).norm() / b.norm()) <= TOL
+        for c in check_channels:
+            assert O.rel_l2(XP[0, c].cpu().numpy(), X_ref[c]) <= TOL
+        del planP, XP
+
+    # ---- M: full size against the oracle's einsum, on an independent random spectrum
+    Xs = torch.from_numpy(I.make_spectrum(w, w.C_in, tag=3).reshape((w.B, w.C_in) + w.K)).to(dev)
+    Yhat = plan.spectral_mul(Xs, W)
+    Y_ref = O.spectral_mul(Xs.cpu().numpy(), W.cpu().numpy().reshape((w.C_in, w.C_out) + w.K))
+    assert O.rel_l2(Yhat.cpu().numpy(), Y_ref) <= TOL
+
+    # ---- I: one whole channel against the separable oracle, sampled points against the literal sum
+    y = plan.inverse(Yhat)
+    torch.cuda.synchronize()
+    co = check_channels[-1] % w.C_out
+    y_ref = O.inverse(Y_ref[0, co][None, None], w.N, w.kmax)[0, 0]
+    assert O.rel_l2(y[0, co].cpu().numpy(), y_ref) <= TOL
+    rms = float(np.sqrt(np.mean(y_ref ** 2)))
+    pts = [tuple(int(rng.integers(0, n)) for n in w.N) for _ in range(24)]
+    lit = _literal_points(Y_ref[0, (co + 1) % w.C_out], w, pts)
+    got = np.array([float(y[(0, (co + 1) % w.C_out) + p].item()) for p in pts])
+    assert np.max(np.abs(got - lit)) <= 2e-5 * rms
+    del y, y_ref
+
+    # ---- B: upstream gradient with two live channels (the others are exactly zero, which keeps the
+    # oracle's share to two forward transforms while every kernel still runs at full size)
+    live = sorted({check_channels[0] % w.C_out, check_channels[-1] % w.C_out})
+    g = torch.zeros((w.B, w.C_out) + w.N, device=dev)
+    for o in live:
+        g[0, o] = I.make_field_channel_torch(w, 0, o, dev, tag=1)
+    gx, gW = plan.backward(g, Xs, W)
+    torch.cuda.synchronize()
+    assert plan.status() == 0
+    cw = O.hermitian_weights(w.N[-1], w.kmax[-1])
+    GY = {o: O.forward(g[0, o].cpu().numpy()[None, None], w.kmax)[0, 0] * cw / float(math.prod(w.N)) for o in live}
+    Xs_h = Xs.cpu().numpy()
+    W_h = W.cpu().numpy().reshape((w.C_in, w.C_out) + w.K)
+    gW_h = gW.cpu().numpy().reshape((w.C_in, w.C_out) + w.K)
+    for o in live:
+        ref = np.conj(Xs_h[0]) * GY[o][None]               # [C_in, K...], B = 1
+        assert O.rel_l2(gW_h[:, o], ref) <= TOL
+    dead = [o for o in range(w.C_out) if o not in live][0]
+    assert float(np.abs(gW_h[:, dead]).max()) == 0.0
+    i0 = check_channels[0] % w.C_in
+    GX = sum(GY[o] * np.conj(W_h[i0, o]) for o in live)
+    gx_ref = O.inverse(GX[None, None], w.N, w.kmax, doubling=False, normalise=False)[0, 0]
+    assert O.rel_l2(gx[0, i0].cpu().numpy(), gx_ref) <= TOL
+    plan.close()
+
+
+def test_cfg5_4d_128_fullsize():
+    w = I.WORKLOADS["cfg5_4d_128"]
+    _check_layer_fullsize(w, P_list=[w.virtual_shards], check_channels=[0, 9], rng_seed=55)
+
+
+def test_cfg4_3d_256_fullsize():
+    w = I.WORKLOADS["cfg4_3d_256"]
+    _check_layer_fullsize(w, P_list=[4], check_channels=[1, 30], rng_seed=44)
