@@ -55,7 +55,7 @@ struct PlaneCfg {
   static constexpr int MT2 = 2;                               // inverse: MMA m-tiles over the 32 quadruples
   static constexpr int GT = K2 / 2;                           // frequencies per parity class
   static constexpr int NS = 4 * NC + 8;                       // floats per combo row: 4 classes x NC, +8 pad
-  static constexpr int ABS = NC + 4;                          // floats between A/B entries
+  static constexpr int ABS = NC + 1;                          // floats between A/B entries (odd: scalar accesses)
   static constexpr int ABP = (2 * K2 + 1) * ABS;
   static constexpr int COMBO_FLOATS = (32 * NS > G * ABP ? 32 * NS : G * ABP);
   static_assert(N3 % 32 == 0 && (N3 == 32 || N3 == 64), "N3");
@@ -204,7 +204,7 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
     double sn, cs;
     sincospi((double)num / (double)((long long)N2 * N3), &sn, &cs);
     const float w = scale * (herm ? herm_weight(f, N3) : 1.0f);
-    rot[e] = make_float2((float)cs * w, (float)sn * w);
+    rot[f * (2 * K2) + r] = make_float2((float)cs * w, (float)sn * w);   // [f][r]: lanes (r) read conflict-free
   }
   __syncthreads();
 
@@ -405,7 +405,7 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
         const float* A = combo + pl2 * Cfg::ABP + g * Cfg::ABS;
         const float* Bp = combo + pl2 * Cfg::ABP + (K2 + g) * Cfg::ABS;
         float2* dst = out + ((task * G + pl2) * (2 * K2) + r) * K3;
-        const float2* rr = rot + r * K3;
+        const float2* rr = rot + r;
 #pragma unroll
         for (int f2 = 0; f2 < K3 / 2; ++f2) {
           float res[4];
@@ -416,7 +416,7 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
             const float BC = g > 0 ? Bp[f] : 0.f, BS = g > 0 ? Bp[K3 + f] : 0.f;
             const float wr = pos ? AC - BS : AC + BS;
             const float wi = pos ? -(AS + BC) : BC - AS;
-            const float2 ro = rr[f];
+            const float2 ro = rr[f * (2 * K2)];
             res[2 * e] = ro.x * wr - ro.y * wi;
             res[2 * e + 1] = ro.x * wi + ro.y * wr;
           }
@@ -521,7 +521,7 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
     double sn, cs;
     sincospi((double)num / (double)((long long)N2 * N3), &sn, &cs);
     const float w = scale * (herm ? herm_weight(f, N3) : 1.0f);
-    rot[e] = make_float2((float)cs * w, -(float)sn * w);
+    rot[f * (2 * K2) + r] = make_float2((float)cs * w, -(float)sn * w);   // [f][r]
   }
   __syncthreads();
 
@@ -576,11 +576,11 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
     // ---- rotate this task's modes, publish V'
     if (actl) {
       float* dst = ab + pll * IC::ABP + rl * IC::ABS;
-      const float2* rr = rot + rl * K3;
+      const float2* rr = rot + rl;
       float re[K3], im[K3];
 #pragma unroll
       for (int i = 0; i < K3 / 2; ++i) {
-        const float2 r0 = rr[2 * i], r1 = rr[2 * i + 1];
+        const float2 r0 = rr[(2 * i) * (2 * K2)], r1 = rr[(2 * i + 1) * (2 * K2)];
         re[2 * i] = vin[i].x * r0.x - vin[i].y * r0.y;
         im[2 * i] = vin[i].x * r0.y + vin[i].y * r0.x;
         re[2 * i + 1] = vin[i].z * r1.x - vin[i].w * r1.y;
