@@ -84,7 +84,7 @@ cudaError_t launch_apply_dim(const DimOp& op_in, bool in_real, bool out_real, co
   if (in_real && !out_real) DTST_LAUNCH(true, false);
   else if (!in_real && out_real) DTST_LAUNCH(false, true);
   else if (!in_real && !out_real) DTST_LAUNCH(false, false);
-  else return cudaErrorInvalidValue;   // real -> real only happens for d == 1; handled by the caller
+  else return cudaErrorInvalidValue;   // real -> real never occurs: a real grid maps to a complex spectrum
 #undef DTST_LAUNCH
   if (err != cudaSuccess) return err;
   return cudaGetLastError();
