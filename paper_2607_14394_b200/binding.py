@@ -366,3 +366,68 @@ class Plan:
             self.close()
         except Exception:
             pass
+
+
+class HostPipeline:
+    """The whole step (F, M, I, B) for callers whose activations live in pinned HOST memory.
+
+    Three CUDA streams - copy-in, compute, copy-out - are chained with events so that the PCIe transfers of
+    x and grad_y in, and of y, grad_x and grad_W out, overlap the kernels and each other, also across
+    consecutive calls of `step`.  Every byte still crosses the bus inside the call; nothing is cached.
+    W stays on the device (it is the layer's parameter).
+    """
+
+    def __init__(self, plan: Plan, W: torch.Tensor):
+        self.plan, self.W = plan, W
+        dev, p = plan.device, plan
+        self.x = torch.empty((p.B, p.C_in) + p.N, dtype=torch.float32, device=dev)
+        self.g = torch.empty((p.B, p.C_out) + p.N, dtype=torch.float32, device=dev)
+        self.Xhat = torch.empty((p.B, p.C_in) + p.K, dtype=torch.complex64, device=dev)
+        self.Yhat = torch.empty((p.B, p.C_out) + p.K, dtype=torch.complex64, device=dev)
+        self.y = torch.empty((p.B, p.C_out) + p.N, dtype=torch.float32, device=dev)
+        self.gx = torch.empty((p.B, p.C_in) + p.N, dtype=torch.float32, device=dev)
+        self.gW = torch.empty((p.C_in, p.C_out, p.M), dtype=torch.complex64, device=dev)
+        self.s_in, self.s_cmp, self.s_out = (torch.cuda.Stream(device=dev) for _ in range(3))
+        ev = lambda: torch.cuda.Event()
+        self.ev_x, self.ev_g, self.ev_fwd_read, self.ev_y, self.ev_b = ev(), ev(), ev(), ev(), ev()
+        self.ev_y_copied, self.ev_done = ev(), ev()
+        self._first = True
+
+    def step(self, hx, hg, hy, hgx, hgW):
+        """Enqueue one step; all five host tensors must be pinned.  Returns immediately; call `wait()`."""
+        p = self.plan
+        with torch.cuda.stream(self.s_in):
+            if not self._first:
+                self.s_in.wait_event(self.ev_fwd_read)     # previous F has consumed x
+            self.x.copy_(hx, non_blocking=True)
+            self.ev_x.record(self.s_in)
+            if not self._first:
+                self.s_in.wait_event(self.ev_b)            # previous B has consumed grad_y
+            self.g.copy_(hg, non_blocking=True)
+            self.ev_g.record(self.s_in)
+        with torch.cuda.stream(self.s_cmp):
+            self.s_cmp.wait_event(self.ev_x)
+            p.forward(self.x, self.Xhat, stream=self.s_cmp)
+            self.ev_fwd_read.record(self.s_cmp)
+            p.spectral_mul(self.Xhat, self.W, self.Yhat, stream=self.s_cmp)
+            if not self._first:
+                self.s_cmp.wait_event(self.ev_y_copied)    # previous y has left the device
+            p.inverse(self.Yhat, self.y, stream=self.s_cmp)
+            self.ev_y.record(self.s_cmp)
+            self.s_cmp.wait_event(self.ev_g)
+            if not self._first:
+                self.s_cmp.wait_event(self.ev_done)        # previous grad_x / grad_W have left the device
+            p.backward(self.g, self.Xhat, self.W, self.gx, self.gW, stream=self.s_cmp)
+            self.ev_b.record(self.s_cmp)
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.ev_y)
+            hy.copy_(self.y, non_blocking=True)
+            self.ev_y_copied.record(self.s_out)
+            self.s_out.wait_event(self.ev_b)
+            hgx.copy_(self.gx, non_blocking=True)
+            hgW.copy_(self.gW, non_blocking=True)
+            self.ev_done.record(self.s_out)
+        self._first = False
+
+    def wait(self):
+        self.ev_done.synchronize()

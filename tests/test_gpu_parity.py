@@ -216,3 +216,35 @@ def test_adjoint_identity_on_device():
     Yc = (Y / c).contiguous()
     rhs = (x.double() * plan.inverse(Yc).double()).sum().item() * float(np.prod(w.N))
     assert abs(lhs - rhs) <= 1e-5 * max(1.0, abs(lhs))
+
+
+def test_host_pipeline_matches_device_path_over_consecutive_steps():
+    # pinned host buffers in and out, copies overlapped with compute on three streams: same bits as the plain path
+    from paper_2607_14394_b200 import Plan
+    from paper_2607_14394_b200.binding import HostPipeline
+    w = I.custom_workload("hostpipe", 1, 2, 2, (16, 16, 64, 32), (2, 3, 8, 4), field="grf", seed=61)
+    plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out)
+    Wd = _dev(I.make_weights(w))
+    pipe = HostPipeline(plan, Wd)
+    outs = []
+    for rep in range(3):
+        wv = I.custom_workload("hostpipe", 1, 2, 2, w.N, w.kmax, field="grf", seed=61 + rep)
+        hx = torch.from_numpy(I.make_field(wv)).pin_memory()
+        hg = torch.from_numpy(I.make_upstream_grad(wv)).pin_memory()
+        hy, hgx = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
+        hgW = torch.empty((w.C_in, w.C_out, w.M), dtype=torch.complex64).pin_memory()
+        pipe.step(hx, hg, hy, hgx, hgW)
+        outs.append((hx, hg, hy, hgx, hgW))
+    pipe.wait()
+    torch.cuda.synchronize()
+    ref_plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out)
+    for hx, hg, hy, hgx, hgW in outs:
+        y, Xhat = ref_plan.layer(hx.cuda(), Wd)
+        gx, gW = ref_plan.backward(hg.cuda(), Xhat, Wd)
+        torch.cuda.synchronize()
+        assert torch.equal(hy, y.cpu()) and torch.equal(hgx, gx.cpu())
+        assert torch.equal(torch.view_as_real(hgW), torch.view_as_real(gW.cpu()))
+    # and the first of them against the oracle
+    hx, hg, hy, hgx, hgW = outs[0]
+    y_ref, X_ref = O.layer_forward(hx.numpy(), Wd.cpu().numpy(), w.kmax)
+    assert O.rel_l2(hy.numpy(), y_ref) <= TOL
