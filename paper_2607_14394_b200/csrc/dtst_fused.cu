@@ -170,7 +170,9 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
   constexpr int SPT = Cfg::SPT, RPS = Cfg::ROWS_PER_STAGE;
 
   extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // 1024-byte alignment for the TMA swizzle, by pointer arithmetic on the shared array itself (an integer
+  // round trip would make the compiler lose the address space and emit generic loads and stores)
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char* ring = smem;
   float* combos_all = reinterpret_cast<float*>(smem + (size_t)stages * kStageBytes);
   float2* rot = reinterpret_cast<float2*>(combos_all + (size_t)W * Cfg::COMBO_FLOATS);
@@ -506,7 +508,9 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
   constexpr int SPT = Cfg::SPT, RPS = Cfg::ROWS_PER_STAGE;
 
   extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // 1024-byte alignment for the TMA swizzle, by pointer arithmetic on the shared array itself (an integer
+  // round trip would make the compiler lose the address space and emit generic loads and stores)
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   char* staging = reinterpret_cast<char*>(smem) + (size_t)warp * IC::WARP_BYTES;
   float* ab = reinterpret_cast<float*>(IC::ALIAS ? staging : staging + IC::STAGING_BYTES);
@@ -796,7 +800,7 @@ void fill_stage1_table(Stage1Table<N3, K3>* t) {
 template <int N3, int K3, int N2, int K2>
 cudaError_t launch_fwd_plane_t(const float* x, float2* out, long long rows, float scale, int herm, int* status,
                                cudaStream_t st) {
-  constexpr int W = 6;
+  constexpr int W = 7;   // 7 consumer warps + the producer warp = 256 threads x 255 registers = the whole file
   using Cfg = PlaneCfg<N3, K3, N2, K2>;
   const SmemPlan sp = smem_plan<Cfg, K2, K3, W>();
   if (sp.stages < 2 * Cfg::SPT) return cudaErrorInvalidConfiguration;
