@@ -89,6 +89,22 @@ SmemPlan smem_plan() {
 
 __device__ __forceinline__ float4 lds128(const char* p) { return *reinterpret_cast<const float4*>(p); }
 
+// 16-byte shared-memory access by 32-bit shared-space address (+ immediate byte offset).  Volatile: a ring
+// slot is refilled by the TMA engine between two reads of the same address, which the compiler cannot see.
+template <int IMM>
+__device__ __forceinline__ float4 lds128_s(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+%5];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "r"(addr), "n"(IMM));
+  return v;
+}
+template <int IMM>
+__device__ __forceinline__ void sts128_s(uint32_t addr, float a, float b, float c, float d) {
+  asm volatile("st.shared.v4.f32 [%0+%1], {%2,%3,%4,%5};" ::"r"(addr), "n"(IMM), "f"(a), "f"(b), "f"(c), "f"(d)
+               : "memory");
+}
+
 // fp32 -> (hi, lo) TF32 pair with hi + lo = v to ~2^-22 relative (error-compensated "3xTF32")
 __device__ __forceinline__ void split_tf32(float v, uint32_t& hi, uint32_t& lo) {
   asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(v));
@@ -105,21 +121,30 @@ __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], 
 }
 
 // One row of N3 reals -> C_f = sum u cos, S_f = sum v sin for f < K3 (half-sample phase deferred).
-template <int N3, int K3>
-__device__ __forceinline__ void stage1_row(const char* stage, int box_rows, int row,
-                                           const Stage1Table<N3, K3>& tab, float (&o)[2 * K3]) {
+// `stage` is the 32-bit shared address of the slot (1024-byte aligned), BOXR its rows per 128-byte panel.
+template <int N3, int K3, int BOXR>
+__device__ __forceinline__ void stage1_row(uint32_t stage, int row, const Stage1Table<N3, K3>& tab,
+                                           float (&o)[2 * K3]) {
   constexpr int CH = N3 / 4;
 #pragma unroll
   for (int i = 0; i < 2 * K3; ++i) o[i] = 0.f;
-  const uint32_t sw = (uint32_t)(row & 7);
-  const char* rbase = stage + (size_t)row * 128;
+  // chunk c of this row sits at row*128 + ((c ^ (row & 7)) << 4) (+ one panel for c >= 8); the row base has
+  // zeros in bits 4..6, so the swizzle is a single XOR of a precomputed base with a constant
+  const uint32_t rx = stage + (uint32_t)row * 128u + (((uint32_t)row & 7u) << 4);
 #pragma unroll
   for (int c = 0; c < CH / 4; ++c) {
+    constexpr int P = BOXR * 128;
     const int c0 = c, c1 = CH / 2 - 1 - c, c2 = CH / 2 + c, c3 = CH - 1 - c;
-    const float4 A = lds128(rbase + (size_t)(c0 / 8) * box_rows * 128 + (((uint32_t)(c0 % 8) ^ sw) << 4));
-    const float4 Bq = lds128(rbase + (size_t)(c1 / 8) * box_rows * 128 + (((uint32_t)(c1 % 8) ^ sw) << 4));
-    const float4 Cq = lds128(rbase + (size_t)(c2 / 8) * box_rows * 128 + (((uint32_t)(c2 % 8) ^ sw) << 4));
-    const float4 D = lds128(rbase + (size_t)(c3 / 8) * box_rows * 128 + (((uint32_t)(c3 % 8) ^ sw) << 4));
+    float4 A, Bq, Cq, D;
+    // (the panel offset is an immediate, the XOR constant depends on c only)
+#define DTST_LD(dst, cc)                                                        \
+    dst = ((cc) / 8 == 0) ? lds128_s<0>(rx ^ (uint32_t)(((cc) % 8) << 4))       \
+                          : lds128_s<P>(rx ^ (uint32_t)(((cc) % 8) << 4));
+    DTST_LD(A, c0)
+    DTST_LD(Bq, c1)
+    DTST_LD(Cq, c2)
+    DTST_LD(D, c3)
+#undef DTST_LD
     const float a[4] = {A.x, A.y, A.z, A.w};
     const float b[4] = {Bq.w, Bq.z, Bq.y, Bq.x};
     const float cc[4] = {Cq.x, Cq.y, Cq.z, Cq.w};
@@ -174,6 +199,7 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
   // round trip would make the compiler lose the address space and emit generic loads and stores)
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char* ring = smem;
+  const uint32_t ring_s = smem_u32(ring);
   float* combos_all = reinterpret_cast<float*>(smem + (size_t)stages * kStageBytes);
   float2* rot = reinterpret_cast<float2*>(combos_all + (size_t)W * Cfg::COMBO_FLOATS);
   uint64_t* full = reinterpret_cast<uint64_t*>(rot + 2 * K2 * K3);
@@ -305,9 +331,9 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
         const float s3 = (r4 == 0 || r4 == 2) ? 1.f : -1.f;
         const int trow = pl1 * N2 + rowq;
         const int sl = (trow / RPS) ? slot1 : slot0;
-        const char* st = reinterpret_cast<const char*>(ring) + (size_t)sl * kStageBytes;
+        const uint32_t st = ring_s + (uint32_t)sl * kStageBytes;
         float o[NC];
-        stage1_row<N3, K3>(st, RPS, trow % RPS, tab, o);
+        stage1_row<N3, K3, RPS>(st, trow % RPS, tab, o);
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
           cpp[c] += o[c];
@@ -439,12 +465,13 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
 // modes, forms alpha_g = V'_{+g} + V'_{-g}, beta_g = i (V'_{+g} - V'_{-g}), expands them to the
 // four rows of each row quadruple (one lane per quadruple), expands every row to N3 reals with
 // the same folded basis, stages the rows in shared memory (TMA swizzle) and stores them with TMA.
-template <int N3, int K3>
-__device__ __forceinline__ void expand_row(char* stage, int box_rows, int row, const Stage1Table<N3, K3>& tab,
+template <int N3, int K3, int BOXR>
+__device__ __forceinline__ void expand_row(uint32_t stage, int row, const Stage1Table<N3, K3>& tab,
                                            const float (&z)[2 * K3]) {
   constexpr int CH = N3 / 4;
-  const uint32_t sw = (uint32_t)(row & 7);
-  char* rbase = stage + (size_t)row * 128;
+  constexpr int P = BOXR * 128;
+  // same single-XOR swizzled addressing as the forward kernel's row loads
+  const uint32_t rx = stage + (uint32_t)row * 128u + (((uint32_t)row & 7u) << 4);
 #pragma unroll
   for (int c = 0; c < CH / 4; ++c) {
     float a[4], b[4], cc[4], d[4];
@@ -469,14 +496,14 @@ __device__ __forceinline__ void expand_row(char* stage, int box_rows, int row, c
       cc[e] = da - db;   // y[N3/2+j]
     }
     const int c0 = c, c1 = CH / 2 - 1 - c, c2 = CH / 2 + c, c3 = CH - 1 - c;
-    *reinterpret_cast<float4*>(rbase + (size_t)(c0 / 8) * box_rows * 128 + (((uint32_t)(c0 % 8) ^ sw) << 4)) =
-        make_float4(a[0], a[1], a[2], a[3]);
-    *reinterpret_cast<float4*>(rbase + (size_t)(c1 / 8) * box_rows * 128 + (((uint32_t)(c1 % 8) ^ sw) << 4)) =
-        make_float4(b[3], b[2], b[1], b[0]);
-    *reinterpret_cast<float4*>(rbase + (size_t)(c2 / 8) * box_rows * 128 + (((uint32_t)(c2 % 8) ^ sw) << 4)) =
-        make_float4(cc[0], cc[1], cc[2], cc[3]);
-    *reinterpret_cast<float4*>(rbase + (size_t)(c3 / 8) * box_rows * 128 + (((uint32_t)(c3 % 8) ^ sw) << 4)) =
-        make_float4(d[3], d[2], d[1], d[0]);
+#define DTST_ST(cidx, v0, v1, v2, v3)                                                         \
+    if ((cidx) / 8 == 0) sts128_s<0>(rx ^ (uint32_t)(((cidx) % 8) << 4), v0, v1, v2, v3);     \
+    else sts128_s<P>(rx ^ (uint32_t)(((cidx) % 8) << 4), v0, v1, v2, v3);
+    DTST_ST(c0, a[0], a[1], a[2], a[3])
+    DTST_ST(c1, b[3], b[2], b[1], b[0])
+    DTST_ST(c2, cc[0], cc[1], cc[2], cc[3])
+    DTST_ST(c3, d[3], d[2], d[1], d[0])
+#undef DTST_ST
   }
 }
 
@@ -513,6 +540,7 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   char* staging = reinterpret_cast<char*>(smem) + (size_t)warp * IC::WARP_BYTES;
+  const uint32_t staging_s = smem_u32(staging);
   float* ab = reinterpret_cast<float*>(IC::ALIAS ? staging : staging + IC::STAGING_BYTES);
   float2* rot = reinterpret_cast<float2*>(smem + (size_t)W * IC::WARP_BYTES);
 
@@ -735,7 +763,7 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
 #pragma unroll
       for (int c = 0; c < NC; ++c) z[c] = fmaf(sQo, Qo[c], fmaf(sQe, Qe[c], fmaf(sPo, Po[c], Pe[c])));
       const int trow = pl1 * N2 + rowq;
-      expand_row<N3, K3>(staging + (size_t)(trow / RPS) * kStageBytes, RPS, trow % RPS, tab, z);
+      expand_row<N3, K3, RPS>(staging_s + (uint32_t)(trow / RPS) * kStageBytes, trow % RPS, tab, z);
     }
     fence_proxy_async_smem();
     __syncwarp();

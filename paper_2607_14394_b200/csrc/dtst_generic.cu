@@ -118,43 +118,46 @@ cudaError_t launch_reduce_partials(const float2* partial, float2* out, long long
 
 // ---------------------------------------------------------------------------
 // Per-mode channel mixing (Eq. 12): Y[b,o,m] = sum_i X[b,i,m] W[i,o,m].
-// One thread per (o, m); W is streamed once per chunk of up to BT batch entries.
+// W-streaming: about B flops per byte of W, so the roof is HBM.  One thread per (o, m); W is read once
+// per chunk of NB batch entries (NB is a compile-time 1..4: a run-time batch predicate inside the channel
+// loop cost a third of the bandwidth).  Full occupancy (about 32 registers) is what keeps enough loads in
+// flight; unrolling or 16-byte accesses measured slower.
 // ---------------------------------------------------------------------------
-template <int BT>
+template <int NB>
 __global__ void __launch_bounds__(256) mix_kernel(const float2* __restrict__ X, const float2* __restrict__ W,
-                                                 float2* __restrict__ Y, int b0, int nb, int Ci, int Co,
-                                                 long long M) {
+                                                 float2* __restrict__ Y, int b0, int Ci, int Co, long long M) {
   const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int o = blockIdx.y;
   if (m >= M) return;
-  float2 acc[BT];
+  float2 acc[NB];
 #pragma unroll
-  for (int b = 0; b < BT; ++b) acc[b] = make_float2(0.f, 0.f);
+  for (int b = 0; b < NB; ++b) acc[b] = make_float2(0.f, 0.f);
   for (int i = 0; i < Ci; ++i) {
-    const float2 w = W[((long long)i * Co + o) * M + m];
+    const float2 w = __ldg(W + ((long long)i * Co + o) * M + m);
 #pragma unroll
-    for (int b = 0; b < BT; ++b) {
-      if (b < nb) {
-        const float2 x = X[((long long)(b0 + b) * Ci + i) * M + m];
-        acc[b].x = fmaf(x.x, w.x, acc[b].x);
-        acc[b].x = fmaf(-x.y, w.y, acc[b].x);
-        acc[b].y = fmaf(x.x, w.y, acc[b].y);
-        acc[b].y = fmaf(x.y, w.x, acc[b].y);
-      }
+    for (int b = 0; b < NB; ++b) {
+      const float2 x = __ldg(X + ((long long)(b0 + b) * Ci + i) * M + m);
+      acc[b].x = fmaf(x.x, w.x, acc[b].x);
+      acc[b].x = fmaf(-x.y, w.y, acc[b].x);
+      acc[b].y = fmaf(x.x, w.y, acc[b].y);
+      acc[b].y = fmaf(x.y, w.x, acc[b].y);
     }
   }
 #pragma unroll
-  for (int b = 0; b < BT; ++b)
-    if (b < nb) Y[((long long)(b0 + b) * Co + o) * M + m] = acc[b];
+  for (int b = 0; b < NB; ++b) Y[((long long)(b0 + b) * Co + o) * M + m] = acc[b];
 }
 
 cudaError_t launch_mix(const float2* X, const float2* W, float2* Y, int B, int Ci, int Co, long long M,
                        cudaStream_t st, long long* launches) {
-  constexpr int BT = 4;
   dim3 grid((unsigned)((M + 255) / 256), (unsigned)Co);
-  for (int b0 = 0; b0 < B; b0 += BT) {
-    const int nb = (B - b0 < BT) ? (B - b0) : BT;
-    mix_kernel<BT><<<grid, 256, 0, st>>>(X, W, Y, b0, nb, Ci, Co, M);
+  for (int b0 = 0; b0 < B; b0 += 4) {
+    const int nb = (B - b0 < 4) ? (B - b0) : 4;
+    switch (nb) {
+      case 1: mix_kernel<1><<<grid, 256, 0, st>>>(X, W, Y, b0, Ci, Co, M); break;
+      case 2: mix_kernel<2><<<grid, 256, 0, st>>>(X, W, Y, b0, Ci, Co, M); break;
+      case 3: mix_kernel<3><<<grid, 256, 0, st>>>(X, W, Y, b0, Ci, Co, M); break;
+      default: mix_kernel<4><<<grid, 256, 0, st>>>(X, W, Y, b0, Ci, Co, M); break;
+    }
     if (launches) ++*launches;
   }
   return cudaGetLastError();
@@ -163,65 +166,93 @@ cudaError_t launch_mix(const float2* X, const float2* W, float2* Y, int B, int C
 // ---------------------------------------------------------------------------
 // Adjoint of the mixing (Section "Backward Pass"):
 //   GX[b,i,m] = sum_o GY[b,o,m] conj(W[i,o,m]);  GW[i,o,m] = sum_b conj(X[b,i,m]) GY[b,o,m]
-// One thread per (i, m) walks o, so W is read once and GW written once.
+// One thread per (i, m) walks o, so W is read once and GW written once.  NB = batch entries of this
+// launch (compile time); ALLB = the launch covers the whole batch, so GW needs no second pass over b.
 // ---------------------------------------------------------------------------
-template <int BT>
+template <int NB, bool ALLB, bool WANT_GX, bool WANT_GW>
 __global__ void __launch_bounds__(256) mix_adjoint_kernel(const float2* __restrict__ GY,
                                                          const float2* __restrict__ X,
                                                          const float2* __restrict__ W, float2* __restrict__ GX,
-                                                         float2* __restrict__ GW, int b0, int nb, int B, int Ci,
-                                                         int Co, long long M, int write_gw) {
+                                                         float2* __restrict__ GW, int b0, int B, int Ci, int Co,
+                                                         long long M) {
   const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int i = blockIdx.y;
   if (m >= M) return;
-  float2 gx[BT];
+  float2 gx[NB], xr[NB];
 #pragma unroll
-  for (int b = 0; b < BT; ++b) gx[b] = make_float2(0.f, 0.f);
+  for (int b = 0; b < NB; ++b) {
+    gx[b] = make_float2(0.f, 0.f);
+    xr[b] = (WANT_GW && ALLB) ? __ldg(X + ((long long)(b0 + b) * Ci + i) * M + m) : make_float2(0.f, 0.f);
+  }
   for (int o = 0; o < Co; ++o) {
-    const float2 w = W[((long long)i * Co + o) * M + m];
-    if (GX != nullptr) {
+    const float2 w = __ldg(W + ((long long)i * Co + o) * M + m);
+    float2 g[NB];
 #pragma unroll
-      for (int b = 0; b < BT; ++b) {
-        if (b < nb) {
-          const float2 g = GY[((long long)(b0 + b) * Co + o) * M + m];
-          // g * conj(w)
-          gx[b].x = fmaf(g.x, w.x, gx[b].x);
-          gx[b].x = fmaf(g.y, w.y, gx[b].x);
-          gx[b].y = fmaf(g.y, w.x, gx[b].y);
-          gx[b].y = fmaf(-g.x, w.y, gx[b].y);
-        }
+    for (int b = 0; b < NB; ++b) g[b] = __ldg(GY + ((long long)(b0 + b) * Co + o) * M + m);
+    if (WANT_GX) {
+#pragma unroll
+      for (int b = 0; b < NB; ++b) {   // g * conj(w)
+        gx[b].x = fmaf(g[b].x, w.x, gx[b].x);
+        gx[b].x = fmaf(g[b].y, w.y, gx[b].x);
+        gx[b].y = fmaf(g[b].y, w.x, gx[b].y);
+        gx[b].y = fmaf(-g[b].x, w.y, gx[b].y);
       }
     }
-    if (write_gw) {
+    if (WANT_GW) {
       float2 acc = make_float2(0.f, 0.f);
-      for (int b = 0; b < B; ++b) {
-        const float2 g = GY[((long long)b * Co + o) * M + m];
-        const float2 x = X[((long long)b * Ci + i) * M + m];
-        // conj(x) * g
-        acc.x = fmaf(x.x, g.x, acc.x);
-        acc.x = fmaf(x.y, g.y, acc.x);
-        acc.y = fmaf(x.x, g.y, acc.y);
-        acc.y = fmaf(-x.y, g.x, acc.y);
+      if (ALLB) {
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {   // conj(x) * g
+          acc.x = fmaf(xr[b].x, g[b].x, acc.x);
+          acc.x = fmaf(xr[b].y, g[b].y, acc.x);
+          acc.y = fmaf(xr[b].x, g[b].y, acc.y);
+          acc.y = fmaf(-xr[b].y, g[b].x, acc.y);
+        }
+      } else {
+        for (int b = 0; b < B; ++b) {
+          const float2 gg = __ldg(GY + ((long long)b * Co + o) * M + m);
+          const float2 xx = __ldg(X + ((long long)b * Ci + i) * M + m);
+          acc.x = fmaf(xx.x, gg.x, acc.x);
+          acc.x = fmaf(xx.y, gg.y, acc.x);
+          acc.y = fmaf(xx.x, gg.y, acc.y);
+          acc.y = fmaf(-xx.y, gg.x, acc.y);
+        }
       }
       GW[((long long)i * Co + o) * M + m] = acc;
     }
   }
-  if (GX != nullptr) {
+  if (WANT_GX) {
 #pragma unroll
-    for (int b = 0; b < BT; ++b)
-      if (b < nb) GX[((long long)(b0 + b) * Ci + i) * M + m] = gx[b];
+    for (int b = 0; b < NB; ++b) GX[((long long)(b0 + b) * Ci + i) * M + m] = gx[b];
   }
+}
+
+template <int NB>
+void launch_mix_adjoint_nb(dim3 grid, cudaStream_t st, const float2* GY, const float2* X, const float2* W,
+                           float2* GX, float2* GW, int b0, int B, int Ci, int Co, long long M, bool want_gw) {
+  const bool allb = (b0 == 0 && NB == B);
+  const bool gx = GX != nullptr;
+#define DTST_MA(AL, WX, WW) \
+  mix_adjoint_kernel<NB, AL, WX, WW><<<grid, 256, 0, st>>>(GY, X, W, GX, GW, b0, B, Ci, Co, M)
+  if (gx && want_gw) { if (allb) DTST_MA(true, true, true); else DTST_MA(false, true, true); }
+  else if (gx) DTST_MA(false, true, false);
+  else if (want_gw) { if (allb) DTST_MA(true, false, true); else DTST_MA(false, false, true); }
+#undef DTST_MA
 }
 
 cudaError_t launch_mix_adjoint(const float2* GY, const float2* X, const float2* W, float2* GX, float2* GW,
                                int B, int Ci, int Co, long long M, cudaStream_t st, long long* launches) {
-  constexpr int BT = 4;
   dim3 grid((unsigned)((M + 255) / 256), (unsigned)Ci);
-  for (int b0 = 0; b0 < B; b0 += BT) {
-    const int nb = (B - b0 < BT) ? (B - b0) : BT;
-    const int write_gw = (GW != nullptr && b0 == 0) ? 1 : 0;
-    if (GX == nullptr && !write_gw) break;
-    mix_adjoint_kernel<BT><<<grid, 256, 0, st>>>(GY, X, W, GX, GW, b0, nb, B, Ci, Co, M, write_gw);
+  for (int b0 = 0; b0 < B; b0 += 4) {
+    const int nb = (B - b0 < 4) ? (B - b0) : 4;
+    const bool want_gw = (GW != nullptr && b0 == 0);
+    if (GX == nullptr && !want_gw) break;
+    switch (nb) {
+      case 1: launch_mix_adjoint_nb<1>(grid, st, GY, X, W, GX, GW, b0, B, Ci, Co, M, want_gw); break;
+      case 2: launch_mix_adjoint_nb<2>(grid, st, GY, X, W, GX, GW, b0, B, Ci, Co, M, want_gw); break;
+      case 3: launch_mix_adjoint_nb<3>(grid, st, GY, X, W, GX, GW, b0, B, Ci, Co, M, want_gw); break;
+      default: launch_mix_adjoint_nb<4>(grid, st, GY, X, W, GX, GW, b0, B, Ci, Co, M, want_gw); break;
+    }
     if (launches) ++*launches;
     if (GX == nullptr) break;
   }
