@@ -59,7 +59,9 @@ enum {
 /* Kernel families selectable with dtst_plan_set_kernel_path. */
 enum {
   DTST_PATH_AUTO = 0,      /* fused streaming kernels where the shape allows, else generic */
-  DTST_PATH_GENERIC = 1    /* one generic contraction kernel per dimension                 */
+  DTST_PATH_GENERIC = 1,   /* one generic contraction kernel per dimension                 */
+  DTST_PATH_ROW = 2        /* reported only: streaming kernel on the contiguous dimension,
+                              folded kernels on the others (shapes without a two-dimension kernel) */
 };
 
 /*
@@ -100,8 +102,9 @@ dtst_status dtst_plan_set_virtual_shards(dtst_plan* plan, int P);
 /* Choose the kernel family (DTST_PATH_*).  Changes workspace_bytes. */
 dtst_status dtst_plan_set_kernel_path(dtst_plan* plan, int path);
 
-/* Reports which family the plan's calls will actually run (DTST_PATH_AUTO is
- * returned only when a fused kernel serves this shape; else DTST_PATH_GENERIC). */
+/* Reports which family the plan's calls will actually run: DTST_PATH_AUTO when the fused
+ * two-dimension streaming kernels serve this shape, DTST_PATH_ROW when the one-dimension streaming
+ * kernels do, else DTST_PATH_GENERIC. */
 dtst_status dtst_plan_kernel_path(const dtst_plan* plan, int* path);
 
 dtst_status dtst_plan_destroy(dtst_plan* plan);

@@ -296,7 +296,7 @@ class Plan:
 
     @property
     def kernel_path(self) -> str:
-        return "fused" if dtst_plan_kernel_path(self._h) == DTST_PATH_AUTO else "generic"
+        return {DTST_PATH_AUTO: "fused", 2: "row"}.get(dtst_plan_kernel_path(self._h), "generic")
 
     def mode_indices(self, dim: int):
         return dtst_plan_mode_indices(self._h, dim, self.K[dim])

@@ -103,6 +103,19 @@ bool use_mid(const dtst_plan* p, int j) {
 
 bool use_fused(const dtst_plan* p) { return p->path_request == DTST_PATH_AUTO && fused_eligible(p); }
 
+// Row kernels: the contiguous dimension alone (whole on this device, zero offset), for shapes without a
+// plane kernel; the other dimensions then run on the reduced tensor.
+bool use_row(const dtst_plan* p) {
+  if (p->path_request != DTST_PATH_AUTO || use_fused(p)) return false;
+  const int a = p->d - 1;
+  if (p->Nl[a] != p->Ng[a] || p->off[a] != 0) return false;
+  if (p->d == 1 && p->P > 1) return false;
+  long long rows = (long long)p->B * (p->C_in > p->C_out ? p->C_in : p->C_out);
+  for (int i = 0; i < a; ++i) rows *= p->Nl[i];
+  if (rows >= (1ll << 31)) return false;   // 32-bit TMA coordinates
+  return row_supported((int)p->Ng[a], p->kmax[a]);
+}
+
 DimOp make_op(const dtst_plan* p, int j, bool forward, int Cn) {
   DimOp op;
   std::memset(&op, 0, sizeof(op));
@@ -300,6 +313,43 @@ dtst_status run_inverse_fused(dtst_plan* p, const float2* Yhat, float* y, int Cn
   return DTST_OK;
 }
 
+// Row path: the row kernel streams the grid once along its contiguous dimension; the rest runs reduced.
+dtst_status run_forward_row(dtst_plan* p, const float* x, float2* Xhat, int Cn, float scale, bool herm,
+                            cudaStream_t st) {
+  const int d = p->d, a = d - 1;
+  const WsLayout L = ws_layout(p);
+  char* ws = static_cast<char*>(p->ws);
+  long long rows = (long long)p->B * Cn;
+  for (int i = 0; i < a; ++i) rows *= p->Nl[i];
+  float2* t1 = (d == 1) ? Xhat : reinterpret_cast<float2*>(ws + L.bufA);
+  {
+    KernelTimer kt(p, DTST_KERNEL_GRID_READ, st);
+    if (cuda_failed(p, launch_row_contract(x, t1, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0,
+                                           reinterpret_cast<int*>(ws + L.status), st)))
+      return DTST_ERR_CUDA;
+  }
+  ++p->launches;
+  if (d == 1) return DTST_OK;
+  return forward_stages(p, t1, d - 2, 1, Xhat, Cn, 1.0f, false, st);
+}
+
+dtst_status run_inverse_row(dtst_plan* p, const float2* Yhat, float* y, int Cn, float scale, bool herm,
+                            cudaStream_t st) {
+  const int d = p->d, a = d - 1;
+  const float2* src = Yhat;
+  if (d > 1) {
+    dtst_status s = inverse_stages_complex(p, Yhat, d - 2, Cn, &src, st);
+    if (s != DTST_OK) return s;
+  }
+  long long rows = (long long)p->B * Cn;
+  for (int i = 0; i < a; ++i) rows *= p->Nl[i];
+  KernelTimer kt(p, DTST_KERNEL_GRID_WRITE, st);
+  if (cuda_failed(p, launch_row_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, st)))
+    return DTST_ERR_CUDA;
+  ++p->launches;
+  return DTST_OK;
+}
+
 dtst_status check_ready(const dtst_plan* p) {
   if (p == nullptr) return DTST_ERR_INVALID_ARG;
   const WsLayout L = ws_layout(p);
@@ -380,7 +430,7 @@ dtst_status dtst_plan_set_kernel_path(dtst_plan* p, int path) {
 
 dtst_status dtst_plan_kernel_path(const dtst_plan* p, int* path) {
   if (p == nullptr || path == nullptr) return DTST_ERR_INVALID_ARG;
-  *path = use_fused(p) ? DTST_PATH_AUTO : DTST_PATH_GENERIC;
+  *path = use_fused(p) ? DTST_PATH_AUTO : (use_row(p) ? DTST_PATH_ROW : DTST_PATH_GENERIC);
   return DTST_OK;
 }
 
@@ -486,6 +536,7 @@ dtst_status dtst_forward(dtst_plan* p, const float* x, void* Xhat, void* stream)
   if (x == nullptr || Xhat == nullptr || !aligned16(x) || !aligned16(Xhat)) return DTST_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (use_fused(p)) return run_forward_fused(p, x, static_cast<float2*>(Xhat), p->C_in, 1.0f, false, st);
+  if (use_row(p)) return run_forward_row(p, x, static_cast<float2*>(Xhat), p->C_in, 1.0f, false, st);
   return run_forward_generic(p, x, static_cast<float2*>(Xhat), p->C_in, 1.0f, false, st);
 }
 
@@ -508,6 +559,7 @@ dtst_status dtst_inverse(dtst_plan* p, const void* Yhat, float* y, void* stream)
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const float scale = (float)(1.0 / (double)p->points_global);
   if (use_fused(p)) return run_inverse_fused(p, static_cast<const float2*>(Yhat), y, p->C_out, scale, true, st);
+  if (use_row(p)) return run_inverse_row(p, static_cast<const float2*>(Yhat), y, p->C_out, scale, true, st);
   return run_inverse_generic(p, static_cast<const float2*>(Yhat), y, p->C_out, scale, true, st);
 }
 
@@ -527,6 +579,7 @@ dtst_status dtst_backward(dtst_plan* p, const float* grad_y, const void* Xhat_sa
   const float scale = (float)(1.0 / (double)p->points_global);
   // adjoint of I: G_Y = (c / prod N) F(grad_y)
   s = use_fused(p) ? run_forward_fused(p, grad_y, GY, p->C_out, scale, true, st)
+      : use_row(p) ? run_forward_row(p, grad_y, GY, p->C_out, scale, true, st)
                    : run_forward_generic(p, grad_y, GY, p->C_out, scale, true, st);
   if (s != DTST_OK) return s;
   // adjoint of M
@@ -539,6 +592,7 @@ dtst_status dtst_backward(dtst_plan* p, const float* grad_y, const void* Xhat_sa
   // adjoint of F: plain expansion, no doubling, no 1/prod N
   if (grad_x != nullptr) {
     s = use_fused(p) ? run_inverse_fused(p, GX, grad_x, p->C_in, 1.0f, false, st)
+        : use_row(p) ? run_inverse_row(p, GX, grad_x, p->C_in, 1.0f, false, st)
                      : run_inverse_generic(p, GX, grad_x, p->C_in, 1.0f, false, st);
     if (s != DTST_OK) return s;
   }

@@ -26,6 +26,8 @@ namespace dtst {
 
 using namespace sm100;
 
+bool make_rows_map(CUtensorMap* map, const void* base, long long rows, int n3, int box_rows);
+
 namespace {
 
 constexpr int kTaskRows = 128;       // rows of the contiguous dimension per warp task
@@ -800,19 +802,6 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// 2-D fp32 tensor [rows][n3] viewed through [box_rows x 32] boxes with the 128-byte swizzle.
-bool make_rows_map(CUtensorMap* map, const void* base, long long rows, int n3, int box_rows) {
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (fn == nullptr) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)n3, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)n3 * 4};
-  cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int N3, int K3>
 void fill_stage1_table(Stage1Table<N3, K3>* t) {
   for (int j = 0; j < N3 / 4; ++j)
@@ -867,6 +856,20 @@ cudaError_t launch_inv_plane_t(const float2* in, float* y, long long rows, float
 }
 
 }  // namespace
+
+// 2-D fp32 tensor [rows][n3] viewed through [box_rows x 32] boxes with the 128-byte swizzle.
+bool make_rows_map(CUtensorMap* map, const void* base, long long rows, int n3, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)n3, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)n3 * 4};
+  cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 
 // Shapes the plane kernels are instantiated for: (N3, k3, N2, k2).
 static bool plane_supported(int N3, int K3, int N2, int K2) {

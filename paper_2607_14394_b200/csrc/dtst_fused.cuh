@@ -1,5 +1,7 @@
 // Fused streaming kernels for the grid-side stages (launchers).
 #pragma once
+#include <cuda.h>
+
 #include "dtst_common.cuh"
 
 namespace dtst {
@@ -13,5 +15,15 @@ cudaError_t launch_fwd_plane(int N3, int K3, int N2, int K2, const float* x, flo
 // Inverse plane kernel: in[planes][2*K2][K3] complex -> real rows [rows][N3].
 cudaError_t launch_inv_plane(int N3, int K3, int N2, int K2, const float2* in, float* y, long long rows,
                              float scale, int herm, int* status, cudaStream_t st);
+
+// 2-D fp32 tensor [rows][n3] viewed through [box_rows x 32 floats] boxes with the 128-byte TMA swizzle.
+bool make_rows_map(CUtensorMap* map, const void* base, long long rows, int n3, int box_rows);
+
+// Row kernels (dtst_row.cu): the contiguous dimension alone, N3 % 32 == 0, N3 <= 256, k3 <= 16.
+bool row_supported(int N3, int K3);
+cudaError_t launch_row_contract(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm,
+                                int* status, cudaStream_t st);
+cudaError_t launch_row_expand(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm,
+                              cudaStream_t st);
 
 }  // namespace dtst

@@ -47,7 +47,7 @@ def _check_layer_fullsize(w, P_list, check_channels, rng_seed):
     x = I.make_field_torch(w, dev, tag=0)
     W = I.make_weights_torch(w, dev)
     plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out)
-    assert plan.kernel_path in ("fused", "generic")
+    assert plan.kernel_path in ("fused", "row", "generic")
     lists = _lists(w)
     for j in range(w.d):
         assert plan.mode_indices(j) == lists[j].tolist()

@@ -86,6 +86,13 @@ EDGE = [
     ("big_batch", 6, 2, 3, (8, 16), (2, 4)),          # B > the mixing kernels' batch tile
     ("tail_rows", 1, 5, 7, (12, 20, 36), (3, 5, 7)),  # nothing a multiple of a tile
     ("wide_last", 1, 2, 2, (8, 8, 520), (2, 3, 9)),
+    # shapes served by the one-dimension streaming kernels: N3 a multiple of 32, ragged row counts
+    ("row_32_k16", 1, 3, 2, (5, 32), (2, 16)),
+    ("row_96_odd_k", 2, 1, 3, (3, 7, 96), (1, 3, 5)),
+    ("row_160", 1, 2, 1, (6, 160), (3, 9)),
+    ("row_256", 1, 1, 2, (4, 6, 256), (2, 3, 16)),
+    ("row_d1", 3, 2, 2, (128,), (7,)),
+    ("row_k1", 1, 2, 2, (9, 64), (4, 1)),
 ]
 
 
