@@ -24,26 +24,36 @@ namespace {
 
 constexpr int kRowSmemLimit = 232448;
 
+// fp32 -> (hi, lo) for the error-compensated TF32 product.  The tensor core reads only the upper 19 bits
+// of an operand, so hi is the value with its low 13 mantissa bits cleared and lo = v - hi is exact in fp32;
+// lo is passed as is (the hardware drops its low bits, an error of 2^-20 |v| at most).  One AND and one
+// subtraction: the rounding conversion (cvt.rna) costs several times more issue slots, which is what
+// bounded these kernels.
 __device__ __forceinline__ void split_tf32_r(float v, uint32_t& hi, uint32_t& lo) {
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(v));
-  const float r = v - __uint_as_float(hi);
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(r));
+  hi = __float_as_uint(v) & 0xffffe000u;
+  lo = __float_as_uint(v - __uint_as_float(hi));
 }
 
+// (not volatile: a pure register-to-register operation the compiler may schedule freely among the loads)
 __device__ __forceinline__ void mma_tf32_r(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ float lds32_s(uint32_t addr) {
-  float v;
-  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-  return v;
+// Plain C++ accesses through a pointer into the shared array (`base` + 32-bit offset): the compiler keeps them
+// on the right side of the barrier waits and arrivals (those are asm statements with a memory clobber) but is
+// free to hoist the next k-step's loads above this k-step's MMAs.
+struct SmemTile {
+  unsigned char* base;   // generic pointer derived from the __shared__ array
+  uint32_t s;            // its 32-bit shared-space address
+};
+__device__ __forceinline__ float lds32_s(const SmemTile& t, uint32_t addr) {
+  return *reinterpret_cast<const float*>(t.base + (addr - t.s));
 }
-__device__ __forceinline__ void sts64_s(uint32_t addr, float a, float b) {
-  asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
+__device__ __forceinline__ void sts64_s(const SmemTile& t, uint32_t addr, float a, float b) {
+  *reinterpret_cast<float2*>(t.base + (addr - t.s)) = make_float2(a, b);
 }
 
 // byte offset of element (row, col) of a [BOXR rows x N3] tile stored as N3/32 panels of [BOXR x 128 B],
@@ -97,6 +107,7 @@ row_contract_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restri
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t ring_s = smem_u32(smem);
+  const SmemTile tl_{smem, ring_s};
   // basis fragments: [cls][ks][lane] float4 = (b0 hi, b1 hi, b0 lo, b1 lo)
   float4* btab = reinterpret_cast<float4*>(smem + (size_t)stages * slot_bytes);
   uint64_t* full = reinterpret_cast<uint64_t*>(btab + (size_t)4 * NKS * 32);
@@ -166,48 +177,86 @@ row_contract_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restri
       const int slot = (int)(tl % stages);
       if (!row_wait_fill(rw, slot, (uint32_t)(tl / stages))) break;
       const uint32_t st = ring_s + (uint32_t)slot * slot_bytes;
+      // two accumulator sets (even / odd k-steps) halve the dependent-MMA chains; summed at the end
+      float acc2[2][MT][4][4];
+#pragma unroll
+      for (int z = 0; z < 2; ++z)
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc2[z][mt][c][e] = 0.f;
+
+      // Gather addressing.  Element (row, j) of the swizzled tile: panel (j >> 5), 16-byte chunk ((j & 31) >> 2)
+      // XOR (row & 7), word j & 3.  With j = 8 ks + t4 + 4 h the chunk is 2 (ks & 3) + h and the word is t4; the
+      // mirrored column N3-1-j has chunk 7 - that and word 3 - t4, i.e. the same XOR term flipped by 0x70.  When
+      // N3 is a multiple of 64 the half-row offsets N3/2 are whole panels, so everything but one XOR and the
+      // panel offsets is a per-lane constant.
+      const bool fastaddr = (N3 % 64) == 0;
+      const uint32_t gx = (uint32_t)g8 << 4;
+      const uint32_t P = (uint32_t)BOXR * 128u;
+      const int NP = N3 / 32;
+#pragma unroll 1
+      for (int ks0 = 0; ks0 < NKS; ks0 += 4) {
+        const uint32_t pa = (uint32_t)(ks0 >> 2);
+        const uint32_t panA = st + pa * P, panD = st + ((uint32_t)NP - 1u - pa) * P;
+        const uint32_t panC = st + ((uint32_t)(NP / 2) + pa) * P, panB = st + ((uint32_t)(NP / 2) - 1u - pa) * P;
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4) {
+          const int ks = ks0 + k4;
+          if (ks >= NKS) break;
+          float4 bf[4];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) bf[c] = btab[(c * NKS + ks) * 32 + lane];
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            uint32_t ah[4][4], al[4][4];   // [class][fragment element]
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int row = 16 * mt + g8 + 8 * (e & 1);
+              float a, b, c, d;
+              if (fastaddr) {
+                const uint32_t xa = ((uint32_t)((2 * k4 + (e >> 1)) << 4)) ^ gx;
+                const uint32_t wa = (uint32_t)row * 128u + ((uint32_t)t4 << 2);
+                const uint32_t wd = (uint32_t)row * 128u + ((uint32_t)(3 - t4) << 2);
+                a = lds32_s(tl_, panA + wa + xa);
+                d = lds32_s(tl_, panD + wd + (xa ^ 0x70u));
+                c = lds32_s(tl_, panC + wa + xa);
+                b = lds32_s(tl_, panB + wd + (xa ^ 0x70u));
+              } else {
+                const int j = 8 * ks + t4 + 4 * (e >> 1);
+                a = lds32_s(tl_, st + tile_off(row, j, BOXR));
+                b = lds32_s(tl_, st + tile_off(row, N3 / 2 - 1 - j, BOXR));
+                c = lds32_s(tl_, st + tile_off(row, N3 / 2 + j, BOXR));
+                d = lds32_s(tl_, st + tile_off(row, N3 - 1 - j, BOXR));
+              }
+              const float u = a + d, v = a - d, up = b + c, vp = b - c;
+              split_tf32_r(u + up, ah[0][e], al[0][e]);   // uu: even-f cos
+              split_tf32_r(u - up, ah[1][e], al[1][e]);   // ud: odd-f cos
+              split_tf32_r(v + vp, ah[2][e], al[2][e]);   // vs: odd-f sin
+              split_tf32_r(v - vp, ah[3][e], al[3][e]);   // vd: even-f sin
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const uint32_t bh0 = __float_as_uint(bf[c].x), bh1 = __float_as_uint(bf[c].y);
+              const uint32_t bl0 = __float_as_uint(bf[c].z), bl1 = __float_as_uint(bf[c].w);
+              mma_tf32_r(acc2[k4 & 1][mt][c], ah[c], bh0, bh1);
+              mma_tf32_r(acc2[k4 & 1][mt][c], al[c], bh0, bh1);
+              mma_tf32_r(acc2[k4 & 1][mt][c], ah[c], bl0, bl1);
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[slot]);
       float acc[MT][4][4];
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
         for (int c = 0; c < 4; ++c)
 #pragma unroll
-          for (int e = 0; e < 4; ++e) acc[mt][c][e] = 0.f;
-
-#pragma unroll 1
-      for (int ks = 0; ks < NKS; ++ks) {
-        float4 bf[4];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) bf[c] = btab[(c * NKS + ks) * 32 + lane];
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
-          uint32_t ah[4][4], al[4][4];   // [class][fragment element]
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int row = 16 * mt + g8 + 8 * (e & 1);
-            const int j = 8 * ks + t4 + 4 * (e >> 1);
-            const float a = lds32_s(st + tile_off(row, j, BOXR));
-            const float b = lds32_s(st + tile_off(row, N3 / 2 - 1 - j, BOXR));
-            const float c = lds32_s(st + tile_off(row, N3 / 2 + j, BOXR));
-            const float d = lds32_s(st + tile_off(row, N3 - 1 - j, BOXR));
-            const float u = a + d, v = a - d, up = b + c, vp = b - c;
-            split_tf32_r(u + up, ah[0][e], al[0][e]);   // uu: even-f cos
-            split_tf32_r(u - up, ah[1][e], al[1][e]);   // ud: odd-f cos
-            split_tf32_r(v + vp, ah[2][e], al[2][e]);   // vs: odd-f sin
-            split_tf32_r(v - vp, ah[3][e], al[3][e]);   // vd: even-f sin
-          }
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const uint32_t bh0 = __float_as_uint(bf[c].x), bh1 = __float_as_uint(bf[c].y);
-            const uint32_t bl0 = __float_as_uint(bf[c].z), bl1 = __float_as_uint(bf[c].w);
-            mma_tf32_r(acc[mt][c], ah[c], bh0, bh1);
-            mma_tf32_r(acc[mt][c], al[c], bh0, bh1);
-            mma_tf32_r(acc[mt][c], ah[c], bl0, bl1);
-          }
-        }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty[slot]);
+          for (int e = 0; e < 4; ++e) acc[mt][c][e] = acc2[0][mt][c][e] + acc2[1][mt][c][e];
 
       // X_f = rot_f (C_f - i S_f); this lane holds f = 4 t4 .. 4 t4 + 3 of rows g8 and g8 + 8 of every m-tile
 #pragma unroll
@@ -259,6 +308,7 @@ row_expand_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __r
   const int g8 = lane >> 2, t4 = lane & 3;
   unsigned char* staging = smem + (size_t)warp * tile_bytes;
   const uint32_t staging_s = smem_u32(staging);
+  const SmemTile tl_{staging, staging_s};
   // basis fragments as MMA B operands: k = frequency slot, n = quadruple; [cls][nt][lane] float4
   float4* btab = reinterpret_cast<float4*>(smem + (size_t)W * tile_bytes);
 
@@ -291,6 +341,23 @@ row_expand_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __r
 
   const long long num_tasks = (rows + BOXR - 1) / BOXR;
   const long long tstride = (long long)gridDim.x * W;
+  // raw input values of a task, fetched one task ahead: element (mt, e) needs frequencies 2 gi, 2 gi + 1
+  float2 vin[MT][4][2];
+  auto load_inputs = [&](long long t) {
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const long long row = t * BOXR + 16 * mt + g8 + 8 * (e & 1);
+        const int gi = t4 + 4 * (e >> 1);
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+          const int f = 2 * gi + p;
+          vin[mt][e][p] = (t < num_tasks && row < rows && f < K3) ? __ldg(in + row * K3 + f) : make_float2(0.f, 0.f);
+        }
+      }
+  };
+  load_inputs((long long)blockIdx.x + (long long)warp * gridDim.x);
   for (long long task = (long long)blockIdx.x + (long long)warp * gridDim.x; task < num_tasks; task += tstride) {
     // A fragments: z'[row][slot] = scale c_f e^{-i pi f / N3} in[row][f]; classes take Re of even f, Re of
     // odd f, Im of odd f, Im of even f.  Element (row, slot): e&1 selects row + 8, e>>1 selects slot + 4.
@@ -299,66 +366,87 @@ row_expand_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __r
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const long long row = task * BOXR + 16 * mt + g8 + 8 * (e & 1);
-        const int gi = t4 + 4 * (e >> 1);
-        float re[2] = {0.f, 0.f}, im[2] = {0.f, 0.f};
+        float re[2], im[2];
 #pragma unroll
         for (int p = 0; p < 2; ++p) {
-          const int f = 2 * gi + p;
-          if (row < rows && f < K3) {
-            const float2 v = __ldg(in + row * K3 + f);
-            const float rx = rotv[e >> 1][p].x, ry = rotv[e >> 1][p].y;
-            re[p] = v.x * rx - v.y * ry;
-            im[p] = v.x * ry + v.y * rx;
-          }
+          const float2 v = vin[mt][e][p];
+          const float rx = rotv[e >> 1][p].x, ry = rotv[e >> 1][p].y;
+          re[p] = v.x * rx - v.y * ry;
+          im[p] = v.x * ry + v.y * rx;
         }
         split_tf32_r(re[0], ah[mt][0][e], al[mt][0][e]);
         split_tf32_r(re[1], ah[mt][1][e], al[mt][1][e]);
         split_tf32_r(im[1], ah[mt][2][e], al[mt][2][e]);
         split_tf32_r(im[0], ah[mt][3][e], al[mt][3][e]);
       }
+    load_inputs(task + tstride);   // the next task's values travel while this one is expanded
     // the previous task's TMA store must have finished reading the staging tile
     if (lane == 0) tma_store_wait_read<0>();
     __syncwarp();
+    // Staging addressing, as in the contraction kernel: quadruple pair j0 = 8 nt + 2 t4 sits in panel nt >> 2,
+    // chunk 2 (nt & 3) + (t4 >> 1), 8-byte slot (t4 & 1); its mirror images flip the chunk (XOR 0x70) and the slot.
+    const bool fastaddr = (N3 % 64) == 0;
+    const uint32_t gx = (uint32_t)g8 << 4;
+    const uint32_t P = (uint32_t)BOXR * 128u;
+    const int NP = N3 / 32;
 #pragma unroll 1
-    for (int nt = 0; nt < NNT; ++nt) {
-      float4 bf[4];
+    for (int nt0 = 0; nt0 < NNT; nt0 += 4) {
+      const uint32_t pa = (uint32_t)(nt0 >> 2);
+      const uint32_t panA = staging_s + pa * P, panD = staging_s + ((uint32_t)NP - 1u - pa) * P;
+      const uint32_t panC = staging_s + ((uint32_t)(NP / 2) + pa) * P;
+      const uint32_t panB = staging_s + ((uint32_t)(NP / 2) - 1u - pa) * P;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) bf[c] = btab[(c * NNT + nt) * 32 + lane];
+      for (int k4 = 0; k4 < 4; ++k4) {
+        const int nt = nt0 + k4;
+        if (nt >= NNT) break;
+        float4 bf[4];
 #pragma unroll
-      for (int mt = 0; mt < MT; ++mt) {
-        float acc[4][4];
+        for (int c = 0; c < 4; ++c) bf[c] = btab[(c * NNT + nt) * 32 + lane];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int mt = 0; mt < MT; ++mt) {
+          float acc[4][4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) acc[c][e] = 0.f;
-          const uint32_t bh0 = __float_as_uint(bf[c].x), bh1 = __float_as_uint(bf[c].y);
-          const uint32_t bl0 = __float_as_uint(bf[c].z), bl1 = __float_as_uint(bf[c].w);
-          mma_tf32_r(acc[c], ah[mt][c], bh0, bh1);
-          mma_tf32_r(acc[c], al[mt][c], bh0, bh1);
-          mma_tf32_r(acc[c], ah[mt][c], bl0, bl1);
-        }
-        // C fragment elements 2h, 2h+1: row = 16 mt + g8 + 8 h, quadruples j0 = 8 nt + 2 t4 and j0 + 1:
-        // their four outputs are pairwise adjacent in the row, so each pair is one 8-byte store
+          for (int c = 0; c < 4; ++c) {
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int row = 16 * mt + g8 + 8 * h;
-          const int j0 = 8 * nt + 2 * t4;
-          float ya[2], yd[2], yb[2], yc[2];
-#pragma unroll
-          for (int q = 0; q < 2; ++q) {
-            const int e = 2 * h + q;
-            const float Ea = acc[0][e], Oa = acc[1][e], Ob = acc[2][e], Eb = acc[3][e];
-            const float sa = Ea + Oa, da = Ea - Oa, sb = Eb + Ob, db = Eb - Ob;
-            ya[q] = sa - sb;   // y[j]
-            yd[q] = sa + sb;   // y[N3-1-j]
-            yb[q] = da + db;   // y[N3/2-1-j]
-            yc[q] = da - db;   // y[N3/2+j]
+            for (int e = 0; e < 4; ++e) acc[c][e] = 0.f;
+            const uint32_t bh0 = __float_as_uint(bf[c].x), bh1 = __float_as_uint(bf[c].y);
+            const uint32_t bl0 = __float_as_uint(bf[c].z), bl1 = __float_as_uint(bf[c].w);
+            mma_tf32_r(acc[c], ah[mt][c], bh0, bh1);
+            mma_tf32_r(acc[c], al[mt][c], bh0, bh1);
+            mma_tf32_r(acc[c], ah[mt][c], bl0, bl1);
           }
-          sts64_s(staging_s + tile_off(row, j0, BOXR), ya[0], ya[1]);
-          sts64_s(staging_s + tile_off(row, N3 - 2 - j0, BOXR), yd[1], yd[0]);
-          sts64_s(staging_s + tile_off(row, N3 / 2 - 2 - j0, BOXR), yb[1], yb[0]);
-          sts64_s(staging_s + tile_off(row, N3 / 2 + j0, BOXR), yc[0], yc[1]);
+          // C fragment elements 2h, 2h+1: row = 16 mt + g8 + 8 h, quadruples j0 = 8 nt + 2 t4 and j0 + 1:
+          // their four outputs are pairwise adjacent in the row, so each pair is one 8-byte store
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int row = 16 * mt + g8 + 8 * h;
+            float ya[2], yd[2], yb[2], yc[2];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              const int e = 2 * h + q;
+              const float Ea = acc[0][e], Oa = acc[1][e], Ob = acc[2][e], Eb = acc[3][e];
+              const float sa = Ea + Oa, da = Ea - Oa, sb = Eb + Ob, db = Eb - Ob;
+              ya[q] = sa - sb;   // y[j]
+              yd[q] = sa + sb;   // y[N3-1-j]
+              yb[q] = da + db;   // y[N3/2-1-j]
+              yc[q] = da - db;   // y[N3/2+j]
+            }
+            if (fastaddr) {
+              const uint32_t xa = ((uint32_t)((2 * k4 + (t4 >> 1)) << 4)) ^ gx;
+              const uint32_t wa = (uint32_t)row * 128u + ((uint32_t)(t4 & 1) << 3);
+              const uint32_t wd = (uint32_t)row * 128u + ((uint32_t)(1 - (t4 & 1)) << 3);
+              sts64_s(tl_, panA + wa + xa, ya[0], ya[1]);
+              sts64_s(tl_, panD + wd + (xa ^ 0x70u), yd[1], yd[0]);
+              sts64_s(tl_, panB + wd + (xa ^ 0x70u), yb[1], yb[0]);
+              sts64_s(tl_, panC + wa + xa, yc[0], yc[1]);
+            } else {
+              const int j0 = 8 * nt + 2 * t4;
+              sts64_s(tl_, staging_s + tile_off(row, j0, BOXR), ya[0], ya[1]);
+              sts64_s(tl_, staging_s + tile_off(row, N3 - 2 - j0, BOXR), yd[1], yd[0]);
+              sts64_s(tl_, staging_s + tile_off(row, N3 / 2 - 2 - j0, BOXR), yb[1], yb[0]);
+              sts64_s(tl_, staging_s + tile_off(row, N3 / 2 + j0, BOXR), yc[0], yc[1]);
+            }
+          }
         }
       }
     }
@@ -383,7 +471,7 @@ cudaError_t launch_row_contract_t(const float* x, float2* out, long long rows, i
   const size_t slot = (size_t)BOXR * N3 * 4;
   const size_t fixed = 1024 + (size_t)4 * (N3 / 32) * 32 * 16 + 512;
   int stages = (int)((kRowSmemLimit - fixed) / slot);
-  if (stages > 14) stages = 14;
+  if (stages > 16) stages = 16;
   if (stages < 3) return cudaErrorInvalidConfiguration;
   const size_t total = (size_t)stages * slot + fixed;
   CUtensorMap map;
@@ -404,7 +492,7 @@ cudaError_t launch_row_expand_t(const float2* in, float* y, long long rows, int 
   const size_t tile = (size_t)BOXR * N3 * 4;
   const size_t fixed = 1024 + (size_t)4 * (N3 / 32) * 32 * 16;
   int W = (int)((kRowSmemLimit - fixed) / tile);
-  if (W > 8) W = 8;
+  if (W > 12) W = 12;
   if (W < 2) return cudaErrorInvalidConfiguration;
   CUtensorMap map;
   if (!make_rows_map(&map, y, rows, N3, BOXR)) return cudaErrorNotSupported;
@@ -418,6 +506,8 @@ cudaError_t launch_row_expand_t(const float2* in, float* y, long long rows, int 
     kern<<<grid, w * 32, total, st>>>(map, in, rows, N3, K3, scale, herm);
     return cudaGetLastError();
   };
+  if (W >= 12 && MT <= 2) return launch(row_expand_kernel<MT, 12>, 12);
+  if (W >= 10 && MT <= 2) return launch(row_expand_kernel<MT, 10>, 10);
   if (W >= 8) return launch(row_expand_kernel<MT, 8>, 8);
   if (W >= 6) return launch(row_expand_kernel<MT, 6>, 6);
   if (W >= 4) return launch(row_expand_kernel<MT, 4>, 4);
