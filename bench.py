@@ -276,6 +276,63 @@ def torch_fft_reference(torch, w, x, W, g, steps=3):
     return out
 
 
+def other_configs_summary(torch, skip_name, steps=10):
+    """Forward and forward+backward time of the other benchmark configurations (parity-test cases, not the
+    headline): seeded device-generated inputs of each shape, CUDA events, 3 warm-ups."""
+    from paper_2607_14394_b200 import Plan, inputs
+    out = {}
+    for name, w in inputs.WORKLOADS.items():
+        if name == skip_name:
+            continue
+        try:
+            dev = torch.device("cuda", torch.cuda.current_device())
+            plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out)
+            gen = torch.Generator(device=dev)
+            gen.manual_seed(w.seed)
+            x = torch.randn((w.B, w.C_in) + w.N, device=dev, generator=gen)
+            g = torch.randn((w.B, w.C_out) + w.N, device=dev, generator=gen)
+            W = inputs.make_weights_torch(w, dev)
+            X = plan.forward(x)
+            Y = plan.spectral_mul(X, W)
+            y = plan.inverse(Y)
+            gx, gW = plan.backward(g, X, W)
+
+            def fwd():
+                plan.forward(x, X)
+                plan.spectral_mul(X, W, Y)
+                plan.inverse(Y, y)
+
+            for _ in range(3):
+                fwd()
+                plan.backward(g, X, W, gx, gW)
+            torch.cuda.synchronize()
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            e[0].record()
+            for _ in range(steps):
+                fwd()
+            e[1].record()
+            for _ in range(steps):
+                plan.backward(g, X, W, gx, gW)
+            e[2].record()
+            torch.cuda.synchronize()
+            tf, tb = e[0].elapsed_time(e[1]) / steps, e[1].elapsed_time(e[2]) / steps
+            ab = algorithmic_bytes(w)
+            pts = w.B * w.points
+            out[name] = {"kernel_path": plan.kernel_path, "fwd_ms": tf, "fwd_bwd_ms": tf + tb,
+                         "fwd_gpoints_per_s": pts / tf / 1e6, "fwd_bwd_gpoints_per_s": pts / (tf + tb) / 1e6,
+                         "fwd_algorithmic_gbs": ab["fwd"] / tf / 1e6,
+                         "fwd_bwd_algorithmic_gbs": ab["fwd_bwd"] / (tf + tb) / 1e6,
+                         "grid_bytes": 4 * w.C_in * pts,
+                         "note": "grid smaller than L2: warm-cache, launch-bound" if 4 * w.C_in * pts < 126e6 else
+                                 "grid larger than L2"}
+            plan.close()
+            del plan, x, g, W, X, Y, y, gx, gW
+            torch.cuda.empty_cache()
+        except Exception as ex:
+            out[name] = {"error": f"{type(ex).__name__}: {ex}"[:160]}
+    return out
+
+
 def main_ours(args, w):
     import torch
     import torch.distributed as dist
@@ -463,6 +520,10 @@ def main_ours(args, w):
         torch.cuda.empty_cache()
         if not args.no_torch_ref:
             line["torch_fft_reference"] = torch_fft_reference(torch, w, x, W, g)
+        if not args.no_other_configs and args.channels == 0:
+            del x, g
+            torch.cuda.empty_cache()
+            line["other_configs"] = other_configs_summary(torch, w.name)
         if not args.no_cpu_baseline:
             try:
                 v, dt, info = time_oracle(w, 1, 0, budget=1.4e8)
@@ -492,6 +553,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-torch-ref", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true")
     args = ap.parse_args()
     from paper_2607_14394_b200 import inputs
     w = inputs.WORKLOADS[args.config]
