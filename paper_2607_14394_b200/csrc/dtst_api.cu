@@ -101,6 +101,12 @@ bool use_mid(const dtst_plan* p, int j) {
   return mid_supported((int)p->Ng[j], p->kmax[j]);
 }
 
+// A two-sided dimension that carries a phase offset, is only partly local, or is cut into virtual slabs.
+bool use_slab(const dtst_plan* p, int j) {
+  if (p->path_request != DTST_PATH_AUTO || j >= p->d - 1 || use_mid(p, j)) return false;
+  return slab_supported((int)p->Nl[j], p->kmax[j]);
+}
+
 bool use_fused(const dtst_plan* p) { return p->path_request == DTST_PATH_AUTO && fused_eligible(p); }
 
 // Row kernels: the contiguous dimension alone (whole on this device, zero offset), for shapes without a
@@ -158,6 +164,18 @@ dtst_status forward_stages(dtst_plan* p, const void* cur, int j_from, int flip, 
     if (in_real) {
       op.scale = scale;
       op.herm = herm ? 1 : 0;
+    }
+    if (!in_real && use_slab(p, j)) {
+      // slabs (or a rank's block) of this dimension: partial spectra formed and summed inside one kernel
+      void* sdst = (j == 0) ? static_cast<void*>(Xhat) : static_cast<void*>(buf[flip]);
+      if (cuda_failed(p, launch_slab(true, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(sdst),
+                                     op.outer, op.inner, (int)p->Nl[j], op.N, (int)p->off[j], j == 0 ? p->P : 1, st)))
+        return DTST_ERR_CUDA;
+      ++p->launches;
+      cur = sdst;
+      flip ^= 1;
+      if (j == 0) return DTST_OK;
+      continue;
     }
     void* dst;
     if (j == 0 && p->P > 1) {
@@ -243,7 +261,12 @@ dtst_status run_inverse_generic(dtst_plan* p, const float2* Yhat, float* y, int 
       op.out_slab_stride = (long long)nl * op.inner;
     }
     void* dst = out_real ? static_cast<void*>(y) : static_cast<void*>(buf[flip]);
-    if (!out_real && use_mid(p, j)) {
+    if (!out_real && use_slab(p, j)) {
+      if (cuda_failed(p, launch_slab(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
+                                     make_op(p, j, false, Cn).outer, make_op(p, j, false, Cn).inner, (int)p->Nl[j],
+                                     (int)p->Ng[j], (int)p->off[j], j == 0 ? p->P : 1, st)))
+        return DTST_ERR_CUDA;
+    } else if (!out_real && use_mid(p, j)) {
       if (cuda_failed(p, launch_mid(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
                                     op.outer, op.inner, op.N, 1.0f, st)))
         return DTST_ERR_CUDA;
@@ -278,7 +301,12 @@ dtst_status inverse_stages_complex(dtst_plan* p, const float2* cur_in, int j_to,
       op.out_slab_stride = (long long)nl * op.inner;
     }
     void* dst = buf[flip];
-    if (use_mid(p, j)) {
+    if (use_slab(p, j)) {
+      if (cuda_failed(p, launch_slab(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
+                                     make_op(p, j, false, Cn).outer, make_op(p, j, false, Cn).inner, (int)p->Nl[j],
+                                     (int)p->Ng[j], (int)p->off[j], j == 0 ? p->P : 1, st)))
+        return DTST_ERR_CUDA;
+    } else if (use_mid(p, j)) {
       if (cuda_failed(p, launch_mid(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
                                     op.outer, op.inner, op.N, 1.0f, st)))
         return DTST_ERR_CUDA;

@@ -136,6 +136,11 @@ cudaError_t launch_mix(const float2* X, const float2* W, float2* Y, int B, int C
 cudaError_t launch_mix_adjoint(const float2* GY, const float2* X, const float2* W, float2* GX, float2* GW,
                                int B, int Ci, int Co, long long M, cudaStream_t st, long long* launches);
 
+// offset / virtual-shard kernels for a two-sided middle dimension (dtst_slab.cu)
+bool slab_supported(int Nl, int K);
+cudaError_t launch_slab(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int Nl,
+                        int N, int off, int P, cudaStream_t st);
+
 // folded register-accumulator kernels for a two-sided middle dimension (dtst_mid.cu)
 bool mid_supported(int N, int K);
 cudaError_t launch_mid(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,

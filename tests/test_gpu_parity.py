@@ -121,14 +121,15 @@ def test_virtual_shards_match_oracle_and_unsharded(N, k, P, path):
 
 
 # ------------------------------------------------------------------ a rank's block with global offsets (Eq. 18)
+@pytest.mark.parametrize("Ng,k,nl,off", [((16, 12, 8), (3, 2, 4), (4, 6, 8), (8, 6, 0)),
+                                         ((32, 24, 32), (4, 8, 4), (8, 12, 32), (16, 12, 0))])
 @pytest.mark.parametrize("path", ["auto", "generic"])
-def test_local_block_plan_gives_partial_spectrum_and_block_inverse(path):
+def test_local_block_plan_gives_partial_spectrum_and_block_inverse(path, Ng, k, nl, off):
     from paper_2607_14394_b200 import Plan
-    Ng, k = (16, 12, 8), (3, 2, 4)
     w = I.custom_workload("local", 1, 2, 2, Ng, k, seed=31)
     x = I.make_field(w)
-    nl, off = (4, 6, 8), (8, 6, 0)
-    blk = np.ascontiguousarray(x[:, :, 8:12, 6:12, :])
+    sl = tuple(slice(o, o + n) for o, n in zip(off, nl))
+    blk = np.ascontiguousarray(x[(slice(None), slice(None)) + sl])
     plan = Plan(nl, k, 1, 2, 2, N_global=Ng, offset=off, path=path)
     part = plan.forward(_dev(blk)).cpu().numpy()
     ref = O.forward(blk, k, N_global=Ng, offsets=off)
@@ -137,6 +138,15 @@ def test_local_block_plan_gives_partial_spectrum_and_block_inverse(path):
     yb = plan.inverse(_dev(Y.astype(np.complex64))).cpu().numpy()
     yref = O.inverse(Y.astype(np.complex64), Ng, k, n_local=nl, offsets=off)
     assert O.rel_l2(yb, yref) <= TOL
+    # and the block's backward pass against the oracle's block statement
+    Wn = I.make_weights(w)
+    g = np.random.default_rng(9).standard_normal((1, 2) + tuple(nl)).astype(np.float32)
+    Xs = _dev(part.astype(np.complex64))
+    gx, gW = plan.backward(_dev(g), Xs, _dev(Wn))
+    gx_ref, gW_ref = O.backward(g, part.astype(np.complex64), Wn.reshape((2, 2) + ref.shape[2:]), k, N_global=Ng,
+                                offsets=off)
+    assert O.rel_l2(gx.cpu().numpy(), gx_ref) <= TOL
+    assert O.rel_l2(gW.cpu().numpy().reshape(gW_ref.shape), gW_ref) <= TOL
 
 
 # ------------------------------------------------------------------ run-to-run determinism and buffer discipline
