@@ -306,11 +306,12 @@ row_expand_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __r
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g8 = lane >> 2, t4 = lane & 3;
-  unsigned char* staging = smem + (size_t)warp * tile_bytes;
-  const uint32_t staging_s = smem_u32(staging);
-  const SmemTile tl_{staging, staging_s};
+  // two staging tiles per warp, used alternately: a tile is rewritten only after the store issued two tasks
+  // ago has read it, so a store's latency hides behind a whole task of work
+  unsigned char* staging0 = smem + (size_t)warp * 2 * tile_bytes;
+  const SmemTile tl_{staging0, smem_u32(staging0)};
   // basis fragments as MMA B operands: k = frequency slot, n = quadruple; [cls][nt][lane] float4
-  float4* btab = reinterpret_cast<float4*>(smem + (size_t)W * tile_bytes);
+  float4* btab = reinterpret_cast<float4*>(smem + (size_t)W * 2 * tile_bytes);
 
   if (threadIdx.x == 0) prefetch_tensormap(&out_map);
   for (int e = threadIdx.x; e < 4 * NNT * 32; e += blockDim.x) {
@@ -341,23 +342,32 @@ row_expand_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __r
 
   const long long num_tasks = (rows + BOXR - 1) / BOXR;
   const long long tstride = (long long)gridDim.x * W;
-  // raw input values of a task, fetched one task ahead: element (mt, e) needs frequencies 2 gi, 2 gi + 1
+  // raw input values of a task, fetched one task ahead: element (mt, e) needs frequencies 2 gi and 2 gi + 1,
+  // which are adjacent in memory: one 16-byte load when k3 is even (every row then starts 16-byte aligned)
   float2 vin[MT][4][2];
+  const bool pairload = (K3 & 1) == 0;
   auto load_inputs = [&](long long t) {
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const long long row = t * BOXR + 16 * mt + g8 + 8 * (e & 1);
-        const int gi = t4 + 4 * (e >> 1);
+        const int f0 = 2 * (t4 + 4 * (e >> 1));
+        const bool live = t < num_tasks && row < rows;
+        if (pairload) {
+          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (live && f0 < K3) v = __ldg(reinterpret_cast<const float4*>(in + row * K3 + f0));
+          vin[mt][e][0] = make_float2(v.x, v.y);
+          vin[mt][e][1] = make_float2(v.z, v.w);
+        } else {
 #pragma unroll
-        for (int p = 0; p < 2; ++p) {
-          const int f = 2 * gi + p;
-          vin[mt][e][p] = (t < num_tasks && row < rows && f < K3) ? __ldg(in + row * K3 + f) : make_float2(0.f, 0.f);
+          for (int p = 0; p < 2; ++p)
+            vin[mt][e][p] = (live && f0 + p < K3) ? __ldg(in + row * K3 + f0 + p) : make_float2(0.f, 0.f);
         }
       }
   };
   load_inputs((long long)blockIdx.x + (long long)warp * gridDim.x);
+  int iter = 0;
   for (long long task = (long long)blockIdx.x + (long long)warp * gridDim.x; task < num_tasks; task += tstride) {
     // A fragments: z'[row][slot] = scale c_f e^{-i pi f / N3} in[row][f]; classes take Re of even f, Re of
     // odd f, Im of odd f, Im of even f.  Element (row, slot): e&1 selects row + 8, e>>1 selects slot + 4.
@@ -380,8 +390,11 @@ row_expand_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __r
         split_tf32_r(im[0], ah[mt][3][e], al[mt][3][e]);
       }
     load_inputs(task + tstride);   // the next task's values travel while this one is expanded
-    // the previous task's TMA store must have finished reading the staging tile
-    if (lane == 0) tma_store_wait_read<0>();
+    // the store issued two tasks ago (same tile) must have finished reading it
+    unsigned char* staging = staging0 + (size_t)(iter & 1) * tile_bytes;
+    const uint32_t staging_s = tl_.s + (uint32_t)(iter & 1) * tile_bytes;
+    ++iter;
+    if (lane == 0) tma_store_wait_read<1>();
     __syncwarp();
     // Staging addressing, as in the contraction kernel: quadruple pair j0 = 8 nt + 2 t4 sits in panel nt >> 2,
     // chunk 2 (nt & 3) + (t4 >> 1), 8-byte slot (t4 & 1); its mirror images flip the chunk (XOR 0x70) and the slot.
@@ -461,7 +474,10 @@ row_expand_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __r
   if (lane == 0) tma_store_wait_all<0>();
 }
 
-int pick_mt(int N3) { return N3 <= 64 ? 4 : (N3 <= 128 ? 2 : 1); }
+// 2 KB TMA load boxes (16 rows) starve the contraction kernel (3.6 instead of 5.9 TB/s at N3 = 256): it uses
+// 32-row tasks; the expansion kernel keeps 16-row tiles at N3 > 128 so that two of them fit per warp.
+int pick_mt(int N3) { return N3 <= 64 ? 4 : 2; }
+int pick_mt_expand(int N3) { return N3 <= 64 ? 4 : (N3 <= 128 ? 2 : 1); }
 
 template <int MT>
 cudaError_t launch_row_contract_t(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm,
@@ -491,14 +507,14 @@ cudaError_t launch_row_expand_t(const float2* in, float* y, long long rows, int 
   constexpr int BOXR = 16 * MT;
   const size_t tile = (size_t)BOXR * N3 * 4;
   const size_t fixed = 1024 + (size_t)4 * (N3 / 32) * 32 * 16;
-  int W = (int)((kRowSmemLimit - fixed) / tile);
+  int W = (int)((kRowSmemLimit - fixed) / (2 * tile));
   if (W > 12) W = 12;
   if (W < 2) return cudaErrorInvalidConfiguration;
   CUtensorMap map;
   if (!make_rows_map(&map, y, rows, N3, BOXR)) return cudaErrorNotSupported;
   const long long tasks = (rows + BOXR - 1) / BOXR;
   auto launch = [&](auto kern, int w) -> cudaError_t {
-    const size_t total = (size_t)w * tile + fixed;
+    const size_t total = (size_t)w * 2 * tile + fixed;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
     if (e != cudaSuccess) return e;
     const long long want = (tasks + w - 1) / w;
@@ -531,7 +547,7 @@ cudaError_t launch_row_contract(const float* x, float2* out, long long rows, int
 
 cudaError_t launch_row_expand(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm,
                               cudaStream_t st) {
-  switch (pick_mt(N3)) {
+  switch (pick_mt_expand(N3)) {
     case 4: return launch_row_expand_t<4>(in, y, rows, N3, K3, scale, herm, st);
     case 2: return launch_row_expand_t<2>(in, y, rows, N3, K3, scale, herm, st);
     default: return launch_row_expand_t<1>(in, y, rows, N3, K3, scale, herm, st);
