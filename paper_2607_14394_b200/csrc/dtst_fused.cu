@@ -59,7 +59,12 @@ struct PlaneCfg {
   static constexpr int NS = 4 * NC + 8;                       // floats per combo row: 4 classes x NC, +8 pad
   static constexpr int ABS = NC + 1;                          // floats between A/B entries (odd: scalar accesses)
   static constexpr int ABP = (2 * K2 + 1) * ABS;
-  static constexpr int COMBO_FLOATS = (32 * NS > G * ABP ? 32 * NS : G * ABP);
+  // forward kernel: one parity class at a time, row stride NSC = 8 mod 16 words (conflict-free fragment loads)
+  static constexpr int NSC = (NC % 16 == 8) ? NC : NC + 8;
+  // per-warp buffer (class combos, later the A/B entries), a multiple of 128 bytes so that every warp's
+  // region stays 16-byte aligned for the vector stores
+  static constexpr int COMBO_FLOATS = (((32 * NSC > G * ABP ? 32 * NSC : G * ABP) + 31) / 32) * 32;
+  static constexpr int BTAB_FLOAT4 = 5 * NKS * 32;            // stage-2 basis fragments, CTA-shared
   static_assert(N3 % 32 == 0 && (N3 == 32 || N3 == 64), "N3");
   static_assert(kTaskRows % N2 == 0 && G * QUADS == 32, "one lane per row quadruple");
   static_assert(G * LPP <= 32 && (G * NC) % 16 == 0, "stage-2 mapping");
@@ -76,7 +81,7 @@ struct SmemPlan {
 template <typename Cfg, int K2, int K3, int W>
 SmemPlan smem_plan() {
   SmemPlan s;
-  const size_t combos = (size_t)W * Cfg::COMBO_FLOATS * 4;
+  const size_t combos = (size_t)W * Cfg::COMBO_FLOATS * 4 + (size_t)Cfg::BTAB_FLOAT4 * 16;
   const size_t rot = (size_t)2 * K2 * K3 * 8;
   const size_t fixed = 1024 /*alignment slack*/ + combos + rot + 512 /*barriers*/;
   s.stages = (int)((kSmemLimit - fixed) / kStageBytes);
@@ -202,7 +207,8 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char* ring = smem;
   const uint32_t ring_s = smem_u32(ring);
-  float* combos_all = reinterpret_cast<float*>(smem + (size_t)stages * kStageBytes);
+  float4* btab = reinterpret_cast<float4*>(smem + (size_t)stages * kStageBytes);
+  float* combos_all = reinterpret_cast<float*>(btab + Cfg::BTAB_FLOAT4);
   float2* rot = reinterpret_cast<float2*>(combos_all + (size_t)W * Cfg::COMBO_FLOATS);
   uint64_t* full = reinterpret_cast<uint64_t*>(rot + 2 * K2 * K3);
   uint64_t* empty = full + 16;
@@ -223,6 +229,30 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tensormap(&in_map);
+  }
+  // Stage-2 basis as MMA B fragments (k = quadruple n, n = frequency slot of the parity class), TF32 hi/lo,
+  // generated once per CTA: entry [cls][ks][lane] = (b0 hi, b1 hi, b0 lo, b1 lo).  Classes: 0 = A even (pp,
+  // cos), 1 = A odd (pd, cos), 2 = B odd (ms, sin), 3 = B even (md, sin); 4 = the unpaired A_{K2} (cos, shares
+  // the pp operand), in column 0 only.
+  for (int e = threadIdx.x; e < Cfg::BTAB_FLOAT4; e += blockDim.x) {
+    const int l = e & 31, ks = (e >> 5) % Cfg::NKS, cls = (e >> 5) / Cfg::NKS;
+    const int lg = l >> 2, lt = l & 3;
+    uint32_t hi[2], lo[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int n = 8 * ks + lt + 4 * h;
+      int g = 0;
+      bool valid = lg < Cfg::GT;
+      if (cls == 0) g = 2 * lg;
+      else if (cls == 1 || cls == 2) g = 2 * lg + 1;
+      else if (cls == 3) g = 2 * lg + 2;
+      else { g = K2; valid = (lg == 0); }
+      double sn, cs;
+      sincospi((double)(((long long)g * (2 * n + 1)) % (2 * N2)) / (double)N2, &sn, &cs);
+      const float v = valid ? ((cls == 2 || cls == 3) ? (float)sn : (float)cs) : 0.f;
+      split_tf32(v, hi[h], lo[h]);
+    }
+    btab[e] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(lo[0]), __uint_as_float(lo[1]));
   }
   // rotation table: the deferred half-sample phases of both dimensions, the scale and the
   // Hermitian weight, one complex factor per (mode position r, last-dim frequency f)
@@ -275,29 +305,6 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
     const int l2 = lane % LPP;
     // MMA fragment coordinates
     const int g8 = lane >> 2, t4 = lane & 3;
-
-    // Stage-2 basis as MMA B fragments (k = quadruple n, n = frequency slot of the parity class), split
-    // into TF32 hi/lo once.  Classes: 0 = A even (pp, cos), 1 = A odd (pd, cos), 2 = B odd (ms, sin),
-    // 3 = B even (md, sin); 4 = the unpaired A_{K2} (cos, shares the pp operand), in column 0 only.
-    uint32_t bhi[5][Cfg::NKS][2], blo[5][Cfg::NKS][2];
-#pragma unroll
-    for (int cls = 0; cls < 5; ++cls)
-#pragma unroll
-      for (int ks = 0; ks < Cfg::NKS; ++ks)
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int n = 8 * ks + t4 + 4 * h;
-          int g = 0;
-          bool valid = g8 < Cfg::GT;
-          if (cls == 0) g = 2 * g8;
-          else if (cls == 1 || cls == 2) g = 2 * g8 + 1;
-          else if (cls == 3) g = 2 * g8 + 2;
-          else { g = K2; valid = (g8 == 0); }
-          double sn, cs;
-          sincospi((double)(((long long)g * (2 * n + 1)) % (2 * N2)) / (double)N2, &sn, &cs);
-          const float v = valid ? ((cls == 2 || cls == 3) ? (float)sn : (float)cs) : 0.f;
-          split_tf32(v, bhi[cls][ks][h], blo[cls][ks][h]);
-        }
 
     for (long long tl = w; tl < n_local; tl += W) {
       const long long task = first + tl * gridDim.x;
@@ -355,24 +362,11 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
         }
       }
 
-      // publish the combos: row (plane, n), 4 classes x NC floats, 16-byte chunks swapped pairwise on
-      // odd groups of four rows so that both these stores and the fragment loads below are conflict-free
-      {
-        float* dst = combo + (size_t)lane * Cfg::NS;
-        const int sw = ((n1 >> 2) & 1);
-#pragma unroll
-        for (int c4 = 0; c4 < NC / 4; ++c4) {
-          const int cc = 4 * (c4 ^ sw);
-          *reinterpret_cast<float4*>(dst + 0 * NC + cc) = make_float4(cpp[4 * c4], cpp[4 * c4 + 1], cpp[4 * c4 + 2], cpp[4 * c4 + 3]);
-          *reinterpret_cast<float4*>(dst + 1 * NC + cc) = make_float4(cpd[4 * c4], cpd[4 * c4 + 1], cpd[4 * c4 + 2], cpd[4 * c4 + 3]);
-          *reinterpret_cast<float4*>(dst + 2 * NC + cc) = make_float4(cms[4 * c4], cms[4 * c4 + 1], cms[4 * c4 + 2], cms[4 * c4 + 3]);
-          *reinterpret_cast<float4*>(dst + 3 * NC + cc) = make_float4(cmd[4 * c4], cmd[4 * c4 + 1], cmd[4 * c4 + 2], cmd[4 * c4 + 3]);
-        }
-      }
-      __syncwarp();
-
-      // ---- stage 2 on the tensor cores (legacy warp-level MMA, TF32 with hi/lo error compensation):
-      // out[(plane, column)][frequency slot] = sum_n combo_cls[n][(plane, column)] * basis_cls[n][slot]
+      // ---- stage 2 on the tensor cores (legacy warp-level MMA, TF32 with hi/lo error compensation), one
+      // parity class at a time through a small per-warp buffer:
+      //   out[(plane, column)][frequency slot] = sum_n combo_cls[n][(plane, column)] * basis_cls[n][slot]
+      // The class's combos are published as rows (plane, n) of NC floats, 16-byte chunks swapped pairwise on
+      // odd groups of four rows so that both the stores and the fragment loads are bank-conflict free.
       float acc[5][Cfg::MT][4];
 #pragma unroll
       for (int cls = 0; cls < 5; ++cls)
@@ -381,9 +375,27 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
 #pragma unroll
           for (int e = 0; e < 4; ++e) acc[cls][mt][e] = 0.f;
 #pragma unroll
-      for (int cls = 0; cls < 4; ++cls)
+      for (int cls = 0; cls < 4; ++cls) {
+        __syncwarp();   // the previous class's fragment loads (or the previous task's epilogue reads) are done
+        {
+          float* dst = combo + (size_t)lane * Cfg::NSC;
+          const int sw = ((n1 >> 2) & 1);
 #pragma unroll
-        for (int ks = 0; ks < Cfg::NKS; ++ks)
+          for (int c4 = 0; c4 < NC / 4; ++c4) {
+            const int cc = 4 * (c4 ^ sw);
+            const float* srcv = (cls == 0) ? cpp : (cls == 1) ? cpd : (cls == 2) ? cms : cmd;
+            *reinterpret_cast<float4*>(dst + cc) =
+                make_float4(srcv[4 * c4], srcv[4 * c4 + 1], srcv[4 * c4 + 2], srcv[4 * c4 + 3]);
+          }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int ks = 0; ks < Cfg::NKS; ++ks) {
+          const float4 bf = btab[(cls * Cfg::NKS + ks) * 32 + lane];
+          const uint32_t bh0 = __float_as_uint(bf.x), bh1 = __float_as_uint(bf.y);
+          const uint32_t bl0 = __float_as_uint(bf.z), bl1 = __float_as_uint(bf.w);
+          float4 bx = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (cls == 0) bx = btab[(4 * Cfg::NKS + ks) * 32 + lane];
 #pragma unroll
           for (int mt = 0; mt < Cfg::MT; ++mt) {
             uint32_t ahi[4], alo[4];
@@ -392,18 +404,20 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
               const int m = 16 * mt + g8 + 8 * (e & 1);
               const int n = 8 * ks + t4 + 4 * (e >> 1);
               const int pl = m / NC, c = m % NC;
-              const float v = combo[(size_t)(pl * QUADS + n) * Cfg::NS + cls * NC + (c ^ ((e >> 1) << 2))];
+              const float v = combo[(size_t)(pl * QUADS + n) * Cfg::NSC + (c ^ ((e >> 1) << 2))];
               split_tf32(v, ahi[e], alo[e]);
             }
-            mma_tf32(acc[cls][mt], ahi, bhi[cls][ks][0], bhi[cls][ks][1]);
-            mma_tf32(acc[cls][mt], alo, bhi[cls][ks][0], bhi[cls][ks][1]);
-            mma_tf32(acc[cls][mt], ahi, blo[cls][ks][0], blo[cls][ks][1]);
+            mma_tf32(acc[cls][mt], ahi, bh0, bh1);
+            mma_tf32(acc[cls][mt], alo, bh0, bh1);
+            mma_tf32(acc[cls][mt], ahi, bl0, bl1);
             if (cls == 0) {   // the pp operand also feeds the unpaired A_{K2}
-              mma_tf32(acc[4][mt], ahi, bhi[4][ks][0], bhi[4][ks][1]);
-              mma_tf32(acc[4][mt], alo, bhi[4][ks][0], bhi[4][ks][1]);
-              mma_tf32(acc[4][mt], ahi, blo[4][ks][0], blo[4][ks][1]);
+              mma_tf32(acc[4][mt], ahi, __float_as_uint(bx.x), __float_as_uint(bx.y));
+              mma_tf32(acc[4][mt], alo, __float_as_uint(bx.x), __float_as_uint(bx.y));
+              mma_tf32(acc[4][mt], ahi, __float_as_uint(bx.z), __float_as_uint(bx.w));
             }
           }
+        }
+      }
       __syncwarp();
 
       // A/B sums -> shared: entry g for A_g (g <= K2), entry K2+g for B_g (g >= 1)
@@ -817,7 +831,7 @@ void fill_stage1_table(Stage1Table<N3, K3>* t) {
 template <int N3, int K3, int N2, int K2>
 cudaError_t launch_fwd_plane_t(const float* x, float2* out, long long rows, float scale, int herm, int* status,
                                cudaStream_t st) {
-  constexpr int W = 7;   // 7 consumer warps + the producer warp = 256 threads x 255 registers = the whole file
+  constexpr int W = 7;   // consumer warps (+ the producer warp = 2 warps per scheduler; 8 or 10 consumers measured slower)
   using Cfg = PlaneCfg<N3, K3, N2, K2>;
   const SmemPlan sp = smem_plan<Cfg, K2, K3, W>();
   if (sp.stages < 2 * Cfg::SPT) return cudaErrorInvalidConfiguration;
