@@ -104,11 +104,12 @@ class ClockSampler:
         return out
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu launch list of this
-# very command at full size; the summary with the command line is profiles/launch_list_cfg5_4d_128.md.
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the two grid-streaming kernels, from one
+# ncu capture of a small case of the same shape (2 channels instead of 16, 1.07 GB of grid: larger than L2, small
+# enough for a multi-pass capture) scaled by the channel ratio 8 - their traffic is proportional to the channel
+# count.  The summary with the command line is profiles/kernels_cfg5_shape_c2_ncu_full.md.
 NCU_TRAFFIC = {
-    "cfg5_4d_128": {"grid_read": 8590074368 + 533445632, "grid_write": 537079040 + 8526035968,
-                    "mix": 661641216 + 28915456, "mix_adjoint": 998619136 + 537102592},
+    "cfg5_4d_128": {"grid_read": 8 * (1073793000 + 64813000), "grid_write": 8 * (67168000 + 1013249000)},
 }
 
 
