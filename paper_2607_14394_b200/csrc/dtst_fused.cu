@@ -34,14 +34,64 @@ constexpr int kTaskRows = 128;       // rows of the contiguous dimension per war
 constexpr int kStageBytes = 16384;   // one ring slot
 constexpr int kSmemLimit = 232448;   // 227 KB opt-in limit per CTA
 
-// Stage-1 coefficients cos/sin(2 pi f (j + 1/2) / N3), j < N3/4, delivered in the kernel
-// parameter constant bank so that every FMA takes its coefficient as a constant operand
-// (a shared-memory operand would cost LDS bandwidth this kernel does not have).
-template <int N3, int K3>
-struct Stage1Table {
-  float cs[N3 / 4][K3];
-  float sn[N3 / 4][K3];
+// Stage-1 coefficients cos/sin(2 pi f (j + 1/2) / N3), j < N3/4, as COMPILE-TIME constants: the row code is fully
+// unrolled over (j, f), so every FMA carries its coefficient as a 32-bit immediate.  No table in HBM, shared or
+// constant memory, no load instruction, no register: a shared-memory operand would cost LDS bandwidth this kernel
+// does not have, and a constant-bank table costs one uniform load per four coefficients (measured: 9 % of the
+// forward kernel's instructions, 22 % of the inverse kernel's).
+namespace ct {
+constexpr double kPi = 3.14159265358979323846264338327950288;
+// Taylor series on |x| <= pi/4 (terms to x^27: below 1e-19)
+constexpr double sin_small(double x) {
+  const double x2 = x * x;
+  double term = x, sum = x;
+  for (int k = 1; k <= 13; ++k) {
+    term *= -x2 / (double)((2 * k) * (2 * k + 1));
+    sum += term;
+  }
+  return sum;
+}
+constexpr double cos_small(double x) {
+  const double x2 = x * x;
+  double term = 1.0, sum = 1.0;
+  for (int k = 1; k <= 13; ++k) {
+    term *= -x2 / (double)((2 * k - 1) * (2 * k));
+    sum += term;
+  }
+  return sum;
+}
+// cos(pi num / den), sin(pi num / den): the argument is reduced exactly in integers to the first octant
+constexpr double cospi_ratio(long long num, long long den) {
+  num %= 2 * den;
+  if (num < 0) num += 2 * den;
+  if (num > den) num = 2 * den - num;          // cos(2 pi - a) = cos a
+  double sign = 1.0;
+  if (2 * num > den) {                         // cos(pi - a) = -cos a
+    num = den - num;
+    sign = -1.0;
+  }
+  if (4 * num <= den) return sign * cos_small(kPi * (double)num / (double)den);
+  return sign * sin_small(kPi * (double)(den - 2 * num) / (double)(2 * den));   // cos a = sin(pi/2 - a)
+}
+constexpr double sinpi_ratio(long long num, long long den) {
+  num %= 2 * den;
+  if (num < 0) num += 2 * den;
+  double sign = 1.0;
+  if (num > den) {                             // sin(2 pi - a) = -sin a
+    num = 2 * den - num;
+    sign = -1.0;
+  }
+  if (2 * num > den) num = den - num;          // sin(pi - a) = sin a
+  if (4 * num <= den) return sign * sin_small(kPi * (double)num / (double)den);
+  return sign * cos_small(kPi * (double)(den - 2 * num) / (double)(2 * den));   // sin a = cos(pi/2 - a)
+}
+// phase (2j+1) f / (2 N3) turns = pi (2j+1) f / N3
+template <int N3, int J, int F>
+struct Coef {
+  static constexpr float cs = (float)cospi_ratio((long long)(2 * J + 1) * F, N3);
+  static constexpr float sn = (float)sinpi_ratio((long long)(2 * J + 1) * F, N3);
 };
+}  // namespace ct
 
 template <int N3, int K3, int N2, int K2>
 struct PlaneCfg {
@@ -114,9 +164,8 @@ __device__ __forceinline__ void sts128_s(uint32_t addr, float a, float b, float 
 
 // fp32 -> (hi, lo) TF32 pair with hi + lo = v to ~2^-22 relative (error-compensated "3xTF32")
 __device__ __forceinline__ void split_tf32(float v, uint32_t& hi, uint32_t& lo) {
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(v));
-  const float r = v - __uint_as_float(hi);
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(r));
+  hi = __float_as_uint(v) & 0xffffe000u;
+  lo = __float_as_uint(v - __uint_as_float(hi));
 }
 
 // D += A(16x8, row) * B(8x8, col), TF32 inputs, fp32 accumulate
@@ -127,53 +176,59 @@ __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], 
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// Forward row code, one quadruple j: o[f] += folded input * coefficient(j, f), f = F .. K3-1 (compile-time recursion
+// so that j and f are constant expressions and the coefficients become immediates).
+template <int N3, int K3, int J, int F>
+__device__ __forceinline__ void s1_freqs(float uu, float ud, float vs, float vd, float (&o)[2 * K3]) {
+  if constexpr (F < K3) {
+    constexpr float cs = ct::Coef<N3, J, F>::cs, sn = ct::Coef<N3, J, F>::sn;
+    if constexpr ((F & 1) == 0) {
+      o[F] = (J == 0) ? uu * cs : fmaf(uu, cs, o[F]);
+      if constexpr (F > 0) o[K3 + F] = (J == 0) ? vd * sn : fmaf(vd, sn, o[K3 + F]);
+    } else {
+      o[F] = (J == 0) ? ud * cs : fmaf(ud, cs, o[F]);
+      o[K3 + F] = (J == 0) ? vs * sn : fmaf(vs, sn, o[K3 + F]);
+    }
+    s1_freqs<N3, K3, J, F + 1>(uu, ud, vs, vd, o);
+  }
+}
+
+// chunks C, CH/2-1-C, CH/2+C, CH-1-C of the row: four quadruples j = 4C .. 4C+3
+template <int N3, int K3, int BOXR, int C>
+__device__ __forceinline__ void s1_chunks(uint32_t rx, float (&o)[2 * K3]) {
+  constexpr int CH = N3 / 4;
+  if constexpr (C < CH / 4) {
+    constexpr int P = BOXR * 128;
+    constexpr int c0 = C, c1 = CH / 2 - 1 - C, c2 = CH / 2 + C, c3 = CH - 1 - C;
+    // (the panel offset is an immediate, the XOR constant depends on the chunk only)
+    const float4 A = lds128_s<(c0 / 8) * P>(rx ^ (uint32_t)((c0 % 8) << 4));
+    const float4 Bq = lds128_s<(c1 / 8) * P>(rx ^ (uint32_t)((c1 % 8) << 4));
+    const float4 Cq = lds128_s<(c2 / 8) * P>(rx ^ (uint32_t)((c2 % 8) << 4));
+    const float4 D = lds128_s<(c3 / 8) * P>(rx ^ (uint32_t)((c3 % 8) << 4));
+#define DTST_QUAD(E, av, bv, cv, dv)                                               \
+    {                                                                              \
+      const float u = (av) + (dv), v = (av) - (dv);                                \
+      const float up = (bv) + (cv), vp = (bv) - (cv);                              \
+      s1_freqs<N3, K3, 4 * C + (E), 0>(u + up, u - up, v + vp, v - vp, o);         \
+    }
+    DTST_QUAD(0, A.x, Bq.w, Cq.x, D.w)
+    DTST_QUAD(1, A.y, Bq.z, Cq.y, D.z)
+    DTST_QUAD(2, A.z, Bq.y, Cq.z, D.y)
+    DTST_QUAD(3, A.w, Bq.x, Cq.w, D.x)
+#undef DTST_QUAD
+    s1_chunks<N3, K3, BOXR, C + 1>(rx, o);
+  }
+}
+
 // One row of N3 reals -> C_f = sum u cos, S_f = sum v sin for f < K3 (half-sample phase deferred).
 // `stage` is the 32-bit shared address of the slot (1024-byte aligned), BOXR its rows per 128-byte panel.
 template <int N3, int K3, int BOXR>
-__device__ __forceinline__ void stage1_row(uint32_t stage, int row, const Stage1Table<N3, K3>& tab,
-                                           float (&o)[2 * K3]) {
-  constexpr int CH = N3 / 4;
-#pragma unroll
-  for (int i = 0; i < 2 * K3; ++i) o[i] = 0.f;
+__device__ __forceinline__ void stage1_row(uint32_t stage, int row, float (&o)[2 * K3]) {
+  o[K3] = 0.f;   // the sine sum of f = 0 has no terms
   // chunk c of this row sits at row*128 + ((c ^ (row & 7)) << 4) (+ one panel for c >= 8); the row base has
   // zeros in bits 4..6, so the swizzle is a single XOR of a precomputed base with a constant
   const uint32_t rx = stage + (uint32_t)row * 128u + (((uint32_t)row & 7u) << 4);
-#pragma unroll
-  for (int c = 0; c < CH / 4; ++c) {
-    constexpr int P = BOXR * 128;
-    const int c0 = c, c1 = CH / 2 - 1 - c, c2 = CH / 2 + c, c3 = CH - 1 - c;
-    float4 A, Bq, Cq, D;
-    // (the panel offset is an immediate, the XOR constant depends on c only)
-#define DTST_LD(dst, cc)                                                        \
-    dst = ((cc) / 8 == 0) ? lds128_s<0>(rx ^ (uint32_t)(((cc) % 8) << 4))       \
-                          : lds128_s<P>(rx ^ (uint32_t)(((cc) % 8) << 4));
-    DTST_LD(A, c0)
-    DTST_LD(Bq, c1)
-    DTST_LD(Cq, c2)
-    DTST_LD(D, c3)
-#undef DTST_LD
-    const float a[4] = {A.x, A.y, A.z, A.w};
-    const float b[4] = {Bq.w, Bq.z, Bq.y, Bq.x};
-    const float cc[4] = {Cq.x, Cq.y, Cq.z, Cq.w};
-    const float d[4] = {D.w, D.z, D.y, D.x};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int j = 4 * c + e;
-      const float u = a[e] + d[e], v = a[e] - d[e];
-      const float up = b[e] + cc[e], vp = b[e] - cc[e];
-      const float uu = u + up, ud = u - up, vs = v + vp, vd = v - vp;
-#pragma unroll
-      for (int f = 0; f < K3; ++f) {
-        if ((f & 1) == 0) {
-          o[f] = fmaf(uu, tab.cs[j][f], o[f]);
-          if (f > 0) o[K3 + f] = fmaf(vd, tab.sn[j][f], o[K3 + f]);
-        } else {
-          o[f] = fmaf(ud, tab.cs[j][f], o[f]);
-          o[K3 + f] = fmaf(vs, tab.sn[j][f], o[K3 + f]);
-        }
-      }
-    }
-  }
+  s1_chunks<N3, K3, BOXR, 0>(rx, o);
 }
 
 // Consumer side of the ring: wait until fill number q (0-based) of `slot` has landed.
@@ -194,8 +249,7 @@ __device__ __forceinline__ bool wait_fill(volatile uint32_t* fill_seq, uint64_t*
 
 template <int N3, int K3, int N2, int K2, int W>
 __global__ void __launch_bounds__((W + 1) * 32, 1)
-fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_constant__ Stage1Table<N3, K3> tab,
-                 float2* __restrict__ out, long long num_tasks, float scale, int herm, int stages,
+fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict__ out, long long num_tasks, float scale, int herm, int stages,
                  int* __restrict__ status) {
   using Cfg = PlaneCfg<N3, K3, N2, K2>;
   constexpr int NC = Cfg::NC, QUADS = Cfg::QUADS, G = Cfg::G, LPP = Cfg::LPP;
@@ -342,7 +396,7 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
         const int sl = (trow / RPS) ? slot1 : slot0;
         const uint32_t st = ring_s + (uint32_t)sl * kStageBytes;
         float o[NC];
-        stage1_row<N3, K3, RPS>(st, trow % RPS, tab, o);
+        stage1_row<N3, K3, RPS>(st, trow % RPS, o);
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
           cpp[c] += o[c];
@@ -481,46 +535,57 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, const __grid_consta
 // modes, forms alpha_g = V'_{+g} + V'_{-g}, beta_g = i (V'_{+g} - V'_{-g}), expands them to the
 // four rows of each row quadruple (one lane per quadruple), expands every row to N3 reals with
 // the same folded basis, stages the rows in shared memory (TMA swizzle) and stores them with TMA.
-template <int N3, int K3, int BOXR>
-__device__ __forceinline__ void expand_row(uint32_t stage, int row, const Stage1Table<N3, K3>& tab,
-                                           const float (&z)[2 * K3]) {
+// Inverse row code, one quadruple j: the four class sums over f = F .. K3-1 with immediate coefficients.
+template <int N3, int K3, int J, int F>
+__device__ __forceinline__ void e1_freqs(const float (&z)[2 * K3], float& Ea, float& Oa, float& Eb, float& Ob) {
+  if constexpr (F < K3) {
+    constexpr float cs = ct::Coef<N3, J, F>::cs, sn = ct::Coef<N3, J, F>::sn;
+    if constexpr ((F & 1) == 0) {
+      Ea = (F == 0) ? z[F] * cs : fmaf(z[F], cs, Ea);
+      if constexpr (F > 0) Eb = (F == 2) ? z[K3 + F] * sn : fmaf(z[K3 + F], sn, Eb);
+    } else {
+      Oa = (F == 1) ? z[F] * cs : fmaf(z[F], cs, Oa);
+      Ob = (F == 1) ? z[K3 + F] * sn : fmaf(z[K3 + F], sn, Ob);
+    }
+    e1_freqs<N3, K3, J, F + 1>(z, Ea, Oa, Eb, Ob);
+  }
+}
+
+template <int N3, int K3, int J>
+__device__ __forceinline__ void e1_quad(const float (&z)[2 * K3], float& ya, float& yb, float& yc, float& yd) {
+  float Ea = 0.f, Oa = 0.f, Eb = 0.f, Ob = 0.f;
+  e1_freqs<N3, K3, J, 0>(z, Ea, Oa, Eb, Ob);
+  const float sa = Ea + Oa, da = Ea - Oa, sb = Eb + Ob, db = Eb - Ob;
+  ya = sa - sb;   // y[j]
+  yd = sa + sb;   // y[N3-1-j]
+  yb = da + db;   // y[N3/2-1-j]
+  yc = da - db;   // y[N3/2+j]
+}
+
+template <int N3, int K3, int BOXR, int C>
+__device__ __forceinline__ void e1_chunks(uint32_t rx, const float (&z)[2 * K3]) {
   constexpr int CH = N3 / 4;
-  constexpr int P = BOXR * 128;
+  if constexpr (C < CH / 4) {
+    constexpr int P = BOXR * 128;
+    constexpr int c0 = C, c1 = CH / 2 - 1 - C, c2 = CH / 2 + C, c3 = CH - 1 - C;
+    float a[4], b[4], cc[4], d[4];
+    e1_quad<N3, K3, 4 * C + 0>(z, a[0], b[0], cc[0], d[0]);
+    e1_quad<N3, K3, 4 * C + 1>(z, a[1], b[1], cc[1], d[1]);
+    e1_quad<N3, K3, 4 * C + 2>(z, a[2], b[2], cc[2], d[2]);
+    e1_quad<N3, K3, 4 * C + 3>(z, a[3], b[3], cc[3], d[3]);
+    sts128_s<(c0 / 8) * P>(rx ^ (uint32_t)((c0 % 8) << 4), a[0], a[1], a[2], a[3]);
+    sts128_s<(c1 / 8) * P>(rx ^ (uint32_t)((c1 % 8) << 4), b[3], b[2], b[1], b[0]);
+    sts128_s<(c2 / 8) * P>(rx ^ (uint32_t)((c2 % 8) << 4), cc[0], cc[1], cc[2], cc[3]);
+    sts128_s<(c3 / 8) * P>(rx ^ (uint32_t)((c3 % 8) << 4), d[3], d[2], d[1], d[0]);
+    e1_chunks<N3, K3, BOXR, C + 1>(rx, z);
+  }
+}
+
+template <int N3, int K3, int BOXR>
+__device__ __forceinline__ void expand_row(uint32_t stage, int row, const float (&z)[2 * K3]) {
   // same single-XOR swizzled addressing as the forward kernel's row loads
   const uint32_t rx = stage + (uint32_t)row * 128u + (((uint32_t)row & 7u) << 4);
-#pragma unroll
-  for (int c = 0; c < CH / 4; ++c) {
-    float a[4], b[4], cc[4], d[4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int j = 4 * c + e;
-      float Ea = 0.f, Oa = 0.f, Eb = 0.f, Ob = 0.f;
-#pragma unroll
-      for (int f = 0; f < K3; ++f) {
-        if ((f & 1) == 0) {
-          Ea = fmaf(z[f], tab.cs[j][f], Ea);
-          if (f > 0) Eb = fmaf(z[K3 + f], tab.sn[j][f], Eb);
-        } else {
-          Oa = fmaf(z[f], tab.cs[j][f], Oa);
-          Ob = fmaf(z[K3 + f], tab.sn[j][f], Ob);
-        }
-      }
-      const float sa = Ea + Oa, da = Ea - Oa, sb = Eb + Ob, db = Eb - Ob;
-      a[e] = sa - sb;    // y[j]
-      d[e] = sa + sb;    // y[N3-1-j]
-      b[e] = da + db;    // y[N3/2-1-j]
-      cc[e] = da - db;   // y[N3/2+j]
-    }
-    const int c0 = c, c1 = CH / 2 - 1 - c, c2 = CH / 2 + c, c3 = CH - 1 - c;
-#define DTST_ST(cidx, v0, v1, v2, v3)                                                         \
-    if ((cidx) / 8 == 0) sts128_s<0>(rx ^ (uint32_t)(((cidx) % 8) << 4), v0, v1, v2, v3);     \
-    else sts128_s<P>(rx ^ (uint32_t)(((cidx) % 8) << 4), v0, v1, v2, v3);
-    DTST_ST(c0, a[0], a[1], a[2], a[3])
-    DTST_ST(c1, b[3], b[2], b[1], b[0])
-    DTST_ST(c2, cc[0], cc[1], cc[2], cc[3])
-    DTST_ST(c3, d[3], d[2], d[1], d[0])
-#undef DTST_ST
-  }
+  e1_chunks<N3, K3, BOXR, 0>(rx, z);
 }
 
 template <int N3, int K3, int N2, int K2>
@@ -543,8 +608,7 @@ struct InvCfg {
 
 template <int N3, int K3, int N2, int K2, int W>
 __global__ void __launch_bounds__(W * 32, 1)
-inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_constant__ Stage1Table<N3, K3> tab,
-                 const float2* __restrict__ in, long long num_tasks, float scale, int herm) {
+inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __restrict__ in, long long num_tasks, float scale, int herm) {
   using Cfg = PlaneCfg<N3, K3, N2, K2>;
   using IC = InvCfg<N3, K3, N2, K2>;
   constexpr int NC = Cfg::NC, QUADS = Cfg::QUADS, G = Cfg::G, LPP = Cfg::LPP;
@@ -779,7 +843,7 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const __grid_const
 #pragma unroll
       for (int c = 0; c < NC; ++c) z[c] = fmaf(sQo, Qo[c], fmaf(sQe, Qe[c], fmaf(sPo, Po[c], Pe[c])));
       const int trow = pl1 * N2 + rowq;
-      expand_row<N3, K3, RPS>(staging_s + (uint32_t)(trow / RPS) * kStageBytes, trow % RPS, tab, z);
+      expand_row<N3, K3, RPS>(staging_s + (uint32_t)(trow / RPS) * kStageBytes, trow % RPS, z);
     }
     fence_proxy_async_smem();
     __syncwarp();
@@ -816,18 +880,6 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-template <int N3, int K3>
-void fill_stage1_table(Stage1Table<N3, K3>* t) {
-  for (int j = 0; j < N3 / 4; ++j)
-    for (int f = 0; f < K3; ++f) {
-      // phase (2j+1) f / (2 N3) turns, reduced exactly before the double-precision evaluation
-      const long long num = ((long long)(2 * j + 1) * f) % (2ll * N3);
-      const double ang = 3.14159265358979323846 * (double)num / (double)N3;
-      t->cs[j][f] = (float)cos(ang);
-      t->sn[j][f] = (float)sin(ang);
-    }
-}
-
 template <int N3, int K3, int N2, int K2>
 cudaError_t launch_fwd_plane_t(const float* x, float2* out, long long rows, float scale, int herm, int* status,
                                cudaStream_t st) {
@@ -837,14 +889,12 @@ cudaError_t launch_fwd_plane_t(const float* x, float2* out, long long rows, floa
   if (sp.stages < 2 * Cfg::SPT) return cudaErrorInvalidConfiguration;
   CUtensorMap map;
   if (!make_rows_map(&map, x, rows, N3, Cfg::ROWS_PER_STAGE)) return cudaErrorNotSupported;
-  Stage1Table<N3, K3> tab;
-  fill_stage1_table(&tab);
   auto kern = fwd_plane_kernel<N3, K3, N2, K2, W>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sp.total);
   if (e != cudaSuccess) return e;
   const long long tasks = rows / kTaskRows;
   const int grid = (int)(tasks < kNumSMs ? tasks : kNumSMs);
-  kern<<<grid, (W + 1) * 32, sp.total, st>>>(map, tab, out, tasks, scale, herm, sp.stages, status);
+  kern<<<grid, (W + 1) * 32, sp.total, st>>>(map, out, tasks, scale, herm, sp.stages, status);
   return cudaGetLastError();
 }
 
@@ -857,15 +907,13 @@ cudaError_t launch_inv_plane_t(const float2* in, float* y, long long rows, float
   static_assert((size_t)W * IC::WARP_BYTES + (size_t)2 * K2 * K3 * 8 + 1024 <= kSmemLimit, "shared memory");
   CUtensorMap map;
   if (!make_rows_map(&map, y, rows, N3, PlaneCfg<N3, K3, N2, K2>::ROWS_PER_STAGE)) return cudaErrorNotSupported;
-  Stage1Table<N3, K3> tab;
-  fill_stage1_table(&tab);
   auto kern = inv_plane_kernel<N3, K3, N2, K2, W>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
   if (e != cudaSuccess) return e;
   const long long tasks = rows / kTaskRows;
   const long long want = (tasks + W - 1) / W;
   const int grid = (int)(want < kNumSMs ? want : kNumSMs);
-  kern<<<grid, W * 32, total, st>>>(map, tab, in, tasks, scale, herm);
+  kern<<<grid, W * 32, total, st>>>(map, in, tasks, scale, herm);
   return cudaGetLastError();
 }
 
