@@ -143,6 +143,10 @@ cudaError_t launch_slab(bool forward, int K, const float2* in, float2* out, long
 
 // folded register-accumulator kernels for a two-sided middle dimension (dtst_mid.cu)
 bool mid_supported(int N, int K);
+// tensor-core variant of the middle-dimension kernels (N % 32 == 0, inner % 4 == 0)
+bool mid_mma_supported(int N, int K, long long inner);
+cudaError_t launch_mid_mma(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
+                           float scale, cudaStream_t st);
 cudaError_t launch_mid(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
                        float scale, cudaStream_t st);
 

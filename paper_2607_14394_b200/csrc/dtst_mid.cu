@@ -349,6 +349,8 @@ bool mid_supported(int N, int K) {
 cudaError_t launch_mid(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
                        float scale, cudaStream_t st) {
   if (outer * inner <= 0) return cudaSuccess;
+  const bool aligned16 = ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
+  if (aligned16 && mid_mma_supported(N, K, inner)) return launch_mid_mma(forward, K, in, out, outer, inner, N, scale, st);
   // two adjacent positions per thread need an even inner extent (then every pair is 16-byte aligned and
   // never straddles two outer slices) and 16-byte aligned tensors
   const bool vec = (inner % 2 == 0) && ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;

@@ -1,0 +1,490 @@
+// Two-sided middle dimension on the tensor cores: the same folded contraction / expansion as dtst_mid.cu
+// (Eq. 18 with zero offset, half-sample phase factored out),
+//     A_g = sum_{q<N/2} (z_q + z_{N-1-q}) cos(psi_g (q + 1/2)),   B_g = sum_{q<N/2} (z_q - z_{N-1-q}) sin(psi_g (q + 1/2)),
+//     Z_{+-g} = e^{+-i psi_g/2} (A_g -+ i B_g),
+// but with the sums over q as warp-level TF32 MMAs (hi/lo compensated, fp32 accumulate).  The complex tensor
+// [outer][N][inner] is read as a REAL matrix with 2*inner columns: the basis is real after the fold, so real
+// and imaginary parts are just neighbouring columns, and a C fragment's column pair (2 t4, 2 t4 + 1) is one
+// complex value.  The cosine frequencies g = 0..K-1 fill one 16-row MMA tile, the sine frequencies g = 1..K a
+// second one (row 0 carries g = K, whose sine partner g = 0 vanishes); the one left over, cos K, runs on FFMA.
+//
+// On the FFMA version this stage was issue-bound (half of all instructions were the multiply-adds, the other
+// half their bookkeeping); here one task of 32 complex positions x N rows needs ~3x fewer instructions and the
+// stage becomes an HBM stream.  Shapes: N % 32 == 0, K in {4, 8, 12, 16}, inner % 4 == 0.
+#include <type_traits>
+
+#include "dtst_common.cuh"
+#include "dtst_mma.cuh"
+
+namespace dtst {
+namespace {
+
+constexpr int kMmaWarps = 12;   // one persistent CTA per SM: the basis tables are built once per SM
+constexpr int kMmaThreads = kMmaWarps * 32;
+constexpr int kNT = 8;              // expansion: MMA n-tiles per task: 64 real columns = 32 complex positions
+constexpr int kTaskPos = 4 * kNT;   // complex positions per task
+constexpr int kCNT = 4;             // contraction: 4 n-tiles per task (one 128-byte line per row), more warps
+constexpr int kCPos = 4 * kCNT;
+constexpr int kCWarps = 16;
+constexpr int kCThreads = kCWarps * 32;
+
+__device__ __forceinline__ float4 as_f4(const uint32_t (&v)[4]) {
+  return make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
+}
+__device__ __forceinline__ void from_f4(const float4 f, uint32_t (&v)[4]) {
+  v[0] = __float_as_uint(f.x);
+  v[1] = __float_as_uint(f.y);
+  v[2] = __float_as_uint(f.z);
+  v[3] = __float_as_uint(f.w);
+}
+
+// cos / sin of pi * g * (2 q + 1) / N with the phase reduced exactly in integers
+__device__ __forceinline__ void basis_cs(int g, int q, int N, float& cs, float& sn) {
+  double s, c;
+  sincospi((double)(((long long)g * (2 * q + 1)) % (2ll * N)) / (double)N, &s, &c);
+  cs = (float)c;
+  sn = (float)s;
+}
+
+// ------------------------------------------------------------------------------------------
+// contraction: in[outer][N][inner] -> out[outer][2K][inner]
+//   MMA roles: M = frequency slot (basis = A operand, from a fragment-ordered shared table),
+//              K = mirrored row pair q, N = real column (data = B operand, straight from global memory).
+// ------------------------------------------------------------------------------------------
+// The contraction streams its input through a per-warp ring of shared-memory stages filled with cp.async
+// (16 bytes per lane and request): one stage = one k-step of one task = 8 rows and their 8 mirror rows, 128 bytes
+// each.  The ring runs ahead across task boundaries, so several kilobytes per warp are in flight at all times
+// without holding them in registers (with register double-buffering this stage was bound by load latency).
+constexpr int kCStages = 4;
+constexpr int kCRow = 8 * kCNT + 8;          // floats per staged row: 40 = 8 mod 32, conflict-free B fragments
+constexpr int kCStageFloats = 16 * kCRow;
+
+__device__ __forceinline__ void cp_async16(float* smem_dst, const float* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// One k-step from a filled stage.  FULL: all kCNT column tiles are valid (no predicates in the instruction stream).
+template <bool FULL>
+__device__ __forceinline__ void contract_step(const float* S, const float4* at, const float* cK, int q0, int ntv,
+                                              float (&accC)[kCNT][4], float (&accS)[kCNT][4], float (&aK)[kCNT]) {
+  uint32_t ch[4], cl[4], sh[4], sl[4];
+  from_f4(at[0], ch);
+  from_f4(at[32], cl);
+  from_f4(at[64], sh);
+  from_f4(at[96], sl);
+  const float ck0 = cK[q0], ck1 = cK[q0 + 4];
+#pragma unroll
+  for (int nt = 0; nt < kCNT; ++nt) {
+    if (FULL || nt < ntv) {
+      // rows t4, t4 + 4 of the k-step and their mirrors (staged 8 rows further down)
+      const float x0 = S[8 * nt], x1 = S[8 * kCRow + 8 * nt];
+      const float x2 = S[4 * kCRow + 8 * nt], x3 = S[12 * kCRow + 8 * nt];
+      const float p0 = x0 + x1, d0 = x0 - x1;
+      const float p1 = x2 + x3, d1 = x2 - x3;
+      uint32_t ph0, pl0, ph1, pl1, dh0, dl0, dh1, dl1;
+      split_tf32_round(p0, ph0, pl0);
+      split_tf32_round(p1, ph1, pl1);
+      split_tf32_round(d0, dh0, dl0);
+      split_tf32_round(d1, dh1, dl1);
+      mma3_tf32(accC[nt], ch, cl, ph0, ph1, pl0, pl1);
+      mma3_tf32(accS[nt], sh, sl, dh0, dh1, dl0, dl1);
+      aK[nt] = fmaf(p0, ck0, fmaf(p1, ck1, aK[nt]));
+    }
+  }
+}
+
+template <int K>
+__global__ void __launch_bounds__(kCThreads, 1)
+mid_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out, long long outer, long long inner,
+                        int N, float scale) {
+  extern __shared__ float4 mm_smem[];
+  const int KS = N / 16;                                    // k-steps of 8 row pairs (even: N % 32 == 0)
+  float4* atab = mm_smem;                                   // [KS][tile cos|sin][hi|lo][lane]
+  float* cK = reinterpret_cast<float*>(atab + (size_t)KS * 4 * 32);   // cos(psi_K (q + 1/2)), q < N/2
+
+  for (int e = threadIdx.x; e < KS * 2 * 32; e += blockDim.x) {
+    const int l = e & 31, tile = (e >> 5) & 1, ks = e >> 6;
+    const int lg = l >> 2, lt = l & 3;
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const int r = lg + 8 * (a & 1), q = 8 * ks + lt + 4 * (a >> 1);
+      const int g = (tile == 1 && r == 0) ? K : r;
+      float cs, sn;
+      basis_cs(g, q, N, cs, sn);
+      const float v = (r < K) ? (tile == 0 ? cs : sn) : 0.f;
+      split_tf32_rna(v, hi[a], lo[a]);
+    }
+    atab[((ks * 2 + tile) * 2 + 0) * 32 + l] = as_f4(hi);
+    atab[((ks * 2 + tile) * 2 + 1) * 32 + l] = as_f4(lo);
+  }
+  for (int q = threadIdx.x; q < N / 2; q += blockDim.x) {
+    float cs, sn;
+    basis_cs(K, q, N, cs, sn);
+    cK[q] = cs;
+  }
+  __syncthreads();
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g8 = lane >> 2, t4 = lane & 3;
+  // e^{i psi_g / 2} * scale for this lane's frequencies g8, g8 + 8 and for K
+  float2 rho_a, rho_b, rho_K;
+  {
+    double s, c;
+    sincospi((double)g8 / (double)N, &s, &c);
+    rho_a = make_float2((float)c * scale, (float)s * scale);
+    sincospi((double)(g8 + 8) / (double)N, &s, &c);
+    rho_b = make_float2((float)c * scale, (float)s * scale);
+    sincospi((double)K / (double)N, &s, &c);
+    rho_K = make_float2((float)c * scale, (float)s * scale);
+  }
+
+  const long long cblocks = (inner + kCPos - 1) / kCPos;
+  const long long tasks = outer * cblocks;
+  const long long rs = 2 * inner;   // floats per row
+  const long long tstride = (long long)gridDim.x * kCWarps;
+  float* ring = cK + N / 2 + (size_t)warp * kCStages * kCStageFloats;   // this warp's stages (16-byte aligned)
+
+  // producer cursor: (task, k-step) of the next stage to request; lane = (row group lane / 8, 16-byte chunk lane % 8)
+  long long ptask = (long long)blockIdx.x * kCWarps + warp;
+  int pks = 0, pstage = 0;
+  const float* ptb = in;
+  bool pchunk_ok = false;
+  auto issue = [&]() {
+    if (ptask < tasks) {
+      if (pks == 0) {
+        const long long o = ptask / cblocks, cb = ptask % cblocks;
+        const long long left = inner - cb * kCPos;
+        const int nch = left >= kCPos ? 2 * kCNT : (int)(left / 2);   // valid 16-byte chunks per row
+        ptb = in + o * N * rs + cb * (2 * kCPos) + 4 * (lane & 7);
+        pchunk_ok = (lane & 7) < nch;
+      }
+      if (pchunk_ok) {
+        float* dst = ring + pstage * kCStageFloats + (lane >> 3) * kCRow + 4 * (lane & 7);
+        const int q = 8 * pks + (lane >> 3);
+        // staged rows: 0..7 = rows q of the k-step, 8..15 = their mirrors N-1-q
+        cp_async16(dst, ptb + (long long)q * rs);
+        cp_async16(dst + 4 * kCRow, ptb + (long long)(q + 4) * rs);
+        cp_async16(dst + 8 * kCRow, ptb + (long long)(N - 1 - q) * rs);
+        cp_async16(dst + 12 * kCRow, ptb + (long long)(N - 5 - q) * rs);
+      }
+      if (++pks == KS) {
+        pks = 0;
+        ptask += tstride;
+      }
+    }
+    cp_async_commit();   // one group per call, also when nothing was requested: the wait below counts groups
+    pstage = pstage + 1 == kCStages ? 0 : pstage + 1;
+  };
+#pragma unroll
+  for (int i = 0; i < kCStages - 1; ++i) issue();
+
+  int cstage = 0;
+  for (long long task = (long long)blockIdx.x * kCWarps + warp; task < tasks; task += tstride) {
+    const long long o = task / cblocks, cb = task % cblocks;
+    const long long left = inner - cb * kCPos;
+    const int ntv = left >= kCPos ? kCNT : (int)(left / 4);   // valid n-tiles
+
+    float accC[kCNT][4], accS[kCNT][4], aK[kCNT];
+#pragma unroll
+    for (int nt = 0; nt < kCNT; ++nt) {
+      aK[nt] = 0.f;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) accC[nt][e] = accS[nt][e] = 0.f;
+    }
+
+    auto body = [&](auto full_tag) {
+      constexpr bool FULL = decltype(full_tag)::value;
+#pragma unroll 1
+      for (int ks = 0; ks < KS; ++ks) {
+        cp_async_wait<kCStages - 2>();   // this k-step's stage has landed (for this lane's requests) ...
+        __syncwarp();                    // ... and for everyone's; all lanes are done with the previous stage
+        issue();                         // refill the stage read in the previous k-step
+        const float* S = ring + cstage * kCStageFloats + t4 * kCRow + g8;
+        contract_step<FULL>(S, atab + (size_t)(ks * 4) * 32 + lane, cK, 8 * ks + t4, ntv, accC, accS, aK);
+        cstage = cstage + 1 == kCStages ? 0 : cstage + 1;
+      }
+    };
+    if (ntv == kCNT) body(std::true_type{});
+    else body(std::false_type{});
+
+    // A_K: sum the quad's partial sums (each lane covered the row pairs t4, t4 + 4 of every k-step)
+#pragma unroll
+    for (int nt = 0; nt < kCNT; ++nt) {
+      aK[nt] += __shfl_xor_sync(0xffffffffu, aK[nt], 1);
+      aK[nt] += __shfl_xor_sync(0xffffffffu, aK[nt], 2);
+    }
+
+    // Z_{+g} = rho_g (A_g - i B_g) -> row g (g < K);  Z_{-g} = conj(rho_g) (A_g + i B_g) -> row 2K - g (g >= 1)
+    float2* ob = out + o * (2 * K) * inner + cb * kCPos + t4;
+    auto emit = [&](int g, float2 rho, float ax, float ay, float bx, float by, float2* dst) {
+      const float pr = ax + by, pi = ay - bx;   // A - iB
+      const float mr = ax - by, mi = ay + bx;   // A + iB
+      if (g < K) dst[(long long)g * inner] = make_float2(rho.x * pr - rho.y * pi, rho.x * pi + rho.y * pr);
+      if (g > 0) dst[(long long)(2 * K - g) * inner] = make_float2(rho.x * mr + rho.y * mi, rho.x * mi - rho.y * mr);
+    };
+#pragma unroll
+    for (int nt = 0; nt < kCNT; ++nt) {
+      // every lane takes part in the shuffles; lanes of row group 0 need A_K of their column pair
+      const float aKr = __shfl_sync(0xffffffffu, aK[nt], (2 * t4) * 4);
+      const float aKi = __shfl_sync(0xffffffffu, aK[nt], (2 * t4 + 1) * 4);
+      if (nt < ntv) {
+        float2* dst = ob + 4 * nt;
+        if (g8 < K) {
+          const float bx = g8 > 0 ? accS[nt][0] : 0.f, by = g8 > 0 ? accS[nt][1] : 0.f;
+          emit(g8, rho_a, accC[nt][0], accC[nt][1], bx, by, dst);
+        }
+        if (g8 + 8 < K) emit(g8 + 8, rho_b, accC[nt][2], accC[nt][3], accS[nt][2], accS[nt][3], dst);
+        if (g8 == 0) emit(K, rho_K, aKr, aKi, accS[nt][0], accS[nt][1], dst);
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// expansion: in[outer][2K][inner] -> out[outer][N][inner]   (B^H along this dimension)
+//   z_n = P_n + Q_n, z_{N-1-n} = P_n - Q_n, n < N/2,
+//   P_n = sum_{g<=K} alpha_g cos(psi_g (n+1/2)), Q_n = sum_{1<=g<=K} beta_g sin(psi_g (n+1/2)),
+//   alpha_g = V'_{+g} + V'_{-g}, beta_g = i (V'_{+g} - V'_{-g}), V'_{+-g} = e^{-+i psi_g/2} V_{+-g}.
+//   MMA roles: M = output row n (basis = A operand, fragment-ordered shared table), K = frequency slot
+//   (cos: g = 0..K-1, sin: g = 1..K, eight per k-step), N = real column.  A warp first forms alpha, beta of its
+//   32 positions in a private shared buffer (one lane per position, coalesced loads), then walks the column
+//   tiles: B fragments from that buffer, all row tiles against them, rows stored straight from the C fragments.
+//   alpha_K cos(psi_K (n+1/2)) is added on FFMA.
+// ------------------------------------------------------------------------------------------
+template <int K>
+struct ExpCfg {
+  static constexpr int KS = (K + 7) / 8;         // k-steps over the frequencies
+  static constexpr int ROW = 2 * kTaskPos + 8;   // floats per buffer row: 72 = 8 mod 32, conflict-free B loads
+  static constexpr int ROWS = 8 * KS + 1;        // alpha rows 0..8KS-1 (zero beyond K-1) + row 8KS for alpha_K
+  static constexpr int WARP_FLOATS = 2 * ROWS * ROW;   // alpha block, beta block (beta row j holds g = j + 1)
+};
+
+template <int K>
+__global__ void __launch_bounds__(kMmaThreads, 1)
+mid_expand_mma_kernel(const float2* __restrict__ in, float* __restrict__ out, long long outer, long long inner,
+                      int N, float scale) {
+  using EC = ExpCfg<K>;
+  constexpr int KS = EC::KS;
+  extern __shared__ float4 mm_smem[];
+  const int MT = N / 32;                                   // 16-row tiles over n < N/2
+  float4* atab = mm_smem;                                  // [MT][KS][tile cos|sin][hi|lo][lane]
+  float* cK = reinterpret_cast<float*>(atab + (size_t)MT * KS * 4 * 32);   // cos(psi_K (n + 1/2)), n < N/2
+  float2* rho = reinterpret_cast<float2*>(cK + N / 2);     // e^{i psi_g / 2} * scale, g <= K
+  float* bufs = reinterpret_cast<float*>(rho + K + 1 + ((K + 1) & 1));     // 16-byte aligned
+
+  for (int e = threadIdx.x; e < MT * KS * 2 * 32; e += blockDim.x) {
+    const int l = e & 31, tile = (e >> 5) & 1, ks = (e >> 6) % KS, mt = (e >> 6) / KS;
+    const int lg = l >> 2, lt = l & 3;
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const int n = 16 * mt + lg + 8 * (a & 1);
+      const int j = 8 * ks + lt + 4 * (a >> 1);      // frequency slot
+      const int g = tile == 0 ? j : j + 1;
+      const bool valid = tile == 0 ? (g < K) : (g <= K);
+      float cs, sn;
+      basis_cs(g, n, N, cs, sn);
+      const float v = valid ? (tile == 0 ? cs : sn) : 0.f;
+      split_tf32_rna(v, hi[a], lo[a]);
+    }
+    atab[(((mt * KS + ks) * 2 + tile) * 2 + 0) * 32 + l] = as_f4(hi);
+    atab[(((mt * KS + ks) * 2 + tile) * 2 + 1) * 32 + l] = as_f4(lo);
+  }
+  for (int n = threadIdx.x; n < N / 2; n += blockDim.x) {
+    float cs, sn;
+    basis_cs(K, n, N, cs, sn);
+    cK[n] = cs;
+  }
+  for (int g = threadIdx.x; g <= K; g += blockDim.x) {
+    double s, c;
+    sincospi((double)g / (double)N, &s, &c);
+    rho[g] = make_float2((float)c * scale, (float)s * scale);
+  }
+  __syncthreads();
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g8 = lane >> 2, t4 = lane & 3;
+  float* al = bufs + (size_t)warp * EC::WARP_FLOATS;       // alpha rows
+  float* be = al + EC::ROWS * EC::ROW;                     // beta rows (row j <-> g = j + 1)
+  // rows that no frequency fills stay zero for the whole kernel
+  for (int e = lane; e < EC::WARP_FLOATS; e += 32) al[e] = 0.f;
+  __syncwarp();
+
+  const long long cblocks = (inner + kTaskPos - 1) / kTaskPos;
+  const long long tasks = outer * cblocks;
+  const long long rs = 2 * inner;   // floats per output row
+  for (long long task = (long long)blockIdx.x * kMmaWarps + warp; task < tasks;
+       task += (long long)gridDim.x * kMmaWarps) {
+    const long long o = task / cblocks, cb = task % cblocks;
+    const long long left = inner - cb * kTaskPos;
+    const int ntv = left >= kTaskPos ? kNT : (int)(left / 4);
+
+    // ---- alpha, beta of this task's positions: lane = position
+    {
+      const bool ok = lane < 4 * ntv;
+      const float2* src = in + o * (2 * K) * inner + cb * kTaskPos + lane;
+#pragma unroll
+      for (int g = 0; g <= K; ++g) {
+        const float2 r = rho[g];
+        float2 v = make_float2(0.f, 0.f), u = make_float2(0.f, 0.f);
+        if (ok && g < K) v = __ldg(src + (long long)g * inner);
+        if (ok && g > 0) u = __ldg(src + (long long)(2 * K - g) * inner);
+        const float2 vp = make_float2(v.x * r.x + v.y * r.y, v.y * r.x - v.x * r.y);   // v * conj(rho)
+        const float2 vm = make_float2(u.x * r.x - u.y * r.y, u.y * r.x + u.x * r.y);   // u * rho
+        const int arow = g < K ? g : 8 * KS;
+        *reinterpret_cast<float2*>(al + arow * EC::ROW + 2 * lane) = make_float2(vp.x + vm.x, vp.y + vm.y);
+        if (g > 0)
+          *reinterpret_cast<float2*>(be + (g - 1) * EC::ROW + 2 * lane) =
+              make_float2(-(vp.y - vm.y), vp.x - vm.x);                                // i (vp - vm)
+      }
+    }
+    __syncwarp();
+
+    // pull the next task's 2K input rows (256 bytes each) into L2 while this one runs on the tensor cores
+    {
+      const long long nt_task = task + (long long)gridDim.x * kMmaWarps;
+      if (nt_task < tasks) {
+        const long long o2 = nt_task / cblocks, cb2 = nt_task % cblocks;
+        const float2* nsrc = in + o2 * (2 * K) * inner + cb2 * kTaskPos;
+        const bool second = inner - cb2 * kTaskPos > 16;   // the second 128-byte line holds valid positions
+        for (int r = lane; r < 2 * K; r += 32) {
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(nsrc + (long long)r * inner));
+          if (second) asm volatile("prefetch.global.L2 [%0];" ::"l"(nsrc + (long long)r * inner + 16));
+        }
+      }
+    }
+
+    float* ob = out + o * N * rs + cb * (2 * kTaskPos) + 2 * t4;
+    const float* alq = al + t4 * EC::ROW + g8;   // B fragment element (slot t4 + 4h + 8ks, column 8nt + g8)
+    const float* beq = be + t4 * EC::ROW + g8;
+    const float* aKp = al + (8 * KS) * EC::ROW + 2 * t4;
+
+    // row tiles outermost: the basis fragments of a tile are loaded once and meet all column tiles, whose
+    // fragments come from the warp's buffer; a row tile's 16 + 16 rows are written 256 bytes at a time
+    auto body = [&](auto full_tag) {
+      constexpr bool FULL = decltype(full_tag)::value;
+#pragma unroll 1
+      for (int mt = 0; mt < MT; ++mt) {
+        uint32_t ch[KS][4], cl[KS][4], sh[KS][4], sl[KS][4];
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+          const float4* t = atab + (size_t)((mt * KS + ks) * 4) * 32 + lane;
+          from_f4(t[0], ch[ks]);
+          from_f4(t[32], cl[ks]);
+          from_f4(t[64], sh[ks]);
+          from_f4(t[96], sl[ks]);
+        }
+        const int n0 = 16 * mt + g8;
+        const float c0 = cK[n0], c1 = cK[n0 + 8];
+        float* da = ob + (long long)n0 * rs;
+        float* db = da + 8 * rs;
+        float* dc = ob + (long long)(N - 1 - n0) * rs;
+        float* dd = dc - 8 * rs;
+#pragma unroll 1
+        for (int nh = 0; nh < kNT; nh += 4)
+#pragma unroll
+        for (int ni = 0; ni < 4; ++ni) {
+          const int nt = nh + ni;
+          if (FULL || nt < ntv) {
+            float P[4] = {0.f, 0.f, 0.f, 0.f}, Q[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+              uint32_t ah0, al0, ah1, al1, bh0, bl0, bh1, bl1;
+              split_tf32_round(alq[(8 * ks) * EC::ROW + 8 * nt], ah0, al0);
+              split_tf32_round(alq[(8 * ks + 4) * EC::ROW + 8 * nt], ah1, al1);
+              split_tf32_round(beq[(8 * ks) * EC::ROW + 8 * nt], bh0, bl0);
+              split_tf32_round(beq[(8 * ks + 4) * EC::ROW + 8 * nt], bh1, bl1);
+              mma3_tf32(P, ch[ks], cl[ks], ah0, ah1, al0, al1);
+              mma3_tf32(Q, sh[ks], sl[ks], bh0, bh1, bl0, bl1);
+            }
+            const float2 aK = *reinterpret_cast<const float2*>(aKp + 8 * nt);
+            P[0] = fmaf(aK.x, c0, P[0]);
+            P[1] = fmaf(aK.y, c0, P[1]);
+            P[2] = fmaf(aK.x, c1, P[2]);
+            P[3] = fmaf(aK.y, c1, P[3]);
+            *reinterpret_cast<float2*>(da + 8 * nt) = make_float2(P[0] + Q[0], P[1] + Q[1]);
+            *reinterpret_cast<float2*>(db + 8 * nt) = make_float2(P[2] + Q[2], P[3] + Q[3]);
+            *reinterpret_cast<float2*>(dc + 8 * nt) = make_float2(P[0] - Q[0], P[1] - Q[1]);
+            *reinterpret_cast<float2*>(dd + 8 * nt) = make_float2(P[2] - Q[2], P[3] - Q[3]);
+          }
+        }
+      }
+    };
+    if (ntv == kNT) body(std::true_type{});
+    else body(std::false_type{});
+    __syncwarp();   // the next task's alpha, beta overwrite the buffer read above
+  }
+}
+
+template <int K>
+size_t contract_smem(int N) {
+  return (size_t)(N / 16) * 4 * 32 * 16 + (size_t)(N / 2) * 4 + (size_t)kCWarps * kCStages * kCStageFloats * 4;
+}
+
+template <int K>
+size_t expand_smem(int N) {
+  return (size_t)(N / 32) * ExpCfg<K>::KS * 4 * 32 * 16 + (size_t)(N / 2) * 4 + (size_t)(K + 1 + ((K + 1) & 1)) * 8 +
+         (size_t)kMmaWarps * ExpCfg<K>::WARP_FLOATS * 4;
+}
+
+template <int K>
+cudaError_t launch_mid_mma_t(bool forward, const float2* in, float2* out, long long outer, long long inner, int N,
+                             float scale, cudaStream_t st) {
+  const size_t smem = forward ? contract_smem<K>(N) : expand_smem<K>(N);
+  const int pos = forward ? kCPos : kTaskPos, warps = forward ? kCWarps : kMmaWarps, threads = warps * 32;
+  const long long tasks = outer * ((inner + pos - 1) / pos);
+  const long long want = (tasks + warps - 1) / warps;
+  // persistent CTAs: exactly as many as are resident at once
+  auto grid_for = [&](auto kern, int* grid) -> cudaError_t {
+    cudaError_t e = cudaSuccess;
+    if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    const long long cap = (long long)kNumSMs * per_sm;
+    *grid = (int)(want < cap ? want : cap);
+    return cudaSuccess;
+  };
+  int grid = 1;
+  if (forward) {
+    auto kern = mid_contract_mma_kernel<K>;
+    cudaError_t e = grid_for(kern, &grid);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, threads, smem, st>>>(reinterpret_cast<const float*>(in), out, outer, inner, N, scale);
+  } else {
+    auto kern = mid_expand_mma_kernel<K>;
+    cudaError_t e = grid_for(kern, &grid);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, threads, smem, st>>>(in, reinterpret_cast<float*>(out), outer, inner, N, scale);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool mid_mma_supported(int N, int K, long long inner) {
+  if (N % 32 != 0 || N < 32 || N > 512 || 2 * K > N) return false;
+  if (!(K == 4 || K == 8 || K == 12 || K == 16)) return false;
+  return inner > 0 && inner % 4 == 0;
+}
+
+cudaError_t launch_mid_mma(bool forward, int K, const float2* in, float2* out, long long outer, long long inner,
+                           int N, float scale, cudaStream_t st) {
+  if (outer * inner <= 0) return cudaSuccess;
+  switch (K) {
+    case 4: return launch_mid_mma_t<4>(forward, in, out, outer, inner, N, scale, st);
+    case 8: return launch_mid_mma_t<8>(forward, in, out, outer, inner, N, scale, st);
+    case 12: return launch_mid_mma_t<12>(forward, in, out, outer, inner, N, scale, st);
+    case 16: return launch_mid_mma_t<16>(forward, in, out, outer, inner, N, scale, st);
+    default: return cudaErrorNotSupported;
+  }
+}
+
+}  // namespace dtst
