@@ -93,6 +93,12 @@ EDGE = [
     ("row_256", 1, 1, 2, (4, 6, 256), (2, 3, 16)),
     ("row_d1", 3, 2, 2, (128,), (7,)),
     ("row_k1", 1, 2, 2, (9, 64), (4, 1)),
+    # middle dimensions on the tensor-core kernels (N % 32 == 0, inner extent a multiple of 4): k = 4 / 8 / 12 / 16,
+    # N not a power of two, column tiles that end inside a task, a single column tile
+    ("mid_mma_k4", 1, 2, 2, (32, 32, 64), (4, 4, 2)),
+    ("mid_mma_n96_k12", 1, 2, 1, (96, 64, 32), (12, 8, 6)),
+    ("mid_mma_tail", 1, 2, 2, (64, 32, 32), (16, 4, 5)),
+    ("mid_mma_thin", 2, 1, 2, (32, 64, 32), (8, 8, 4)),
 ]
 
 
