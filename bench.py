@@ -18,9 +18,7 @@ import json
 import math
 import os
 import statistics
-import subprocess
 import sys
-import tempfile
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -45,60 +43,99 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples SM clock, power and throttle reasons while the timed region runs (read-only NVML queries from a
+    thread, every 10 ms: a child nvidia-smi takes longer to start than a short timed region lasts)."""
 
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    REASONS = ((0x8, "hw_slowdown"), (0x40, "hw_thermal_slowdown"), (0x20, "sw_thermal_slowdown"),
+               (0x4, "sw_power_cap"))
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index: int, uuid=None):
         self.gpu = gpu_index
-        self.proc = None
-        self.path = None
+        self.uuid = uuid
+        self.thread = None
+        self.samples = []
+        self.stop_flag = False
+        self.nvml = None
+        self.handle = None
+
+    def _open(self):
+        import pynvml
+        pynvml.nvmlInit()
+        self.nvml = pynvml
+        handle = None
+        if self.uuid:
+            for cand in (f"GPU-{self.uuid}", str(self.uuid)):
+                try:
+                    handle = pynvml.nvmlDeviceGetHandleByUUID(cand)
+                    break
+                except Exception:
+                    handle = None
+        if handle is None:
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            idx = self.gpu
+            parts = [t for t in visible.split(",") if t.strip()]
+            if parts and self.gpu < len(parts) and parts[self.gpu].strip().isdigit():
+                idx = int(parts[self.gpu])
+            handle = pynvml.nvmlDeviceGetHandleByIndex(idx)
+        self.handle = handle
+        self.max_sm = pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM)
+
+    def _sample(self):
+        n, h = self.nvml, self.handle
+        sm = n.nvmlDeviceGetClockInfo(h, n.NVML_CLOCK_SM)
+        try:
+            power = n.nvmlDeviceGetPowerUsage(h) / 1000.0
+        except Exception:
+            power = None
+        try:
+            getter = getattr(n, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                n.nvmlDeviceGetCurrentClocksThrottleReasons
+            mask = int(getter(h))
+        except Exception:
+            mask = 0
+        self.samples.append((sm, power, mask))
+
+    def _run(self):
+        import time as _t
+        while not self.stop_flag:
+            try:
+                self._sample()
+            except Exception:
+                break
+            _t.sleep(0.01)
 
     def start(self):
         try:
-            fd, self.path = tempfile.mkstemp(prefix="dtst_clocks_", suffix=".csv")
-            os.close(fd)
-            self.fh = open(self.path, "w")
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "20"], stdout=self.fh, stderr=subprocess.DEVNULL)
+            self._open()
+            self._sample()
+            import threading
+            self.thread = threading.Thread(target=self._run, daemon=True)
+            self.thread.start()
         except Exception:
-            self.proc = None
+            self.thread = None
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
+        if self.nvml is None or self.handle is None:
             return out
         try:
-            self.proc.terminate()          # the exact child we started
-            self.proc.wait(timeout=5)
+            self._sample()
         except Exception:
             pass
+        self.stop_flag = True
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        if self.samples:
+            sm = [t[0] for t in self.samples]
+            power = [t[1] for t in self.samples if t[1] is not None]
+            mask = 0
+            for t in self.samples:
+                mask |= t[2]
+            out = {"sm_mhz": statistics.median(sm), "sm_max_mhz": self.max_sm,
+                   "reasons": sorted(name for bit, name in self.REASONS if mask & bit),
+                   "samples": len(sm), "power_w_max": max(power) if power else None}
         try:
-            self.fh.close()
-            sm, mx, power = [], [], []
-            reasons = set()
-            with open(self.path) as fh:
-                for line in fh:
-                    p = [t.strip() for t in line.split(",")]
-                    if len(p) < 9:
-                        continue
-                    try:
-                        sm.append(float(p[1]))
-                        mx.append(float(p[2]))
-                        power.append(float(p[3]))
-                    except ValueError:
-                        continue
-                    for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
-                                         p[5:9]):
-                        if val.lower().startswith("active"):
-                            reasons.add(name)
-            os.unlink(self.path)
-            if sm:
-                out = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                       "samples": len(sm), "power_w_max": max(power) if power else None}
+            self.nvml.nvmlShutdown()
         except Exception:
             pass
         return out
@@ -109,7 +146,7 @@ class ClockSampler:
 # enough for a multi-pass capture) scaled by the channel ratio 8 - their traffic is proportional to the channel
 # count.  The summary with the command line is profiles/kernels_cfg5_shape_c2_ncu_full.md.
 NCU_TRAFFIC = {
-    "cfg5_4d_128": {"grid_read": 8 * (1073793000 + 64813000), "grid_write": 8 * (67168000 + 1013249000)},
+    "cfg5_4d_128": {"grid_read": 8 * (1073788000 + 64662000), "grid_write": 8 * (67159000 + 1018316000)},
 }
 
 
@@ -389,7 +426,7 @@ def main_ours(args, w):
 
     plan.enable_kernel_timing(2 * steps + 2)
     phase_events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(local_rank, uuid=getattr(torch.cuda.get_device_properties(local_rank), "uuid", None))
     launches0 = plan.launch_count()
     barrier()
     torch.cuda.synchronize()
