@@ -46,5 +46,28 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+# ---- the plain-C driver (tests/c_driver): proves the library is usable without Python or C++
+REPO = os.path.dirname(HERE)
+C_DRIVER_SRC = os.path.join(REPO, "tests", "c_driver", "dtst_c_driver.c")
+C_DRIVER_BIN = os.path.join(HERE, "dtst_c_driver")
+
+
+def build_c_driver(force: bool = False) -> str:
+    """gcc -std=c99 against include/dtst.h, libdtst.so (found through an $ORIGIN rpath) and the CUDA runtime."""
+    build()
+    if not force and os.path.exists(C_DRIVER_BIN) and \
+            os.path.getmtime(C_DRIVER_BIN) >= max(os.path.getmtime(C_DRIVER_SRC), os.path.getmtime(LIB)):
+        return C_DRIVER_BIN
+    cuda = os.path.dirname(os.path.dirname(_nvcc()))
+    cmd = ["gcc", "-std=c99", "-O2", "-Wall", "-I", os.path.join(REPO, "include"), "-I", os.path.join(cuda, "include"),
+           C_DRIVER_SRC, "-o", C_DRIVER_BIN, "-L", HERE, "-ldtst", "-L", os.path.join(cuda, "lib64"), "-lcudart",
+           "-Wl,-rpath,$ORIGIN", "-Wl,-rpath," + os.path.join(cuda, "lib64")]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError("gcc failed:\n" + res.stdout + res.stderr)
+    return C_DRIVER_BIN
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_c_driver(force="--force" in sys.argv))
