@@ -585,7 +585,7 @@ def main():
     ap.add_argument("--config", default=DEFAULT_WORKLOAD)
     ap.add_argument("--shards", type=int, default=1, help="virtual shards along dim 0")
     ap.add_argument("--path", default="auto", choices=["auto", "generic"])
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--channels", type=int, default=0,
                     help="override C_in = C_out (smaller cases for profiler captures; not a bench configuration)")
     ap.add_argument("--no-e2e", action="store_true")

@@ -55,9 +55,9 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
                                                   uint32_t limit = (1u << 24)) {
   for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(40);
     if ((it & 63u) == 63u) {
       if (*abort_flag) return false;
-      __nanosleep(64);
     }
   }
   *abort_flag = 1;
