@@ -3,8 +3,9 @@
 // Forward ("plane") kernel: contracts the last two grid dimensions in one pass.  The real
 // grid is read from HBM exactly once through a TMA-fed shared-memory ring; each consumer
 // warp owns a task of 128 consecutive rows (one or two [N2 x N3] planes), contracts the
-// contiguous dimension with one thread per row, then the next dimension with one thread
-// per retained frequency, and writes only the [2*k2 x k3] complex result of each plane.
+// contiguous dimension with one thread per row (folded FFMA with immediate coefficients),
+// then the next dimension on the tensor cores (TF32 hi/lo compensated warp MMAs), and writes
+// only the [2*k2 x k3] complex result of each plane.
 //
 // Both contractions use the symmetries of the DFT basis (Eq. 18 with zero offset): with the
 // half-sample phase factored out,
@@ -20,6 +21,7 @@
 #include <cuda.h>
 
 #include "dtst_fused.cuh"
+#include "dtst_mma.cuh"
 #include "dtst_sm100.cuh"
 
 namespace dtst {
@@ -144,8 +146,6 @@ SmemPlan smem_plan() {
   return s;
 }
 
-__device__ __forceinline__ float4 lds128(const char* p) { return *reinterpret_cast<const float4*>(p); }
-
 // 16-byte shared-memory access by 32-bit shared-space address (+ immediate byte offset).  Volatile: a ring
 // slot is refilled by the TMA engine between two reads of the same address, which the compiler cannot see.
 template <int IMM>
@@ -162,11 +162,9 @@ __device__ __forceinline__ void sts128_s(uint32_t addr, float a, float b, float 
                : "memory");
 }
 
-// fp32 -> (hi, lo) TF32 pair with hi + lo = v to ~2^-22 relative (error-compensated "3xTF32")
-__device__ __forceinline__ void split_tf32(float v, uint32_t& hi, uint32_t& lo) {
-  hi = __float_as_uint(v) & 0xffffe000u;
-  lo = __float_as_uint(v - __uint_as_float(hi));
-}
+// fp32 -> (hi, lo) TF32 pair for the error-compensated product hi*hi + lo*hi + hi*lo: the truncating split
+// (two instructions) for operands split in the inner loop, the rounding one for the basis tables built once
+__device__ __forceinline__ void split_tf32(float v, uint32_t& hi, uint32_t& lo) { split_tf32_trunc(v, hi, lo); }
 
 // D += A(16x8, row) * B(8x8, col), TF32 inputs, fp32 accumulate
 __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
@@ -304,7 +302,7 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
       double sn, cs;
       sincospi((double)(((long long)g * (2 * n + 1)) % (2 * N2)) / (double)N2, &sn, &cs);
       const float v = valid ? ((cls == 2 || cls == 3) ? (float)sn : (float)cs) : 0.f;
-      split_tf32(v, hi[h], lo[h]);
+      split_tf32_rna(v, hi[h], lo[h]);
     }
     btab[e] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(lo[0]), __uint_as_float(lo[1]));
   }
@@ -663,7 +661,7 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __re
         double sn, cs;
         sincospi((double)(((long long)g * (2 * n + 1)) % (2 * N2)) / (double)N2, &sn, &cs);
         const float v = valid ? ((cls == 2 || cls == 3) ? (float)sn : (float)cs) : 0.f;
-        split_tf32(v, ahi[cls][mt][e], alo[cls][mt][e]);
+        split_tf32_rna(v, ahi[cls][mt][e], alo[cls][mt][e]);
       }
 
   // loader role: lane = (plane, mode position r)
