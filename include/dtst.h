@@ -167,6 +167,34 @@ dtst_status dtst_backward(dtst_plan* plan, const float* grad_y, const void* Xhat
                           const void* W, float* grad_x, void* grad_W, void* stream);
 
 /*
+ * The same steps one by one, for a caller that runs the layer across several ranks (Algorithm 1: each
+ * rank owns a slab of the grid and an equal, contiguous share S_p of the flattened modes, Eq. 12) and
+ * exchanges spectra between the steps with its own collectives:
+ *   forward:  dtst_forward on the slab (plan from dtst_plan_create_local)  -> partial spectrum
+ *             all-reduce(sum) over ranks (Eq. 7)                           -> Xhat, full [B, C_in, M]
+ *             dtst_spectral_mul_modes on [m0, m0 + count)                  -> Yhat chunk [B, C_out, count]
+ *             all-gather of the chunks                                     -> Yhat, full
+ *             dtst_inverse on the slab                                     -> y on the slab
+ *   backward: dtst_backward_spectrum (partial G_Y), all-reduce, dtst_backward_mix_modes on the rank's
+ *             modes (grad_W shard stays local: no all-reduce of weight gradients), all-gather of the
+ *             G_X chunks, dtst_backward_input on the slab.
+ * Layouts: full spectra [B, C, M]; W_shard, grad_W_shard [C_in, C_out, count]; chunks [B, C, count];
+ * all complex64, device, 16-byte aligned.  0 <= m0, count >= 1, m0 + count <= M, else
+ * DTST_ERR_INVALID_ARG.  Outputs are assigned.  dtst_backward_mix_modes: GX_chunk or grad_W_shard may be
+ * NULL to skip it (not both); Xhat_saved is only read for grad_W_shard.
+ */
+dtst_status dtst_spectral_mul_modes(dtst_plan* plan, const void* Xhat, const void* W_shard,
+                                    void* Yhat_chunk, int64_t m0, int64_t count, void* stream);
+/* G_Y = (c / prod N_global) * F(grad_y) of this plan's block: [B, C_out, M] (the adjoint of dtst_inverse). */
+dtst_status dtst_backward_spectrum(dtst_plan* plan, const float* grad_y, void* GY, void* stream);
+dtst_status dtst_backward_mix_modes(dtst_plan* plan, const void* GY, const void* Xhat_saved,
+                                    const void* W_shard, void* GX_chunk, void* grad_W_shard,
+                                    int64_t m0, int64_t count, void* stream);
+/* grad_x = Re sum_m G_X[m] e^{+i theta_m n} on this plan's block: no doubling, no 1 / prod N
+ * (the adjoint of dtst_forward).  GX [B, C_in, M]. */
+dtst_status dtst_backward_input(dtst_plan* plan, const void* GX, float* grad_x, void* stream);
+
+/*
  * The forward partial DFT without any caller-provided or allocated scratch.
  * (The paper has no counterpart to this call; it exists for integration reasons.)
  *

@@ -37,7 +37,8 @@ EXPORTED = [
     "dtst_plan_set_workspace", "dtst_forward", "dtst_spectral_mul", "dtst_inverse",
     "dtst_backward", "dtst_plan_status", "dtst_plan_launch_count", "dtst_status_string",
     "dtst_version", "dtst_plan_enable_kernel_timing", "dtst_plan_kernel_timing", "dtst_forward_static",
-    "dtst_plan_last_cuda_error",
+    "dtst_plan_last_cuda_error", "dtst_spectral_mul_modes", "dtst_backward_spectrum", "dtst_backward_mix_modes",
+    "dtst_backward_input",
 ]
 
 
@@ -76,6 +77,10 @@ def lib() -> ctypes.CDLL:
     L.dtst_spectral_mul.argtypes = [vp, vp, vp, vp, vp]
     L.dtst_inverse.argtypes = [vp, vp, vp, vp]
     L.dtst_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.dtst_spectral_mul_modes.argtypes = [vp, vp, vp, vp, ctypes.c_int64, ctypes.c_int64, vp]
+    L.dtst_backward_spectrum.argtypes = [vp, vp, vp, vp]
+    L.dtst_backward_mix_modes.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_int64, ctypes.c_int64, vp]
+    L.dtst_backward_input.argtypes = [vp, vp, vp, vp]
     L.dtst_plan_status.argtypes = [vp, vp]
     L.dtst_plan_launch_count.argtypes = [vp, i64p]
     L.dtst_plan_enable_kernel_timing.argtypes = [vp, i32]
@@ -225,6 +230,32 @@ def dtst_backward(plan, grad_y, Xhat_saved, W, grad_x, grad_W, stream=None) -> N
                                _stream_ptr(stream)), "dtst_backward", plan)
 
 
+def dtst_spectral_mul_modes(plan, Xhat, W_shard, Yhat_chunk, m0, count, stream=None) -> None:
+    _check(lib().dtst_spectral_mul_modes(plan, _ptr(Xhat, torch.complex64, "Xhat"),
+                                         _ptr(W_shard, torch.complex64, "W_shard"),
+                                         _ptr(Yhat_chunk, torch.complex64, "Yhat_chunk"), int(m0), int(count),
+                                         _stream_ptr(stream)), "dtst_spectral_mul_modes", plan)
+
+
+def dtst_backward_spectrum(plan, grad_y, GY, stream=None) -> None:
+    _check(lib().dtst_backward_spectrum(plan, _ptr(grad_y, torch.float32, "grad_y"), _ptr(GY, torch.complex64, "GY"),
+                                        _stream_ptr(stream)), "dtst_backward_spectrum", plan)
+
+
+def dtst_backward_mix_modes(plan, GY, Xhat_saved, W_shard, GX_chunk, grad_W_shard, m0, count, stream=None) -> None:
+    _check(lib().dtst_backward_mix_modes(plan, _ptr(GY, torch.complex64, "GY"),
+                                         _ptr(Xhat_saved, torch.complex64, "Xhat_saved"),
+                                         _ptr(W_shard, torch.complex64, "W_shard"),
+                                         _ptr(GX_chunk, torch.complex64, "GX_chunk"),
+                                         _ptr(grad_W_shard, torch.complex64, "grad_W_shard"), int(m0), int(count),
+                                         _stream_ptr(stream)), "dtst_backward_mix_modes", plan)
+
+
+def dtst_backward_input(plan, GX, grad_x, stream=None) -> None:
+    _check(lib().dtst_backward_input(plan, _ptr(GX, torch.complex64, "GX"), _ptr(grad_x, torch.float32, "grad_x"),
+                                     _stream_ptr(stream)), "dtst_backward_input", plan)
+
+
 def dtst_plan_status(plan, stream=None) -> int:
     return int(lib().dtst_plan_status(plan, _stream_ptr(stream)))
 
@@ -348,6 +379,33 @@ class Plan:
             grad_W = torch.empty((self.C_in, self.C_out, self.M), dtype=torch.complex64, device=self.device)
         dtst_backward(self._h, grad_y, Xhat_saved, W, grad_x, grad_W, stream)
         return grad_x, grad_W
+
+    # -- the steps one by one (a rank of a slab-sharded layer exchanges spectra between them)
+    def spectral_mul_modes(self, Xhat, W_shard, m0, count, out=None, stream=None):
+        if out is None:
+            out = torch.empty((self.B, self.C_out, count), dtype=torch.complex64, device=self.device)
+        dtst_spectral_mul_modes(self._h, Xhat, W_shard, out, m0, count, stream)
+        return out
+
+    def backward_spectrum(self, grad_y, out=None, stream=None):
+        if out is None:
+            out = torch.empty((self.B, self.C_out) + self.K, dtype=torch.complex64, device=self.device)
+        dtst_backward_spectrum(self._h, grad_y, out, stream)
+        return out
+
+    def backward_mix_modes(self, GY, Xhat_saved, W_shard, m0, count, GX_chunk=None, grad_W_shard=None, stream=None):
+        if GX_chunk is None:
+            GX_chunk = torch.empty((self.B, self.C_in, count), dtype=torch.complex64, device=self.device)
+        if grad_W_shard is None:
+            grad_W_shard = torch.empty((self.C_in, self.C_out, count), dtype=torch.complex64, device=self.device)
+        dtst_backward_mix_modes(self._h, GY, Xhat_saved, W_shard, GX_chunk, grad_W_shard, m0, count, stream)
+        return GX_chunk, grad_W_shard
+
+    def backward_input(self, GX, out=None, stream=None):
+        if out is None:
+            out = torch.empty((self.B, self.C_in) + self.N, dtype=torch.float32, device=self.device)
+        dtst_backward_input(self._h, GX, out, stream)
+        return out
 
     def layer(self, x, W, Xhat=None, Yhat=None, y=None, stream=None):
         """y = I(M(F(x), W)); returns (y, Xhat)."""

@@ -627,6 +627,64 @@ dtst_status dtst_backward(dtst_plan* p, const float* grad_y, const void* Xhat_sa
   return DTST_OK;
 }
 
+// ---- the steps of the layer one by one, for a caller that exchanges spectra between ranks in between them
+dtst_status dtst_spectral_mul_modes(dtst_plan* p, const void* Xhat, const void* W_shard, void* Yhat_chunk,
+                                    int64_t m0, int64_t count, void* stream) {
+  if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  if (Xhat == nullptr || W_shard == nullptr || Yhat_chunk == nullptr || !aligned16(Xhat) || !aligned16(W_shard) ||
+      !aligned16(Yhat_chunk) || Yhat_chunk == Xhat || Yhat_chunk == W_shard)
+    return DTST_ERR_INVALID_ARG;
+  if (m0 < 0 || count < 1 || m0 + count > p->M) return DTST_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cuda_failed(p, launch_mix_modes(static_cast<const float2*>(Xhat), static_cast<const float2*>(W_shard),
+                                      static_cast<float2*>(Yhat_chunk), p->B, p->C_in, p->C_out, p->M, m0, count, st,
+                                      &p->launches)))
+    return DTST_ERR_CUDA;
+  return DTST_OK;
+}
+
+dtst_status dtst_backward_spectrum(dtst_plan* p, const float* grad_y, void* GY, void* stream) {
+  dtst_status s = check_ready(p);
+  if (s != DTST_OK) return s;
+  if (grad_y == nullptr || GY == nullptr || !aligned16(grad_y) || !aligned16(GY)) return DTST_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const float scale = (float)(1.0 / (double)p->points_global);
+  float2* out = static_cast<float2*>(GY);
+  return use_fused(p) ? run_forward_fused(p, grad_y, out, p->C_out, scale, true, st)
+         : use_row(p) ? run_forward_row(p, grad_y, out, p->C_out, scale, true, st)
+                      : run_forward_generic(p, grad_y, out, p->C_out, scale, true, st);
+}
+
+dtst_status dtst_backward_mix_modes(dtst_plan* p, const void* GY, const void* Xhat_saved, const void* W_shard,
+                                    void* GX_chunk, void* grad_W_shard, int64_t m0, int64_t count, void* stream) {
+  if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  if (GY == nullptr || W_shard == nullptr || (GX_chunk == nullptr && grad_W_shard == nullptr) ||
+      (grad_W_shard != nullptr && Xhat_saved == nullptr))
+    return DTST_ERR_INVALID_ARG;
+  if (!aligned16(GY) || !aligned16(Xhat_saved) || !aligned16(W_shard) || !aligned16(GX_chunk) ||
+      !aligned16(grad_W_shard))
+    return DTST_ERR_INVALID_ARG;
+  if (m0 < 0 || count < 1 || m0 + count > p->M) return DTST_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cuda_failed(p, launch_mix_adjoint_modes(static_cast<const float2*>(GY), static_cast<const float2*>(Xhat_saved),
+                                              static_cast<const float2*>(W_shard), static_cast<float2*>(GX_chunk),
+                                              static_cast<float2*>(grad_W_shard), p->B, p->C_in, p->C_out, p->M, m0,
+                                              count, st, &p->launches)))
+    return DTST_ERR_CUDA;
+  return DTST_OK;
+}
+
+dtst_status dtst_backward_input(dtst_plan* p, const void* GX, float* grad_x, void* stream) {
+  dtst_status s = check_ready(p);
+  if (s != DTST_OK) return s;
+  if (GX == nullptr || grad_x == nullptr || !aligned16(GX) || !aligned16(grad_x)) return DTST_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const float2* in = static_cast<const float2*>(GX);
+  return use_fused(p) ? run_inverse_fused(p, in, grad_x, p->C_in, 1.0f, false, st)
+         : use_row(p) ? run_inverse_row(p, in, grad_x, p->C_in, 1.0f, false, st)
+                      : run_inverse_generic(p, in, grad_x, p->C_in, 1.0f, false, st);
+}
+
 dtst_status dtst_plan_status(dtst_plan* p, void* stream) {
   if (p == nullptr) return DTST_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -133,6 +133,11 @@ cudaError_t launch_apply_dim(const DimOp& op, bool in_real, bool out_real, const
 cudaError_t launch_reduce_partials(const float2* partial, float2* out, long long n, int P, cudaStream_t st);
 cudaError_t launch_mix(const float2* X, const float2* W, float2* Y, int B, int Ci, int Co, long long M,
                        cudaStream_t st, long long* launches);
+cudaError_t launch_mix_modes(const float2* X, const float2* W, float2* Y, int B, int Ci, int Co, long long M,
+                             long long m0, long long cnt, cudaStream_t st, long long* launches);
+cudaError_t launch_mix_adjoint_modes(const float2* GY, const float2* X, const float2* W, float2* GX, float2* GW,
+                                     int B, int Ci, int Co, long long M, long long m0, long long cnt,
+                                     cudaStream_t st, long long* launches);
 cudaError_t launch_mix_adjoint(const float2* GY, const float2* X, const float2* W, float2* GX, float2* GW,
                                int B, int Ci, int Co, long long M, cudaStream_t st, long long* launches);
 

@@ -259,4 +259,95 @@ cudaError_t launch_mix_adjoint(const float2* GY, const float2* X, const float2* 
   return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------------
+// Mixing on a contiguous chunk [m0, m0 + cnt) of the flattened modes: the equal partition of the
+// modes among ranks (Eq. 12 applied by rank p to its S_p).  The spectra are the full tensors
+// [B][C][M] every rank holds after the reduction; the weight tensors are the rank's shards
+// [C_in][C_out][cnt]; outputs are contiguous chunks [B][C][cnt], ready to be gathered.
+// Not on the single-GPU hot path: plain one-thread-per-output kernels.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) mix_modes_kernel(const float2* __restrict__ X, const float2* __restrict__ W,
+                                                       float2* __restrict__ Y, int Ci, int Co, long long M,
+                                                       long long m0, long long cnt) {
+  const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int o = blockIdx.y, b = blockIdx.z;
+  if (m >= cnt) return;
+  float2 acc = make_float2(0.f, 0.f);
+  for (int i = 0; i < Ci; ++i) {
+    const float2 w = __ldg(W + ((long long)i * Co + o) * cnt + m);
+    const float2 x = __ldg(X + ((long long)b * Ci + i) * M + m0 + m);
+    acc.x = fmaf(x.x, w.x, acc.x);
+    acc.x = fmaf(-x.y, w.y, acc.x);
+    acc.y = fmaf(x.x, w.y, acc.y);
+    acc.y = fmaf(x.y, w.x, acc.y);
+  }
+  Y[((long long)b * Co + o) * cnt + m] = acc;
+}
+
+// G_X[b][i][m] = sum_o G_Y[b][o][m0 + m] conj(W[i][o][m])
+__global__ void __launch_bounds__(256) mix_adjoint_gx_modes_kernel(const float2* __restrict__ GY,
+                                                                  const float2* __restrict__ W,
+                                                                  float2* __restrict__ GX, int Ci, int Co,
+                                                                  long long M, long long m0, long long cnt) {
+  const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int i = blockIdx.y, b = blockIdx.z;
+  if (m >= cnt) return;
+  float2 acc = make_float2(0.f, 0.f);
+  for (int o = 0; o < Co; ++o) {
+    const float2 w = __ldg(W + ((long long)i * Co + o) * cnt + m);
+    const float2 g = __ldg(GY + ((long long)b * Co + o) * M + m0 + m);
+    acc.x = fmaf(g.x, w.x, acc.x);
+    acc.x = fmaf(g.y, w.y, acc.x);
+    acc.y = fmaf(g.y, w.x, acc.y);
+    acc.y = fmaf(-g.x, w.y, acc.y);
+  }
+  GX[((long long)b * Ci + i) * cnt + m] = acc;
+}
+
+// G_W[i][o][m] = sum_b conj(X[b][i][m0 + m]) G_Y[b][o][m0 + m]
+__global__ void __launch_bounds__(256) mix_adjoint_gw_modes_kernel(const float2* __restrict__ GY,
+                                                                  const float2* __restrict__ X,
+                                                                  float2* __restrict__ GW, int B, int Ci, int Co,
+                                                                  long long M, long long m0, long long cnt) {
+  const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int o = blockIdx.y, i = blockIdx.z;
+  if (m >= cnt) return;
+  float2 acc = make_float2(0.f, 0.f);
+  for (int b = 0; b < B; ++b) {
+    const float2 x = __ldg(X + ((long long)b * Ci + i) * M + m0 + m);
+    const float2 g = __ldg(GY + ((long long)b * Co + o) * M + m0 + m);
+    acc.x = fmaf(x.x, g.x, acc.x);
+    acc.x = fmaf(x.y, g.y, acc.x);
+    acc.y = fmaf(x.x, g.y, acc.y);
+    acc.y = fmaf(-x.y, g.x, acc.y);
+  }
+  GW[((long long)i * Co + o) * cnt + m] = acc;
+}
+
+cudaError_t launch_mix_modes(const float2* X, const float2* W, float2* Y, int B, int Ci, int Co, long long M,
+                             long long m0, long long cnt, cudaStream_t st, long long* launches) {
+  if (cnt <= 0 || B <= 0) return cudaSuccess;
+  dim3 grid((unsigned)((cnt + 255) / 256), (unsigned)Co, (unsigned)B);
+  mix_modes_kernel<<<grid, 256, 0, st>>>(X, W, Y, Ci, Co, M, m0, cnt);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_mix_adjoint_modes(const float2* GY, const float2* X, const float2* W, float2* GX, float2* GW,
+                                     int B, int Ci, int Co, long long M, long long m0, long long cnt,
+                                     cudaStream_t st, long long* launches) {
+  if (cnt <= 0 || B <= 0) return cudaSuccess;
+  if (GX != nullptr) {
+    dim3 grid((unsigned)((cnt + 255) / 256), (unsigned)Ci, (unsigned)B);
+    mix_adjoint_gx_modes_kernel<<<grid, 256, 0, st>>>(GY, W, GX, Ci, Co, M, m0, cnt);
+    if (launches) ++*launches;
+  }
+  if (GW != nullptr) {
+    dim3 grid((unsigned)((cnt + 255) / 256), (unsigned)Co, (unsigned)Ci);
+    mix_adjoint_gw_modes_kernel<<<grid, 256, 0, st>>>(GY, X, GW, B, Ci, Co, M, m0, cnt);
+    if (launches) ++*launches;
+  }
+  return cudaGetLastError();
+}
+
 }  // namespace dtst
