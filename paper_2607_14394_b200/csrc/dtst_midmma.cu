@@ -472,7 +472,12 @@ cudaError_t launch_mid_mma_t(bool forward, const float2* in, float2* out, long l
 bool mid_mma_supported(int N, int K, long long inner) {
   if (N % 32 != 0 || N < 32 || N > 512 || 2 * K > N) return false;
   if (!(K == 4 || K == 8 || K == 12 || K == 16)) return false;
-  return inner > 0 && inner % 4 == 0;
+  if (inner <= 0 || inner % 4 != 0) return false;
+  // both kernels must fit the 227 KB of shared memory a CTA can opt into
+  const size_t lim = 227 * 1024;
+  const size_t c = contract_smem<16>(N);
+  const size_t e = K == 4 ? expand_smem<4>(N) : K == 8 ? expand_smem<8>(N) : K == 12 ? expand_smem<12>(N) : expand_smem<16>(N);
+  return c <= lim && e <= lim;
 }
 
 cudaError_t launch_mid_mma(bool forward, int K, const float2* in, float2* out, long long outer, long long inner,
