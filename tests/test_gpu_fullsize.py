@@ -132,3 +132,51 @@ def test_cfg5_4d_128_fullsize():
 def test_cfg4_3d_256_fullsize():
     w = I.WORKLOADS["cfg4_3d_256"]
     _check_layer_fullsize(w, P_list=[4], check_channels=[1, 30], rng_seed=44)
+
+
+@pytest.mark.parametrize("name", ["cfg5_4d_128", "cfg4_3d_256"])
+def test_fullsize_properties_that_hold_at_any_size(name):
+    """At the benchmark's full sizes, in its launch configuration, on every channel at once (no oracle needed):
+    the adjoint identity <F x, Y> = <x, F^H Y> with F^H = dtst_backward_input, the pair
+    <I Y, g> = <Y, G_Y(g)> with G_Y = dtst_backward_spectrum, and linearity of F."""
+    from paper_2607_14394_b200 import Plan
+    w = I.WORKLOADS[name]
+    dev = torch.device("cuda")
+    plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out)
+    gen = torch.Generator(device=dev).manual_seed(2024)
+    x = torch.randn((w.B, w.C_in) + w.N, device=dev, generator=gen)
+    Y = torch.randn((w.B, w.C_in) + w.K, dtype=torch.complex64, device=dev, generator=gen)
+
+    def cdot(a, b):   # Re <a, b> over complex tensors, accumulated in float64
+        return float((torch.view_as_real(a).double() * torch.view_as_real(b).double()).sum().item())
+
+    def rdot(a, b):
+        return float(torch.dot(a.reshape(-1).double(), b.reshape(-1).double()).item()) if a.numel() < 2 ** 31 else \
+            float(sum(torch.dot(a[:, c].reshape(-1).double(), b[:, c].reshape(-1).double()).item()
+                      for c in range(a.shape[1])))
+
+    Fx = plan.forward(x)
+    FhY = plan.backward_input(Y)                       # F^H Y on the grid (needs C_in channels)
+    lhs, rhs = cdot(Fx, Y), rdot(x, FhY)
+    assert abs(lhs - rhs) <= 2e-5 * max(abs(lhs), float(torch.view_as_real(Fx).double().norm() *
+                                                      torch.view_as_real(Y).double().norm()) * 1e-2)
+    del FhY
+    torch.cuda.empty_cache()
+
+    # linearity: F(2 x) = 2 F(x) bit for bit (a power of two scales exactly through every fp32 operation)
+    x.mul_(2.0)
+    F2 = plan.forward(x)
+    assert torch.equal(torch.view_as_real(F2), 2.0 * torch.view_as_real(Fx))
+    del F2, Fx
+    torch.cuda.empty_cache()
+
+    if w.C_in == w.C_out:
+        g = x                                           # any real field serves as the upstream gradient
+        y = plan.inverse(Y)
+        GY = plan.backward_spectrum(g)
+        lhs, rhs = rdot(y, g), cdot(Y, GY)
+        scale = float(y.double().norm() * g.double().norm())
+        assert abs(lhs - rhs) <= 2e-5 * max(abs(lhs), 1e-2 * scale)
+    torch.cuda.synchronize()
+    assert plan.status() == 0
+    plan.close()
