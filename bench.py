@@ -485,16 +485,39 @@ def main_ours(args, w):
     if args.no_e2e:
         e2e = {"value": None, "unit": UNIT, "skipped": "--no-e2e"}
     elif rank == 0 or world > 1:
+        # Every rank pins five host buffers (43 GB at this workload); all ranks of the node must get theirs, and
+        # they decide TOGETHER whether to run, so that no rank waits at a barrier for one that gave up.
+        hx = hg = hy = hgx = hgW = None
+        pinned_ok = 1.0
+        try:
+            need = 4 * (x.numel() + g.numel() + y.numel() + gx.numel()) + 8 * gW.numel()
+            try:
+                import psutil
+                if need * world > 0.7 * psutil.virtual_memory().available:
+                    pinned_ok = 0.0
+            except ImportError:
+                pass
+            if pinned_ok:
+                hx = torch.empty(x.shape, dtype=torch.float32, pin_memory=True)
+                hg = torch.empty(g.shape, dtype=torch.float32, pin_memory=True)
+                hy = torch.empty(y.shape, dtype=torch.float32, pin_memory=True)
+                hgx = torch.empty(gx.shape, dtype=torch.float32, pin_memory=True)
+                hgW = torch.empty(gW.shape, dtype=torch.complex64, pin_memory=True)
+        except Exception:
+            pinned_ok = 0.0
+        if world > 1:
+            flag = torch.tensor([pinned_ok], device=dev)
+            dist.all_reduce(flag, op=dist.ReduceOp.MIN)
+            pinned_ok = float(flag.item())
+        if not pinned_ok:
+            hx = hg = hy = hgx = hgW = None
+            e2e = {"value": None, "unit": UNIT, "skipped": "pinned host buffers for every rank did not fit host memory"}
+    if e2e is None and (rank == 0 or world > 1):
         try:
             e2e_steps = max(1, min(steps, args.e2e_steps))
             from paper_2607_14394_b200.binding import HostPipeline
-            hx = torch.empty(x.shape, dtype=torch.float32, pin_memory=True)
-            hg = torch.empty(g.shape, dtype=torch.float32, pin_memory=True)
             hx.copy_(x)
             hg.copy_(g)
-            hy = torch.empty(y.shape, dtype=torch.float32, pin_memory=True)
-            hgx = torch.empty(gx.shape, dtype=torch.float32, pin_memory=True)
-            hgW = torch.empty(gW.shape, dtype=torch.complex64, pin_memory=True)
             del x, g, y, gx, gW
             torch.cuda.empty_cache()
             pipe = HostPipeline(plan, W)
