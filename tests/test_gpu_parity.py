@@ -109,6 +109,41 @@ def test_edge_shapes(case, path):
     run_layer_and_check(I.custom_workload(name, B, Ci, Co, N, k, seed=11), path)
 
 
+# ------------------------------------------------------------------ a seeded sweep of shapes nobody picked by hand
+def _random_cases(count, seed):
+    """Seeded draw of (B, C_in, C_out, N, kmax, P): d = 1..4, extents that mix multiples of 32 / 16 / 4 with odd
+    numbers where the ABI allows them, retained counts from 1 up to the full band, a virtual-shard count that
+    divides N_0.  Sizes stay small enough for the oracle to take a fraction of a second each."""
+    rng = np.random.default_rng(seed)
+    last_choices = [4, 8, 12, 20, 32, 36, 64, 96, 128]          # the contiguous extent must be a multiple of 4
+    mid_choices = [3, 4, 5, 6, 8, 9, 12, 16, 24, 32, 33, 64]
+    cases = []
+    while len(cases) < count:
+        d = int(rng.integers(1, 5))
+        N = [int(rng.choice(mid_choices)) for _ in range(d - 1)] + [int(rng.choice(last_choices))]
+        if np.prod(N) > 300_000:
+            continue
+        k = []
+        for j, n in enumerate(N):
+            hi = n // 2 if j < d - 1 else n // 2 + 1
+            k.append(int(rng.integers(1, max(1, min(hi, 16)) + 1)))
+        B, Ci, Co = int(rng.integers(1, 4)), int(rng.integers(1, 5)), int(rng.integers(1, 5))
+        divs = [p for p in (1, 2, 3, 4, 8) if N[0] % p == 0]
+        P = int(rng.choice(divs))
+        cases.append((B, Ci, Co, tuple(N), tuple(k), P))
+    return cases
+
+
+RANDOM_CASES = _random_cases(28, seed=20260714)
+
+
+@pytest.mark.parametrize("case", RANDOM_CASES, ids=[f"r{i}_" + "x".join(map(str, c[3])) for i, c in enumerate(RANDOM_CASES)])
+def test_random_shapes(case):
+    B, Ci, Co, N, k, P = case
+    w = I.custom_workload("random", B, Ci, Co, N, k, field="grf" if len(N) > 1 else "iid", seed=sum(N) + 7 * P)
+    run_layer_and_check(w, "auto", P=P)
+
+
 # ------------------------------------------------------------------ virtual shards (Eq. 6-7 on one GPU)
 @pytest.mark.parametrize("N,k,P", [((16, 8, 12), (3, 2, 4), 4), ((16, 8, 12), (3, 2, 4), 16),
                                    ((64, 64), (8, 8), 8), ((8,), (3,), 2),
