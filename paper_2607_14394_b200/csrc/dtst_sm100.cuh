@@ -73,11 +73,15 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       : "memory");
 }
 
-// 2-D tiled TMA store shared -> global (bulk async group).
+// 2-D tiled TMA store shared -> global (bulk async group).  The output is written once and not read again by
+// this kernel: an evict-first L2 policy lets the write-back stream drain sooner (measured: 1.5 % on the
+// inverse plane kernel; the same hint on the forward kernel's loads costs 1 %).
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, const void* smem_src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%1, %2}], [%3], %4;" ::"l"(
                    reinterpret_cast<uint64_t>(map)),
-               "r"(x), "r"(y), "r"(smem_u32(smem_src))
+               "r"(x), "r"(y), "r"(smem_u32(smem_src)), "l"(pol)
                : "memory");
 }
 
