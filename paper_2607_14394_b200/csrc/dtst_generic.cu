@@ -133,7 +133,7 @@ __global__ void __launch_bounds__(256) mix_kernel(const float2* __restrict__ X, 
 #pragma unroll
   for (int b = 0; b < NB; ++b) acc[b] = make_float2(0.f, 0.f);
   for (int i = 0; i < Ci; ++i) {
-    const float2 w = __ldg(W + ((long long)i * Co + o) * M + m);
+    const float2 w = __ldcs(W + ((long long)i * Co + o) * M + m);   // streamed once: do not displace the spectra in L2
 #pragma unroll
     for (int b = 0; b < NB; ++b) {
       const float2 x = __ldg(X + ((long long)(b0 + b) * Ci + i) * M + m);
@@ -185,7 +185,7 @@ __global__ void __launch_bounds__(256) mix_adjoint_kernel(const float2* __restri
     xr[b] = (WANT_GW && ALLB) ? __ldg(X + ((long long)(b0 + b) * Ci + i) * M + m) : make_float2(0.f, 0.f);
   }
   for (int o = 0; o < Co; ++o) {
-    const float2 w = __ldg(W + ((long long)i * Co + o) * M + m);
+    const float2 w = __ldcs(W + ((long long)i * Co + o) * M + m);   // streamed once: do not displace the spectra in L2
     float2 g[NB];
 #pragma unroll
     for (int b = 0; b < NB; ++b) g[b] = __ldg(GY + ((long long)(b0 + b) * Co + o) * M + m);
@@ -218,7 +218,7 @@ __global__ void __launch_bounds__(256) mix_adjoint_kernel(const float2* __restri
           acc.y = fmaf(-xx.y, gg.x, acc.y);
         }
       }
-      GW[((long long)i * Co + o) * M + m] = acc;
+      __stcs(GW + ((long long)i * Co + o) * M + m, acc);
     }
   }
   if (WANT_GX) {
