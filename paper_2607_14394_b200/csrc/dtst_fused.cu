@@ -674,7 +674,7 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __re
   if (task < num_tasks && actl) {
     const float4* src = reinterpret_cast<const float4*>(in + ((task * G + pll) * (2 * K2) + rl) * K3);
 #pragma unroll
-    for (int i = 0; i < K3 / 2; ++i) vin[i] = __ldg(src + i);
+    for (int i = 0; i < K3 / 2; ++i) vin[i] = __ldcs(src + i);
   }
 
   for (; task < num_tasks; task += tstride) {
@@ -709,7 +709,7 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __re
       if (nt < num_tasks && actl) {
         const float4* src = reinterpret_cast<const float4*>(in + ((nt * G + pll) * (2 * K2) + rl) * K3);
 #pragma unroll
-        for (int i = 0; i < K3 / 2; ++i) vin[i] = __ldg(src + i);
+        for (int i = 0; i < K3 / 2; ++i) vin[i] = __ldcs(src + i);
       }
     }
     __syncwarp();

@@ -267,7 +267,7 @@ struct ExpCfg {
 template <int K>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 mid_expand_mma_kernel(const float2* __restrict__ in, float* __restrict__ out, long long outer, long long inner,
-                      int N, float scale) {
+                      int N, float scale, int streaming) {
   using EC = ExpCfg<K>;
   constexpr int KS = EC::KS;
   extern __shared__ float4 mm_smem[];
@@ -332,8 +332,8 @@ mid_expand_mma_kernel(const float2* __restrict__ in, float* __restrict__ out, lo
       for (int g = 0; g <= K; ++g) {
         const float2 r = rho[g];
         float2 v = make_float2(0.f, 0.f), u = make_float2(0.f, 0.f);
-        if (ok && g < K) v = __ldg(src + (long long)g * inner);
-        if (ok && g > 0) u = __ldg(src + (long long)(2 * K - g) * inner);
+        if (ok && g < K) v = __ldcs(src + (long long)g * inner);
+        if (ok && g > 0) u = __ldcs(src + (long long)(2 * K - g) * inner);
         const float2 vp = make_float2(v.x * r.x + v.y * r.y, v.y * r.x - v.x * r.y);   // v * conj(rho)
         const float2 vm = make_float2(u.x * r.x - u.y * r.y, u.y * r.x + u.x * r.y);   // u * rho
         const int arow = g < K ? g : 8 * KS;
@@ -407,10 +407,19 @@ mid_expand_mma_kernel(const float2* __restrict__ in, float* __restrict__ out, lo
             P[1] = fmaf(aK.y, c0, P[1]);
             P[2] = fmaf(aK.x, c1, P[2]);
             P[3] = fmaf(aK.y, c1, P[3]);
-            *reinterpret_cast<float2*>(da + 8 * nt) = make_float2(P[0] + Q[0], P[1] + Q[1]);
-            *reinterpret_cast<float2*>(db + 8 * nt) = make_float2(P[2] + Q[2], P[3] + Q[3]);
-            *reinterpret_cast<float2*>(dc + 8 * nt) = make_float2(P[0] - Q[0], P[1] - Q[1]);
-            *reinterpret_cast<float2*>(dd + 8 * nt) = make_float2(P[2] - Q[2], P[3] - Q[3]);
+            const float2 va = make_float2(P[0] + Q[0], P[1] + Q[1]), vb = make_float2(P[2] + Q[2], P[3] + Q[3]);
+            const float2 vc = make_float2(P[0] - Q[0], P[1] - Q[1]), vd = make_float2(P[2] - Q[2], P[3] - Q[3]);
+            if (streaming) {   // an output far larger than L2 is not worth keeping there for the next kernel
+              __stcs(reinterpret_cast<float2*>(da + 8 * nt), va);
+              __stcs(reinterpret_cast<float2*>(db + 8 * nt), vb);
+              __stcs(reinterpret_cast<float2*>(dc + 8 * nt), vc);
+              __stcs(reinterpret_cast<float2*>(dd + 8 * nt), vd);
+            } else {
+              *reinterpret_cast<float2*>(da + 8 * nt) = va;
+              *reinterpret_cast<float2*>(db + 8 * nt) = vb;
+              *reinterpret_cast<float2*>(dc + 8 * nt) = vc;
+              *reinterpret_cast<float2*>(dd + 8 * nt) = vd;
+            }
           }
         }
       }
@@ -462,7 +471,8 @@ cudaError_t launch_mid_mma_t(bool forward, const float2* in, float2* out, long l
     auto kern = mid_expand_mma_kernel<K>;
     cudaError_t e = grid_for(kern, &grid);
     if (e != cudaSuccess) return e;
-    kern<<<grid, threads, smem, st>>>(in, reinterpret_cast<float*>(out), outer, inner, N, scale);
+    const int streaming = (double)outer * N * inner * 8.0 > 2.0 * 126e6 ? 1 : 0;
+    kern<<<grid, threads, smem, st>>>(in, reinterpret_cast<float*>(out), outer, inner, N, scale, streaming);
   }
   return cudaGetLastError();
 }
