@@ -23,10 +23,6 @@ constexpr int kMmaWarps = 12;   // one persistent CTA per SM: the basis tables a
 constexpr int kMmaThreads = kMmaWarps * 32;
 constexpr int kNT = 8;              // expansion: MMA n-tiles per task: 64 real columns = 32 complex positions
 constexpr int kTaskPos = 4 * kNT;   // complex positions per task
-constexpr int kCNT = 4;             // contraction: 4 n-tiles per task (one 128-byte line per row), more warps
-constexpr int kCPos = 4 * kCNT;
-constexpr int kCWarps = 16;
-constexpr int kCThreads = kCWarps * 32;
 
 __device__ __forceinline__ float4 as_f4(const uint32_t (&v)[4]) {
   return make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
@@ -48,16 +44,31 @@ __device__ __forceinline__ void basis_cs(int g, int q, int N, float& cs, float& 
 
 // ------------------------------------------------------------------------------------------
 // contraction: in[outer][N][inner] -> out[outer][2K][inner]
-//   MMA roles: M = frequency slot (basis = A operand, from a fragment-ordered shared table),
-//              K = mirrored row pair q, N = real column (data = B operand, straight from global memory).
+//
+// Second fold: psi_g (N/2-1-q + 1/2) = pi g - psi_g (q + 1/2), so the cosine is even (odd) and the sine odd (even)
+// about the quarter points for even (odd) g.  The four rows a = z_q, b = z_{N/2-1-q}, c = z_{N/2+q}, d = z_{N-1-q}
+// (q < N/4) fold into
+//     uu = (a+d)+(b+c) -> A_g, g even      ud = (a+d)-(b+c) -> A_g, g odd
+//     vs = (a-d)+(b-c) -> B_g, g odd       vd = (a-d)-(b-c) -> B_g, g even
+// and each of the four parity classes has K/2 <= 8 frequencies: exactly one MMA n-tile.  MMA roles:
+//   M = 16 real columns = 8 complex positions (rows 0..7 = real parts, 8..15 = imaginary parts: a C fragment
+//       then holds whole complex values), the folded DATA as A operand;
+//   K = 8 row quadruples per k-step;  N = the class's frequency slots, the BASIS as B operand (shared table).
+// Half the MMAs of the single fold (which needs two 16-row frequency tiles per 8 columns), and half the row pairs.
+// The left-over cos K (even class, ninth slot) runs on FFMA.
+//
+// The input streams through a per-warp ring of shared-memory stages filled with cp.async (16 bytes per lane and
+// request): one stage = one k-step of one task = 4 x 8 rows of 128 bytes.  The ring runs ahead across task
+// boundaries, so several kilobytes per warp are in flight at all times without holding them in registers (with
+// register double-buffering this stage was bound by load latency).
 // ------------------------------------------------------------------------------------------
-// The contraction streams its input through a per-warp ring of shared-memory stages filled with cp.async
-// (16 bytes per lane and request): one stage = one k-step of one task = 8 rows and their 8 mirror rows, 128 bytes
-// each.  The ring runs ahead across task boundaries, so several kilobytes per warp are in flight at all times
-// without holding them in registers (with register double-buffering this stage was bound by load latency).
-constexpr int kCStages = 4;
-constexpr int kCRow = 8 * kCNT + 8;          // floats per staged row: 40 = 8 mod 32, conflict-free B fragments
-constexpr int kCStageFloats = 16 * kCRow;
+constexpr int kCMT = 2;                       // MMA m-tiles per task: 16 complex positions = 128 bytes per row
+constexpr int kCPos = 8 * kCMT;
+constexpr int kCWarps = 12;
+constexpr int kCThreads = kCWarps * 32;
+constexpr int kCStages = 3;
+constexpr int kCRow = 2 * kCPos + 8;          // floats per staged row: 40 = 8 mod 32, conflict-free 8-byte loads
+constexpr int kCStageFloats = 32 * kCRow;     // [a | b | c | d][8 quadruples]
 
 __device__ __forceinline__ void cp_async16(float* smem_dst, const float* gsrc) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
@@ -67,33 +78,46 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// One k-step from a filled stage.  FULL: all kCNT column tiles are valid (no predicates in the instruction stream).
-template <bool FULL>
-__device__ __forceinline__ void contract_step(const float* S, const float4* at, const float* cK, int q0, int ntv,
-                                              float (&accC)[kCNT][4], float (&accS)[kCNT][4], float (&aK)[kCNT]) {
-  uint32_t ch[4], cl[4], sh[4], sl[4];
-  from_f4(at[0], ch);
-  from_f4(at[32], cl);
-  from_f4(at[64], sh);
-  from_f4(at[96], sl);
-  const float ck0 = cK[q0], ck1 = cK[q0 + 4];
+// frequency of slot s in parity class cls (0: even cos, 1: odd cos, 2: odd sin, 3: even sin)
+__device__ __forceinline__ int class_freq(int cls, int s) { return cls == 0 ? 2 * s : (cls == 3 ? 2 * s + 2 : 2 * s + 1); }
+
+// One k-step (8 quadruples) of one m-tile (8 complex positions) from a filled stage.
+__device__ __forceinline__ void contract_step(const float* S, const float4* bt, float ck0, float ck1,
+                                              float (&acc)[4][4], float (&aK)[2]) {
+  // S points at this lane's (quadruple t4, position g8): rows of group g sit 8 * kCRow floats apart
+  float X[4][4];   // [class][A-fragment element: (re, t4) (im, t4) (re, t4+4) (im, t4+4)]
 #pragma unroll
-  for (int nt = 0; nt < kCNT; ++nt) {
-    if (FULL || nt < ntv) {
-      // rows t4, t4 + 4 of the k-step and their mirrors (staged 8 rows further down)
-      const float x0 = S[8 * nt], x1 = S[8 * kCRow + 8 * nt];
-      const float x2 = S[4 * kCRow + 8 * nt], x3 = S[12 * kCRow + 8 * nt];
-      const float p0 = x0 + x1, d0 = x0 - x1;
-      const float p1 = x2 + x3, d1 = x2 - x3;
-      uint32_t ph0, pl0, ph1, pl1, dh0, dl0, dh1, dl1;
-      split_tf32_round(p0, ph0, pl0);
-      split_tf32_round(p1, ph1, pl1);
-      split_tf32_round(d0, dh0, dl0);
-      split_tf32_round(d1, dh1, dl1);
-      mma3_tf32(accC[nt], ch, cl, ph0, ph1, pl0, pl1);
-      mma3_tf32(accS[nt], sh, sl, dh0, dh1, dl0, dl1);
-      aK[nt] = fmaf(p0, ck0, fmaf(p1, ck1, aK[nt]));
+  for (int h = 0; h < 2; ++h) {
+    const float2 a = *reinterpret_cast<const float2*>(S + (0 * 8 + 4 * h) * kCRow);
+    const float2 b = *reinterpret_cast<const float2*>(S + (1 * 8 + 4 * h) * kCRow);
+    const float2 c = *reinterpret_cast<const float2*>(S + (2 * 8 + 4 * h) * kCRow);
+    const float2 d = *reinterpret_cast<const float2*>(S + (3 * 8 + 4 * h) * kCRow);
+    {
+      const float u = a.x + d.x, v = a.x - d.x, up = b.x + c.x, vp = b.x - c.x;
+      X[0][2 * h] = u + up;
+      X[1][2 * h] = u - up;
+      X[2][2 * h] = v + vp;
+      X[3][2 * h] = v - vp;
     }
+    {
+      const float u = a.y + d.y, v = a.y - d.y, up = b.y + c.y, vp = b.y - c.y;
+      X[0][2 * h + 1] = u + up;
+      X[1][2 * h + 1] = u - up;
+      X[2][2 * h + 1] = v + vp;
+      X[3][2 * h + 1] = v - vp;
+    }
+  }
+  aK[0] = fmaf(X[0][0], ck0, fmaf(X[0][2], ck1, aK[0]));
+  aK[1] = fmaf(X[0][1], ck0, fmaf(X[0][3], ck1, aK[1]));
+#pragma unroll
+  for (int cls = 0; cls < 4; ++cls) {
+    uint32_t ah[4], al[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) split_tf32_round(X[cls][e], ah[e], al[e]);
+    const float4 b = bt[cls * 32];   // (b0 hi, b1 hi, b0 lo, b1 lo)
+    mma_m16n8k8_tf32(acc[cls], ah, __float_as_uint(b.x), __float_as_uint(b.y));
+    mma_m16n8k8_tf32(acc[cls], al, __float_as_uint(b.x), __float_as_uint(b.y));
+    mma_m16n8k8_tf32(acc[cls], ah, __float_as_uint(b.z), __float_as_uint(b.w));
   }
 }
 
@@ -101,28 +125,28 @@ template <int K>
 __global__ void __launch_bounds__(kCThreads, 1)
 mid_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out, long long outer, long long inner,
                         int N, float scale) {
+  static_assert(K % 4 == 0 && K <= 16, "parity classes of K/2 <= 8 frequencies");
   extern __shared__ float4 mm_smem[];
-  const int KS = N / 16;                                    // k-steps of 8 row pairs (even: N % 32 == 0)
-  float4* atab = mm_smem;                                   // [KS][tile cos|sin][hi|lo][lane]
-  float* cK = reinterpret_cast<float*>(atab + (size_t)KS * 4 * 32);   // cos(psi_K (q + 1/2)), q < N/2
+  const int KS = N / 32;                                    // k-steps of 8 row quadruples
+  float4* btab = mm_smem;                                   // [KS][class][lane]
+  float* cK = reinterpret_cast<float*>(btab + (size_t)KS * 4 * 32);   // cos(psi_K (q + 1/2)), q < N/4
 
-  for (int e = threadIdx.x; e < KS * 2 * 32; e += blockDim.x) {
-    const int l = e & 31, tile = (e >> 5) & 1, ks = e >> 6;
-    const int lg = l >> 2, lt = l & 3;
-    uint32_t hi[4], lo[4];
+  for (int e = threadIdx.x; e < KS * 4 * 32; e += blockDim.x) {
+    const int l = e & 31, cls = (e >> 5) & 3, ks = e >> 7;
+    const int lg = l >> 2, lt = l & 3;                      // B fragment: k = lt (+4), n = lg
+    const int g = class_freq(cls, lg);
+    const bool valid = lg < K / 2;
+    uint32_t hi[2], lo[2];
 #pragma unroll
-    for (int a = 0; a < 4; ++a) {
-      const int r = lg + 8 * (a & 1), q = 8 * ks + lt + 4 * (a >> 1);
-      const int g = (tile == 1 && r == 0) ? K : r;
+    for (int h = 0; h < 2; ++h) {
       float cs, sn;
-      basis_cs(g, q, N, cs, sn);
-      const float v = (r < K) ? (tile == 0 ? cs : sn) : 0.f;
-      split_tf32_rna(v, hi[a], lo[a]);
+      basis_cs(g, 8 * ks + lt + 4 * h, N, cs, sn);
+      const float v = valid ? ((cls == 0 || cls == 1) ? cs : sn) : 0.f;
+      split_tf32_rna(v, hi[h], lo[h]);
     }
-    atab[((ks * 2 + tile) * 2 + 0) * 32 + l] = as_f4(hi);
-    atab[((ks * 2 + tile) * 2 + 1) * 32 + l] = as_f4(lo);
+    btab[e] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(lo[0]), __uint_as_float(lo[1]));
   }
-  for (int q = threadIdx.x; q < N / 2; q += blockDim.x) {
+  for (int q = threadIdx.x; q < N / 4; q += blockDim.x) {
     float cs, sn;
     basis_cs(K, q, N, cs, sn);
     cK[q] = cs;
@@ -131,25 +155,22 @@ mid_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out, 
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g8 = lane >> 2, t4 = lane & 3;
-  // e^{i psi_g / 2} * scale for this lane's frequencies g8, g8 + 8 and for K
-  float2 rho_a, rho_b, rho_K;
-  {
+  // e^{i psi_g / 2} * scale for this lane's frequencies 4 t4 .. 4 t4 + 3 and for K
+  float2 rho[5];
+#pragma unroll
+  for (int j = 0; j < 5; ++j) {
     double s, c;
-    sincospi((double)g8 / (double)N, &s, &c);
-    rho_a = make_float2((float)c * scale, (float)s * scale);
-    sincospi((double)(g8 + 8) / (double)N, &s, &c);
-    rho_b = make_float2((float)c * scale, (float)s * scale);
-    sincospi((double)K / (double)N, &s, &c);
-    rho_K = make_float2((float)c * scale, (float)s * scale);
+    sincospi((double)(j < 4 ? 4 * t4 + j : K) / (double)N, &s, &c);
+    rho[j] = make_float2((float)c * scale, (float)s * scale);
   }
 
   const long long cblocks = (inner + kCPos - 1) / kCPos;
   const long long tasks = outer * cblocks;
   const long long rs = 2 * inner;   // floats per row
   const long long tstride = (long long)gridDim.x * kCWarps;
-  float* ring = cK + N / 2 + (size_t)warp * kCStages * kCStageFloats;   // this warp's stages (16-byte aligned)
+  float* ring = cK + N / 4 + (size_t)warp * kCStages * kCStageFloats;   // this warp's stages (16-byte aligned)
 
-  // producer cursor: (task, k-step) of the next stage to request; lane = (row group lane / 8, 16-byte chunk lane % 8)
+  // producer cursor: (task, k-step) of the next stage to request; lane = (row lane / 8, 16-byte chunk lane % 8)
   long long ptask = (long long)blockIdx.x * kCWarps + warp;
   int pks = 0, pstage = 0;
   const float* ptb = in;
@@ -159,18 +180,22 @@ mid_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out, 
       if (pks == 0) {
         const long long o = ptask / cblocks, cb = ptask % cblocks;
         const long long left = inner - cb * kCPos;
-        const int nch = left >= kCPos ? 2 * kCNT : (int)(left / 2);   // valid 16-byte chunks per row
+        const int nch = left >= kCPos ? kCPos / 2 : (int)(left / 2);   // valid 16-byte chunks per row
         ptb = in + o * N * rs + cb * (2 * kCPos) + 4 * (lane & 7);
         pchunk_ok = (lane & 7) < nch;
       }
       if (pchunk_ok) {
         float* dst = ring + pstage * kCStageFloats + (lane >> 3) * kCRow + 4 * (lane & 7);
         const int q = 8 * pks + (lane >> 3);
-        // staged rows: 0..7 = rows q of the k-step, 8..15 = their mirrors N-1-q
-        cp_async16(dst, ptb + (long long)q * rs);
-        cp_async16(dst + 4 * kCRow, ptb + (long long)(q + 4) * rs);
-        cp_async16(dst + 8 * kCRow, ptb + (long long)(N - 1 - q) * rs);
-        cp_async16(dst + 12 * kCRow, ptb + (long long)(N - 5 - q) * rs);
+        // staged rows: group a = rows q, b = N/2-1-q, c = N/2+q, d = N-1-q (8 quadruples each; this lane: q, q+4)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int qq = q + 4 * h;
+          cp_async16(dst + (0 * 8 + 4 * h) * kCRow, ptb + (long long)qq * rs);
+          cp_async16(dst + (1 * 8 + 4 * h) * kCRow, ptb + (long long)(N / 2 - 1 - qq) * rs);
+          cp_async16(dst + (2 * 8 + 4 * h) * kCRow, ptb + (long long)(N / 2 + qq) * rs);
+          cp_async16(dst + (3 * 8 + 4 * h) * kCRow, ptb + (long long)(N - 1 - qq) * rs);
+        }
       }
       if (++pks == KS) {
         pks = 0;
@@ -187,59 +212,63 @@ mid_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out, 
   for (long long task = (long long)blockIdx.x * kCWarps + warp; task < tasks; task += tstride) {
     const long long o = task / cblocks, cb = task % cblocks;
     const long long left = inner - cb * kCPos;
-    const int ntv = left >= kCPos ? kCNT : (int)(left / 4);   // valid n-tiles
+    const int mtv = left >= kCPos ? kCMT : (int)((left + 7) / 8);   // m-tiles with at least one valid position
 
-    float accC[kCNT][4], accS[kCNT][4], aK[kCNT];
+    float acc[kCMT][4][4], aK[kCMT][2];
 #pragma unroll
-    for (int nt = 0; nt < kCNT; ++nt) {
-      aK[nt] = 0.f;
+    for (int mt = 0; mt < kCMT; ++mt) {
+      aK[mt][0] = aK[mt][1] = 0.f;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) accC[nt][e] = accS[nt][e] = 0.f;
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[mt][c][e] = 0.f;
     }
 
-    auto body = [&](auto full_tag) {
-      constexpr bool FULL = decltype(full_tag)::value;
 #pragma unroll 1
-      for (int ks = 0; ks < KS; ++ks) {
-        cp_async_wait<kCStages - 2>();   // this k-step's stage has landed (for this lane's requests) ...
-        __syncwarp();                    // ... and for everyone's; all lanes are done with the previous stage
-        issue();                         // refill the stage read in the previous k-step
-        const float* S = ring + cstage * kCStageFloats + t4 * kCRow + g8;
-        contract_step<FULL>(S, atab + (size_t)(ks * 4) * 32 + lane, cK, 8 * ks + t4, ntv, accC, accS, aK);
-        cstage = cstage + 1 == kCStages ? 0 : cstage + 1;
-      }
-    };
-    if (ntv == kCNT) body(std::true_type{});
-    else body(std::false_type{});
-
-    // A_K: sum the quad's partial sums (each lane covered the row pairs t4, t4 + 4 of every k-step)
+    for (int ks = 0; ks < KS; ++ks) {
+      cp_async_wait<kCStages - 2>();   // this k-step's stage has landed (for this lane's requests) ...
+      __syncwarp();                    // ... and for everyone's; all lanes are done with the previous stage
+      issue();                         // refill the stage read in the previous k-step
+      const float* S = ring + cstage * kCStageFloats + t4 * kCRow + 2 * g8;
+      const float4* bt = btab + (size_t)(ks * 4) * 32 + lane;
+      const float ck0 = cK[8 * ks + t4], ck1 = cK[8 * ks + t4 + 4];
 #pragma unroll
-    for (int nt = 0; nt < kCNT; ++nt) {
-      aK[nt] += __shfl_xor_sync(0xffffffffu, aK[nt], 1);
-      aK[nt] += __shfl_xor_sync(0xffffffffu, aK[nt], 2);
+      for (int mt = 0; mt < kCMT; ++mt)
+        if (mt < mtv) contract_step(S + 16 * mt, bt, ck0, ck1, acc[mt], aK[mt]);
+      cstage = cstage + 1 == kCStages ? 0 : cstage + 1;
     }
 
+    // ---- epilogue.  acc[mt][cls] = (re, slot 2 t4), (re, slot 2 t4 + 1), (im, 2 t4), (im, 2 t4 + 1) of position g8.
     // Z_{+g} = rho_g (A_g - i B_g) -> row g (g < K);  Z_{-g} = conj(rho_g) (A_g + i B_g) -> row 2K - g (g >= 1)
-    float2* ob = out + o * (2 * K) * inner + cb * kCPos + t4;
-    auto emit = [&](int g, float2 rho, float ax, float ay, float bx, float by, float2* dst) {
-      const float pr = ax + by, pi = ay - bx;   // A - iB
-      const float mr = ax - by, mi = ay + bx;   // A + iB
-      if (g < K) dst[(long long)g * inner] = make_float2(rho.x * pr - rho.y * pi, rho.x * pi + rho.y * pr);
-      if (g > 0) dst[(long long)(2 * K - g) * inner] = make_float2(rho.x * mr + rho.y * mi, rho.x * mi - rho.y * mr);
-    };
 #pragma unroll
-    for (int nt = 0; nt < kCNT; ++nt) {
-      // every lane takes part in the shuffles; lanes of row group 0 need A_K of their column pair
-      const float aKr = __shfl_sync(0xffffffffu, aK[nt], (2 * t4) * 4);
-      const float aKi = __shfl_sync(0xffffffffu, aK[nt], (2 * t4 + 1) * 4);
-      if (nt < ntv) {
-        float2* dst = ob + 4 * nt;
-        if (g8 < K) {
-          const float bx = g8 > 0 ? accS[nt][0] : 0.f, by = g8 > 0 ? accS[nt][1] : 0.f;
-          emit(g8, rho_a, accC[nt][0], accC[nt][1], bx, by, dst);
+    for (int mt = 0; mt < kCMT; ++mt) {
+      // A_K: sum the quad's partial sums (each lane covered the quadruples t4, t4 + 4 of every k-step)
+      float aKr = aK[mt][0], aKi = aK[mt][1];
+      aKr += __shfl_xor_sync(0xffffffffu, aKr, 1);
+      aKr += __shfl_xor_sync(0xffffffffu, aKr, 2);
+      aKi += __shfl_xor_sync(0xffffffffu, aKi, 1);
+      aKi += __shfl_xor_sync(0xffffffffu, aKi, 2);
+      // B of the even frequency 4 t4 is the even-sine slot 2 t4 - 1: the second slot of the lane below
+      float bpr = __shfl_up_sync(0xffffffffu, acc[mt][3][1], 1);
+      float bpi = __shfl_up_sync(0xffffffffu, acc[mt][3][3], 1);
+      if (t4 == 0) bpr = bpi = 0.f;   // B_0 = 0
+      const long long pos = cb * kCPos + 8 * mt + g8;
+      if (mt < mtv && pos < inner) {
+        float2* dst = out + o * (2 * K) * inner + pos;
+        auto emit = [&](int g, float2 r, float ax, float ay, float bx, float by) {
+          const float pr = ax + by, pi = ay - bx;   // A - iB
+          const float mr = ax - by, mi = ay + bx;   // A + iB
+          if (g < K) dst[(long long)g * inner] = make_float2(r.x * pr - r.y * pi, r.x * pi + r.y * pr);
+          if (g > 0) dst[(long long)(2 * K - g) * inner] = make_float2(r.x * mr + r.y * mi, r.x * mi - r.y * mr);
+        };
+        const int g0 = 4 * t4;
+        if (g0 < K) {
+          emit(g0, rho[0], acc[mt][0][0], acc[mt][0][2], bpr, bpi);                                   // even, slot 2 t4
+          emit(g0 + 1, rho[1], acc[mt][1][0], acc[mt][1][2], acc[mt][2][0], acc[mt][2][2]);           // odd
+          emit(g0 + 2, rho[2], acc[mt][0][1], acc[mt][0][3], acc[mt][3][0], acc[mt][3][2]);           // even, slot 2 t4 + 1
+          emit(g0 + 3, rho[3], acc[mt][1][1], acc[mt][1][3], acc[mt][2][1], acc[mt][2][3]);           // odd
         }
-        if (g8 + 8 < K) emit(g8 + 8, rho_b, accC[nt][2], accC[nt][3], accS[nt][2], accS[nt][3], dst);
-        if (g8 == 0) emit(K, rho_K, aKr, aKi, accS[nt][0], accS[nt][1], dst);
+        if (t4 == K / 4 - 1) emit(K, rho[4], aKr, aKi, acc[mt][3][1], acc[mt][3][3]);                 // -K only
       }
     }
   }
@@ -432,7 +461,7 @@ mid_expand_mma_kernel(const float2* __restrict__ in, float* __restrict__ out, lo
 
 template <int K>
 size_t contract_smem(int N) {
-  return (size_t)(N / 16) * 4 * 32 * 16 + (size_t)(N / 2) * 4 + (size_t)kCWarps * kCStages * kCStageFloats * 4;
+  return (size_t)(N / 32) * 4 * 32 * 16 + (size_t)(N / 4) * 4 + (size_t)kCWarps * kCStages * kCStageFloats * 4;
 }
 
 template <int K>
