@@ -19,10 +19,6 @@
 namespace dtst {
 namespace {
 
-constexpr int kMmaWarps = 12;   // one persistent CTA per SM: the basis tables are built once per SM
-constexpr int kMmaThreads = kMmaWarps * 32;
-constexpr int kNT = 8;              // expansion: MMA n-tiles per task: 64 real columns = 32 complex positions
-constexpr int kTaskPos = 4 * kNT;   // complex positions per task
 
 __device__ __forceinline__ float4 as_f4(const uint32_t (&v)[4]) {
   return make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
@@ -275,187 +271,182 @@ mid_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out, 
 }
 
 // ------------------------------------------------------------------------------------------
-// expansion: in[outer][2K][inner] -> out[outer][N][inner]   (B^H along this dimension)
-//   z_n = P_n + Q_n, z_{N-1-n} = P_n - Q_n, n < N/2,
-//   P_n = sum_{g<=K} alpha_g cos(psi_g (n+1/2)), Q_n = sum_{1<=g<=K} beta_g sin(psi_g (n+1/2)),
-//   alpha_g = V'_{+g} + V'_{-g}, beta_g = i (V'_{+g} - V'_{-g}), V'_{+-g} = e^{-+i psi_g/2} V_{+-g}.
-//   MMA roles: M = output row n (basis = A operand, fragment-ordered shared table), K = frequency slot
-//   (cos: g = 0..K-1, sin: g = 1..K, eight per k-step), N = real column.  A warp first forms alpha, beta of its
-//   32 positions in a private shared buffer (one lane per position, coalesced loads), then walks the column
-//   tiles: B fragments from that buffer, all row tiles against them, rows stored straight from the C fragments.
-//   alpha_K cos(psi_K (n+1/2)) is added on FFMA.
+// expansion: in[outer][2K][inner] -> out[outer][N][inner]   (B^H along this dimension), the transpose of the
+// contraction above with the same two folds.  With
+//   alpha_g = V'_{+g} + V'_{-g}, beta_g = i (V'_{+g} - V'_{-g}), V'_{+-g} = e^{-+i psi_g/2} V_{+-g}
+// and, for a row quadruple n < N/4, the four class sums
+//   Pe = sum_{g even} alpha_g cos(psi_g (n+1/2)),  Po = sum_{g odd} alpha_g cos,
+//   Qo = sum_{g odd} beta_g sin(psi_g (n+1/2)),    Qe = sum_{g even} beta_g sin,
+// the four output rows are
+//   z_n = Pe+Po+Qo+Qe,  z_{N/2-1-n} = Pe-Po+Qo-Qe,  z_{N/2+n} = Pe-Po-Qo+Qe,  z_{N-1-n} = Pe+Po-Qo-Qe.
+// MMA roles: M = 16 real columns = 8 complex positions (real parts | imaginary parts), alpha / beta of a class as
+// the A operand, built once per task straight from global memory into registers; K = the class's 8 frequency
+// slots; N = 8 row quadruples, the basis as B operand from a fragment-ordered shared table.  The left-over
+// alpha_K cos(psi_K (n+1/2)) is added on FFMA.  Rows are written from the C fragments, 64 contiguous bytes per row
+// and store instruction.
 // ------------------------------------------------------------------------------------------
-template <int K>
-struct ExpCfg {
-  static constexpr int KS = (K + 7) / 8;         // k-steps over the frequencies
-  static constexpr int ROW = 2 * kTaskPos + 8;   // floats per buffer row: 72 = 8 mod 32, conflict-free B loads
-  static constexpr int ROWS = 8 * KS + 1;        // alpha rows 0..8KS-1 (zero beyond K-1) + row 8KS for alpha_K
-  static constexpr int WARP_FLOATS = 2 * ROWS * ROW;   // alpha block, beta block (beta row j holds g = j + 1)
-};
+constexpr int kEMT = 2;                       // m-tiles per task: 16 complex positions
+constexpr int kEPos = 8 * kEMT;
+constexpr int kEWarps = 12;
+constexpr int kEThreads = kEWarps * 32;
 
 template <int K>
-__global__ void __launch_bounds__(kMmaThreads, 1)
-mid_expand_mma_kernel(const float2* __restrict__ in, float* __restrict__ out, long long outer, long long inner,
+__global__ void __launch_bounds__(kEThreads, 1)
+mid_expand_mma_kernel(const float2* __restrict__ in, float2* __restrict__ out, long long outer, long long inner,
                       int N, float scale, int streaming) {
-  using EC = ExpCfg<K>;
-  constexpr int KS = EC::KS;
+  static_assert(K % 4 == 0 && K <= 16, "parity classes of K/2 <= 8 frequencies");
   extern __shared__ float4 mm_smem[];
-  const int MT = N / 32;                                   // 16-row tiles over n < N/2
-  float4* atab = mm_smem;                                  // [MT][KS][tile cos|sin][hi|lo][lane]
-  float* cK = reinterpret_cast<float*>(atab + (size_t)MT * KS * 4 * 32);   // cos(psi_K (n + 1/2)), n < N/2
-  float2* rho = reinterpret_cast<float2*>(cK + N / 2);     // e^{i psi_g / 2} * scale, g <= K
-  float* bufs = reinterpret_cast<float*>(rho + K + 1 + ((K + 1) & 1));     // 16-byte aligned
+  const int NT = N / 32;                                   // n-tiles of 8 row quadruples
+  float4* btab = mm_smem;                                  // [NT][class][lane]
+  float* cK = reinterpret_cast<float*>(btab + (size_t)NT * 4 * 32);   // cos(psi_K (n + 1/2)), n < N/4
 
-  for (int e = threadIdx.x; e < MT * KS * 2 * 32; e += blockDim.x) {
-    const int l = e & 31, tile = (e >> 5) & 1, ks = (e >> 6) % KS, mt = (e >> 6) / KS;
-    const int lg = l >> 2, lt = l & 3;
-    uint32_t hi[4], lo[4];
+  for (int e = threadIdx.x; e < NT * 4 * 32; e += blockDim.x) {
+    const int l = e & 31, cls = (e >> 5) & 3, nt = e >> 7;
+    const int lg = l >> 2, lt = l & 3;                      // B fragment: k = slot lt (+4), n = quadruple lg
+    uint32_t hi[2], lo[2];
 #pragma unroll
-    for (int a = 0; a < 4; ++a) {
-      const int n = 16 * mt + lg + 8 * (a & 1);
-      const int j = 8 * ks + lt + 4 * (a >> 1);      // frequency slot
-      const int g = tile == 0 ? j : j + 1;
-      const bool valid = tile == 0 ? (g < K) : (g <= K);
+    for (int h = 0; h < 2; ++h) {
+      const int slot = lt + 4 * h;
       float cs, sn;
-      basis_cs(g, n, N, cs, sn);
-      const float v = valid ? (tile == 0 ? cs : sn) : 0.f;
-      split_tf32_rna(v, hi[a], lo[a]);
+      basis_cs(class_freq(cls, slot), 8 * nt + lg, N, cs, sn);
+      const float v = slot < K / 2 ? ((cls == 0 || cls == 1) ? cs : sn) : 0.f;
+      split_tf32_rna(v, hi[h], lo[h]);
     }
-    atab[(((mt * KS + ks) * 2 + tile) * 2 + 0) * 32 + l] = as_f4(hi);
-    atab[(((mt * KS + ks) * 2 + tile) * 2 + 1) * 32 + l] = as_f4(lo);
+    btab[e] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(lo[0]), __uint_as_float(lo[1]));
   }
-  for (int n = threadIdx.x; n < N / 2; n += blockDim.x) {
+  for (int n = threadIdx.x; n < N / 4; n += blockDim.x) {
     float cs, sn;
     basis_cs(K, n, N, cs, sn);
     cK[n] = cs;
-  }
-  for (int g = threadIdx.x; g <= K; g += blockDim.x) {
-    double s, c;
-    sincospi((double)g / (double)N, &s, &c);
-    rho[g] = make_float2((float)c * scale, (float)s * scale);
   }
   __syncthreads();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g8 = lane >> 2, t4 = lane & 3;
-  float* al = bufs + (size_t)warp * EC::WARP_FLOATS;       // alpha rows
-  float* be = al + EC::ROWS * EC::ROW;                     // beta rows (row j <-> g = j + 1)
-  // rows that no frequency fills stay zero for the whole kernel
-  for (int e = lane; e < EC::WARP_FLOATS; e += 32) al[e] = 0.f;
-  __syncwarp();
-
-  const long long cblocks = (inner + kTaskPos - 1) / kTaskPos;
-  const long long tasks = outer * cblocks;
-  const long long rs = 2 * inner;   // floats per output row
-  for (long long task = (long long)blockIdx.x * kMmaWarps + warp; task < tasks;
-       task += (long long)gridDim.x * kMmaWarps) {
-    const long long o = task / cblocks, cb = task % cblocks;
-    const long long left = inner - cb * kTaskPos;
-    const int ntv = left >= kTaskPos ? kNT : (int)(left / 4);
-
-    // ---- alpha, beta of this task's positions: lane = position
-    {
-      const bool ok = lane < 4 * ntv;
-      const float2* src = in + o * (2 * K) * inner + cb * kTaskPos + lane;
+  // the six frequencies whose alpha / beta this lane turns into A fragments: 2 t4 + {0, 1, 2} and the same + 8
+  float2 rho[7];   // e^{i psi_g / 2} * scale; [6] = frequency K
 #pragma unroll
-      for (int g = 0; g <= K; ++g) {
-        const float2 r = rho[g];
+  for (int j = 0; j < 7; ++j) {
+    const int g = j < 6 ? 2 * t4 + (j % 3) + 8 * (j / 3) : K;
+    double s, c;
+    sincospi((double)g / (double)N, &s, &c);
+    rho[j] = make_float2((float)c * scale, (float)s * scale);
+  }
+
+  const long long cblocks = (inner + kEPos - 1) / kEPos;
+  const long long tasks = outer * cblocks;
+  const long long tstride = (long long)gridDim.x * kEWarps;
+  for (long long task = (long long)blockIdx.x * kEWarps + warp; task < tasks; task += tstride) {
+    const long long o = task / cblocks, cb = task % cblocks;
+    const long long left = inner - cb * kEPos;
+    const int mtv = left >= kEPos ? kEMT : (int)((left + 7) / 8);
+
+    // pull the next task's 2K input rows (128 bytes each) into L2 while this one runs on the tensor cores
+    {
+      const long long nx = task + tstride;
+      if (nx < tasks) {
+        const float2* nsrc = in + (nx / cblocks) * (2 * K) * inner + (nx % cblocks) * kEPos;
+        for (int r = lane; r < 2 * K; r += 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(nsrc + (long long)r * inner));
+      }
+    }
+
+    // ---- A fragments: alpha (classes 0, 1) and beta (classes 2, 3) of this lane's position, hi / lo
+    uint32_t ah[kEMT][4][4], al[kEMT][4][4];
+    float2 aKv[kEMT];
+#pragma unroll
+    for (int mt = 0; mt < kEMT; ++mt) {
+      const long long pos = cb * kEPos + 8 * mt + g8;
+      const bool ok = mt < mtv && pos < inner;
+      const float2* src = in + o * (2 * K) * inner + (ok ? pos : 0);
+      float2 alpha[6], beta[6];
+#pragma unroll
+      for (int j = 0; j < 6; ++j) {
+        const int g = 2 * t4 + (j % 3) + 8 * (j / 3);
         float2 v = make_float2(0.f, 0.f), u = make_float2(0.f, 0.f);
         if (ok && g < K) v = __ldcs(src + (long long)g * inner);
-        if (ok && g > 0) u = __ldcs(src + (long long)(2 * K - g) * inner);
+        if (ok && g > 0 && g <= K) u = __ldcs(src + (long long)(2 * K - g) * inner);
+        const float2 r = rho[j];
         const float2 vp = make_float2(v.x * r.x + v.y * r.y, v.y * r.x - v.x * r.y);   // v * conj(rho)
         const float2 vm = make_float2(u.x * r.x - u.y * r.y, u.y * r.x + u.x * r.y);   // u * rho
-        const int arow = g < K ? g : 8 * KS;
-        *reinterpret_cast<float2*>(al + arow * EC::ROW + 2 * lane) = make_float2(vp.x + vm.x, vp.y + vm.y);
-        if (g > 0)
-          *reinterpret_cast<float2*>(be + (g - 1) * EC::ROW + 2 * lane) =
-              make_float2(-(vp.y - vm.y), vp.x - vm.x);                                // i (vp - vm)
+        alpha[j] = make_float2(vp.x + vm.x, vp.y + vm.y);
+        beta[j] = make_float2(-(vp.y - vm.y), vp.x - vm.x);                            // i (vp - vm)
+      }
+      {
+        float2 u = make_float2(0.f, 0.f);
+        if (ok) u = __ldcs(src + (long long)K * inner);                                // V_{-K}
+        const float2 r = rho[6];
+        aKv[mt] = make_float2(u.x * r.x - u.y * r.y, u.y * r.x + u.x * r.y);           // alpha_K = rho_K V_{-K}
+      }
+      // class slots t4 (h = 0) and t4 + 4 (h = 1): even cos g = 2 slot, odd g = 2 slot + 1, even sin g = 2 slot + 2
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        split_tf32_round(alpha[3 * h + 0].x, ah[mt][0][2 * h], al[mt][0][2 * h]);
+        split_tf32_round(alpha[3 * h + 0].y, ah[mt][0][2 * h + 1], al[mt][0][2 * h + 1]);
+        split_tf32_round(alpha[3 * h + 1].x, ah[mt][1][2 * h], al[mt][1][2 * h]);
+        split_tf32_round(alpha[3 * h + 1].y, ah[mt][1][2 * h + 1], al[mt][1][2 * h + 1]);
+        split_tf32_round(beta[3 * h + 1].x, ah[mt][2][2 * h], al[mt][2][2 * h]);
+        split_tf32_round(beta[3 * h + 1].y, ah[mt][2][2 * h + 1], al[mt][2][2 * h + 1]);
+        split_tf32_round(beta[3 * h + 2].x, ah[mt][3][2 * h], al[mt][3][2 * h]);
+        split_tf32_round(beta[3 * h + 2].y, ah[mt][3][2 * h + 1], al[mt][3][2 * h + 1]);
       }
     }
-    __syncwarp();
 
-    // pull the next task's 2K input rows (256 bytes each) into L2 while this one runs on the tensor cores
-    {
-      const long long nt_task = task + (long long)gridDim.x * kMmaWarps;
-      if (nt_task < tasks) {
-        const long long o2 = nt_task / cblocks, cb2 = nt_task % cblocks;
-        const float2* nsrc = in + o2 * (2 * K) * inner + cb2 * kTaskPos;
-        const bool second = inner - cb2 * kTaskPos > 16;   // the second 128-byte line holds valid positions
-        for (int r = lane; r < 2 * K; r += 32) {
-          asm volatile("prefetch.global.L2 [%0];" ::"l"(nsrc + (long long)r * inner));
-          if (second) asm volatile("prefetch.global.L2 [%0];" ::"l"(nsrc + (long long)r * inner + 16));
-        }
-      }
-    }
-
-    float* ob = out + o * N * rs + cb * (2 * kTaskPos) + 2 * t4;
-    const float* alq = al + t4 * EC::ROW + g8;   // B fragment element (slot t4 + 4h + 8ks, column 8nt + g8)
-    const float* beq = be + t4 * EC::ROW + g8;
-    const float* aKp = al + (8 * KS) * EC::ROW + 2 * t4;
-
-    // row tiles outermost: the basis fragments of a tile are loaded once and meet all column tiles, whose
-    // fragments come from the warp's buffer; a row tile's 16 + 16 rows are written 256 bytes at a time
-    auto body = [&](auto full_tag) {
-      constexpr bool FULL = decltype(full_tag)::value;
+    float2* ob = out + o * N * inner + cb * kEPos + g8;
 #pragma unroll 1
-      for (int mt = 0; mt < MT; ++mt) {
-        uint32_t ch[KS][4], cl[KS][4], sh[KS][4], sl[KS][4];
+    for (int nt = 0; nt < NT; ++nt) {
+      float4 bf[4];
 #pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-          const float4* t = atab + (size_t)((mt * KS + ks) * 4) * 32 + lane;
-          from_f4(t[0], ch[ks]);
-          from_f4(t[32], cl[ks]);
-          from_f4(t[64], sh[ks]);
-          from_f4(t[96], sl[ks]);
-        }
-        const int n0 = 16 * mt + g8;
-        const float c0 = cK[n0], c1 = cK[n0 + 8];
-        float* da = ob + (long long)n0 * rs;
-        float* db = da + 8 * rs;
-        float* dc = ob + (long long)(N - 1 - n0) * rs;
-        float* dd = dc - 8 * rs;
-#pragma unroll 1
-        for (int nh = 0; nh < kNT; nh += 4)
+      for (int c = 0; c < 4; ++c) bf[c] = btab[(size_t)(nt * 4 + c) * 32 + lane];
+      const int n0 = 8 * nt + 2 * t4;                      // this lane's two quadruples: n0, n0 + 1
+      const float c0 = cK[n0], c1 = cK[n0 + 1];
 #pragma unroll
-        for (int ni = 0; ni < 4; ++ni) {
-          const int nt = nh + ni;
-          if (FULL || nt < ntv) {
-            float P[4] = {0.f, 0.f, 0.f, 0.f}, Q[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int mt = 0; mt < kEMT; ++mt) {
+        if (mt < mtv) {
+          float acc[4][4];
 #pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-              uint32_t ah0, al0, ah1, al1, bh0, bl0, bh1, bl1;
-              split_tf32_round(alq[(8 * ks) * EC::ROW + 8 * nt], ah0, al0);
-              split_tf32_round(alq[(8 * ks + 4) * EC::ROW + 8 * nt], ah1, al1);
-              split_tf32_round(beq[(8 * ks) * EC::ROW + 8 * nt], bh0, bl0);
-              split_tf32_round(beq[(8 * ks + 4) * EC::ROW + 8 * nt], bh1, bl1);
-              mma3_tf32(P, ch[ks], cl[ks], ah0, ah1, al0, al1);
-              mma3_tf32(Q, sh[ks], sl[ks], bh0, bh1, bl0, bl1);
-            }
-            const float2 aK = *reinterpret_cast<const float2*>(aKp + 8 * nt);
-            P[0] = fmaf(aK.x, c0, P[0]);
-            P[1] = fmaf(aK.y, c0, P[1]);
-            P[2] = fmaf(aK.x, c1, P[2]);
-            P[3] = fmaf(aK.y, c1, P[3]);
-            const float2 va = make_float2(P[0] + Q[0], P[1] + Q[1]), vb = make_float2(P[2] + Q[2], P[3] + Q[3]);
-            const float2 vc = make_float2(P[0] - Q[0], P[1] - Q[1]), vd = make_float2(P[2] - Q[2], P[3] - Q[3]);
-            if (streaming) {   // an output far larger than L2 is not worth keeping there for the next kernel
-              __stcs(reinterpret_cast<float2*>(da + 8 * nt), va);
-              __stcs(reinterpret_cast<float2*>(db + 8 * nt), vb);
-              __stcs(reinterpret_cast<float2*>(dc + 8 * nt), vc);
-              __stcs(reinterpret_cast<float2*>(dd + 8 * nt), vd);
-            } else {
-              *reinterpret_cast<float2*>(da + 8 * nt) = va;
-              *reinterpret_cast<float2*>(db + 8 * nt) = vb;
-              *reinterpret_cast<float2*>(dc + 8 * nt) = vc;
-              *reinterpret_cast<float2*>(dd + 8 * nt) = vd;
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[c][e] = 0.f;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) mma_m16n8k8_tf32(acc[c], ah[mt][c], __float_as_uint(bf[c].x), __float_as_uint(bf[c].y));
+#pragma unroll
+          for (int c = 0; c < 4; ++c) mma_m16n8k8_tf32(acc[c], al[mt][c], __float_as_uint(bf[c].x), __float_as_uint(bf[c].y));
+#pragma unroll
+          for (int c = 0; c < 4; ++c) mma_m16n8k8_tf32(acc[c], ah[mt][c], __float_as_uint(bf[c].z), __float_as_uint(bf[c].w));
+          // acc[cls] = (re, n0) (re, n0 + 1) (im, n0) (im, n0 + 1); the left-over alpha_K term joins Pe
+          acc[0][0] = fmaf(aKv[mt].x, c0, acc[0][0]);
+          acc[0][1] = fmaf(aKv[mt].x, c1, acc[0][1]);
+          acc[0][2] = fmaf(aKv[mt].y, c0, acc[0][2]);
+          acc[0][3] = fmaf(aKv[mt].y, c1, acc[0][3]);
+          if (cb * kEPos + 8 * mt + g8 < inner) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              const int n = n0 + q;
+              const float per = acc[0][q], pei = acc[0][2 + q], por = acc[1][q], poi = acc[1][2 + q];
+              const float qor = acc[2][q], qoi = acc[2][2 + q], qer = acc[3][q], qei = acc[3][2 + q];
+              const float spr = per + por, dpr = per - por, sqr = qor + qer, dqr = qor - qer;
+              const float spi = pei + poi, dpi = pei - poi, sqi = qoi + qei, dqi = qoi - qei;
+              const float2 za = make_float2(spr + sqr, spi + sqi);     // z_n          = Pe+Po+Qo+Qe
+              const float2 zd = make_float2(spr - sqr, spi - sqi);     // z_{N-1-n}    = Pe+Po-Qo-Qe
+              const float2 zb = make_float2(dpr + dqr, dpi + dqi);     // z_{N/2-1-n}  = Pe-Po+Qo-Qe
+              const float2 zc = make_float2(dpr - dqr, dpi - dqi);     // z_{N/2+n}    = Pe-Po-Qo+Qe
+              float2* d = ob + 8 * mt;
+              if (streaming) {   // an output far larger than L2 is not worth keeping there for the next kernel
+                __stcs(d + (long long)n * inner, za);
+                __stcs(d + (long long)(N / 2 - 1 - n) * inner, zb);
+                __stcs(d + (long long)(N / 2 + n) * inner, zc);
+                __stcs(d + (long long)(N - 1 - n) * inner, zd);
+              } else {
+                d[(long long)n * inner] = za;
+                d[(long long)(N / 2 - 1 - n) * inner] = zb;
+                d[(long long)(N / 2 + n) * inner] = zc;
+                d[(long long)(N - 1 - n) * inner] = zd;
+              }
             }
           }
         }
       }
-    };
-    if (ntv == kNT) body(std::true_type{});
-    else body(std::false_type{});
-    __syncwarp();   // the next task's alpha, beta overwrite the buffer read above
+    }
   }
 }
 
@@ -465,16 +456,13 @@ size_t contract_smem(int N) {
 }
 
 template <int K>
-size_t expand_smem(int N) {
-  return (size_t)(N / 32) * ExpCfg<K>::KS * 4 * 32 * 16 + (size_t)(N / 2) * 4 + (size_t)(K + 1 + ((K + 1) & 1)) * 8 +
-         (size_t)kMmaWarps * ExpCfg<K>::WARP_FLOATS * 4;
-}
+size_t expand_smem(int N) { return (size_t)(N / 32) * 4 * 32 * 16 + (size_t)(N / 4) * 4; }
 
 template <int K>
 cudaError_t launch_mid_mma_t(bool forward, const float2* in, float2* out, long long outer, long long inner, int N,
                              float scale, cudaStream_t st) {
   const size_t smem = forward ? contract_smem<K>(N) : expand_smem<K>(N);
-  const int pos = forward ? kCPos : kTaskPos, warps = forward ? kCWarps : kMmaWarps, threads = warps * 32;
+  const int pos = forward ? kCPos : kEPos, warps = forward ? kCWarps : kEWarps, threads = warps * 32;
   const long long tasks = outer * ((inner + pos - 1) / pos);
   const long long want = (tasks + warps - 1) / warps;
   // persistent CTAs: exactly as many as are resident at once
@@ -501,7 +489,7 @@ cudaError_t launch_mid_mma_t(bool forward, const float2* in, float2* out, long l
     cudaError_t e = grid_for(kern, &grid);
     if (e != cudaSuccess) return e;
     const int streaming = (double)outer * N * inner * 8.0 > 2.0 * 126e6 ? 1 : 0;
-    kern<<<grid, threads, smem, st>>>(in, reinterpret_cast<float*>(out), outer, inner, N, scale, streaming);
+    kern<<<grid, threads, smem, st>>>(in, out, outer, inner, N, scale, streaming);
   }
   return cudaGetLastError();
 }
