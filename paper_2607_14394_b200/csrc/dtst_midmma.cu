@@ -1,34 +1,24 @@
-// Two-sided middle dimension on the tensor cores: the same folded contraction / expansion as dtst_mid.cu
+// Two-sided middle dimension on the tensor cores: the folded contraction / expansion of dtst_mid.cu
 // (Eq. 18 with zero offset, half-sample phase factored out),
 //     A_g = sum_{q<N/2} (z_q + z_{N-1-q}) cos(psi_g (q + 1/2)),   B_g = sum_{q<N/2} (z_q - z_{N-1-q}) sin(psi_g (q + 1/2)),
 //     Z_{+-g} = e^{+-i psi_g/2} (A_g -+ i B_g),
-// but with the sums over q as warp-level TF32 MMAs (hi/lo compensated, fp32 accumulate).  The complex tensor
-// [outer][N][inner] is read as a REAL matrix with 2*inner columns: the basis is real after the fold, so real
-// and imaginary parts are just neighbouring columns, and a C fragment's column pair (2 t4, 2 t4 + 1) is one
-// complex value.  The cosine frequencies g = 0..K-1 fill one 16-row MMA tile, the sine frequencies g = 1..K a
-// second one (row 0 carries g = K, whose sine partner g = 0 vanishes); the one left over, cos K, runs on FFMA.
+// folded a second time about the quarter points (even g: cosine even, sine odd; odd g the other way round), with the
+// sums over the row quadruples as warp-level TF32 MMAs (hi/lo compensated, fp32 accumulate).  The folded DATA is
+// the 16-row operand (8 complex positions: real parts in rows 0..7, imaginary parts in rows 8..15, so that a C
+// fragment holds whole complex values); the BASIS of one parity class (even cos, odd cos, odd sin, even sin:
+// K/2 <= 8 frequencies each) is the 8-column operand from a fragment-ordered shared table built once per persistent
+// CTA; the one frequency left over, cos K, runs on FFMA.
 //
-// On the FFMA version this stage was issue-bound (half of all instructions were the multiply-adds, the other
-// half their bookkeeping); here one task of 32 complex positions x N rows needs ~3x fewer instructions and the
-// stage becomes an HBM stream.  Shapes: N % 32 == 0, K in {4, 8, 12, 16}, inner % 4 == 0.
-#include <type_traits>
-
+// The FFMA version of this stage was issue-bound (half of all instructions were the multiply-adds, the other half
+// their bookkeeping); a first MMA version with one fold and the frequencies as the 16-row operand needed twice the
+// MMAs and was bound by the tensor pipe of the warp-level path.  Shapes: N % 32 == 0, K in {4, 8, 12, 16},
+// inner % 4 == 0.
 #include "dtst_common.cuh"
 #include "dtst_mma.cuh"
 
 namespace dtst {
 namespace {
 
-
-__device__ __forceinline__ float4 as_f4(const uint32_t (&v)[4]) {
-  return make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
-}
-__device__ __forceinline__ void from_f4(const float4 f, uint32_t (&v)[4]) {
-  v[0] = __float_as_uint(f.x);
-  v[1] = __float_as_uint(f.y);
-  v[2] = __float_as_uint(f.z);
-  v[3] = __float_as_uint(f.w);
-}
 
 // cos / sin of pi * g * (2 q + 1) / N with the phase reduced exactly in integers
 __device__ __forceinline__ void basis_cs(int g, int q, int N, float& cs, float& sn) {
