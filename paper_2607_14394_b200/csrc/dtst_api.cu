@@ -101,6 +101,14 @@ bool use_mid(const dtst_plan* p, int j) {
   return mid_supported((int)p->Ng[j], p->kmax[j]);
 }
 
+// Expansion of such a dimension: virtual slabs change nothing here - slab p's rows are the rows [p nl, (p+1) nl) of
+// the plain expansion (same global phases, no reduction between slabs), so the folded kernel serves them too.
+bool use_mid_expand(const dtst_plan* p, int j) {
+  if (p->path_request != DTST_PATH_AUTO || j >= p->d - 1) return false;
+  if (p->Nl[j] != p->Ng[j] || p->off[j] != 0) return false;
+  return mid_supported((int)p->Ng[j], p->kmax[j]);
+}
+
 // A two-sided dimension that carries a phase offset, is only partly local, or is cut into virtual slabs.
 bool use_slab(const dtst_plan* p, int j) {
   if (p->path_request != DTST_PATH_AUTO || j >= p->d - 1 || use_mid(p, j)) return false;
@@ -261,7 +269,12 @@ dtst_status run_inverse_generic(dtst_plan* p, const float2* Yhat, float* y, int 
       op.out_slab_stride = (long long)nl * op.inner;
     }
     void* dst = out_real ? static_cast<void*>(y) : static_cast<void*>(buf[flip]);
-    if (!out_real && use_slab(p, j)) {
+    if (!out_real && use_mid_expand(p, j)) {
+      if (cuda_failed(p, launch_mid(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
+                                    make_op(p, j, false, Cn).outer, make_op(p, j, false, Cn).inner, (int)p->Ng[j], 1.0f,
+                                    st)))
+        return DTST_ERR_CUDA;
+    } else if (!out_real && use_slab(p, j)) {
       if (cuda_failed(p, launch_slab(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
                                      make_op(p, j, false, Cn).outer, make_op(p, j, false, Cn).inner, (int)p->Nl[j],
                                      (int)p->Ng[j], (int)p->off[j], j == 0 ? p->P : 1, st)))
@@ -301,7 +314,12 @@ dtst_status inverse_stages_complex(dtst_plan* p, const float2* cur_in, int j_to,
       op.out_slab_stride = (long long)nl * op.inner;
     }
     void* dst = buf[flip];
-    if (use_slab(p, j)) {
+    if (use_mid_expand(p, j)) {
+      if (cuda_failed(p, launch_mid(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
+                                    make_op(p, j, false, Cn).outer, make_op(p, j, false, Cn).inner, (int)p->Ng[j], 1.0f,
+                                    st)))
+        return DTST_ERR_CUDA;
+    } else if (use_slab(p, j)) {
       if (cuda_failed(p, launch_slab(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
                                      make_op(p, j, false, Cn).outer, make_op(p, j, false, Cn).inner, (int)p->Nl[j],
                                      (int)p->Ng[j], (int)p->off[j], j == 0 ? p->P : 1, st)))
