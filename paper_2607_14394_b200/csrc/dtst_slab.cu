@@ -9,6 +9,7 @@
 // already reduced one, so this stays a small share of a step.  The basis table E[n][r] is generated on the
 // device into shared memory once per persistent CTA.
 #include "dtst_common.cuh"
+#include "dtst_mma.cuh"
 
 namespace dtst {
 namespace {
@@ -118,6 +119,188 @@ __global__ void __launch_bounds__(kSlabThreads) slab_expand_kernel(const float2*
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// The contraction on the tensor cores, for slabs whose row count is a multiple of 8 (and inner % 4 == 0).
+// No fold is possible, so this is the plain complex product written with real MMAs:
+//   M = 16 real columns = 8 complex positions (real parts | imaginary parts), the data as A operand;
+//   K = 8 rows of the slab per step;  N = 8 of the 2k retained frequencies, cos and sin tables as B operands.
+// A slab's partial spectrum is accumulated from zero (C = sum x cos, S = sum x sin; Z = (C_re + S_im) + i (C_im -
+// S_re)) and then added to the running total: Eq. 7, slabs in ascending order.  The input streams through a
+// per-warp cp.async ring as in the folded kernel.
+// ------------------------------------------------------------------------------------------
+constexpr int kSMT = 2;                       // m-tiles per task: 16 complex positions = 128 bytes per row
+constexpr int kSPos = 8 * kSMT;
+constexpr int kSWarps = 10;
+constexpr int kSStages = 6;
+constexpr int kSRow = 2 * kSPos + 8;          // floats per staged row (8 mod 32: conflict-free 8-byte loads)
+constexpr int kSStageFloats = 8 * kSRow;
+
+__device__ __forceinline__ void slab_cp_async16(float* smem_dst, const float* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+               : "memory");
+}
+
+template <int K>
+__global__ void __launch_bounds__(kSWarps * 32, 1)
+slab_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out, long long outer, long long inner,
+                         int Nl, int N, int off, int P) {
+  constexpr int NT = 2 * K / 8;                 // n-tiles over the 2k retained frequencies
+  extern __shared__ float4 slab_smem4[];
+  const int KS = Nl / 8;                        // k-steps over all local rows
+  const int ksl = KS / P;                       // k-steps per slab
+  float4* btab = slab_smem4;                    // [KS][NT][cos | sin][lane]
+  float* ringbase = reinterpret_cast<float*>(btab + (size_t)KS * NT * 2 * 32);
+
+  for (int e = threadIdx.x; e < KS * NT * 2 * 32; e += blockDim.x) {
+    const int l = e & 31, sn_tab = (e >> 5) & 1, nt = (e >> 6) % NT, ks = (e >> 6) / NT;
+    const int lg = l >> 2, lt = l & 3;          // B fragment: k = row lt (+4), n = frequency slot lg
+    const int sidx = mode_at(8 * nt + lg, K, N, 1);
+    uint32_t hi[2], lo[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const float2 t = twiddle(sidx, (long long)off + 8 * ks + lt + 4 * h, N, +1);   // (cos, sin) of the phase
+      split_tf32_rna(sn_tab ? t.y : t.x, hi[h], lo[h]);
+    }
+    btab[e] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(lo[0]), __uint_as_float(lo[1]));
+  }
+  __syncthreads();
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g8 = lane >> 2, t4 = lane & 3;
+  const long long cblocks = (inner + kSPos - 1) / kSPos;
+  const long long tasks = outer * cblocks;
+  const long long rs = 2 * inner;               // floats per row
+  const long long tstride = (long long)gridDim.x * kSWarps;
+  float* ring = ringbase + (size_t)warp * kSStages * kSStageFloats;
+
+  long long ptask = (long long)blockIdx.x * kSWarps + warp;
+  int pks = 0, pstage = 0;
+  const float* ptb = in;
+  bool pchunk_ok = false;
+  auto issue = [&]() {
+    if (ptask < tasks) {
+      if (pks == 0) {
+        const long long o = ptask / cblocks, cb = ptask % cblocks;
+        const long long left = inner - cb * kSPos;
+        const int nch = left >= kSPos ? kSPos / 2 : (int)(left / 2);
+        ptb = in + o * Nl * rs + cb * (2 * kSPos) + 4 * (lane & 7);
+        pchunk_ok = (lane & 7) < nch;
+      }
+      if (pchunk_ok) {
+        float* dst = ring + pstage * kSStageFloats + (lane >> 3) * kSRow + 4 * (lane & 7);
+        const int n = 8 * pks + (lane >> 3);
+        slab_cp_async16(dst, ptb + (long long)n * rs);
+        slab_cp_async16(dst + 4 * kSRow, ptb + (long long)(n + 4) * rs);
+      }
+      if (++pks == KS) {
+        pks = 0;
+        ptask += tstride;
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    pstage = pstage + 1 == kSStages ? 0 : pstage + 1;
+  };
+#pragma unroll
+  for (int i = 0; i < kSStages - 1; ++i) issue();
+
+  int cstage = 0;
+  for (long long task = (long long)blockIdx.x * kSWarps + warp; task < tasks; task += tstride) {
+    const long long o = task / cblocks, cb = task % cblocks;
+    const long long left = inner - cb * kSPos;
+    const int mtv = left >= kSPos ? kSMT : (int)((left + 7) / 8);
+    float tot[kSMT][NT][4];
+#pragma unroll
+    for (int mt = 0; mt < kSMT; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) tot[mt][nt][e] = 0.f;
+
+#pragma unroll 1
+    for (int slab = 0; slab < P; ++slab) {
+      float aC[kSMT][NT][4], aS[kSMT][NT][4];
+#pragma unroll
+      for (int mt = 0; mt < kSMT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) aC[mt][nt][e] = aS[mt][nt][e] = 0.f;
+#pragma unroll 1
+      for (int k = 0; k < ksl; ++k) {
+        const int ks = slab * ksl + k;
+        asm volatile("cp.async.wait_group %0;" ::"n"(kSStages - 2) : "memory");
+        __syncwarp();
+        issue();
+        const float* S = ring + cstage * kSStageFloats + t4 * kSRow + 2 * g8;
+        const float4* bt = btab + (size_t)(ks * NT * 2) * 32 + lane;
+#pragma unroll
+        for (int mt = 0; mt < kSMT; ++mt) {
+          if (mt < mtv) {
+            const float2 lo_row = *reinterpret_cast<const float2*>(S + 16 * mt);
+            const float2 hi_row = *reinterpret_cast<const float2*>(S + 4 * kSRow + 16 * mt);
+            uint32_t ah[4], al[4];
+            split_tf32_round(lo_row.x, ah[0], al[0]);
+            split_tf32_round(lo_row.y, ah[1], al[1]);
+            split_tf32_round(hi_row.x, ah[2], al[2]);
+            split_tf32_round(hi_row.y, ah[3], al[3]);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              const float4 bc = bt[(nt * 2 + 0) * 32], bs = bt[(nt * 2 + 1) * 32];
+              mma3_tf32(aC[mt][nt], ah, al, __float_as_uint(bc.x), __float_as_uint(bc.y), __float_as_uint(bc.z),
+                        __float_as_uint(bc.w));
+              mma3_tf32(aS[mt][nt], ah, al, __float_as_uint(bs.x), __float_as_uint(bs.y), __float_as_uint(bs.z),
+                        __float_as_uint(bs.w));
+            }
+          }
+        }
+        cstage = cstage + 1 == kSStages ? 0 : cstage + 1;
+      }
+      // Eq. 7: this slab's partial spectrum, then onto the total (slabs in ascending order).
+      // Fragments: (re, slot 2 t4) (re, slot 2 t4 + 1) (im, 2 t4) (im, 2 t4 + 1) of position g8.
+#pragma unroll
+      for (int mt = 0; mt < kSMT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          tot[mt][nt][0] += aC[mt][nt][0] + aS[mt][nt][2];
+          tot[mt][nt][1] += aC[mt][nt][1] + aS[mt][nt][3];
+          tot[mt][nt][2] += aC[mt][nt][2] - aS[mt][nt][0];
+          tot[mt][nt][3] += aC[mt][nt][3] - aS[mt][nt][1];
+        }
+    }
+#pragma unroll
+    for (int mt = 0; mt < kSMT; ++mt) {
+      const long long pos = cb * kSPos + 8 * mt + g8;
+      if (mt < mtv && pos < inner) {
+        float2* dst = out + o * (2 * K) * inner + pos;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          dst[(long long)(8 * nt + 2 * t4) * inner] = make_float2(tot[mt][nt][0], tot[mt][nt][2]);
+          dst[(long long)(8 * nt + 2 * t4 + 1) * inner] = make_float2(tot[mt][nt][1], tot[mt][nt][3]);
+        }
+      }
+    }
+  }
+}
+
+template <int K>
+size_t slab_mma_smem(int Nl) {
+  return (size_t)(Nl / 8) * (2 * K / 8) * 2 * 32 * 16 + (size_t)kSWarps * kSStages * kSStageFloats * 4;
+}
+
+template <int K>
+cudaError_t launch_slab_mma_t(const float2* in, float2* out, long long outer, long long inner, int Nl, int N, int off,
+                              int P, cudaStream_t st) {
+  const size_t smem = slab_mma_smem<K>(Nl);
+  auto kern = slab_contract_mma_kernel<K>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  const long long tasks = outer * ((inner + kSPos - 1) / kSPos);
+  const long long want = (tasks + kSWarps - 1) / kSWarps;
+  const int grid = (int)(want < kNumSMs ? want : kNumSMs);
+  kern<<<grid, kSWarps * 32, smem, st>>>(reinterpret_cast<const float*>(in), out, outer, inner, Nl, N, off, P);
+  return cudaGetLastError();
+}
+
 template <int K>
 cudaError_t launch_slab_t(bool forward, const float2* in, float2* out, long long outer, long long inner, int Nl, int N,
                           int off, int P, cudaStream_t st) {
@@ -149,6 +332,18 @@ bool slab_supported(int Nl, int K) {
 cudaError_t launch_slab(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int Nl,
                         int N, int off, int P, cudaStream_t st) {
   if (outer * inner <= 0) return cudaSuccess;
+  // contraction of slabs that are whole k-steps of 8 rows: tensor-core kernel
+  const bool aligned16 = ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
+  if (forward && aligned16 && inner % 4 == 0 && P >= 1 && Nl % P == 0 && (Nl / P) % 8 == 0) {
+    const size_t lim = 227 * 1024;
+    switch (K) {
+      case 4: if (slab_mma_smem<4>(Nl) <= lim) return launch_slab_mma_t<4>(in, out, outer, inner, Nl, N, off, P, st); break;
+      case 8: if (slab_mma_smem<8>(Nl) <= lim) return launch_slab_mma_t<8>(in, out, outer, inner, Nl, N, off, P, st); break;
+      case 12: if (slab_mma_smem<12>(Nl) <= lim) return launch_slab_mma_t<12>(in, out, outer, inner, Nl, N, off, P, st); break;
+      case 16: if (slab_mma_smem<16>(Nl) <= lim) return launch_slab_mma_t<16>(in, out, outer, inner, Nl, N, off, P, st); break;
+      default: break;
+    }
+  }
   switch (K) {
     case 4: return launch_slab_t<4>(forward, in, out, outer, inner, Nl, N, off, P, st);
     case 8: return launch_slab_t<8>(forward, in, out, outer, inner, Nl, N, off, P, st);
