@@ -146,7 +146,8 @@ bool slab_supported(int Nl, int K);
 cudaError_t launch_slab(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int Nl,
                         int N, int off, int P, cudaStream_t st);
 
-// folded register-accumulator kernels for a two-sided middle dimension (dtst_mid.cu)
+// folded kernels for a two-sided middle dimension: tensor-core version (dtst_midmma.cu) where the shape allows,
+// else the FFMA register-accumulator version (dtst_mid.cu)
 bool mid_supported(int N, int K);
 // tensor-core variant of the middle-dimension kernels (N % 32 == 0, inner % 4 == 0)
 bool mid_mma_supported(int N, int K, long long inner);
