@@ -314,6 +314,42 @@ def torch_fft_reference(torch, w, x, W, g, steps=3):
     return out
 
 
+def virtual_shard_summary(torch, w, x, g, W, P, steps=10):
+    """The headline workload once more with its dimension 0 cut into P virtual slabs (partial spectra with global
+    phase offsets, summed on the device in ascending order): step time beside the unsharded one."""
+    from paper_2607_14394_b200 import Plan
+    try:
+        plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out, virtual_shards=P)
+        X = plan.forward(x)
+        Y = plan.spectral_mul(X, W)
+        y = plan.inverse(Y)
+        gx, gW = plan.backward(g, X, W)
+
+        def step():
+            plan.forward(x, X)
+            plan.spectral_mul(X, W, Y)
+            plan.inverse(Y, y)
+            plan.backward(g, X, W, gx, gW)
+
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        ok = plan.status() == 0
+        plan.close()
+        del plan, X, Y, y, gx, gW
+        torch.cuda.empty_cache()
+        return {"P": P, "ms_per_step": ms, "gpoints_per_s": w.B * w.points / ms / 1e6, "status_ok": ok, "steps": steps}
+    except Exception as ex:
+        return {"P": P, "error": f"{type(ex).__name__}: {ex}"[:200]}
+
+
 def other_configs_summary(torch, skip_name, steps=10):
     """Forward and forward+backward time of the other benchmark configurations (parity-test cases, not the
     headline): seeded device-generated inputs of each shape, CUDA events, 3 warm-ups."""
@@ -579,6 +615,8 @@ def main_ours(args, w):
     # secondary reference and CPU baseline: rank 0, single GPU only
     if rank == 0 and world == 1:
         torch.cuda.empty_cache()
+        if not args.no_other_configs and args.channels == 0 and P == 1 and w.virtual_shards > 1:
+            line["virtual_shards"] = virtual_shard_summary(torch, w, x, g, W, w.virtual_shards, steps=min(steps, 10))
         if not args.no_torch_ref:
             line["torch_fft_reference"] = torch_fft_reference(torch, w, x, W, g)
         if not args.no_other_configs and args.channels == 0:
