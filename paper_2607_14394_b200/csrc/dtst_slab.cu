@@ -128,9 +128,9 @@ __global__ void __launch_bounds__(kSlabThreads) slab_expand_kernel(const float2*
 // S_re)) and then added to the running total: Eq. 7, slabs in ascending order.  The input streams through a
 // per-warp cp.async ring as in the folded kernel.
 // ------------------------------------------------------------------------------------------
-constexpr int kSMT = 2;                       // m-tiles per task: 16 complex positions = 128 bytes per row
+constexpr int kSMT = 1;                       // m-tiles per task: 8 complex positions = 64 bytes per row
 constexpr int kSPos = 8 * kSMT;
-constexpr int kSWarps = 10;
+constexpr int kSWarps = 16;
 constexpr int kSStages = 6;
 constexpr int kSRow = 2 * kSPos + 8;          // floats per staged row (8 mod 32: conflict-free 8-byte loads)
 constexpr int kSStageFloats = 8 * kSRow;
@@ -144,25 +144,30 @@ template <int K>
 __global__ void __launch_bounds__(kSWarps * 32, 1)
 slab_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out, long long outer, long long inner,
                          int Nl, int N, int off, int P) {
-  constexpr int NT = 2 * K / 8;                 // n-tiles over the 2k retained frequencies
+  // +g and -g share their sums: C_g = sum_n z_n cos(phi_g (off + n)), S_g = sum_n z_n sin(phi_g (off + n)),
+  // Z_{+g} = C_g - i S_g, Z_{-g} = C_g + i S_g, phi_g = 2 pi g / N.  The MMA n-tiles cover g = 0..K-1; g = K (only
+  // -K is retained) runs on FFMA.
+  constexpr int NT = (K + 7) / 8;
   extern __shared__ float4 slab_smem4[];
   const int KS = Nl / 8;                        // k-steps over all local rows
   const int ksl = KS / P;                       // k-steps per slab
   float4* btab = slab_smem4;                    // [KS][NT][cos | sin][lane]
-  float* ringbase = reinterpret_cast<float*>(btab + (size_t)KS * NT * 2 * 32);
+  float2* tK = reinterpret_cast<float2*>(btab + (size_t)KS * NT * 2 * 32);   // (cos, sin)(phi_K (off + n)), n < Nl
+  float* ringbase = reinterpret_cast<float*>(tK + Nl);
 
   for (int e = threadIdx.x; e < KS * NT * 2 * 32; e += blockDim.x) {
     const int l = e & 31, sn_tab = (e >> 5) & 1, nt = (e >> 6) % NT, ks = (e >> 6) / NT;
     const int lg = l >> 2, lt = l & 3;          // B fragment: k = row lt (+4), n = frequency slot lg
-    const int sidx = mode_at(8 * nt + lg, K, N, 1);
+    const int g = 8 * nt + lg;
     uint32_t hi[2], lo[2];
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      const float2 t = twiddle(sidx, (long long)off + 8 * ks + lt + 4 * h, N, +1);   // (cos, sin) of the phase
-      split_tf32_rna(sn_tab ? t.y : t.x, hi[h], lo[h]);
+      const float2 t = twiddle(g, (long long)off + 8 * ks + lt + 4 * h, N, +1);   // (cos, sin) of the phase
+      split_tf32_rna(g < K ? (sn_tab ? t.y : t.x) : 0.f, hi[h], lo[h]);
     }
     btab[e] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(lo[0]), __uint_as_float(lo[1]));
   }
+  for (int n = threadIdx.x; n < Nl; n += blockDim.x) tK[n] = twiddle(K, (long long)off + n, N, +1);
   __syncthreads();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -208,23 +213,28 @@ slab_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out,
     const long long o = task / cblocks, cb = task % cblocks;
     const long long left = inner - cb * kSPos;
     const int mtv = left >= kSPos ? kSMT : (int)((left + 7) / 8);
-    float tot[kSMT][NT][4];
+    // totals: Z_{+g} and Z_{-g} as (re, slot 2 t4) (re, slot 2 t4 + 1) (im, 2 t4) (im, 2 t4 + 1); Z_{-K} as (re, im)
+    float totp[kSMT][NT][4], totm[kSMT][NT][4], totK[kSMT][2];
 #pragma unroll
-    for (int mt = 0; mt < kSMT; ++mt)
+    for (int mt = 0; mt < kSMT; ++mt) {
+      totK[mt][0] = totK[mt][1] = 0.f;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) tot[mt][nt][e] = 0.f;
+        for (int e = 0; e < 4; ++e) totp[mt][nt][e] = totm[mt][nt][e] = 0.f;
+    }
 
 #pragma unroll 1
     for (int slab = 0; slab < P; ++slab) {
-      float aC[kSMT][NT][4], aS[kSMT][NT][4];
+      float aC[kSMT][NT][4], aS[kSMT][NT][4], cK[kSMT][2], sK[kSMT][2];
 #pragma unroll
-      for (int mt = 0; mt < kSMT; ++mt)
+      for (int mt = 0; mt < kSMT; ++mt) {
+        cK[mt][0] = cK[mt][1] = sK[mt][0] = sK[mt][1] = 0.f;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
           for (int e = 0; e < 4; ++e) aC[mt][nt][e] = aS[mt][nt][e] = 0.f;
+      }
 #pragma unroll 1
       for (int k = 0; k < ksl; ++k) {
         const int ks = slab * ksl + k;
@@ -233,11 +243,16 @@ slab_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out,
         issue();
         const float* S = ring + cstage * kSStageFloats + t4 * kSRow + 2 * g8;
         const float4* bt = btab + (size_t)(ks * NT * 2) * 32 + lane;
+        const float2 tk0 = tK[8 * ks + t4], tk1 = tK[8 * ks + t4 + 4];
 #pragma unroll
         for (int mt = 0; mt < kSMT; ++mt) {
           if (mt < mtv) {
             const float2 lo_row = *reinterpret_cast<const float2*>(S + 16 * mt);
             const float2 hi_row = *reinterpret_cast<const float2*>(S + 4 * kSRow + 16 * mt);
+            cK[mt][0] = fmaf(lo_row.x, tk0.x, fmaf(hi_row.x, tk1.x, cK[mt][0]));
+            cK[mt][1] = fmaf(lo_row.y, tk0.x, fmaf(hi_row.y, tk1.x, cK[mt][1]));
+            sK[mt][0] = fmaf(lo_row.x, tk0.y, fmaf(hi_row.x, tk1.y, sK[mt][0]));
+            sK[mt][1] = fmaf(lo_row.y, tk0.y, fmaf(hi_row.y, tk1.y, sK[mt][1]));
             uint32_t ah[4], al[4];
             split_tf32_round(lo_row.x, ah[0], al[0]);
             split_tf32_round(lo_row.y, ah[1], al[1]);
@@ -255,17 +270,33 @@ slab_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out,
         }
         cstage = cstage + 1 == kSStages ? 0 : cstage + 1;
       }
-      // Eq. 7: this slab's partial spectrum, then onto the total (slabs in ascending order).
-      // Fragments: (re, slot 2 t4) (re, slot 2 t4 + 1) (im, 2 t4) (im, 2 t4 + 1) of position g8.
+      // Eq. 7: this slab's partial spectrum, then onto the totals (slabs in ascending order).
 #pragma unroll
-      for (int mt = 0; mt < kSMT; ++mt)
+      for (int mt = 0; mt < kSMT; ++mt) {
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-          tot[mt][nt][0] += aC[mt][nt][0] + aS[mt][nt][2];
-          tot[mt][nt][1] += aC[mt][nt][1] + aS[mt][nt][3];
-          tot[mt][nt][2] += aC[mt][nt][2] - aS[mt][nt][0];
-          tot[mt][nt][3] += aC[mt][nt][3] - aS[mt][nt][1];
+          // Z_{+g} = C - iS: (C_re + S_im, C_im - S_re);  Z_{-g} = C + iS: (C_re - S_im, C_im + S_re)
+          totp[mt][nt][0] += aC[mt][nt][0] + aS[mt][nt][2];
+          totp[mt][nt][1] += aC[mt][nt][1] + aS[mt][nt][3];
+          totp[mt][nt][2] += aC[mt][nt][2] - aS[mt][nt][0];
+          totp[mt][nt][3] += aC[mt][nt][3] - aS[mt][nt][1];
+          totm[mt][nt][0] += aC[mt][nt][0] - aS[mt][nt][2];
+          totm[mt][nt][1] += aC[mt][nt][1] - aS[mt][nt][3];
+          totm[mt][nt][2] += aC[mt][nt][2] + aS[mt][nt][0];
+          totm[mt][nt][3] += aC[mt][nt][3] + aS[mt][nt][1];
         }
+        // Z_{-K} of this slab: the quad's lanes covered rows t4, t4 + 4 of every k-step
+        float cr = cK[mt][0], ci = cK[mt][1], sr = sK[mt][0], si = sK[mt][1];
+#pragma unroll
+        for (int m = 1; m <= 2; m <<= 1) {
+          cr += __shfl_xor_sync(0xffffffffu, cr, m);
+          ci += __shfl_xor_sync(0xffffffffu, ci, m);
+          sr += __shfl_xor_sync(0xffffffffu, sr, m);
+          si += __shfl_xor_sync(0xffffffffu, si, m);
+        }
+        totK[mt][0] += cr - si;
+        totK[mt][1] += ci + sr;
+      }
     }
 #pragma unroll
     for (int mt = 0; mt < kSMT; ++mt) {
@@ -273,10 +304,16 @@ slab_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out,
       if (mt < mtv && pos < inner) {
         float2* dst = out + o * (2 * K) * inner + pos;
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-          dst[(long long)(8 * nt + 2 * t4) * inner] = make_float2(tot[mt][nt][0], tot[mt][nt][2]);
-          dst[(long long)(8 * nt + 2 * t4 + 1) * inner] = make_float2(tot[mt][nt][1], tot[mt][nt][3]);
-        }
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            const int g = 8 * nt + 2 * t4 + q;
+            if (g < K) {
+              dst[(long long)g * inner] = make_float2(totp[mt][nt][q], totp[mt][nt][2 + q]);
+              if (g > 0) dst[(long long)(2 * K - g) * inner] = make_float2(totm[mt][nt][q], totm[mt][nt][2 + q]);
+            }
+          }
+        if (t4 == 0) dst[(long long)K * inner] = make_float2(totK[mt][0], totK[mt][1]);
       }
     }
   }
@@ -284,7 +321,7 @@ slab_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out,
 
 template <int K>
 size_t slab_mma_smem(int Nl) {
-  return (size_t)(Nl / 8) * (2 * K / 8) * 2 * 32 * 16 + (size_t)kSWarps * kSStages * kSStageFloats * 4;
+  return (size_t)(Nl / 8) * ((K + 7) / 8) * 2 * 32 * 16 + (size_t)Nl * 8 + (size_t)kSWarps * kSStages * kSStageFloats * 4;
 }
 
 template <int K>
