@@ -258,13 +258,28 @@ slab_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out,
             split_tf32_round(lo_row.y, ah[1], al[1]);
             split_tf32_round(hi_row.x, ah[2], al[2]);
             split_tf32_round(hi_row.y, ah[3], al[3]);
+            // the three compensated products of an accumulator depend on one another: issue them interleaved
+            // over the 2 NT accumulators
+            float4 bc[NT], bs[NT];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-              const float4 bc = bt[(nt * 2 + 0) * 32], bs = bt[(nt * 2 + 1) * 32];
-              mma3_tf32(aC[mt][nt], ah, al, __float_as_uint(bc.x), __float_as_uint(bc.y), __float_as_uint(bc.z),
-                        __float_as_uint(bc.w));
-              mma3_tf32(aS[mt][nt], ah, al, __float_as_uint(bs.x), __float_as_uint(bs.y), __float_as_uint(bs.z),
-                        __float_as_uint(bs.w));
+              bc[nt] = bt[(nt * 2 + 0) * 32];
+              bs[nt] = bt[(nt * 2 + 1) * 32];
+            }
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              mma_m16n8k8_tf32(aC[mt][nt], ah, __float_as_uint(bc[nt].x), __float_as_uint(bc[nt].y));
+              mma_m16n8k8_tf32(aS[mt][nt], ah, __float_as_uint(bs[nt].x), __float_as_uint(bs[nt].y));
+            }
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              mma_m16n8k8_tf32(aC[mt][nt], al, __float_as_uint(bc[nt].x), __float_as_uint(bc[nt].y));
+              mma_m16n8k8_tf32(aS[mt][nt], al, __float_as_uint(bs[nt].x), __float_as_uint(bs[nt].y));
+            }
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              mma_m16n8k8_tf32(aC[mt][nt], ah, __float_as_uint(bc[nt].z), __float_as_uint(bc[nt].w));
+              mma_m16n8k8_tf32(aS[mt][nt], ah, __float_as_uint(bs[nt].z), __float_as_uint(bs[nt].w));
             }
           }
         }
