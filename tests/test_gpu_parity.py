@@ -147,7 +147,10 @@ def test_random_shapes(case):
 # ------------------------------------------------------------------ virtual shards (Eq. 6-7 on one GPU)
 @pytest.mark.parametrize("N,k,P", [((16, 8, 12), (3, 2, 4), 4), ((16, 8, 12), (3, 2, 4), 16),
                                    ((64, 64), (8, 8), 8), ((8,), (3,), 2),
-                                   ((64, 32, 32, 16), (8, 4, 4, 4), 8)])
+                                   ((64, 32, 32, 16), (8, 4, 4, 4), 8),
+                                   # slabs of whole 8-row steps: the tensor-core slab contraction, with column tails
+                                   ((128, 64, 32), (16, 16, 4), 8), ((96, 32, 36), (12, 4, 9), 3),
+                                   ((64, 128), (16, 12), 8)])
 @pytest.mark.parametrize("path", ["auto", "generic"])
 def test_virtual_shards_match_oracle_and_unsharded(N, k, P, path):
     w = I.custom_workload("shards", 2, 2, 3, N, k, field="grf", seed=23)
