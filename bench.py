@@ -314,6 +314,34 @@ def torch_fft_reference(torch, w, x, W, g, steps=3):
     return out
 
 
+def graph_step_ms(torch, step_fn, steps=10):
+    """One step captured in a CUDA graph (the compute calls allocate nothing and never synchronise, so they can be
+    captured as they are) and replayed: the step time without per-launch host overhead."""
+    try:
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            step_fn()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                step_fn()
+        torch.cuda.synchronize()
+        for _ in range(3):
+            graph.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        del graph
+        return ms
+    except Exception as ex:
+        return f"{type(ex).__name__}: {ex}"[:160]
+
+
 def virtual_shard_summary(torch, w, x, g, W, P, steps=10):
     """The headline workload once more with its dimension 0 cut into P virtual slabs (partial spectra with global
     phase offsets, summed on the device in ascending order): step time beside the unsharded one."""
@@ -390,12 +418,19 @@ def other_configs_summary(torch, skip_name, steps=10):
             e[2].record()
             torch.cuda.synchronize()
             tf, tb = e[0].elapsed_time(e[1]) / steps, e[1].elapsed_time(e[2]) / steps
+
+            def whole_step():
+                fwd()
+                plan.backward(g, X, W, gx, gW)
+
+            tg = graph_step_ms(torch, whole_step, steps)
             ab = algorithmic_bytes(w)
             pts = w.B * w.points
             out[name] = {"kernel_path": plan.kernel_path, "fwd_ms": tf, "fwd_bwd_ms": tf + tb,
                          "fwd_gpoints_per_s": pts / tf / 1e6, "fwd_bwd_gpoints_per_s": pts / (tf + tb) / 1e6,
                          "fwd_algorithmic_gbs": ab["fwd"] / tf / 1e6,
                          "fwd_bwd_algorithmic_gbs": ab["fwd_bwd"] / (tf + tb) / 1e6,
+                         "fwd_bwd_cuda_graph_ms": tg,
                          "grid_bytes": 4 * w.C_in * pts,
                          "note": "grid smaller than L2: warm-cache, launch-bound" if 4 * w.C_in * pts < 126e6 else
                                  "grid larger than L2"}
@@ -482,6 +517,8 @@ def main_ours(args, w):
     ph = [sum(phase_events[i][j].elapsed_time(phase_events[i][j + 1]) for i in range(steps)) / steps for j in range(4)]
     kt = {k: plan.kernel_timing(k) for k in ("grid_read", "grid_write", "mix", "mix_adjoint")}
     plan.enable_kernel_timing(0)
+    graph_ms = graph_step_ms(torch, step, min(steps, 10)) if (rank == 0 and world == 1 and
+                                                             not args.no_other_configs) else None
 
     red = D.max_over_ranks([ms_step] + ph, device=dev)
     ms_step, ph = red[0], red[1:]
@@ -615,6 +652,9 @@ def main_ours(args, w):
     # secondary reference and CPU baseline: rank 0, single GPU only
     if rank == 0 and world == 1:
         torch.cuda.empty_cache()
+        if graph_ms is not None:
+            line["cuda_graph"] = {"ms_per_step": graph_ms,
+                                  "what": "the same step captured once in a CUDA graph and replayed"}
         if not args.no_other_configs and args.channels == 0 and P == 1 and w.virtual_shards > 1:
             line["virtual_shards"] = virtual_shard_summary(torch, w, x, g, W, w.virtual_shards, steps=min(steps, 10))
         if not args.no_torch_ref:

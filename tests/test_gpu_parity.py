@@ -279,6 +279,42 @@ def test_adjoint_identity_on_device():
     assert abs(lhs - rhs) <= 1e-5 * max(1.0, abs(lhs))
 
 
+def test_step_can_be_captured_in_a_cuda_graph():
+    # the compute calls allocate nothing and never synchronise: a whole step captures as it is and replays bit for bit
+    w = I.custom_workload("graph", 2, 3, 2, (32, 32, 64), (4, 8, 8), field="grf", seed=41)
+    plan = _plan(w)
+    x, W, g = _dev(I.make_field(w)), _dev(I.make_weights(w)), _dev(I.make_upstream_grad(w))
+    X = plan.forward(x)
+    Y = plan.spectral_mul(X, W)
+    y = plan.inverse(Y)
+    gx, gW = plan.backward(g, X, W)
+
+    def step():
+        plan.forward(x, X)
+        plan.spectral_mul(X, W, Y)
+        plan.inverse(Y, y)
+        plan.backward(g, X, W, gx, gW)
+
+    step()
+    torch.cuda.synchronize()
+    ref = [t.clone() for t in (X, Y, y, gx, gW)]
+    side, graph = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        step()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    torch.cuda.synchronize()
+    for t in (X, Y, y, gx, gW):
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert plan.status() == 0
+    for got, want in zip((X, Y, y, gx, gW), ref):
+        assert torch.equal(torch.view_as_real(got) if got.is_complex() else got,
+                           torch.view_as_real(want) if want.is_complex() else want)
+
+
 def test_host_pipeline_matches_device_path_over_consecutive_steps():
     # pinned host buffers in and out, copies overlapped with compute on three streams: same bits as the plain path
     from paper_2607_14394_b200 import Plan
