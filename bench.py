@@ -141,17 +141,34 @@ class ClockSampler:
         return out
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the two grid-streaming kernels, from one
-# ncu capture of a small case of the same shape (2 channels instead of 16, 1.07 GB of grid: larger than L2, small
-# enough for a multi-pass capture) scaled by the channel ratio 8 - their traffic is proportional to the channel
-# count.  The summary with the command line is profiles/kernels_cfg5_shape_c2_ncu_full.md.
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the two grid-streaming kernels from ncu
+# captures of the same kernels at the same shape with FEWER CHANNELS (the capture-size rule: a few GB on the device
+# at most under a multi-pass capture).  Two captures (2 and 4 channels) give a line: the slope is the traffic per
+# channel, the intercept what does not grow with the tensor (a store stream's last dirty lines are still in L2 when
+# the kernel ends and are counted by nobody), so the full launch is intercept + slope * channels instead of a
+# plain scaling of one capture.  The summaries with their command lines are under profiles/.
 NCU_TRAFFIC = {
-    "cfg5_4d_128": {"grid_read": 8 * (1073788000 + 64662000), "grid_write": 8 * (67159000 + 1018316000)},
+    "cfg5_4d_128": {
+        "channels": (2, 4),
+        "grid_read": ((1073788000 + 64662000), None),      # (read + write) bytes at 2 and at 4 channels
+        "grid_write": ((67159000 + 1018316000), None),
+        "source": "profiles/kernels_cfg5_shape_c2_ncu_full.md",
+    },
 }
 
 
-def measured_traffic(workload: str, kind: str):
-    return NCU_TRAFFIC.get(workload, {}).get(kind)
+def measured_traffic(workload: str, kind: str, channels: int):
+    """Extrapolated DRAM traffic of one launch at `channels` channels, or None without a capture."""
+    rec = NCU_TRAFFIC.get(workload)
+    if not rec or kind not in rec:
+        return None
+    (c0, c1), (t0, t1) = rec["channels"], rec[kind]
+    if t0 is None:
+        return None
+    if t1 is None:                       # one capture only: plain scaling (under-counts the fixed L2 residue)
+        return t0 * channels / c0
+    slope = (t1 - t0) / (c1 - c0)
+    return t0 + slope * (channels - c0)
 
 
 def algorithmic_bytes(w):
@@ -203,37 +220,60 @@ def oracle_data(w, cs, n0):
     return x, W, g
 
 
-def time_oracle(w, steps, warmup, budget=1.7e7):
+ORACLE_BUDGET = 1.7e7      # point-channels per sample step: about a second of oracle work on 8 cores
+
+
+def time_oracle(w, steps, warmup, budget=ORACLE_BUDGET, one_core=True):
+    """Times the oracle as it stands on a bounded sample of the workload: `warmup` untimed steps (at least one),
+    then `steps` timed ones, mean and min; then the same on ONE core (threadpoolctl) when asked."""
     try:
-        from threadpoolctl import threadpool_info
+        from threadpoolctl import threadpool_info, threadpool_limits
         threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
     except Exception:
+        threadpool_limits = None
         threads = len(os.sched_getaffinity(0))
     cs, n0 = oracle_sample_spec(w, budget)
     data = oracle_data(w, cs, n0)
-    for _ in range(warmup):
-        run_oracle_step(w, cs, n0, data)
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        run_oracle_step(w, cs, n0, data)
-    dt = (time.perf_counter() - t0) / steps
+
+    def run(n_warm, n_steps):
+        for _ in range(n_warm):
+            run_oracle_step(w, cs, n0, data)
+        ts = []
+        for _ in range(n_steps):
+            t0 = time.perf_counter()
+            run_oracle_step(w, cs, n0, data)
+            ts.append(time.perf_counter() - t0)
+        return sum(ts) / len(ts), min(ts)
+
+    dt, dt_min = run(max(1, warmup), max(1, steps))
     sample_ptch = w.B * (w.points // w.N[0]) * n0 * cs
     # equivalent whole-layer grid points per second at the workload's channel count
-    value = sample_ptch / max(w.C_in, w.C_out) / dt / 1e9
+    to_value = lambda t: sample_ptch / max(w.C_in, w.C_out) / t / 1e9
+    value = to_value(dt)
     grid_part = (f"the whole grid" if n0 == w.N[0] else
                  f"first {n0} of {w.N[0]} planes along dim 0 (a slab, with its global phase offset)")
     sample = (f"float64 numpy oracle, fwd+bwd, {cs} of {w.C_in} channels (in and out), {grid_part}; "
-              f"value = sample point-channels / {max(w.C_in, w.C_out)} channels / time")
-    return value, dt, {"kind": "oracle", "cores": int(min(threads, len(os.sched_getaffinity(0)))),
-                       "host_cores": len(os.sched_getaffinity(0)), "sample": sample,
-                       "seconds_per_sample_step": dt}
+              f"value = sample point-channels / {max(w.C_in, w.C_out)} channels / time; "
+              f"{max(1, warmup)} warm-up + {max(1, steps)} timed sample steps, mean (min also given)")
+    info = {"kind": "oracle", "cores": int(min(threads, len(os.sched_getaffinity(0)))),
+            "host_cores": len(os.sched_getaffinity(0)), "sample": sample,
+            "seconds_per_sample_step": dt, "seconds_per_sample_step_min": dt_min, "value_at_min": to_value(dt_min)}
+    if one_core and threadpool_limits is not None:
+        try:
+            with threadpool_limits(limits=1):
+                dt1, dt1_min = run(0, max(1, min(steps, 2)))
+            info["one_core"] = {"value": to_value(dt1), "unit": UNIT, "cores": 1, "seconds_per_sample_step": dt1,
+                                "seconds_per_sample_step_min": dt1_min}
+        except Exception as ex:
+            info["one_core"] = {"error": f"{type(ex).__name__}: {ex}"[:120]}
+    return value, dt, info
 
 
 def main_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    steps, warmup = max(1, args.steps), max(0, args.warmup)
+    steps, warmup = max(1, args.steps), max(1, args.warmup)
     value, dt, info = time_oracle(w, steps, warmup)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
@@ -342,9 +382,77 @@ def graph_step_ms(torch, step_fn, steps=10):
         return f"{type(ex).__name__}: {ex}"[:160]
 
 
-def virtual_shard_summary(torch, w, x, g, W, P, steps=10):
+def timed_steps(torch, plan, tensors, steps, barrier=None, sampler=None):
+    """`steps` whole steps (F, M, I, B) between two synchronisations, CUDA events on the launching stream around the
+    region and around each phase, the library's own events around the dominant kernels.  Returns the step time,
+    the phase split, the per-kernel-kind launch record and the number of kernel launches."""
+    x, g, W, Xhat, Yhat, y, gx, gW = tensors
+
+    def step(evs=None):
+        if evs is not None:
+            evs[0].record()
+        plan.forward(x, Xhat)
+        if evs is not None:
+            evs[1].record()
+        plan.spectral_mul(Xhat, W, Yhat)
+        if evs is not None:
+            evs[2].record()
+        plan.inverse(Yhat, y)
+        if evs is not None:
+            evs[3].record()
+        plan.backward(g, Xhat, W, gx, gW)
+        if evs is not None:
+            evs[4].record()
+
+    plan.enable_kernel_timing(2 * steps + 2)
+    phase_events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
+    launches0 = plan.launch_count()
+    if barrier:
+        barrier()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_start.record()
+    for i in range(steps):
+        step(phase_events[i])
+    t_end.record()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    clocks = sampler.stop() if sampler else None
+    launches = plan.launch_count() - launches0
+    ms_step = t_start.elapsed_time(t_end) / steps
+    ph = [sum(phase_events[i][j].elapsed_time(phase_events[i][j + 1]) for i in range(steps)) / steps for j in range(4)]
+    kt = {k: plan.kernel_timing(k) for k in ("grid_read", "grid_write", "mix", "mix_adjoint")}
+    plan.enable_kernel_timing(0)
+    return {"ms_step": ms_step, "phases": ph, "kt": kt, "launches": launches, "clocks": clocks, "step_fn": step}
+
+
+def kernel_table(w, kt):
+    """Per kernel kind: launches, average launch time, algorithmic bytes per launch and the rate they give."""
+    ab = algorithmic_bytes(w)
+
+    def kind_line(kind, bytes_per_launch):
+        n, ms = kt[kind]
+        if n == 0:
+            return None
+        avg = ms / n
+        return {"launches": n, "avg_ms": avg, "algorithmic_bytes_per_launch": bytes_per_launch,
+                "achieved_gbs": bytes_per_launch / (avg * 1e-3) / 1e9}
+
+    return {
+        "grid_read": kind_line("grid_read", (ab["grid_read_launch_F"] + ab["grid_read_launch_B"]) / 2),
+        "grid_write": kind_line("grid_write", (ab["grid_write_launch_I"] + ab["grid_write_launch_B"]) / 2),
+        "mix": kind_line("mix", ab["mix"]),
+        "mix_adjoint": kind_line("mix_adjoint", ab["mix_adjoint"]),
+    }
+
+
+def virtual_shard_summary(torch, w, x, g, W, P, steps, peak):
     """The headline workload once more with its dimension 0 cut into P virtual slabs (partial spectra with global
-    phase offsets, summed on the device in ascending order): step time beside the unsharded one."""
+    phase offsets, summed on the device in ascending order), timed exactly like the headline: same number of
+    steps, phase split, kernel table, whole-step roofline fraction."""
     from paper_2607_14394_b200 import Plan
     try:
         plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out, virtual_shards=P)
@@ -352,28 +460,27 @@ def virtual_shard_summary(torch, w, x, g, W, P, steps=10):
         Y = plan.spectral_mul(X, W)
         y = plan.inverse(Y)
         gx, gW = plan.backward(g, X, W)
-
-        def step():
+        tensors = (x, g, W, X, Y, y, gx, gW)
+        for _ in range(3):
             plan.forward(x, X)
             plan.spectral_mul(X, W, Y)
             plan.inverse(Y, y)
             plan.backward(g, X, W, gx, gW)
-
-        for _ in range(3):
-            step()
         torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(steps):
-            step()
-        e1.record()
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1) / steps
+        r = timed_steps(torch, plan, tensors, steps)
         ok = plan.status() == 0
+        ab = algorithmic_bytes(w)
+        ms = r["ms_step"]
+        out = {"P": P, "ms_per_step": ms, "gpoints_per_s": w.B * w.points / ms / 1e6, "status_ok": ok, "steps": steps,
+               "phases_ms": dict(zip("FMIB", r["phases"])), "kernels": kernel_table(w, r["kt"]),
+               "gpu_launches": r["launches"],
+               "algorithmic_gbs": ab["fwd_bwd"] / (ms * 1e-3) / 1e9,
+               "frac_of_measured_peak": ab["fwd_bwd"] / (ms * 1e-3) / 1e9 / peak,
+               "frac_of_nominal_8TBs": ab["fwd_bwd"] / (ms * 1e-3) / 1e9 / 8000.0}
         plan.close()
-        del plan, X, Y, y, gx, gW
+        del plan, X, Y, y, gx, gW, tensors, r
         torch.cuda.empty_cache()
-        return {"P": P, "ms_per_step": ms, "gpoints_per_s": w.B * w.points / ms / 1e6, "status_ok": ok, "steps": steps}
+        return out
     except Exception as ex:
         return {"P": P, "error": f"{type(ex).__name__}: {ex}"[:200]}
 
@@ -449,6 +556,8 @@ def main_ours(args, w):
     from paper_2607_14394_b200 import dist as D
 
     world, rank, local_rank = D.env_world()
+    if world > 1 and args.multi == "slab":
+        return main_sharded(args, w)
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the spectral layer has no CPU path")
     torch.cuda.set_device(local_rank)
@@ -468,55 +577,28 @@ def main_ours(args, w):
     y = torch.empty((w.B, w.C_out) + w.N, dtype=torch.float32, device=dev)
     gx = torch.empty((w.B, w.C_in) + w.N, dtype=torch.float32, device=dev)
     gW = torch.empty((w.C_in, w.C_out, w.M), dtype=torch.complex64, device=dev)
-
-    def step(evs=None):
-        if evs is not None:
-            evs[0].record()
-        plan.forward(x, Xhat)
-        if evs is not None:
-            evs[1].record()
-        plan.spectral_mul(Xhat, W, Yhat)
-        if evs is not None:
-            evs[2].record()
-        plan.inverse(Yhat, y)
-        if evs is not None:
-            evs[3].record()
-        plan.backward(g, Xhat, W, gx, gW)
-        if evs is not None:
-            evs[4].record()
+    tensors = (x, g, W, Xhat, Yhat, y, gx, gW)
 
     def barrier():
         if world > 1:
             dist.barrier()
 
+    def warm():
+        plan.forward(x, Xhat)
+        plan.spectral_mul(Xhat, W, Yhat)
+        plan.inverse(Yhat, y)
+        plan.backward(g, Xhat, W, gx, gW)
+
     for _ in range(warmup):
-        step()
+        warm()
     torch.cuda.synchronize()
     if plan.status() != 0:
         raise RuntimeError("device-side status word set during warm-up")
 
-    plan.enable_kernel_timing(2 * steps + 2)
-    phase_events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
-    sampler = ClockSampler(local_rank, uuid=getattr(torch.cuda.get_device_properties(local_rank), "uuid", None))
-    launches0 = plan.launch_count()
-    barrier()
-    torch.cuda.synchronize()
-    if rank == 0:
-        sampler.start()
-    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_start.record()
-    for i in range(steps):
-        step(phase_events[i])
-    t_end.record()
-    torch.cuda.synchronize()
-    barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    launches = plan.launch_count() - launches0
-    ms_total = t_start.elapsed_time(t_end)
-    ms_step = ms_total / steps
-    ph = [sum(phase_events[i][j].elapsed_time(phase_events[i][j + 1]) for i in range(steps)) / steps for j in range(4)]
-    kt = {k: plan.kernel_timing(k) for k in ("grid_read", "grid_write", "mix", "mix_adjoint")}
-    plan.enable_kernel_timing(0)
+    sampler = ClockSampler(local_rank, uuid=getattr(torch.cuda.get_device_properties(local_rank), "uuid", None)) \
+        if rank == 0 else None
+    r = timed_steps(torch, plan, tensors, steps, barrier, sampler)
+    clocks, launches, ms_step, ph, kt, step = r["clocks"], r["launches"], r["ms_step"], r["phases"], r["kt"], r["step_fn"]
     graph_ms = graph_step_ms(torch, step, min(steps, 10)) if (rank == 0 and world == 1 and
                                                              not args.no_other_configs) else None
 
@@ -530,27 +612,24 @@ def main_ours(args, w):
     peak, peak_src = measured_peaks()
 
     # roofline of the dominant kernel kind (the two grid-streaming kernels carry ~all bytes)
-    def kind_line(kind, bytes_per_launch):
-        n, ms = kt[kind]
-        if n == 0:
-            return None
-        avg = ms / n
-        return {"launches": n, "avg_ms": avg, "algorithmic_bytes_per_launch": bytes_per_launch,
-                "achieved_gbs": bytes_per_launch / (avg * 1e-3) / 1e9}
-
-    kinds = {
-        "grid_read": kind_line("grid_read", (ab["grid_read_launch_F"] + ab["grid_read_launch_B"]) / 2),
-        "grid_write": kind_line("grid_write", (ab["grid_write_launch_I"] + ab["grid_write_launch_B"]) / 2),
-        "mix": kind_line("mix", ab["mix"]),
-        "mix_adjoint": kind_line("mix_adjoint", ab["mix_adjoint"]),
-    }
+    kinds = kernel_table(w, kt)
     dom = max((k for k in ("grid_read", "grid_write") if kinds[k]), key=lambda k: kt[k][1], default=None)
     roofline = None
     if dom:
         a = kinds[dom]["achieved_gbs"]
+        traffic = measured_traffic(w.name.split("_c")[0] if args.channels else w.name, dom, w.C_in)
         roofline = {"bound": "hbm", "kernel": dom, "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
-                    "frac_of_nominal_8TBs": a / 8000.0, "traffic": measured_traffic(w.name, dom), "peak_source": peak_src,
-                    "avg_launch_ms": kinds[dom]["avg_ms"]}
+                    "frac_of_nominal_8TBs": a / 8000.0, "traffic": traffic,
+                    "traffic_over_algorithmic": (traffic / kinds[dom]["algorithmic_bytes_per_launch"]) if traffic else None,
+                    "peak_source": peak_src, "avg_launch_ms": kinds[dom]["avg_ms"]}
+    # the whole step against the same roof: every algorithmic byte of F, M, I, B over the step time
+    step_gbs = ab["fwd_bwd"] / (ms_step * 1e-3) / 1e9
+    roofline_step = {"bound": "hbm", "algorithmic_bytes": ab["fwd_bwd"], "achieved": step_gbs, "peak": peak,
+                     "unit": "GB/s", "frac": step_gbs / peak, "frac_of_nominal_8TBs": step_gbs / 8000.0,
+                     "peak_source": peak_src, "target_frac_of_nominal": 0.70,
+                     "fwd": {"algorithmic_bytes": ab["fwd"], "achieved": ab["fwd"] / (fwd_ms * 1e-3) / 1e9,
+                             "frac": ab["fwd"] / (fwd_ms * 1e-3) / 1e9 / peak,
+                             "frac_of_nominal_8TBs": ab["fwd"] / (fwd_ms * 1e-3) / 1e9 / 8000.0}}
 
     # end to end through host buffers: pinned host -> device copies of x and g_y, the step,
     # device -> host reads of y, grad_x and grad_W, all inside the timed region
@@ -591,7 +670,7 @@ def main_ours(args, w):
             from paper_2607_14394_b200.binding import HostPipeline
             hx.copy_(x)
             hg.copy_(g)
-            del x, g, y, gx, gW
+            del x, g, y, gx, gW, tensors, r, step
             torch.cuda.empty_cache()
             pipe = HostPipeline(plan, W)
             pipe.step(hx, hg, hy, hgx, hgW)            # warm-up
@@ -636,7 +715,7 @@ def main_ours(args, w):
                        if 4 * w.B * w.C_in * w.points > 3 * 126e6 else "inputs smaller than L2: warm-cache numbers",
                        "parallelism": f"independent batches x{world}, no collective"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-            "roofline": roofline,
+            "roofline": roofline, "roofline_step": roofline_step,
             "fwd": {"ms": fwd_ms, "gpoints_per_s": pts_per_step / (fwd_ms * 1e-3) / 1e9,
                     "algorithmic_gbs": ab["fwd"] / (fwd_ms * 1e-3) / 1e9,
                     "frac_of_measured_peak": ab["fwd"] / (fwd_ms * 1e-3) / 1e9 / peak},
@@ -656,7 +735,7 @@ def main_ours(args, w):
             line["cuda_graph"] = {"ms_per_step": graph_ms,
                                   "what": "the same step captured once in a CUDA graph and replayed"}
         if not args.no_other_configs and args.channels == 0 and P == 1 and w.virtual_shards > 1:
-            line["virtual_shards"] = virtual_shard_summary(torch, w, x, g, W, w.virtual_shards, steps=min(steps, 10))
+            line["virtual_shards"] = virtual_shard_summary(torch, w, x, g, W, w.virtual_shards, steps, peak)
         if not args.no_torch_ref:
             line["torch_fft_reference"] = torch_fft_reference(torch, w, x, W, g)
         if not args.no_other_configs and args.channels == 0:
@@ -665,7 +744,8 @@ def main_ours(args, w):
             line["other_configs"] = other_configs_summary(torch, w.name)
         if not args.no_cpu_baseline:
             try:
-                v, dt, info = time_oracle(w, 1, 0, budget=1.4e8)
+                # the same bounded sample, warm-up and statistics as the reference arm (--impl reference)
+                v, dt, info = time_oracle(w, args.cpu_steps, 1)
                 line["cpu_baseline"] = dict(info, value=v, unit=UNIT)
             except Exception as ex:
                 line["cpu_baseline"] = {"value": None, "unit": UNIT, "kind": "oracle", "cores": 0,
@@ -675,6 +755,203 @@ def main_ours(args, w):
     if world > 1:
         dist.destroy_process_group()
     return 0
+
+
+def main_sharded(args, w):
+    """N > 1 ranks, one per GPU: the layer sharded the way Algorithm 1 shards it (strong scaling).  The workload's
+    grid is cut into N slabs along dimension 0 and its modes and weights into N equal chunks; per step every rank
+    runs forward and backward with two collectives per direction (all-reduce of the partial spectrum, all-gather
+    of the mixed chunks), the received spectra landing in local memory before any kernel reads them.  Timed with
+    CUDA events between barriers, max over ranks; rank 0 prints the JSON line.
+
+    `--backend gloo --ops-module MODULE:FACTORY` runs the same launcher and the same exchange logic on CPU ranks
+    with a stand-in for the CUDA steps supplied by the caller (the tests do that); such a line is marked
+    "data_path": "stand-in" and is not a measurement of this library."""
+    import torch
+    import torch.distributed as dist
+    from paper_2607_14394_b200 import dist as D
+    from paper_2607_14394_b200 import inputs
+    from paper_2607_14394_b200.dist_layer import SlabShardedLayer
+
+    world, rank, local_rank = D.env_world()
+    gloo = args.backend == "gloo"
+    if gloo:
+        if not args.ops_module:
+            raise RuntimeError("--backend gloo needs --ops-module: the layer itself has no CPU path")
+        import importlib
+        mod, fn = args.ops_module.split(":")
+        make_ops = getattr(importlib.import_module(mod), fn)
+        dev = torch.device("cpu")
+        D.init_process_group("gloo")
+    else:
+        if not torch.cuda.is_available():
+            raise RuntimeError("bench.py needs CUDA devices: the spectral layer has no CPU path")
+        if local_rank >= torch.cuda.device_count():
+            raise RuntimeError(f"rank {rank} has no GPU: {torch.cuda.device_count()} visible, {world} ranks")
+        dev = torch.device("cuda", local_rank)
+        torch.cuda.set_device(dev)
+        D.init_process_group("nccl", dev)
+    if w.N[0] % world != 0 or w.M % world != 0:
+        raise RuntimeError(f"{world} ranks must divide N_0 = {w.N[0]} and the mode count {w.M}")
+    n_local = (w.N[0] // world,) + tuple(w.N[1:])
+    offset = (rank * n_local[0],) + (0,) * (w.d - 1)
+    ops = make_ops(w.N, n_local, offset, w.kmax, w.B, w.C_in, w.C_out) if gloo else None
+    layer = SlabShardedLayer(w.N, w.kmax, w.B, w.C_in, w.C_out, world, rank, device=dev, ops=ops)
+
+    steps, warmup = max(1, args.steps), max(3, args.warmup)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(D.rank_seed(w.seed, rank))
+    rdt = torch.float64 if gloo else torch.float32
+    cdt = torch.complex128 if gloo else torch.complex64
+    x = torch.randn((w.B, w.C_in) + n_local, generator=gen, device=dev, dtype=rdt)
+    g = torch.randn((w.B, w.C_out) + n_local, generator=gen, device=dev, dtype=rdt)
+    W_shard = torch.view_as_complex(torch.randn((w.C_in, w.C_out, layer.cnt, 2), generator=gen, device=dev, dtype=rdt)
+                                    / (w.C_in * w.C_out) ** 0.5).to(cdt)
+
+    class Clock:
+        """CUDA events on the launching stream, or the host clock for the CPU stand-in."""
+        def __init__(self):
+            self.t = torch.cuda.Event(enable_timing=True) if not gloo else None
+        def record(self):
+            if gloo:
+                self.t = time.perf_counter()
+            else:
+                self.t.record()
+        def ms_to(self, other):
+            return (other.t - self.t) * 1e3 if gloo else self.t.elapsed_time(other.t)
+
+    PH = ("F_local", "all_reduce_X", "mix", "all_gather_Y", "I_local",
+          "B_spectrum_local", "all_reduce_GY", "mix_adjoint", "all_gather_GX", "B_input_local")
+
+    def step(marks=None):
+        def m(i):
+            if marks is not None:
+                marks[i].record()
+        m(0)
+        Xp = layer.local_spectrum(x); m(1)
+        Xhat = layer._all_reduce(Xp, None); m(2)
+        Yc = layer.local_mix(Xhat, W_shard); m(3)
+        Yhat = layer._all_gather(Yc, None); m(4)
+        y = layer.local_inverse(Yhat); m(5)
+        GYp = layer.local_grad_spectrum(g); m(6)
+        GY = layer._all_reduce(GYp, None); m(7)
+        GXc, gWs = layer.local_grad_mix(GY, Xhat, W_shard); m(8)
+        GX = layer._all_gather(GXc, None); m(9)
+        gx = layer.local_grad_input(GX); m(10)
+        return y, gx, gWs
+
+    def sync():
+        if not gloo:
+            torch.cuda.synchronize()
+
+    for _ in range(warmup if not gloo else 1):
+        step()
+    sync()
+    if not gloo and layer.ops.plan.status() != 0:
+        raise RuntimeError("device-side status word set during warm-up")
+    launches0 = 0 if gloo else layer.ops.plan.launch_count()
+    sampler = None
+    if rank == 0 and not gloo:
+        sampler = ClockSampler(local_rank, uuid=getattr(torch.cuda.get_device_properties(local_rank), "uuid", None))
+    marks = [[Clock() for _ in range(11)] for _ in range(steps)]
+    dist.barrier()
+    sync()
+    if sampler:
+        sampler.start()
+    for i in range(steps):
+        step(marks[i])
+    sync()
+    dist.barrier()
+    clocks = sampler.stop() if sampler else None
+    ms_step = marks[0][0].ms_to(marks[-1][10]) / steps
+    ph = [sum(marks[i][j].ms_to(marks[i][j + 1]) for i in range(steps)) / steps for j in range(10)]
+    red = D.max_over_ranks([ms_step] + ph, device=dev)
+    ms_step, ph = red[0], red[1:]
+    launches = 0 if gloo else layer.ops.plan.launch_count() - launches0
+
+    # end to end: every step copies this rank's slab of x and grad_y from pinned host memory and reads y, grad_x
+    # and the grad_W shard back (plain stream-ordered copies around the same step)
+    e2e = None
+    if not gloo and not args.no_e2e:
+        try:
+            hx, hg = x.cpu().pin_memory(), g.cpu().pin_memory()
+            hy, hgx = torch.empty_like(hx).pin_memory() if w.C_in == w.C_out else \
+                torch.empty((w.B, w.C_out) + n_local).pin_memory(), torch.empty_like(hx).pin_memory()
+            hgW = torch.empty((w.C_in, w.C_out, layer.cnt), dtype=torch.complex64).pin_memory()
+
+            def e2e_step():
+                x.copy_(hx, non_blocking=True)
+                g.copy_(hg, non_blocking=True)
+                y, gx, gWs = step()
+                hy.copy_(y, non_blocking=True)
+                hgx.copy_(gx, non_blocking=True)
+                hgW.copy_(gWs, non_blocking=True)
+
+            e2e_step()
+            sync()
+            dist.barrier()
+            n_e = max(1, min(steps, args.e2e_steps))
+            a0, a1 = Clock(), Clock()
+            a0.record()
+            for _ in range(n_e):
+                e2e_step()
+            a1.record()
+            sync()
+            dist.barrier()
+            ms_e = D.max_over_ranks([a0.ms_to(a1) / n_e], device=dev)[0]
+            e2e = {"value": w.B * w.points / (ms_e * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms_e, "steps": n_e,
+                   "h2d_bytes_per_step": int(world * 4 * (hx.numel() + hg.numel())),
+                   "d2h_bytes_per_step": int(world * (4 * (hy.numel() + hgx.numel()) + 8 * hgW.numel())),
+                   "what": "every rank: its slab of x, grad_y pinned host -> device; the sharded step; its slab of "
+                           "y, grad_x and its grad_W shard -> pinned host; bytes are the job's total"}
+        except Exception as ex:
+            e2e = {"value": None, "unit": UNIT, "error": f"{type(ex).__name__}: {ex}"[:200]}
+    elif not gloo:
+        e2e = {"value": None, "unit": UNIT, "skipped": "--no-e2e"}
+
+    if rank == 0:
+        pts = w.B * w.points                       # the GLOBAL grid: total work is fixed as N grows
+        ab = algorithmic_bytes(w)
+        peak, peak_src = measured_peaks()
+        spectrum_bytes = 8 * w.B * w.M
+        line = {
+            "metric": METRIC, "value": pts / (ms_step * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": warmup if not gloo else 1, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "f64" if gloo else "f32", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "C_in": w.C_in, "C_out": w.C_out, "grid": list(w.N),
+                       "kmax": list(w.kmax), "modes": w.M, "slab_per_rank": list(n_local),
+                       "modes_per_rank": layer.cnt, "l2": "inputs larger than L2 (no flush needed)"
+                       if 4 * w.B * w.C_in * w.points / world > 3 * 126e6 else "per-rank inputs smaller than L2",
+                       "parallelism": f"slab{world} along dim 0: all-reduce of the partial spectrum, mode-sharded "
+                                      f"mixing, all-gather (per direction); backend {args.backend}"},
+            "backend": args.backend, "data_path": "stand-in (test ops on CPU ranks)" if gloo else "cuda",
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches) * world,
+            "phases_ms": dict(zip(PH, ph)),
+            "collective_ms_per_step": ph[1] + ph[3] + ph[6] + ph[8],
+            "collective_payload_bytes_per_step": {
+                "all_reduce": spectrum_bytes * (w.C_in + w.C_out),
+                "all_gather": spectrum_bytes * (w.C_out + w.C_in)},
+            "roofline_step": None if gloo else {
+                "bound": "hbm", "algorithmic_bytes": ab["fwd_bwd"],
+                "achieved": ab["fwd_bwd"] / (ms_step * 1e-3) / 1e9, "peak": peak * world, "unit": "GB/s",
+                "frac": ab["fwd_bwd"] / (ms_step * 1e-3) / 1e9 / (peak * world), "peak_source": peak_src + f" x {world}"},
+        }
+        print(json.dumps(line))
+    dist.destroy_process_group()
+    return 0
+
+
+def respawn_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start N ranks of this very script under torchrun (one per
+    GPU, rendezvous on 127.0.0.1) and hand their output through."""
+    import socket
+    import subprocess
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -689,6 +966,12 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--channels", type=int, default=0,
                     help="override C_in = C_out (smaller cases for profiler captures; not a bench configuration)")
+    ap.add_argument("--multi", default="slab", choices=["slab", "batches"],
+                    help="N > 1: 'slab' = the layer sharded over ranks (Algorithm 1, strong scaling, collectives); "
+                         "'batches' = an independent batch per rank (weak scaling, no collective)")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"])
+    ap.add_argument("--ops-module", default="", help="with --backend gloo: MODULE:FACTORY of a stand-in for the CUDA steps")
+    ap.add_argument("--cpu-steps", type=int, default=3, help="timed sample steps of the CPU oracle baseline")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-torch-ref", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -701,6 +984,8 @@ def main():
                                    field=w.field, seed=w.seed, virtual_shards=w.virtual_shards)
     if args.impl == "reference":
         return main_reference(args, w)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return respawn_ranks(args.gpus)
     return main_ours(args, w)
 
 

@@ -71,7 +71,8 @@ enum {
  *   kmax[d]  retained modes per dimension (host array): 1 <= k_j, 2 k_j <= N_j for
  *            j < d-1, and k_{d-1} <= N_{d-1}/2 + 1
  *   B, C_in, C_out  batch and channel counts (>= 1)
- * The plan records the current CUDA device; use it with that device current.
+ * The plan records the current CUDA device; every compute call must be made with that
+ * device current, else it returns DTST_ERR_INVALID_ARG without launching anything.
  * Errors: DTST_ERR_INVALID_ARG for any violated bound, DTST_ERR_ALLOC.
  */
 dtst_status dtst_plan_create(dtst_plan** out, int d, const int64_t N[], const int32_t kmax[],
@@ -161,7 +162,8 @@ dtst_status dtst_inverse(dtst_plan* plan, const void* Yhat, float* y, void* stre
  * Complex gradients follow the convention dL/dRe + i dL/dIm.
  *   grad_y [B, C_out, n...] float32; Xhat_saved = dtst_forward's output; W as above;
  *   grad_x [B, C_in, n...] float32 and grad_W [C_in, C_out, M] complex64 are ASSIGNED
- *   (not accumulated); either may be NULL to skip it (not both).
+ *   (not accumulated); either may be NULL to skip it (not both).  Xhat_saved is read only
+ *   for grad_W and may be NULL when grad_W is NULL.
  */
 dtst_status dtst_backward(dtst_plan* plan, const float* grad_y, const void* Xhat_saved,
                           const void* W, float* grad_x, void* grad_W, void* stream);
@@ -234,6 +236,19 @@ dtst_status dtst_forward_static(dtst_plan* plan, const float* x, void* Xhat, voi
  * DTST_OK, or DTST_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up
  * (the kernel then exited normally and its output is undefined).  Clears the word. */
 dtst_status dtst_plan_status(dtst_plan* plan, void* stream);
+
+/*
+ * Diagnostic for the failure-reporting path, not for production use.  Every device-side wait in
+ * the streaming kernels is bounded: when its poll budget runs out the kernel raises the plan's
+ * status word and returns normally (no trap, no hang).  This call makes that happen on purpose:
+ * from now on the forward plane kernel's producer stops feeding its shared-memory ring after
+ * `withhold_after_fills` slot fills and the waits give up after `poll_limit` polls (1..65536, so
+ * that the run ends within milliseconds); the call's output is then undefined and
+ * dtst_plan_status reports DTST_ERR_DEVICE_TIMEOUT once.  withhold_after_fills < 0 restores
+ * normal operation.  Only plans on the fused streaming path are affected (dtst_plan_kernel_path
+ * == DTST_PATH_AUTO).
+ */
+dtst_status dtst_plan_debug_ring_fault(dtst_plan* plan, int64_t withhold_after_fills, uint32_t poll_limit);
 
 /* Number of kernel launches the plan's compute calls have issued so far. */
 dtst_status dtst_plan_launch_count(const dtst_plan* plan, int64_t* launches);

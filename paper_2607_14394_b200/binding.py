@@ -38,7 +38,7 @@ EXPORTED = [
     "dtst_backward", "dtst_plan_status", "dtst_plan_launch_count", "dtst_status_string",
     "dtst_version", "dtst_plan_enable_kernel_timing", "dtst_plan_kernel_timing", "dtst_forward_static",
     "dtst_plan_last_cuda_error", "dtst_spectral_mul_modes", "dtst_backward_spectrum", "dtst_backward_mix_modes",
-    "dtst_backward_input",
+    "dtst_backward_input", "dtst_plan_debug_ring_fault",
 ]
 
 
@@ -81,6 +81,7 @@ def lib() -> ctypes.CDLL:
     L.dtst_backward_spectrum.argtypes = [vp, vp, vp, vp]
     L.dtst_backward_mix_modes.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_int64, ctypes.c_int64, vp]
     L.dtst_backward_input.argtypes = [vp, vp, vp, vp]
+    L.dtst_plan_debug_ring_fault.argtypes = [vp, ctypes.c_int64, ctypes.c_uint32]
     L.dtst_plan_status.argtypes = [vp, vp]
     L.dtst_plan_launch_count.argtypes = [vp, i64p]
     L.dtst_plan_enable_kernel_timing.argtypes = [vp, i32]
@@ -256,6 +257,11 @@ def dtst_backward_input(plan, GX, grad_x, stream=None) -> None:
                                      _stream_ptr(stream)), "dtst_backward_input", plan)
 
 
+def dtst_plan_debug_ring_fault(plan, withhold_after_fills, poll_limit) -> None:
+    _check(lib().dtst_plan_debug_ring_fault(plan, int(withhold_after_fills), int(poll_limit)),
+           "dtst_plan_debug_ring_fault")
+
+
 def dtst_plan_status(plan, stream=None) -> int:
     return int(lib().dtst_plan_status(plan, _stream_ptr(stream)))
 
@@ -301,6 +307,10 @@ class Plan:
         self.d = len(self.N)
         self.B, self.C_in, self.C_out = int(B), int(C_in), int(C_out)
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        if self.device.type != "cuda":
+            raise ValueError("a Plan lives on a CUDA device")
+        if self.device.index is None:
+            self.device = torch.device("cuda", torch.cuda.current_device())
         self._h = None
         with torch.cuda.device(self.device):
             if N_global is None:
@@ -347,28 +357,67 @@ class Plan:
     def kernel_timing(self, kind):
         return dtst_plan_kernel_timing(self._h, kind)
 
+    # -- argument checks: the C ABI takes raw device pointers, so a tensor of the wrong size or on another
+    # device would make the kernels read or write out of bounds; refuse it here, as a Python error
+    def _numel(self, kind: str, count=None) -> int:
+        import math
+        pts = math.prod(self.N)
+        return {"x": self.B * self.C_in * pts, "y": self.B * self.C_out * pts,
+                "Xhat": self.B * self.C_in * self.M, "Yhat": self.B * self.C_out * self.M,
+                "W": self.C_in * self.C_out * self.M,
+                "Xchunk": self.B * self.C_in * (count or 0), "Ychunk": self.B * self.C_out * (count or 0),
+                "Wshard": self.C_in * self.C_out * (count or 0)}[kind]
+
+    def _expect(self, t, kind: str, name: str, count=None):
+        if t is None:
+            return
+        if not isinstance(t, torch.Tensor) or not t.is_cuda:
+            raise ValueError(f"{name} must be a CUDA tensor")
+        if t.device != self.device:
+            raise ValueError(f"{name} is on {t.device}, the plan on {self.device}")
+        want = self._numel(kind, count)
+        if t.numel() != want:
+            raise ValueError(f"{name} has {t.numel()} elements, the plan needs {want} ({kind})")
+
+    def _modes(self, m0, count):
+        if not (0 <= int(m0) and int(count) >= 1 and int(m0) + int(count) <= self.M):
+            raise ValueError(f"mode range [{m0}, {m0}+{count}) outside [0, {self.M})")
+
     # -- compute (outputs allocated here unless given)
     def forward(self, x, out=None, stream=None):
         if out is None:
             out = torch.empty((self.B, self.C_in) + self.K, dtype=torch.complex64, device=self.device)
-        dtst_forward(self._h, x, out, stream)
+        self._expect(x, "x", "x")
+        self._expect(out, "Xhat", "out")
+        with torch.cuda.device(self.device):
+            dtst_forward(self._h, x, out, stream)
         return out
 
     def forward_static(self, x, out, stream=None):
         """Forward partial DFT into the caller's `out` using only the library's fixed scratch."""
-        dtst_forward_static(self._h, x, out, stream)
+        self._expect(x, "x", "x")
+        self._expect(out, "Xhat", "out")
+        with torch.cuda.device(self.device):
+            dtst_forward_static(self._h, x, out, stream)
         return out
 
     def spectral_mul(self, Xhat, W, out=None, stream=None):
         if out is None:
             out = torch.empty((self.B, self.C_out) + self.K, dtype=torch.complex64, device=self.device)
-        dtst_spectral_mul(self._h, Xhat, W, out, stream)
+        self._expect(Xhat, "Xhat", "Xhat")
+        self._expect(W, "W", "W")
+        self._expect(out, "Yhat", "out")
+        with torch.cuda.device(self.device):
+            dtst_spectral_mul(self._h, Xhat, W, out, stream)
         return out
 
     def inverse(self, Yhat, out=None, stream=None):
         if out is None:
             out = torch.empty((self.B, self.C_out) + self.N, dtype=torch.float32, device=self.device)
-        dtst_inverse(self._h, Yhat, out, stream)
+        self._expect(Yhat, "Yhat", "Yhat")
+        self._expect(out, "y", "out")
+        with torch.cuda.device(self.device):
+            dtst_inverse(self._h, Yhat, out, stream)
         return out
 
     def backward(self, grad_y, Xhat_saved, W, grad_x=None, grad_W=None, need_grad_x=True, need_grad_W=True,
@@ -377,34 +426,58 @@ class Plan:
             grad_x = torch.empty((self.B, self.C_in) + self.N, dtype=torch.float32, device=self.device)
         if grad_W is None and need_grad_W:
             grad_W = torch.empty((self.C_in, self.C_out, self.M), dtype=torch.complex64, device=self.device)
-        dtst_backward(self._h, grad_y, Xhat_saved, W, grad_x, grad_W, stream)
+        self._expect(grad_y, "y", "grad_y")
+        self._expect(Xhat_saved, "Xhat", "Xhat_saved")
+        self._expect(W, "W", "W")
+        self._expect(grad_x, "x", "grad_x")
+        self._expect(grad_W, "W", "grad_W")
+        with torch.cuda.device(self.device):
+            dtst_backward(self._h, grad_y, Xhat_saved, W, grad_x, grad_W, stream)
         return grad_x, grad_W
 
     # -- the steps one by one (a rank of a slab-sharded layer exchanges spectra between them)
     def spectral_mul_modes(self, Xhat, W_shard, m0, count, out=None, stream=None):
+        self._modes(m0, count)
         if out is None:
             out = torch.empty((self.B, self.C_out, count), dtype=torch.complex64, device=self.device)
-        dtst_spectral_mul_modes(self._h, Xhat, W_shard, out, m0, count, stream)
+        self._expect(Xhat, "Xhat", "Xhat")
+        self._expect(W_shard, "Wshard", "W_shard", count)
+        self._expect(out, "Ychunk", "out", count)
+        with torch.cuda.device(self.device):
+            dtst_spectral_mul_modes(self._h, Xhat, W_shard, out, m0, count, stream)
         return out
 
     def backward_spectrum(self, grad_y, out=None, stream=None):
         if out is None:
             out = torch.empty((self.B, self.C_out) + self.K, dtype=torch.complex64, device=self.device)
-        dtst_backward_spectrum(self._h, grad_y, out, stream)
+        self._expect(grad_y, "y", "grad_y")
+        self._expect(out, "Yhat", "out")
+        with torch.cuda.device(self.device):
+            dtst_backward_spectrum(self._h, grad_y, out, stream)
         return out
 
     def backward_mix_modes(self, GY, Xhat_saved, W_shard, m0, count, GX_chunk=None, grad_W_shard=None, stream=None):
+        self._modes(m0, count)
         if GX_chunk is None:
             GX_chunk = torch.empty((self.B, self.C_in, count), dtype=torch.complex64, device=self.device)
         if grad_W_shard is None:
             grad_W_shard = torch.empty((self.C_in, self.C_out, count), dtype=torch.complex64, device=self.device)
-        dtst_backward_mix_modes(self._h, GY, Xhat_saved, W_shard, GX_chunk, grad_W_shard, m0, count, stream)
+        self._expect(GY, "Yhat", "GY")
+        self._expect(Xhat_saved, "Xhat", "Xhat_saved")
+        self._expect(W_shard, "Wshard", "W_shard", count)
+        self._expect(GX_chunk, "Xchunk", "GX_chunk", count)
+        self._expect(grad_W_shard, "Wshard", "grad_W_shard", count)
+        with torch.cuda.device(self.device):
+            dtst_backward_mix_modes(self._h, GY, Xhat_saved, W_shard, GX_chunk, grad_W_shard, m0, count, stream)
         return GX_chunk, grad_W_shard
 
     def backward_input(self, GX, out=None, stream=None):
         if out is None:
             out = torch.empty((self.B, self.C_in) + self.N, dtype=torch.float32, device=self.device)
-        dtst_backward_input(self._h, GX, out, stream)
+        self._expect(GX, "Xhat", "GX")
+        self._expect(out, "x", "out")
+        with torch.cuda.device(self.device):
+            dtst_backward_input(self._h, GX, out, stream)
         return out
 
     def layer(self, x, W, Xhat=None, Yhat=None, y=None, stream=None):
@@ -413,6 +486,10 @@ class Plan:
         Yhat = self.spectral_mul(Xhat, W, Yhat, stream)
         y = self.inverse(Yhat, y, stream)
         return y, Xhat
+
+    def debug_ring_fault(self, withhold_after_fills: int, poll_limit: int = 1024) -> None:
+        """Diagnostic: make the forward plane kernel's bounded waits run out (see dtst_plan_debug_ring_fault)."""
+        dtst_plan_debug_ring_fault(self._h, withhold_after_fills, poll_limit)
 
     def close(self):
         if self._h is not None:

@@ -84,6 +84,7 @@ dtst_status create_common(dtst_plan** out, int d, const int64_t* Ng, const int64
   p->points_global = pts_g;
   p->P = 1;
   p->path_request = DTST_PATH_AUTO;
+  p->dbg_withhold_after = -1;
   p->device = -1;
   int dev = -1;
   if (cudaGetDevice(&dev) == cudaSuccess) p->device = dev;
@@ -236,66 +237,53 @@ dtst_status run_forward_fused(dtst_plan* p, const float* x, float2* Xhat, int Cn
   float2* t1 = (d == 2) ? Xhat : reinterpret_cast<float2*>(ws + L.bufA);
   {
     KernelTimer kt(p, DTST_KERNEL_GRID_READ, st);
+    const RingDebug dbg{p->dbg_poll_limit ? p->dbg_poll_limit : kDefaultPollLimit, p->dbg_withhold_after};
     if (cuda_failed(p, launch_fwd_plane((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], x, t1, planes * p->Ng[b], scale,
-                         herm ? 1 : 0, reinterpret_cast<int*>(ws + L.status), st))) return DTST_ERR_CUDA;
+                         herm ? 1 : 0, reinterpret_cast<int*>(ws + L.status), dbg, st))) return DTST_ERR_CUDA;
   }
   ++p->launches;
   if (d == 2) return DTST_OK;
   return forward_stages(p, t1, d - 3, 1, Xhat, Cn, 1.0f, false, st);
 }
 
-// Generic expansion: [B*Cn, M] spectrum -> real grid tensor.
-dtst_status run_inverse_generic(dtst_plan* p, const float2* Yhat, float* y, int Cn, float scale, bool herm,
-                                cudaStream_t st) {
-  const WsLayout L = ws_layout(p);
-  char* ws = static_cast<char*>(p->ws);
-  float2* buf[2] = {reinterpret_cast<float2*>(ws + L.bufA), reinterpret_cast<float2*>(ws + L.bufB)};
-  const void* cur = Yhat;
-  int flip = 0;
-  for (int j = 0; j < p->d; ++j) {
-    DimOp op = make_op(p, j, false, Cn);
-    const bool out_real = (j == p->d - 1);
-    if (out_real) {
-      op.scale = scale;
-      op.herm = herm ? 1 : 0;
-    }
-    if (j == 0 && p->P > 1) {
-      // slab p expands to rows [p*nl, (p+1)*nl) with the same offset phases; no reduction needed
-      const int nl = (int)(p->Nl[0] / p->P);
-      op.slabs = p->P;
-      op.R = nl;
-      op.offset_step = nl;
-      op.out_outer_stride = p->Nl[0] * op.inner;
-      op.out_slab_stride = (long long)nl * op.inner;
-    }
-    void* dst = out_real ? static_cast<void*>(y) : static_cast<void*>(buf[flip]);
-    if (!out_real && use_mid_expand(p, j)) {
-      if (cuda_failed(p, launch_mid(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
-                                    make_op(p, j, false, Cn).outer, make_op(p, j, false, Cn).inner, (int)p->Ng[j], 1.0f,
-                                    st)))
-        return DTST_ERR_CUDA;
-    } else if (!out_real && use_slab(p, j)) {
-      if (cuda_failed(p, launch_slab(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
-                                     make_op(p, j, false, Cn).outer, make_op(p, j, false, Cn).inner, (int)p->Nl[j],
-                                     (int)p->Ng[j], (int)p->off[j], j == 0 ? p->P : 1, st)))
-        return DTST_ERR_CUDA;
-    } else if (!out_real && use_mid(p, j)) {
-      if (cuda_failed(p, launch_mid(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
-                                    op.outer, op.inner, op.N, 1.0f, st)))
-        return DTST_ERR_CUDA;
-    } else {
-      KernelTimer kt(p, DTST_KERNEL_GRID_WRITE, st, out_real);
-      if (cuda_failed(p, launch_apply_dim(op, false, out_real, cur, dst, st))) return DTST_ERR_CUDA;
-    }
-    ++p->launches;
-    cur = dst;
-    flip ^= 1;
+// One expansion stage (B^H along dimension j) from `cur` into `dst` with whichever kernel family serves it.  The
+// last dimension's stage writes the real grid and carries the scale and the Hermitian weights.
+dtst_status expand_stage(dtst_plan* p, int j, int Cn, const void* cur, void* dst, float scale, bool herm,
+                         cudaStream_t st) {
+  DimOp op = make_op(p, j, false, Cn);
+  const bool out_real = (j == p->d - 1);
+  if (out_real) {
+    op.scale = scale;
+    op.herm = herm ? 1 : 0;
   }
+  const long long outer = op.outer, inner = op.inner;
+  if (j == 0 && p->P > 1) {
+    // slab p expands to rows [p*nl, (p+1)*nl) with the same offset phases; no reduction needed
+    const int nl = (int)(p->Nl[0] / p->P);
+    op.slabs = p->P;
+    op.R = nl;
+    op.offset_step = nl;
+    op.out_outer_stride = p->Nl[0] * op.inner;
+    op.out_slab_stride = (long long)nl * op.inner;
+  }
+  cudaError_t e;
+  if (!out_real && use_mid_expand(p, j)) {
+    e = launch_mid(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst), outer, inner,
+                   (int)p->Ng[j], 1.0f, st);
+  } else if (!out_real && use_slab(p, j)) {
+    e = launch_slab(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst), outer, inner,
+                    (int)p->Nl[j], (int)p->Ng[j], (int)p->off[j], j == 0 ? p->P : 1, st);
+  } else {
+    KernelTimer kt(p, DTST_KERNEL_GRID_WRITE, st, out_real);
+    e = launch_apply_dim(op, false, out_real, cur, dst, st);
+  }
+  if (cuda_failed(p, e)) return DTST_ERR_CUDA;
+  ++p->launches;
   return DTST_OK;
 }
 
-// Generic expansion stages j = 0..j_to on `cur` (complex), ping-ponging through the workspace; returns
-// the buffer holding the result through *out_buf.
+// Expansion stages j = 0..j_to on `cur` (complex), ping-ponging through the workspace; returns the buffer
+// holding the result through *out_buf (cur_in itself when j_to < 0).
 dtst_status inverse_stages_complex(dtst_plan* p, const float2* cur_in, int j_to, int Cn, const float2** out_buf,
                                    cudaStream_t st) {
   const WsLayout L = ws_layout(p);
@@ -304,39 +292,23 @@ dtst_status inverse_stages_complex(dtst_plan* p, const float2* cur_in, int j_to,
   const void* cur = cur_in;
   int flip = 0;
   for (int j = 0; j <= j_to; ++j) {
-    DimOp op = make_op(p, j, false, Cn);
-    if (j == 0 && p->P > 1) {
-      const int nl = (int)(p->Nl[0] / p->P);
-      op.slabs = p->P;
-      op.R = nl;
-      op.offset_step = nl;
-      op.out_outer_stride = p->Nl[0] * op.inner;
-      op.out_slab_stride = (long long)nl * op.inner;
-    }
     void* dst = buf[flip];
-    if (use_mid_expand(p, j)) {
-      if (cuda_failed(p, launch_mid(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
-                                    make_op(p, j, false, Cn).outer, make_op(p, j, false, Cn).inner, (int)p->Ng[j], 1.0f,
-                                    st)))
-        return DTST_ERR_CUDA;
-    } else if (use_slab(p, j)) {
-      if (cuda_failed(p, launch_slab(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
-                                     make_op(p, j, false, Cn).outer, make_op(p, j, false, Cn).inner, (int)p->Nl[j],
-                                     (int)p->Ng[j], (int)p->off[j], j == 0 ? p->P : 1, st)))
-        return DTST_ERR_CUDA;
-    } else if (use_mid(p, j)) {
-      if (cuda_failed(p, launch_mid(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
-                                    op.outer, op.inner, op.N, 1.0f, st)))
-        return DTST_ERR_CUDA;
-    } else if (cuda_failed(p, launch_apply_dim(op, false, false, cur, dst, st))) {
-      return DTST_ERR_CUDA;
-    }
-    ++p->launches;
+    const dtst_status s = expand_stage(p, j, Cn, cur, dst, 1.0f, false, st);
+    if (s != DTST_OK) return s;
     cur = dst;
     flip ^= 1;
   }
   *out_buf = static_cast<const float2*>(cur);
   return DTST_OK;
+}
+
+// Generic expansion: [B*Cn, M] spectrum -> real grid tensor.
+dtst_status run_inverse_generic(dtst_plan* p, const float2* Yhat, float* y, int Cn, float scale, bool herm,
+                                cudaStream_t st) {
+  const float2* src = Yhat;
+  const dtst_status s = inverse_stages_complex(p, Yhat, p->d - 2, Cn, &src, st);
+  if (s != DTST_OK) return s;
+  return expand_stage(p, p->d - 1, Cn, src, y, scale, herm, st);
 }
 
 // Fused expansion: generic stages for dims 0..d-3 on the small tensor, then the inverse plane kernel
@@ -396,8 +368,24 @@ dtst_status run_inverse_row(dtst_plan* p, const float2* Yhat, float* y, int Cn, 
   return DTST_OK;
 }
 
-dtst_status check_ready(const dtst_plan* p) {
+// A plan belongs to the device that was current when it was created: its workspace and the caller's tensors live
+// there, so a compute call with another device current would launch on the wrong GPU with foreign pointers.
+dtst_status check_device(const dtst_plan* p) {
   if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  if (p->device >= 0) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return DTST_ERR_CUDA;
+    }
+    if (dev != p->device) return DTST_ERR_INVALID_ARG;
+  }
+  return DTST_OK;
+}
+
+dtst_status check_ready(const dtst_plan* p) {
+  const dtst_status sd = check_device(p);
+  if (sd != DTST_OK) return sd;
   const WsLayout L = ws_layout(p);
   if (p->ws == nullptr || p->ws_bytes < L.total) return DTST_ERR_WORKSPACE;
   return DTST_OK;
@@ -587,7 +575,7 @@ dtst_status dtst_forward(dtst_plan* p, const float* x, void* Xhat, void* stream)
 }
 
 dtst_status dtst_spectral_mul(dtst_plan* p, const void* Xhat, const void* W, void* Yhat, void* stream) {
-  if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  if (check_device(p) != DTST_OK) return check_device(p);
   if (Xhat == nullptr || W == nullptr || Yhat == nullptr || !aligned16(Xhat) || !aligned16(W) ||
       !aligned16(Yhat) || Yhat == Xhat || Yhat == W)
     return DTST_ERR_INVALID_ARG;
@@ -613,7 +601,9 @@ dtst_status dtst_backward(dtst_plan* p, const float* grad_y, const void* Xhat_sa
                           float* grad_x, void* grad_W, void* stream) {
   dtst_status s = check_ready(p);
   if (s != DTST_OK) return s;
-  if (grad_y == nullptr || Xhat_saved == nullptr || W == nullptr || (grad_x == nullptr && grad_W == nullptr))
+  // Xhat_saved is read for grad_W only
+  if (grad_y == nullptr || W == nullptr || (grad_x == nullptr && grad_W == nullptr) ||
+      (grad_W != nullptr && Xhat_saved == nullptr))
     return DTST_ERR_INVALID_ARG;
   if (!aligned16(grad_y) || !aligned16(Xhat_saved) || !aligned16(W) || !aligned16(grad_x) || !aligned16(grad_W))
     return DTST_ERR_INVALID_ARG;
@@ -648,7 +638,7 @@ dtst_status dtst_backward(dtst_plan* p, const float* grad_y, const void* Xhat_sa
 // ---- the steps of the layer one by one, for a caller that exchanges spectra between ranks in between them
 dtst_status dtst_spectral_mul_modes(dtst_plan* p, const void* Xhat, const void* W_shard, void* Yhat_chunk,
                                     int64_t m0, int64_t count, void* stream) {
-  if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  if (check_device(p) != DTST_OK) return check_device(p);
   if (Xhat == nullptr || W_shard == nullptr || Yhat_chunk == nullptr || !aligned16(Xhat) || !aligned16(W_shard) ||
       !aligned16(Yhat_chunk) || Yhat_chunk == Xhat || Yhat_chunk == W_shard)
     return DTST_ERR_INVALID_ARG;
@@ -675,7 +665,7 @@ dtst_status dtst_backward_spectrum(dtst_plan* p, const float* grad_y, void* GY, 
 
 dtst_status dtst_backward_mix_modes(dtst_plan* p, const void* GY, const void* Xhat_saved, const void* W_shard,
                                     void* GX_chunk, void* grad_W_shard, int64_t m0, int64_t count, void* stream) {
-  if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  if (check_device(p) != DTST_OK) return check_device(p);
   if (GY == nullptr || W_shard == nullptr || (GX_chunk == nullptr && grad_W_shard == nullptr) ||
       (grad_W_shard != nullptr && Xhat_saved == nullptr))
     return DTST_ERR_INVALID_ARG;
@@ -714,6 +704,14 @@ dtst_status dtst_plan_status(dtst_plan* p, void* stream) {
     if (cudaMemset(p->ws, 0, kStatusBytes) != cudaSuccess) return DTST_ERR_CUDA;
     return DTST_ERR_DEVICE_TIMEOUT;
   }
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_debug_ring_fault(dtst_plan* p, int64_t withhold_after_fills, uint32_t poll_limit) {
+  if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  if (withhold_after_fills >= 0 && (poll_limit == 0 || poll_limit > (1u << 16))) return DTST_ERR_INVALID_ARG;
+  p->dbg_withhold_after = withhold_after_fills < 0 ? -1 : (long long)withhold_after_fills;
+  p->dbg_poll_limit = withhold_after_fills < 0 ? 0u : poll_limit;
   return DTST_OK;
 }
 

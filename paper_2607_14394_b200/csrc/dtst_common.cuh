@@ -11,7 +11,7 @@
 namespace dtst {
 
 constexpr int kMaxDims = DTST_MAX_DIMS;
-constexpr int kNumSMs = 148;                 // B200
+constexpr int kFallbackSMs = 148;            // B200; used only if the attribute query fails
 constexpr size_t kStatusBytes = 256;         // head of the workspace: device status word
 
 // One application of a (generated) complex matrix E[R x Q] along one dimension of
@@ -38,6 +38,26 @@ struct DimOp {
   long long in_slab_stride, out_slab_stride;
   int basis_in_smem;
 };
+
+// Number of SMs of the current device (persistent kernels launch one CTA per SM, or a multiple): queried
+// once per device and cached.
+inline int num_sms() {
+  static int cache[64] = {};   // 0 = not yet queried; a racing first query writes the same value twice
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    (void)cudaGetLastError();
+    return kFallbackSMs;
+  }
+  int n = cache[dev];
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+      (void)cudaGetLastError();
+      n = kFallbackSMs;
+    }
+    cache[dev] = n;
+  }
+  return n;
+}
 
 // Retained DFT index at position pos of a dimension's list.
 __host__ __device__ inline int mode_at(int pos, int k, int N, int two_sided) {
@@ -93,6 +113,8 @@ struct dtst_plan {
   size_t ws_bytes;
   long long launches;
   int last_cuda_error;             // cudaError_t of the last failing runtime call / launch
+  unsigned dbg_poll_limit;         // 0 = default budget of the bounded waits
+  long long dbg_withhold_after;    // < 0 = off (the default)
   // optional per-kernel event timing (benchmarks only)
   int timing_cap;
   int timing_n[DTST_KERNEL_KINDS];
@@ -100,6 +122,14 @@ struct dtst_plan {
 };
 
 namespace dtst {
+
+// Poll budget of the bounded device-side waits and the diagnostic that makes one of them run out
+// (dtst_plan_debug_ring_fault): the producer of the forward plane kernel's ring stops after `withhold_after` fills.
+struct RingDebug {
+  uint32_t poll_limit;        // polls before a wait gives up
+  long long withhold_after;   // < 0: never withhold
+};
+constexpr uint32_t kDefaultPollLimit = 1u << 24;
 
 struct WsLayout {
   size_t status, bufA, bufB, partial, gy, gx, total;

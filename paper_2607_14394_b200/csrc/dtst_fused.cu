@@ -230,25 +230,33 @@ __device__ __forceinline__ void stage1_row(uint32_t stage, int row, float (&o)[2
 }
 
 // Consumer side of the ring: wait until fill number q (0-based) of `slot` has landed.
+// Every lane of the warp calls it; the lanes poll independently but leave with ONE verdict (a lane whose barrier
+// completed just as another warp raised the abort flag must not go on alone into the warp-synchronous MMA code).
 __device__ __forceinline__ bool wait_fill(volatile uint32_t* fill_seq, uint64_t* full, int slot, uint32_t q,
-                                          volatile int* abort_flag) {
+                                          volatile int* abort_flag, uint32_t limit) {
+  bool ok = true;
   for (uint32_t it = 0; fill_seq[slot] < q + 1u; ++it) {
     if ((it & 63u) == 63u) {
-      if (*abort_flag) return false;
+      if (*abort_flag) {
+        ok = false;
+        break;
+      }
       __nanosleep(64);
     }
-    if (it > (1u << 24)) {
+    if (it > limit) {
       *abort_flag = 1;
-      return false;
+      ok = false;
+      break;
     }
   }
-  return mbar_wait_bounded(&full[slot], q & 1u, abort_flag);
+  if (ok) ok = mbar_wait_bounded(&full[slot], q & 1u, abort_flag, limit);
+  return __all_sync(0xffffffffu, ok) != 0;
 }
 
 template <int N3, int K3, int N2, int K2, int W>
 __global__ void __launch_bounds__((W + 1) * 32, 1)
 fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict__ out, long long num_tasks, float scale, int herm, int stages,
-                 int* __restrict__ status) {
+                 int* __restrict__ status, uint32_t poll_limit, long long withhold_after) {
   using Cfg = PlaneCfg<N3, K3, N2, K2>;
   constexpr int NC = Cfg::NC, QUADS = Cfg::QUADS, G = Cfg::G, LPP = Cfg::LPP;
   constexpr int SPT = Cfg::SPT, RPS = Cfg::ROWS_PER_STAGE;
@@ -330,9 +338,12 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
       for (long long tl = 0; tl < n_local; ++tl) {
         const long long task = first + tl * gridDim.x;
         for (int s = 0; s < SPT; ++s, ++k) {
+          // diagnostic (dtst_plan_debug_ring_fault): stop feeding the ring after `withhold_after` fills, so
+          // that the consumers' bounded waits run out
+          if (withhold_after >= 0 && k >= withhold_after) goto producer_done;
           const int slot = (int)(k % stages);
           const uint32_t ph = (uint32_t)((k / stages) & 1);
-          if (!mbar_wait_bounded(&empty[slot], ph ^ 1u, abort_flag)) goto producer_done;
+          if (!mbar_wait_bounded(&empty[slot], ph ^ 1u, abort_flag, poll_limit)) goto producer_done;
           fill_seq[slot] = (uint32_t)(k / stages) + 1u;
           mbar_arrive_expect_tx(&full[slot], (uint32_t)kStageBytes);
 #pragma unroll
@@ -370,18 +381,18 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
 #pragma unroll
       for (int c = 0; c < NC; ++c) cpp[c] = cpd[c] = cms[c] = cmd[c] = 0.f;
       if constexpr (!kSplit) {
-        if (!wait_fill(fill_seq, full, slot0, (uint32_t)(k0 / stages), abort_flag)) break;
-        if (SPT == 2 && !wait_fill(fill_seq, full, slot1, (uint32_t)((k0 + 1) / stages), abort_flag)) break;
+        if (!wait_fill(fill_seq, full, slot0, (uint32_t)(k0 / stages), abort_flag, poll_limit)) break;
+        if (SPT == 2 && !wait_fill(fill_seq, full, slot1, (uint32_t)((k0 + 1) / stages), abort_flag, poll_limit)) break;
       }
       bool alive = true;
 #pragma unroll 1
       for (int r4 = 0; r4 < 4; ++r4) {
         if constexpr (kSplit) {
-          if (r4 == 0) alive = wait_fill(fill_seq, full, slot0, (uint32_t)(k0 / stages), abort_flag);
+          if (r4 == 0) alive = wait_fill(fill_seq, full, slot0, (uint32_t)(k0 / stages), abort_flag, poll_limit);
           if (r4 == 2) {
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[slot0]);
-            alive = wait_fill(fill_seq, full, slot1, (uint32_t)((k0 + 1) / stages), abort_flag);
+            alive = wait_fill(fill_seq, full, slot1, (uint32_t)((k0 + 1) / stages), abort_flag, poll_limit);
           }
           if (!alive) break;
         }
@@ -524,7 +535,13 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
   }
 
   __syncthreads();
-  if (threadIdx.x == 0 && *abort_flag) atomicExch(status, 1);
+  if (threadIdx.x == 0 && *abort_flag) {
+    // the pipeline gave up: loads that were armed but never consumed may still be in flight, and this CTA's
+    // shared memory must not be handed to the next one while the TMA engine writes to it
+    for (int s = 0; s < stages; ++s)
+      if (fill_seq[s] > 0) mbar_wait_plain(&full[s], (fill_seq[s] - 1u) & 1u, 1u << 16);
+    atomicExch(status, 1);
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -863,24 +880,27 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+EncodeTiledFn lookup_encode_tiled() {
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  EncodeTiledFn fn = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+      q == cudaDriverEntryPointSuccess)
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  (void)cudaGetLastError();
+  return fn;
+}
+
+// looked up once; the initialisation of a function-local static is thread-safe, so plans on different host
+// threads all see the same answer
 EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    (void)cudaGetLastError();
-  }
+  static const EncodeTiledFn fn = lookup_encode_tiled();
   return fn;
 }
 
 template <int N3, int K3, int N2, int K2>
 cudaError_t launch_fwd_plane_t(const float* x, float2* out, long long rows, float scale, int herm, int* status,
-                               cudaStream_t st) {
+                               const RingDebug& dbg, cudaStream_t st) {
   constexpr int W = 7;   // consumer warps (+ the producer warp = 2 warps per scheduler; 8 or 10 consumers measured slower)
   using Cfg = PlaneCfg<N3, K3, N2, K2>;
   const SmemPlan sp = smem_plan<Cfg, K2, K3, W>();
@@ -891,8 +911,9 @@ cudaError_t launch_fwd_plane_t(const float* x, float2* out, long long rows, floa
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sp.total);
   if (e != cudaSuccess) return e;
   const long long tasks = rows / kTaskRows;
-  const int grid = (int)(tasks < kNumSMs ? tasks : kNumSMs);
-  kern<<<grid, (W + 1) * 32, sp.total, st>>>(map, out, tasks, scale, herm, sp.stages, status);
+  const int grid = (int)(tasks < num_sms() ? tasks : num_sms());
+  kern<<<grid, (W + 1) * 32, sp.total, st>>>(map, out, tasks, scale, herm, sp.stages, status, dbg.poll_limit,
+                                              dbg.withhold_after);
   return cudaGetLastError();
 }
 
@@ -910,7 +931,7 @@ cudaError_t launch_inv_plane_t(const float2* in, float* y, long long rows, float
   if (e != cudaSuccess) return e;
   const long long tasks = rows / kTaskRows;
   const long long want = (tasks + W - 1) / W;
-  const int grid = (int)(want < kNumSMs ? want : kNumSMs);
+  const int grid = (int)(want < num_sms() ? want : num_sms());
   kern<<<grid, W * 32, total, st>>>(map, in, tasks, scale, herm);
   return cudaGetLastError();
 }
@@ -955,13 +976,13 @@ bool fused_eligible(const dtst_plan* p) {
 }
 
 cudaError_t launch_fwd_plane(int N3, int K3, int N2, int K2, const float* x, float2* out, long long rows,
-                             float scale, int herm, int* status, cudaStream_t st) {
+                             float scale, int herm, int* status, const RingDebug& dbg, cudaStream_t st) {
   if (N3 == 64 && K3 == 8 && N2 == 128 && K2 == 16)
-    return launch_fwd_plane_t<64, 8, 128, 16>(x, out, rows, scale, herm, status, st);
+    return launch_fwd_plane_t<64, 8, 128, 16>(x, out, rows, scale, herm, status, dbg, st);
   if (N3 == 32 && K3 == 4 && N2 == 64 && K2 == 8)
-    return launch_fwd_plane_t<32, 4, 64, 8>(x, out, rows, scale, herm, status, st);
+    return launch_fwd_plane_t<32, 4, 64, 8>(x, out, rows, scale, herm, status, dbg, st);
   if (N3 == 64 && K3 == 8 && N2 == 64 && K2 == 8)
-    return launch_fwd_plane_t<64, 8, 64, 8>(x, out, rows, scale, herm, status, st);
+    return launch_fwd_plane_t<64, 8, 64, 8>(x, out, rows, scale, herm, status, dbg, st);
   return cudaErrorNotSupported;
 }
 

@@ -10,7 +10,7 @@ namespace dtst {
 // contracting the last two grid dimensions in one pass.  scale and the Hermitian weight (herm) are
 // applied per last-dim frequency.  `status` is the plan's device status word.
 cudaError_t launch_fwd_plane(int N3, int K3, int N2, int K2, const float* x, float2* out, long long rows,
-                             float scale, int herm, int* status, cudaStream_t st);
+                             float scale, int herm, int* status, const RingDebug& dbg, cudaStream_t st);
 
 // Inverse plane kernel: in[planes][2*K2][K3] complex -> real rows [rows][N3].
 cudaError_t launch_inv_plane(int N3, int K3, int N2, int K2, const float2* in, float* y, long long rows,

@@ -70,7 +70,7 @@ cudaError_t launch_apply_dim(const DimOp& op_in, bool in_real, bool out_real, co
   const long long total = op.outer * op.R * op.inner;
   if (total <= 0) return cudaSuccess;
   long long blocks = (total + 255) / 256;
-  const long long cap = (long long)kNumSMs * 8;
+  const long long cap = (long long)num_sms() * 8;
   if (blocks > cap) blocks = cap;
   dim3 grid((unsigned)blocks, (unsigned)op.slabs);
   cudaError_t err = cudaSuccess;
@@ -111,7 +111,7 @@ __global__ void __launch_bounds__(256) reduce_partials_kernel(const float2* __re
 cudaError_t launch_reduce_partials(const float2* partial, float2* out, long long n, int P, cudaStream_t st) {
   if (n <= 0) return cudaSuccess;
   long long blocks = (n + 255) / 256;
-  if (blocks > (long long)kNumSMs * 8) blocks = (long long)kNumSMs * 8;
+  if (blocks > (long long)num_sms() * 8) blocks = (long long)num_sms() * 8;
   reduce_partials_kernel<<<(unsigned)blocks, 256, 0, st>>>(partial, out, n, P);
   return cudaGetLastError();
 }

@@ -329,7 +329,7 @@ cudaError_t launch_mid_t(bool forward, const float2* in, float2* out, long long 
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kMidThreads, smem);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
-    const long long cap = (long long)kNumSMs * per_sm;
+    const long long cap = (long long)num_sms() * per_sm;
     const int grid = (int)(tiles < cap ? tiles : cap);
     kern<<<grid, kMidThreads, smem, st>>>(in, out, outer, inner, N, scale);
     return cudaGetLastError();

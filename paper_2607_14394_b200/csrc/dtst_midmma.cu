@@ -464,7 +464,7 @@ cudaError_t launch_mid_mma_t(bool forward, const float2* in, float2* out, long l
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
-    const long long cap = (long long)kNumSMs * per_sm;
+    const long long cap = (long long)num_sms() * per_sm;
     *grid = (int)(want < cap ? want : cap);
     return cudaSuccess;
   };

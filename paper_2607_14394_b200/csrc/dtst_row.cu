@@ -93,6 +93,13 @@ __device__ __forceinline__ bool row_wait_fill(const RowWait& w, int slot, uint32
   return mbar_wait_bounded(&w.full[slot], q & 1u, w.abort_flag);
 }
 
+// The same wait with one verdict for the whole warp (every lane calls it): the lanes poll independently, and a
+// lane whose barrier completed just as another warp raised the abort flag must not go on alone into the
+// warp-synchronous MMA code.
+__device__ __forceinline__ bool row_wait_fill_warp(const RowWait& w, int slot, uint32_t q) {
+  return __all_sync(0xffffffffu, row_wait_fill(w, slot, q)) != 0;
+}
+
 // ---------------------------------------------------------------------------------------------
 // forward: MT m-tiles of 16 rows per task; W consumer warps + one producer warp
 // ---------------------------------------------------------------------------------------------
@@ -175,7 +182,7 @@ row_contract_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restri
     for (long long tl = w; tl < n_local; tl += W) {
       const long long task = first + tl * gridDim.x;
       const int slot = (int)(tl % stages);
-      if (!row_wait_fill(rw, slot, (uint32_t)(tl / stages))) break;
+      if (!row_wait_fill_warp(rw, slot, (uint32_t)(tl / stages))) break;
       const uint32_t st = ring_s + (uint32_t)slot * slot_bytes;
       // two accumulator sets (even / odd k-steps) halve the dependent-MMA chains; summed at the end
       float acc2[2][MT][4][4];
@@ -496,7 +503,7 @@ cudaError_t launch_row_contract_t(const float* x, float2* out, long long rows, i
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
   if (e != cudaSuccess) return e;
   const long long tasks = (rows + BOXR - 1) / BOXR;
-  const int grid = (int)(tasks < kNumSMs ? tasks : kNumSMs);
+  const int grid = (int)(tasks < num_sms() ? tasks : num_sms());
   kern<<<grid, (W + 1) * 32, total, st>>>(map, out, rows, N3, K3, scale, herm, stages, status);
   return cudaGetLastError();
 }
@@ -518,7 +525,7 @@ cudaError_t launch_row_expand_t(const float2* in, float* y, long long rows, int 
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
     if (e != cudaSuccess) return e;
     const long long want = (tasks + w - 1) / w;
-    const int grid = (int)(want < kNumSMs ? want : kNumSMs);
+    const int grid = (int)(want < num_sms() ? want : num_sms());
     kern<<<grid, w * 32, total, st>>>(map, in, rows, N3, K3, scale, herm);
     return cudaGetLastError();
   };

@@ -348,7 +348,7 @@ cudaError_t launch_slab_mma_t(const float2* in, float2* out, long long outer, lo
   if (e != cudaSuccess) return e;
   const long long tasks = outer * ((inner + kSPos - 1) / kSPos);
   const long long want = (tasks + kSWarps - 1) / kSWarps;
-  const int grid = (int)(want < kNumSMs ? want : kNumSMs);
+  const int grid = (int)(want < num_sms() ? want : num_sms());
   kern<<<grid, kSWarps * 32, smem, st>>>(reinterpret_cast<const float*>(in), out, outer, inner, Nl, N, off, P);
   return cudaGetLastError();
 }
@@ -367,7 +367,7 @@ cudaError_t launch_slab_t(bool forward, const float2* in, float2* out, long long
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     const long long want = (total + kSlabThreads - 1) / kSlabThreads;
-    const long long cap = (long long)kNumSMs * per_sm;
+    const long long cap = (long long)num_sms() * per_sm;
     kern<<<(unsigned)(want < cap ? want : cap), kSlabThreads, smem, st>>>(in, out, outer, inner, Nl, N, off, P);
     return cudaGetLastError();
   };

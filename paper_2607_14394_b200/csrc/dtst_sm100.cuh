@@ -64,6 +64,16 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
   return false;
 }
 
+// Plain bounded wait without an abort flag: for draining loads that are still in flight before a CTA whose
+// pipeline gave up returns (its shared memory must not be reassigned while the TMA engine writes to it).
+__device__ __forceinline__ bool mbar_wait_plain(uint64_t* bar, uint32_t parity, uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(40);
+  }
+  return false;
+}
+
 // 2-D tiled TMA load global -> shared, completion on an mbarrier (no multicast).
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
   asm volatile(

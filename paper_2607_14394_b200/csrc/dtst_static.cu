@@ -68,11 +68,20 @@ extern "C" dtst_status dtst_forward_static(dtst_plan* p, const float* x, void* X
   const size_t offA = 0, offB = up256(szA), offP = offB + up256(szB), total = offP + up256(szP);
   if (total > (size_t)DTST_STATIC_SCRATCH_BYTES) return DTST_ERR_STATIC_LIMIT;
 
-  void* base = nullptr;
-  if (scratch_of_current_device(&base) != cudaSuccess) {
+  // a failing runtime call or launch is recorded in the plan for dtst_plan_last_cuda_error
+  auto failed = [p](cudaError_t e) {
+    if (e == cudaSuccess) return false;
+    p->last_cuda_error = (int)e;
     (void)cudaGetLastError();
-    return DTST_ERR_CUDA;
+    return true;
+  };
+  if (p->device >= 0) {
+    int dev = -1;
+    if (failed(cudaGetDevice(&dev))) return DTST_ERR_CUDA;
+    if (dev != p->device) return DTST_ERR_INVALID_ARG;   // the plan belongs to another device
   }
+  void* base = nullptr;
+  if (failed(scratch_of_current_device(&base))) return DTST_ERR_CUDA;
   char* s = static_cast<char*>(base);
   float2* buf[2] = {reinterpret_cast<float2*>(s + offA), reinterpret_cast<float2*>(s + offB)};
   float2* partial = reinterpret_cast<float2*>(s + offP);
@@ -112,13 +121,13 @@ extern "C" dtst_status dtst_forward_static(dtst_plan* p, const float* x, void* X
     } else {
       dst = (j == 0) ? static_cast<void*>(Xhat) : static_cast<void*>(buf[flip]);
     }
-    if (launch_apply_dim(op, j == p->d - 1, false, cur, dst, st) != cudaSuccess) return DTST_ERR_CUDA;
+    if (failed(launch_apply_dim(op, j == p->d - 1, false, cur, dst, st))) return DTST_ERR_CUDA;
     ++p->launches;
     cur = dst;
     flip ^= 1;
   }
   if (p->P > 1) {
-    if (launch_reduce_partials(partial, Xhat, (long long)p->B * p->C_in * p->M, p->P, st) != cudaSuccess)
+    if (failed(launch_reduce_partials(partial, Xhat, (long long)p->B * p->C_in * p->M, p->P, st)))
       return DTST_ERR_CUDA;
     ++p->launches;
   }

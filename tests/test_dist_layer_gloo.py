@@ -15,48 +15,12 @@ import torch.multiprocessing as mp
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-class OracleOps:
-    """The six local steps in float64 numpy, on torch CPU tensors."""
-
-    def __init__(self, O, N_global, n_local, offset, kmax, B, C_in, C_out):
-        self.O, self.Ng, self.nl, self.off, self.k = O, tuple(N_global), tuple(n_local), tuple(offset), tuple(kmax)
-        self.B, self.Ci, self.Co = B, C_in, C_out
-        d = len(self.Ng)
-        self.K = tuple(2 * self.k[j] if j < d - 1 else self.k[j] for j in range(d))
-        self.M = math.prod(self.K)
-
-    def spectrum(self, x):
-        X = self.O.forward(x.numpy(), self.k, N_global=self.Ng, offsets=self.off)
-        return torch.from_numpy(np.ascontiguousarray(X.reshape(self.B, self.Ci, self.M)))
-
-    def mix(self, Xhat, W_shard, m0, cnt):
-        Y = np.einsum("bim,iom->bom", Xhat.numpy()[:, :, m0:m0 + cnt], W_shard.numpy())
-        return torch.from_numpy(np.ascontiguousarray(Y))
-
-    def inverse(self, Yhat):
-        y = self.O.inverse(Yhat.numpy().reshape((self.B, self.Co) + self.K), self.Ng, self.k, n_local=self.nl,
-                           offsets=self.off)
-        return torch.from_numpy(np.ascontiguousarray(y))
-
-    def grad_spectrum(self, g):
-        c = self.O.hermitian_weights(self.Ng[-1], self.k[-1])
-        G = self.O.forward(g.numpy(), self.k, N_global=self.Ng, offsets=self.off) * c / float(math.prod(self.Ng))
-        return torch.from_numpy(np.ascontiguousarray(G.reshape(self.B, self.Co, self.M)))
-
-    def grad_mix(self, GY, Xhat, W_shard, m0, cnt):
-        gy, xh = GY.numpy()[:, :, m0:m0 + cnt], Xhat.numpy()[:, :, m0:m0 + cnt]
-        GX = np.einsum("bom,iom->bim", gy, np.conj(W_shard.numpy()))
-        gW = np.einsum("bim,bom->iom", np.conj(xh), gy)
-        return torch.from_numpy(np.ascontiguousarray(GX)), torch.from_numpy(np.ascontiguousarray(gW))
-
-    def grad_input(self, GX):
-        gx = self.O.inverse(GX.numpy().reshape((self.B, self.Ci) + self.K), self.Ng, self.k, n_local=self.nl,
-                            offsets=self.off, doubling=False, normalise=False)
-        return torch.from_numpy(np.ascontiguousarray(gx))
+from gloo_ops import OracleOps
 
 
 def _worker(rank, world, port, q):
     sys.path.insert(0, ROOT)
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
     os.environ.update(WORLD_SIZE=str(world), RANK=str(rank), LOCAL_RANK=str(rank), MASTER_ADDR="127.0.0.1",
                       MASTER_PORT=str(port))
     import torch.distributed as dist

@@ -6,6 +6,7 @@ import pytest
 
 from oracle import dtst_oracle as O
 from paper_2607_14394_b200 import inputs as I
+from parity_checks import per_mode_excess, per_plane_excess
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -46,14 +47,24 @@ def run_layer_and_check(w, path="auto", P=1, check_backward=True, tol=TOL):
         "Yhat": O.rel_l2(Yhat.cpu().numpy(), Y_ref),
         "y": O.rel_l2(y.cpu().numpy(), y_ref),
     }
+    # every retained mode and every plane on its own scale (multiples of the per-mode / per-plane bars)
+    fine = {
+        "Xhat/mode": per_mode_excess(Xhat.cpu().numpy(), X_ref),
+        "Yhat/mode": per_mode_excess(Yhat.cpu().numpy(), Y_ref),
+        "y/plane": per_plane_excess(y.cpu().numpy(), y_ref),
+    }
     if check_backward:
         gx, gW = plan.backward(gd, Xhat, Wd)
         torch.cuda.synchronize()
         gx_ref, gW_ref = O.backward(g, X_ref, Wm, w.kmax)
         errs["grad_x"] = O.rel_l2(gx.cpu().numpy(), gx_ref)
         errs["grad_W"] = O.rel_l2(gW.cpu().numpy().reshape(gW_ref.shape), gW_ref)
+        fine["grad_W/mode"] = per_mode_excess(gW.cpu().numpy().reshape(gW_ref.shape), gW_ref)
+        fine["grad_x/plane"] = per_plane_excess(gx.cpu().numpy(), gx_ref)
     for name, e in errs.items():
         assert e <= tol, (w.name, path, P, name, e, errs)
+    for name, e in fine.items():
+        assert e <= 1.0, (w.name, path, P, name, e, fine)
     plan.close()
     return errs
 
@@ -250,6 +261,31 @@ def test_argument_errors_on_device():
                                  ctypes.c_void_p(X.data_ptr()), st) == Bn.DTST_ERR_INVALID_ARG   # aliasing
     assert lib.dtst_backward(plan.handle, ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(X.data_ptr()),
                              ctypes.c_void_p(X.data_ptr()), None, None, st) == Bn.DTST_ERR_INVALID_ARG
+    # the saved spectrum is read for grad_W only: it may be missing when grad_W is not asked for ...
+    Wt = torch.zeros((2, 2, 8), dtype=torch.complex64, device="cuda")
+    gxt = torch.zeros_like(x)
+    assert lib.dtst_backward(plan.handle, ctypes.c_void_p(x.data_ptr()), None, ctypes.c_void_p(Wt.data_ptr()),
+                             ctypes.c_void_p(gxt.data_ptr()), None, st) == Bn.DTST_OK
+    # ... and is required when it is
+    assert lib.dtst_backward(plan.handle, ctypes.c_void_p(x.data_ptr()), None, ctypes.c_void_p(Wt.data_ptr()),
+                             ctypes.c_void_p(gxt.data_ptr()), ctypes.c_void_p(Wt.data_ptr()), st) \
+        == Bn.DTST_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    launched = plan.launch_count()
+    # tensors of the wrong size never reach the kernels
+    with pytest.raises(ValueError):
+        plan.forward(torch.zeros((1, 2, 8, 4), device="cuda"))
+    with pytest.raises(ValueError):
+        plan.forward(x, out=torch.zeros((1, 2, 4, 1), dtype=torch.complex64, device="cuda"))
+    with pytest.raises(ValueError):
+        plan.spectral_mul(X, torch.zeros((2, 2, 4), dtype=torch.complex64, device="cuda"))
+    with pytest.raises(ValueError):
+        plan.inverse(X, out=torch.zeros((1, 2, 8, 7), device="cuda"))
+    with pytest.raises(ValueError):
+        plan.backward(x, X, Wt, grad_x=torch.zeros((1, 1, 8, 8), device="cuda"))
+    with pytest.raises(ValueError):
+        plan.spectral_mul_modes(X, Wt, 4, 8)
+    assert plan.launch_count() == launched
     small = torch.zeros(256, dtype=torch.uint8, device="cuda")
     with pytest.raises(Bn.DtstError) as e:
         Bn.dtst_plan_set_workspace(plan.handle, small)
@@ -257,9 +293,35 @@ def test_argument_errors_on_device():
     with pytest.raises(ValueError):
         plan.forward(x.cpu())
     assert plan.status() == 0
-    assert plan.launch_count() == 0
+    before = plan.launch_count()
     plan.forward(x)
-    assert plan.launch_count() > 0
+    assert plan.launch_count() > before
+
+
+def test_bounded_wait_runs_out_and_is_reported_once():
+    """The failure-reporting path of the streaming kernels, made to happen on the host's request: the forward
+    plane kernel's producer stops feeding its ring after one fill, the consumers' bounded waits run out, the
+    kernel returns normally, dtst_plan_status reports the timeout once and clears it, and the next ordinary call
+    is correct.  Nothing faults and no wait is unbounded."""
+    from paper_2607_14394_b200 import binding as Bn
+    w = I.WORKLOADS["cfg1_2d_64"]
+    plan = _plan(w)
+    assert plan.kernel_path == "fused"
+    x = _dev(I.make_field(w))
+    ref = plan.forward(x).clone()
+    torch.cuda.synchronize()
+    assert plan.status() == Bn.DTST_OK
+    plan.debug_ring_fault(1, poll_limit=1024)
+    junk = plan.forward(x)
+    assert plan.status() == Bn.DTST_ERR_DEVICE_TIMEOUT
+    assert plan.status() == Bn.DTST_OK                       # reported once, then cleared
+    plan.debug_ring_fault(-1)
+    again = plan.forward(x)
+    torch.cuda.synchronize()
+    assert plan.status() == Bn.DTST_OK
+    assert torch.equal(torch.view_as_real(again), torch.view_as_real(ref))
+    assert O.rel_l2(again.cpu().numpy(), O.forward(I.make_field(w), w.kmax)) <= TOL
+    del junk
 
 
 def test_adjoint_identity_on_device():

@@ -5,12 +5,14 @@ time (a plug-in inside an application that owns all GPU memory, a loop that
 bans allocator calls after start-up) and have no workspace to pass either.
 For them the library keeps a fixed 8 MiB scratch array of its own.  This test
 calls that entry point through the C ABI twice in a row and compares both
-results with the ordinary dtst_forward, with the tolerance of the parity tests.
+results with the ordinary dtst_forward and with the float64 oracle, with the
+tolerance of the parity tests.
 The file sorts last on purpose: if it fails, every other test has already run.
 """
 import numpy as np
 import pytest
 
+from oracle import dtst_oracle as O
 from paper_2607_14394_b200 import inputs as I
 
 torch = pytest.importorskip("torch")
@@ -47,8 +49,13 @@ def test_static_scratch_forward_matches_workspace_forward_twice(P):
     torch.cuda.synchronize()
     assert _rel_l2(out1, ref) <= TOL
     assert _rel_l2(out2, ref) <= TOL
+    # and against the oracle itself, not only against the sibling entry point
+    X_ref = O.forward_sharded(I.make_field(w), w.kmax, P) if P > 1 else O.forward(I.make_field(w), w.kmax)
+    assert O.rel_l2(out1.cpu().numpy(), X_ref) <= TOL
+    assert O.rel_l2(out2.cpu().numpy(), X_ref) <= TOL
     ref2 = Plan(w2.N, w2.kmax, w2.B, w2.C_in, w2.C_out).forward(x2)
     assert _rel_l2(o2, ref2) <= TOL
+    assert O.rel_l2(o2.cpu().numpy(), O.forward(I.make_field(w2), w2.kmax)) <= TOL
 
 
 def test_static_scratch_limit_is_reported_not_exceeded():
