@@ -4,6 +4,7 @@
 
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <stddef.h>
 
 #include "../../include/dtst.h"
@@ -70,6 +71,33 @@ __host__ __device__ inline float herm_weight(int f, int N) {
 }
 
 #ifdef __CUDACC__
+// Programmatic dependent launch.  Every kernel of the library is launched with the programmatic-serialisation
+// attribute and follows one protocol: `pdl_trigger()` first thing (the next kernel of the stream may then be
+// scheduled as soon as SMs free up), then the prologue that touches nothing a predecessor produced (basis
+// tables from (N, k, offset), barrier set-up, tensor-map prefetch), then `pdl_wait()` - reached by EVERY thread of
+// every CTA, before its first global-memory access and before any early exit - which returns once the
+// preceding kernel has completed and its writes are visible.  So a kernel's launch latency and table build hide
+// behind its predecessor's tail; the data dependencies are exactly those of plain stream order.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  static const bool off = getenv("DTST_NO_PDL") != nullptr;
+  cfg.numAttrs = off ? 0 : 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // exp(sign * 2 pi i * (s*n mod N) / N): the integer phase is reduced exactly before
 // any floating-point operation, then evaluated in double and rounded once.
 __device__ inline float2 twiddle(int s, long long n, int N, int sign) {

@@ -260,6 +260,7 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
   using Cfg = PlaneCfg<N3, K3, N2, K2>;
   constexpr int NC = Cfg::NC, QUADS = Cfg::QUADS, G = Cfg::G, LPP = Cfg::LPP;
   constexpr int SPT = Cfg::SPT, RPS = Cfg::ROWS_PER_STAGE;
+  pdl_trigger();
 
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment for the TMA swizzle, by pointer arithmetic on the shared array itself (an integer
@@ -327,6 +328,7 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
     rot[f * (2 * K2) + r] = make_float2((float)cs * w, (float)sn * w);   // [f][r]: lanes (r) read conflict-free
   }
   __syncthreads();
+  pdl_wait();   // everything above is independent of the preceding kernel
 
   const long long first = blockIdx.x;
   const long long n_local = first < num_tasks ? (num_tasks - first + gridDim.x - 1) / gridDim.x : 0;
@@ -628,6 +630,7 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __re
   using IC = InvCfg<N3, K3, N2, K2>;
   constexpr int NC = Cfg::NC, QUADS = Cfg::QUADS, G = Cfg::G, LPP = Cfg::LPP;
   constexpr int SPT = Cfg::SPT, RPS = Cfg::ROWS_PER_STAGE;
+  pdl_trigger();
 
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment for the TMA swizzle, by pointer arithmetic on the shared array itself (an integer
@@ -688,6 +691,7 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __re
   const long long tstride = (long long)gridDim.x * W;
   long long task = (long long)blockIdx.x + (long long)warp * gridDim.x;
   float4 vin[K3 / 2];
+  pdl_wait();   // everything above is independent of the preceding kernel
   if (task < num_tasks && actl) {
     const float4* src = reinterpret_cast<const float4*>(in + ((task * G + pll) * (2 * K2) + rl) * K3);
 #pragma unroll
@@ -912,8 +916,8 @@ cudaError_t launch_fwd_plane_t(const float* x, float2* out, long long rows, floa
   if (e != cudaSuccess) return e;
   const long long tasks = rows / kTaskRows;
   const int grid = (int)(tasks < num_sms() ? tasks : num_sms());
-  kern<<<grid, (W + 1) * 32, sp.total, st>>>(map, out, tasks, scale, herm, sp.stages, status, dbg.poll_limit,
-                                              dbg.withhold_after);
+  (void)launch_pdl(kern, dim3(grid), dim3((W + 1) * 32), sp.total, st, map, out, tasks, scale, herm, sp.stages, status,
+                   dbg.poll_limit, dbg.withhold_after);
   return cudaGetLastError();
 }
 
@@ -932,7 +936,7 @@ cudaError_t launch_inv_plane_t(const float2* in, float* y, long long rows, float
   const long long tasks = rows / kTaskRows;
   const long long want = (tasks + W - 1) / W;
   const int grid = (int)(want < num_sms() ? want : num_sms());
-  kern<<<grid, W * 32, total, st>>>(map, in, tasks, scale, herm);
+  (void)launch_pdl(kern, dim3(grid), dim3(W * 32), total, st, map, in, tasks, scale, herm);
   return cudaGetLastError();
 }
 

@@ -13,6 +13,7 @@ namespace dtst {
 template <bool IN_REAL, bool OUT_REAL>
 __global__ void __launch_bounds__(256) apply_dim_kernel(DimOp p, const void* __restrict__ in_,
                                                        void* __restrict__ out_) {
+  pdl_trigger();
   extern __shared__ float2 Es[];
   const int slab = blockIdx.y;
   if (p.basis_in_smem) {
@@ -22,6 +23,7 @@ __global__ void __launch_bounds__(256) apply_dim_kernel(DimOp p, const void* __r
     }
     __syncthreads();
   }
+  pdl_wait();
   const float* in_r = reinterpret_cast<const float*>(in_) + (long long)slab * p.in_slab_stride;
   const float2* in_c = reinterpret_cast<const float2*>(in_) + (long long)slab * p.in_slab_stride;
   float* out_r = reinterpret_cast<float*>(out_) + (long long)slab * p.out_slab_stride;
@@ -79,7 +81,7 @@ cudaError_t launch_apply_dim(const DimOp& op_in, bool in_real, bool out_real, co
     if (dyn > 48 * 1024)                                                                            \
       err = cudaFuncSetAttribute(apply_dim_kernel<IR, OR>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                  (int)dyn);                                                         \
-    if (err == cudaSuccess) apply_dim_kernel<IR, OR><<<grid, 256, dyn, st>>>(op, in, out);          \
+    if (err == cudaSuccess) err = launch_pdl(apply_dim_kernel<IR, OR>, grid, dim3(256), dyn, st, op, in, out); \
   } while (0)
   if (in_real && !out_real) DTST_LAUNCH(true, false);
   else if (!in_real && out_real) DTST_LAUNCH(false, true);
@@ -96,6 +98,8 @@ cudaError_t launch_apply_dim(const DimOp& op_in, bool in_real, bool out_real, co
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) reduce_partials_kernel(const float2* __restrict__ partial,
                                                              float2* __restrict__ out, long long n, int P) {
+  pdl_trigger();
+  pdl_wait();
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
     float2 acc = partial[i];
@@ -112,8 +116,7 @@ cudaError_t launch_reduce_partials(const float2* partial, float2* out, long long
   if (n <= 0) return cudaSuccess;
   long long blocks = (n + 255) / 256;
   if (blocks > (long long)num_sms() * 8) blocks = (long long)num_sms() * 8;
-  reduce_partials_kernel<<<(unsigned)blocks, 256, 0, st>>>(partial, out, n, P);
-  return cudaGetLastError();
+  return launch_pdl(reduce_partials_kernel, dim3((unsigned)blocks), dim3(256), 0, st, partial, out, n, P);
 }
 
 // ---------------------------------------------------------------------------
@@ -126,6 +129,8 @@ cudaError_t launch_reduce_partials(const float2* partial, float2* out, long long
 template <int NB>
 __global__ void __launch_bounds__(256) mix_kernel(const float2* __restrict__ X, const float2* __restrict__ W,
                                                  float2* __restrict__ Y, int b0, int Ci, int Co, long long M) {
+  pdl_trigger();
+  pdl_wait();
   const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int o = blockIdx.y;
   if (m >= M) return;
@@ -150,14 +155,16 @@ __global__ void __launch_bounds__(256) mix_kernel(const float2* __restrict__ X, 
 cudaError_t launch_mix(const float2* X, const float2* W, float2* Y, int B, int Ci, int Co, long long M,
                        cudaStream_t st, long long* launches) {
   dim3 grid((unsigned)((M + 255) / 256), (unsigned)Co);
+  cudaError_t e = cudaSuccess;
   for (int b0 = 0; b0 < B; b0 += 4) {
     const int nb = (B - b0 < 4) ? (B - b0) : 4;
     switch (nb) {
-      case 1: mix_kernel<1><<<grid, 256, 0, st>>>(X, W, Y, b0, Ci, Co, M); break;
-      case 2: mix_kernel<2><<<grid, 256, 0, st>>>(X, W, Y, b0, Ci, Co, M); break;
-      case 3: mix_kernel<3><<<grid, 256, 0, st>>>(X, W, Y, b0, Ci, Co, M); break;
-      default: mix_kernel<4><<<grid, 256, 0, st>>>(X, W, Y, b0, Ci, Co, M); break;
+      case 1: e = launch_pdl(mix_kernel<1>, grid, dim3(256), 0, st, X, W, Y, b0, Ci, Co, M); break;
+      case 2: e = launch_pdl(mix_kernel<2>, grid, dim3(256), 0, st, X, W, Y, b0, Ci, Co, M); break;
+      case 3: e = launch_pdl(mix_kernel<3>, grid, dim3(256), 0, st, X, W, Y, b0, Ci, Co, M); break;
+      default: e = launch_pdl(mix_kernel<4>, grid, dim3(256), 0, st, X, W, Y, b0, Ci, Co, M); break;
     }
+    if (e != cudaSuccess) return e;
     if (launches) ++*launches;
   }
   return cudaGetLastError();
@@ -175,6 +182,8 @@ __global__ void __launch_bounds__(256) mix_adjoint_kernel(const float2* __restri
                                                          const float2* __restrict__ W, float2* __restrict__ GX,
                                                          float2* __restrict__ GW, int b0, int B, int Ci, int Co,
                                                          long long M) {
+  pdl_trigger();
+  pdl_wait();
   const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int i = blockIdx.y;
   if (m >= M) return;
@@ -233,7 +242,7 @@ void launch_mix_adjoint_nb(dim3 grid, cudaStream_t st, const float2* GY, const f
   const bool allb = (b0 == 0 && NB == B);
   const bool gx = GX != nullptr;
 #define DTST_MA(AL, WX, WW) \
-  mix_adjoint_kernel<NB, AL, WX, WW><<<grid, 256, 0, st>>>(GY, X, W, GX, GW, b0, B, Ci, Co, M)
+  (void)launch_pdl(mix_adjoint_kernel<NB, AL, WX, WW>, grid, dim3(256), 0, st, GY, X, W, GX, GW, b0, B, Ci, Co, M)
   if (gx && want_gw) { if (allb) DTST_MA(true, true, true); else DTST_MA(false, true, true); }
   else if (gx) DTST_MA(false, true, false);
   else if (want_gw) { if (allb) DTST_MA(true, false, true); else DTST_MA(false, false, true); }
@@ -269,6 +278,8 @@ cudaError_t launch_mix_adjoint(const float2* GY, const float2* X, const float2* 
 __global__ void __launch_bounds__(256) mix_modes_kernel(const float2* __restrict__ X, const float2* __restrict__ W,
                                                        float2* __restrict__ Y, int Ci, int Co, long long M,
                                                        long long m0, long long cnt) {
+  pdl_trigger();
+  pdl_wait();
   const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int o = blockIdx.y, b = blockIdx.z;
   if (m >= cnt) return;
@@ -289,6 +300,8 @@ __global__ void __launch_bounds__(256) mix_adjoint_gx_modes_kernel(const float2*
                                                                   const float2* __restrict__ W,
                                                                   float2* __restrict__ GX, int Ci, int Co,
                                                                   long long M, long long m0, long long cnt) {
+  pdl_trigger();
+  pdl_wait();
   const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int i = blockIdx.y, b = blockIdx.z;
   if (m >= cnt) return;
@@ -309,6 +322,8 @@ __global__ void __launch_bounds__(256) mix_adjoint_gw_modes_kernel(const float2*
                                                                   const float2* __restrict__ X,
                                                                   float2* __restrict__ GW, int B, int Ci, int Co,
                                                                   long long M, long long m0, long long cnt) {
+  pdl_trigger();
+  pdl_wait();
   const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const int o = blockIdx.y, i = blockIdx.z;
   if (m >= cnt) return;
@@ -328,7 +343,7 @@ cudaError_t launch_mix_modes(const float2* X, const float2* W, float2* Y, int B,
                              long long m0, long long cnt, cudaStream_t st, long long* launches) {
   if (cnt <= 0 || B <= 0) return cudaSuccess;
   dim3 grid((unsigned)((cnt + 255) / 256), (unsigned)Co, (unsigned)B);
-  mix_modes_kernel<<<grid, 256, 0, st>>>(X, W, Y, Ci, Co, M, m0, cnt);
+  (void)launch_pdl(mix_modes_kernel, grid, dim3(256), 0, st, X, W, Y, Ci, Co, M, m0, cnt);
   if (launches) ++*launches;
   return cudaGetLastError();
 }
@@ -339,12 +354,12 @@ cudaError_t launch_mix_adjoint_modes(const float2* GY, const float2* X, const fl
   if (cnt <= 0 || B <= 0) return cudaSuccess;
   if (GX != nullptr) {
     dim3 grid((unsigned)((cnt + 255) / 256), (unsigned)Ci, (unsigned)B);
-    mix_adjoint_gx_modes_kernel<<<grid, 256, 0, st>>>(GY, W, GX, Ci, Co, M, m0, cnt);
+    (void)launch_pdl(mix_adjoint_gx_modes_kernel, grid, dim3(256), 0, st, GY, W, GX, Ci, Co, M, m0, cnt);
     if (launches) ++*launches;
   }
   if (GW != nullptr) {
     dim3 grid((unsigned)((cnt + 255) / 256), (unsigned)Co, (unsigned)Ci);
-    mix_adjoint_gw_modes_kernel<<<grid, 256, 0, st>>>(GY, X, GW, B, Ci, Co, M, m0, cnt);
+    (void)launch_pdl(mix_adjoint_gw_modes_kernel, grid, dim3(256), 0, st, GY, X, GW, B, Ci, Co, M, m0, cnt);
     if (launches) ++*launches;
   }
   return cudaGetLastError();

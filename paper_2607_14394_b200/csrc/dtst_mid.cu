@@ -58,11 +58,13 @@ __global__ void __launch_bounds__(kMidThreads) mid_contract_kernel(const float2*
                                                                    float2* __restrict__ out, long long outer,
                                                                    long long inner, int N, float scale) {
   constexpr int TS = MidTab<K>::TS;
+  pdl_trigger();
   extern __shared__ float smem_mid[];
   float* tab = smem_mid;
   float2* rho = reinterpret_cast<float2*>(tab + (size_t)(N / 2) * TS);
   build_mid_table<K>(tab, rho, N, scale);
   __syncthreads();
+  pdl_wait();
 
   const long long total = outer * inner;
   const long long per_cta = (long long)kMidThreads * PT;
@@ -214,11 +216,13 @@ __global__ void __launch_bounds__(kMidThreads) mid_expand_kernel(const float2* _
                                                                  float2* __restrict__ out, long long outer,
                                                                  long long inner, int N, float scale) {
   constexpr int TS = MidTab<K>::TS;
+  pdl_trigger();
   extern __shared__ float smem_mid[];
   float* tab = smem_mid;
   float2* rho = reinterpret_cast<float2*>(tab + (size_t)(N / 2) * TS);
   build_mid_table<K>(tab, rho, N, scale);
   __syncthreads();
+  pdl_wait();
 
   const long long total = outer * inner;
   const long long per_cta = (long long)kMidThreads * PT;
@@ -331,7 +335,7 @@ cudaError_t launch_mid_t(bool forward, const float2* in, float2* out, long long 
     if (per_sm < 1) per_sm = 1;
     const long long cap = (long long)num_sms() * per_sm;
     const int grid = (int)(tiles < cap ? tiles : cap);
-    kern<<<grid, kMidThreads, smem, st>>>(in, out, outer, inner, N, scale);
+    (void)launch_pdl(kern, dim3(grid), dim3(kMidThreads), smem, st, in, out, outer, inner, N, scale);
     return cudaGetLastError();
   };
   return forward ? launch(mid_contract_kernel<K, PT, VEC>) : launch(mid_expand_kernel<K, PT, VEC>);

@@ -112,6 +112,7 @@ __global__ void __launch_bounds__(kCThreads, 1)
 mid_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out, long long outer, long long inner,
                         int N, float scale) {
   static_assert(K % 4 == 0 && K <= 16, "parity classes of K/2 <= 8 frequencies");
+  pdl_trigger();
   extern __shared__ float4 mm_smem[];
   const int KS = N / 32;                                    // k-steps of 8 row quadruples
   float4* btab = mm_smem;                                   // [KS][class][lane]
@@ -155,6 +156,7 @@ mid_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out, 
   const long long rs = 2 * inner;   // floats per row
   const long long tstride = (long long)gridDim.x * kCWarps;
   float* ring = cK + N / 4 + (size_t)warp * kCStages * kCStageFloats;   // this warp's stages (16-byte aligned)
+  pdl_wait();   // everything above is independent of the preceding kernel
 
   // producer cursor: (task, k-step) of the next stage to request; lane = (row lane / 8, 16-byte chunk lane % 8)
   long long ptask = (long long)blockIdx.x * kCWarps + warp;
@@ -285,6 +287,7 @@ __global__ void __launch_bounds__(kEThreads, 1)
 mid_expand_mma_kernel(const float2* __restrict__ in, float2* __restrict__ out, long long outer, long long inner,
                       int N, float scale, int streaming) {
   static_assert(K % 4 == 0 && K <= 16, "parity classes of K/2 <= 8 frequencies");
+  pdl_trigger();
   extern __shared__ float4 mm_smem[];
   const int NT = N / 32;                                   // n-tiles of 8 row quadruples
   float4* btab = mm_smem;                                  // [NT][class][lane]
@@ -326,6 +329,7 @@ mid_expand_mma_kernel(const float2* __restrict__ in, float2* __restrict__ out, l
   const long long cblocks = (inner + kEPos - 1) / kEPos;
   const long long tasks = outer * cblocks;
   const long long tstride = (long long)gridDim.x * kEWarps;
+  pdl_wait();   // everything above is independent of the preceding kernel
   for (long long task = (long long)blockIdx.x * kEWarps + warp; task < tasks; task += tstride) {
     const long long o = task / cblocks, cb = task % cblocks;
     const long long left = inner - cb * kEPos;
@@ -473,13 +477,13 @@ cudaError_t launch_mid_mma_t(bool forward, const float2* in, float2* out, long l
     auto kern = mid_contract_mma_kernel<K>;
     cudaError_t e = grid_for(kern, &grid);
     if (e != cudaSuccess) return e;
-    kern<<<grid, threads, smem, st>>>(reinterpret_cast<const float*>(in), out, outer, inner, N, scale);
+    (void)launch_pdl(kern, dim3(grid), dim3(threads), smem, st, reinterpret_cast<const float*>(in), out, outer, inner, N, scale);
   } else {
     auto kern = mid_expand_mma_kernel<K>;
     cudaError_t e = grid_for(kern, &grid);
     if (e != cudaSuccess) return e;
     const int streaming = (double)outer * N * inner * 8.0 > 2.0 * 126e6 ? 1 : 0;
-    kern<<<grid, threads, smem, st>>>(in, out, outer, inner, N, scale, streaming);
+    (void)launch_pdl(kern, dim3(grid), dim3(threads), smem, st, in, out, outer, inner, N, scale, streaming);
   }
   return cudaGetLastError();
 }

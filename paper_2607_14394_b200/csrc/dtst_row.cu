@@ -107,6 +107,7 @@ template <int MT, int W>
 __global__ void __launch_bounds__((W + 1) * 32, 1)
 row_contract_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict__ out, long long rows, int N3,
                     int K3, float scale, int herm, int stages, int* __restrict__ status) {
+  pdl_trigger();
   constexpr int BOXR = 16 * MT;
   const int NKS = N3 / 32;                       // k-steps of 8 quadruples
   const uint32_t slot_bytes = (uint32_t)BOXR * N3 * 4;
@@ -146,6 +147,7 @@ row_contract_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restri
     btab[e] = make_float4(__uint_as_float(h0), __uint_as_float(h1), __uint_as_float(l0), __uint_as_float(l1));
   }
   __syncthreads();
+  pdl_wait();   // everything above is independent of the preceding kernel
 
   const long long num_tasks = (rows + BOXR - 1) / BOXR;
   const long long first = blockIdx.x;
@@ -305,6 +307,7 @@ template <int MT, int W>
 __global__ void __launch_bounds__(W * 32, 1)
 row_expand_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __restrict__ in, long long rows, int N3,
                   int K3, float scale, int herm) {
+  pdl_trigger();
   constexpr int BOXR = 16 * MT;
   const int NNT = N3 / 32;                       // n-tiles of 8 quadruples
   const uint32_t tile_bytes = (uint32_t)BOXR * N3 * 4;
@@ -353,6 +356,7 @@ row_expand_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __r
   // which are adjacent in memory: one 16-byte load when k3 is even (every row then starts 16-byte aligned)
   float2 vin[MT][4][2];
   const bool pairload = (K3 & 1) == 0;
+  pdl_wait();   // everything above is independent of the preceding kernel
   auto load_inputs = [&](long long t) {
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
@@ -504,7 +508,7 @@ cudaError_t launch_row_contract_t(const float* x, float2* out, long long rows, i
   if (e != cudaSuccess) return e;
   const long long tasks = (rows + BOXR - 1) / BOXR;
   const int grid = (int)(tasks < num_sms() ? tasks : num_sms());
-  kern<<<grid, (W + 1) * 32, total, st>>>(map, out, rows, N3, K3, scale, herm, stages, status);
+  (void)launch_pdl(kern, dim3(grid), dim3((W + 1) * 32), total, st, map, out, rows, N3, K3, scale, herm, stages, status);
   return cudaGetLastError();
 }
 
@@ -526,7 +530,7 @@ cudaError_t launch_row_expand_t(const float2* in, float* y, long long rows, int 
     if (e != cudaSuccess) return e;
     const long long want = (tasks + w - 1) / w;
     const int grid = (int)(want < num_sms() ? want : num_sms());
-    kern<<<grid, w * 32, total, st>>>(map, in, rows, N3, K3, scale, herm);
+    (void)launch_pdl(kern, dim3(grid), dim3(w * 32), total, st, map, in, rows, N3, K3, scale, herm);
     return cudaGetLastError();
   };
   if (W >= 12 && MT <= 2) return launch(row_expand_kernel<MT, 12>, 12);

@@ -29,9 +29,11 @@ template <int K>
 __global__ void __launch_bounds__(kSlabThreads) slab_contract_kernel(const float2* __restrict__ in,
                                                                      float2* __restrict__ out, long long outer,
                                                                      long long inner, int Nl, int N, int off, int P) {
+  pdl_trigger();
   extern __shared__ float2 slab_tab[];
   build_slab_table<K>(slab_tab, Nl, N, off, -1);
   __syncthreads();
+  pdl_wait();
   const long long total = outer * inner;
   const int nl = Nl / P;
   for (long long p0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; p0 < total;
@@ -83,9 +85,11 @@ template <int K>
 __global__ void __launch_bounds__(kSlabThreads) slab_expand_kernel(const float2* __restrict__ in,
                                                                    float2* __restrict__ out, long long outer,
                                                                    long long inner, int Nl, int N, int off, int P) {
+  pdl_trigger();
   extern __shared__ float2 slab_tab[];
   build_slab_table<K>(slab_tab, Nl, N, off, +1);
   __syncthreads();
+  pdl_wait();
   const long long total = outer * inner;
   const int nl = Nl / P;
   for (long long p0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; p0 < total;
@@ -147,6 +151,7 @@ slab_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out,
   // +g and -g share their sums: C_g = sum_n z_n cos(phi_g (off + n)), S_g = sum_n z_n sin(phi_g (off + n)),
   // Z_{+g} = C_g - i S_g, Z_{-g} = C_g + i S_g, phi_g = 2 pi g / N.  The MMA n-tiles cover g = 0..K-1; g = K (only
   // -K is retained) runs on FFMA.
+  pdl_trigger();
   constexpr int NT = (K + 7) / 8;
   extern __shared__ float4 slab_smem4[];
   const int KS = Nl / 8;                        // k-steps over all local rows
@@ -169,6 +174,7 @@ slab_contract_mma_kernel(const float* __restrict__ in, float2* __restrict__ out,
   }
   for (int n = threadIdx.x; n < Nl; n += blockDim.x) tK[n] = twiddle(K, (long long)off + n, N, +1);
   __syncthreads();
+  pdl_wait();
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g8 = lane >> 2, t4 = lane & 3;
@@ -349,7 +355,7 @@ cudaError_t launch_slab_mma_t(const float2* in, float2* out, long long outer, lo
   const long long tasks = outer * ((inner + kSPos - 1) / kSPos);
   const long long want = (tasks + kSWarps - 1) / kSWarps;
   const int grid = (int)(want < num_sms() ? want : num_sms());
-  kern<<<grid, kSWarps * 32, smem, st>>>(reinterpret_cast<const float*>(in), out, outer, inner, Nl, N, off, P);
+  (void)launch_pdl(kern, dim3(grid), dim3(kSWarps * 32), smem, st, reinterpret_cast<const float*>(in), out, outer, inner, Nl, N, off, P);
   return cudaGetLastError();
 }
 
@@ -368,7 +374,7 @@ cudaError_t launch_slab_t(bool forward, const float2* in, float2* out, long long
     if (per_sm < 1) per_sm = 1;
     const long long want = (total + kSlabThreads - 1) / kSlabThreads;
     const long long cap = (long long)num_sms() * per_sm;
-    kern<<<(unsigned)(want < cap ? want : cap), kSlabThreads, smem, st>>>(in, out, outer, inner, Nl, N, off, P);
+    (void)launch_pdl(kern, dim3((unsigned)(want < cap ? want : cap)), dim3(kSlabThreads), smem, st, in, out, outer, inner, Nl, N, off, P);
     return cudaGetLastError();
   };
   return forward ? launch(slab_contract_kernel<K>) : launch(slab_expand_kernel<K>);
