@@ -108,6 +108,30 @@ dtst_status dtst_plan_set_kernel_path(dtst_plan* plan, int path);
  * kernels do, else DTST_PATH_GENERIC. */
 dtst_status dtst_plan_kernel_path(const dtst_plan* plan, int* path);
 
+/*
+ * "Fast path or fail".  Shapes outside the streaming kernels' reach (odd extents, a contiguous extent that is not
+ * a multiple of 32, k outside {4, 8, 12, 16} on a middle dimension, offsets on the contiguous dimension) are
+ * served by a generic kernel that is an order of magnitude slower.  With required != 0 this call returns
+ * DTST_ERR_UNSUPPORTED if ANY stage of the plan's forward- or inverse-type transforms would take that kernel,
+ * and otherwise DTST_OK, after which the compute calls of this plan return DTST_ERR_UNSUPPORTED (launching
+ * nothing) should a later option change (virtual shards, kernel path) make a stage fall back.  required = 0
+ * lifts the requirement.  dtst_plan_kernel_path tells which family serves the grid-side stage.
+ */
+dtst_status dtst_plan_require_fast_path(dtst_plan* plan, int required);
+
+/*
+ * Optional variant of the inverse-type stage (dtst_inverse and the last stage of dtst_backward) for plans on
+ * the fused streaming path with d >= 3: the expansion of dimension d-3 (B^H along it, Eq. 14) runs INSIDE the
+ * kernel that writes the grid, on one extra warp per CTA that stays a few columns ahead of the warps expanding
+ * the last two dimensions, through a ring of `ring_columns` columns that is consumed from L2; the separate
+ * launch for that dimension and its full-size intermediate in HBM disappear.  Same arithmetic, same bits.
+ * Off by default (ring_columns = 0): measured on the largest benchmark shape it shortens an isolated inverse
+ * call by 6 % (ring of 48-64 columns) but a whole step not at all - the single helper warp is the pipeline's
+ * bottleneck under the power cap - and it slows small grids down.  Returns DTST_ERR_UNSUPPORTED (and stays off)
+ * when the plan's shape has no such kernel.  Call it before querying workspace_bytes.
+ */
+dtst_status dtst_plan_set_column_expansion(dtst_plan* plan, int ring_columns);
+
 dtst_status dtst_plan_destroy(dtst_plan* plan);
 
 /* M = number of retained modes; K[d] (host, may be NULL) = entries kept per dim. */

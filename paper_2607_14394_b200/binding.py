@@ -38,7 +38,7 @@ EXPORTED = [
     "dtst_backward", "dtst_plan_status", "dtst_plan_launch_count", "dtst_status_string",
     "dtst_version", "dtst_plan_enable_kernel_timing", "dtst_plan_kernel_timing", "dtst_forward_static",
     "dtst_plan_last_cuda_error", "dtst_spectral_mul_modes", "dtst_backward_spectrum", "dtst_backward_mix_modes",
-    "dtst_backward_input", "dtst_plan_debug_ring_fault",
+    "dtst_backward_input", "dtst_plan_debug_ring_fault", "dtst_plan_set_column_expansion", "dtst_plan_require_fast_path",
 ]
 
 
@@ -81,6 +81,8 @@ def lib() -> ctypes.CDLL:
     L.dtst_backward_spectrum.argtypes = [vp, vp, vp, vp]
     L.dtst_backward_mix_modes.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_int64, ctypes.c_int64, vp]
     L.dtst_backward_input.argtypes = [vp, vp, vp, vp]
+    L.dtst_plan_set_column_expansion.argtypes = [vp, i32]
+    L.dtst_plan_require_fast_path.argtypes = [vp, i32]
     L.dtst_plan_debug_ring_fault.argtypes = [vp, ctypes.c_int64, ctypes.c_uint32]
     L.dtst_plan_status.argtypes = [vp, vp]
     L.dtst_plan_launch_count.argtypes = [vp, i64p]
@@ -165,6 +167,14 @@ def dtst_plan_set_virtual_shards(plan, P) -> None:
 
 def dtst_plan_set_kernel_path(plan, path) -> None:
     _check(lib().dtst_plan_set_kernel_path(plan, int(path)), "dtst_plan_set_kernel_path")
+
+
+def dtst_plan_require_fast_path(plan, required=True) -> None:
+    _check(lib().dtst_plan_require_fast_path(plan, 1 if required else 0), "dtst_plan_require_fast_path")
+
+
+def dtst_plan_set_column_expansion(plan, ring_columns) -> None:
+    _check(lib().dtst_plan_set_column_expansion(plan, int(ring_columns)), "dtst_plan_set_column_expansion")
 
 
 def dtst_plan_kernel_path(plan) -> int:
@@ -301,7 +311,7 @@ class Plan:
     """
 
     def __init__(self, N, kmax, B, C_in, C_out, N_global=None, offset=None, virtual_shards: int = 1,
-                 path: str = "auto", device=None, allocate_workspace: bool = True):
+                 path: str = "auto", device=None, allocate_workspace: bool = True, column_expansion: int = 0):
         self.N = tuple(int(n) for n in N)
         self.kmax = tuple(int(k) for k in kmax)
         self.d = len(self.N)
@@ -322,6 +332,8 @@ class Plan:
         dtst_plan_set_kernel_path(self._h, DTST_PATH_AUTO if path == "auto" else DTST_PATH_GENERIC)
         if virtual_shards != 1:
             dtst_plan_set_virtual_shards(self._h, virtual_shards)
+        if column_expansion:
+            dtst_plan_set_column_expansion(self._h, column_expansion)
         self.M, self.K = dtst_plan_num_modes(self._h, self.d)
         self.workspace = None
         if allocate_workspace:
@@ -486,6 +498,10 @@ class Plan:
         Yhat = self.spectral_mul(Xhat, W, Yhat, stream)
         y = self.inverse(Yhat, y, stream)
         return y, Xhat
+
+    def require_fast_path(self, required: bool = True) -> None:
+        """Raises DtstError(DTST_ERR_UNSUPPORTED) if any stage of this plan would run on the slow generic kernel."""
+        dtst_plan_require_fast_path(self._h, required)
 
     def debug_ring_fault(self, withhold_after_fills: int, poll_limit: int = 1024) -> None:
         """Diagnostic: make the forward plane kernel's bounded waits run out (see dtst_plan_debug_ring_fault)."""

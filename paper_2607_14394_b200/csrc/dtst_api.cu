@@ -131,6 +131,21 @@ bool use_row(const dtst_plan* p) {
   return row_supported((int)p->Ng[a], p->kmax[a]);
 }
 
+// True when no stage of any transform of this plan falls back to the generic one-thread-per-output kernel: the
+// grid-side stage runs on a plane or row kernel and every other dimension on a folded or slab kernel, in both
+// directions.
+bool all_streaming(const dtst_plan* p) {
+  int first;
+  if (use_fused(p)) first = p->d - 3;
+  else if (use_row(p)) first = p->d - 2;
+  else return false;
+  for (int j = first; j >= 0; --j) {
+    if (!(use_slab(p, j) || use_mid(p, j))) return false;          // contraction
+    if (!(use_mid_expand(p, j) || use_slab(p, j))) return false;   // expansion
+  }
+  return true;
+}
+
 DimOp make_op(const dtst_plan* p, int j, bool forward, int Cn) {
   DimOp op;
   std::memset(&op, 0, sizeof(op));
@@ -311,22 +326,51 @@ dtst_status run_inverse_generic(dtst_plan* p, const float2* Yhat, float* y, int 
   return expand_stage(p, p->d - 1, Cn, src, y, scale, herm, st);
 }
 
-// Fused expansion: generic stages for dims 0..d-3 on the small tensor, then the inverse plane kernel
-// expands the last two dimensions and writes the grid once.
+// The dimension in front of the plane can be expanded inside the inverse plane kernel by a helper warp
+// (dtst_plan_set_column_expansion): when the caller asked for it, the dimension is whole on this device with zero
+// offset, and the kernel is built for its shape.
+bool use_colexp(const dtst_plan* p) {
+  if (p->colexp_ring <= 0 || p->d < 3 || !use_fused(p)) return false;
+  const int c = p->d - 3, a = p->d - 1, b = p->d - 2;
+  if (!use_mid_expand(p, c)) return false;
+  return inv_plane_colexp_supported((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], (int)p->Ng[c], p->kmax[c]);
+}
+
+// Fused expansion: stages for the leading dimensions on the small tensor, then the inverse plane kernel
+// expands the last two dimensions and writes the grid once; where the shape allows, the dimension in front of
+// them is expanded inside that kernel too.
 dtst_status run_inverse_fused(dtst_plan* p, const float2* Yhat, float* y, int Cn, float scale, bool herm,
                               cudaStream_t st) {
   const int d = p->d, a = d - 1, b = d - 2;
+  const bool colexp = use_colexp(p);
   const float2* src = Yhat;
-  if (d > 2) {
-    dtst_status s = inverse_stages_complex(p, Yhat, d - 3, Cn, &src, st);
+  const int j_to = colexp ? d - 4 : d - 3;
+  if (j_to >= 0) {
+    dtst_status s = inverse_stages_complex(p, Yhat, j_to, Cn, &src, st);
     if (s != DTST_OK) return s;
   }
   long long planes = (long long)p->B * Cn;
   for (int i = 0; i < b; ++i) planes *= p->Nl[i];
+  const WsLayout L = ws_layout(p);
+  char* ws = static_cast<char*>(p->ws);
   KernelTimer kt(p, DTST_KERNEL_GRID_WRITE, st);
-  if (cuda_failed(p, launch_inv_plane((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], src, y,
-                                      planes * p->Ng[b], scale, herm ? 1 : 0, nullptr, st)))
+  if (colexp) {
+    const int c = d - 3;
+    // the ping-pong buffer the separate expansion of dimension c would have written: its first ring_cols columns
+    float2* ring = reinterpret_cast<float2*>(ws + (((j_to + 1) & 1) ? L.bufB : L.bufA));
+    const long long cols = planes / p->Nl[c];
+    long long ring_cols = p->colexp_ring;
+    if (ring_cols > cols) ring_cols = cols;
+    if (cuda_failed(p, launch_inv_plane_colexp((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], (int)p->Ng[c],
+                                               p->kmax[c], src, ring, (int)ring_cols,
+                                               reinterpret_cast<int*>(ws + L.counters), cols, y, planes * p->Ng[b],
+                                               scale, herm ? 1 : 0, reinterpret_cast<int*>(ws + L.status),
+                                               p->dbg_poll_limit ? p->dbg_poll_limit : kDefaultPollLimit, st)))
+      return DTST_ERR_CUDA;
+  } else if (cuda_failed(p, launch_inv_plane((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], src, y,
+                                             planes * p->Ng[b], scale, herm ? 1 : 0, nullptr, st))) {
     return DTST_ERR_CUDA;
+  }
   ++p->launches;
   return DTST_OK;
 }
@@ -386,6 +430,7 @@ dtst_status check_device(const dtst_plan* p) {
 dtst_status check_ready(const dtst_plan* p) {
   const dtst_status sd = check_device(p);
   if (sd != DTST_OK) return sd;
+  if (p->require_fast && !all_streaming(p)) return DTST_ERR_UNSUPPORTED;
   const WsLayout L = ws_layout(p);
   if (p->ws == nullptr || p->ws_bytes < L.total) return DTST_ERR_WORKSPACE;
   return DTST_OK;
@@ -428,6 +473,14 @@ WsLayout ws_layout(const dtst_plan* p) {
   L.partial = o; o += align256(L.szPartial);
   L.gy = o; o += align256(L.szG);
   L.gx = o; o += align256(L.szG);
+  // flow-control counters of the kernels that expand or contract a leading dimension inside a plane kernel:
+  // two ints per column (a column = one index tuple of batch, channel and the dimensions in front of the last three)
+  {
+    long long cols = (long long)p->B * Cn;
+    for (int i = 0; i + 3 < p->d; ++i) cols *= p->Nl[i];
+    L.szCounters = p->d >= 3 ? (size_t)2 * cols * sizeof(int) : 0;
+  }
+  L.counters = o; o += align256(L.szCounters);
   L.total = o;
   return L;
 }
@@ -459,6 +512,25 @@ dtst_status dtst_plan_set_virtual_shards(dtst_plan* p, int P) {
 dtst_status dtst_plan_set_kernel_path(dtst_plan* p, int path) {
   if (p == nullptr || (path != DTST_PATH_AUTO && path != DTST_PATH_GENERIC)) return DTST_ERR_INVALID_ARG;
   p->path_request = path;
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_require_fast_path(dtst_plan* p, int required) {
+  if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  p->require_fast = 0;
+  if (!required) return DTST_OK;
+  if (!all_streaming(p)) return DTST_ERR_UNSUPPORTED;
+  p->require_fast = 1;
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_set_column_expansion(dtst_plan* p, int ring_columns) {
+  if (p == nullptr || ring_columns < 0) return DTST_ERR_INVALID_ARG;
+  p->colexp_ring = ring_columns;
+  if (ring_columns > 0 && !use_colexp(p)) {
+    p->colexp_ring = 0;
+    return DTST_ERR_UNSUPPORTED;
+  }
   return DTST_OK;
 }
 

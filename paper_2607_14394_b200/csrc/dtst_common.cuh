@@ -143,6 +143,8 @@ struct dtst_plan {
   int last_cuda_error;             // cudaError_t of the last failing runtime call / launch
   unsigned dbg_poll_limit;         // 0 = default budget of the bounded waits
   long long dbg_withhold_after;    // < 0 = off (the default)
+  int require_fast;                // 1: compute calls refuse to run if any stage would take the generic kernel
+  int colexp_ring;                 // > 0: expand the dimension in front of the plane inside the inverse plane kernel
   // optional per-kernel event timing (benchmarks only)
   int timing_cap;
   int timing_n[DTST_KERNEL_KINDS];
@@ -160,8 +162,8 @@ struct RingDebug {
 constexpr uint32_t kDefaultPollLimit = 1u << 24;
 
 struct WsLayout {
-  size_t status, bufA, bufB, partial, gy, gx, total;
-  size_t szA, szB, szPartial, szG;
+  size_t status, bufA, bufB, partial, gy, gx, counters, total;
+  size_t szA, szB, szPartial, szG, szCounters;
 };
 
 bool fused_eligible(const dtst_plan* p);

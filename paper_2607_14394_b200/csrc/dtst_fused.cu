@@ -1,883 +1,17 @@
-// Fused streaming kernels for the grid-side stages of the truncated spectral layer.
-//
-// Forward ("plane") kernel: contracts the last two grid dimensions in one pass.  The real
-// grid is read from HBM exactly once through a TMA-fed shared-memory ring; each consumer
-// warp owns a task of 128 consecutive rows (one or two [N2 x N3] planes), contracts the
-// contiguous dimension with one thread per row (folded FFMA with immediate coefficients),
-// then the next dimension on the tensor cores (TF32 hi/lo compensated warp MMAs), and writes
-// only the [2*k2 x k3] complex result of each plane.
-//
-// Both contractions use the symmetries of the DFT basis (Eq. 18 with zero offset): with the
-// half-sample phase factored out,
-//     sum_n x[n] e^{-i phi n} = e^{+i phi/2} sum_n x[n] e^{-i phi (n + 1/2)},
-// the cos/sin factors are even/odd about the centre of the row and again (up to (-1)^f)
-// about the centre of each half, so four inputs (n, N/2-1-n, N/2+n, N-1-n) are folded with
-// 8 additions and then need one multiply-add per retained frequency and parity class instead
-// of four.  Frequencies +g and -g of a two-sided dimension share their cos and sin sums.
-// This cuts the multiply count roughly fourfold and keeps the arithmetic in exact fp32 FMAs,
-// which is what lets an HBM-bound kernel afford a dense contraction with only 8..16 output
-// columns (far too narrow for the tensor cores to help: the MMA would be bound by reading
-// its 128 x 8 A tile from shared memory, which costs as much as the FMAs done here).
+// Dispatcher of the fused streaming kernels: which plane shapes exist, tensor-map construction, and the run-time
+// selection of the instantiation for a plan's shape.  The kernels themselves are templates in dtst_plane.cuh,
+// instantiated in dtst_plane_inst_*.cu.
 #include <cuda.h>
 
-#include "dtst_fused.cuh"
-#include "dtst_mma.cuh"
-#include "dtst_sm100.cuh"
+#include "dtst_plane.cuh"
 
 namespace dtst {
 
-using namespace sm100;
-
-bool make_rows_map(CUtensorMap* map, const void* base, long long rows, int n3, int box_rows);
+namespace plane {
+DTST_PLANE_SHAPES(DTST_PLANE_EXTERN)
+}
 
 namespace {
-
-constexpr int kTaskRows = 128;       // rows of the contiguous dimension per warp task
-constexpr int kStageBytes = 16384;   // one ring slot
-constexpr int kSmemLimit = 232448;   // 227 KB opt-in limit per CTA
-
-// Stage-1 coefficients cos/sin(2 pi f (j + 1/2) / N3), j < N3/4, as COMPILE-TIME constants: the row code is fully
-// unrolled over (j, f), so every FMA carries its coefficient as a 32-bit immediate.  No table in HBM, shared or
-// constant memory, no load instruction, no register: a shared-memory operand would cost LDS bandwidth this kernel
-// does not have, and a constant-bank table costs one uniform load per four coefficients (measured: 9 % of the
-// forward kernel's instructions, 22 % of the inverse kernel's).
-namespace ct {
-constexpr double kPi = 3.14159265358979323846264338327950288;
-// Taylor series on |x| <= pi/4 (terms to x^27: below 1e-19)
-constexpr double sin_small(double x) {
-  const double x2 = x * x;
-  double term = x, sum = x;
-  for (int k = 1; k <= 13; ++k) {
-    term *= -x2 / (double)((2 * k) * (2 * k + 1));
-    sum += term;
-  }
-  return sum;
-}
-constexpr double cos_small(double x) {
-  const double x2 = x * x;
-  double term = 1.0, sum = 1.0;
-  for (int k = 1; k <= 13; ++k) {
-    term *= -x2 / (double)((2 * k - 1) * (2 * k));
-    sum += term;
-  }
-  return sum;
-}
-// cos(pi num / den), sin(pi num / den): the argument is reduced exactly in integers to the first octant
-constexpr double cospi_ratio(long long num, long long den) {
-  num %= 2 * den;
-  if (num < 0) num += 2 * den;
-  if (num > den) num = 2 * den - num;          // cos(2 pi - a) = cos a
-  double sign = 1.0;
-  if (2 * num > den) {                         // cos(pi - a) = -cos a
-    num = den - num;
-    sign = -1.0;
-  }
-  if (4 * num <= den) return sign * cos_small(kPi * (double)num / (double)den);
-  return sign * sin_small(kPi * (double)(den - 2 * num) / (double)(2 * den));   // cos a = sin(pi/2 - a)
-}
-constexpr double sinpi_ratio(long long num, long long den) {
-  num %= 2 * den;
-  if (num < 0) num += 2 * den;
-  double sign = 1.0;
-  if (num > den) {                             // sin(2 pi - a) = -sin a
-    num = 2 * den - num;
-    sign = -1.0;
-  }
-  if (2 * num > den) num = den - num;          // sin(pi - a) = sin a
-  if (4 * num <= den) return sign * sin_small(kPi * (double)num / (double)den);
-  return sign * cos_small(kPi * (double)(den - 2 * num) / (double)(2 * den));   // sin a = cos(pi/2 - a)
-}
-// phase (2j+1) f / (2 N3) turns = pi (2j+1) f / N3
-template <int N3, int J, int F>
-struct Coef {
-  static constexpr float cs = (float)cospi_ratio((long long)(2 * J + 1) * F, N3);
-  static constexpr float sn = (float)sinpi_ratio((long long)(2 * J + 1) * F, N3);
-};
-}  // namespace ct
-
-template <int N3, int K3, int N2, int K2>
-struct PlaneCfg {
-  static constexpr int ROWS_PER_STAGE = kStageBytes / (N3 * 4);
-  static constexpr int SPT = kTaskRows / ROWS_PER_STAGE;      // ring slots per task
-  static constexpr int BOXES = N3 / 32;                       // 128-byte column panels per row
-  static constexpr int G = kTaskRows / N2;                    // planes per task
-  static constexpr int QUADS = N2 / 4;                        // row quadruples per plane
-  static constexpr int NC = 2 * K3;                           // real columns after stage 1 (C | S)
-  static constexpr int LPP = 2 * K2;                          // output rows (modes) per plane
-  static constexpr int NKS = QUADS / 8;                       // MMA k-steps over the quadruples
-  static constexpr int MT = G * NC / 16;                      // MMA m-tiles over (plane, column)
-  static constexpr int MT2 = 2;                               // inverse: MMA m-tiles over the 32 quadruples
-  static constexpr int GT = K2 / 2;                           // frequencies per parity class
-  static constexpr int NS = 4 * NC + 8;                       // floats per combo row: 4 classes x NC, +8 pad
-  static constexpr int ABS = NC + 1;                          // floats between A/B entries (odd: scalar accesses)
-  static constexpr int ABP = (2 * K2 + 1) * ABS;
-  // forward kernel: one parity class at a time, row stride NSC = 8 mod 16 words (conflict-free fragment loads)
-  static constexpr int NSC = (NC % 16 == 8) ? NC : NC + 8;
-  // per-warp buffer (class combos, later the A/B entries), a multiple of 128 bytes so that every warp's
-  // region stays 16-byte aligned for the vector stores
-  static constexpr int COMBO_FLOATS = (((32 * NSC > G * ABP ? 32 * NSC : G * ABP) + 31) / 32) * 32;
-  static constexpr int BTAB_FLOAT4 = 5 * NKS * 32;            // stage-2 basis fragments, CTA-shared
-  static_assert(N3 % 32 == 0 && (N3 == 32 || N3 == 64), "N3");
-  static_assert(kTaskRows % N2 == 0 && G * QUADS == 32, "one lane per row quadruple");
-  static_assert(G * LPP <= 32 && (G * NC) % 16 == 0, "stage-2 mapping");
-  static_assert(K3 % 2 == 0 && NC % 8 == 0 && K2 % 2 == 0 && GT <= 8 && QUADS % 8 == 0, "shape");
-  static_assert(NS % 32 == 8, "combo row stride must be 8 mod 32 words for conflict-free fragment loads");
-  static_assert(SPT == 1 || SPT == 2, "SPT");
-};
-
-struct SmemPlan {
-  int stages;
-  size_t ring, combos, rot, bars, total;
-};
-
-template <typename Cfg, int K2, int K3, int W>
-SmemPlan smem_plan() {
-  SmemPlan s;
-  const size_t combos = (size_t)W * Cfg::COMBO_FLOATS * 4 + (size_t)Cfg::BTAB_FLOAT4 * 16;
-  const size_t rot = (size_t)2 * K2 * K3 * 8;
-  const size_t fixed = 1024 /*alignment slack*/ + combos + rot + 512 /*barriers*/;
-  s.stages = (int)((kSmemLimit - fixed) / kStageBytes);
-  if (s.stages > 12) s.stages = 12;
-  s.ring = 0;
-  s.combos = (size_t)s.stages * kStageBytes;
-  s.rot = s.combos + combos;
-  s.bars = s.rot + rot;
-  s.total = s.bars + 512 + 1024;
-  return s;
-}
-
-// 16-byte shared-memory access by 32-bit shared-space address (+ immediate byte offset).  Volatile: a ring
-// slot is refilled by the TMA engine between two reads of the same address, which the compiler cannot see.
-template <int IMM>
-__device__ __forceinline__ float4 lds128_s(uint32_t addr) {
-  float4 v;
-  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4+%5];"
-               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-               : "r"(addr), "n"(IMM));
-  return v;
-}
-template <int IMM>
-__device__ __forceinline__ void sts128_s(uint32_t addr, float a, float b, float c, float d) {
-  asm volatile("st.shared.v4.f32 [%0+%1], {%2,%3,%4,%5};" ::"r"(addr), "n"(IMM), "f"(a), "f"(b), "f"(c), "f"(d)
-               : "memory");
-}
-
-// fp32 -> (hi, lo) TF32 pair for the error-compensated product hi*hi + lo*hi + hi*lo: the truncating split
-// (two instructions) for operands split in the inner loop, the rounding one for the basis tables built once
-__device__ __forceinline__ void split_tf32(float v, uint32_t& hi, uint32_t& lo) { split_tf32_trunc(v, hi, lo); }
-
-// D += A(16x8, row) * B(8x8, col), TF32 inputs, fp32 accumulate
-__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// Forward row code, one quadruple j: o[f] += folded input * coefficient(j, f), f = F .. K3-1 (compile-time recursion
-// so that j and f are constant expressions and the coefficients become immediates).
-template <int N3, int K3, int J, int F>
-__device__ __forceinline__ void s1_freqs(float uu, float ud, float vs, float vd, float (&o)[2 * K3]) {
-  if constexpr (F < K3) {
-    constexpr float cs = ct::Coef<N3, J, F>::cs, sn = ct::Coef<N3, J, F>::sn;
-    if constexpr ((F & 1) == 0) {
-      o[F] = (J == 0) ? uu * cs : fmaf(uu, cs, o[F]);
-      if constexpr (F > 0) o[K3 + F] = (J == 0) ? vd * sn : fmaf(vd, sn, o[K3 + F]);
-    } else {
-      o[F] = (J == 0) ? ud * cs : fmaf(ud, cs, o[F]);
-      o[K3 + F] = (J == 0) ? vs * sn : fmaf(vs, sn, o[K3 + F]);
-    }
-    s1_freqs<N3, K3, J, F + 1>(uu, ud, vs, vd, o);
-  }
-}
-
-// chunks C, CH/2-1-C, CH/2+C, CH-1-C of the row: four quadruples j = 4C .. 4C+3
-template <int N3, int K3, int BOXR, int C>
-__device__ __forceinline__ void s1_chunks(uint32_t rx, float (&o)[2 * K3]) {
-  constexpr int CH = N3 / 4;
-  if constexpr (C < CH / 4) {
-    constexpr int P = BOXR * 128;
-    constexpr int c0 = C, c1 = CH / 2 - 1 - C, c2 = CH / 2 + C, c3 = CH - 1 - C;
-    // (the panel offset is an immediate, the XOR constant depends on the chunk only)
-    const float4 A = lds128_s<(c0 / 8) * P>(rx ^ (uint32_t)((c0 % 8) << 4));
-    const float4 Bq = lds128_s<(c1 / 8) * P>(rx ^ (uint32_t)((c1 % 8) << 4));
-    const float4 Cq = lds128_s<(c2 / 8) * P>(rx ^ (uint32_t)((c2 % 8) << 4));
-    const float4 D = lds128_s<(c3 / 8) * P>(rx ^ (uint32_t)((c3 % 8) << 4));
-#define DTST_QUAD(E, av, bv, cv, dv)                                               \
-    {                                                                              \
-      const float u = (av) + (dv), v = (av) - (dv);                                \
-      const float up = (bv) + (cv), vp = (bv) - (cv);                              \
-      s1_freqs<N3, K3, 4 * C + (E), 0>(u + up, u - up, v + vp, v - vp, o);         \
-    }
-    DTST_QUAD(0, A.x, Bq.w, Cq.x, D.w)
-    DTST_QUAD(1, A.y, Bq.z, Cq.y, D.z)
-    DTST_QUAD(2, A.z, Bq.y, Cq.z, D.y)
-    DTST_QUAD(3, A.w, Bq.x, Cq.w, D.x)
-#undef DTST_QUAD
-    s1_chunks<N3, K3, BOXR, C + 1>(rx, o);
-  }
-}
-
-// One row of N3 reals -> C_f = sum u cos, S_f = sum v sin for f < K3 (half-sample phase deferred).
-// `stage` is the 32-bit shared address of the slot (1024-byte aligned), BOXR its rows per 128-byte panel.
-template <int N3, int K3, int BOXR>
-__device__ __forceinline__ void stage1_row(uint32_t stage, int row, float (&o)[2 * K3]) {
-  o[K3] = 0.f;   // the sine sum of f = 0 has no terms
-  // chunk c of this row sits at row*128 + ((c ^ (row & 7)) << 4) (+ one panel for c >= 8); the row base has
-  // zeros in bits 4..6, so the swizzle is a single XOR of a precomputed base with a constant
-  const uint32_t rx = stage + (uint32_t)row * 128u + (((uint32_t)row & 7u) << 4);
-  s1_chunks<N3, K3, BOXR, 0>(rx, o);
-}
-
-// Consumer side of the ring: wait until fill number q (0-based) of `slot` has landed.
-// Every lane of the warp calls it; the lanes poll independently but leave with ONE verdict (a lane whose barrier
-// completed just as another warp raised the abort flag must not go on alone into the warp-synchronous MMA code).
-__device__ __forceinline__ bool wait_fill(volatile uint32_t* fill_seq, uint64_t* full, int slot, uint32_t q,
-                                          volatile int* abort_flag, uint32_t limit) {
-  bool ok = true;
-  for (uint32_t it = 0; fill_seq[slot] < q + 1u; ++it) {
-    if ((it & 63u) == 63u) {
-      if (*abort_flag) {
-        ok = false;
-        break;
-      }
-      __nanosleep(64);
-    }
-    if (it > limit) {
-      *abort_flag = 1;
-      ok = false;
-      break;
-    }
-  }
-  if (ok) ok = mbar_wait_bounded(&full[slot], q & 1u, abort_flag, limit);
-  return __all_sync(0xffffffffu, ok) != 0;
-}
-
-template <int N3, int K3, int N2, int K2, int W>
-__global__ void __launch_bounds__((W + 1) * 32, 1)
-fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict__ out, long long num_tasks, float scale, int herm, int stages,
-                 int* __restrict__ status, uint32_t poll_limit, long long withhold_after) {
-  using Cfg = PlaneCfg<N3, K3, N2, K2>;
-  constexpr int NC = Cfg::NC, QUADS = Cfg::QUADS, G = Cfg::G, LPP = Cfg::LPP;
-  constexpr int SPT = Cfg::SPT, RPS = Cfg::ROWS_PER_STAGE;
-  pdl_trigger();
-
-  extern __shared__ unsigned char smem_raw[];
-  // 1024-byte alignment for the TMA swizzle, by pointer arithmetic on the shared array itself (an integer
-  // round trip would make the compiler lose the address space and emit generic loads and stores)
-  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-  unsigned char* ring = smem;
-  const uint32_t ring_s = smem_u32(ring);
-  float4* btab = reinterpret_cast<float4*>(smem + (size_t)stages * kStageBytes);
-  float* combos_all = reinterpret_cast<float*>(btab + Cfg::BTAB_FLOAT4);
-  float2* rot = reinterpret_cast<float2*>(combos_all + (size_t)W * Cfg::COMBO_FLOATS);
-  uint64_t* full = reinterpret_cast<uint64_t*>(rot + 2 * K2 * K3);
-  uint64_t* empty = full + 16;
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(empty + 16);
-  // fill_seq[slot] = number of fills the producer has armed for that slot.  A parity wait can only
-  // tell "this phase" from "the previous one", so a consumer that is a whole lap of the ring ahead
-  // must first see its fill armed (which implies every earlier fill of the slot has landed).
-  volatile uint32_t* fill_seq = reinterpret_cast<volatile uint32_t*>(empty + 16) + 4;
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < stages; ++s) {
-      mbar_init(&full[s], 1);
-      mbar_init(&empty[s], 1);
-      fill_seq[s] = 0;
-    }
-    *abort_flag = 0;
-    fence_barrier_init();
-    prefetch_tensormap(&in_map);
-  }
-  // Stage-2 basis as MMA B fragments (k = quadruple n, n = frequency slot of the parity class), TF32 hi/lo,
-  // generated once per CTA: entry [cls][ks][lane] = (b0 hi, b1 hi, b0 lo, b1 lo).  Classes: 0 = A even (pp,
-  // cos), 1 = A odd (pd, cos), 2 = B odd (ms, sin), 3 = B even (md, sin); 4 = the unpaired A_{K2} (cos, shares
-  // the pp operand), in column 0 only.
-  for (int e = threadIdx.x; e < Cfg::BTAB_FLOAT4; e += blockDim.x) {
-    const int l = e & 31, ks = (e >> 5) % Cfg::NKS, cls = (e >> 5) / Cfg::NKS;
-    const int lg = l >> 2, lt = l & 3;
-    uint32_t hi[2], lo[2];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int n = 8 * ks + lt + 4 * h;
-      int g = 0;
-      bool valid = lg < Cfg::GT;
-      if (cls == 0) g = 2 * lg;
-      else if (cls == 1 || cls == 2) g = 2 * lg + 1;
-      else if (cls == 3) g = 2 * lg + 2;
-      else { g = K2; valid = (lg == 0); }
-      double sn, cs;
-      sincospi((double)(((long long)g * (2 * n + 1)) % (2 * N2)) / (double)N2, &sn, &cs);
-      const float v = valid ? ((cls == 2 || cls == 3) ? (float)sn : (float)cs) : 0.f;
-      split_tf32_rna(v, hi[h], lo[h]);
-    }
-    btab[e] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(lo[0]), __uint_as_float(lo[1]));
-  }
-  // rotation table: the deferred half-sample phases of both dimensions, the scale and the
-  // Hermitian weight, one complex factor per (mode position r, last-dim frequency f)
-  for (int e = threadIdx.x; e < 2 * K2 * K3; e += blockDim.x) {
-    const int r = e / K3, f = e % K3;
-    const int sg = (r < K2) ? r : -(2 * K2 - r);
-    // angle / pi = sg / N2 + f / N3, reduced as an exact rational
-    const long long num = (long long)sg * N3 + (long long)f * N2;
-    double sn, cs;
-    sincospi((double)num / (double)((long long)N2 * N3), &sn, &cs);
-    const float w = scale * (herm ? herm_weight(f, N3) : 1.0f);
-    rot[f * (2 * K2) + r] = make_float2((float)cs * w, (float)sn * w);   // [f][r]: lanes (r) read conflict-free
-  }
-  __syncthreads();
-  pdl_wait();   // everything above is independent of the preceding kernel
-
-  const long long first = blockIdx.x;
-  const long long n_local = first < num_tasks ? (num_tasks - first + gridDim.x - 1) / gridDim.x : 0;
-
-  if (warp == 0) {
-    // ---------------- producer: one thread feeds the ring in task order ----------------
-    if (lane == 0) {
-      long long k = 0;
-      for (long long tl = 0; tl < n_local; ++tl) {
-        const long long task = first + tl * gridDim.x;
-        for (int s = 0; s < SPT; ++s, ++k) {
-          // diagnostic (dtst_plan_debug_ring_fault): stop feeding the ring after `withhold_after` fills, so
-          // that the consumers' bounded waits run out
-          if (withhold_after >= 0 && k >= withhold_after) goto producer_done;
-          const int slot = (int)(k % stages);
-          const uint32_t ph = (uint32_t)((k / stages) & 1);
-          if (!mbar_wait_bounded(&empty[slot], ph ^ 1u, abort_flag, poll_limit)) goto producer_done;
-          fill_seq[slot] = (uint32_t)(k / stages) + 1u;
-          mbar_arrive_expect_tx(&full[slot], (uint32_t)kStageBytes);
-#pragma unroll
-          for (int h = 0; h < Cfg::BOXES; ++h)
-            tma_load_2d(ring + (size_t)slot * kStageBytes + (size_t)h * RPS * 128, &in_map, h * 32,
-                        (int)(task * kTaskRows + (long long)s * RPS), &full[slot]);
-        }
-      }
-    }
-  producer_done:
-    __syncwarp();
-  } else {
-    // ---------------- consumers: one warp per task ----------------
-    const int w = warp - 1;
-    float* combo = combos_all + (size_t)w * Cfg::COMBO_FLOATS;
-
-    // stage-1 role: lane = (plane in task, row quadruple)
-    const int pl1 = lane / QUADS, n1 = lane % QUADS;
-    // epilogue role: lane = (plane, mode position r)
-    const bool act2 = lane < G * LPP;
-    const int pl2 = act2 ? lane / LPP : 0;
-    const int l2 = lane % LPP;
-    // MMA fragment coordinates
-    const int g8 = lane >> 2, t4 = lane & 3;
-
-    for (long long tl = w; tl < n_local; tl += W) {
-      const long long task = first + tl * gridDim.x;
-      const long long k0 = tl * SPT;
-      const int slot0 = (int)(k0 % stages), slot1 = (int)((k0 + SPT - 1) % stages);
-      constexpr bool kSplit = (SPT == 2 && N2 == 128);   // rows a, b in the first slot, c, d in the second
-
-      // ---- stage 1: the four rows of this lane's quadruple, accumulated straight into the four
-      // parity combos  pp = a+d+b+c, pd = a+d-b-c, ms = a-d+b-c, md = a-d-b+c  (one copy of the row code)
-      float cpp[NC], cpd[NC], cms[NC], cmd[NC];
-#pragma unroll
-      for (int c = 0; c < NC; ++c) cpp[c] = cpd[c] = cms[c] = cmd[c] = 0.f;
-      if constexpr (!kSplit) {
-        if (!wait_fill(fill_seq, full, slot0, (uint32_t)(k0 / stages), abort_flag, poll_limit)) break;
-        if (SPT == 2 && !wait_fill(fill_seq, full, slot1, (uint32_t)((k0 + 1) / stages), abort_flag, poll_limit)) break;
-      }
-      bool alive = true;
-#pragma unroll 1
-      for (int r4 = 0; r4 < 4; ++r4) {
-        if constexpr (kSplit) {
-          if (r4 == 0) alive = wait_fill(fill_seq, full, slot0, (uint32_t)(k0 / stages), abort_flag, poll_limit);
-          if (r4 == 2) {
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&empty[slot0]);
-            alive = wait_fill(fill_seq, full, slot1, (uint32_t)((k0 + 1) / stages), abort_flag, poll_limit);
-          }
-          if (!alive) break;
-        }
-        // order a, b, c, d = rows n, N2/2-1-n, N2/2+n, N2-1-n of the plane
-        const int rowq = (r4 == 0) ? n1 : (r4 == 1) ? (N2 / 2 - 1 - n1) : (r4 == 2) ? (N2 / 2 + n1) : (N2 - 1 - n1);
-        const float s1 = (r4 == 0 || r4 == 3) ? 1.f : -1.f;
-        const float s2 = (r4 <= 1) ? 1.f : -1.f;
-        const float s3 = (r4 == 0 || r4 == 2) ? 1.f : -1.f;
-        const int trow = pl1 * N2 + rowq;
-        const int sl = (trow / RPS) ? slot1 : slot0;
-        const uint32_t st = ring_s + (uint32_t)sl * kStageBytes;
-        float o[NC];
-        stage1_row<N3, K3, RPS>(st, trow % RPS, o);
-#pragma unroll
-        for (int c = 0; c < NC; ++c) {
-          cpp[c] += o[c];
-          cpd[c] = fmaf(s1, o[c], cpd[c]);
-          cms[c] = fmaf(s2, o[c], cms[c]);
-          cmd[c] = fmaf(s3, o[c], cmd[c]);
-        }
-      }
-      if (!alive) break;
-      __syncwarp();
-      if (lane == 0) {
-        if constexpr (kSplit) {
-          mbar_arrive(&empty[slot1]);
-        } else {
-          mbar_arrive(&empty[slot0]);
-          if (SPT == 2) mbar_arrive(&empty[slot1]);
-        }
-      }
-
-      // ---- stage 2 on the tensor cores (legacy warp-level MMA, TF32 with hi/lo error compensation), one
-      // parity class at a time through a small per-warp buffer:
-      //   out[(plane, column)][frequency slot] = sum_n combo_cls[n][(plane, column)] * basis_cls[n][slot]
-      // The class's combos are published as rows (plane, n) of NC floats, 16-byte chunks swapped pairwise on
-      // odd groups of four rows so that both the stores and the fragment loads are bank-conflict free.
-      float acc[5][Cfg::MT][4];
-#pragma unroll
-      for (int cls = 0; cls < 5; ++cls)
-#pragma unroll
-        for (int mt = 0; mt < Cfg::MT; ++mt)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) acc[cls][mt][e] = 0.f;
-#pragma unroll
-      for (int cls = 0; cls < 4; ++cls) {
-        __syncwarp();   // the previous class's fragment loads (or the previous task's epilogue reads) are done
-        {
-          float* dst = combo + (size_t)lane * Cfg::NSC;
-          const int sw = ((n1 >> 2) & 1);
-#pragma unroll
-          for (int c4 = 0; c4 < NC / 4; ++c4) {
-            const int cc = 4 * (c4 ^ sw);
-            const float* srcv = (cls == 0) ? cpp : (cls == 1) ? cpd : (cls == 2) ? cms : cmd;
-            *reinterpret_cast<float4*>(dst + cc) =
-                make_float4(srcv[4 * c4], srcv[4 * c4 + 1], srcv[4 * c4 + 2], srcv[4 * c4 + 3]);
-          }
-        }
-        __syncwarp();
-#pragma unroll
-        for (int ks = 0; ks < Cfg::NKS; ++ks) {
-          const float4 bf = btab[(cls * Cfg::NKS + ks) * 32 + lane];
-          const uint32_t bh0 = __float_as_uint(bf.x), bh1 = __float_as_uint(bf.y);
-          const uint32_t bl0 = __float_as_uint(bf.z), bl1 = __float_as_uint(bf.w);
-          float4 bx = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (cls == 0) bx = btab[(4 * Cfg::NKS + ks) * 32 + lane];
-#pragma unroll
-          for (int mt = 0; mt < Cfg::MT; ++mt) {
-            uint32_t ahi[4], alo[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int m = 16 * mt + g8 + 8 * (e & 1);
-              const int n = 8 * ks + t4 + 4 * (e >> 1);
-              const int pl = m / NC, c = m % NC;
-              const float v = combo[(size_t)(pl * QUADS + n) * Cfg::NSC + (c ^ ((e >> 1) << 2))];
-              split_tf32(v, ahi[e], alo[e]);
-            }
-            mma_tf32(acc[cls][mt], ahi, bh0, bh1);
-            mma_tf32(acc[cls][mt], alo, bh0, bh1);
-            mma_tf32(acc[cls][mt], ahi, bl0, bl1);
-            if (cls == 0) {   // the pp operand also feeds the unpaired A_{K2}
-              mma_tf32(acc[4][mt], ahi, __float_as_uint(bx.x), __float_as_uint(bx.y));
-              mma_tf32(acc[4][mt], alo, __float_as_uint(bx.x), __float_as_uint(bx.y));
-              mma_tf32(acc[4][mt], ahi, __float_as_uint(bx.z), __float_as_uint(bx.w));
-            }
-          }
-        }
-      }
-      __syncwarp();
-
-      // A/B sums -> shared: entry g for A_g (g <= K2), entry K2+g for B_g (g >= 1)
-#pragma unroll
-      for (int cls = 0; cls < 5; ++cls)
-#pragma unroll
-        for (int mt = 0; mt < Cfg::MT; ++mt)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int m = 16 * mt + g8 + 8 * (e >> 1);
-            const int gi = 2 * t4 + (e & 1);
-            const int pl = m / NC, c = m % NC;
-            int entry;
-            bool valid = gi < Cfg::GT;
-            if (cls == 0) entry = 2 * gi;
-            else if (cls == 1) entry = 2 * gi + 1;
-            else if (cls == 2) entry = K2 + 2 * gi + 1;
-            else if (cls == 3) entry = K2 + 2 * gi + 2;
-            else { entry = K2; valid = (gi == 0); }
-            if (valid) combo[pl * Cfg::ABP + entry * Cfg::ABS + c] = acc[cls][mt][e];
-          }
-      __syncwarp();
-
-      // epilogue: Z_{+g} = rho (A - iB), Z_{-g} = rho (A + iB) with A = AC - i AS, B = BC - i BS
-      if (act2) {
-        const int r = l2;
-        const bool pos = r < K2;
-        const int g = pos ? r : 2 * K2 - r;
-        const float* A = combo + pl2 * Cfg::ABP + g * Cfg::ABS;
-        const float* Bp = combo + pl2 * Cfg::ABP + (K2 + g) * Cfg::ABS;
-        float2* dst = out + ((task * G + pl2) * (2 * K2) + r) * K3;
-        const float2* rr = rot + r;
-#pragma unroll
-        for (int f2 = 0; f2 < K3 / 2; ++f2) {
-          float res[4];
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int f = 2 * f2 + e;
-            const float AC = A[f], AS = A[K3 + f];
-            const float BC = g > 0 ? Bp[f] : 0.f, BS = g > 0 ? Bp[K3 + f] : 0.f;
-            const float wr = pos ? AC - BS : AC + BS;
-            const float wi = pos ? -(AS + BC) : BC - AS;
-            const float2 ro = rr[f * (2 * K2)];
-            res[2 * e] = ro.x * wr - ro.y * wi;
-            res[2 * e + 1] = ro.x * wi + ro.y * wr;
-          }
-          *reinterpret_cast<float4*>(dst + 2 * f2) = make_float4(res[0], res[1], res[2], res[3]);
-        }
-      }
-      __syncwarp();   // the next task's combos overwrite the A/B entries read above
-    }
-  }
-
-  __syncthreads();
-  if (threadIdx.x == 0 && *abort_flag) {
-    // the pipeline gave up: loads that were armed but never consumed may still be in flight, and this CTA's
-    // shared memory must not be handed to the next one while the TMA engine writes to it
-    for (int s = 0; s < stages; ++s)
-      if (fill_seq[s] > 0) mbar_wait_plain(&full[s], (fill_seq[s] - 1u) & 1u, 1u << 16);
-    atomicExch(status, 1);
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Inverse plane kernel: the transpose of the forward one.  in[planes][2*K2][K3] complex ->
-// real rows [planes*N2][N3].  Each warp owns a task of 128 output rows: it pre-rotates the plane's
-// modes, forms alpha_g = V'_{+g} + V'_{-g}, beta_g = i (V'_{+g} - V'_{-g}), expands them to the
-// four rows of each row quadruple (one lane per quadruple), expands every row to N3 reals with
-// the same folded basis, stages the rows in shared memory (TMA swizzle) and stores them with TMA.
-// Inverse row code, one quadruple j: the four class sums over f = F .. K3-1 with immediate coefficients.
-template <int N3, int K3, int J, int F>
-__device__ __forceinline__ void e1_freqs(const float (&z)[2 * K3], float& Ea, float& Oa, float& Eb, float& Ob) {
-  if constexpr (F < K3) {
-    constexpr float cs = ct::Coef<N3, J, F>::cs, sn = ct::Coef<N3, J, F>::sn;
-    if constexpr ((F & 1) == 0) {
-      Ea = (F == 0) ? z[F] * cs : fmaf(z[F], cs, Ea);
-      if constexpr (F > 0) Eb = (F == 2) ? z[K3 + F] * sn : fmaf(z[K3 + F], sn, Eb);
-    } else {
-      Oa = (F == 1) ? z[F] * cs : fmaf(z[F], cs, Oa);
-      Ob = (F == 1) ? z[K3 + F] * sn : fmaf(z[K3 + F], sn, Ob);
-    }
-    e1_freqs<N3, K3, J, F + 1>(z, Ea, Oa, Eb, Ob);
-  }
-}
-
-template <int N3, int K3, int J>
-__device__ __forceinline__ void e1_quad(const float (&z)[2 * K3], float& ya, float& yb, float& yc, float& yd) {
-  float Ea = 0.f, Oa = 0.f, Eb = 0.f, Ob = 0.f;
-  e1_freqs<N3, K3, J, 0>(z, Ea, Oa, Eb, Ob);
-  const float sa = Ea + Oa, da = Ea - Oa, sb = Eb + Ob, db = Eb - Ob;
-  ya = sa - sb;   // y[j]
-  yd = sa + sb;   // y[N3-1-j]
-  yb = da + db;   // y[N3/2-1-j]
-  yc = da - db;   // y[N3/2+j]
-}
-
-template <int N3, int K3, int BOXR, int C>
-__device__ __forceinline__ void e1_chunks(uint32_t rx, const float (&z)[2 * K3]) {
-  constexpr int CH = N3 / 4;
-  if constexpr (C < CH / 4) {
-    constexpr int P = BOXR * 128;
-    constexpr int c0 = C, c1 = CH / 2 - 1 - C, c2 = CH / 2 + C, c3 = CH - 1 - C;
-    float a[4], b[4], cc[4], d[4];
-    e1_quad<N3, K3, 4 * C + 0>(z, a[0], b[0], cc[0], d[0]);
-    e1_quad<N3, K3, 4 * C + 1>(z, a[1], b[1], cc[1], d[1]);
-    e1_quad<N3, K3, 4 * C + 2>(z, a[2], b[2], cc[2], d[2]);
-    e1_quad<N3, K3, 4 * C + 3>(z, a[3], b[3], cc[3], d[3]);
-    sts128_s<(c0 / 8) * P>(rx ^ (uint32_t)((c0 % 8) << 4), a[0], a[1], a[2], a[3]);
-    sts128_s<(c1 / 8) * P>(rx ^ (uint32_t)((c1 % 8) << 4), b[3], b[2], b[1], b[0]);
-    sts128_s<(c2 / 8) * P>(rx ^ (uint32_t)((c2 % 8) << 4), cc[0], cc[1], cc[2], cc[3]);
-    sts128_s<(c3 / 8) * P>(rx ^ (uint32_t)((c3 % 8) << 4), d[3], d[2], d[1], d[0]);
-    e1_chunks<N3, K3, BOXR, C + 1>(rx, z);
-  }
-}
-
-template <int N3, int K3, int BOXR>
-__device__ __forceinline__ void expand_row(uint32_t stage, int row, const float (&z)[2 * K3]) {
-  // same single-XOR swizzled addressing as the forward kernel's row loads
-  const uint32_t rx = stage + (uint32_t)row * 128u + (((uint32_t)row & 7u) << 4);
-  e1_chunks<N3, K3, BOXR, 0>(rx, z);
-}
-
-template <int N3, int K3, int N2, int K2>
-struct InvCfg {
-  using P = PlaneCfg<N3, K3, N2, K2>;
-  static constexpr int ABS = P::NC + 4;                     // floats between entries
-  static constexpr int ENTRIES = 2 * K2 + 2;                // alpha_0..alpha_K2, beta_0..beta_K2 (beta_0 unused)
-  static constexpr int ABP = ENTRIES * ABS + 4;             // floats between planes
-  static constexpr int AB_FLOATS = ((P::G * ABP + 3) / 4) * 4;
-  static constexpr int COMBO_FLOATS = 32 * P::NS;           // expanded combos, one row per quadruple
-  static constexpr int NT = P::NC / 8;                      // MMA n-tiles over the columns
-  static constexpr int STAGING_BYTES = kTaskRows * N3 * 4;  // 128 output rows
-  // With two staging blocks that are stored one after the other (rows a, b then rows c, d) the small
-  // alpha/beta and combo buffers live inside the first block: its store is issued half a task before the
-  // next task needs the space, so one bounded wait on that store group is all the aliasing costs.
-  static constexpr bool ALIAS = (P::SPT == 2 && N2 == 128) && ((AB_FLOATS + COMBO_FLOATS) * 4 <= kStageBytes);
-  static constexpr int WARP_BYTES =
-      ALIAS ? STAGING_BYTES : STAGING_BYTES + (((AB_FLOATS + COMBO_FLOATS) * 4 + 1023) / 1024) * 1024;
-};
-
-template <int N3, int K3, int N2, int K2, int W>
-__global__ void __launch_bounds__(W * 32, 1)
-inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __restrict__ in, long long num_tasks, float scale, int herm) {
-  using Cfg = PlaneCfg<N3, K3, N2, K2>;
-  using IC = InvCfg<N3, K3, N2, K2>;
-  constexpr int NC = Cfg::NC, QUADS = Cfg::QUADS, G = Cfg::G, LPP = Cfg::LPP;
-  constexpr int SPT = Cfg::SPT, RPS = Cfg::ROWS_PER_STAGE;
-  pdl_trigger();
-
-  extern __shared__ unsigned char smem_raw[];
-  // 1024-byte alignment for the TMA swizzle, by pointer arithmetic on the shared array itself (an integer
-  // round trip would make the compiler lose the address space and emit generic loads and stores)
-  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  char* staging = reinterpret_cast<char*>(smem) + (size_t)warp * IC::WARP_BYTES;
-  const uint32_t staging_s = smem_u32(staging);
-  float* ab = reinterpret_cast<float*>(IC::ALIAS ? staging : staging + IC::STAGING_BYTES);
-  float2* rot = reinterpret_cast<float2*>(smem + (size_t)W * IC::WARP_BYTES);
-
-  if (threadIdx.x == 0) prefetch_tensormap(&out_map);
-  // conjugate rotation table: exp(-i pi (sg/N2 + f/N3)) * scale * Hermitian weight
-  for (int e = threadIdx.x; e < 2 * K2 * K3; e += blockDim.x) {
-    const int r = e / K3, f = e % K3;
-    const int sg = (r < K2) ? r : -(2 * K2 - r);
-    const long long num = (long long)sg * N3 + (long long)f * N2;
-    double sn, cs;
-    sincospi((double)num / (double)((long long)N2 * N3), &sn, &cs);
-    const float w = scale * (herm ? herm_weight(f, N3) : 1.0f);
-    rot[f * (2 * K2) + r] = make_float2((float)cs * w, -(float)sn * w);   // [f][r]
-  }
-  __syncthreads();
-
-  // roles: row quadruple (stage 1 / unfold), MMA fragment coordinates, mode loader
-  const int pl1 = lane / QUADS, n1 = lane % QUADS;
-  const int g8 = lane >> 2, t4 = lane & 3;
-  float* combo = ab + IC::AB_FLOATS;
-
-  // Second-dimension basis as MMA A fragments (row = quadruple n, col = frequency slot of the parity class),
-  // TF32 hi/lo.  Classes: 0 = Pe (even g, cos), 1 = Po (odd g, cos), 2 = Qo (odd g, sin), 3 = Qe (even g, sin);
-  // index 4 = the unpaired g = K2 cosine, which adds into Pe through one extra k-step.
-  uint32_t ahi[5][Cfg::MT2][4], alo[5][Cfg::MT2][4];
-#pragma unroll
-  for (int cls = 0; cls < 5; ++cls)
-#pragma unroll
-    for (int mt = 0; mt < Cfg::MT2; ++mt)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int n = (16 * mt + g8 + 8 * (e & 1)) % QUADS;
-        const int gi = t4 + 4 * (e >> 1);
-        int g = 0;
-        bool valid = gi < Cfg::GT;
-        if (cls == 0) g = 2 * gi;
-        else if (cls == 1 || cls == 2) g = 2 * gi + 1;
-        else if (cls == 3) g = 2 * gi + 2;
-        else { g = K2; valid = (gi == 0); }
-        double sn, cs;
-        sincospi((double)(((long long)g * (2 * n + 1)) % (2 * N2)) / (double)N2, &sn, &cs);
-        const float v = valid ? ((cls == 2 || cls == 3) ? (float)sn : (float)cs) : 0.f;
-        split_tf32_rna(v, ahi[cls][mt][e], alo[cls][mt][e]);
-      }
-
-  // loader role: lane = (plane, mode position r)
-  const bool actl = lane < G * LPP;
-  const int pll = actl ? lane / LPP : 0, rl = lane % LPP;
-
-  const long long tstride = (long long)gridDim.x * W;
-  long long task = (long long)blockIdx.x + (long long)warp * gridDim.x;
-  float4 vin[K3 / 2];
-  pdl_wait();   // everything above is independent of the preceding kernel
-  if (task < num_tasks && actl) {
-    const float4* src = reinterpret_cast<const float4*>(in + ((task * G + pll) * (2 * K2) + rl) * K3);
-#pragma unroll
-    for (int i = 0; i < K3 / 2; ++i) vin[i] = __ldcs(src + i);
-  }
-
-  for (; task < num_tasks; task += tstride) {
-    if constexpr (IC::ALIAS) {
-      // the store of the previous task's first block (committed second to last) must have read its rows
-      if (lane == 0) tma_store_wait_read<1>();
-      __syncwarp();
-    }
-    // ---- rotate this task's modes, publish V'
-    if (actl) {
-      float* dst = ab + pll * IC::ABP + rl * IC::ABS;
-      const float2* rr = rot + rl;
-      float re[K3], im[K3];
-#pragma unroll
-      for (int i = 0; i < K3 / 2; ++i) {
-        const float2 r0 = rr[(2 * i) * (2 * K2)], r1 = rr[(2 * i + 1) * (2 * K2)];
-        re[2 * i] = vin[i].x * r0.x - vin[i].y * r0.y;
-        im[2 * i] = vin[i].x * r0.y + vin[i].y * r0.x;
-        re[2 * i + 1] = vin[i].z * r1.x - vin[i].w * r1.y;
-        im[2 * i + 1] = vin[i].z * r1.y + vin[i].w * r1.x;
-      }
-#pragma unroll
-      for (int i = 0; i < K3 / 4; ++i) {
-        *reinterpret_cast<float4*>(dst + 4 * i) = make_float4(re[4 * i], re[4 * i + 1], re[4 * i + 2], re[4 * i + 3]);
-        *reinterpret_cast<float4*>(dst + K3 + 4 * i) =
-            make_float4(im[4 * i], im[4 * i + 1], im[4 * i + 2], im[4 * i + 3]);
-      }
-    }
-    // prefetch the next task's modes while this one is expanded
-    {
-      const long long nt = task + tstride;
-      if (nt < num_tasks && actl) {
-        const float4* src = reinterpret_cast<const float4*>(in + ((nt * G + pll) * (2 * K2) + rl) * K3);
-#pragma unroll
-        for (int i = 0; i < K3 / 2; ++i) vin[i] = __ldcs(src + i);
-      }
-    }
-    __syncwarp();
-    // ---- alpha_g = V'_{+g} + V'_{-g}, beta_g = i (V'_{+g} - V'_{-g}); lane (plane, g), g = 0..K2
-    {
-      const bool acta = lane < G * LPP && (lane % LPP) <= K2;
-      const int pla = acta ? lane / LPP : 0, g = acta ? lane % LPP : 0;
-      float vp[NC], vm[NC];
-      const float* srcp = ab + pla * IC::ABP + g * IC::ABS;
-      const float* srcm = ab + pla * IC::ABP + ((2 * K2 - g) % (2 * K2)) * IC::ABS;
-#pragma unroll
-      for (int c = 0; c < NC; ++c) {
-        vp[c] = (g < K2) ? srcp[c] : 0.f;
-        vm[c] = (g > 0) ? srcm[c] : 0.f;
-      }
-      __syncwarp();
-      if (acta) {
-        float* da = ab + pla * IC::ABP + g * IC::ABS;
-        float* db = ab + pla * IC::ABP + (K2 + 1 + g) * IC::ABS;
-#pragma unroll
-        for (int f = 0; f < K3; ++f) {
-          const float pr = vp[f], pi = vp[K3 + f], mr = vm[f], mi = vm[K3 + f];
-          da[f] = pr + mr;
-          da[K3 + f] = pi + mi;
-          // i * ((pr - mr) + i (pi - mi)) = -(pi - mi) + i (pr - mr)
-          db[f] = -(pi - mi);
-          db[K3 + f] = pr - mr;
-        }
-      }
-    }
-    __syncwarp();
-
-    // ---- expand the second dimension on the tensor cores (warp-level MMA, TF32 hi/lo compensated):
-    // combo_cls[quadruple n][(plane, column)] = sum_slot basis_cls[n][slot] * (alpha|beta)_cls[slot][column]
-#pragma unroll
-    for (int cls = 0; cls < 4; ++cls)
-#pragma unroll
-      for (int nt = 0; nt < IC::NT; ++nt)
-#pragma unroll
-        for (int mt = 0; mt < Cfg::MT2; ++mt) {
-          const int pl = (16 * mt) / QUADS;
-          float acc[4] = {0.f, 0.f, 0.f, 0.f};
-          const int c = 8 * nt + g8;
-          {
-            uint32_t bh[2], bl[2];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              const int gi = t4 + 4 * h;
-              int entry = 0;
-              if (cls == 0) entry = 2 * gi;
-              else if (cls == 1) entry = 2 * gi + 1;
-              else if (cls == 2) entry = K2 + 1 + 2 * gi + 1;
-              else entry = K2 + 1 + 2 * gi + 2;
-              const float v = (gi < Cfg::GT) ? ab[pl * IC::ABP + entry * IC::ABS + c] : 0.f;
-              split_tf32(v, bh[h], bl[h]);
-            }
-            mma_tf32(acc, ahi[cls][mt], bh[0], bh[1]);
-            mma_tf32(acc, alo[cls][mt], bh[0], bh[1]);
-            mma_tf32(acc, ahi[cls][mt], bl[0], bl[1]);
-          }
-          if (cls == 0) {   // unpaired g = K2: slot 0 of an extra k-step, all other slots are zero
-            uint32_t bh[2], bl[2];
-            const float v = (t4 == 0) ? ab[pl * IC::ABP + K2 * IC::ABS + c] : 0.f;
-            split_tf32(v, bh[0], bl[0]);
-            bh[1] = 0u;
-            bl[1] = 0u;
-            mma_tf32(acc, ahi[4][mt], bh[0], bh[1]);
-            mma_tf32(acc, alo[4][mt], bh[0], bh[1]);
-            mma_tf32(acc, ahi[4][mt], bl[0], bl[1]);
-          }
-          // C fragment -> combos row (quadruple), 16-byte chunks swapped pairwise on odd groups of four rows
-          const int colp = (8 * nt + 2 * t4) ^ (((g8 >> 2) & 1) << 2);
-          float* d0 = combo + (size_t)(16 * mt + g8) * Cfg::NS + cls * NC + colp;
-          *reinterpret_cast<float2*>(d0) = make_float2(acc[0], acc[1]);
-          *reinterpret_cast<float2*>(d0 + 8 * Cfg::NS) = make_float2(acc[2], acc[3]);
-        }
-    __syncwarp();
-
-    // this lane's quadruple: Pe, Po, Qo, Qe
-    float Pe[NC], Po[NC], Qo[NC], Qe[NC];
-    {
-      const float* src = combo + (size_t)lane * Cfg::NS;
-      const int sw = (n1 >> 2) & 1;
-#pragma unroll
-      for (int c4 = 0; c4 < NC / 4; ++c4) {
-        const int cc = 4 * (c4 ^ sw);
-        const float4 v0 = *reinterpret_cast<const float4*>(src + 0 * NC + cc);
-        const float4 v1 = *reinterpret_cast<const float4*>(src + 1 * NC + cc);
-        const float4 v2 = *reinterpret_cast<const float4*>(src + 2 * NC + cc);
-        const float4 v3 = *reinterpret_cast<const float4*>(src + 3 * NC + cc);
-        Pe[4 * c4] = v0.x; Pe[4 * c4 + 1] = v0.y; Pe[4 * c4 + 2] = v0.z; Pe[4 * c4 + 3] = v0.w;
-        Po[4 * c4] = v1.x; Po[4 * c4 + 1] = v1.y; Po[4 * c4 + 2] = v1.z; Po[4 * c4 + 3] = v1.w;
-        Qo[4 * c4] = v2.x; Qo[4 * c4 + 1] = v2.y; Qo[4 * c4 + 2] = v2.z; Qo[4 * c4 + 3] = v2.w;
-        Qe[4 * c4] = v3.x; Qe[4 * c4 + 1] = v3.y; Qe[4 * c4 + 2] = v3.z; Qe[4 * c4 + 3] = v3.w;
-      }
-    }
-    // the previous task's TMA stores must have finished reading the staging rows before they are rewritten
-    // (aliased layout: the first block is already free, and every lane has its combos in registers now)
-    if constexpr (!IC::ALIAS) {
-      if (lane == 0) tma_store_wait_read<0>();
-    }
-    __syncwarp();
-
-    // ---- unfold to the four rows (a: n, b: N2/2-1-n, c: N2/2+n, d: N2-1-n) and expand each along the
-    // contiguous dimension; one copy of the row code, signs select the row
-    constexpr bool kSplit = (SPT == 2 && N2 == 128);   // rows a, b fill the first staging block: store it early
-#pragma unroll 1
-    for (int r4 = 0; r4 < 4; ++r4) {
-      if constexpr (kSplit) {
-        if (r4 == 2) {
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) {
-#pragma unroll
-            for (int h = 0; h < Cfg::BOXES; ++h)
-              tma_store_2d(&out_map, h * 32, (int)(task * kTaskRows), staging + (size_t)h * RPS * 128);
-            tma_store_commit();
-            // rows c, d go to the second block: the previous task's store of it must be done reading
-            if constexpr (IC::ALIAS) tma_store_wait_read<1>();
-          }
-          if constexpr (IC::ALIAS) __syncwarp();
-        }
-      }
-      const int rowq = (r4 == 0) ? n1 : (r4 == 1) ? (N2 / 2 - 1 - n1) : (r4 == 2) ? (N2 / 2 + n1) : (N2 - 1 - n1);
-      const float sPo = (r4 == 0 || r4 == 3) ? 1.f : -1.f;   // a, d: +Po;  b, c: -Po
-      const float sQe = (r4 == 0 || r4 == 2) ? 1.f : -1.f;   // a, c: +Qe;  b, d: -Qe
-      const float sQo = (r4 <= 1) ? 1.f : -1.f;              // a, b: +Qo;  c, d: -Qo
-      float z[NC];
-#pragma unroll
-      for (int c = 0; c < NC; ++c) z[c] = fmaf(sQo, Qo[c], fmaf(sQe, Qe[c], fmaf(sPo, Po[c], Pe[c])));
-      const int trow = pl1 * N2 + rowq;
-      expand_row<N3, K3, RPS>(staging_s + (uint32_t)(trow / RPS) * kStageBytes, trow % RPS, z);
-    }
-    fence_proxy_async_smem();
-    __syncwarp();
-    if (lane == 0) {
-#pragma unroll
-      for (int rb = kSplit ? 1 : 0; rb < SPT; ++rb)
-#pragma unroll
-        for (int h = 0; h < Cfg::BOXES; ++h)
-          tma_store_2d(&out_map, h * 32, (int)(task * kTaskRows + (long long)rb * RPS),
-                       staging + (size_t)rb * kStageBytes + (size_t)h * RPS * 128);
-      tma_store_commit();
-    }
-  }
-  if (lane == 0) tma_store_wait_all<0>();
-}
 
 // ---------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -902,44 +36,6 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-template <int N3, int K3, int N2, int K2>
-cudaError_t launch_fwd_plane_t(const float* x, float2* out, long long rows, float scale, int herm, int* status,
-                               const RingDebug& dbg, cudaStream_t st) {
-  constexpr int W = 7;   // consumer warps (+ the producer warp = 2 warps per scheduler; 8 or 10 consumers measured slower)
-  using Cfg = PlaneCfg<N3, K3, N2, K2>;
-  const SmemPlan sp = smem_plan<Cfg, K2, K3, W>();
-  if (sp.stages < 2 * Cfg::SPT) return cudaErrorInvalidConfiguration;
-  CUtensorMap map;
-  if (!make_rows_map(&map, x, rows, N3, Cfg::ROWS_PER_STAGE)) return cudaErrorNotSupported;
-  auto kern = fwd_plane_kernel<N3, K3, N2, K2, W>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sp.total);
-  if (e != cudaSuccess) return e;
-  const long long tasks = rows / kTaskRows;
-  const int grid = (int)(tasks < num_sms() ? tasks : num_sms());
-  (void)launch_pdl(kern, dim3(grid), dim3((W + 1) * 32), sp.total, st, map, out, tasks, scale, herm, sp.stages, status,
-                   dbg.poll_limit, dbg.withhold_after);
-  return cudaGetLastError();
-}
-
-template <int N3, int K3, int N2, int K2>
-cudaError_t launch_inv_plane_t(const float2* in, float* y, long long rows, float scale, int herm, cudaStream_t st) {
-  using IC = InvCfg<N3, K3, N2, K2>;
-  constexpr int W = (IC::WARP_BYTES * 7 + 2 * K2 * K3 * 8 + 1024 <= kSmemLimit) ? 7
-                    : (IC::WARP_BYTES * 6 + 2 * K2 * K3 * 8 + 1024 <= kSmemLimit) ? 6 : 5;
-  const size_t total = (size_t)W * IC::WARP_BYTES + (size_t)2 * K2 * K3 * 8 + 1024;
-  static_assert((size_t)W * IC::WARP_BYTES + (size_t)2 * K2 * K3 * 8 + 1024 <= kSmemLimit, "shared memory");
-  CUtensorMap map;
-  if (!make_rows_map(&map, y, rows, N3, PlaneCfg<N3, K3, N2, K2>::ROWS_PER_STAGE)) return cudaErrorNotSupported;
-  auto kern = inv_plane_kernel<N3, K3, N2, K2, W>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
-  if (e != cudaSuccess) return e;
-  const long long tasks = rows / kTaskRows;
-  const long long want = (tasks + W - 1) / W;
-  const int grid = (int)(want < num_sms() ? want : num_sms());
-  (void)launch_pdl(kern, dim3(grid), dim3(W * 32), total, st, map, in, tasks, scale, herm);
-  return cudaGetLastError();
-}
-
 }  // namespace
 
 // 2-D fp32 tensor [rows][n3] viewed through [box_rows x 32] boxes with the 128-byte swizzle.
@@ -958,8 +54,10 @@ bool make_rows_map(CUtensorMap* map, const void* base, long long rows, int n3, i
 
 // Shapes the plane kernels are instantiated for: (N3, k3, N2, k2).
 static bool plane_supported(int N3, int K3, int N2, int K2) {
-  return (N3 == 64 && K3 == 8 && N2 == 128 && K2 == 16) || (N3 == 32 && K3 == 4 && N2 == 64 && K2 == 8) ||
-         (N3 == 64 && K3 == 8 && N2 == 64 && K2 == 8);
+#define DTST_MATCH(a, b, c, d) if (N3 == a && K3 == b && N2 == c && K2 == d) return true;
+  DTST_PLANE_SHAPES(DTST_MATCH)
+#undef DTST_MATCH
+  return false;
 }
 
 bool fused_eligible(const dtst_plan* p) {
@@ -969,35 +67,59 @@ bool fused_eligible(const dtst_plan* p) {
   if (p->Nl[a] != p->Ng[a] || p->Nl[b] != p->Ng[b] || p->off[a] != 0 || p->off[b] != 0) return false;
   if (p->d == 2 && p->P > 1) return false;   // slabs would cut the second-last dimension
   if (!plane_supported((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b])) return false;
-  const int Cmin = 1;
-  long long planes = (long long)p->B * Cmin;
+  long long planes = (long long)p->B;
   for (int i = 0; i < b; ++i) planes *= p->Nl[i];
   // tasks are 128 rows: with 64-row planes every tensor must hold an even number of planes
   long long pin = planes * p->C_in, pout = planes * p->C_out;
-  if ((pin * p->Ng[b]) % kTaskRows != 0 || (pout * p->Ng[b]) % kTaskRows != 0) return false;
+  if ((pin * p->Ng[b]) % plane::kTaskRows != 0 || (pout * p->Ng[b]) % plane::kTaskRows != 0) return false;
   if (pin * p->Ng[b] >= (1ll << 31) || pout * p->Ng[b] >= (1ll << 31)) return false;   // 32-bit TMA coordinates
   return encode_tiled_fn() != nullptr;
 }
 
 cudaError_t launch_fwd_plane(int N3, int K3, int N2, int K2, const float* x, float2* out, long long rows,
                              float scale, int herm, int* status, const RingDebug& dbg, cudaStream_t st) {
-  if (N3 == 64 && K3 == 8 && N2 == 128 && K2 == 16)
-    return launch_fwd_plane_t<64, 8, 128, 16>(x, out, rows, scale, herm, status, dbg, st);
-  if (N3 == 32 && K3 == 4 && N2 == 64 && K2 == 8)
-    return launch_fwd_plane_t<32, 4, 64, 8>(x, out, rows, scale, herm, status, dbg, st);
-  if (N3 == 64 && K3 == 8 && N2 == 64 && K2 == 8)
-    return launch_fwd_plane_t<64, 8, 64, 8>(x, out, rows, scale, herm, status, dbg, st);
+#define DTST_CALL(a, b, c, d) \
+  if (N3 == a && K3 == b && N2 == c && K2 == d) return plane::plane_fwd<a, b, c, d>(x, out, rows, scale, herm, status, dbg, st);
+  DTST_PLANE_SHAPES(DTST_CALL)
+#undef DTST_CALL
   return cudaErrorNotSupported;
 }
 
-}  // namespace dtst
-
-namespace dtst {
 cudaError_t launch_inv_plane(int N3, int K3, int N2, int K2, const float2* in, float* y, long long rows, float scale,
                              int herm, int* /*status*/, cudaStream_t st) {
-  if (N3 == 64 && K3 == 8 && N2 == 128 && K2 == 16) return launch_inv_plane_t<64, 8, 128, 16>(in, y, rows, scale, herm, st);
-  if (N3 == 32 && K3 == 4 && N2 == 64 && K2 == 8) return launch_inv_plane_t<32, 4, 64, 8>(in, y, rows, scale, herm, st);
-  if (N3 == 64 && K3 == 8 && N2 == 64 && K2 == 8) return launch_inv_plane_t<64, 8, 64, 8>(in, y, rows, scale, herm, st);
+  const plane::ColExpandArgs none{};
+#define DTST_CALL(a, b, c, d) \
+  if (N3 == a && K3 == b && N2 == c && K2 == d) return plane::plane_inv<a, b, c, d, 0, 1>(in, y, rows, scale, herm, none, st);
+  DTST_PLANE_SHAPES(DTST_CALL)
+#undef DTST_CALL
   return cudaErrorNotSupported;
 }
+
+// The helper-warp variant is built for a leading dimension of the same shape as the second plane dimension.
+bool inv_plane_colexp_supported(int N3, int K3, int N2, int K2, int N1, int K1) {
+  if (!plane_supported(N3, K3, N2, K2)) return false;
+  return N1 == N2 && K1 == K2 && (2 * K2 * K3) % (8 * plane::kColExpandMT) == 0;
+}
+
+cudaError_t launch_inv_plane_colexp(int N3, int K3, int N2, int K2, int N1, int K1, const float2* in1, float2* ring,
+                                    int ring_cols, int* counters, long long cols, float* y, long long rows,
+                                    float scale, int herm, int* status, uint32_t poll_limit, cudaStream_t st) {
+  if (!inv_plane_colexp_supported(N3, K3, N2, K2, N1, K1)) return cudaErrorNotSupported;
+  plane::ColExpandArgs ce{};
+  ce.in1 = in1;
+  ce.ring = ring;
+  ce.ready = counters;
+  ce.done = counters + cols;
+  ce.status = status;
+  ce.cols = cols;
+  ce.N1 = N1;
+  ce.R = ring_cols < 1 ? 1 : ring_cols;
+  ce.poll_limit = poll_limit;
+#define DTST_CALL(a, b, c, d) \
+  if (N3 == a && K3 == b && N2 == c && K2 == d) return plane::plane_inv<a, b, c, d, d, c / 32>(ring, y, rows, scale, herm, ce, st);
+  DTST_PLANE_SHAPES(DTST_CALL)
+#undef DTST_CALL
+  return cudaErrorNotSupported;
+}
+
 }  // namespace dtst

@@ -16,6 +16,14 @@ cudaError_t launch_fwd_plane(int N3, int K3, int N2, int K2, const float* x, flo
 cudaError_t launch_inv_plane(int N3, int K3, int N2, int K2, const float2* in, float* y, long long rows,
                              float scale, int herm, int* status, cudaStream_t st);
 
+// The same with the expansion of the dimension in front of the plane (extent N1, 2 K1 retained entries) done inside
+// the kernel by a helper warp per CTA: in1[cols][2 K1][2 K2 K3] is expanded column by column into `ring`
+// ([ring_cols][N1][2 K2 K3], consumed from L2); `counters` holds 2 * cols ints (zeroed by the launch).
+bool inv_plane_colexp_supported(int N3, int K3, int N2, int K2, int N1, int K1);
+cudaError_t launch_inv_plane_colexp(int N3, int K3, int N2, int K2, int N1, int K1, const float2* in1, float2* ring,
+                                    int ring_cols, int* counters, long long cols, float* y, long long rows,
+                                    float scale, int herm, int* status, uint32_t poll_limit, cudaStream_t st);
+
 // 2-D fp32 tensor [rows][n3] viewed through [box_rows x 32 floats] boxes with the 128-byte TMA swizzle.
 bool make_rows_map(CUtensorMap* map, const void* base, long long rows, int n3, int box_rows);
 

@@ -20,14 +20,6 @@ namespace dtst {
 namespace {
 
 
-// cos / sin of pi * g * (2 q + 1) / N with the phase reduced exactly in integers
-__device__ __forceinline__ void basis_cs(int g, int q, int N, float& cs, float& sn) {
-  double s, c;
-  sincospi((double)(((long long)g * (2 * q + 1)) % (2ll * N)) / (double)N, &s, &c);
-  cs = (float)c;
-  sn = (float)s;
-}
-
 // ------------------------------------------------------------------------------------------
 // contraction: in[outer][N][inner] -> out[outer][2K][inner]
 //
@@ -63,9 +55,6 @@ __device__ __forceinline__ void cp_async16(float* smem_dst, const float* gsrc) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-// frequency of slot s in parity class cls (0: even cos, 1: odd cos, 2: odd sin, 3: even sin)
-__device__ __forceinline__ int class_freq(int cls, int s) { return cls == 0 ? 2 * s : (cls == 3 ? 2 * s + 2 : 2 * s + 1); }
 
 // One k-step (8 quadruples) of one m-tile (8 complex positions) from a filled stage.
 __device__ __forceinline__ void contract_step(const float* S, const float4* bt, float ck0, float ck1,

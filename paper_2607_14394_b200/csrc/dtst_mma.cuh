@@ -48,4 +48,16 @@ __device__ __forceinline__ void mma3_tf32(float (&d)[4], const uint32_t (&ahi)[4
   mma_m16n8k8_tf32(d, ahi, bl0, bl1);
 }
 
+// cos / sin of pi * g * (2 q + 1) / N (the half-sample phase psi_g (q + 1/2), psi_g = 2 pi g / N) with the phase
+// reduced exactly in integers: the basis of the folded two-sided dimensions
+__device__ __forceinline__ void basis_cs(int g, int q, int N, float& cs, float& sn) {
+  double s, c;
+  sincospi((double)(((long long)g * (2 * q + 1)) % (2ll * N)) / (double)N, &s, &c);
+  cs = (float)c;
+  sn = (float)s;
+}
+
+// frequency of slot s in parity class cls (0: even cos, 1: odd cos, 2: odd sin, 3: even sin)
+__device__ __forceinline__ int class_freq(int cls, int s) { return cls == 0 ? 2 * s : (cls == 3 ? 2 * s + 2 : 2 * s + 1); }
+
 }  // namespace dtst

@@ -324,6 +324,95 @@ def test_bounded_wait_runs_out_and_is_reported_once():
     del junk
 
 
+def test_in_kernel_column_expansion_gives_the_same_bits():
+    """The optional inverse-type kernel that expands dimension d-3 on a helper warp inside the plane kernel
+    (flow control through per-column counters in global memory, a ring of columns consumed from L2) does the
+    same arithmetic as the separate launch: same bits, for rings smaller and larger than the column count, and
+    against the oracle."""
+    from paper_2607_14394_b200 import Plan, binding as Bn
+    w = I.WORKLOADS["cfg3_4d_64"]
+    Wd, g = _dev(I.make_weights(w)), _dev(I.make_upstream_grad(w))
+    x = _dev(I.make_field(w))
+    ref_plan = _plan(w)
+    Xhat = ref_plan.forward(x)
+    Yhat = ref_plan.spectral_mul(Xhat, Wd)
+    y_ref = ref_plan.inverse(Yhat)
+    gx_ref, gW_ref = ref_plan.backward(g, Xhat, Wd)
+    torch.cuda.synchronize()
+    launches_ref = ref_plan.launch_count()
+    for ring in (3, 16, 10_000):
+        plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out, column_expansion=ring)
+        y = plan.inverse(Yhat)
+        y2 = plan.inverse(Yhat)                       # the counters start every launch from zero
+        gx, gW = plan.backward(g, Xhat, Wd)
+        torch.cuda.synchronize()
+        assert plan.status() == 0
+        assert torch.equal(y, y_ref) and torch.equal(y2, y_ref) and torch.equal(gx, gx_ref)
+        assert torch.equal(torch.view_as_real(gW), torch.view_as_real(gW_ref))
+        plan.close()
+    y_or = O.inverse(O.spectral_mul(O.forward(I.make_field(w), w.kmax), I.make_weights(w).reshape((w.C_in, w.C_out) + w.K)),
+                     w.N, w.kmax)
+    assert O.rel_l2(y_ref.cpu().numpy(), y_or) <= TOL
+    # shapes without such a kernel say so
+    w2 = I.custom_workload("nocolexp", 1, 2, 2, (16, 24, 40), (3, 5, 6))
+    p2 = _plan(w2)
+    with pytest.raises(Bn.DtstError) as e:
+        Bn.dtst_plan_set_column_expansion(p2.handle, 8)
+    assert e.value.status == Bn.DTST_ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------ more plane shapes than the benchmark's three
+PLANE_SHAPES = [
+    # name, B, Ci, Co, N, kmax: (N3, k3, N2, k2) of the last two dimensions is a shape the plane kernels exist for
+    ("p_64_8_128_8", 1, 2, 2, (32, 128, 64), (4, 8, 8)),
+    ("p_32_8_64_8", 1, 2, 3, (32, 32, 64, 32), (4, 8, 8, 8)),
+    ("p_32_8_128_16", 1, 1, 2, (64, 128, 32), (8, 16, 8)),
+    ("p_32_8_128_8", 2, 1, 1, (32, 128, 32), (16, 8, 8)),
+    ("p_64_4_64_8", 1, 2, 2, (32, 64, 64), (12, 8, 4)),
+    ("p_64_8_64_8_d3", 1, 2, 2, (64, 64, 64), (8, 8, 8)),
+]
+
+
+@pytest.mark.parametrize("case", PLANE_SHAPES, ids=[c[0] for c in PLANE_SHAPES])
+def test_more_plane_shapes_run_fused_and_match_the_oracle(case):
+    name, B, Ci, Co, N, k = case
+    w = I.custom_workload(name, B, Ci, Co, N, k, field="grf", seed=29)
+    plan = _plan(w)
+    assert plan.kernel_path == "fused"
+    plan.require_fast_path()            # every stage on a streaming kernel, or this raises
+    plan.close()
+    run_layer_and_check(w, "auto")
+    run_layer_and_check(w, "auto", P=4)
+
+
+def test_fast_path_or_fail():
+    from paper_2607_14394_b200 import binding as Bn
+    # an odd extent in the middle: the generic kernel would serve that dimension
+    w = I.custom_workload("slowmid", 1, 2, 2, (9, 64, 64), (3, 8, 8))
+    plan = _plan(w)
+    with pytest.raises(Bn.DtstError) as e:
+        plan.require_fast_path()
+    assert e.value.status == Bn.DTST_ERR_UNSUPPORTED
+    plan.forward(_dev(I.make_field(w)))                      # not required: still runs (on the generic kernel)
+    # all stages streaming: accepted; switching the plan to the generic family afterwards makes the calls refuse
+    w2 = I.WORKLOADS["cfg3_4d_64"]
+    p2 = _plan(w2)
+    p2.require_fast_path()
+    x2 = _dev(I.make_field(w2))
+    p2.forward(x2)
+    Bn.dtst_plan_set_kernel_path(p2.handle, Bn.DTST_PATH_GENERIC)
+    before = p2.launch_count()
+    with pytest.raises(Bn.DtstError) as e:
+        p2.forward(x2)
+    assert e.value.status == Bn.DTST_ERR_UNSUPPORTED and p2.launch_count() == before
+    p2.require_fast_path(False)
+    p2.forward(x2)
+    # the row family counts as fast as well
+    p4 = _plan(I.WORKLOADS["cfg2_3d_64"])
+    assert p4.kernel_path == "row"
+    p4.require_fast_path()
+
+
 def test_adjoint_identity_on_device():
     # <F x, Y> = <x, F^H Y> holds for the kernels themselves at a size the oracle need not touch
     w = I.custom_workload("adj", 1, 2, 2, (32, 32, 64), (4, 6, 8), seed=77)
