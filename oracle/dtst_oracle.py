@@ -16,8 +16,8 @@ Conventions (d transformed dims, grid N = (N_0..N_{d-1}), last one contiguous):
 Every function below is pinned by tests that do not re-use its own formula:
 numpy.fft (rfftn-then-slice, irfftn of the zero-padded spectrum), closed forms,
 brute force on tiny grids, the adjoint identity, Parseval, slab linearity,
-finite differences and torch float64 autograd.  Nothing here is "parity
-unpinned".
+finite differences and torch float64 autograd (the block of Algorithm 1 with
+its bypass and GELU included).  Nothing here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -253,6 +253,60 @@ def backward(grad_y: np.ndarray, Xhat: np.ndarray, W: np.ndarray, kmax, N_global
     g_x = inverse(G_X.reshape((B, Ci) + G_Y.shape[2:]), N, kmax, n_local=n_local, offsets=offsets,
                   doubling=False, normalise=False)
     return g_x, G_W.reshape(W.shape)
+
+
+# --------------------------------------------------------------------------
+# The whole block (Section "Block Structure", Algorithm 1 lines 1 and 8; Eq. 1):
+#     x_next = GELU(W_bypass x + y),   y = I(M(F(x), W))
+# W_bypass is the point-wise linear operator: [C_out, C_in], applied at every grid point; no bias is mentioned in
+# the paper and none is applied.  GELU is the exact (erf) form, z Phi(z).
+# --------------------------------------------------------------------------
+def _erf(z: np.ndarray) -> np.ndarray:
+    from scipy.special import erf      # a library primitive as one step; pinned against math.erf and torch
+    return erf(z)
+
+
+def gelu(z: np.ndarray) -> np.ndarray:
+    """GELU(z) = z * Phi(z) = z/2 * (1 + erf(z / sqrt 2))."""
+    z = np.asarray(z, dtype=np.float64)
+    return 0.5 * z * (1.0 + _erf(z / math.sqrt(2.0)))
+
+
+def gelu_grad(z: np.ndarray) -> np.ndarray:
+    """d GELU / dz = Phi(z) + z * phi(z), phi the standard normal density."""
+    z = np.asarray(z, dtype=np.float64)
+    return 0.5 * (1.0 + _erf(z / math.sqrt(2.0))) + z * np.exp(-0.5 * z * z) / math.sqrt(2.0 * math.pi)
+
+
+def bypass(x: np.ndarray, Wb: np.ndarray) -> np.ndarray:
+    """(W_bypass x)[b, o, n] = sum_i Wb[o, i] x[b, i, n]  (Algorithm 1 line 1)."""
+    return np.einsum("oi,bi...->bo...", np.asarray(Wb, dtype=np.float64), np.asarray(x, dtype=np.float64))
+
+
+def block_forward(x: np.ndarray, W: np.ndarray, Wb: np.ndarray, kmax, N_global=None, offsets=None):
+    """Returns (out, z, Xhat): z = W_bypass x + I(M(F(x), W)) is the pre-activation, out = GELU(z)
+    (Algorithm 1 lines 1-8 without the collectives; with N_global/offsets, x is one rank's block and Xhat its
+    partial spectrum, so z and out are only meaningful once the partial spectra have been summed)."""
+    y, Xhat = layer_forward(x, W, kmax, N_global=N_global, offsets=offsets)
+    z = bypass(x, Wb) + y
+    return gelu(z), z, Xhat
+
+
+def block_backward(grad_out: np.ndarray, x: np.ndarray, z: np.ndarray, Xhat: np.ndarray, W: np.ndarray,
+                   Wb: np.ndarray, kmax, N_global=None, offsets=None):
+    """Gradients of L = sum(out * grad_out) w.r.t. x, W (spectral) and W_bypass.
+
+    g_z = grad_out * GELU'(z)                                  adjoint of the activation
+    grad_Wb[o, i] = sum_{b, n} g_z[b, o, n] x[b, i, n]         the bypass is linear in Wb
+    grad_x = Wb^T g_z + (adjoint of the spectral layer)(g_z)   (Section "Backward Pass")
+    """
+    gz = np.asarray(grad_out, dtype=np.float64) * gelu_grad(z)
+    gx_spec, gW = backward(gz, Xhat, W, kmax, N_global=N_global, offsets=offsets)
+    xb = np.asarray(x, dtype=np.float64)
+    B = xb.shape[0]
+    gWb = np.einsum("bon,bin->oi", gz.reshape(B, gz.shape[1], -1), xb.reshape(B, xb.shape[1], -1))
+    gx = np.einsum("oi,bo...->bi...", np.asarray(Wb, dtype=np.float64), gz) + gx_spec
+    return gx, gW, gWb
 
 
 # --------------------------------------------------------------------------

@@ -276,6 +276,106 @@ def test_layer_and_backward_match_torch_autograd(N, kmax):
     assert O.rel_l2(gW, gW_ref) < 1e-12
 
 
+# ---------------------------------------------------------------- the whole block (bypass + GELU)
+def test_gelu_against_math_erf_closed_forms_and_torch():
+    import torch
+    z = np.concatenate([np.linspace(-9, 9, 721), RNG.standard_normal(300) * 3])
+    want = np.array([0.5 * v * (1.0 + math.erf(v / math.sqrt(2.0))) for v in z])
+    assert np.max(np.abs(O.gelu(z) - want)) < 1e-15
+    assert O.gelu(0.0) == 0.0
+    assert np.allclose(O.gelu(z) - O.gelu(-z), z, atol=1e-14)          # z Phi(z) + z Phi(-z) = z
+    assert abs(O.gelu(40.0) - 40.0) < 1e-12 and abs(O.gelu(-40.0)) < 1e-12
+    t = torch.tensor(z, dtype=torch.float64, requires_grad=True)
+    out = torch.nn.functional.gelu(t)                                  # exact (erf) form
+    out.sum().backward()
+    assert np.max(np.abs(O.gelu(z) - out.detach().numpy())) < 1e-14
+    assert np.max(np.abs(O.gelu_grad(z) - t.grad.numpy())) < 1e-13
+    h = 1e-6                                                           # and a central difference
+    assert np.max(np.abs((O.gelu(z + h) - O.gelu(z - h)) / (2 * h) - O.gelu_grad(z))) < 1e-8
+
+
+def test_bypass_is_a_pointwise_matrix_product():
+    x = RNG.standard_normal((2, 3, 4, 5))
+    Wb = RNG.standard_normal((2, 3))
+    z = O.bypass(x, Wb)
+    for b in range(2):
+        for n0 in range(4):
+            for n1 in range(5):
+                assert np.allclose(z[b, :, n0, n1], Wb @ x[b, :, n0, n1])
+    assert np.allclose(O.bypass(x[:, :, :, :], np.eye(3)), x)
+
+
+def _torch_block_grads(x, W, Wb, g, kmax):
+    import torch
+    N = x.shape[2:]
+    d = len(N)
+    dims = tuple(range(2, 2 + d))
+    lists = O.mode_index_lists(N, kmax)
+    xt = torch.tensor(x, dtype=torch.float64, requires_grad=True)
+    Wt = torch.tensor(W, dtype=torch.complex128, requires_grad=True)
+    Wbt = torch.tensor(Wb, dtype=torch.float64, requires_grad=True)
+    Xf = torch.fft.rfftn(xt, dim=dims)
+    ix = torch.meshgrid(*[torch.tensor(l) for l in lists], indexing="ij")
+    Xs = Xf[(slice(None), slice(None)) + tuple(ix)]
+    K = Xs.shape[2:]
+    Ys = torch.einsum("bim,iom->bom", Xs.reshape(x.shape[0], x.shape[1], -1), Wt.reshape(W.shape[0], W.shape[1], -1))
+    full = torch.zeros((x.shape[0], W.shape[1]) + tuple(N[:-1]) + (N[-1] // 2 + 1,), dtype=torch.complex128)
+    full[(slice(None), slice(None)) + tuple(ix)] = Ys.reshape((x.shape[0], W.shape[1]) + tuple(K))
+    y = torch.fft.irfftn(full, s=N, dim=dims)
+    lin = torch.nn.functional.linear(xt.movedim(1, -1), Wbt).movedim(-1, 1)     # a 1x1 convolution, no bias
+    out = torch.nn.functional.gelu(lin + y)
+    (out * torch.tensor(g)).sum().backward()
+    return out.detach().numpy(), xt.grad.numpy(), Wt.grad.numpy(), Wbt.grad.numpy()
+
+
+@pytest.mark.parametrize("N,kmax", [((8, 6, 10), (2, 3, 3)), ((4, 6, 5, 8), (2, 1, 2, 3)), ((6, 8), (3, 5))])
+def test_block_forward_and_backward_match_torch_autograd(N, kmax):
+    B, Ci, Co = 2, 3, 2
+    x = _rand_x(N, B, Ci)
+    M = O.num_modes(N, kmax)
+    W = (RNG.standard_normal((Ci, Co, M)) + 1j * RNG.standard_normal((Ci, Co, M))) * 3.0
+    Wb = RNG.standard_normal((Co, Ci))
+    g = RNG.standard_normal((B, Co) + tuple(N))
+    out_ref, gx_ref, gW_ref, gWb_ref = _torch_block_grads(x, W, Wb, g, kmax)
+    out, z, Xhat = O.block_forward(x, W, Wb, kmax)
+    gx, gW, gWb = O.block_backward(g, x, z, Xhat, W, Wb, kmax)
+    assert O.rel_l2(out, out_ref) < 1e-12
+    assert O.rel_l2(gx, gx_ref) < 1e-12
+    assert O.rel_l2(gW, gW_ref) < 1e-12
+    assert O.rel_l2(gWb, gWb_ref) < 1e-12
+    # with the bypass and the activation switched off the block is the layer itself
+    y, _ = O.layer_forward(x, W, kmax)
+    _, z0, _ = O.block_forward(x, W, np.zeros_like(Wb), kmax)
+    assert np.allclose(z0, y, atol=1e-13)
+
+
+def test_block_backward_matches_finite_differences():
+    N, kmax, B, Ci, Co = (4, 6), (2, 2), 1, 2, 2
+    x = _rand_x(N, B, Ci)
+    M = O.num_modes(N, kmax)
+    W = (RNG.standard_normal((Ci, Co, M)) + 1j * RNG.standard_normal((Ci, Co, M)))
+    Wb = RNG.standard_normal((Co, Ci))
+    g = RNG.standard_normal((B, Co) + N)
+    loss = lambda xx, ww, wb: float(np.sum(O.block_forward(xx, ww, wb, kmax)[0] * g))
+    out, z, Xhat = O.block_forward(x, W, Wb, kmax)
+    gx, gW, gWb = O.block_backward(g, x, z, Xhat, W, Wb, kmax)
+    h = 1e-6
+    for idx in [(0, 0, 1, 2), (0, 1, 3, 5)]:
+        e = np.zeros_like(x)
+        e[idx] = h
+        assert abs((loss(x + e, W, Wb) - loss(x - e, W, Wb)) / (2 * h) - gx[idx]) < 1e-7
+    for idx in [(0, 1), (1, 0)]:
+        e = np.zeros_like(Wb)
+        e[idx] = h
+        assert abs((loss(x, W, Wb + e) - loss(x, W, Wb - e)) / (2 * h) - gWb[idx]) < 1e-7
+    for idx in [(0, 1, 3), (1, 0, 5)]:
+        e = np.zeros_like(W)
+        e[idx] = h
+        re = (loss(x, W + e, Wb) - loss(x, W - e, Wb)) / (2 * h)
+        im = (loss(x, W + 1j * e, Wb) - loss(x, W - 1j * e, Wb)) / (2 * h)
+        assert abs(re - gW[idx].real) < 1e-7 and abs(im - gW[idx].imag) < 1e-7
+
+
 def test_block_layer_and_backward_are_slices_and_sums_of_the_global_ones():
     # a rank's block (Eq. 18): y and grad_x of the block are slices of the global results when the
     # block's spectrum is replaced by the summed one; partial spectra and grad_W sum over blocks
