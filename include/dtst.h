@@ -193,6 +193,38 @@ dtst_status dtst_backward(dtst_plan* plan, const float* grad_y, const void* Xhat
                           const void* W, float* grad_x, void* grad_W, void* stream);
 
 /*
+ * The whole block around the layer (Section "Block Structure"; Algorithm 1 lines 1 and 8; Eq. 1):
+ *   z   = W_bypass x + I(M(F(x), W))        z[b,o,n] = sum_i W_bypass[o,i] x[b,i,n] + y[b,o,n]
+ *   out = GELU(z) = z Phi(z)                 (exact erf form; the paper names GELU and no bias)
+ *   x [B, C_in, n...] float32; W [C_in, C_out, M] complex64 (the spectral weights of dtst_spectral_mul);
+ *   W_bypass [C_out, C_in] float32, row-major (the point-wise linear operator, a 1x1 convolution's weight);
+ *   out [B, C_out, n...] float32 (written); Xhat_saved [B, C_in, M] complex64 (written: F(x), needed by
+ *   the backward pass); z_saved [B, C_out, n...] float32, the pre-activation, written when not NULL (pass NULL
+ *   for inference).  out and z_saved must not alias x or each other.
+ * The mixed spectrum lives in the plan's workspace.  Needs grid points per (b, c) % 4 == 0 (always true, the
+ * contiguous extent is a multiple of 4) and C_in * C_out <= 4096, else DTST_ERR_UNSUPPORTED.
+ */
+dtst_status dtst_block_forward(dtst_plan* plan, const float* x, const void* W, const float* W_bypass,
+                               float* out, void* Xhat_saved, float* z_saved, void* stream);
+
+/*
+ * Backward pass of the block for upstream gradient grad_out = dL/d out (Section "Backward Pass": the linear
+ * steps are replaced by their adjoints; the activation by its derivative):
+ *   g_z            = grad_out * GELU'(z_saved),   GELU'(z) = Phi(z) + z phi(z)
+ *   grad_W_bypass[o,i] = sum_{b,n} g_z[b,o,n] x[b,i,n]
+ *   (grad_x, grad_W)   = dtst_backward(g_z, ...);   grad_x += W_bypass^T g_z
+ *   scratch [B, C_out, n...] float32: caller-owned, overwritten with g_z (it may be grad_out itself when the
+ *   caller no longer needs grad_out); it must not alias x, z_saved or grad_x.
+ *   grad_x [B, C_in, n...], grad_W [C_in, C_out, M] complex64, grad_W_bypass [C_out, C_in] are ASSIGNED; any of
+ *   them may be NULL to skip it (not all three).  Xhat_saved is read for grad_W only.
+ * The sum over grid points for grad_W_bypass runs in a fixed order (per-CTA partial sums in the workspace,
+ * added in ascending CTA order): repeated calls give the same bits.
+ */
+dtst_status dtst_block_backward(dtst_plan* plan, const float* grad_out, const float* x, const float* z_saved,
+                                const void* Xhat_saved, const void* W, const float* W_bypass, float* scratch,
+                                float* grad_x, void* grad_W, float* grad_W_bypass, void* stream);
+
+/*
  * The same steps one by one, for a caller that runs the layer across several ranks (Algorithm 1: each
  * rank owns a slab of the grid and an equal, contiguous share S_p of the flattened modes, Eq. 12) and
  * exchanges spectra between the steps with its own collectives:

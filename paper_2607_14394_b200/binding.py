@@ -38,7 +38,7 @@ EXPORTED = [
     "dtst_backward", "dtst_plan_status", "dtst_plan_launch_count", "dtst_status_string",
     "dtst_version", "dtst_plan_enable_kernel_timing", "dtst_plan_kernel_timing", "dtst_forward_static",
     "dtst_plan_last_cuda_error", "dtst_spectral_mul_modes", "dtst_backward_spectrum", "dtst_backward_mix_modes",
-    "dtst_backward_input", "dtst_plan_debug_ring_fault", "dtst_plan_set_column_expansion", "dtst_plan_require_fast_path",
+    "dtst_backward_input", "dtst_plan_debug_ring_fault", "dtst_plan_set_column_expansion", "dtst_plan_require_fast_path", "dtst_block_forward", "dtst_block_backward",
 ]
 
 
@@ -77,6 +77,8 @@ def lib() -> ctypes.CDLL:
     L.dtst_spectral_mul.argtypes = [vp, vp, vp, vp, vp]
     L.dtst_inverse.argtypes = [vp, vp, vp, vp]
     L.dtst_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.dtst_block_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+    L.dtst_block_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.dtst_spectral_mul_modes.argtypes = [vp, vp, vp, vp, ctypes.c_int64, ctypes.c_int64, vp]
     L.dtst_backward_spectrum.argtypes = [vp, vp, vp, vp]
     L.dtst_backward_mix_modes.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_int64, ctypes.c_int64, vp]
@@ -241,6 +243,25 @@ def dtst_backward(plan, grad_y, Xhat_saved, W, grad_x, grad_W, stream=None) -> N
                                _stream_ptr(stream)), "dtst_backward", plan)
 
 
+def dtst_block_forward(plan, x, W, W_bypass, out, Xhat_saved, z_saved, stream=None) -> None:
+    _check(lib().dtst_block_forward(plan, _ptr(x, torch.float32, "x"), _ptr(W, torch.complex64, "W"),
+                                    _ptr(W_bypass, torch.float32, "W_bypass"), _ptr(out, torch.float32, "out"),
+                                    _ptr(Xhat_saved, torch.complex64, "Xhat_saved"),
+                                    _ptr(z_saved, torch.float32, "z_saved"), _stream_ptr(stream)),
+           "dtst_block_forward", plan)
+
+
+def dtst_block_backward(plan, grad_out, x, z_saved, Xhat_saved, W, W_bypass, scratch, grad_x, grad_W, grad_W_bypass,
+                        stream=None) -> None:
+    _check(lib().dtst_block_backward(plan, _ptr(grad_out, torch.float32, "grad_out"), _ptr(x, torch.float32, "x"),
+                                     _ptr(z_saved, torch.float32, "z_saved"),
+                                     _ptr(Xhat_saved, torch.complex64, "Xhat_saved"), _ptr(W, torch.complex64, "W"),
+                                     _ptr(W_bypass, torch.float32, "W_bypass"), _ptr(scratch, torch.float32, "scratch"),
+                                     _ptr(grad_x, torch.float32, "grad_x"), _ptr(grad_W, torch.complex64, "grad_W"),
+                                     _ptr(grad_W_bypass, torch.float32, "grad_W_bypass"), _stream_ptr(stream)),
+           "dtst_block_backward", plan)
+
+
 def dtst_spectral_mul_modes(plan, Xhat, W_shard, Yhat_chunk, m0, count, stream=None) -> None:
     _check(lib().dtst_spectral_mul_modes(plan, _ptr(Xhat, torch.complex64, "Xhat"),
                                          _ptr(W_shard, torch.complex64, "W_shard"),
@@ -376,7 +397,7 @@ class Plan:
         pts = math.prod(self.N)
         return {"x": self.B * self.C_in * pts, "y": self.B * self.C_out * pts,
                 "Xhat": self.B * self.C_in * self.M, "Yhat": self.B * self.C_out * self.M,
-                "W": self.C_in * self.C_out * self.M,
+                "W": self.C_in * self.C_out * self.M, "Wb": self.C_in * self.C_out,
                 "Xchunk": self.B * self.C_in * (count or 0), "Ychunk": self.B * self.C_out * (count or 0),
                 "Wshard": self.C_in * self.C_out * (count or 0)}[kind]
 
@@ -446,6 +467,43 @@ class Plan:
         with torch.cuda.device(self.device):
             dtst_backward(self._h, grad_y, Xhat_saved, W, grad_x, grad_W, stream)
         return grad_x, grad_W
+
+    # -- the whole block of Algorithm 1: GELU(W_bypass x + layer(x))
+    def block_forward(self, x, W, W_bypass, out=None, Xhat=None, z=None, save_z=True, stream=None):
+        """Returns (out, Xhat, z); z (the pre-activation, needed by block_backward) is None with save_z=False."""
+        if out is None:
+            out = torch.empty((self.B, self.C_out) + self.N, dtype=torch.float32, device=self.device)
+        if Xhat is None:
+            Xhat = torch.empty((self.B, self.C_in) + self.K, dtype=torch.complex64, device=self.device)
+        if z is None and save_z:
+            z = torch.empty((self.B, self.C_out) + self.N, dtype=torch.float32, device=self.device)
+        for t, kind, name in ((x, "x", "x"), (W, "W", "W"), (W_bypass, "Wb", "W_bypass"), (out, "y", "out"),
+                              (Xhat, "Xhat", "Xhat"), (z, "y", "z")):
+            self._expect(t, kind, name)
+        with torch.cuda.device(self.device):
+            dtst_block_forward(self._h, x, W, W_bypass, out, Xhat, z, stream)
+        return out, Xhat, z
+
+    def block_backward(self, grad_out, x, z, Xhat, W, W_bypass, scratch=None, grad_x=None, grad_W=None,
+                       grad_W_bypass=None, stream=None):
+        """Returns (grad_x, grad_W, grad_W_bypass); `scratch` ([B, C_out, n...]) receives g_z."""
+        dev = self.device
+        if scratch is None:
+            scratch = torch.empty((self.B, self.C_out) + self.N, dtype=torch.float32, device=dev)
+        if grad_x is None:
+            grad_x = torch.empty((self.B, self.C_in) + self.N, dtype=torch.float32, device=dev)
+        if grad_W is None:
+            grad_W = torch.empty((self.C_in, self.C_out, self.M), dtype=torch.complex64, device=dev)
+        if grad_W_bypass is None:
+            grad_W_bypass = torch.empty((self.C_out, self.C_in), dtype=torch.float32, device=dev)
+        for t, kind, name in ((grad_out, "y", "grad_out"), (x, "x", "x"), (z, "y", "z"), (Xhat, "Xhat", "Xhat"),
+                              (W, "W", "W"), (W_bypass, "Wb", "W_bypass"), (scratch, "y", "scratch"),
+                              (grad_x, "x", "grad_x"), (grad_W, "W", "grad_W"), (grad_W_bypass, "Wb", "grad_W_bypass")):
+            self._expect(t, kind, name)
+        with torch.cuda.device(self.device):
+            dtst_block_backward(self._h, grad_out, x, z, Xhat, W, W_bypass, scratch, grad_x, grad_W, grad_W_bypass,
+                                stream)
+        return grad_x, grad_W, grad_W_bypass
 
     # -- the steps one by one (a rank of a slab-sharded layer exchanges spectra between them)
     def spectral_mul_modes(self, Xhat, W_shard, m0, count, out=None, stream=None):

@@ -481,6 +481,9 @@ WsLayout ws_layout(const dtst_plan* p) {
     L.szCounters = p->d >= 3 ? (size_t)2 * cols * sizeof(int) : 0;
   }
   L.counters = o; o += align256(L.szCounters);
+  // per-CTA partial sums of the bypass weight gradient (dtst_block_backward)
+  L.szWbPartial = (size_t)kBlockPartialRows * p->C_in * p->C_out * sizeof(float);
+  L.wb_partial = o; o += align256(L.szWbPartial);
   L.total = o;
   return L;
 }
@@ -703,6 +706,67 @@ dtst_status dtst_backward(dtst_plan* p, const float* grad_y, const void* Xhat_sa
         : use_row(p) ? run_inverse_row(p, GX, grad_x, p->C_in, 1.0f, false, st)
                      : run_inverse_generic(p, GX, grad_x, p->C_in, 1.0f, false, st);
     if (s != DTST_OK) return s;
+  }
+  return DTST_OK;
+}
+
+// ---- the whole block: GELU(W_bypass x + I(M(F(x), W))) and its backward pass
+dtst_status dtst_block_forward(dtst_plan* p, const float* x, const void* W, const float* W_bypass, float* out,
+                               void* Xhat_saved, float* z_saved, void* stream) {
+  dtst_status s = check_ready(p);
+  if (s != DTST_OK) return s;
+  if (x == nullptr || W == nullptr || W_bypass == nullptr || out == nullptr || Xhat_saved == nullptr)
+    return DTST_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(W) || !aligned16(W_bypass) || !aligned16(out) || !aligned16(Xhat_saved) ||
+      !aligned16(z_saved) || out == x || z_saved == x || (z_saved != nullptr && z_saved == out))
+    return DTST_ERR_INVALID_ARG;
+  if (!block_supported(p->C_in, p->C_out, p->points_local)) return DTST_ERR_UNSUPPORTED;
+  const WsLayout L = ws_layout(p);
+  void* Yhat = static_cast<char*>(p->ws) + L.gy;
+  s = dtst_forward(p, x, Xhat_saved, stream);
+  if (s != DTST_OK) return s;
+  s = dtst_spectral_mul(p, Xhat_saved, W, Yhat, stream);
+  if (s != DTST_OK) return s;
+  s = dtst_inverse(p, Yhat, out, stream);          // out holds y; the epilogue turns it into the activation in place
+  if (s != DTST_OK) return s;
+  if (cuda_failed(p, launch_block_epilogue(x, out, z_saved, W_bypass, p->B, p->C_in, p->C_out, p->points_local,
+                                           static_cast<cudaStream_t>(stream))))
+    return DTST_ERR_CUDA;
+  ++p->launches;
+  return DTST_OK;
+}
+
+dtst_status dtst_block_backward(dtst_plan* p, const float* grad_out, const float* x, const float* z_saved,
+                                const void* Xhat_saved, const void* W, const float* W_bypass, float* scratch,
+                                float* grad_x, void* grad_W, float* grad_W_bypass, void* stream) {
+  dtst_status s = check_ready(p);
+  if (s != DTST_OK) return s;
+  if (grad_out == nullptr || x == nullptr || z_saved == nullptr || W == nullptr || W_bypass == nullptr ||
+      scratch == nullptr || (grad_x == nullptr && grad_W == nullptr && grad_W_bypass == nullptr) ||
+      (grad_W != nullptr && Xhat_saved == nullptr))
+    return DTST_ERR_INVALID_ARG;
+  if (!aligned16(grad_out) || !aligned16(x) || !aligned16(z_saved) || !aligned16(Xhat_saved) || !aligned16(W) ||
+      !aligned16(W_bypass) || !aligned16(scratch) || !aligned16(grad_x) || !aligned16(grad_W) ||
+      !aligned16(grad_W_bypass) || scratch == x || scratch == z_saved || scratch == grad_x)
+    return DTST_ERR_INVALID_ARG;
+  if (!block_supported(p->C_in, p->C_out, p->points_local)) return DTST_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const WsLayout L = ws_layout(p);
+  // adjoint of the activation: g_z = grad_out * GELU'(z)
+  if (cuda_failed(p, launch_gelu_backward(grad_out, z_saved, scratch, (long long)p->B * p->C_out * p->points_local, st)))
+    return DTST_ERR_CUDA;
+  ++p->launches;
+  // adjoint of the spectral layer on g_z
+  if (grad_x != nullptr || grad_W != nullptr) {
+    s = dtst_backward(p, scratch, Xhat_saved, W, grad_x, grad_W, stream);
+    if (s != DTST_OK) return s;
+  }
+  // adjoint of the bypass: grad_x += W_bypass^T g_z, grad_W_bypass = sum g_z x^T
+  if (grad_x != nullptr || grad_W_bypass != nullptr) {
+    if (cuda_failed(p, launch_bypass_backward(scratch, x, grad_x, W_bypass, grad_W_bypass,
+                                              reinterpret_cast<float*>(static_cast<char*>(p->ws) + L.wb_partial), p->B,
+                                              p->C_in, p->C_out, p->points_local, st, &p->launches)))
+      return DTST_ERR_CUDA;
   }
   return DTST_OK;
 }

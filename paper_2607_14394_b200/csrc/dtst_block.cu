@@ -1,0 +1,253 @@
+// The rest of the block around the spectral layer (Section "Block Structure", Algorithm 1 lines 1 and 8):
+//     out = GELU(W_bypass x + y),   y = I(M(F(x), W))  the spectral layer's output,
+// and its backward pass.  W_bypass is the point-wise linear operator [C_out][C_in] (no bias), GELU the exact
+// erf form z Phi(z).  Everything here is HBM-bound element-wise work over the grid: one pass that reads x and y
+// and writes the activation (and, for training, the pre-activation), one pass for GELU', and one pass that adds
+// W_bypass^T g_z to grad_x while it reduces grad_W_bypass.
+//
+// Kernels in this file serve any channel count in exact fp32 FFMA; dtst_block_umma.cu holds the tensor-core
+// (tcgen05, accumulator in TMEM) version of the forward pass's bypass product for channel counts it fits.
+#include "dtst_common.cuh"
+
+namespace dtst {
+namespace {
+
+__device__ __forceinline__ float gelu_f(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f)); }
+
+// d GELU / dz = Phi(z) + z phi(z)
+__device__ __forceinline__ float gelu_grad_f(float v) {
+  return 0.5f * (1.0f + erff(v * 0.70710678118654752f)) + v * __expf(-0.5f * v * v) * 0.39894228040143268f;
+}
+
+constexpr int kOC = 4;   // output channels per register tile of the FFMA kernels
+
+// out[b,o,p] = GELU(sum_i Wb[o,i] x[b,i,p] + out[b,o,p]) in place (out holds y on entry); z (optional) gets the
+// pre-activation.  One thread owns four consecutive points and walks the output channels four at a time; the
+// input channels of its points are re-read from L1 for every group of four outputs.
+__global__ void __launch_bounds__(256) block_epilogue_kernel(const float* __restrict__ x, float* __restrict__ out,
+                                                            float* __restrict__ z, const float* __restrict__ Wb,
+                                                            int B, int Ci, int Co, long long P) {
+  pdl_trigger();
+  extern __shared__ float wb_s[];   // [Co][Ci]
+  pdl_wait();
+  for (int e = threadIdx.x; e < Co * Ci; e += blockDim.x) wb_s[e] = Wb[e];
+  __syncthreads();
+  const long long quads = P / 4;
+  const long long total = (long long)B * quads;
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+       t += (long long)gridDim.x * blockDim.x) {
+    const long long b = t / quads, q = t % quads;
+    const float4* xb = reinterpret_cast<const float4*>(x + b * Ci * P) + q;
+    float4* ob = reinterpret_cast<float4*>(out + b * Co * P) + q;
+    float4* zb = z ? reinterpret_cast<float4*>(z + b * Co * P) + q : nullptr;
+    for (int o0 = 0; o0 < Co; o0 += kOC) {
+      float4 acc[kOC];
+#pragma unroll
+      for (int k = 0; k < kOC; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int i = 0; i < Ci; ++i) {
+        const float4 xv = __ldg(xb + (long long)i * quads);
+#pragma unroll
+        for (int k = 0; k < kOC; ++k) {
+          const float w = (o0 + k < Co) ? wb_s[(o0 + k) * Ci + i] : 0.f;
+          acc[k].x = fmaf(w, xv.x, acc[k].x);
+          acc[k].y = fmaf(w, xv.y, acc[k].y);
+          acc[k].z = fmaf(w, xv.z, acc[k].z);
+          acc[k].w = fmaf(w, xv.w, acc[k].w);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < kOC; ++k) {
+        if (o0 + k < Co) {
+          const long long off = (long long)(o0 + k) * quads;
+          const float4 yv = ob[off];
+          const float4 zv = make_float4(acc[k].x + yv.x, acc[k].y + yv.y, acc[k].z + yv.z, acc[k].w + yv.w);
+          if (zb) __stcs(zb + off, zv);
+          __stcs(ob + off, make_float4(gelu_f(zv.x), gelu_f(zv.y), gelu_f(zv.z), gelu_f(zv.w)));
+        }
+      }
+    }
+  }
+}
+
+// g_z = grad_out * GELU'(z), element-wise, 16 bytes per access (gz may alias grad_out)
+__global__ void __launch_bounds__(256) gelu_backward_kernel(const float4* __restrict__ g, const float4* __restrict__ z,
+                                                           float4* gz, long long n4) {
+  pdl_trigger();
+  pdl_wait();
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < n4; t += (long long)gridDim.x * blockDim.x) {
+    const float4 gv = __ldcs(g + t), zv = __ldcs(z + t);
+    gz[t] = make_float4(gv.x * gelu_grad_f(zv.x), gv.y * gelu_grad_f(zv.y), gv.z * gelu_grad_f(zv.z),
+                        gv.w * gelu_grad_f(zv.w));
+  }
+}
+
+// The bypass in the backward pass, one pass over the grid:
+//   grad_x[b,i,p] += sum_o Wb[o,i] g_z[b,o,p]          (added to what the spectral layer's adjoint left there)
+//   partial[cta][o][i] = sum over this CTA's points of g_z[b,o,p] x[b,i,p]
+// A CTA stages tiles of kTP points of g_z (all C_out channels) and x (all C_in channels) in shared memory; every
+// thread owns up to kMaxPairs (o, i) pairs of the weight gradient across all its tiles (fixed order: the sum over
+// a CTA's tiles and then over CTAs is the same on every run) and a group of four input channels times four points
+// of grad_x per tile.
+constexpr int kTP = 128;
+constexpr int kMaxPairs = 16;    // per thread: C_in * C_out <= 256 * 16
+
+__global__ void __launch_bounds__(256) bypass_backward_kernel(const float* __restrict__ gz, const float* __restrict__ x,
+                                                             float* __restrict__ gx, const float* __restrict__ Wb,
+                                                             float* __restrict__ partial, int B, int Ci, int Co,
+                                                             long long P, int want_gx, int want_gw) {
+  pdl_trigger();
+  extern __shared__ float bb_s[];
+  float* wb_s = bb_s;                       // [Co][Ci]
+  float* gz_s = wb_s + ((Co * Ci + 3) & ~3);   // [Co][kTP], 16-byte aligned
+  float* x_s = gz_s + Co * kTP;             // [Ci][kTP]
+  pdl_wait();
+  for (int e = threadIdx.x; e < Co * Ci; e += blockDim.x) wb_s[e] = Wb[e];
+  const int pairs = Co * Ci;
+  float acc[kMaxPairs];
+#pragma unroll
+  for (int k = 0; k < kMaxPairs; ++k) acc[k] = 0.f;
+  const long long tiles_per_b = (P + kTP - 1) / kTP;
+  const long long tiles = (long long)B * tiles_per_b;
+  for (long long t = blockIdx.x; t < tiles; t += gridDim.x) {
+    const long long b = t / tiles_per_b, p0 = (t % tiles_per_b) * kTP;
+    const int np = (int)((P - p0) < kTP ? (P - p0) : kTP);   // a multiple of 4
+    __syncthreads();   // the previous tile has been consumed (and wb_s is complete)
+    for (int e = threadIdx.x; e < (Co + Ci) * (kTP / 4); e += blockDim.x) {
+      const int c = e / (kTP / 4), q = e % (kTP / 4);
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (4 * q < np) {
+        const float* src = c < Co ? gz + (b * Co + c) * P : x + (b * Ci + (c - Co)) * P;
+        v = __ldcs(reinterpret_cast<const float4*>(src + p0) + q);
+      }
+      reinterpret_cast<float4*>(c < Co ? gz_s + c * kTP : x_s + (c - Co) * kTP)[q] = v;
+    }
+    __syncthreads();
+    if (want_gw) {
+#pragma unroll
+      for (int k = 0; k < kMaxPairs; ++k) {
+        const int pr = threadIdx.x + k * 256;
+        if (pr < pairs) {
+          const float4* ga = reinterpret_cast<const float4*>(gz_s + (pr / Ci) * kTP);
+          const float4* xa = reinterpret_cast<const float4*>(x_s + (pr % Ci) * kTP);
+          float s = 0.f;
+          for (int q = 0; q < kTP / 4; ++q) {
+            const float4 a = ga[q], c = xa[q];
+            s = fmaf(a.x, c.x, fmaf(a.y, c.y, fmaf(a.z, c.z, fmaf(a.w, c.w, s))));
+          }
+          acc[k] += s;
+        }
+      }
+    }
+    if (want_gx) {
+      // (group of four input channels, quad of points) per thread, as many rounds as the tile needs
+      const int groups = (Ci + 3) / 4;
+      for (int e = threadIdx.x; e < groups * (kTP / 4); e += blockDim.x) {
+        const int gi = e / (kTP / 4), q = e % (kTP / 4);
+        if (4 * q >= np) continue;
+        float4 a[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) a[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int o = 0; o < Co; ++o) {
+          const float4 gv = reinterpret_cast<const float4*>(gz_s + o * kTP)[q];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float w = (4 * gi + k < Ci) ? wb_s[o * Ci + 4 * gi + k] : 0.f;
+            a[k].x = fmaf(w, gv.x, a[k].x);
+            a[k].y = fmaf(w, gv.y, a[k].y);
+            a[k].z = fmaf(w, gv.z, a[k].z);
+            a[k].w = fmaf(w, gv.w, a[k].w);
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (4 * gi + k < Ci) {
+            float4* dst = reinterpret_cast<float4*>(gx + (b * Ci + 4 * gi + k) * P + p0) + q;
+            const float4 old = *dst;
+            __stcs(dst, make_float4(old.x + a[k].x, old.y + a[k].y, old.z + a[k].z, old.w + a[k].w));
+          }
+        }
+      }
+    }
+  }
+  if (want_gw) {
+#pragma unroll
+    for (int k = 0; k < kMaxPairs; ++k) {
+      const int pr = threadIdx.x + k * 256;
+      if (pr < pairs) partial[(long long)blockIdx.x * pairs + pr] = acc[k];
+    }
+  }
+}
+
+// grad_Wb[pair] = sum over CTAs (ascending) of partial[cta][pair]
+__global__ void __launch_bounds__(256) reduce_wb_kernel(const float* __restrict__ partial, float* __restrict__ gWb,
+                                                       int pairs, int ctas) {
+  pdl_trigger();
+  pdl_wait();
+  const int pr = blockIdx.x * blockDim.x + threadIdx.x;
+  if (pr >= pairs) return;
+  float s = 0.f;
+  for (int c = 0; c < ctas; ++c) s += partial[(long long)c * pairs + pr];
+  gWb[pr] = s;
+}
+
+}  // namespace
+
+bool block_supported(int Ci, int Co, long long P) {
+  return P % 4 == 0 && (long long)Ci * Co <= 256 * kMaxPairs && (size_t)(((Ci * Co + 3) & ~3) + (Ci + Co) * kTP) * 4 <= 200 * 1024;
+}
+
+cudaError_t launch_block_epilogue(const float* x, float* out, float* z, const float* Wb, int B, int Ci, int Co,
+                                  long long P, cudaStream_t st) {
+  const long long total = (long long)B * (P / 4);
+  if (total <= 0) return cudaSuccess;
+  long long blocks = (total + 255) / 256;
+  const long long cap = (long long)num_sms() * 8;
+  if (blocks > cap) blocks = cap;
+  const size_t smem = (size_t)Ci * Co * 4;
+  cudaError_t e = cudaSuccess;
+  if (smem > 48 * 1024) e = cudaFuncSetAttribute(block_epilogue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  (void)launch_pdl(block_epilogue_kernel, dim3((unsigned)blocks), dim3(256), smem, st, x, out, z, Wb, B, Ci, Co, P);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gelu_backward(const float* g, const float* z, float* gz, long long n, cudaStream_t st) {
+  const long long n4 = n / 4;
+  if (n4 <= 0) return cudaSuccess;
+  long long blocks = (n4 + 255) / 256;
+  const long long cap = (long long)num_sms() * 16;
+  if (blocks > cap) blocks = cap;
+  (void)launch_pdl(gelu_backward_kernel, dim3((unsigned)blocks), dim3(256), 0, st, reinterpret_cast<const float4*>(g),
+                   reinterpret_cast<const float4*>(z), reinterpret_cast<float4*>(gz), n4);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_bypass_backward(const float* gz, const float* x, float* gx, const float* Wb, float* gWb,
+                                   float* partial, int B, int Ci, int Co, long long P, cudaStream_t st,
+                                   long long* launches) {
+  const long long tiles = (long long)B * ((P + kTP - 1) / kTP);
+  if (tiles <= 0) return cudaSuccess;
+  const size_t smem = (size_t)(((Ci * Co + 3) & ~3) + (Ci + Co) * kTP) * 4;
+  cudaError_t e = cudaSuccess;
+  if (smem > 48 * 1024) e = cudaFuncSetAttribute(bypass_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  int per_sm = 1;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bypass_backward_kernel, 256, smem);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) per_sm = 1;
+  long long ctas = (long long)num_sms() * per_sm;
+  if (ctas > kBlockPartialRows) ctas = kBlockPartialRows;
+  if (ctas > tiles) ctas = tiles;
+  (void)launch_pdl(bypass_backward_kernel, dim3((unsigned)ctas), dim3(256), smem, st, gz, x, gx, Wb, partial, B, Ci, Co, P,
+                   gx != nullptr ? 1 : 0, gWb != nullptr ? 1 : 0);
+  if (launches) ++*launches;
+  if (gWb != nullptr) {
+    const int pairs = Ci * Co;
+    (void)launch_pdl(reduce_wb_kernel, dim3((unsigned)((pairs + 255) / 256)), dim3(256), 0, st,
+                     static_cast<const float*>(partial), gWb, pairs, (int)ctas);
+    if (launches) ++*launches;
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace dtst

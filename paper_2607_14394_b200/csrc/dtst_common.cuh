@@ -162,9 +162,11 @@ struct RingDebug {
 constexpr uint32_t kDefaultPollLimit = 1u << 24;
 
 struct WsLayout {
-  size_t status, bufA, bufB, partial, gy, gx, counters, total;
-  size_t szA, szB, szPartial, szG, szCounters;
+  size_t status, bufA, bufB, partial, gy, gx, counters, wb_partial, total;
+  size_t szA, szB, szPartial, szG, szCounters, szWbPartial;
 };
+
+constexpr int kBlockPartialRows = 1024;   // most CTAs the bypass weight-gradient reduction is spread over
 
 bool fused_eligible(const dtst_plan* p);
 
@@ -200,6 +202,15 @@ cudaError_t launch_mix_adjoint_modes(const float2* GY, const float2* X, const fl
                                      cudaStream_t st, long long* launches);
 cudaError_t launch_mix_adjoint(const float2* GY, const float2* X, const float2* W, float2* GX, float2* GW,
                                int B, int Ci, int Co, long long M, cudaStream_t st, long long* launches);
+
+// the block around the layer: bypass + GELU and their backward pass (dtst_block.cu)
+bool block_supported(int Ci, int Co, long long P);
+cudaError_t launch_block_epilogue(const float* x, float* out, float* z, const float* Wb, int B, int Ci, int Co,
+                                  long long P, cudaStream_t st);
+cudaError_t launch_gelu_backward(const float* g, const float* z, float* gz, long long n, cudaStream_t st);
+cudaError_t launch_bypass_backward(const float* gz, const float* x, float* gx, const float* Wb, float* gWb,
+                                   float* partial, int B, int Ci, int Co, long long P, cudaStream_t st,
+                                   long long* launches);
 
 // offset / virtual-shard kernels for a two-sided middle dimension (dtst_slab.cu)
 bool slab_supported(int Nl, int K);
