@@ -729,9 +729,16 @@ dtst_status dtst_block_forward(dtst_plan* p, const float* x, const void* W, cons
   if (s != DTST_OK) return s;
   s = dtst_inverse(p, Yhat, out, stream);          // out holds y; the epilogue turns it into the activation in place
   if (s != DTST_OK) return s;
-  if (cuda_failed(p, launch_block_epilogue(x, out, z_saved, W_bypass, p->B, p->C_in, p->C_out, p->points_local,
-                                           static_cast<cudaStream_t>(stream))))
+  // the bypass product on the tensor cores where the channel counts fit an MMA tile, else exact-fp32 FFMA
+  if (p->path_request == DTST_PATH_AUTO && block_umma_supported(p->C_in, p->C_out, p->points_local, p->B)) {
+    if (cuda_failed(p, launch_block_epilogue_umma(x, out, z_saved, W_bypass, p->B, p->C_in, p->C_out, p->points_local,
+                                                  reinterpret_cast<int*>(static_cast<char*>(p->ws) + L.status),
+                                                  static_cast<cudaStream_t>(stream))))
+      return DTST_ERR_CUDA;
+  } else if (cuda_failed(p, launch_block_epilogue(x, out, z_saved, W_bypass, p->B, p->C_in, p->C_out,
+                                                  p->points_local, static_cast<cudaStream_t>(stream)))) {
     return DTST_ERR_CUDA;
+  }
   ++p->launches;
   return DTST_OK;
 }

@@ -51,6 +51,20 @@ bool make_rows_map(CUtensorMap* map, const void* base, long long rows, int n3, i
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool tma_encode_available() { return encode_tiled_fn() != nullptr; }
+
+// fp32 tensor [rows][P] with P contiguous, viewed through [box_rows x 32 floats] boxes with the 128-byte swizzle
+bool make_points_map(CUtensorMap* map, const float* base, long long rows, long long P, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)P, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)P * 4};
+  cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 // Shapes the plane kernels are instantiated for: (N3, k3, N2, k2).
 static bool plane_supported(int N3, int K3, int N2, int K2) {

@@ -27,6 +27,16 @@ cudaError_t launch_inv_plane_colexp(int N3, int K3, int N2, int K2, int N1, int 
 // 2-D fp32 tensor [rows][n3] viewed through [box_rows x 32 floats] boxes with the 128-byte TMA swizzle.
 bool make_rows_map(CUtensorMap* map, const void* base, long long rows, int n3, int box_rows);
 
+// whether the driver's tensor-map encoder could be found (no TMA kernel runs without it)
+bool tma_encode_available();
+// fp32 tensor [rows][P] with P contiguous, viewed through [box_rows x 32 floats] boxes with the 128-byte swizzle
+bool make_points_map(CUtensorMap* map, const float* base, long long rows, long long P, int box_rows);
+
+// Tensor-core version of the block's forward epilogue (dtst_block_umma.cu): C_in in {8, 16, 32}, C_out in {16, 32}
+bool block_umma_supported(int Ci, int Co, long long P, int B);
+cudaError_t launch_block_epilogue_umma(const float* x, float* out, float* z, const float* Wb, int B, int Ci, int Co,
+                                       long long P, int* status, cudaStream_t st);
+
 // Row kernels (dtst_row.cu): the contiguous dimension alone, N3 % 32 == 0, N3 <= 256, k3 <= 16.
 bool row_supported(int N3, int K3);
 cudaError_t launch_row_contract(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm,
