@@ -492,6 +492,91 @@ def virtual_shard_summary(torch, w, x, g, W, P, steps, peak):
         return {"P": P, "error": f"{type(ex).__name__}: {ex}"[:200]}
 
 
+def block_summary(torch, w, x, g, W, steps, peak):
+    """The whole block of Algorithm 1 on the headline workload - GELU(W_bypass x + layer(x)) with the pre-activation
+    kept for training, and its backward pass - timed like the headline (K uninstrumented steps, then K with the
+    library's events around the block's own kernels).  Algorithmic bytes: the layer's, plus one more read of x for
+    the bypass, plus (training) the pre-activation written once and read once, g_z written and read once, x and
+    grad_x read once more for the bypass adjoint."""
+    from paper_2607_14394_b200 import Plan
+    try:
+        dev = x.device
+        plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out)
+        gen = torch.Generator(device=dev).manual_seed(w.seed + 77)
+        Wb = torch.randn((w.C_out, w.C_in), device=dev, generator=gen) / w.C_in ** 0.5
+        out, Xhat, z = plan.block_forward(x, W, Wb)
+        scratch = torch.empty_like(z)
+        gx, gW, gWb = plan.block_backward(g, x, z, Xhat, W, Wb, scratch=scratch)
+
+        def fwd():
+            plan.block_forward(x, W, Wb, out, Xhat, z)
+
+        def bwd():
+            plan.block_backward(g, x, z, Xhat, W, Wb, scratch, gx, gW, gWb)
+
+        for _ in range(3):
+            fwd()
+            bwd()
+        torch.cuda.synchronize()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        for _ in range(steps):
+            fwd()
+        e[1].record()
+        for _ in range(steps):
+            bwd()
+        e[2].record()
+        torch.cuda.synchronize()
+        tf, tb = e[0].elapsed_time(e[1]) / steps, e[1].elapsed_time(e[2]) / steps
+        plan.enable_kernel_timing(steps + 2)
+        for _ in range(steps):
+            fwd()
+            bwd()
+        torch.cuda.synchronize()
+        kt = {k: plan.kernel_timing(k) for k in ("block_epilogue", "gelu_backward", "bypass_backward")}
+        # the forward epilogue once more with each of its two kernels asked for explicitly
+        epi = {}
+        for mode in ("ffma", "tensor"):
+            try:
+                plan.set_block_epilogue(mode)
+                fwd()
+                torch.cuda.synchronize()
+                plan.kernel_timing("block_epilogue")
+                for _ in range(steps):
+                    fwd()
+                n_e, ms_e = plan.kernel_timing("block_epilogue")
+                epi[mode] = ms_e / max(1, n_e)
+            except Exception as ex:
+                epi[mode] = f"{type(ex).__name__}"[:60]
+        plan.set_block_epilogue("auto")
+        plan.enable_kernel_timing(0)
+        ok = plan.status() == 0
+        ab = algorithmic_bytes(w)
+        pts = w.B * w.points
+        gin, gout = 4 * w.C_in * pts, 4 * w.C_out * pts
+        bytes_f = ab["fwd"] + gin + 2 * gout                  # x once more; z written; y/out read-modify-written
+        bytes_b = (ab["fwd_bwd"] - ab["fwd"]) + 3 * gout + gout + gin + 2 * gin   # gelu' pass, bypass adjoint pass
+        kernel_bytes = {"block_epilogue": gin + 3 * gout, "gelu_backward": 3 * gout, "bypass_backward": gout + 3 * gin}
+        res = {"fwd_ms": tf, "fwd_bwd_ms": tf + tb, "status_ok": ok, "steps": steps,
+               "fwd_gpoints_per_s": pts / tf / 1e6, "fwd_bwd_gpoints_per_s": pts / (tf + tb) / 1e6,
+               "bytes_moved_model": {"fwd": bytes_f, "fwd_bwd": bytes_f + bytes_b},
+               "fwd_gbs": bytes_f / tf / 1e6, "fwd_bwd_gbs": (bytes_f + bytes_b) / (tf + tb) / 1e6,
+               "fwd_bwd_frac_of_measured_peak": (bytes_f + bytes_b) / (tf + tb) / 1e6 / peak,
+               "bypass_product": "auto: tcgen05.mma kind::tf32 (3xTF32, accumulator in TMEM) from 32 input channels "
+                                 "on, fp32 FFMA below",
+               "epilogue_kernel_ms": {"ffma": epi.get("ffma"), "tcgen05": epi.get("tensor")},
+               "kernels": {k: {"launches": n, "avg_ms": ms / n, "bytes_per_launch": kernel_bytes[k],
+                               "achieved_gbs": kernel_bytes[k] / (ms / n) / 1e6,
+                               "frac_of_measured_peak": kernel_bytes[k] / (ms / n) / 1e6 / peak}
+                           for k, (n, ms) in kt.items() if n}}
+        plan.close()
+        del plan, out, Xhat, z, scratch, gx, gW, gWb
+        torch.cuda.empty_cache()
+        return res
+    except Exception as ex:
+        return {"error": f"{type(ex).__name__}: {ex}"[:200]}
+
+
 def other_configs_summary(torch, skip_name, steps=10):
     """Forward and forward+backward time of the other benchmark configurations (parity-test cases, not the
     headline): seeded device-generated inputs of each shape, CUDA events, 3 warm-ups."""
@@ -760,6 +845,8 @@ def main_ours(args, w):
                                   "what": "the same step captured once in a CUDA graph and replayed"}
         if not args.no_other_configs and args.channels == 0 and P == 1 and w.virtual_shards > 1:
             line["virtual_shards"] = virtual_shard_summary(torch, w, x, g, W, w.virtual_shards, steps, peak)
+        if not args.no_other_configs:
+            line["block"] = block_summary(torch, w, x, g, W, min(steps, 10), peak)
         if not args.no_torch_ref:
             line["torch_fft_reference"] = torch_fft_reference(torch, w, x, W, g)
         if not args.no_other_configs and args.channels == 0:

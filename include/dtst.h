@@ -202,10 +202,23 @@ dtst_status dtst_backward(dtst_plan* plan, const float* grad_y, const void* Xhat
  *   the backward pass); z_saved [B, C_out, n...] float32, the pre-activation, written when not NULL (pass NULL
  *   for inference).  out and z_saved must not alias x or each other.
  * The mixed spectrum lives in the plan's workspace.  Needs grid points per (b, c) % 4 == 0 (always true, the
- * contiguous extent is a multiple of 4) and C_in * C_out <= 4096, else DTST_ERR_UNSUPPORTED.
+ * contiguous extent is a multiple of 4) and C_in + C_out <= 64, else DTST_ERR_UNSUPPORTED.
  */
 dtst_status dtst_block_forward(dtst_plan* plan, const float* x, const void* W, const float* W_bypass,
                                float* out, void* Xhat_saved, float* z_saved, void* stream);
+
+/*
+ * Which kernel forms the bypass product W_bypass x inside dtst_block_forward:
+ *   DTST_BLOCK_EPILOGUE_FFMA    exact fp32 multiply-adds, any channel count;
+ *   DTST_BLOCK_EPILOGUE_TENSOR  the tensor cores (tcgen05.mma kind::tf32 with the accumulator in tensor memory,
+ *                               three TF32 products per fp32 product): C_in in {8, 16, 32}, C_out in {16, 32},
+ *                               plans on the streaming kernel family; DTST_ERR_UNSUPPORTED otherwise;
+ *   DTST_BLOCK_EPILOGUE_AUTO    (default) the tensor cores from 32 input channels on, where the product stops
+ *                               fitting into the memory time of the FFMA kernel; FFMA below.
+ * Both meet the same tolerance against the float64 statement of the block.
+ */
+enum { DTST_BLOCK_EPILOGUE_AUTO = 0, DTST_BLOCK_EPILOGUE_FFMA = 1, DTST_BLOCK_EPILOGUE_TENSOR = 2 };
+dtst_status dtst_plan_set_block_epilogue(dtst_plan* plan, int mode);
 
 /*
  * Backward pass of the block for upstream gradient grad_out = dL/d out (Section "Backward Pass": the linear
@@ -324,7 +337,10 @@ enum {
   DTST_KERNEL_GRID_WRITE = 1,
   DTST_KERNEL_MIX = 2,
   DTST_KERNEL_MIX_ADJOINT = 3,
-  DTST_KERNEL_KINDS = 4
+  DTST_KERNEL_BLOCK_EPILOGUE = 4,   /* dtst_block_forward: bypass product + add + GELU                 */
+  DTST_KERNEL_GELU_BACKWARD = 5,    /* dtst_block_backward: g_z = grad_out * GELU'(z)                   */
+  DTST_KERNEL_BYPASS_BACKWARD = 6,  /* dtst_block_backward: grad_x += W_bypass^T g_z, grad_W_bypass      */
+  DTST_KERNEL_KINDS = 7
 };
 dtst_status dtst_plan_enable_kernel_timing(dtst_plan* plan, int capacity);
 
@@ -336,6 +352,10 @@ dtst_status dtst_plan_kernel_timing(dtst_plan* plan, int kind, int64_t* launches
  * failing runtime call or launch of this plan (0 / "no error" otherwise).  The string is static. */
 dtst_status dtst_plan_last_cuda_error(const dtst_plan* plan, int* code, const char** text);
 
+/*
+ * Diagnostics read once from the environment (for A/B measurements; not for production use):
+ *   DTST_NO_PDL=1            launch every kernel without the programmatic-dependent-launch attribute
+ */
 const char* dtst_status_string(dtst_status s);
 
 /* Library version as major*10000 + minor*100 + patch. */

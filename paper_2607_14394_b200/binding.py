@@ -39,6 +39,7 @@ EXPORTED = [
     "dtst_version", "dtst_plan_enable_kernel_timing", "dtst_plan_kernel_timing", "dtst_forward_static",
     "dtst_plan_last_cuda_error", "dtst_spectral_mul_modes", "dtst_backward_spectrum", "dtst_backward_mix_modes",
     "dtst_backward_input", "dtst_plan_debug_ring_fault", "dtst_plan_set_column_expansion", "dtst_plan_require_fast_path", "dtst_block_forward", "dtst_block_backward",
+    "dtst_plan_set_block_epilogue",
 ]
 
 
@@ -85,6 +86,7 @@ def lib() -> ctypes.CDLL:
     L.dtst_backward_input.argtypes = [vp, vp, vp, vp]
     L.dtst_plan_set_column_expansion.argtypes = [vp, i32]
     L.dtst_plan_require_fast_path.argtypes = [vp, i32]
+    L.dtst_plan_set_block_epilogue.argtypes = [vp, i32]
     L.dtst_plan_debug_ring_fault.argtypes = [vp, ctypes.c_int64, ctypes.c_uint32]
     L.dtst_plan_status.argtypes = [vp, vp]
     L.dtst_plan_launch_count.argtypes = [vp, i64p]
@@ -169,6 +171,14 @@ def dtst_plan_set_virtual_shards(plan, P) -> None:
 
 def dtst_plan_set_kernel_path(plan, path) -> None:
     _check(lib().dtst_plan_set_kernel_path(plan, int(path)), "dtst_plan_set_kernel_path")
+
+
+BLOCK_EPILOGUE = {"auto": 0, "ffma": 1, "tensor": 2}
+
+
+def dtst_plan_set_block_epilogue(plan, mode) -> None:
+    m = BLOCK_EPILOGUE[mode] if isinstance(mode, str) else int(mode)
+    _check(lib().dtst_plan_set_block_epilogue(plan, m), "dtst_plan_set_block_epilogue")
 
 
 def dtst_plan_require_fast_path(plan, required=True) -> None:
@@ -303,7 +313,8 @@ def dtst_plan_launch_count(plan) -> int:
     return int(v.value)
 
 
-KERNEL_KINDS = {"grid_read": 0, "grid_write": 1, "mix": 2, "mix_adjoint": 3}
+KERNEL_KINDS = {"grid_read": 0, "grid_write": 1, "mix": 2, "mix_adjoint": 3, "block_epilogue": 4,
+                "gelu_backward": 5, "bypass_backward": 6}
 
 
 def dtst_plan_enable_kernel_timing(plan, capacity: int) -> None:
@@ -556,6 +567,10 @@ class Plan:
         Yhat = self.spectral_mul(Xhat, W, Yhat, stream)
         y = self.inverse(Yhat, y, stream)
         return y, Xhat
+
+    def set_block_epilogue(self, mode) -> None:
+        """'auto', 'ffma' or 'tensor': which kernel forms the bypass product of block_forward."""
+        dtst_plan_set_block_epilogue(self._h, mode)
 
     def require_fast_path(self, required: bool = True) -> None:
         """Raises DtstError(DTST_ERR_UNSUPPORTED) if any stage of this plan would run on the slow generic kernel."""

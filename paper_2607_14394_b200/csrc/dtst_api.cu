@@ -518,6 +518,15 @@ dtst_status dtst_plan_set_kernel_path(dtst_plan* p, int path) {
   return DTST_OK;
 }
 
+dtst_status dtst_plan_set_block_epilogue(dtst_plan* p, int mode) {
+  if (p == nullptr || mode < DTST_BLOCK_EPILOGUE_AUTO || mode > DTST_BLOCK_EPILOGUE_TENSOR) return DTST_ERR_INVALID_ARG;
+  if (mode == DTST_BLOCK_EPILOGUE_TENSOR &&
+      (p->path_request != DTST_PATH_AUTO || !block_umma_supported(p->C_in, p->C_out, p->points_local, p->B)))
+    return DTST_ERR_UNSUPPORTED;
+  p->block_epilogue = mode;
+  return DTST_OK;
+}
+
 dtst_status dtst_plan_require_fast_path(dtst_plan* p, int required) {
   if (p == nullptr) return DTST_ERR_INVALID_ARG;
   p->require_fast = 0;
@@ -710,6 +719,17 @@ dtst_status dtst_backward(dtst_plan* p, const float* grad_y, const void* Xhat_sa
   return DTST_OK;
 }
 
+// Which kernel forms the bypass product of dtst_block_forward: the tensor-core one (tcgen05) when asked for, or,
+// left to the library, from 32 input channels on - below that the exact-fp32 FFMA kernel is the faster one
+// (measured at 16 channels on the largest benchmark shape: 7.4 ms against 12.0 ms for 34 GB moved; the product is
+// 16 multiply-adds per output value there, which the FFMA pipe does within the memory time, while the tensor-core
+// kernel's per-tile chain of split, product and epilogue is latency-bound at four CTAs per SM).
+static bool use_block_tensor(const dtst_plan* p) {
+  if (p->path_request != DTST_PATH_AUTO || p->block_epilogue == DTST_BLOCK_EPILOGUE_FFMA) return false;
+  if (!block_umma_supported(p->C_in, p->C_out, p->points_local, p->B)) return false;
+  return p->block_epilogue == DTST_BLOCK_EPILOGUE_TENSOR || p->C_in >= 32;
+}
+
 // ---- the whole block: GELU(W_bypass x + I(M(F(x), W))) and its backward pass
 dtst_status dtst_block_forward(dtst_plan* p, const float* x, const void* W, const float* W_bypass, float* out,
                                void* Xhat_saved, float* z_saved, void* stream) {
@@ -729,8 +749,8 @@ dtst_status dtst_block_forward(dtst_plan* p, const float* x, const void* W, cons
   if (s != DTST_OK) return s;
   s = dtst_inverse(p, Yhat, out, stream);          // out holds y; the epilogue turns it into the activation in place
   if (s != DTST_OK) return s;
-  // the bypass product on the tensor cores where the channel counts fit an MMA tile, else exact-fp32 FFMA
-  if (p->path_request == DTST_PATH_AUTO && block_umma_supported(p->C_in, p->C_out, p->points_local, p->B)) {
+  KernelTimer kt(p, DTST_KERNEL_BLOCK_EPILOGUE, static_cast<cudaStream_t>(stream));
+  if (use_block_tensor(p)) {
     if (cuda_failed(p, launch_block_epilogue_umma(x, out, z_saved, W_bypass, p->B, p->C_in, p->C_out, p->points_local,
                                                   reinterpret_cast<int*>(static_cast<char*>(p->ws) + L.status),
                                                   static_cast<cudaStream_t>(stream))))
@@ -760,8 +780,12 @@ dtst_status dtst_block_backward(dtst_plan* p, const float* grad_out, const float
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const WsLayout L = ws_layout(p);
   // adjoint of the activation: g_z = grad_out * GELU'(z)
-  if (cuda_failed(p, launch_gelu_backward(grad_out, z_saved, scratch, (long long)p->B * p->C_out * p->points_local, st)))
-    return DTST_ERR_CUDA;
+  {
+    KernelTimer kt(p, DTST_KERNEL_GELU_BACKWARD, st);
+    if (cuda_failed(p, launch_gelu_backward(grad_out, z_saved, scratch,
+                                            (long long)p->B * p->C_out * p->points_local, st)))
+      return DTST_ERR_CUDA;
+  }
   ++p->launches;
   // adjoint of the spectral layer on g_z
   if (grad_x != nullptr || grad_W != nullptr) {
@@ -770,6 +794,7 @@ dtst_status dtst_block_backward(dtst_plan* p, const float* grad_out, const float
   }
   // adjoint of the bypass: grad_x += W_bypass^T g_z, grad_W_bypass = sum g_z x^T
   if (grad_x != nullptr || grad_W_bypass != nullptr) {
+    KernelTimer kt(p, DTST_KERNEL_BYPASS_BACKWARD, st);
     if (cuda_failed(p, launch_bypass_backward(scratch, x, grad_x, W_bypass, grad_W_bypass,
                                               reinterpret_cast<float*>(static_cast<char*>(p->ws) + L.wb_partial), p->B,
                                               p->C_in, p->C_out, p->points_local, st, &p->launches)))

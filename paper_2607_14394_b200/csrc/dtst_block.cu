@@ -84,96 +84,139 @@ __global__ void __launch_bounds__(256) gelu_backward_kernel(const float4* __rest
 // The bypass in the backward pass, one pass over the grid:
 //   grad_x[b,i,p] += sum_o Wb[o,i] g_z[b,o,p]          (added to what the spectral layer's adjoint left there)
 //   partial[cta][o][i] = sum over this CTA's points of g_z[b,o,p] x[b,i,p]
-// A CTA stages tiles of kTP points of g_z (all C_out channels) and x (all C_in channels) in shared memory; every
-// thread owns up to kMaxPairs (o, i) pairs of the weight gradient across all its tiles (fixed order: the sum over
-// a CTA's tiles and then over CTAs is the same on every run) and a group of four input channels times four points
-// of grad_x per tile.
+// A CTA stages tiles of kTP points of g_z (all C_out channels) and x (all C_in channels) in shared memory.
+// Weight gradient: the (o, i) pairs are cut into 4 x 4 blocks; a thread owns one block for every npg-th quad of
+// points (npg = 256 / blocks point groups work side by side), so that 8 shared-memory loads of 16 bytes feed 64
+// multiply-adds; its 16 sums live in registers across all tiles of the CTA and are added over the point groups in
+// ascending order at the end - a fixed order, so repeated runs give the same bits.  Input gradient: a thread owns
+// four input channels times four points per round.
 constexpr int kTP = 128;
-constexpr int kMaxPairs = 16;    // per thread: C_in * C_out <= 256 * 16
+constexpr int kTS = kTP + 4;     // row stride of the staged tiles in floats (rows shifted by 16 bytes in the banks)
 
-__global__ void __launch_bounds__(256) bypass_backward_kernel(const float* __restrict__ gz, const float* __restrict__ x,
+__global__ void __launch_bounds__(256, 3) bypass_backward_kernel(const float* __restrict__ gz, const float* __restrict__ x,
                                                              float* __restrict__ gx, const float* __restrict__ Wb,
                                                              float* __restrict__ partial, int B, int Ci, int Co,
                                                              long long P, int want_gx, int want_gw) {
   pdl_trigger();
   extern __shared__ float bb_s[];
   float* wb_s = bb_s;                       // [Co][Ci]
-  float* gz_s = wb_s + ((Co * Ci + 3) & ~3);   // [Co][kTP], 16-byte aligned
-  float* x_s = gz_s + Co * kTP;             // [Ci][kTP]
+  float* gz_s = wb_s + ((Co * Ci + 3) & ~3);   // [Co][kTP], rows kTS apart, 16-byte aligned
+  float* x_s = gz_s + Co * kTS;             // [Ci][kTP], rows kTS apart
   pdl_wait();
   for (int e = threadIdx.x; e < Co * Ci; e += blockDim.x) wb_s[e] = Wb[e];
-  const int pairs = Co * Ci;
-  float acc[kMaxPairs];
+  const int ob_n = (Co + 3) / 4, ib_n = (Ci + 3) / 4;
+  const int blocks = ob_n * ib_n;                       // <= 256 (C_in * C_out <= 4096)
+  const int npg = 256 / blocks;                         // point groups
+  const int pg = threadIdx.x / blocks, blk = threadIdx.x % blocks;
+  const bool gw_thread = want_gw && pg < npg;
+  const int o0 = 4 * (blk / ib_n), i0 = 4 * (blk % ib_n);
+  float acc[4][4];
 #pragma unroll
-  for (int k = 0; k < kMaxPairs; ++k) acc[k] = 0.f;
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) acc[a][c] = 0.f;
   const long long tiles_per_b = (P + kTP - 1) / kTP;
   const long long tiles = (long long)B * tiles_per_b;
+  // Each thread stages up to kLd 16-byte pieces of a tile; the pieces of the NEXT tile are requested before the
+  // current one is worked on, so that their latency hides behind the arithmetic (C_in + C_out <= 8 * kLd).
+  constexpr int kLd = 8;
+  const int pieces = (Co + Ci) * (kTP / 4);
+  float4 nxt[kLd];
+  auto fetch = [&](long long tt) {
+    const long long bb = tt / tiles_per_b, pp0 = (tt % tiles_per_b) * kTP;
+    const int nnp = (int)((P - pp0) < kTP ? (P - pp0) : kTP);
+#pragma unroll
+    for (int k = 0; k < kLd; ++k) {
+      const int e = threadIdx.x + 256 * k;
+      nxt[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (e < pieces) {
+        const int c = e / (kTP / 4), q = e % (kTP / 4);
+        if (4 * q < nnp) {
+          const float* src = c < Co ? gz + (bb * Co + c) * P : x + (bb * Ci + (c - Co)) * P;
+          nxt[k] = __ldcs(reinterpret_cast<const float4*>(src + pp0) + q);
+        }
+      }
+    }
+  };
+  if ((long long)blockIdx.x < tiles) fetch(blockIdx.x);
   for (long long t = blockIdx.x; t < tiles; t += gridDim.x) {
     const long long b = t / tiles_per_b, p0 = (t % tiles_per_b) * kTP;
     const int np = (int)((P - p0) < kTP ? (P - p0) : kTP);   // a multiple of 4
     __syncthreads();   // the previous tile has been consumed (and wb_s is complete)
-    for (int e = threadIdx.x; e < (Co + Ci) * (kTP / 4); e += blockDim.x) {
-      const int c = e / (kTP / 4), q = e % (kTP / 4);
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (4 * q < np) {
-        const float* src = c < Co ? gz + (b * Co + c) * P : x + (b * Ci + (c - Co)) * P;
-        v = __ldcs(reinterpret_cast<const float4*>(src + p0) + q);
+#pragma unroll
+    for (int k = 0; k < kLd; ++k) {
+      const int e = threadIdx.x + 256 * k;
+      if (e < pieces) {
+        const int c = e / (kTP / 4), q = e % (kTP / 4);
+        reinterpret_cast<float4*>(c < Co ? gz_s + c * kTS : x_s + (c - Co) * kTS)[q] = nxt[k];
       }
-      reinterpret_cast<float4*>(c < Co ? gz_s + c * kTP : x_s + (c - Co) * kTP)[q] = v;
     }
     __syncthreads();
-    if (want_gw) {
+    if (t + gridDim.x < tiles) fetch(t + gridDim.x);
+    if (gw_thread) {
+      for (int q = pg; q < kTP / 4; q += npg) {     // quads beyond the end of a ragged tile hold zeros
+        float4 gv[4], xv[4];
 #pragma unroll
-      for (int k = 0; k < kMaxPairs; ++k) {
-        const int pr = threadIdx.x + k * 256;
-        if (pr < pairs) {
-          const float4* ga = reinterpret_cast<const float4*>(gz_s + (pr / Ci) * kTP);
-          const float4* xa = reinterpret_cast<const float4*>(x_s + (pr % Ci) * kTP);
-          float s = 0.f;
-          for (int q = 0; q < kTP / 4; ++q) {
-            const float4 a = ga[q], c = xa[q];
-            s = fmaf(a.x, c.x, fmaf(a.y, c.y, fmaf(a.z, c.z, fmaf(a.w, c.w, s))));
-          }
-          acc[k] += s;
+        for (int a = 0; a < 4; ++a) {
+          gv[a] = (o0 + a < Co) ? reinterpret_cast<const float4*>(gz_s + (o0 + a) * kTS)[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+          xv[a] = (i0 + a < Ci) ? reinterpret_cast<const float4*>(x_s + (i0 + a) * kTS)[q] : make_float4(0.f, 0.f, 0.f, 0.f);
         }
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+            acc[a][c] = fmaf(gv[a].x, xv[c].x, fmaf(gv[a].y, xv[c].y, fmaf(gv[a].z, xv[c].z, fmaf(gv[a].w, xv[c].w, acc[a][c]))));
       }
     }
     if (want_gx) {
-      // (group of four input channels, quad of points) per thread, as many rounds as the tile needs
-      const int groups = (Ci + 3) / 4;
+      // (pair of input channels, quad of points) per thread, as many rounds as the tile needs; what the spectral
+      // layer's adjoint left in grad_x is requested first and added last, so that its latency hides behind the sums
+      const int groups = (Ci + 1) / 2;
       for (int e = threadIdx.x; e < groups * (kTP / 4); e += blockDim.x) {
         const int gi = e / (kTP / 4), q = e % (kTP / 4);
         if (4 * q >= np) continue;
-        float4 a[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) a[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        const int i0g = 2 * gi;
+        const bool two = i0g + 1 < Ci;
+        float4* d0 = reinterpret_cast<float4*>(gx + (b * Ci + i0g) * P + p0) + q;
+        float4* d1 = reinterpret_cast<float4*>(gx + (b * Ci + i0g + (two ? 1 : 0)) * P + p0) + q;
+        const float4 old0 = *d0;
+        const float4 old1 = two ? *d1 : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
         for (int o = 0; o < Co; ++o) {
-          const float4 gv = reinterpret_cast<const float4*>(gz_s + o * kTP)[q];
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const float w = (4 * gi + k < Ci) ? wb_s[o * Ci + 4 * gi + k] : 0.f;
-            a[k].x = fmaf(w, gv.x, a[k].x);
-            a[k].y = fmaf(w, gv.y, a[k].y);
-            a[k].z = fmaf(w, gv.z, a[k].z);
-            a[k].w = fmaf(w, gv.w, a[k].w);
-          }
+          const float4 gv = reinterpret_cast<const float4*>(gz_s + o * kTS)[q];
+          const float w0 = wb_s[o * Ci + i0g], w1 = two ? wb_s[o * Ci + i0g + 1] : 0.f;
+          a0.x = fmaf(w0, gv.x, a0.x);
+          a0.y = fmaf(w0, gv.y, a0.y);
+          a0.z = fmaf(w0, gv.z, a0.z);
+          a0.w = fmaf(w0, gv.w, a0.w);
+          a1.x = fmaf(w1, gv.x, a1.x);
+          a1.y = fmaf(w1, gv.y, a1.y);
+          a1.z = fmaf(w1, gv.z, a1.z);
+          a1.w = fmaf(w1, gv.w, a1.w);
         }
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          if (4 * gi + k < Ci) {
-            float4* dst = reinterpret_cast<float4*>(gx + (b * Ci + 4 * gi + k) * P + p0) + q;
-            const float4 old = *dst;
-            __stcs(dst, make_float4(old.x + a[k].x, old.y + a[k].y, old.z + a[k].z, old.w + a[k].w));
-          }
-        }
+        __stcs(d0, make_float4(old0.x + a0.x, old0.y + a0.y, old0.z + a0.z, old0.w + a0.w));
+        if (two) __stcs(d1, make_float4(old1.x + a1.x, old1.y + a1.y, old1.z + a1.z, old1.w + a1.w));
       }
     }
   }
   if (want_gw) {
+    // add the point groups in ascending order through shared memory (the staged tiles are no longer needed)
+    __syncthreads();
+    float* red = gz_s;                                  // [npg][blocks][16] floats <= 256 * 16
+    if (gw_thread) {
 #pragma unroll
-    for (int k = 0; k < kMaxPairs; ++k) {
-      const int pr = threadIdx.x + k * 256;
-      if (pr < pairs) partial[(long long)blockIdx.x * pairs + pr] = acc[k];
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) red[(pg * blocks + blk) * 16 + 4 * a + c] = acc[a][c];
+    }
+    __syncthreads();
+    const int pairs = Co * Ci;
+    for (int pr = threadIdx.x; pr < pairs; pr += blockDim.x) {
+      const int o = pr / Ci, i = pr % Ci;
+      const int bk = (o / 4) * ib_n + (i / 4), el = 4 * (o % 4) + (i % 4);
+      float s = 0.f;
+      for (int g = 0; g < npg; ++g) s += red[(g * blocks + bk) * 16 + el];
+      partial[(long long)blockIdx.x * pairs + pr] = s;
     }
   }
 }
@@ -193,7 +236,7 @@ __global__ void __launch_bounds__(256) reduce_wb_kernel(const float* __restrict_
 }  // namespace
 
 bool block_supported(int Ci, int Co, long long P) {
-  return P % 4 == 0 && (long long)Ci * Co <= 256 * kMaxPairs && (size_t)(((Ci * Co + 3) & ~3) + (Ci + Co) * kTP) * 4 <= 200 * 1024;
+  return P % 4 == 0 && ((Ci + 3) / 4) * ((Co + 3) / 4) <= 256 && Ci + Co <= 64 && (size_t)(((Ci * Co + 3) & ~3) + (Ci + Co) * kTS) * 4 <= 200 * 1024;
 }
 
 cudaError_t launch_block_epilogue(const float* x, float* out, float* z, const float* Wb, int B, int Ci, int Co,
@@ -227,7 +270,9 @@ cudaError_t launch_bypass_backward(const float* gz, const float* x, float* gx, c
                                    long long* launches) {
   const long long tiles = (long long)B * ((P + kTP - 1) / kTP);
   if (tiles <= 0) return cudaSuccess;
-  const size_t smem = (size_t)(((Ci * Co + 3) & ~3) + (Ci + Co) * kTP) * 4;
+  size_t smem = (size_t)(((Ci * Co + 3) & ~3) + (Ci + Co) * kTS) * 4;
+  const size_t red_bytes = (size_t)(((Ci * Co + 3) & ~3) + 256 * 16) * 4;   // the final reduction's scratch
+  if (smem < red_bytes) smem = red_bytes;
   cudaError_t e = cudaSuccess;
   if (smem > 48 * 1024) e = cudaFuncSetAttribute(bypass_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;

@@ -20,7 +20,7 @@
 // One elected thread issues the TMA loads, one the MMAs; completion travels through mbarriers (tcgen05.commit for
 // the tensor core).  Every wait is bounded: on expiry the kernel raises the plan's status word, drains its loads,
 // frees its tensor memory and returns.  Several CTAs share an SM (about 52 KB of shared memory and 32 TMEM
-// columns each at 16 channels), which is what overlaps one CTA's epilogue with another's loads.
+// columns each at 16 channels), and inside a CTA the A operands and the accumulator are double-buffered, which is what overlaps one CTA's epilogue with another's loads.
 #include <cuda.h>
 
 #include "dtst_common.cuh"
@@ -34,7 +34,7 @@ using namespace sm100;
 namespace {
 
 constexpr int kPts = 128;          // points per tile = MMA M
-constexpr int kStages = 4;         // x tiles in flight per CTA
+constexpr int kStages = 2;         // x tiles in flight per CTA (several CTAs share an SM)
 constexpr int kWorkers = 4;        // worker warps (one per TMEM lane quarter)
 constexpr int kThreads = (2 + kWorkers) * 32;
 
@@ -92,8 +92,8 @@ struct UmmaCfg {
   static constexpr int A_KSTEP_BYTES = kPts * 32;         // [128 points][8 channels] as core matrices
   static constexpr int B_KSTEP_BYTES = CO * 32;           // [CO][8 channels] as core matrices
   static constexpr int B_BYTES = 2 * KS * B_KSTEP_BYTES;  // hi and lo
-  static constexpr int TCOLS = CO < 32 ? 32 : CO;         // TMEM columns (a power of two >= 32)
-  static constexpr size_t SMEM = 1024 + (size_t)(kStages + 2) * TILE_BYTES + B_BYTES + 256;
+  static constexpr int TCOLS = 2 * CO < 32 ? 32 : 2 * CO;  // TMEM columns: two accumulators (a power of two >= 32)
+  static constexpr size_t SMEM = 1024 + (size_t)(kStages + 4) * TILE_BYTES + B_BYTES + 256;
 };
 
 template <int CI, int CO>
@@ -106,15 +106,16 @@ block_epilogue_umma_kernel(const __grid_constant__ CUtensorMap x_map, float* __r
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char* ring = smem;                                         // kStages x tile as TMA delivers it
-  unsigned char* hi_tile = smem + (size_t)kStages * Cfg::TILE_BYTES;  // A operand of the tile being multiplied
-  unsigned char* lo_tile = hi_tile + Cfg::TILE_BYTES;
-  unsigned char* bmat = lo_tile + Cfg::TILE_BYTES;                    // [hi | lo][k-step][core matrices]
+  // the A operands, double-buffered: [buffer][hi | lo]; tile j uses buffer j & 1 (and accumulator j & 1), so that
+  // the split of tile j + 1 overlaps the products and the epilogue of tile j
+  unsigned char* a_tiles = smem + (size_t)kStages * Cfg::TILE_BYTES;
+  unsigned char* bmat = a_tiles + 4 * (size_t)Cfg::TILE_BYTES;         // [hi | lo][k-step][core matrices]
   uint64_t* full = reinterpret_cast<uint64_t*>(bmat + Cfg::B_BYTES);
   uint64_t* empty = full + kStages;
-  uint64_t* lo_ready = empty + kStages;
-  uint64_t* mma_done = lo_ready + 1;
-  uint64_t* tmem_free = mma_done + 1;
-  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tmem_free + 1);
+  uint64_t* lo_ready = empty + kStages;     // [2]
+  uint64_t* mma_done = lo_ready + 2;        // [2]
+  uint64_t* tmem_free = mma_done + 2;       // [2]
+  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(tmem_free + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_s + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -123,9 +124,11 @@ block_epilogue_umma_kernel(const __grid_constant__ CUtensorMap x_map, float* __r
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], kWorkers);
     }
-    mbar_init(lo_ready, kWorkers);
-    mbar_init(mma_done, 1);
-    mbar_init(tmem_free, kWorkers);
+    for (int k = 0; k < 2; ++k) {
+      mbar_init(&lo_ready[k], kWorkers);
+      mbar_init(&mma_done[k], 1);
+      mbar_init(&tmem_free[k], kWorkers);
+    }
     *abort_flag = 0;
     fence_barrier_init();
     prefetch_tensormap(&x_map);
@@ -177,11 +180,16 @@ block_epilogue_umma_kernel(const __grid_constant__ CUtensorMap x_map, float* __r
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc(kPts, CO);
-      const uint32_t b_addr = smem_u32(bmat), hi_addr = smem_u32(hi_tile), lo_addr = smem_u32(lo_tile);
+      const uint32_t b_addr = smem_u32(bmat);
       for (long long j = 0; j < n_local; ++j) {
-        if (!mbar_wait_bounded(lo_ready, (uint32_t)(j & 1), abort_flag, poll_limit)) break;      // split done
-        if (j > 0 && !mbar_wait_bounded(tmem_free, (uint32_t)((j - 1) & 1), abort_flag, poll_limit)) break;
+        const int k2 = (int)(j & 1);
+        const uint32_t ph = (uint32_t)((j >> 1) & 1);
+        if (!mbar_wait_bounded(&lo_ready[k2], ph, abort_flag, poll_limit)) break;                // split done
+        if (j >= 2 && !mbar_wait_bounded(&tmem_free[k2], ph ^ 1u, abort_flag, poll_limit)) break;  // accumulator read
         tc_fence_after();
+        const uint32_t hi_addr = smem_u32(a_tiles + (size_t)(2 * k2) * Cfg::TILE_BYTES);
+        const uint32_t lo_addr = hi_addr + Cfg::TILE_BYTES;
+        const uint32_t d_addr = tmem_base + (uint32_t)(k2 * CO);
 #pragma unroll
         for (int ks = 0; ks < Cfg::KS; ++ks) {
           // K-major, no swizzle: core matrices 128 bytes apart along K, 256 bytes apart along M / N
@@ -189,58 +197,74 @@ block_epilogue_umma_kernel(const __grid_constant__ CUtensorMap x_map, float* __r
           const uint64_t a_lo = smem_desc(lo_addr + ks * Cfg::A_KSTEP_BYTES, 128, 256, kLayoutNone);
           const uint64_t b_hi = smem_desc(b_addr + ks * Cfg::B_KSTEP_BYTES, 128, 256, kLayoutNone);
           const uint64_t b_lo = smem_desc(b_addr + (Cfg::KS + ks) * Cfg::B_KSTEP_BYTES, 128, 256, kLayoutNone);
-          umma_tf32(tmem_base, a_hi, b_hi, idesc, ks > 0 ? 1u : 0u);
-          umma_tf32(tmem_base, a_hi, b_lo, idesc, 1u);
-          umma_tf32(tmem_base, a_lo, b_hi, idesc, 1u);
+          umma_tf32(d_addr, a_hi, b_hi, idesc, ks > 0 ? 1u : 0u);
+          umma_tf32(d_addr, a_hi, b_lo, idesc, 1u);
+          umma_tf32(d_addr, a_lo, b_hi, idesc, 1u);
         }
-        umma_commit(mma_done);     // the accumulator is complete (and the hi / lo tiles may be rewritten)
+        umma_commit(&mma_done[k2]);   // accumulator k2 is complete (and A buffer k2 may be rewritten)
       }
     }
   } else {
-    // ---------------- workers: split the tile, then the epilogue ----------------
-    const int wt = threadIdx.x - 64;                       // 0..127
+    // ---------------- workers: split tile j + 1, then the epilogue of tile j ----------------
     const int quarter = warp & 3;                          // the TMEM lanes this warp may read
     const int pt = quarter * 32 + lane;                    // this thread's point within a tile
-    for (long long j = 0; j < n_local; ++j) {
+    // y of this thread's point of tile j for every output channel (requested long before it is needed)
+    auto load_y = [&](long long j, float (&yv)[CO]) {
       const long long t = first + j * gridDim.x;
-      const int s = (int)(j % kStages);
       const long long b = t / tiles_per_b, p0 = (t % tiles_per_b) * kPts;
       const bool live = p0 + pt < P;
-      // y of this thread's point for every output channel, requested before anything else
-      float yv[CO];
       const float* yb = out + (b * CO) * P + p0 + pt;
 #pragma unroll
       for (int o = 0; o < CO; ++o) yv[o] = live ? yb[(long long)o * P] : 0.f;
+    };
+    // this thread's point of tile j: its channels from the swizzled x tile (channel c of point p sits in panel
+    // p / 32, row c, 16-byte chunk ((p % 32) / 4) ^ (c % 8)), split into hi = tf32 truncation and lo = x - hi, and
+    // written four channels at a time into the K-major core matrices of A buffer j & 1:
+    //   k-step (c / 8): + (p / 8) * 256 + ((c % 8) / 4) * 128 + (p % 8) * 16 bytes
+    auto split = [&](long long j) -> bool {
+      const int s = (int)(j % kStages);
       bool ok = mbar_wait_bounded(&full[s], (uint32_t)((j / kStages) & 1), abort_flag, poll_limit);
       ok = __all_sync(0xffffffffu, ok) != 0;
-      if (!ok) break;
-      // this thread's point: its channels from the swizzled tile (channel c of point p sits in panel p / 32, row c,
-      // 16-byte chunk ((p % 32) / 4) ^ (c % 8)), split into hi = tf32 truncation and lo = x - hi, and written four
-      // channels at a time into the K-major core matrices of the two A operands:
-      //   k-step (c / 8): + (p / 8) * 256 + ((c % 8) / 4) * 128 + (p % 8) * 16 bytes
-      {
-        const unsigned char* srcb = ring + (size_t)s * Cfg::TILE_BYTES + (pt / 32) * Cfg::PANEL_BYTES + (pt % 4) * 4;
-        const int chunk = (pt % 32) / 4;
+      if (!ok) return false;
+      unsigned char* hi_tile = a_tiles + (size_t)(2 * (j & 1)) * Cfg::TILE_BYTES;
+      unsigned char* lo_tile = hi_tile + Cfg::TILE_BYTES;
+      const unsigned char* srcb = ring + (size_t)s * Cfg::TILE_BYTES + (pt / 32) * Cfg::PANEL_BYTES + (pt % 4) * 4;
+      const int chunk = (pt % 32) / 4;
 #pragma unroll
-        for (int c4 = 0; c4 < CI / 4; ++c4) {
-          float v[4], h[4];
+      for (int c4 = 0; c4 < CI / 4; ++c4) {
+        float v[4], h[4];
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const int c = 4 * c4 + k;
-            v[k] = *reinterpret_cast<const float*>(srcb + c * 128 + ((chunk ^ (c & 7)) << 4));
-            h[k] = __uint_as_float(__float_as_uint(v[k]) & 0xffffe000u);
-          }
-          const int off = (c4 / 2) * Cfg::A_KSTEP_BYTES + (pt / 8) * 256 + (c4 % 2) * 128 + (pt % 8) * 16;
-          *reinterpret_cast<float4*>(hi_tile + off) = make_float4(h[0], h[1], h[2], h[3]);
-          *reinterpret_cast<float4*>(lo_tile + off) = make_float4(v[0] - h[0], v[1] - h[1], v[2] - h[2], v[3] - h[3]);
+        for (int k = 0; k < 4; ++k) {
+          const int c = 4 * c4 + k;
+          v[k] = *reinterpret_cast<const float*>(srcb + c * 128 + ((chunk ^ (c & 7)) << 4));
+          h[k] = __uint_as_float(__float_as_uint(v[k]) & 0xffffe000u);
         }
+        const int off = (c4 / 2) * Cfg::A_KSTEP_BYTES + (pt / 8) * 256 + (c4 % 2) * 128 + (pt % 8) * 16;
+        *reinterpret_cast<float4*>(hi_tile + off) = make_float4(h[0], h[1], h[2], h[3]);
+        *reinterpret_cast<float4*>(lo_tile + off) = make_float4(v[0] - h[0], v[1] - h[1], v[2] - h[2], v[3] - h[3]);
       }
+      fence_proxy_async_smem();   // the tensor core reads the A tiles through the async proxy
       __syncwarp();
-      if (lane == 0) mbar_arrive(&empty[s]);   // this warp has read its quarter of the x tile
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(lo_ready);
-      ok = mbar_wait_bounded(mma_done, (uint32_t)(j & 1), abort_flag, poll_limit);
+      if (lane == 0) {
+        mbar_arrive(&empty[s]);            // this warp has read its quarter of the x tile
+        mbar_arrive(&lo_ready[j & 1]);     // and written its quarter of the A tiles
+      }
+      return true;
+    };
+    float y_cur[CO], y_next[CO];
+    bool alive = n_local > 0;
+    if (alive) {
+      load_y(0, y_cur);
+      alive = split(0);
+    }
+    for (long long j = 0; alive && j < n_local; ++j) {
+      if (j + 1 < n_local) {
+        load_y(j + 1, y_next);
+        alive = split(j + 1);
+        if (!alive) break;
+      }
+      const int k2 = (int)(j & 1);
+      bool ok = mbar_wait_bounded(&mma_done[k2], (uint32_t)((j >> 1) & 1), abort_flag, poll_limit);
       ok = __all_sync(0xffffffffu, ok) != 0;
       if (!ok) break;
       tc_fence_after();
@@ -248,23 +272,27 @@ block_epilogue_umma_kernel(const __grid_constant__ CUtensorMap x_map, float* __r
 #pragma unroll
       for (int c0 = 0; c0 < CO; c0 += 16) {
         float part[16];
-        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, part);
+        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(k2 * CO + c0), part);
 #pragma unroll
         for (int i = 0; i < 16; ++i) acc[c0 + i] = part[i];
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tmem_free);   // the next tile's products may overwrite the accumulator
-      if (live) {
+      if (lane == 0) mbar_arrive(&tmem_free[k2]);   // products of tile j + 2 may overwrite this accumulator
+      const long long t = first + j * gridDim.x;
+      const long long b = t / tiles_per_b, p0 = (t % tiles_per_b) * kPts;
+      if (p0 + pt < P) {
         float* ob = out + (b * CO) * P + p0 + pt;
         float* zb = z ? z + (b * CO) * P + p0 + pt : nullptr;
 #pragma unroll
         for (int o = 0; o < CO; ++o) {
-          const float v = acc[o] + yv[o];
+          const float v = acc[o] + y_cur[o];
           if (zb) __stcs(zb + (long long)o * P, v);
           __stcs(ob + (long long)o * P, gelu_f(v));
         }
       }
+#pragma unroll
+      for (int o = 0; o < CO; ++o) y_cur[o] = y_next[o];
     }
   }
 

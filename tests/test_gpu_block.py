@@ -23,11 +23,12 @@ def _bypass_weights(w, seed=5):
     return (rng.standard_normal((w.C_out, w.C_in)) / np.sqrt(w.C_in)).astype(np.float32)
 
 
-def run_block_and_check(w, path="auto", P=1, w_scale=1.0):
+def run_block_and_check(w, path="auto", P=1, w_scale=1.0, epilogue="auto"):
     from paper_2607_14394_b200 import Plan
     x, W, g = I.make_field(w), I.make_weights(w) * np.float32(w_scale), I.make_upstream_grad(w)
     Wb = _bypass_weights(w)
     plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out, virtual_shards=P, path=path)
+    plan.set_block_epilogue(epilogue)
     xd, Wd, Wbd, gd = _dev(x), _dev(W), _dev(Wb), _dev(g)
     out, Xhat, z = plan.block_forward(xd, Wd, Wbd)
     out_nz, _, z_none = plan.block_forward(xd, Wd, Wbd, save_z=False)
@@ -87,6 +88,35 @@ def test_block_edge_shapes(case):
     name, B, Ci, Co, N, k = case
     run_block_and_check(I.custom_workload(name, B, Ci, Co, N, k, field="grf" if len(N) > 1 else "iid", seed=13),
                         w_scale=4.0)
+
+
+TENSOR_CASES = [
+    ("t_16_16", 1, 16, 16, (16, 32, 32), (4, 8, 8)),
+    ("t_8_16_tail", 2, 8, 16, (10, 6, 44), (2, 3, 3)),     # points per channel not a multiple of the 128-point tile
+    ("t_32_32", 1, 32, 32, (8, 16, 32), (2, 4, 8)),
+    ("t_16_32_many_tiles", 1, 16, 32, (64, 64, 32), (4, 8, 8)),   # more tiles than CTAs: the pipelines wrap around
+]
+
+
+@pytest.mark.parametrize("case", TENSOR_CASES, ids=[c[0] for c in TENSOR_CASES])
+def test_block_epilogue_on_the_tensor_cores(case):
+    """The bypass product as tcgen05.mma kind::tf32 with the accumulator in tensor memory, asked for explicitly,
+    against the oracle; and the FFMA epilogue on the same inputs."""
+    name, B, Ci, Co, N, k = case
+    w = I.custom_workload(name, B, Ci, Co, N, k, field="grf", seed=17)
+    run_block_and_check(w, w_scale=4.0, epilogue="tensor")
+    run_block_and_check(w, w_scale=4.0, epilogue="ffma")
+
+
+def test_block_epilogue_choice_is_validated():
+    from paper_2607_14394_b200 import Plan, binding as Bn
+    plan = Plan((8, 16), (2, 4), 1, 3, 5)
+    with pytest.raises(Bn.DtstError) as e:
+        plan.set_block_epilogue("tensor")           # channel counts the MMA tile does not fit
+    assert e.value.status == Bn.DTST_ERR_UNSUPPORTED
+    plan.set_block_epilogue("ffma")
+    with pytest.raises(Bn.DtstError):
+        Bn.dtst_plan_set_block_epilogue(plan.handle, 7)
 
 
 def test_block_with_virtual_shards():
