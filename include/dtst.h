@@ -54,7 +54,7 @@ enum {
   DTST_ERR_STATIC_LIMIT = -7     /* dtst_forward_static: the plan needs more than DTST_STATIC_SCRATCH_BYTES */
 };
 
-#define DTST_MAX_DIMS 4
+#define DTST_MAX_DIMS 6
 
 /* Kernel families selectable with dtst_plan_set_kernel_path. */
 enum {
@@ -236,6 +236,27 @@ dtst_status dtst_plan_set_block_epilogue(dtst_plan* plan, int mode);
 dtst_status dtst_block_backward(dtst_plan* plan, const float* grad_out, const float* x, const float* z_saved,
                                 const void* Xhat_saved, const void* W, const float* W_bypass, float* scratch,
                                 float* grad_x, void* grad_W, float* grad_W_bypass, void* stream);
+
+/*
+ * Point-wise linear layers: the lifting network P and the projection network Q around the blocks of an FNO
+ * (Section "Background and Motivation", Eq. 1: "lifted ... via a pointwise network P ... projected ... via a
+ * pointwise network Q"; taken here as one linear map each, with an optional bias).  No plan is involved.
+ *   out[b,o,p] = sum_i W[o,i] x[b,i,p] + bias[o]
+ *   x [B, C_in, points], out [B, C_out, points] float32 (device, 16-byte aligned, points % 4 == 0, out != x);
+ *   W [C_out, C_in] row-major; bias [C_out] or NULL.
+ * Backward for upstream gradient grad_out [B, C_out, points]:
+ *   grad_x[b,i,p] = sum_o W[o,i] grad_out[b,o,p]   (assigned)
+ *   grad_W[o,i]   = sum_{b,p} grad_out[b,o,p] x[b,i,p],   grad_bias[o] = sum_{b,p} grad_out[b,o,p]
+ * any of the three may be NULL (not all).  The two sums over points run in a fixed order through `scratch`
+ * (device, dtst_pointwise_linear_scratch_bytes; DTST_ERR_WORKSPACE if missing or too small): same bits on every
+ * run.  Needs C_in + C_out <= 64 for the backward pass, else DTST_ERR_UNSUPPORTED.
+ */
+dtst_status dtst_pointwise_linear(int B, int C_in, int C_out, int64_t points, const float* x, const float* W,
+                                  const float* bias, float* out, void* stream);
+dtst_status dtst_pointwise_linear_scratch_bytes(int C_in, int C_out, size_t* bytes);
+dtst_status dtst_pointwise_linear_backward(int B, int C_in, int C_out, int64_t points, const float* grad_out,
+                                           const float* x, const float* W, float* grad_x, float* grad_W,
+                                           float* grad_bias, void* scratch, size_t scratch_bytes, void* stream);
 
 /*
  * The same steps one by one, for a caller that runs the layer across several ranks (Algorithm 1: each

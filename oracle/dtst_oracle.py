@@ -310,6 +310,52 @@ def block_backward(grad_out: np.ndarray, x: np.ndarray, z: np.ndarray, Xhat: np.
 
 
 # --------------------------------------------------------------------------
+# A whole Fourier neural operator (Section "Background and Motivation": the input is lifted to d_v channels by a
+# point-wise network P, passed through L Fourier layers (Eq. 1) and projected back by a point-wise network Q).
+# P and Q are taken as one linear map with bias each; every Fourier layer is the block above, activation included.
+# params = {"P_w": [d_v, C_a], "P_b": [d_v], "blocks": [(W_l [d_v, d_v, M] complex, Wb_l [d_v, d_v]), ...],
+#           "Q_w": [C_u, d_v], "Q_b": [C_u]}
+# --------------------------------------------------------------------------
+def pointwise_linear(x: np.ndarray, W: np.ndarray, b=None) -> np.ndarray:
+    y = bypass(x, W)
+    if b is not None:
+        y = y + np.asarray(b, dtype=np.float64).reshape((1, -1) + (1,) * (x.ndim - 2))
+    return y
+
+
+def fno_forward(a: np.ndarray, params: dict, kmax):
+    """Returns (u, saved): u = Q(block_L(... block_1(P(a)))), saved = what fno_backward needs."""
+    v = pointwise_linear(a, params["P_w"], params["P_b"])
+    saved = {"a": np.asarray(a, dtype=np.float64), "v": [], "z": [], "Xhat": []}
+    for (W, Wb) in params["blocks"]:
+        out, z, Xhat = block_forward(v, W, Wb, kmax)
+        saved["v"].append(v)
+        saved["z"].append(z)
+        saved["Xhat"].append(Xhat)
+        v = out
+    saved["v_last"] = v
+    return pointwise_linear(v, params["Q_w"], params["Q_b"]), saved
+
+
+def fno_backward(grad_u: np.ndarray, params: dict, saved: dict, kmax) -> dict:
+    """Gradients of L = sum(u * grad_u) w.r.t. every parameter (and the input a)."""
+    g = np.asarray(grad_u, dtype=np.float64)
+    B = g.shape[0]
+    flat = lambda t: t.reshape(B, t.shape[1], -1)
+    grads = {"Q_w": np.einsum("bon,bin->oi", flat(g), flat(saved["v_last"])), "Q_b": flat(g).sum(axis=(0, 2)),
+             "blocks": [None] * len(params["blocks"])}
+    g = bypass(g, np.asarray(params["Q_w"]).T)
+    for l in reversed(range(len(params["blocks"]))):
+        W, Wb = params["blocks"][l]
+        g, gW, gWb = block_backward(g, saved["v"][l], saved["z"][l], saved["Xhat"][l], W, Wb, kmax)
+        grads["blocks"][l] = (gW, gWb)
+    grads["P_w"] = np.einsum("bon,bin->oi", flat(g), flat(saved["a"]))
+    grads["P_b"] = flat(g).sum(axis=(0, 2))
+    grads["a"] = bypass(g, np.asarray(params["P_w"]).T)
+    return grads
+
+
+# --------------------------------------------------------------------------
 # Flop model of the per-dimension gemm pipeline (Table 2)
 # --------------------------------------------------------------------------
 def gemm_flops_per_stage(shape, order, K, channels: int):

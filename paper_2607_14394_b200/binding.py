@@ -39,7 +39,8 @@ EXPORTED = [
     "dtst_version", "dtst_plan_enable_kernel_timing", "dtst_plan_kernel_timing", "dtst_forward_static",
     "dtst_plan_last_cuda_error", "dtst_spectral_mul_modes", "dtst_backward_spectrum", "dtst_backward_mix_modes",
     "dtst_backward_input", "dtst_plan_debug_ring_fault", "dtst_plan_set_column_expansion", "dtst_plan_require_fast_path", "dtst_block_forward", "dtst_block_backward",
-    "dtst_plan_set_block_epilogue",
+    "dtst_plan_set_block_epilogue", "dtst_pointwise_linear", "dtst_pointwise_linear_scratch_bytes",
+    "dtst_pointwise_linear_backward",
 ]
 
 
@@ -80,6 +81,10 @@ def lib() -> ctypes.CDLL:
     L.dtst_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.dtst_block_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     L.dtst_block_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.dtst_pointwise_linear.argtypes = [i32, i32, i32, ctypes.c_int64, vp, vp, vp, vp, vp]
+    L.dtst_pointwise_linear_scratch_bytes.argtypes = [i32, i32, ctypes.POINTER(ctypes.c_size_t)]
+    L.dtst_pointwise_linear_backward.argtypes = [i32, i32, i32, ctypes.c_int64, vp, vp, vp, vp, vp, vp, vp,
+                                                 ctypes.c_size_t, vp]
     L.dtst_spectral_mul_modes.argtypes = [vp, vp, vp, vp, ctypes.c_int64, ctypes.c_int64, vp]
     L.dtst_backward_spectrum.argtypes = [vp, vp, vp, vp]
     L.dtst_backward_mix_modes.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_int64, ctypes.c_int64, vp]
@@ -270,6 +275,43 @@ def dtst_block_backward(plan, grad_out, x, z_saved, Xhat_saved, W, W_bypass, scr
                                      _ptr(grad_x, torch.float32, "grad_x"), _ptr(grad_W, torch.complex64, "grad_W"),
                                      _ptr(grad_W_bypass, torch.float32, "grad_W_bypass"), _stream_ptr(stream)),
            "dtst_block_backward", plan)
+
+
+def dtst_pointwise_linear(x, W, bias, out, stream=None) -> None:
+    """out[b, o, ...] = sum_i W[o, i] x[b, i, ...] + bias[o]; x [B, C_in, ...], out [B, C_out, ...]."""
+    B, Ci = x.shape[0], x.shape[1]
+    Co = W.shape[0]
+    P = x[0, 0].numel()
+    if W.shape != (Co, Ci) or out.shape[0] != B or out.shape[1] != Co or out[0, 0].numel() != P or \
+            (bias is not None and bias.numel() != Co):
+        raise ValueError("pointwise linear: shapes do not fit")
+    with torch.cuda.device(x.device):
+        _check(lib().dtst_pointwise_linear(B, Ci, Co, P, _ptr(x, torch.float32, "x"), _ptr(W, torch.float32, "W"),
+                                           _ptr(bias, torch.float32, "bias"), _ptr(out, torch.float32, "out"),
+                                           _stream_ptr(stream)), "dtst_pointwise_linear")
+
+
+def dtst_pointwise_linear_scratch_bytes(C_in, C_out) -> int:
+    v = ctypes.c_size_t(0)
+    _check(lib().dtst_pointwise_linear_scratch_bytes(int(C_in), int(C_out), ctypes.byref(v)),
+           "dtst_pointwise_linear_scratch_bytes")
+    return int(v.value)
+
+
+def dtst_pointwise_linear_backward(grad_out, x, W, grad_x, grad_W, grad_bias, scratch, stream=None) -> None:
+    B, Ci = x.shape[0], x.shape[1]
+    Co = W.shape[0]
+    P = x[0, 0].numel()
+    if W.shape != (Co, Ci) or grad_out.shape[0] != B or grad_out.shape[1] != Co or grad_out[0, 0].numel() != P or \
+            (grad_x is not None and grad_x.shape != x.shape) or (grad_W is not None and grad_W.shape != W.shape) or \
+            (grad_bias is not None and grad_bias.numel() != Co):
+        raise ValueError("pointwise linear backward: shapes do not fit")
+    with torch.cuda.device(x.device):
+        _check(lib().dtst_pointwise_linear_backward(
+            B, Ci, Co, P, _ptr(grad_out, torch.float32, "grad_out"), _ptr(x, torch.float32, "x"),
+            _ptr(W, torch.float32, "W"), _ptr(grad_x, torch.float32, "grad_x"), _ptr(grad_W, torch.float32, "grad_W"),
+            _ptr(grad_bias, torch.float32, "grad_bias"), _ptr(scratch, torch.uint8, "scratch"),
+            0 if scratch is None else scratch.numel(), _stream_ptr(stream)), "dtst_pointwise_linear_backward")
 
 
 def dtst_spectral_mul_modes(plan, Xhat, W_shard, Yhat_chunk, m0, count, stream=None) -> None:

@@ -482,7 +482,7 @@ WsLayout ws_layout(const dtst_plan* p) {
   }
   L.counters = o; o += align256(L.szCounters);
   // per-CTA partial sums of the bypass weight gradient (dtst_block_backward)
-  L.szWbPartial = (size_t)kBlockPartialRows * p->C_in * p->C_out * sizeof(float);
+  L.szWbPartial = (size_t)kBlockPartialRows * ((size_t)p->C_in * p->C_out + p->C_out) * sizeof(float);
   L.wb_partial = o; o += align256(L.szWbPartial);
   L.total = o;
   return L;
@@ -799,6 +799,49 @@ dtst_status dtst_block_backward(dtst_plan* p, const float* grad_out, const float
                                               reinterpret_cast<float*>(static_cast<char*>(p->ws) + L.wb_partial), p->B,
                                               p->C_in, p->C_out, p->points_local, st, &p->launches)))
       return DTST_ERR_CUDA;
+  }
+  return DTST_OK;
+}
+
+// ---- point-wise linear layers (the lifting and projection layers around the blocks of an FNO)
+dtst_status dtst_pointwise_linear(int B, int C_in, int C_out, int64_t points, const float* x, const float* W,
+                                  const float* bias, float* out, void* stream) {
+  if (B < 1 || C_in < 1 || C_out < 1 || points < 4 || points % 4 != 0 || x == nullptr || W == nullptr ||
+      out == nullptr || out == x || !aligned16(x) || !aligned16(out) || !aligned16(W) ||
+      (reinterpret_cast<uintptr_t>(bias) & 3u) != 0)
+    return DTST_ERR_INVALID_ARG;
+  if ((size_t)C_in * C_out * 4 > 200 * 1024) return DTST_ERR_UNSUPPORTED;
+  if (launch_pointwise_linear(x, out, bias, W, B, C_in, C_out, points, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return DTST_ERR_CUDA;
+  }
+  return DTST_OK;
+}
+
+dtst_status dtst_pointwise_linear_scratch_bytes(int C_in, int C_out, size_t* bytes) {
+  if (C_in < 1 || C_out < 1 || bytes == nullptr) return DTST_ERR_INVALID_ARG;
+  *bytes = align256((size_t)kBlockPartialRows * ((size_t)C_in * C_out + C_out) * sizeof(float));
+  return DTST_OK;
+}
+
+dtst_status dtst_pointwise_linear_backward(int B, int C_in, int C_out, int64_t points, const float* grad_out,
+                                           const float* x, const float* W, float* grad_x, float* grad_W,
+                                           float* grad_bias, void* scratch, size_t scratch_bytes, void* stream) {
+  if (B < 1 || C_in < 1 || C_out < 1 || points < 4 || points % 4 != 0 || grad_out == nullptr || x == nullptr ||
+      W == nullptr || (grad_x == nullptr && grad_W == nullptr && grad_bias == nullptr) || grad_x == grad_out ||
+      grad_x == x)
+    return DTST_ERR_INVALID_ARG;
+  if (!aligned16(grad_out) || !aligned16(x) || !aligned16(W) || !aligned16(grad_x) || !aligned16(grad_W) ||
+      (reinterpret_cast<uintptr_t>(grad_bias) & 3u) != 0 || !aligned16(scratch))
+    return DTST_ERR_INVALID_ARG;
+  if (!block_supported(C_in, C_out, points)) return DTST_ERR_UNSUPPORTED;
+  size_t need = 0;
+  dtst_pointwise_linear_scratch_bytes(C_in, C_out, &need);
+  if ((grad_W != nullptr || grad_bias != nullptr) && (scratch == nullptr || scratch_bytes < need)) return DTST_ERR_WORKSPACE;
+  if (launch_linear_backward(grad_out, x, grad_x, 2, W, grad_W, grad_bias, static_cast<float*>(scratch), B, C_in, C_out,
+                             points, static_cast<cudaStream_t>(stream), nullptr) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return DTST_ERR_CUDA;
   }
   return DTST_OK;
 }

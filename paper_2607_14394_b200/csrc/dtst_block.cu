@@ -24,6 +24,9 @@ constexpr int kOC = 4;   // output channels per register tile of the FFMA kernel
 // out[b,o,p] = GELU(sum_i Wb[o,i] x[b,i,p] + out[b,o,p]) in place (out holds y on entry); z (optional) gets the
 // pre-activation.  One thread owns four consecutive points and walks the output channels four at a time; the
 // input channels of its points are re-read from L1 for every group of four outputs.
+// With LINEAR the same loop is a plain point-wise linear layer (the lifting and projection layers of an FNO):
+// out[b,o,p] = sum_i Wb[o,i] x[b,i,p] + bias[o], `z` then carries the bias (or NULL) and out is write-only.
+template <bool LINEAR>
 __global__ void __launch_bounds__(256) block_epilogue_kernel(const float* __restrict__ x, float* __restrict__ out,
                                                             float* __restrict__ z, const float* __restrict__ Wb,
                                                             int B, int Ci, int Co, long long P) {
@@ -39,7 +42,7 @@ __global__ void __launch_bounds__(256) block_epilogue_kernel(const float* __rest
     const long long b = t / quads, q = t % quads;
     const float4* xb = reinterpret_cast<const float4*>(x + b * Ci * P) + q;
     float4* ob = reinterpret_cast<float4*>(out + b * Co * P) + q;
-    float4* zb = z ? reinterpret_cast<float4*>(z + b * Co * P) + q : nullptr;
+    float4* zb = (!LINEAR && z) ? reinterpret_cast<float4*>(z + b * Co * P) + q : nullptr;
     for (int o0 = 0; o0 < Co; o0 += kOC) {
       float4 acc[kOC];
 #pragma unroll
@@ -59,10 +62,15 @@ __global__ void __launch_bounds__(256) block_epilogue_kernel(const float* __rest
       for (int k = 0; k < kOC; ++k) {
         if (o0 + k < Co) {
           const long long off = (long long)(o0 + k) * quads;
-          const float4 yv = ob[off];
-          const float4 zv = make_float4(acc[k].x + yv.x, acc[k].y + yv.y, acc[k].z + yv.z, acc[k].w + yv.w);
-          if (zb) __stcs(zb + off, zv);
-          __stcs(ob + off, make_float4(gelu_f(zv.x), gelu_f(zv.y), gelu_f(zv.z), gelu_f(zv.w)));
+          if constexpr (LINEAR) {
+            const float bo = z ? z[o0 + k] : 0.f;
+            ob[off] = make_float4(acc[k].x + bo, acc[k].y + bo, acc[k].z + bo, acc[k].w + bo);
+          } else {
+            const float4 yv = ob[off];
+            const float4 zv = make_float4(acc[k].x + yv.x, acc[k].y + yv.y, acc[k].z + yv.z, acc[k].w + yv.w);
+            if (zb) __stcs(zb + off, zv);
+            __stcs(ob + off, make_float4(gelu_f(zv.x), gelu_f(zv.y), gelu_f(zv.z), gelu_f(zv.w)));
+          }
         }
       }
     }
@@ -96,7 +104,7 @@ constexpr int kTS = kTP + 4;     // row stride of the staged tiles in floats (ro
 __global__ void __launch_bounds__(256, 3) bypass_backward_kernel(const float* __restrict__ gz, const float* __restrict__ x,
                                                              float* __restrict__ gx, const float* __restrict__ Wb,
                                                              float* __restrict__ partial, int B, int Ci, int Co,
-                                                             long long P, int want_gx, int want_gw) {
+                                                             long long P, int want_gx, int want_gw, int want_gb) {
   pdl_trigger();
   extern __shared__ float bb_s[];
   float* wb_s = bb_s;                       // [Co][Ci]
@@ -115,6 +123,7 @@ __global__ void __launch_bounds__(256, 3) bypass_backward_kernel(const float* __
   for (int a = 0; a < 4; ++a)
 #pragma unroll
     for (int c = 0; c < 4; ++c) acc[a][c] = 0.f;
+  float bsum[4] = {0.f, 0.f, 0.f, 0.f};   // sum over points of g_z (the gradient of a bias), on the threads with i0 == 0
   const long long tiles_per_b = (P + kTP - 1) / kTP;
   const long long tiles = (long long)B * tiles_per_b;
   // Each thread stages up to kLd 16-byte pieces of a tile; the pieces of the NEXT tile are requested before the
@@ -166,6 +175,10 @@ __global__ void __launch_bounds__(256, 3) bypass_backward_kernel(const float* __
 #pragma unroll
           for (int c = 0; c < 4; ++c)
             acc[a][c] = fmaf(gv[a].x, xv[c].x, fmaf(gv[a].y, xv[c].y, fmaf(gv[a].z, xv[c].z, fmaf(gv[a].w, xv[c].w, acc[a][c]))));
+        if (want_gb && i0 == 0) {
+#pragma unroll
+          for (int a = 0; a < 4; ++a) bsum[a] += (gv[a].x + gv[a].y) + (gv[a].z + gv[a].w);
+        }
       }
     }
     if (want_gx) {
@@ -179,8 +192,9 @@ __global__ void __launch_bounds__(256, 3) bypass_backward_kernel(const float* __
         const bool two = i0g + 1 < Ci;
         float4* d0 = reinterpret_cast<float4*>(gx + (b * Ci + i0g) * P + p0) + q;
         float4* d1 = reinterpret_cast<float4*>(gx + (b * Ci + i0g + (two ? 1 : 0)) * P + p0) + q;
-        const float4 old0 = *d0;
-        const float4 old1 = two ? *d1 : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 old0 = want_gx == 1 ? *d0 : zero4;          // 1: add to what is there, 2: assign
+        const float4 old1 = (two && want_gx == 1) ? *d1 : zero4;
         float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
         for (int o = 0; o < Co; ++o) {
           const float4 gv = reinterpret_cast<const float4*>(gz_s + o * kTS)[q];
@@ -216,21 +230,40 @@ __global__ void __launch_bounds__(256, 3) bypass_backward_kernel(const float* __
       const int bk = (o / 4) * ib_n + (i / 4), el = 4 * (o % 4) + (i % 4);
       float s = 0.f;
       for (int g = 0; g < npg; ++g) s += red[(g * blocks + bk) * 16 + el];
-      partial[(long long)blockIdx.x * pairs + pr] = s;
+      partial[(long long)blockIdx.x * (pairs + Co) + pr] = s;
+    }
+    if (want_gb) {
+      __syncthreads();
+      if (gw_thread && i0 == 0) {
+#pragma unroll
+        for (int a = 0; a < 4; ++a) red[pg * 4 * ob_n + (o0 + a)] = bsum[a];
+      }
+      __syncthreads();
+      for (int o = threadIdx.x; o < Co; o += blockDim.x) {
+        float s = 0.f;
+        for (int g = 0; g < npg; ++g) s += red[g * 4 * ob_n + o];
+        partial[(long long)blockIdx.x * (pairs + Co) + pairs + o] = s;
+      }
     }
   }
 }
 
 // grad_Wb[pair] = sum over CTAs (ascending) of partial[cta][pair]
+// (entries [pairs, pairs + n_bias) of a row are the bias gradient)
 __global__ void __launch_bounds__(256) reduce_wb_kernel(const float* __restrict__ partial, float* __restrict__ gWb,
-                                                       int pairs, int ctas) {
+                                                       float* __restrict__ gb, int pairs, int n_bias, int ctas) {
   pdl_trigger();
   pdl_wait();
   const int pr = blockIdx.x * blockDim.x + threadIdx.x;
-  if (pr >= pairs) return;
+  const int row = pairs + n_bias;
+  if (pr >= row) return;
   float s = 0.f;
-  for (int c = 0; c < ctas; ++c) s += partial[(long long)c * pairs + pr];
-  gWb[pr] = s;
+  for (int c = 0; c < ctas; ++c) s += partial[(long long)c * row + pr];
+  if (pr < pairs) {
+    if (gWb) gWb[pr] = s;
+  } else if (gb) {
+    gb[pr - pairs] = s;
+  }
 }
 
 }  // namespace
@@ -239,8 +272,8 @@ bool block_supported(int Ci, int Co, long long P) {
   return P % 4 == 0 && ((Ci + 3) / 4) * ((Co + 3) / 4) <= 256 && Ci + Co <= 64 && (size_t)(((Ci * Co + 3) & ~3) + (Ci + Co) * kTS) * 4 <= 200 * 1024;
 }
 
-cudaError_t launch_block_epilogue(const float* x, float* out, float* z, const float* Wb, int B, int Ci, int Co,
-                                  long long P, cudaStream_t st) {
+static cudaError_t launch_epilogue_any(bool linear, const float* x, float* out, float* z, const float* Wb, int B, int Ci,
+                                       int Co, long long P, cudaStream_t st) {
   const long long total = (long long)B * (P / 4);
   if (total <= 0) return cudaSuccess;
   long long blocks = (total + 255) / 256;
@@ -248,10 +281,21 @@ cudaError_t launch_block_epilogue(const float* x, float* out, float* z, const fl
   if (blocks > cap) blocks = cap;
   const size_t smem = (size_t)Ci * Co * 4;
   cudaError_t e = cudaSuccess;
-  if (smem > 48 * 1024) e = cudaFuncSetAttribute(block_epilogue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  auto kern = linear ? block_epilogue_kernel<true> : block_epilogue_kernel<false>;
+  if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  (void)launch_pdl(block_epilogue_kernel, dim3((unsigned)blocks), dim3(256), smem, st, x, out, z, Wb, B, Ci, Co, P);
+  (void)launch_pdl(kern, dim3((unsigned)blocks), dim3(256), smem, st, x, out, z, Wb, B, Ci, Co, P);
   return cudaGetLastError();
+}
+
+cudaError_t launch_block_epilogue(const float* x, float* out, float* z, const float* Wb, int B, int Ci, int Co,
+                                  long long P, cudaStream_t st) {
+  return launch_epilogue_any(false, x, out, z, Wb, B, Ci, Co, P, st);
+}
+
+cudaError_t launch_pointwise_linear(const float* x, float* out, const float* bias, const float* W, int B, int Ci,
+                                    int Co, long long P, cudaStream_t st) {
+  return launch_epilogue_any(true, x, out, const_cast<float*>(bias), W, B, Ci, Co, P, st);
 }
 
 cudaError_t launch_gelu_backward(const float* g, const float* z, float* gz, long long n, cudaStream_t st) {
@@ -265,8 +309,10 @@ cudaError_t launch_gelu_backward(const float* g, const float* z, float* gz, long
   return cudaGetLastError();
 }
 
-cudaError_t launch_bypass_backward(const float* gz, const float* x, float* gx, const float* Wb, float* gWb,
-                                   float* partial, int B, int Ci, int Co, long long P, cudaStream_t st,
+// mode_gx: 0 = no input gradient, 1 = add it to gx, 2 = assign it.  gb (optional): the sum of gz over batch and points
+// per output channel.  `partial` holds kBlockPartialRows rows of C_in * C_out + C_out floats.
+cudaError_t launch_linear_backward(const float* gz, const float* x, float* gx, int mode_gx, const float* Wb, float* gWb,
+                                   float* gb, float* partial, int B, int Ci, int Co, long long P, cudaStream_t st,
                                    long long* launches) {
   const long long tiles = (long long)B * ((P + kTP - 1) / kTP);
   if (tiles <= 0) return cudaSuccess;
@@ -283,16 +329,23 @@ cudaError_t launch_bypass_backward(const float* gz, const float* x, float* gx, c
   long long ctas = (long long)num_sms() * per_sm;
   if (ctas > kBlockPartialRows) ctas = kBlockPartialRows;
   if (ctas > tiles) ctas = tiles;
+  const int want_gw = (gWb != nullptr || gb != nullptr) ? 1 : 0;
   (void)launch_pdl(bypass_backward_kernel, dim3((unsigned)ctas), dim3(256), smem, st, gz, x, gx, Wb, partial, B, Ci, Co, P,
-                   gx != nullptr ? 1 : 0, gWb != nullptr ? 1 : 0);
+                   gx != nullptr ? mode_gx : 0, want_gw, gb != nullptr ? 1 : 0);
   if (launches) ++*launches;
-  if (gWb != nullptr) {
+  if (want_gw) {
     const int pairs = Ci * Co;
-    (void)launch_pdl(reduce_wb_kernel, dim3((unsigned)((pairs + 255) / 256)), dim3(256), 0, st,
-                     static_cast<const float*>(partial), gWb, pairs, (int)ctas);
+    (void)launch_pdl(reduce_wb_kernel, dim3((unsigned)((pairs + Co + 255) / 256)), dim3(256), 0, st,
+                     static_cast<const float*>(partial), gWb, gb, pairs, Co, (int)ctas);
     if (launches) ++*launches;
   }
   return cudaGetLastError();
+}
+
+cudaError_t launch_bypass_backward(const float* gz, const float* x, float* gx, const float* Wb, float* gWb,
+                                   float* partial, int B, int Ci, int Co, long long P, cudaStream_t st,
+                                   long long* launches) {
+  return launch_linear_backward(gz, x, gx, 1, Wb, gWb, nullptr, partial, B, Ci, Co, P, st, launches);
 }
 
 }  // namespace dtst

@@ -208,6 +208,11 @@ cudaError_t launch_mix_adjoint(const float2* GY, const float2* X, const float2* 
 bool block_supported(int Ci, int Co, long long P);
 cudaError_t launch_block_epilogue(const float* x, float* out, float* z, const float* Wb, int B, int Ci, int Co,
                                   long long P, cudaStream_t st);
+cudaError_t launch_pointwise_linear(const float* x, float* out, const float* bias, const float* W, int B, int Ci,
+                                    int Co, long long P, cudaStream_t st);
+cudaError_t launch_linear_backward(const float* gz, const float* x, float* gx, int mode_gx, const float* Wb, float* gWb,
+                                   float* gb, float* partial, int B, int Ci, int Co, long long P, cudaStream_t st,
+                                   long long* launches);
 cudaError_t launch_gelu_backward(const float* g, const float* z, float* gz, long long n, cudaStream_t st);
 cudaError_t launch_bypass_backward(const float* gz, const float* x, float* gx, const float* Wb, float* gWb,
                                    float* partial, int B, int Ci, int Co, long long P, cudaStream_t st,

@@ -50,12 +50,12 @@ static void write_file(const char* path, const void* buf, size_t bytes) {
 int main(int argc, char** argv) {
   if (argc < 2) return 64;
   const int d = atoi(argv[1]);
-  if (d < 1 || d > 4 || argc != 2 + 2 * d + 3 + 4) {
+  if (d < 1 || d > DTST_MAX_DIMS || argc != 2 + 2 * d + 3 + 4) {
     fprintf(stderr, "usage: %s d N.. k.. B C_in C_out x.bin W.bin Xhat.bin y.bin\n", argv[0]);
     return 64;
   }
-  int64_t N[4], K[4], M = 0;
-  int32_t kmax[4];
+  int64_t N[DTST_MAX_DIMS], K[DTST_MAX_DIMS], M = 0;
+  int32_t kmax[DTST_MAX_DIMS];
   size_t points = 1;
   for (int j = 0; j < d; ++j) {
     N[j] = atoll(argv[2 + j]);

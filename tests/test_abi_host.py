@@ -66,7 +66,7 @@ def test_edge_mode_tables():
 
 @pytest.mark.parametrize("d,N,k,B,Ci,Co", [
     (0, (8,), (2,), 1, 1, 1),            # d out of range
-    (5, (8,) * 5, (2,) * 5, 1, 1, 1),
+    (7, (8,) * 7, (2,) * 7, 1, 1, 1),
     (2, (8, 8), (5, 2), 1, 1, 1),        # 2k > N on a two-sided dim
     (2, (8, 8), (2, 6), 1, 1, 1),        # beyond Nyquist on the one-sided dim
     (2, (8, 8), (0, 2), 1, 1, 1),        # k < 1

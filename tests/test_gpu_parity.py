@@ -94,6 +94,9 @@ EDGE = [
     ("d2_k1", 2, 1, 1, (5, 6), (1, 1)),
     ("d3_ragged", 1, 3, 2, (10, 6, 12), (2, 3, 3)),
     ("d4_small", 1, 2, 2, (4, 6, 5, 8), (2, 1, 2, 3)),
+    ("d5", 1, 2, 1, (4, 3, 6, 4, 8), (2, 1, 2, 2, 3)),            # more dimensions than the benchmark uses
+    ("d6", 1, 1, 2, (2, 4, 3, 4, 2, 8), (1, 2, 1, 1, 1, 2)),
+    ("d5_fused_tail", 1, 1, 1, (2, 2, 32, 64, 32), (1, 1, 4, 8, 4)),   # d = 5 with plane + folded kernels inside
     ("big_batch", 6, 2, 3, (8, 16), (2, 4)),          # B > the mixing kernels' batch tile
     ("tail_rows", 1, 5, 7, (12, 20, 36), (3, 5, 7)),  # nothing a multiple of a tile
     ("wide_last", 1, 2, 2, (8, 8, 520), (2, 3, 9)),

@@ -376,6 +376,47 @@ def test_block_backward_matches_finite_differences():
         assert abs(re - gW[idx].real) < 1e-7 and abs(im - gW[idx].imag) < 1e-7
 
 
+def test_fno_forward_and_backward_match_torch_autograd():
+    """A whole small FNO (lift, two Fourier layers, projection) against torch float64 autograd through
+    rfftn / irfftn, linear layers and the exact GELU."""
+    import torch
+    N, kmax, B, Ca, dv, Cu, L = (6, 8, 10), (2, 3, 4), 2, 3, 4, 2, 2
+    M = O.num_modes(N, kmax)
+    a = _rand_x(N, B, Ca)
+    params = {"P_w": RNG.standard_normal((dv, Ca)), "P_b": RNG.standard_normal(dv),
+              "blocks": [((RNG.standard_normal((dv, dv, M)) + 1j * RNG.standard_normal((dv, dv, M))),
+                          RNG.standard_normal((dv, dv)) / 2) for _ in range(L)],
+              "Q_w": RNG.standard_normal((Cu, dv)), "Q_b": RNG.standard_normal(Cu)}
+    g = RNG.standard_normal((B, Cu) + N)
+    u, saved = O.fno_forward(a, params, kmax)
+    grads = O.fno_backward(g, params, saved, kmax)
+
+    d = len(N)
+    dims = tuple(range(2, 2 + d))
+    lists = O.mode_index_lists(N, kmax)
+    ix = torch.meshgrid(*[torch.tensor(l) for l in lists], indexing="ij")
+    t = lambda v, c=False: torch.tensor(v, dtype=torch.complex128 if c else torch.float64, requires_grad=True)
+    at, Pw, Pb, Qw, Qb = t(a), t(params["P_w"]), t(params["P_b"]), t(params["Q_w"]), t(params["Q_b"])
+    Ws = [(t(W, True), t(Wb)) for W, Wb in params["blocks"]]
+    lin = lambda x, w, b=None: torch.nn.functional.linear(x.movedim(1, -1), w, b).movedim(-1, 1)
+    v = lin(at, Pw, Pb)
+    for W, Wb in Ws:
+        Xs = torch.fft.rfftn(v, dim=dims)[(slice(None), slice(None)) + tuple(ix)]
+        Ys = torch.einsum("bim,iom->bom", Xs.reshape(B, dv, -1), W)
+        full = torch.zeros((B, dv) + tuple(N[:-1]) + (N[-1] // 2 + 1,), dtype=torch.complex128)
+        full[(slice(None), slice(None)) + tuple(ix)] = Ys.reshape((B, dv) + tuple(Xs.shape[2:]))
+        v = torch.nn.functional.gelu(lin(v, Wb) + torch.fft.irfftn(full, s=N, dim=dims))
+    ut = lin(v, Qw, Qb)
+    (ut * torch.tensor(g)).sum().backward()
+    assert O.rel_l2(u, ut.detach().numpy()) < 1e-12
+    assert O.rel_l2(grads["a"], at.grad.numpy()) < 1e-11
+    for name, tt in (("P_w", Pw), ("P_b", Pb), ("Q_w", Qw), ("Q_b", Qb)):
+        assert O.rel_l2(grads[name], tt.grad.numpy()) < 1e-11, name
+    for l in range(L):
+        assert O.rel_l2(grads["blocks"][l][0], Ws[l][0].grad.numpy()) < 1e-11
+        assert O.rel_l2(grads["blocks"][l][1], Ws[l][1].grad.numpy()) < 1e-11
+
+
 def test_block_layer_and_backward_are_slices_and_sums_of_the_global_ones():
     # a rank's block (Eq. 18): y and grad_x of the block are slices of the global results when the
     # block's spectrum is replaced by the summed one; partial spectra and grad_W sum over blocks
