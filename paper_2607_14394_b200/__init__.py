@@ -6,13 +6,16 @@ input generators.  The binding is imported lazily so that the input generators
 can be used without torch or the built library.
 """
 
-__all__ = ["Plan", "binding", "inputs", "build"]
+__all__ = ["Plan", "FNO", "binding", "inputs", "build"]
 
 
 def __getattr__(name):
     if name == "Plan":
         from .binding import Plan
         return Plan
+    if name == "FNO":
+        from .fno import FNO
+        return FNO
     if name in ("binding", "inputs", "build"):
         import importlib
         return importlib.import_module("." + name, __name__)

@@ -78,7 +78,7 @@ __global__ void __launch_bounds__(256) block_epilogue_kernel(const float* __rest
 }
 
 // g_z = grad_out * GELU'(z), element-wise, 16 bytes per access (gz may alias grad_out)
-__global__ void __launch_bounds__(256) gelu_backward_kernel(const float4* __restrict__ g, const float4* __restrict__ z,
+__global__ void __launch_bounds__(256) gelu_backward_kernel(const float4* g, const float4* __restrict__ z,
                                                            float4* gz, long long n4) {
   pdl_trigger();
   pdl_wait();
