@@ -215,6 +215,67 @@ def inverse_literal(Yhat: np.ndarray, N_global, kmax) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------
+# The DTST primitive as the paper states it (Section "Distributed Truncated Spectral Transforms"): a COMPLEX
+# d-dimensional tensor and the two-sided retained set S_j on EVERY dimension, the last one included
+# (K_j = 2 k_j for all j).  No Hermitian symmetry, hence no doubling: the inverse is the plain complex sum of Eq. 14.
+# --------------------------------------------------------------------------
+def mode_index_lists_complex(N, kmax):
+    return [retained_indices(int(N[j]), int(kmax[j]), one_sided=False) for j in range(len(N))]
+
+
+def forward_complex(x: np.ndarray, kmax, N_global=None, offsets=None) -> np.ndarray:
+    """Xhat[B, C, 2k_0..2k_{d-1}] from complex x[B, C, n_local...] (Eq. 5-6 with the basis of Eq. 18)."""
+    n_local = x.shape[2:]
+    d = len(n_local)
+    N_global = tuple(n_local) if N_global is None else tuple(N_global)
+    offsets = (0,) * d if offsets is None else tuple(offsets)
+    lists = mode_index_lists_complex(N_global, kmax)
+    t = x.astype(np.complex128)
+    for j in range(d - 1, -1, -1):
+        t = _apply_along(basis_matrix(N_global[j], lists[j], n_local[j], offsets[j]), t, 2 + j)
+    return t
+
+
+def inverse_complex(Yhat: np.ndarray, N_global, kmax, n_local=None, offsets=None, normalise: bool = True) -> np.ndarray:
+    """y[B, C, n_local...] complex = (1/prod N) sum_m Yhat[m] prod_j W_{N_j}^{-s_j n_j} (Eq. 14, B^{-1} = B^H / N)."""
+    d = len(N_global)
+    N_global = tuple(N_global)
+    n_local = N_global if n_local is None else tuple(n_local)
+    offsets = (0,) * d if offsets is None else tuple(offsets)
+    lists = mode_index_lists_complex(N_global, kmax)
+    t = Yhat.astype(np.complex128)
+    for j in range(d):
+        t = _apply_along(basis_matrix(N_global[j], lists[j], n_local[j], offsets[j]).conj().T, t, 2 + j)
+    return t / float(math.prod(N_global)) if normalise else t
+
+
+def layer_forward_complex(x: np.ndarray, W: np.ndarray, kmax, N_global=None, offsets=None):
+    n_local = x.shape[2:]
+    N = tuple(n_local) if N_global is None else tuple(N_global)
+    Xhat = forward_complex(x, kmax, N_global=N, offsets=offsets)
+    Yhat = spectral_mul(Xhat, W.reshape((W.shape[0], W.shape[1]) + Xhat.shape[2:]))
+    return inverse_complex(Yhat, N, kmax, n_local=n_local, offsets=offsets), Xhat
+
+
+def backward_complex(grad_y: np.ndarray, Xhat: np.ndarray, W: np.ndarray, kmax, N_global=None, offsets=None):
+    """Gradients of a real loss with upstream gradient grad_y = dL/dRe(y) + i dL/dIm(y) (the same convention for
+    every complex quantity): each linear step is replaced by its adjoint (Section "Backward Pass")."""
+    n_local = grad_y.shape[2:]
+    N = tuple(n_local) if N_global is None else tuple(N_global)
+    B = grad_y.shape[0]
+    G_Y = forward_complex(grad_y, kmax, N_global=N, offsets=offsets) / float(math.prod(N))
+    Ci, Co = W.shape[:2]
+    Wm = W.reshape(Ci, Co, -1).astype(np.complex128)
+    GYf = G_Y.reshape(B, Co, -1)
+    Xf = Xhat.reshape(B, Ci, -1).astype(np.complex128)
+    G_X = np.einsum("bom,iom->bim", GYf, Wm.conj())
+    G_W = np.einsum("bim,bom->iom", Xf.conj(), GYf)
+    g_x = inverse_complex(G_X.reshape((B, Ci) + G_Y.shape[2:]), N, kmax, n_local=n_local, offsets=offsets,
+                          normalise=False)
+    return g_x, G_W.reshape(W.shape)
+
+
+# --------------------------------------------------------------------------
 # The whole layer and its backward pass (Section "Backward Pass": adjoints)
 # --------------------------------------------------------------------------
 def layer_forward(x: np.ndarray, W: np.ndarray, kmax, N_global=None, offsets=None):

@@ -276,6 +276,63 @@ def test_layer_and_backward_match_torch_autograd(N, kmax):
     assert O.rel_l2(gW, gW_ref) < 1e-12
 
 
+# ---------------------------------------------------------------- the complex primitive (two-sided on every dim)
+@pytest.mark.parametrize("N,kmax", [((8,), (3,)), ((6, 8), (3, 2)), ((5, 6, 8), (2, 3, 4)), ((4, 6, 5, 8), (2, 1, 2, 3))])
+def test_complex_forward_and_inverse_against_fftn(N, kmax):
+    B, C = 2, 2
+    x = RNG.standard_normal((B, C) + N) + 1j * RNG.standard_normal((B, C) + N)
+    lists = O.mode_index_lists_complex(N, kmax)
+    dims = tuple(range(2, 2 + len(N)))
+    full = np.fft.fftn(x, axes=dims)
+    want = full[(slice(None), slice(None)) + np.ix_(*lists)]
+    X = O.forward_complex(x, kmax)
+    assert X.shape == (B, C) + tuple(2 * k for k in kmax)
+    assert O.rel_l2(X, want) < 1e-12
+    # inverse: ifftn of the spectrum zero-padded outside the retained set
+    Y = RNG.standard_normal(X.shape) + 1j * RNG.standard_normal(X.shape)
+    pad = np.zeros((B, C) + N, dtype=complex)
+    pad[(slice(None), slice(None)) + np.ix_(*lists)] = Y
+    assert O.rel_l2(O.inverse_complex(Y, N, kmax), np.fft.ifftn(pad, axes=dims)) < 1e-12
+    # slabs along dim 0 with global offsets sum to the whole (Eq. 6-7), and a block of the inverse is a slice
+    if N[0] % 2 == 0:
+        h = N[0] // 2
+        parts = sum(O.forward_complex(x[:, :, p * h:(p + 1) * h], kmax, N_global=N, offsets=(p * h,) + (0,) * (len(N) - 1))
+                    for p in range(2))
+        assert O.rel_l2(parts, X) < 1e-12
+        blk = O.inverse_complex(Y, N, kmax, n_local=(h,) + N[1:], offsets=(h,) + (0,) * (len(N) - 1))
+        assert O.rel_l2(blk, O.inverse_complex(Y, N, kmax)[:, :, h:]) < 1e-12
+    # a real field's complex transform agrees with the real path on the modes both keep (f >= 0 on the last dim)
+    xr = RNG.standard_normal((B, C) + N)
+    if kmax[-1] <= N[-1] // 2:
+        assert O.rel_l2(O.forward_complex(xr, kmax)[..., :kmax[-1]], O.forward(xr, kmax)) < 1e-12
+
+
+def test_complex_layer_backward_matches_torch_autograd():
+    import torch
+    N, kmax, B, Ci, Co = (6, 8, 10), (2, 3, 4), 2, 3, 2
+    x = RNG.standard_normal((B, Ci) + N) + 1j * RNG.standard_normal((B, Ci) + N)
+    M = int(np.prod([2 * k for k in kmax]))
+    W = RNG.standard_normal((Ci, Co, M)) + 1j * RNG.standard_normal((Ci, Co, M))
+    g = RNG.standard_normal((B, Co) + N) + 1j * RNG.standard_normal((B, Co) + N)
+    y, Xhat = O.layer_forward_complex(x, W, kmax)
+    gx, gW = O.backward_complex(g, Xhat, W, kmax)
+    lists = O.mode_index_lists_complex(N, kmax)
+    dims = tuple(range(2, 5))
+    xt = torch.tensor(x, requires_grad=True)
+    Wt = torch.tensor(W, requires_grad=True)
+    ix = torch.meshgrid(*[torch.tensor(l) for l in lists], indexing="ij")
+    Xs = torch.fft.fftn(xt, dim=dims)[(slice(None), slice(None)) + tuple(ix)]
+    Ys = torch.einsum("bim,iom->bom", Xs.reshape(B, Ci, -1), Wt)
+    full = torch.zeros((B, Co) + N, dtype=torch.complex128)
+    full[(slice(None), slice(None)) + tuple(ix)] = Ys.reshape((B, Co) + tuple(Xs.shape[2:]))
+    yt = torch.fft.ifftn(full, dim=dims)
+    gt = torch.tensor(g)
+    (yt.real * gt.real + yt.imag * gt.imag).sum().backward()      # L with dL/dRe y = Re g, dL/dIm y = Im g
+    assert O.rel_l2(y, yt.detach().numpy()) < 1e-12
+    assert O.rel_l2(gx, xt.grad.numpy()) < 1e-12
+    assert O.rel_l2(gW, Wt.grad.numpy()) < 1e-12
+
+
 # ---------------------------------------------------------------- the whole block (bypass + GELU)
 def test_gelu_against_math_erf_closed_forms_and_torch():
     import torch
