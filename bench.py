@@ -150,9 +150,9 @@ class ClockSampler:
 NCU_TRAFFIC = {
     "cfg5_4d_128": {
         "channels": (2, 4),
-        "grid_read": ((1073788000 + 64662000), None),      # (read + write) bytes at 2 and at 4 channels
-        "grid_write": ((67159000 + 1018316000), None),
-        "source": "profiles/kernels_cfg5_shape_c2_ncu_full.md",
+        "grid_read": (1138479500, 2277482880),      # read + write bytes per launch at 2 and at 4 channels
+        "grid_write": (1080677000, 2218299264),
+        "source": "profiles/plane_kernels_cfg5_shape_c2_c4_ncu.md",
     },
 }
 

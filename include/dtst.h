@@ -91,6 +91,29 @@ dtst_status dtst_plan_create_local(dtst_plan** out, int d, const int64_t N_globa
                                    const int32_t kmax[], int B, int C_in, int C_out);
 
 /*
+ * The DTST primitive as Section "Distributed Truncated Spectral Transforms" states it: a COMPLEX d-dimensional
+ * tensor and the two-sided retained set S_j = [0..k_j-1, N_j-k_j..N_j-1] on EVERY dimension, the last one included
+ * (K_j = 2 k_j for all j, 2 k_j <= N_j).  Arguments as dtst_plan_create_local; N_local and offset may both be NULL
+ * for a grid that lives entirely on this device.  Such a plan is used with dtst_forward_complex,
+ * dtst_spectral_mul (unchanged), dtst_inverse_complex and dtst_backward_complex; the real-field entry points
+ * return DTST_ERR_INVALID_ARG for it.  Virtual shards and per-rank blocks work as for real plans.  The contiguous
+ * dimension of a complex plan runs on the generic kernel family (the streaming kernels read real grids); the
+ * other dimensions on the folded and slab kernels.
+ *   F: Xhat[b,c,m] = sum_n x[b,c,n] prod_j exp(-2 pi i s_j(m) (off_j + n_j) / N_j)        (Eq. 5-6, Eq. 18)
+ *   I: y[b,o,n]    = (1/prod N) sum_m Yhat[b,o,m] prod_j exp(+2 pi i s_j(m) (off_j + n_j) / N_j)   (Eq. 14)
+ *      - no Hermitian doubling: nothing is implied by symmetry;
+ *   B: G_Y = F(grad_y) / prod N,  G_X and grad_W as in dtst_backward,  grad_x = sum_m G_X[m] e^{+i theta_m n}
+ *      (complex), gradients in the convention dL/dRe + i dL/dIm.
+ *   x, y, grad_y, grad_x: [B, C, n_0..n_{d-1}] complex64; spectra [B, C, K_0..K_{d-1}] complex64.
+ */
+dtst_status dtst_plan_create_complex(dtst_plan** out, int d, const int64_t N_global[], const int64_t N_local[],
+                                     const int64_t offset[], const int32_t kmax[], int B, int C_in, int C_out);
+dtst_status dtst_forward_complex(dtst_plan* plan, const void* x, void* Xhat, void* stream);
+dtst_status dtst_inverse_complex(dtst_plan* plan, const void* Yhat, void* y, void* stream);
+dtst_status dtst_backward_complex(dtst_plan* plan, const void* grad_y, const void* Xhat_saved, const void* W,
+                                  void* grad_x, void* grad_W, void* stream);
+
+/*
  * Virtual shards: split the (local) grid into P slabs along dim 0, compute each
  * slab's partial spectrum with its global phase offset and sum the P partials on
  * the device in ascending slab order (Eq. 6-7 without a collective).  The inverse

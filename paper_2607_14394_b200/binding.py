@@ -40,7 +40,8 @@ EXPORTED = [
     "dtst_plan_last_cuda_error", "dtst_spectral_mul_modes", "dtst_backward_spectrum", "dtst_backward_mix_modes",
     "dtst_backward_input", "dtst_plan_debug_ring_fault", "dtst_plan_set_column_expansion", "dtst_plan_require_fast_path", "dtst_block_forward", "dtst_block_backward",
     "dtst_plan_set_block_epilogue", "dtst_pointwise_linear", "dtst_pointwise_linear_scratch_bytes",
-    "dtst_pointwise_linear_backward",
+    "dtst_pointwise_linear_backward", "dtst_plan_create_complex", "dtst_forward_complex", "dtst_inverse_complex",
+    "dtst_backward_complex",
 ]
 
 
@@ -66,6 +67,10 @@ def lib() -> ctypes.CDLL:
     vp, i32, i64p, i32p = ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int32)
     L.dtst_plan_create.argtypes = [ctypes.POINTER(vp), i32, i64p, i32p, i32, i32, i32]
     L.dtst_plan_create_local.argtypes = [ctypes.POINTER(vp), i32, i64p, i64p, i64p, i32p, i32, i32, i32]
+    L.dtst_plan_create_complex.argtypes = [ctypes.POINTER(vp), i32, i64p, i64p, i64p, i32p, i32, i32, i32]
+    L.dtst_forward_complex.argtypes = [vp, vp, vp, vp]
+    L.dtst_inverse_complex.argtypes = [vp, vp, vp, vp]
+    L.dtst_backward_complex.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.dtst_plan_set_virtual_shards.argtypes = [vp, i32]
     L.dtst_plan_set_kernel_path.argtypes = [vp, i32]
     L.dtst_plan_kernel_path.argtypes = [vp, ctypes.POINTER(i32)]
@@ -168,6 +173,32 @@ def dtst_plan_create_local(d, N_global, N_local, offset, kmax, B, C_in, C_out) -
     _check(lib().dtst_plan_create_local(ctypes.byref(h), int(d), _i64(N_global), _i64(N_local), _i64(offset),
                                         _i32(kmax), int(B), int(C_in), int(C_out)), "dtst_plan_create_local")
     return h
+
+
+def dtst_plan_create_complex(d, N_global, N_local, offset, kmax, B, C_in, C_out) -> ctypes.c_void_p:
+    h = ctypes.c_void_p(0)
+    _check(lib().dtst_plan_create_complex(ctypes.byref(h), int(d), _i64(N_global),
+                                          None if N_local is None else _i64(N_local),
+                                          None if offset is None else _i64(offset), _i32(kmax), int(B), int(C_in),
+                                          int(C_out)), "dtst_plan_create_complex")
+    return h
+
+
+def dtst_forward_complex(plan, x, Xhat, stream=None) -> None:
+    _check(lib().dtst_forward_complex(plan, _ptr(x, torch.complex64, "x"), _ptr(Xhat, torch.complex64, "Xhat"),
+                                      _stream_ptr(stream)), "dtst_forward_complex", plan)
+
+
+def dtst_inverse_complex(plan, Yhat, y, stream=None) -> None:
+    _check(lib().dtst_inverse_complex(plan, _ptr(Yhat, torch.complex64, "Yhat"), _ptr(y, torch.complex64, "y"),
+                                      _stream_ptr(stream)), "dtst_inverse_complex", plan)
+
+
+def dtst_backward_complex(plan, grad_y, Xhat_saved, W, grad_x, grad_W, stream=None) -> None:
+    _check(lib().dtst_backward_complex(plan, _ptr(grad_y, torch.complex64, "grad_y"),
+                                       _ptr(Xhat_saved, torch.complex64, "Xhat_saved"), _ptr(W, torch.complex64, "W"),
+                                       _ptr(grad_x, torch.complex64, "grad_x"), _ptr(grad_W, torch.complex64, "grad_W"),
+                                       _stream_ptr(stream)), "dtst_backward_complex", plan)
 
 
 def dtst_plan_set_virtual_shards(plan, P) -> None:
@@ -385,7 +416,8 @@ class Plan:
     """
 
     def __init__(self, N, kmax, B, C_in, C_out, N_global=None, offset=None, virtual_shards: int = 1,
-                 path: str = "auto", device=None, allocate_workspace: bool = True, column_expansion: int = 0):
+                 path: str = "auto", device=None, allocate_workspace: bool = True, column_expansion: int = 0,
+                 complex_fields: bool = False):
         self.N = tuple(int(n) for n in N)
         self.kmax = tuple(int(k) for k in kmax)
         self.d = len(self.N)
@@ -396,8 +428,14 @@ class Plan:
         if self.device.index is None:
             self.device = torch.device("cuda", torch.cuda.current_device())
         self._h = None
+        self.complex_fields = bool(complex_fields)
+        self.grid_dtype = torch.complex64 if complex_fields else torch.float32
         with torch.cuda.device(self.device):
-            if N_global is None:
+            if complex_fields:
+                self._h = dtst_plan_create_complex(self.d, self.N if N_global is None else N_global,
+                                                   None if N_global is None else self.N, offset, self.kmax, B, C_in,
+                                                   C_out)
+            elif N_global is None:
                 self._h = dtst_plan_create(self.d, self.N, self.kmax, B, C_in, C_out)
             else:
                 self._h = dtst_plan_create_local(self.d, N_global, self.N, offset, self.kmax, B, C_in, C_out)
@@ -476,7 +514,7 @@ class Plan:
         self._expect(x, "x", "x")
         self._expect(out, "Xhat", "out")
         with torch.cuda.device(self.device):
-            dtst_forward(self._h, x, out, stream)
+            (dtst_forward_complex if self.complex_fields else dtst_forward)(self._h, x, out, stream)
         return out
 
     def forward_static(self, x, out, stream=None):
@@ -499,17 +537,17 @@ class Plan:
 
     def inverse(self, Yhat, out=None, stream=None):
         if out is None:
-            out = torch.empty((self.B, self.C_out) + self.N, dtype=torch.float32, device=self.device)
+            out = torch.empty((self.B, self.C_out) + self.N, dtype=self.grid_dtype, device=self.device)
         self._expect(Yhat, "Yhat", "Yhat")
         self._expect(out, "y", "out")
         with torch.cuda.device(self.device):
-            dtst_inverse(self._h, Yhat, out, stream)
+            (dtst_inverse_complex if self.complex_fields else dtst_inverse)(self._h, Yhat, out, stream)
         return out
 
     def backward(self, grad_y, Xhat_saved, W, grad_x=None, grad_W=None, need_grad_x=True, need_grad_W=True,
                  stream=None):
         if grad_x is None and need_grad_x:
-            grad_x = torch.empty((self.B, self.C_in) + self.N, dtype=torch.float32, device=self.device)
+            grad_x = torch.empty((self.B, self.C_in) + self.N, dtype=self.grid_dtype, device=self.device)
         if grad_W is None and need_grad_W:
             grad_W = torch.empty((self.C_in, self.C_out, self.M), dtype=torch.complex64, device=self.device)
         self._expect(grad_y, "y", "grad_y")
@@ -518,7 +556,8 @@ class Plan:
         self._expect(grad_x, "x", "grad_x")
         self._expect(grad_W, "W", "grad_W")
         with torch.cuda.device(self.device):
-            dtst_backward(self._h, grad_y, Xhat_saved, W, grad_x, grad_W, stream)
+            (dtst_backward_complex if self.complex_fields else dtst_backward)(self._h, grad_y, Xhat_saved, W, grad_x,
+                                                                               grad_W, stream)
         return grad_x, grad_W
 
     # -- the whole block of Algorithm 1: GELU(W_bypass x + layer(x))

@@ -37,7 +37,7 @@ bool mul_overflows(long long a, long long b) {
 }
 
 dtst_status create_common(dtst_plan** out, int d, const int64_t* Ng, const int64_t* Nl, const int64_t* off,
-                          const int32_t* kmax, int B, int C_in, int C_out) {
+                          const int32_t* kmax, int B, int C_in, int C_out, bool complex_io = false) {
   if (out == nullptr) return DTST_ERR_INVALID_ARG;
   *out = nullptr;
   if (Ng == nullptr || kmax == nullptr || d < 1 || d > kMaxDims) return DTST_ERR_INVALID_ARG;
@@ -50,12 +50,12 @@ dtst_status create_common(dtst_plan** out, int d, const int64_t* Ng, const int64
     if (ng < 1 || ng > (1ll << 30) || nl < 1 || o < 0 || o + nl > ng) return DTST_ERR_INVALID_ARG;
     const long long k = kmax[j];
     if (k < 1) return DTST_ERR_INVALID_ARG;
-    if (j < d - 1) {
+    if (j < d - 1 || complex_io) {
       if (2 * k > ng) return DTST_ERR_INVALID_ARG;     // the two halves of S_j must not overlap
     } else {
       if (k > ng / 2 + 1) return DTST_ERR_INVALID_ARG; // one-sided: at most up to Nyquist
     }
-    const long long K = (j < d - 1) ? 2 * k : k;
+    const long long K = (j < d - 1 || complex_io) ? 2 * k : k;
     if (mul_overflows(pts_l, nl) || mul_overflows(pts_g, ng) || mul_overflows(M, K)) return DTST_ERR_INVALID_ARG;
     pts_l *= nl;
     pts_g *= ng;
@@ -77,7 +77,7 @@ dtst_status create_common(dtst_plan** out, int d, const int64_t* Ng, const int64
     p->Nl[j] = Nl ? Nl[j] : Ng[j];
     p->off[j] = off ? off[j] : 0;
     p->kmax[j] = kmax[j];
-    p->K[j] = (j < d - 1) ? 2 * kmax[j] : kmax[j];
+    p->K[j] = (j < d - 1 || complex_io) ? 2 * kmax[j] : kmax[j];
   }
   p->M = M;
   p->points_local = pts_l;
@@ -85,6 +85,7 @@ dtst_status create_common(dtst_plan** out, int d, const int64_t* Ng, const int64
   p->P = 1;
   p->path_request = DTST_PATH_AUTO;
   p->dbg_withhold_after = -1;
+  p->complex_io = complex_io ? 1 : 0;
   p->device = -1;
   int dev = -1;
   if (cudaGetDevice(&dev) == cudaSuccess) p->device = dev;
@@ -116,12 +117,13 @@ bool use_slab(const dtst_plan* p, int j) {
   return slab_supported((int)p->Nl[j], p->kmax[j]);
 }
 
-bool use_fused(const dtst_plan* p) { return p->path_request == DTST_PATH_AUTO && fused_eligible(p); }
+// (the plane and row kernels read a REAL grid: complex plans take the generic kernel on the contiguous dimension)
+bool use_fused(const dtst_plan* p) { return p->path_request == DTST_PATH_AUTO && !p->complex_io && fused_eligible(p); }
 
 // Row kernels: the contiguous dimension alone (whole on this device, zero offset), for shapes without a
 // plane kernel; the other dimensions then run on the reduced tensor.
 bool use_row(const dtst_plan* p) {
-  if (p->path_request != DTST_PATH_AUTO || use_fused(p)) return false;
+  if (p->path_request != DTST_PATH_AUTO || p->complex_io || use_fused(p)) return false;
   const int a = p->d - 1;
   if (p->Nl[a] != p->Ng[a] || p->off[a] != 0) return false;
   if (p->d == 1 && p->P > 1) return false;
@@ -135,6 +137,7 @@ bool use_row(const dtst_plan* p) {
 // grid-side stage runs on a plane or row kernel and every other dimension on a folded or slab kernel, in both
 // directions.
 bool all_streaming(const dtst_plan* p) {
+  if (p->complex_io) return false;   // the contiguous dimension of a complex plan runs on the generic kernel
   int first;
   if (use_fused(p)) first = p->d - 3;
   else if (use_row(p)) first = p->d - 2;
@@ -160,7 +163,7 @@ DimOp make_op(const dtst_plan* p, int j, bool forward, int Cn) {
   op.R = forward ? p->K[j] : (int)p->Nl[j];
   op.N = (int)p->Ng[j];
   op.k = p->kmax[j];
-  op.two_sided = (j < p->d - 1) ? 1 : 0;
+  op.two_sided = (j < p->d - 1 || p->complex_io) ? 1 : 0;
   op.offset = (int)p->off[j];
   op.offset_step = 0;
   op.forward = forward ? 1 : 0;
@@ -184,8 +187,8 @@ dtst_status forward_stages(dtst_plan* p, const void* cur, int j_from, int flip, 
   float2* partial = reinterpret_cast<float2*>(ws + L.partial);
   for (int j = j_from; j >= 0; --j) {
     DimOp op = make_op(p, j, true, Cn);
-    const bool in_real = (j == p->d - 1);
-    if (in_real) {
+    const bool in_real = (j == p->d - 1) && !p->complex_io;
+    if (j == p->d - 1) {
       op.scale = scale;
       op.herm = herm ? 1 : 0;
     }
@@ -266,8 +269,8 @@ dtst_status run_forward_fused(dtst_plan* p, const float* x, float2* Xhat, int Cn
 dtst_status expand_stage(dtst_plan* p, int j, int Cn, const void* cur, void* dst, float scale, bool herm,
                          cudaStream_t st) {
   DimOp op = make_op(p, j, false, Cn);
-  const bool out_real = (j == p->d - 1);
-  if (out_real) {
+  const bool out_real = (j == p->d - 1) && !p->complex_io;
+  if (j == p->d - 1) {
     op.scale = scale;
     op.herm = herm ? 1 : 0;
   }
@@ -625,7 +628,7 @@ dtst_status dtst_plan_num_modes(const dtst_plan* p, int64_t* M, int64_t K[]) {
 dtst_status dtst_plan_mode_indices(const dtst_plan* p, int dim, int64_t* idx) {
   if (p == nullptr || idx == nullptr || dim < 0 || dim >= p->d) return DTST_ERR_INVALID_ARG;
   for (int r = 0; r < p->K[dim]; ++r)
-    idx[r] = mode_at(r, p->kmax[dim], (int)p->Ng[dim], dim < p->d - 1 ? 1 : 0);
+    idx[r] = mode_at(r, p->kmax[dim], (int)p->Ng[dim], (dim < p->d - 1 || p->complex_io) ? 1 : 0);
   return DTST_OK;
 }
 
@@ -648,9 +651,57 @@ dtst_status dtst_plan_set_workspace(dtst_plan* p, void* dev_ptr, size_t bytes) {
   return DTST_OK;
 }
 
+dtst_status dtst_plan_create_complex(dtst_plan** out, int d, const int64_t N_global[], const int64_t N_local[],
+                                     const int64_t offset[], const int32_t kmax[], int B, int C_in, int C_out) {
+  return create_common(out, d, N_global, N_local, offset, kmax, B, C_in, C_out, true);
+}
+
+dtst_status dtst_forward_complex(dtst_plan* p, const void* x, void* Xhat, void* stream) {
+  dtst_status s = check_ready(p);
+  if (s != DTST_OK) return s;
+  if (!p->complex_io || x == nullptr || Xhat == nullptr || !aligned16(x) || !aligned16(Xhat)) return DTST_ERR_INVALID_ARG;
+  return run_forward_generic(p, static_cast<const float*>(x), static_cast<float2*>(Xhat), p->C_in, 1.0f, false,
+                             static_cast<cudaStream_t>(stream));
+}
+
+dtst_status dtst_inverse_complex(dtst_plan* p, const void* Yhat, void* y, void* stream) {
+  dtst_status s = check_ready(p);
+  if (s != DTST_OK) return s;
+  if (!p->complex_io || Yhat == nullptr || y == nullptr || !aligned16(Yhat) || !aligned16(y)) return DTST_ERR_INVALID_ARG;
+  return run_inverse_generic(p, static_cast<const float2*>(Yhat), static_cast<float*>(y), p->C_out,
+                             (float)(1.0 / (double)p->points_global), false, static_cast<cudaStream_t>(stream));
+}
+
+dtst_status dtst_backward_complex(dtst_plan* p, const void* grad_y, const void* Xhat_saved, const void* W, void* grad_x,
+                                  void* grad_W, void* stream) {
+  dtst_status s = check_ready(p);
+  if (s != DTST_OK) return s;
+  if (!p->complex_io || grad_y == nullptr || W == nullptr || (grad_x == nullptr && grad_W == nullptr) ||
+      (grad_W != nullptr && Xhat_saved == nullptr))
+    return DTST_ERR_INVALID_ARG;
+  if (!aligned16(grad_y) || !aligned16(Xhat_saved) || !aligned16(W) || !aligned16(grad_x) || !aligned16(grad_W))
+    return DTST_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const WsLayout L = ws_layout(p);
+  char* ws = static_cast<char*>(p->ws);
+  float2* GY = reinterpret_cast<float2*>(ws + L.gy);
+  float2* GX = reinterpret_cast<float2*>(ws + L.gx);
+  // adjoint of the inverse: G_Y = F(grad_y) / prod N (no Hermitian weights: nothing was doubled)
+  s = run_forward_generic(p, static_cast<const float*>(grad_y), GY, p->C_out, (float)(1.0 / (double)p->points_global),
+                          false, st);
+  if (s != DTST_OK) return s;
+  if (cuda_failed(p, launch_mix_adjoint(GY, static_cast<const float2*>(Xhat_saved), static_cast<const float2*>(W),
+                                        grad_x ? GX : nullptr, static_cast<float2*>(grad_W), p->B, p->C_in, p->C_out,
+                                        p->M, st, &p->launches)))
+    return DTST_ERR_CUDA;
+  if (grad_x != nullptr) return run_inverse_generic(p, GX, static_cast<float*>(grad_x), p->C_in, 1.0f, false, st);
+  return DTST_OK;
+}
+
 dtst_status dtst_forward(dtst_plan* p, const float* x, void* Xhat, void* stream) {
   dtst_status s = check_ready(p);
   if (s != DTST_OK) return s;
+  if (p->complex_io) return DTST_ERR_INVALID_ARG;   // a complex plan: dtst_forward_complex
   if (x == nullptr || Xhat == nullptr || !aligned16(x) || !aligned16(Xhat)) return DTST_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (use_fused(p)) return run_forward_fused(p, x, static_cast<float2*>(Xhat), p->C_in, 1.0f, false, st);
@@ -673,7 +724,7 @@ dtst_status dtst_spectral_mul(dtst_plan* p, const void* Xhat, const void* W, voi
 dtst_status dtst_inverse(dtst_plan* p, const void* Yhat, float* y, void* stream) {
   dtst_status s = check_ready(p);
   if (s != DTST_OK) return s;
-  if (Yhat == nullptr || y == nullptr || !aligned16(Yhat) || !aligned16(y)) return DTST_ERR_INVALID_ARG;
+  if (p->complex_io || Yhat == nullptr || y == nullptr || !aligned16(Yhat) || !aligned16(y)) return DTST_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const float scale = (float)(1.0 / (double)p->points_global);
   if (use_fused(p)) return run_inverse_fused(p, static_cast<const float2*>(Yhat), y, p->C_out, scale, true, st);
@@ -686,7 +737,7 @@ dtst_status dtst_backward(dtst_plan* p, const float* grad_y, const void* Xhat_sa
   dtst_status s = check_ready(p);
   if (s != DTST_OK) return s;
   // Xhat_saved is read for grad_W only
-  if (grad_y == nullptr || W == nullptr || (grad_x == nullptr && grad_W == nullptr) ||
+  if (p->complex_io || grad_y == nullptr || W == nullptr || (grad_x == nullptr && grad_W == nullptr) ||
       (grad_W != nullptr && Xhat_saved == nullptr))
     return DTST_ERR_INVALID_ARG;
   if (!aligned16(grad_y) || !aligned16(Xhat_saved) || !aligned16(W) || !aligned16(grad_x) || !aligned16(grad_W))
@@ -865,7 +916,7 @@ dtst_status dtst_spectral_mul_modes(dtst_plan* p, const void* Xhat, const void* 
 dtst_status dtst_backward_spectrum(dtst_plan* p, const float* grad_y, void* GY, void* stream) {
   dtst_status s = check_ready(p);
   if (s != DTST_OK) return s;
-  if (grad_y == nullptr || GY == nullptr || !aligned16(grad_y) || !aligned16(GY)) return DTST_ERR_INVALID_ARG;
+  if (p->complex_io || grad_y == nullptr || GY == nullptr || !aligned16(grad_y) || !aligned16(GY)) return DTST_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const float scale = (float)(1.0 / (double)p->points_global);
   float2* out = static_cast<float2*>(GY);
@@ -896,7 +947,7 @@ dtst_status dtst_backward_mix_modes(dtst_plan* p, const void* GY, const void* Xh
 dtst_status dtst_backward_input(dtst_plan* p, const void* GX, float* grad_x, void* stream) {
   dtst_status s = check_ready(p);
   if (s != DTST_OK) return s;
-  if (GX == nullptr || grad_x == nullptr || !aligned16(GX) || !aligned16(grad_x)) return DTST_ERR_INVALID_ARG;
+  if (p->complex_io || GX == nullptr || grad_x == nullptr || !aligned16(GX) || !aligned16(grad_x)) return DTST_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const float2* in = static_cast<const float2*>(GX);
   return use_fused(p) ? run_inverse_fused(p, in, grad_x, p->C_in, 1.0f, false, st)

@@ -50,7 +50,7 @@ long long stage_elems(const dtst_plan* p, int j) {
 }  // namespace
 
 extern "C" dtst_status dtst_forward_static(dtst_plan* p, const float* x, void* Xhat_, void* stream) {
-  if (p == nullptr || x == nullptr || Xhat_ == nullptr) return DTST_ERR_INVALID_ARG;
+  if (p == nullptr || x == nullptr || Xhat_ == nullptr || p->complex_io) return DTST_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(x) & 15u) || (reinterpret_cast<uintptr_t>(Xhat_) & 15u))
     return DTST_ERR_INVALID_ARG;
   float2* Xhat = static_cast<float2*>(Xhat_);
