@@ -132,6 +132,23 @@ dtst_status dtst_plan_set_kernel_path(dtst_plan* plan, int path);
 dtst_status dtst_plan_kernel_path(const dtst_plan* plan, int* path);
 
 /*
+ * Contraction order (Section "cuBLAS vs cuFFT", paragraph on dimension ordering: the result does not depend on
+ * the order, the work does - contracting the most compressing dimension first shrinks the tensor soonest).
+ * The grid-side kernel always takes the contiguous dimension (and, on the fused path, the one in front of it);
+ * `order` lists the remaining candidates, the dimensions 0..d-2 (n = d-1 entries, a permutation), in the order
+ * the forward-type transforms contract them; the inverse-type transforms expand in the reverse order.  On the
+ * fused path the position of dimension d-2 in the list is ignored.  Default: d-2, d-3, .., 0 (Algorithm 1
+ * line 2).  With virtual shards dimension 0 must come last (the slab partial spectra are summed after the last
+ * stage), else DTST_ERR_INVALID_ARG.  Changes workspace_bytes: query it again.
+ * dtst_plan_tune_contraction_order picks the order by ascending K_j / n_j (local extent), dimension 0 last if it
+ * carries virtual shards, and reports the bytes the stages behind the grid-side kernel move per forward-type
+ * transform before and after (either pointer may be NULL).
+ */
+dtst_status dtst_plan_set_contraction_order(dtst_plan* plan, const int32_t order[], int n);
+dtst_status dtst_plan_get_contraction_order(const dtst_plan* plan, int32_t order[]);
+dtst_status dtst_plan_tune_contraction_order(dtst_plan* plan, double* bytes_before, double* bytes_after);
+
+/*
  * "Fast path or fail".  Shapes outside the streaming kernels' reach (odd extents, a contiguous extent that is not
  * a multiple of 32, k outside {4, 8, 12, 16} on a middle dimension, offsets on the contiguous dimension) are
  * served by a generic kernel that is an order of magnitude slower.  With required != 0 this call returns

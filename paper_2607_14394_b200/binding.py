@@ -41,7 +41,8 @@ EXPORTED = [
     "dtst_backward_input", "dtst_plan_debug_ring_fault", "dtst_plan_set_column_expansion", "dtst_plan_require_fast_path", "dtst_block_forward", "dtst_block_backward",
     "dtst_plan_set_block_epilogue", "dtst_pointwise_linear", "dtst_pointwise_linear_scratch_bytes",
     "dtst_pointwise_linear_backward", "dtst_plan_create_complex", "dtst_forward_complex", "dtst_inverse_complex",
-    "dtst_backward_complex",
+    "dtst_backward_complex", "dtst_plan_set_contraction_order", "dtst_plan_get_contraction_order",
+    "dtst_plan_tune_contraction_order",
 ]
 
 
@@ -71,6 +72,9 @@ def lib() -> ctypes.CDLL:
     L.dtst_forward_complex.argtypes = [vp, vp, vp, vp]
     L.dtst_inverse_complex.argtypes = [vp, vp, vp, vp]
     L.dtst_backward_complex.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.dtst_plan_set_contraction_order.argtypes = [vp, i32p, i32]
+    L.dtst_plan_get_contraction_order.argtypes = [vp, i32p]
+    L.dtst_plan_tune_contraction_order.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     L.dtst_plan_set_virtual_shards.argtypes = [vp, i32]
     L.dtst_plan_set_kernel_path.argtypes = [vp, i32]
     L.dtst_plan_kernel_path.argtypes = [vp, ctypes.POINTER(i32)]
@@ -199,6 +203,24 @@ def dtst_backward_complex(plan, grad_y, Xhat_saved, W, grad_x, grad_W, stream=No
                                        _ptr(Xhat_saved, torch.complex64, "Xhat_saved"), _ptr(W, torch.complex64, "W"),
                                        _ptr(grad_x, torch.complex64, "grad_x"), _ptr(grad_W, torch.complex64, "grad_W"),
                                        _stream_ptr(stream)), "dtst_backward_complex", plan)
+
+
+def dtst_plan_set_contraction_order(plan, order) -> None:
+    _check(lib().dtst_plan_set_contraction_order(plan, _i32(order), len(order)), "dtst_plan_set_contraction_order")
+
+
+def dtst_plan_get_contraction_order(plan, d):
+    buf = (ctypes.c_int32 * max(1, d - 1))()
+    _check(lib().dtst_plan_get_contraction_order(plan, buf), "dtst_plan_get_contraction_order")
+    return [int(v) for v in buf][:d - 1]
+
+
+def dtst_plan_tune_contraction_order(plan):
+    """Returns (bytes_before, bytes_after) of the stages behind the grid-side kernel per forward-type transform."""
+    a, b = ctypes.c_double(0), ctypes.c_double(0)
+    _check(lib().dtst_plan_tune_contraction_order(plan, ctypes.byref(a), ctypes.byref(b)),
+           "dtst_plan_tune_contraction_order")
+    return float(a.value), float(b.value)
 
 
 def dtst_plan_set_virtual_shards(plan, P) -> None:
@@ -648,6 +670,28 @@ class Plan:
         Yhat = self.spectral_mul(Xhat, W, Yhat, stream)
         y = self.inverse(Yhat, y, stream)
         return y, Xhat
+
+    def _reset_workspace(self) -> None:
+        if self.workspace is not None:
+            nbytes = dtst_plan_workspace_bytes(self._h)
+            if nbytes > self.workspace.numel():
+                self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            with torch.cuda.device(self.device):
+                dtst_plan_set_workspace(self._h, self.workspace)
+
+    def set_contraction_order(self, order) -> None:
+        """Order in which the forward-type transforms contract the dimensions 0..d-2 (a permutation)."""
+        dtst_plan_set_contraction_order(self._h, order)
+        self._reset_workspace()
+
+    def contraction_order(self):
+        return dtst_plan_get_contraction_order(self._h, self.d)
+
+    def tune_contraction_order(self):
+        """Most compressing dimension first; returns the modelled (bytes_before, bytes_after) of the stages."""
+        r = dtst_plan_tune_contraction_order(self._h)
+        self._reset_workspace()
+        return r
 
     def set_block_epilogue(self, mode) -> None:
         """'auto', 'ffma' or 'tensor': which kernel forms the bypass product of block_forward."""

@@ -84,6 +84,7 @@ dtst_status create_common(dtst_plan** out, int d, const int64_t* Ng, const int64
   p->points_global = pts_g;
   p->P = 1;
   p->path_request = DTST_PATH_AUTO;
+  for (int j = 0; j < kMaxDims; ++j) p->order_rank[j] = d - 1 - j;   // default: d-2 first, dimension 0 last
   p->dbg_withhold_after = -1;
   p->complex_io = complex_io ? 1 : 0;
   p->device = -1;
@@ -149,14 +150,35 @@ bool all_streaming(const dtst_plan* p) {
   return true;
 }
 
-DimOp make_op(const dtst_plan* p, int j, bool forward, int Cn) {
+// The dimensions 0..j_top in the order the forward transform contracts them (the expansion walks it backwards):
+// ascending rank, the plan's contraction order (dtst_plan_set_contraction_order; default d-2, d-3, .., 0).
+int middle_order(const dtst_plan* p, int j_top, int* out) {
+  int n = 0;
+  for (int j = 0; j <= j_top; ++j) out[n++] = j;
+  for (int a = 1; a < n; ++a)          // insertion sort by rank
+    for (int b = a; b > 0 && p->order_rank[out[b]] < p->order_rank[out[b - 1]]; --b) {
+      const int t = out[b];
+      out[b] = out[b - 1];
+      out[b - 1] = t;
+    }
+  return n;
+}
+
+// complex elements of a tensor in which dimension i has its retained entries (contracted[i]) or its local grid extent
+long long state_elems(const dtst_plan* p, int Cn, const bool* contracted) {
+  long long n = (long long)p->B * Cn;
+  for (int i = 0; i < p->d; ++i) n *= contracted[i] ? p->K[i] : p->Nl[i];
+  return n;
+}
+
+// One per-dimension operation on a tensor whose other dimensions are in the state `contracted` says.
+DimOp make_op(const dtst_plan* p, int j, bool forward, int Cn, const bool* contracted) {
   DimOp op;
   std::memset(&op, 0, sizeof(op));
   long long outer = (long long)p->B * Cn;
-  for (int i = 0; i < j; ++i) outer *= p->Nl[i];
+  for (int i = 0; i < j; ++i) outer *= contracted[i] ? p->K[i] : p->Nl[i];
   long long inner = 1;
-  for (int i = j + 1; i < p->d; ++i) inner *= forward ? p->K[i] : p->K[i];
-  // forward: dims after j are already contracted (K); expand: dims after j are not yet expanded (K)
+  for (int i = j + 1; i < p->d; ++i) inner *= contracted[i] ? p->K[i] : p->Nl[i];
   op.outer = outer;
   op.inner = inner;
   op.Q = forward ? (int)p->Nl[j] : p->K[j];
@@ -177,16 +199,26 @@ DimOp make_op(const dtst_plan* p, int j, bool forward, int Cn) {
   return op;
 }
 
-// Forward stages j_from..0 on `cur` (real iff j_from is the last dimension), ping-ponging through the
-// workspace; the result lands in Xhat.  scale/herm apply on the one-sided dimension's stage only.
+// Forward stages on `cur`: the last dimension first when j_from == d-1 (then `cur` is the grid itself), then the
+// dimensions 0..min(j_from, d-2) in the plan's contraction order, ping-ponging through the workspace; the result
+// lands in Xhat.  scale/herm apply on the last dimension's stage only.
 dtst_status forward_stages(dtst_plan* p, const void* cur, int j_from, int flip, float2* Xhat, int Cn,
                            float scale, bool herm, cudaStream_t st) {
   const WsLayout L = ws_layout(p);
   char* ws = static_cast<char*>(p->ws);
   float2* buf[2] = {reinterpret_cast<float2*>(ws + L.bufA), reinterpret_cast<float2*>(ws + L.bufB)};
   float2* partial = reinterpret_cast<float2*>(ws + L.partial);
-  for (int j = j_from; j >= 0; --j) {
-    DimOp op = make_op(p, j, true, Cn);
+  int list[kMaxDims + 1], n = 0;
+  if (j_from == p->d - 1) list[n++] = p->d - 1;
+  n += middle_order(p, j_from < p->d - 1 ? j_from : p->d - 2, list + n);
+  bool contracted[kMaxDims];
+  for (int i = 0; i < p->d; ++i) contracted[i] = i > j_from;
+  bool need_reduce = false;
+  for (int idx = 0; idx < n; ++idx) {
+    const int j = list[idx];
+    const bool last = idx == n - 1;
+    DimOp op = make_op(p, j, true, Cn, contracted);
+    contracted[j] = true;
     const bool in_real = (j == p->d - 1) && !p->complex_io;
     if (j == p->d - 1) {
       op.scale = scale;
@@ -194,19 +226,19 @@ dtst_status forward_stages(dtst_plan* p, const void* cur, int j_from, int flip, 
     }
     if (!in_real && use_slab(p, j)) {
       // slabs (or a rank's block) of this dimension: partial spectra formed and summed inside one kernel
-      void* sdst = (j == 0) ? static_cast<void*>(Xhat) : static_cast<void*>(buf[flip]);
+      void* sdst = last ? static_cast<void*>(Xhat) : static_cast<void*>(buf[flip]);
       if (cuda_failed(p, launch_slab(true, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(sdst),
                                      op.outer, op.inner, (int)p->Nl[j], op.N, (int)p->off[j], j == 0 ? p->P : 1, st)))
         return DTST_ERR_CUDA;
       ++p->launches;
       cur = sdst;
       flip ^= 1;
-      if (j == 0) return DTST_OK;
       continue;
     }
     void* dst;
     if (j == 0 && p->P > 1) {
-      // slab p contracts rows [p*nl, (p+1)*nl) of dim 0 with its own phase offset (Eq. 6, Eq. 18)
+      // slab p contracts rows [p*nl, (p+1)*nl) of dim 0 with its own phase offset (Eq. 6, Eq. 18); the P partial
+      // spectra are summed afterwards, so this stage is the last one (the contraction order guarantees it)
       const int nl = (int)(p->Nl[0] / p->P);
       op.slabs = p->P;
       op.Q = nl;
@@ -215,8 +247,9 @@ dtst_status forward_stages(dtst_plan* p, const void* cur, int j_from, int flip, 
       op.in_slab_stride = (long long)nl * op.inner;
       op.out_slab_stride = (long long)p->B * Cn * p->M;
       dst = partial;
+      need_reduce = true;
     } else {
-      dst = (j == 0) ? static_cast<void*>(Xhat) : static_cast<void*>(buf[flip]);
+      dst = last ? static_cast<void*>(Xhat) : static_cast<void*>(buf[flip]);
     }
     if (!in_real && use_mid(p, j)) {
       if (cuda_failed(p, launch_mid(true, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
@@ -230,7 +263,7 @@ dtst_status forward_stages(dtst_plan* p, const void* cur, int j_from, int flip, 
     cur = dst;
     flip ^= 1;
   }
-  if (p->P > 1) {
+  if (need_reduce) {
     if (cuda_failed(p, launch_reduce_partials(partial, Xhat, (long long)p->B * Cn * p->M, p->P, st))) return DTST_ERR_CUDA;
     ++p->launches;
   }
@@ -264,11 +297,12 @@ dtst_status run_forward_fused(dtst_plan* p, const float* x, float2* Xhat, int Cn
   return forward_stages(p, t1, d - 3, 1, Xhat, Cn, 1.0f, false, st);
 }
 
-// One expansion stage (B^H along dimension j) from `cur` into `dst` with whichever kernel family serves it.  The
-// last dimension's stage writes the real grid and carries the scale and the Hermitian weights.
+// One expansion stage (B^H along dimension j) from `cur` into `dst` with whichever kernel family serves it; the
+// other dimensions are in the state `contracted` says.  The last dimension's stage writes the grid and carries the
+// scale and the Hermitian weights.
 dtst_status expand_stage(dtst_plan* p, int j, int Cn, const void* cur, void* dst, float scale, bool herm,
-                         cudaStream_t st) {
-  DimOp op = make_op(p, j, false, Cn);
+                         const bool* contracted, cudaStream_t st) {
+  DimOp op = make_op(p, j, false, Cn, contracted);
   const bool out_real = (j == p->d - 1) && !p->complex_io;
   if (j == p->d - 1) {
     op.scale = scale;
@@ -300,23 +334,32 @@ dtst_status expand_stage(dtst_plan* p, int j, int Cn, const void* cur, void* dst
   return DTST_OK;
 }
 
-// Expansion stages j = 0..j_to on `cur` (complex), ping-ponging through the workspace; returns the buffer
-// holding the result through *out_buf (cur_in itself when j_to < 0).
-dtst_status inverse_stages_complex(dtst_plan* p, const float2* cur_in, int j_to, int Cn, const float2** out_buf,
-                                   cudaStream_t st) {
+// Expansion of the dimensions 0..j_top (the forward contraction order walked backwards; `skip`, if >= 0, is left to
+// the caller and must come last) on `cur`, ping-ponging through the workspace; returns the buffer holding the
+// result through *out_buf (cur_in itself when nothing is expanded) and the number of stages through *stages.
+dtst_status inverse_stages_complex(dtst_plan* p, const float2* cur_in, int j_top, int skip, int Cn,
+                                   const float2** out_buf, int* stages, cudaStream_t st) {
   const WsLayout L = ws_layout(p);
   char* ws = static_cast<char*>(p->ws);
   float2* buf[2] = {reinterpret_cast<float2*>(ws + L.bufA), reinterpret_cast<float2*>(ws + L.bufB)};
   const void* cur = cur_in;
-  int flip = 0;
-  for (int j = 0; j <= j_to; ++j) {
+  int list[kMaxDims], n = j_top >= 0 ? middle_order(p, j_top, list) : 0;
+  bool contracted[kMaxDims];
+  for (int i = 0; i < p->d; ++i) contracted[i] = true;
+  int flip = 0, done = 0;
+  for (int idx = n - 1; idx >= 0; --idx) {
+    const int j = list[idx];
+    if (j == skip) continue;
     void* dst = buf[flip];
-    const dtst_status s = expand_stage(p, j, Cn, cur, dst, 1.0f, false, st);
+    const dtst_status s = expand_stage(p, j, Cn, cur, dst, 1.0f, false, contracted, st);
     if (s != DTST_OK) return s;
+    contracted[j] = false;
     cur = dst;
     flip ^= 1;
+    ++done;
   }
   *out_buf = static_cast<const float2*>(cur);
+  if (stages) *stages = done;
   return DTST_OK;
 }
 
@@ -324,9 +367,11 @@ dtst_status inverse_stages_complex(dtst_plan* p, const float2* cur_in, int j_to,
 dtst_status run_inverse_generic(dtst_plan* p, const float2* Yhat, float* y, int Cn, float scale, bool herm,
                                 cudaStream_t st) {
   const float2* src = Yhat;
-  const dtst_status s = inverse_stages_complex(p, Yhat, p->d - 2, Cn, &src, st);
+  const dtst_status s = inverse_stages_complex(p, Yhat, p->d - 2, -1, Cn, &src, nullptr, st);
   if (s != DTST_OK) return s;
-  return expand_stage(p, p->d - 1, Cn, src, y, scale, herm, st);
+  bool contracted[kMaxDims];
+  for (int i = 0; i < p->d; ++i) contracted[i] = i == p->d - 1;
+  return expand_stage(p, p->d - 1, Cn, src, y, scale, herm, contracted, st);
 }
 
 // The dimension in front of the plane can be expanded inside the inverse plane kernel by a helper warp
@@ -336,6 +381,8 @@ bool use_colexp(const dtst_plan* p) {
   if (p->colexp_ring <= 0 || p->d < 3 || !use_fused(p)) return false;
   const int c = p->d - 3, a = p->d - 1, b = p->d - 2;
   if (!use_mid_expand(p, c)) return false;
+  int list[kMaxDims];
+  if (middle_order(p, c, list) < 1 || list[0] != c) return false;   // it must be the last dimension to be expanded
   return inv_plane_colexp_supported((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], (int)p->Ng[c], p->kmax[c]);
 }
 
@@ -347,9 +394,9 @@ dtst_status run_inverse_fused(dtst_plan* p, const float2* Yhat, float* y, int Cn
   const int d = p->d, a = d - 1, b = d - 2;
   const bool colexp = use_colexp(p);
   const float2* src = Yhat;
-  const int j_to = colexp ? d - 4 : d - 3;
-  if (j_to >= 0) {
-    dtst_status s = inverse_stages_complex(p, Yhat, j_to, Cn, &src, st);
+  int stages = 0;
+  if (d > 2) {
+    dtst_status s = inverse_stages_complex(p, Yhat, d - 3, colexp ? d - 3 : -1, Cn, &src, &stages, st);
     if (s != DTST_OK) return s;
   }
   long long planes = (long long)p->B * Cn;
@@ -360,7 +407,7 @@ dtst_status run_inverse_fused(dtst_plan* p, const float2* Yhat, float* y, int Cn
   if (colexp) {
     const int c = d - 3;
     // the ping-pong buffer the separate expansion of dimension c would have written: its first ring_cols columns
-    float2* ring = reinterpret_cast<float2*>(ws + (((j_to + 1) & 1) ? L.bufB : L.bufA));
+    float2* ring = reinterpret_cast<float2*>(ws + ((stages & 1) ? L.bufB : L.bufA));
     const long long cols = planes / p->Nl[c];
     long long ring_cols = p->colexp_ring;
     if (ring_cols > cols) ring_cols = cols;
@@ -403,7 +450,7 @@ dtst_status run_inverse_row(dtst_plan* p, const float2* Yhat, float* y, int Cn, 
   const int d = p->d, a = d - 1;
   const float2* src = Yhat;
   if (d > 1) {
-    dtst_status s = inverse_stages_complex(p, Yhat, d - 2, Cn, &src, st);
+    dtst_status s = inverse_stages_complex(p, Yhat, d - 2, -1, Cn, &src, nullptr, st);
     if (s != DTST_OK) return s;
   }
   long long rows = (long long)p->B * Cn;
@@ -447,21 +494,37 @@ WsLayout ws_layout(const dtst_plan* p) {
   WsLayout L;
   std::memset(&L, 0, sizeof(L));
   const int Cn = p->C_in > p->C_out ? p->C_in : p->C_out;
+  // Ping-pong buffers A and B: walk the stage chains of every kernel family (a plan option may switch families
+  // later) in the plan's contraction order and keep the largest tensor each buffer ever receives.
   long long a = 0, b = 0;
-  {
-    // ping-pong buffers: the forward writes stage d-1 into A, d-2 into B, ...; the
-    // expansion writes stage 0 into A, 1 into B, ...  Both directions produce the same
-    // set of intermediate shapes, walked in opposite order.
+  auto put = [&](int which, long long n) {
+    if (which == 0) a = n > a ? n : a; else b = n > b ? n : b;
+  };
+  for (int j_from = p->d - 1; j_from >= p->d - 3 && j_from >= -1; --j_from) {
+    bool contracted[kMaxDims];
+    // forward: the grid-side kernel (if any) leaves its result in A, the following stages alternate from B
+    for (int i = 0; i < p->d; ++i) contracted[i] = i > j_from;
+    int list[kMaxDims + 1], n = 0;
+    if (j_from == p->d - 1) list[n++] = p->d - 1;
+    if (j_from >= 0 || p->d >= 2) n += middle_order(p, j_from < p->d - 1 ? j_from : p->d - 2, list + n);
     int flip = 0;
-    for (int j = p->d - 1; j >= 1; --j) {
-      const long long n = fwd_stage_elems(p, j, Cn);
-      if (flip == 0) a = n > a ? n : a; else b = n > b ? n : b;
+    if (j_from < p->d - 1) {
+      put(0, state_elems(p, Cn, contracted));
+      flip = 1;
+    }
+    for (int idx = 0; idx < n; ++idx) {
+      contracted[list[idx]] = true;
+      if (idx != n - 1) put(flip, state_elems(p, Cn, contracted));
       flip ^= 1;
     }
+    // expansion: the same order backwards, every stage into a buffer, starting with A
+    for (int i = 0; i < p->d; ++i) contracted[i] = true;
+    const int j_top = j_from < p->d - 1 ? j_from : p->d - 2;
+    int m = j_top >= 0 ? middle_order(p, j_top, list) : 0;
     flip = 0;
-    for (int j = 0; j < p->d - 1; ++j) {
-      const long long n = fwd_stage_elems(p, j + 1, Cn);
-      if (flip == 0) a = n > a ? n : a; else b = n > b ? n : b;
+    for (int idx = m - 1; idx >= 0; --idx) {
+      contracted[list[idx]] = false;
+      put(flip, state_elems(p, Cn, contracted));
       flip ^= 1;
     }
   }
@@ -511,6 +574,11 @@ dtst_status dtst_plan_create_local(dtst_plan** out, int d, const int64_t N_globa
 
 dtst_status dtst_plan_set_virtual_shards(dtst_plan* p, int P) {
   if (p == nullptr || P < 1 || p->Nl[0] % P != 0) return DTST_ERR_INVALID_ARG;
+  if (P > 1 && p->d >= 2) {   // dimension 0 must be the last one contracted (see dtst_plan_set_contraction_order)
+    int list[kMaxDims];
+    const int n = middle_order(p, p->d - 2, list);
+    if (list[n - 1] != 0) return DTST_ERR_INVALID_ARG;
+  }
   p->P = P;
   return DTST_OK;
 }
@@ -518,6 +586,68 @@ dtst_status dtst_plan_set_virtual_shards(dtst_plan* p, int P) {
 dtst_status dtst_plan_set_kernel_path(dtst_plan* p, int path) {
   if (p == nullptr || (path != DTST_PATH_AUTO && path != DTST_PATH_GENERIC)) return DTST_ERR_INVALID_ARG;
   p->path_request = path;
+  return DTST_OK;
+}
+
+// bytes the stages behind the grid-side kernel move in one forward-type transform (complex64 in and out per stage)
+static double middle_stage_bytes(const dtst_plan* p) {
+  const int j_top = use_fused(p) ? p->d - 3 : p->d - 2;
+  if (j_top < 0) return 0.0;
+  int list[kMaxDims];
+  const int n = middle_order(p, j_top, list);
+  bool contracted[kMaxDims];
+  for (int i = 0; i < p->d; ++i) contracted[i] = i > j_top;
+  double bytes = 0.0;
+  for (int idx = 0; idx < n; ++idx) {
+    bytes += 8.0 * (double)state_elems(p, p->C_in, contracted);
+    contracted[list[idx]] = true;
+    bytes += 8.0 * (double)state_elems(p, p->C_in, contracted);
+  }
+  return bytes;
+}
+
+dtst_status dtst_plan_set_contraction_order(dtst_plan* p, const int32_t order[], int n) {
+  if (p == nullptr || order == nullptr || n != p->d - 1) return DTST_ERR_INVALID_ARG;
+  bool seen[kMaxDims] = {};
+  for (int i = 0; i < n; ++i) {
+    if (order[i] < 0 || order[i] > p->d - 2 || seen[order[i]]) return DTST_ERR_INVALID_ARG;
+    seen[order[i]] = true;
+  }
+  // the slab partial sums of virtual shards are added after the last stage: dimension 0 then has to be that stage
+  if (p->P > 1 && n > 0 && order[n - 1] != 0) return DTST_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) p->order_rank[order[i]] = i;
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_get_contraction_order(const dtst_plan* p, int32_t order[]) {
+  if (p == nullptr || (order == nullptr && p->d > 1)) return DTST_ERR_INVALID_ARG;
+  int list[kMaxDims];
+  const int n = p->d >= 2 ? middle_order(p, p->d - 2, list) : 0;
+  for (int i = 0; i < n; ++i) order[i] = list[i];
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_tune_contraction_order(dtst_plan* p, double* bytes_before, double* bytes_after) {
+  if (p == nullptr) return DTST_ERR_INVALID_ARG;
+  if (bytes_before) *bytes_before = middle_stage_bytes(p);
+  // the most compressing dimension first: ascending K_j / n_j; ties keep the default (higher dimension first);
+  // dimension 0 stays last when it carries virtual shards
+  int list[kMaxDims], n = 0;
+  for (int j = p->d - 2; j >= 0; --j) list[n++] = j;
+  auto before = [&](int x, int y) {
+    if (p->P > 1 && (x == 0 || y == 0)) return y == 0 && x != 0;
+    const long long lhs = (long long)p->K[x] * p->Nl[y], rhs = (long long)p->K[y] * p->Nl[x];   // K_x/n_x < K_y/n_y
+    if (lhs != rhs) return lhs < rhs;
+    return x > y;
+  };
+  for (int a = 1; a < n; ++a)
+    for (int b = a; b > 0 && before(list[b], list[b - 1]); --b) {
+      const int t = list[b];
+      list[b] = list[b - 1];
+      list[b - 1] = t;
+    }
+  for (int i = 0; i < n; ++i) p->order_rank[list[i]] = i;
+  if (bytes_after) *bytes_after = middle_stage_bytes(p);
   return DTST_OK;
 }
 

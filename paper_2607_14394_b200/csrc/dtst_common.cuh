@@ -143,6 +143,7 @@ struct dtst_plan {
   int last_cuda_error;             // cudaError_t of the last failing runtime call / launch
   unsigned dbg_poll_limit;         // 0 = default budget of the bounded waits
   long long dbg_withhold_after;    // < 0 = off (the default)
+  int order_rank[dtst::kMaxDims];  // contraction order of the dimensions behind the grid-side kernel: lower = earlier
   int complex_io;                  // 1: complex fields, two-sided retained set on the last dimension too
   int block_epilogue;              // DTST_BLOCK_EPILOGUE_*
   int require_fast;                // 1: compute calls refuse to run if any stage would take the generic kernel

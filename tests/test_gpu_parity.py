@@ -388,6 +388,81 @@ def test_more_plane_shapes_run_fused_and_match_the_oracle(case):
     run_layer_and_check(w, "auto", P=4)
 
 
+# ------------------------------------------------------------------ contraction order and pencils
+@pytest.mark.parametrize("N,k,order", [
+    ((32, 64, 16), (4, 8, 3), (0, 1)),                 # generic/folded: dimension 0 before dimension 1
+    ((32, 64, 64, 32), (8, 4, 8, 4), (0, 2, 1)),       # fused: the plane kernel keeps dims 2, 3; 0 before 1
+    ((16, 12, 8, 20), (2, 5, 3, 6), (1, 0, 2)),        # generic kernels, mixed
+    ((6, 8), (3, 4), (0,)),
+])
+def test_any_contraction_order_gives_the_same_layer(N, k, order):
+    """The result does not depend on the contraction order (Section "cuBLAS vs cuFFT"): every order meets the
+    tolerance against the oracle, forward, inverse and backward."""
+    w = I.custom_workload("order", 1, 2, 2, N, k, field="grf", seed=37)
+    x, W, g = I.make_field(w), I.make_weights(w), I.make_upstream_grad(w)
+    plan = _plan(w)
+    default = plan.contraction_order()
+    assert default == list(range(len(N) - 2, -1, -1))
+    plan.set_contraction_order(order)
+    assert plan.contraction_order() == list(order)
+    Xhat = plan.forward(_dev(x))
+    y = plan.inverse(plan.spectral_mul(Xhat, _dev(W)))
+    gx, gW = plan.backward(_dev(g), Xhat, _dev(W))
+    torch.cuda.synchronize()
+    assert plan.status() == 0
+    Wm = W.reshape((w.C_in, w.C_out) + w.K)
+    y_ref, X_ref = O.layer_forward(x, Wm, w.kmax)
+    gx_ref, gW_ref = O.backward(g, X_ref, Wm, w.kmax)
+    assert O.rel_l2(Xhat.cpu().numpy(), X_ref) <= TOL and O.rel_l2(y.cpu().numpy(), y_ref) <= TOL
+    assert O.rel_l2(gx.cpu().numpy(), gx_ref) <= TOL
+    assert O.rel_l2(gW.cpu().numpy().reshape(gW_ref.shape), gW_ref) <= TOL
+
+
+def test_order_tuner_contracts_the_most_compressing_dimension_first():
+    from paper_2607_14394_b200 import Plan, binding as Bn
+    # dimension 0 keeps 2*2 of 64 entries (ratio 1/16), dimension 1 keeps 2*12 of 32 (3/4): 0 should go first
+    w = I.custom_workload("tune", 1, 2, 2, (64, 32, 16), (2, 12, 3), field="grf", seed=41)
+    plan = _plan(w)
+    before, after = plan.tune_contraction_order()
+    assert plan.contraction_order() == [0, 1] and after < before
+    # modelled bytes: 8 bytes per complex element read and written by every stage behind the grid-side kernel
+    row = plan.kernel_path != "generic"
+    k_last = w.K[-1]
+    elems = lambda n0, n1: 2 * n0 * n1 * k_last
+    want_after = 8 * (elems(64, 32) + elems(4, 32) + elems(4, 32) + elems(4, 24))
+    want_before = 8 * (elems(64, 32) + elems(64, 24) + elems(64, 24) + elems(4, 24))
+    assert (before, after) == (want_before, want_after), (row, before, after)
+    run = plan.forward(_dev(I.make_field(w)))
+    assert O.rel_l2(run.cpu().numpy(), O.forward(I.make_field(w), w.kmax)) <= TOL
+    # with virtual shards dimension 0 has to stay last
+    p2 = Plan(w.N, w.kmax, 1, 2, 2, virtual_shards=4)
+    p2.tune_contraction_order()
+    assert p2.contraction_order()[-1] == 0
+    with pytest.raises(Bn.DtstError) as e:
+        p2.set_contraction_order((0, 1))
+    assert e.value.status == Bn.DTST_ERR_INVALID_ARG
+    with pytest.raises(Bn.DtstError):
+        plan.set_contraction_order((0, 0))
+
+
+def test_pencil_block_runs_on_the_tensor_core_slab_kernels():
+    """A rank's pencil (offsets on dimensions 0 AND 1, Section "Computing the Local Partial Spectrum") stays on the
+    streaming family: plane kernel on the last two dimensions, slab kernels with global phases on the cut ones."""
+    from paper_2607_14394_b200 import Plan
+    Ng, k, nl, off = (64, 64, 64, 32), (8, 8, 8, 4), (16, 32, 64, 32), (32, 32, 0, 0)
+    w = I.custom_workload("pencil", 1, 2, 2, Ng, k, field="grf", seed=43)
+    x = I.make_field(w)
+    blk = np.ascontiguousarray(x[:, :, 32:48, 32:64])
+    plan = Plan(nl, k, 1, 2, 2, N_global=Ng, offset=off)
+    assert plan.kernel_path == "fused"
+    plan.require_fast_path()
+    part = plan.forward(_dev(blk)).cpu().numpy()
+    assert O.rel_l2(part, O.forward(blk, k, N_global=Ng, offsets=off)) <= TOL
+    Y = I.make_spectrum(w, 2, tag=5).reshape((1, 2) + part.shape[2:])
+    yb = plan.inverse(_dev(Y)).cpu().numpy()
+    assert O.rel_l2(yb, O.inverse(Y, Ng, k, n_local=nl, offsets=off)) <= TOL
+
+
 def test_fast_path_or_fail():
     from paper_2607_14394_b200 import binding as Bn
     # an odd extent in the middle: the generic kernel would serve that dimension
