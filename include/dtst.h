@@ -327,6 +327,29 @@ dtst_status dtst_backward_mix_modes(dtst_plan* plan, const void* GY, const void*
 dtst_status dtst_backward_input(dtst_plan* plan, const void* GX, float* grad_x, void* stream);
 
 /*
+ * The whole step for callers whose activations live in HOST memory.  One step = F, M, I (Eq. 5-14) and B
+ * (Section "Backward Pass") on inputs x and grad_y that are copied in from the host and results y, grad_x and
+ * grad_W that are copied back, inside the call's work:
+ *   dtst_plan_host_io_bytes   device staging the step needs (x, grad_y, y, grad_x, two spectra, grad_W);
+ *   dtst_plan_enable_host_io  hands that staging over (device pointer, 256-byte aligned, caller-owned) and creates
+ *                             the three internal streams (copy-in, compute, copy-out) and their events - the only
+ *                             allocation; NULL switches the facility off and releases them;
+ *   dtst_step_host            enqueues one step and returns at once: hx [B, C_in, n...], hgy [B, C_out, n...] host
+ *                             (read), dW [C_in, C_out, M] complex64 DEVICE (the layer's parameter), hy, hgx, hgW
+ *                             host (written).  Transfers overlap the kernels and each other, also across
+ *                             consecutive steps (a step's copy-in runs under the previous step's backward pass).
+ *                             Use page-locked host buffers: pageable ones make the copies synchronous.  The host
+ *                             buffers of a step must stay untouched until dtst_host_io_wait has returned.
+ *   dtst_host_io_wait         blocks until the outputs of every enqueued step are in host memory.
+ * The plan needs its workspace as for the device-pointer calls.  Real plans only.
+ */
+dtst_status dtst_plan_host_io_bytes(const dtst_plan* plan, size_t* bytes);
+dtst_status dtst_plan_enable_host_io(dtst_plan* plan, void* dev_staging, size_t bytes);
+dtst_status dtst_step_host(dtst_plan* plan, const float* hx, const float* hgy, const void* dW, float* hy,
+                           float* hgx, void* hgW);
+dtst_status dtst_host_io_wait(dtst_plan* plan);
+
+/*
  * The forward partial DFT without any caller-provided or allocated scratch.
  * (The paper has no counterpart to this call; it exists for integration reasons.)
  *

@@ -42,7 +42,8 @@ EXPORTED = [
     "dtst_plan_set_block_epilogue", "dtst_pointwise_linear", "dtst_pointwise_linear_scratch_bytes",
     "dtst_pointwise_linear_backward", "dtst_plan_create_complex", "dtst_forward_complex", "dtst_inverse_complex",
     "dtst_backward_complex", "dtst_plan_set_contraction_order", "dtst_plan_get_contraction_order",
-    "dtst_plan_tune_contraction_order",
+    "dtst_plan_tune_contraction_order", "dtst_plan_host_io_bytes", "dtst_plan_enable_host_io", "dtst_step_host",
+    "dtst_host_io_wait",
 ]
 
 
@@ -98,6 +99,10 @@ def lib() -> ctypes.CDLL:
     L.dtst_backward_spectrum.argtypes = [vp, vp, vp, vp]
     L.dtst_backward_mix_modes.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_int64, ctypes.c_int64, vp]
     L.dtst_backward_input.argtypes = [vp, vp, vp, vp]
+    L.dtst_plan_host_io_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
+    L.dtst_plan_enable_host_io.argtypes = [vp, vp, ctypes.c_size_t]
+    L.dtst_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.dtst_host_io_wait.argtypes = [vp]
     L.dtst_plan_set_column_expansion.argtypes = [vp, i32]
     L.dtst_plan_require_fast_path.argtypes = [vp, i32]
     L.dtst_plan_set_block_epilogue.argtypes = [vp, i32]
@@ -720,63 +725,43 @@ class Plan:
 class HostPipeline:
     """The whole step (F, M, I, B) for callers whose activations live in pinned HOST memory.
 
-    Three CUDA streams - copy-in, compute, copy-out - are chained with events so that the PCIe transfers of
-    x and grad_y in, and of y, grad_x and grad_W out, overlap the kernels and each other, also across
-    consecutive calls of `step`.  Every byte still crosses the bus inside the call; nothing is cached.
-    W stays on the device (it is the layer's parameter).
+    A thin wrapper over `dtst_step_host`: the library chains three internal streams - copy-in, compute, copy-out -
+    with events so that the PCIe transfers of x and grad_y in, and of y, grad_x and grad_W out, overlap the
+    kernels and each other, also across consecutive calls of `step`.  Every byte still crosses the bus inside the
+    call; nothing is cached.  W stays on the device (it is the layer's parameter).
     """
 
     def __init__(self, plan: Plan, W: torch.Tensor):
         self.plan, self.W = plan, W
-        dev, p = plan.device, plan
-        self.x = torch.empty((p.B, p.C_in) + p.N, dtype=torch.float32, device=dev)
-        self.g = torch.empty((p.B, p.C_out) + p.N, dtype=torch.float32, device=dev)
-        self.Xhat = torch.empty((p.B, p.C_in) + p.K, dtype=torch.complex64, device=dev)
-        self.Yhat = torch.empty((p.B, p.C_out) + p.K, dtype=torch.complex64, device=dev)
-        self.y = torch.empty((p.B, p.C_out) + p.N, dtype=torch.float32, device=dev)
-        self.gx = torch.empty((p.B, p.C_in) + p.N, dtype=torch.float32, device=dev)
-        self.gW = torch.empty((p.C_in, p.C_out, p.M), dtype=torch.complex64, device=dev)
-        self.s_in, self.s_cmp, self.s_out = (torch.cuda.Stream(device=dev) for _ in range(3))
-        ev = lambda: torch.cuda.Event()
-        self.ev_x, self.ev_g, self.ev_fwd_read, self.ev_y, self.ev_b = ev(), ev(), ev(), ev(), ev()
-        self.ev_y_copied, self.ev_done = ev(), ev()
-        self._first = True
+        n = ctypes.c_size_t()
+        _check(lib().dtst_plan_host_io_bytes(plan.handle, ctypes.byref(n)), "dtst_plan_host_io_bytes")
+        self.staging = torch.empty(max(1, n.value), dtype=torch.uint8, device=plan.device)
+        with torch.cuda.device(plan.device):
+            _check(lib().dtst_plan_enable_host_io(plan.handle, _ptr(self.staging, torch.uint8, "staging"), n.value),
+                   "dtst_plan_enable_host_io", plan.handle)
+        self._keep = []
 
     def step(self, hx, hg, hy, hgx, hgW):
-        """Enqueue one step; all five host tensors must be pinned.  Returns immediately; call `wait()`."""
+        """Enqueue one step; all five host tensors should be pinned.  Returns immediately; call `wait()`."""
         p = self.plan
-        with torch.cuda.stream(self.s_in):
-            if not self._first:
-                self.s_in.wait_event(self.ev_fwd_read)     # previous F has consumed x
-            self.x.copy_(hx, non_blocking=True)
-            self.ev_x.record(self.s_in)
-            if not self._first:
-                self.s_in.wait_event(self.ev_b)            # previous B has consumed grad_y
-            self.g.copy_(hg, non_blocking=True)
-            self.ev_g.record(self.s_in)
-        with torch.cuda.stream(self.s_cmp):
-            self.s_cmp.wait_event(self.ev_x)
-            p.forward(self.x, self.Xhat, stream=self.s_cmp)
-            self.ev_fwd_read.record(self.s_cmp)
-            p.spectral_mul(self.Xhat, self.W, self.Yhat, stream=self.s_cmp)
-            if not self._first:
-                self.s_cmp.wait_event(self.ev_y_copied)    # previous y has left the device
-            p.inverse(self.Yhat, self.y, stream=self.s_cmp)
-            self.ev_y.record(self.s_cmp)
-            self.s_cmp.wait_event(self.ev_g)
-            if not self._first:
-                self.s_cmp.wait_event(self.ev_done)        # previous grad_x / grad_W have left the device
-            p.backward(self.g, self.Xhat, self.W, self.gx, self.gW, stream=self.s_cmp)
-            self.ev_b.record(self.s_cmp)
-        with torch.cuda.stream(self.s_out):
-            self.s_out.wait_event(self.ev_y)
-            hy.copy_(self.y, non_blocking=True)
-            self.ev_y_copied.record(self.s_out)
-            self.s_out.wait_event(self.ev_b)
-            hgx.copy_(self.gx, non_blocking=True)
-            hgW.copy_(self.gW, non_blocking=True)
-            self.ev_done.record(self.s_out)
-        self._first = False
+        for t, shape, name in ((hx, (p.B, p.C_in) + p.N, "hx"), (hgx, (p.B, p.C_in) + p.N, "hgx"),
+                               (hg, (p.B, p.C_out) + p.N, "hg"), (hy, (p.B, p.C_out) + p.N, "hy")):
+            if t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous() or tuple(t.shape) != tuple(shape):
+                raise ValueError(f"{name}: expected a contiguous float32 host tensor of shape {tuple(shape)}")
+        if (hgW.is_cuda or hgW.dtype != torch.complex64 or not hgW.is_contiguous()
+                or hgW.numel() != p.C_in * p.C_out * p.M):
+            raise ValueError("hgW: expected a contiguous complex64 host tensor of C_in*C_out*M elements")
+        p._expect(self.W, "W", "W")
+        self._keep.append((hx, hg, hy, hgx, hgW))
+        hp = lambda t: ctypes.c_void_p(t.data_ptr())
+        with torch.cuda.device(p.device):
+            _check(lib().dtst_step_host(p.handle, hp(hx), hp(hg), _ptr(self.W, torch.complex64, "W"), hp(hy), hp(hgx),
+                                        hp(hgW)), "dtst_step_host", p.handle)
 
     def wait(self):
-        self.ev_done.synchronize()
+        _check(lib().dtst_host_io_wait(self.plan.handle), "dtst_host_io_wait", self.plan.handle)
+        self._keep.clear()
+
+    def close(self):
+        if self.plan._h:
+            lib().dtst_plan_enable_host_io(self.plan._h, None, 0)

@@ -743,6 +743,7 @@ dtst_status dtst_plan_kernel_timing(dtst_plan* p, int kind, int64_t* launches, d
 dtst_status dtst_plan_destroy(dtst_plan* p) {
   if (p == nullptr) return DTST_ERR_INVALID_ARG;
   free_timing(p);
+  host_io_release(p);
   delete p;
   return DTST_OK;
 }

@@ -122,6 +122,8 @@ __device__ inline float2 dimop_entry(const DimOp& p, int r, int q, int slab) {
 
 }  // namespace dtst
 
+struct dtst_host_io;   // streams, events and staging offsets of dtst_step_host (dtst_hostio.cu)
+
 // The plan: pure host-side configuration plus a caller-owned workspace pointer.
 struct dtst_plan {
   int d;
@@ -143,6 +145,7 @@ struct dtst_plan {
   int last_cuda_error;             // cudaError_t of the last failing runtime call / launch
   unsigned dbg_poll_limit;         // 0 = default budget of the bounded waits
   long long dbg_withhold_after;    // < 0 = off (the default)
+  dtst_host_io* host_io;           // non-null after dtst_plan_enable_host_io
   int order_rank[dtst::kMaxDims];  // contraction order of the dimensions behind the grid-side kernel: lower = earlier
   int complex_io;                  // 1: complex fields, two-sided retained set on the last dimension too
   int block_epilogue;              // DTST_BLOCK_EPILOGUE_*
@@ -172,6 +175,7 @@ struct WsLayout {
 constexpr int kBlockPartialRows = 1024;   // most CTAs the bypass weight-gradient reduction is spread over
 
 bool fused_eligible(const dtst_plan* p);
+void host_io_release(dtst_plan* p);
 
 // Brackets one kernel launch with events when timing is enabled (no-ops otherwise).
 struct KernelTimer {

@@ -108,3 +108,23 @@ def test_null_handles_are_errors_not_crashes():
     assert lib.dtst_spectral_mul(h, null, null, null, null) == Bn.DTST_ERR_INVALID_ARG
     assert lib.dtst_plan_set_workspace(h, ctypes.c_void_p(128), 1 << 20) == Bn.DTST_ERR_INVALID_ARG  # misaligned
     Bn.dtst_plan_destroy(h)
+
+
+def test_host_io_argument_checks_need_no_gpu():
+    import ctypes
+    lib = Bn.lib()
+    n = ctypes.c_size_t()
+    assert lib.dtst_plan_host_io_bytes(None, ctypes.byref(n)) == Bn.DTST_ERR_INVALID_ARG
+    h = Bn.dtst_plan_create(2, (32, 64), (4, 8), 1, 2, 3)
+    try:
+        assert lib.dtst_plan_host_io_bytes(h, ctypes.byref(n)) == Bn.DTST_OK
+        grid_in, grid_out, M = 2 * 32 * 64 * 4, 3 * 32 * 64 * 4, 8 * 8
+        want = 2 * grid_in + 2 * grid_out + (2 + 3 + 6) * M * 8
+        assert want <= n.value <= want + 7 * 256       # seven regions, each rounded up to 256 bytes
+        # not enabled: a step is refused, nothing runs
+        assert lib.dtst_step_host(h, None, None, None, None, None, None) == Bn.DTST_ERR_INVALID_ARG
+        assert lib.dtst_host_io_wait(h) == Bn.DTST_ERR_INVALID_ARG
+        assert lib.dtst_plan_enable_host_io(h, ctypes.c_void_p(4), n.value) == Bn.DTST_ERR_INVALID_ARG   # misaligned
+        assert lib.dtst_plan_enable_host_io(h, None, 0) == Bn.DTST_OK                                  # off: no-op
+    finally:
+        Bn.dtst_plan_destroy(h)
