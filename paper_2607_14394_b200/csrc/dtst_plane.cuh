@@ -260,7 +260,6 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
   using Cfg = PlaneCfg<N3, K3, N2, K2>;
   constexpr int NC = Cfg::NC, QUADS = Cfg::QUADS, G = Cfg::G, LPP = Cfg::LPP;
   constexpr int SPT = Cfg::SPT, RPS = Cfg::ROWS_PER_STAGE;
-  pdl_trigger();
 
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment for the TMA swizzle, by pointer arithmetic on the shared array itself (an integer
@@ -336,22 +335,27 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
   if (warp == 0) {
     // ---------------- producer: one thread feeds the ring in task order ----------------
     if (lane == 0) {
-      long long k = 0;
-      for (long long tl = 0; tl < n_local; ++tl) {
-        const long long task = first + tl * gridDim.x;
-        for (int s = 0; s < SPT; ++s, ++k) {
-          // diagnostic (dtst_plan_debug_ring_fault): stop feeding the ring after `withhold_after` fills, so
-          // that the consumers' bounded waits run out
-          if (withhold_after >= 0 && k >= withhold_after) goto producer_done;
-          const int slot = (int)(k % stages);
-          const uint32_t ph = (uint32_t)((k / stages) & 1);
-          if (!mbar_wait_bounded(&empty[slot], ph ^ 1u, abort_flag, poll_limit)) goto producer_done;
-          fill_seq[slot] = (uint32_t)(k / stages) + 1u;
+      // slot and lap (fill number of that slot) advance incrementally: no division on the thread every load of
+      // this CTA waits for.  The diagnostic of dtst_plan_debug_ring_fault shortens the loop instead of testing
+      // inside it: after `withhold_after` fills (rounded down to whole tasks) the ring is fed no more and the
+      // consumers' bounded waits run out.
+      const long long n_feed = (withhold_after >= 0 && withhold_after / SPT < n_local) ? withhold_after / SPT : n_local;
+      uint32_t slot = 0, lap = 0;
+      for (long long tl = 0; tl < n_feed; ++tl) {
+        const int row0 = (int)((first + tl * gridDim.x) * kTaskRows);
+#pragma unroll
+        for (int s = 0; s < SPT; ++s) {
+          if (!mbar_wait_bounded(&empty[slot], (lap & 1u) ^ 1u, abort_flag)) goto producer_done;
+          fill_seq[slot] = lap + 1u;
           mbar_arrive_expect_tx(&full[slot], (uint32_t)kStageBytes);
 #pragma unroll
           for (int h = 0; h < Cfg::BOXES; ++h)
-            tma_load_2d(ring + (size_t)slot * kStageBytes + (size_t)h * RPS * 128, &in_map, h * 32,
-                        (int)(task * kTaskRows + (long long)s * RPS), &full[slot]);
+            tma_load_2d(ring + (size_t)slot * kStageBytes + (size_t)h * RPS * 128, &in_map, h * 32, row0 + s * RPS,
+                        &full[slot]);
+          if (++slot == (uint32_t)stages) {
+            slot = 0;
+            ++lap;
+          }
         }
       }
     }
@@ -371,10 +375,15 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
     // MMA fragment coordinates
     const int g8 = lane >> 2, t4 = lane & 3;
 
+    // this warp's position in the ring, advanced by W tasks per trip (no division in the loop)
+    uint32_t slot0 = (uint32_t)((w * SPT) % stages), lap0 = (uint32_t)((w * SPT) / stages);
     for (long long tl = w; tl < n_local; tl += W) {
       const long long task = first + tl * gridDim.x;
-      const long long k0 = tl * SPT;
-      const int slot0 = (int)(k0 % stages), slot1 = (int)((k0 + SPT - 1) % stages);
+      uint32_t slot1 = slot0, lap1 = lap0;
+      if (SPT == 2 && ++slot1 == (uint32_t)stages) {
+        slot1 = 0;
+        ++lap1;
+      }
       constexpr bool kSplit = (SPT == 2 && N2 == 128);   // rows a, b in the first slot, c, d in the second
 
       // ---- stage 1: the four rows of this lane's quadruple, accumulated straight into the four
@@ -383,18 +392,18 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
 #pragma unroll
       for (int c = 0; c < NC; ++c) cpp[c] = cpd[c] = cms[c] = cmd[c] = 0.f;
       if constexpr (!kSplit) {
-        if (!wait_fill(fill_seq, full, slot0, (uint32_t)(k0 / stages), abort_flag, poll_limit)) break;
-        if (SPT == 2 && !wait_fill(fill_seq, full, slot1, (uint32_t)((k0 + 1) / stages), abort_flag, poll_limit)) break;
+        if (!wait_fill(fill_seq, full, slot0, lap0, abort_flag, poll_limit)) break;
+        if (SPT == 2 && !wait_fill(fill_seq, full, slot1, lap1, abort_flag, poll_limit)) break;
       }
       bool alive = true;
 #pragma unroll 1
       for (int r4 = 0; r4 < 4; ++r4) {
         if constexpr (kSplit) {
-          if (r4 == 0) alive = wait_fill(fill_seq, full, slot0, (uint32_t)(k0 / stages), abort_flag, poll_limit);
+          if (r4 == 0) alive = wait_fill(fill_seq, full, slot0, lap0, abort_flag, poll_limit);
           if (r4 == 2) {
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[slot0]);
-            alive = wait_fill(fill_seq, full, slot1, (uint32_t)((k0 + 1) / stages), abort_flag, poll_limit);
+            alive = wait_fill(fill_seq, full, slot1, lap1, abort_flag, poll_limit);
           }
           if (!alive) break;
         }
@@ -533,9 +542,17 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
         }
       }
       __syncwarp();   // the next task's combos overwrite the A/B entries read above
+      slot0 += (uint32_t)(W * SPT);
+      while (slot0 >= (uint32_t)stages) {
+        slot0 -= (uint32_t)stages;
+        ++lap0;
+      }
     }
   }
 
+  // the dependent kernel may be scheduled from here on: triggering at the start of this kernel instead was measured
+  // slower (its blocks become resident beside this kernel's and compete for the issue slots of a kernel that needs them)
+  pdl_trigger();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) {
     // the pipeline gave up: loads that were armed but never consumed may still be in flight, and this CTA's
@@ -790,7 +807,6 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __re
   using IC = InvCfg<N3, K3, N2, K2>;
   constexpr int NC = Cfg::NC, QUADS = Cfg::QUADS, G = Cfg::G, LPP = Cfg::LPP;
   constexpr int SPT = Cfg::SPT, RPS = Cfg::ROWS_PER_STAGE;
-  pdl_trigger();
 
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment for the TMA swizzle, by pointer arithmetic on the shared array itself (an integer
@@ -1117,6 +1133,7 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __re
       tma_store_commit();
     }
   }
+  pdl_trigger();   // late, as in the forward kernel
   if (lane == 0) tma_store_wait_all<0>();
 }
 
