@@ -276,6 +276,19 @@ dtst_status run_forward_generic(dtst_plan* p, const float* x, float2* Xhat, int 
   return forward_stages(p, x, p->d - 1, 0, Xhat, Cn, scale, herm, st);
 }
 
+// Whether the forward plane kernel also contracts the dimension in front of the plane: that dimension must be the
+// first of the middle stages in the plan's order, whole on this device, without offset and not cut into slabs.
+bool use_fwd_col(const dtst_plan* p) {
+  const int d = p->d;
+  if (d < 3 || !use_fused(p)) return false;
+  const int c = d - 3;
+  int list[kMaxDims];
+  if (middle_order(p, c, list) < 1 || list[0] != c) return false;
+  if (!use_mid(p, c)) return false;
+  return fwd_plane_col_supported((int)p->Ng[d - 1], p->kmax[d - 1], (int)p->Ng[d - 2], p->kmax[d - 2], (int)p->Ng[c],
+                                 p->kmax[c]);
+}
+
 // Fused forward: the plane kernel streams the grid once and contracts the last two dimensions;
 // the remaining dimensions run on the reduced tensor.
 dtst_status run_forward_fused(dtst_plan* p, const float* x, float2* Xhat, int Cn, float scale, bool herm,
@@ -286,6 +299,22 @@ dtst_status run_forward_fused(dtst_plan* p, const float* x, float2* Xhat, int Cn
   long long planes = (long long)p->B * Cn;
   for (int i = 0; i < b; ++i) planes *= p->Nl[i];
   float2* t1 = (d == 2) ? Xhat : reinterpret_cast<float2*>(ws + L.bufA);
+  if (use_fwd_col(p)) {
+    // the third dimension is contracted inside the plane kernel: no reduced tensor in HBM, one launch less
+    const int c = d - 3;
+    float2* dst = (d == 3) ? Xhat : t1;
+    {
+      KernelTimer kt(p, DTST_KERNEL_GRID_READ, st);
+      const RingDebug dbg{p->dbg_poll_limit ? p->dbg_poll_limit : kDefaultPollLimit, p->dbg_withhold_after};
+      if (cuda_failed(p, launch_fwd_plane_col((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], (int)p->Ng[c],
+                                              p->kmax[c], x, dst, planes * p->Ng[b], scale, herm ? 1 : 0,
+                                              reinterpret_cast<int*>(ws + L.status), dbg, st)))
+        return DTST_ERR_CUDA;
+    }
+    ++p->launches;
+    if (d == 3) return DTST_OK;
+    return forward_stages(p, t1, d - 4, 1, Xhat, Cn, 1.0f, false, st);
+  }
   {
     KernelTimer kt(p, DTST_KERNEL_GRID_READ, st);
     const RingDebug dbg{p->dbg_poll_limit ? p->dbg_poll_limit : kDefaultPollLimit, p->dbg_withhold_after};

@@ -3,12 +3,15 @@
 // instantiated in dtst_plane_inst_*.cu.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "dtst_plane.cuh"
 
 namespace dtst {
 
 namespace plane {
 DTST_PLANE_SHAPES(DTST_PLANE_EXTERN)
+DTST_PLANE_COL_SHAPES(DTST_PLANE_COL_EXTERN)
 }
 
 namespace {
@@ -95,6 +98,29 @@ cudaError_t launch_fwd_plane(int N3, int K3, int N2, int K2, const float* x, flo
 #define DTST_CALL(a, b, c, d) \
   if (N3 == a && K3 == b && N2 == c && K2 == d) return plane::plane_fwd<a, b, c, d>(x, out, rows, scale, herm, status, dbg, st);
   DTST_PLANE_SHAPES(DTST_CALL)
+#undef DTST_CALL
+  return cudaErrorNotSupported;
+}
+
+// N1 must divide 8 K1 (the unpaired mode's phase then depends on a plane's place in its batch of 8 only), hold both
+// retained halves and fit the kernel's cosine table.
+bool fwd_plane_col_supported(int N3, int K3, int N2, int K2, int N1, int K1) {
+  static const bool off = std::getenv("DTST_NO_COLFUSE") != nullptr;   // diagnostic: keep the two-launch path
+  if (off) return false;
+  bool shape = false;
+#define DTST_MATCH(a, b, c, d, e) if (N3 == a && K3 == b && N2 == c && K2 == d && K1 == e) shape = true;
+  DTST_PLANE_COL_SHAPES(DTST_MATCH)
+#undef DTST_MATCH
+  return shape && N1 % 8 == 0 && N1 <= 128 && N1 >= 2 * K1 && (8 * K1) % N1 == 0;
+}
+
+cudaError_t launch_fwd_plane_col(int N3, int K3, int N2, int K2, int N1, int K1, const float* x, float2* out,
+                                 long long rows, float scale, int herm, int* status, const RingDebug& dbg,
+                                 cudaStream_t st) {
+#define DTST_CALL(a, b, c, d, e)                                    \
+  if (N3 == a && K3 == b && N2 == c && K2 == d && K1 == e)          \
+    return plane::plane_fwd_col<a, b, c, d, e>(x, out, rows, N1, scale, herm, status, dbg, st);
+  DTST_PLANE_COL_SHAPES(DTST_CALL)
 #undef DTST_CALL
   return cudaErrorNotSupported;
 }

@@ -12,6 +12,13 @@ namespace dtst {
 cudaError_t launch_fwd_plane(int N3, int K3, int N2, int K2, const float* x, float2* out, long long rows,
                              float scale, int herm, int* status, const RingDebug& dbg, cudaStream_t st);
 
+// The same with the third dimension (the one in front of the plane: extent N1, whole and without offset, K1 modes
+// per side) contracted inside the kernel: out[columns][2 K1][2 K2][K3], columns = rows / (N2 N1).
+bool fwd_plane_col_supported(int N3, int K3, int N2, int K2, int N1, int K1);
+cudaError_t launch_fwd_plane_col(int N3, int K3, int N2, int K2, int N1, int K1, const float* x, float2* out,
+                                 long long rows, float scale, int herm, int* status, const RingDebug& dbg,
+                                 cudaStream_t st);
+
 // Inverse plane kernel: in[planes][2*K2][K3] complex -> real rows [rows][N3].
 cudaError_t launch_inv_plane(int N3, int K3, int N2, int K2, const float2* in, float* y, long long rows,
                              float scale, int herm, int* status, cudaStream_t st);

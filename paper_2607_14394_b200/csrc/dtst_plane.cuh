@@ -33,6 +33,7 @@ namespace plane {
 using namespace sm100;
 
 constexpr int kTaskRows = 128;       // rows of the contiguous dimension per warp task
+constexpr int kColAccWarps = 4;      // accumulator warps of the forward kernel's fused third dimension
 constexpr int kStageBytes = 16384;   // one ring slot
 constexpr int kSmemLimit = 232448;   // 227 KB opt-in limit per CTA
 
@@ -131,18 +132,18 @@ struct SmemPlan {
 };
 
 template <typename Cfg, int K2, int K3, int W>
-SmemPlan smem_plan() {
+SmemPlan smem_plan(size_t extra = 0) {   // extra: bytes behind the barrier block (fused third dimension)
   SmemPlan s;
   const size_t combos = (size_t)W * Cfg::COMBO_FLOATS * 4 + (size_t)Cfg::BTAB_FLOAT4 * 16;
   const size_t rot = (size_t)2 * K2 * K3 * 8;
-  const size_t fixed = 1024 /*alignment slack*/ + combos + rot + 512 /*barriers*/;
+  const size_t fixed = 1024 /*alignment slack*/ + combos + rot + 512 /*barriers*/ + extra;
   s.stages = (int)((kSmemLimit - fixed) / kStageBytes);
   if (s.stages > 12) s.stages = 12;
   s.ring = 0;
   s.combos = (size_t)s.stages * kStageBytes;
   s.rot = s.combos + combos;
   s.bars = s.rot + rot;
-  s.total = s.bars + 512 + 1024;
+  s.total = s.bars + 512 + extra + 1024;
   return s;
 }
 
@@ -253,13 +254,31 @@ __device__ __forceinline__ bool wait_fill(volatile uint32_t* fill_seq, uint64_t*
   return __all_sync(0xffffffffu, ok) != 0;
 }
 
-template <int N3, int K3, int N2, int K2, int W>
-__global__ void __launch_bounds__((W + 1) * 32, 1)
+// All lanes of a warp wait for a phase of an mbarrier and leave with one verdict.
+__device__ __forceinline__ bool wait_bar_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
+  const bool ok = mbar_wait_bounded(bar, parity, abort_flag, limit);
+  return __all_sync(0xffffffffu, ok) != 0;
+}
+
+// K1 > 0: the THIRD dimension (the one in front of the plane, extent N1, K1 retained modes per side) is contracted
+// inside this kernel too.  A CTA then takes whole columns (the N1 consecutive planes that share their leading
+// indices); the consumer warps put each finished plane - [2 k2][k3] complex, 2 KB - into a double-buffered batch of
+// 8 planes in shared memory instead of writing it to HBM, and kColAccWarps further warps contract every complete
+// batch into the column's [2 k1][2 k2][k3] accumulator, which lives in their MMA C fragments:
+//   C_g[m] += sum_k cos(2 pi g n_k / N1) v_k[m],  S_g[m] += sum_k sin(..) v_k[m]     (TF32 hi/lo, 16 x 8 x 8 MMAs)
+//   Z_{+g} = C_g - i S_g,  Z_{-g} = C_g + i S_g  at the column's end;  Z_{-K1} = sum_n v_n e^{+2 pi i K1 n / N1} in FFMA.
+// The reduced tensor of the plane stage ([planes][2 k2][k3], 6 % of the bytes of a transform, written and read once)
+// and the launch that contracted it disappear.  Twelve warps: every warp is capped at 168 registers.
+template <int N3, int K3, int N2, int K2, int W, int K1>
+__global__ void __launch_bounds__((W + 1 + (K1 > 0 ? kColAccWarps : 0)) * 32, 1)
 fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict__ out, long long num_tasks, float scale, int herm, int stages,
-                 int* __restrict__ status, uint32_t poll_limit, long long withhold_after) {
+                 int* __restrict__ status, uint32_t poll_limit, long long withhold_after, int N1) {
   using Cfg = PlaneCfg<N3, K3, N2, K2>;
   constexpr int NC = Cfg::NC, QUADS = Cfg::QUADS, G = Cfg::G, LPP = Cfg::LPP;
   constexpr int SPT = Cfg::SPT, RPS = Cfg::ROWS_PER_STAGE;
+  constexpr bool COLS = K1 > 0;
+  constexpr int PCOLS = 2 * (2 * K2) * K3;   // floats of one finished plane
+  static_assert(!COLS || (G == 1 && K1 == 16 && PCOLS % (64 * kColAccWarps) == 0), "fused third dimension: shape");
 
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment for the TMA swizzle, by pointer arithmetic on the shared array itself (an integer
@@ -277,6 +296,12 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
   // tell "this phase" from "the previous one", so a consumer that is a whole lap of the ring ahead
   // must first see its fill armed (which implies every earlier fill of the slot has landed).
   volatile uint32_t* fill_seq = reinterpret_cast<volatile uint32_t*>(empty + 16) + 4;
+  // fused third dimension: batch complete / batch consumed barriers (inside the 512-byte barrier block), the two
+  // batches of finished planes and the cosine table cos(2 pi j / N1)
+  uint64_t* pfull = full + 44;
+  uint64_t* pfree = full + 46;
+  float* pbuf = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(full) + 512);
+  float* ctab = pbuf + 2 * 8 * PCOLS;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -287,9 +312,17 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
       fill_seq[s] = 0;
     }
     *abort_flag = 0;
+    if constexpr (COLS) {
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(&pfull[i], 8);
+        mbar_init(&pfree[i], kColAccWarps);
+      }
+    }
     fence_barrier_init();
     prefetch_tensormap(&in_map);
   }
+  if constexpr (COLS)
+    for (int e = threadIdx.x; e < N1; e += blockDim.x) ctab[e] = (float)cospi(2.0 * (double)e / (double)N1);
   // Stage-2 basis as MMA B fragments (k = quadruple n, n = frequency slot of the parity class), TF32 hi/lo,
   // generated once per CTA: entry [cls][ks][lane] = (b0 hi, b1 hi, b0 lo, b1 lo).  Classes: 0 = A even (pp,
   // cos), 1 = A odd (pd, cos), 2 = B odd (ms, sin), 3 = B even (md, sin); 4 = the unpaired A_{K2} (cos, shares
@@ -330,7 +363,14 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
   pdl_wait();   // everything above is independent of the preceding kernel
 
   const long long first = blockIdx.x;
-  const long long n_local = first < num_tasks ? (num_tasks - first + gridDim.x - 1) / gridDim.x : 0;
+  long long n_local;
+  if constexpr (COLS) {
+    // a task is one plane; this CTA takes the columns first, first + grid, ..: N1 consecutive planes each
+    const long long cols = num_tasks / N1;
+    n_local = first < cols ? ((cols - first + gridDim.x - 1) / gridDim.x) * N1 : 0;
+  } else {
+    n_local = first < num_tasks ? (num_tasks - first + gridDim.x - 1) / gridDim.x : 0;
+  }
 
   if (warp == 0) {
     // ---------------- producer: one thread feeds the ring in task order ----------------
@@ -341,8 +381,19 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
       // consumers' bounded waits run out.
       const long long n_feed = (withhold_after >= 0 && withhold_after / SPT < n_local) ? withhold_after / SPT : n_local;
       uint32_t slot = 0, lap = 0;
+      long long pcol0 = first * N1;   // fused third dimension: first plane of the current column, plane within it
+      int pn = 0;
       for (long long tl = 0; tl < n_feed; ++tl) {
-        const int row0 = (int)((first + tl * gridDim.x) * kTaskRows);
+        int row0;
+        if constexpr (COLS) {
+          row0 = (int)((pcol0 + pn) * kTaskRows);
+          if (++pn == N1) {
+            pn = 0;
+            pcol0 += (long long)gridDim.x * N1;
+          }
+        } else {
+          row0 = (int)((first + tl * gridDim.x) * kTaskRows);
+        }
 #pragma unroll
         for (int s = 0; s < SPT; ++s) {
           if (!mbar_wait_bounded(&empty[slot], (lap & 1u) ^ 1u, abort_flag)) goto producer_done;
@@ -361,9 +412,10 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
     }
   producer_done:
     __syncwarp();
-  } else {
+  } else if (!COLS || warp <= W) {
     // ---------------- consumers: one warp per task ----------------
     const int w = warp - 1;
+    int ct = w;   // fused third dimension: this warp's task as a CTA-local count (batch = ct / 8, place = ct % 8)
     float* combo = combos_all + (size_t)w * Cfg::COMBO_FLOATS;
 
     // stage-1 role: lane = (plane in task, row quadruple)
@@ -515,6 +567,11 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
           }
       __syncwarp();
 
+      if constexpr (COLS) {
+        // the accumulator warps must be done with the batch that used this buffer before
+        const int u = ct >> 4;
+        if (u > 0 && !wait_bar_warp(&pfree[(ct >> 3) & 1], (uint32_t)(u - 1) & 1u, abort_flag, poll_limit)) break;
+      }
       // epilogue: Z_{+g} = rho (A - iB), Z_{-g} = rho (A + iB) with A = AC - i AS, B = BC - i BS
       if (act2) {
         const int r = l2;
@@ -523,6 +580,11 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
         const float* A = combo + pl2 * Cfg::ABP + g * Cfg::ABS;
         const float* Bp = combo + pl2 * Cfg::ABP + (K2 + g) * Cfg::ABS;
         float2* dst = out + ((task * G + pl2) * (2 * K2) + r) * K3;
+        // fused third dimension: place ct % 8 of batch ct / 8; the 8-float groups of a plane are permuted by its
+        // place so that the accumulator warps' fragment loads (four planes x eight columns per request) hit 32
+        // different banks
+        float* prow = pbuf + (size_t)(((ct >> 3) & 1) * 8 + (ct & 7)) * PCOLS;
+        const int swz = (ct & 3) << 3;
         const float2* rr = rot + r;
 #pragma unroll
         for (int f2 = 0; f2 < K3 / 2; ++f2) {
@@ -538,14 +600,99 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
             res[2 * e] = ro.x * wr - ro.y * wi;
             res[2 * e + 1] = ro.x * wi + ro.y * wr;
           }
-          *reinterpret_cast<float4*>(dst + 2 * f2) = make_float4(res[0], res[1], res[2], res[3]);
+          if constexpr (COLS)
+            *reinterpret_cast<float4*>(prow + ((r * 2 * K3 + 4 * f2) ^ swz)) = make_float4(res[0], res[1], res[2], res[3]);
+          else
+            *reinterpret_cast<float4*>(dst + 2 * f2) = make_float4(res[0], res[1], res[2], res[3]);
         }
       }
       __syncwarp();   // the next task's combos overwrite the A/B entries read above
+      if constexpr (COLS) {
+        if (lane == 0) mbar_arrive(&pfull[(ct >> 3) & 1]);   // this plane is in its batch (release after the __syncwarp)
+        ct += W;
+      }
       slot0 += (uint32_t)(W * SPT);
       while (slot0 >= (uint32_t)stages) {
         slot0 -= (uint32_t)stages;
         ++lap0;
+      }
+    }
+  } else {
+    if constexpr (COLS) {
+      // ---------------- accumulator warps: contract every complete batch of 8 planes along the third dimension ---
+      const int a = warp - (W + 1);
+      const int g8 = lane >> 2, t4 = lane & 3;
+      constexpr int NTW = (PCOLS / 8) / kColAccWarps;   // n-tiles of 8 real columns per warp
+      constexpr int INNER = PCOLS / 2;                  // complex values per plane
+      const int qN = N1 - (N1 >> 2);                    // sin x = cos(x - pi/2): index shift in the cosine table
+      float accC[NTW][4], accS[NTW][4];
+      float z16[4];                                     // Z_{-K1} of this lane's two complex columns
+#pragma unroll
+      for (int nt = 0; nt < NTW; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) accC[nt][e] = accS[nt][e] = 0.f;
+      z16[0] = z16[1] = z16[2] = z16[3] = 0.f;
+      const int nb = (int)(n_local >> 3), bpc = N1 >> 3;
+      long long col = first;
+      int bc = 0;                                       // batch within the column
+      for (int b = 0; b < nb; ++b) {
+        const int buf = b & 1;
+        if (!wait_bar_warp(&pfull[buf], (uint32_t)(b >> 1) & 1u, abort_flag, poll_limit)) break;
+        const float* pb = pbuf + (size_t)buf * 8 * PCOLS;
+        // basis fragments of this batch: rows = frequencies g8, g8 + 8; columns = planes n = 8 bc + t4, + 4
+        uint32_t chi[4], clo[4], shi[4], slo[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int g = g8 + 8 * (e & 1), n = 8 * bc + t4 + 4 * (e >> 1);
+          const int idx = (g * n) % N1;
+          split_tf32_rna(ctab[idx], chi[e], clo[e]);
+          split_tf32_rna(ctab[(idx + qN) % N1], shi[e], slo[e]);
+        }
+        const int sw = t4 << 3;   // planes t4 and t4 + 4 carry the same permutation
+#pragma unroll
+        for (int nt = 0; nt < NTW; ++nt) {
+          const int c0 = (8 * (NTW * a + nt) + g8) ^ sw;
+          uint32_t bh0, bl0, bh1, bl1;
+          split_tf32_round(pb[t4 * PCOLS + c0], bh0, bl0);
+          split_tf32_round(pb[(t4 + 4) * PCOLS + c0], bh1, bl1);
+          mma3_tf32(accC[nt], chi, clo, bh0, bh1, bl0, bl1);
+          mma3_tf32(accS[nt], shi, slo, bh0, bh1, bl0, bl1);
+        }
+        // the unpaired mode -K1: e^{+2 pi i K1 n / N1} depends on the place in the batch only (8 K1 / N1 is whole)
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int idx = (K1 * k) % N1;
+          const float cs = ctab[idx], sn = ctab[(idx + qN) % N1];
+          const float4 v = *reinterpret_cast<const float4*>(pb + k * PCOLS + ((2 * INNER / kColAccWarps * a + 4 * lane) ^ ((k & 3) << 3)));
+          z16[0] = fmaf(v.x, cs, fmaf(-v.y, sn, z16[0]));
+          z16[1] = fmaf(v.x, sn, fmaf(v.y, cs, z16[1]));
+          z16[2] = fmaf(v.z, cs, fmaf(-v.w, sn, z16[2]));
+          z16[3] = fmaf(v.z, sn, fmaf(v.w, cs, z16[3]));
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&pfree[buf]);
+        if (++bc == bpc) {
+          // the column is complete: Z_{+g} = C_g - i S_g (position g), Z_{-g} = C_g + i S_g (position 2 K1 - g)
+          float2* ob = out + col * (2 * K1) * INNER;
+#pragma unroll
+          for (int nt = 0; nt < NTW; ++nt) {
+            const int m = 4 * (NTW * a + nt) + t4;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int g = g8 + 8 * h;
+              const float cx = accC[nt][2 * h], cy = accC[nt][2 * h + 1];
+              const float sx = accS[nt][2 * h], sy = accS[nt][2 * h + 1];
+              ob[(long long)g * INNER + m] = make_float2(cx + sy, cy - sx);
+              if (g > 0) ob[(long long)(2 * K1 - g) * INNER + m] = make_float2(cx - sy, cy + sx);
+              accC[nt][2 * h] = accC[nt][2 * h + 1] = accS[nt][2 * h] = accS[nt][2 * h + 1] = 0.f;
+            }
+          }
+          *reinterpret_cast<float4*>(ob + (long long)K1 * INNER + INNER / kColAccWarps * a + 2 * lane) =
+              make_float4(z16[0], z16[1], z16[2], z16[3]);
+          z16[0] = z16[1] = z16[2] = z16[3] = 0.f;
+          bc = 0;
+          col += gridDim.x;
+        }
       }
     }
   }
@@ -1148,13 +1295,37 @@ cudaError_t plane_fwd(const float* x, float2* out, long long rows, float scale, 
   if (sp.stages < 2 * Cfg::SPT) return cudaErrorInvalidConfiguration;
   CUtensorMap map;
   if (!make_rows_map(&map, x, rows, N3, Cfg::ROWS_PER_STAGE)) return cudaErrorNotSupported;
-  auto kern = fwd_plane_kernel<N3, K3, N2, K2, W>;
+  auto kern = fwd_plane_kernel<N3, K3, N2, K2, W, 0>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sp.total);
   if (e != cudaSuccess) return e;
   const long long tasks = rows / kTaskRows;
   const int grid = (int)(tasks < num_sms() ? tasks : num_sms());
   (void)launch_pdl(kern, dim3(grid), dim3((W + 1) * 32), sp.total, st, map, out, tasks, scale, herm, sp.stages, status,
-                   dbg.poll_limit, dbg.withhold_after);
+                   dbg.poll_limit, dbg.withhold_after, 0);
+  return cudaGetLastError();
+}
+
+// The forward kernel with the third dimension (extent N1, K1 modes per side) contracted on chip: x rows as above,
+// out [columns][2 K1][2 k2][k3] complex, columns = rows / (N2 N1).
+template <int N3, int K3, int N2, int K2, int K1>
+cudaError_t plane_fwd_col(const float* x, float2* out, long long rows, int N1, float scale, int herm, int* status,
+                          const RingDebug& dbg, cudaStream_t st) {
+  constexpr int W = 7;
+  using Cfg = PlaneCfg<N3, K3, N2, K2>;
+  static_assert(Cfg::G == 1, "one plane per task");
+  const size_t extra = (size_t)2 * 8 * (2 * 2 * K2 * K3) * 4 + 512;   // two batches of 8 planes, the cosine table
+  const SmemPlan sp = smem_plan<Cfg, K2, K3, W>(extra);
+  if (sp.stages < 2 * Cfg::SPT || N1 > 128) return cudaErrorInvalidConfiguration;
+  CUtensorMap map;
+  if (!make_rows_map(&map, x, rows, N3, Cfg::ROWS_PER_STAGE)) return cudaErrorNotSupported;
+  auto kern = fwd_plane_kernel<N3, K3, N2, K2, W, K1>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sp.total);
+  if (e != cudaSuccess) return e;
+  const long long tasks = rows / kTaskRows;   // planes
+  const long long cols = tasks / N1;
+  const int grid = (int)(cols < num_sms() ? cols : num_sms());
+  (void)launch_pdl(kern, dim3(grid), dim3((W + 1 + kColAccWarps) * 32), sp.total, st, map, out, tasks, scale, herm,
+                   sp.stages, status, dbg.poll_limit, dbg.withhold_after, N1);
   return cudaGetLastError();
 }
 
@@ -1206,6 +1377,15 @@ cudaError_t plane_inv(const float2* in, float* y, long long rows, float scale, i
                                                                const ColExpandArgs&, cudaStream_t);                      \
   extern template cudaError_t plane_inv<N3, K3, N2, K2, K2, N2 / 32>(const float2*, float*, long long, float, int,       \
                                                                       const ColExpandArgs&, cudaStream_t);
+
+// The forward kernel with the third dimension fused is built for the largest benchmark shape.
+#define DTST_PLANE_COL_SHAPES(X) X(64, 8, 128, 16, 16)
+#define DTST_PLANE_COL_INSTANTIATE(N3, K3, N2, K2, K1)                                                                  \
+  template cudaError_t plane_fwd_col<N3, K3, N2, K2, K1>(const float*, float2*, long long, int, float, int, int*,       \
+                                                          const RingDebug&, cudaStream_t);
+#define DTST_PLANE_COL_EXTERN(N3, K3, N2, K2, K1)                                                                       \
+  extern template cudaError_t plane_fwd_col<N3, K3, N2, K2, K1>(const float*, float2*, long long, int, float, int,      \
+                                                                 int*, const RingDebug&, cudaStream_t);
 
 }  // namespace plane
 }  // namespace dtst

@@ -388,6 +388,28 @@ def test_more_plane_shapes_run_fused_and_match_the_oracle(case):
     run_layer_and_check(w, "auto", P=4)
 
 
+# ------------------------------------------------------------------ third dimension inside the forward plane kernel
+@pytest.mark.parametrize("N,k,B,C,P", [
+    ((32, 128, 64), (16, 16, 8), 1, 3, 1),        # d = 3: the kernel writes the spectrum itself; N1 = 2 k1 (all of dim 0)
+    ((64, 128, 64), (16, 16, 8), 2, 2, 1),        # four columns on four CTAs
+    ((3, 128, 128, 64), (1, 16, 16, 8), 1, 1, 1), # N1 = 128: sixteen batches per column; a stage behind the kernel
+    ((4, 64, 128, 64), (2, 16, 16, 8), 1, 2, 2),  # virtual shards on dimension 0 behind the fused kernel
+])
+def test_forward_with_the_third_dimension_fused(N, k, B, C, P):
+    """Shapes whose forward-type transforms contract three dimensions in one kernel (columns of planes accumulated
+    in the MMA fragments of extra warps): forward, inverse and backward against the oracle."""
+    w = I.custom_workload("colfuse", B, C, C, N, k, field="grf", seed=47)
+    plan = _plan(w, "auto", P)
+    assert plan.kernel_path == "fused"
+    # one launch per forward: plane kernel (+ one per remaining dimension)
+    before = plan.launch_count()
+    plan.forward(_dev(I.make_field(w)))
+    torch.cuda.synchronize()
+    assert plan.launch_count() - before <= 1 + (len(N) - 3) + (1 if P > 1 else 0)   # (+ the slab reduction)
+    plan.close()
+    run_layer_and_check(w, "auto", P=P)
+
+
 # ------------------------------------------------------------------ contraction order and pencils
 @pytest.mark.parametrize("N,k,order", [
     ((32, 64, 16), (4, 8, 3), (0, 1)),                 # generic/folded: dimension 0 before dimension 1
