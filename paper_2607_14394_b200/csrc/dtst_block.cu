@@ -316,6 +316,22 @@ cudaError_t launch_linear_backward(const float* gz, const float* x, float* gx, i
                                    long long* launches) {
   const long long tiles = (long long)B * ((P + kTP - 1) / kTP);
   if (tiles <= 0) return cudaSuccess;
+  if (linear_backward_mma_supported(Ci, Co, P)) {
+    // 16 or 32 channels on both sides: both products on the tensor cores (dtst_block_mma.cu)
+    const int want = (gWb != nullptr || gb != nullptr) ? 1 : 0;
+    int rows = 0;
+    cudaError_t em = launch_linear_backward_mma(gz, x, gx, gx != nullptr ? mode_gx : 0, Wb, partial, B, Ci, Co, P, want,
+                                                gb != nullptr ? 1 : 0, kBlockPartialRows, &rows, st);
+    if (em != cudaSuccess) return em;
+    if (launches) ++*launches;
+    if (want) {
+      const int pairs = Ci * Co;
+      (void)launch_pdl(reduce_wb_kernel, dim3((unsigned)((pairs + Co + 255) / 256)), dim3(256), 0, st,
+                       static_cast<const float*>(partial), gWb, gb, pairs, Co, rows);
+      if (launches) ++*launches;
+    }
+    return cudaGetLastError();
+  }
   size_t smem = (size_t)(((Ci * Co + 3) & ~3) + (Ci + Co) * kTS) * 4;
   const size_t red_bytes = (size_t)(((Ci * Co + 3) & ~3) + 256 * 16) * 4;   // the final reduction's scratch
   if (smem < red_bytes) smem = red_bytes;

@@ -102,8 +102,8 @@ cudaError_t launch_fwd_plane(int N3, int K3, int N2, int K2, const float* x, flo
   return cudaErrorNotSupported;
 }
 
-// N1 must divide 8 K1 (the unpaired mode's phase then depends on a plane's place in its batch of 8 only), hold both
-// retained halves and fit the kernel's cosine table.
+// N1 must be a power of two that divides 8 K1 (the unpaired mode's phase then depends on a plane's place in its
+// batch of 8 only), hold both retained halves and fit the kernel's cosine table.
 bool fwd_plane_col_supported(int N3, int K3, int N2, int K2, int N1, int K1) {
   static const bool off = std::getenv("DTST_NO_COLFUSE") != nullptr;   // diagnostic: keep the two-launch path
   if (off) return false;
@@ -111,7 +111,7 @@ bool fwd_plane_col_supported(int N3, int K3, int N2, int K2, int N1, int K1) {
 #define DTST_MATCH(a, b, c, d, e) if (N3 == a && K3 == b && N2 == c && K2 == d && K1 == e) shape = true;
   DTST_PLANE_COL_SHAPES(DTST_MATCH)
 #undef DTST_MATCH
-  return shape && N1 % 8 == 0 && N1 <= 128 && N1 >= 2 * K1 && (8 * K1) % N1 == 0;
+  return shape && N1 >= 8 && (N1 & (N1 - 1)) == 0 && N1 <= 128 && N1 >= 2 * K1 && (8 * K1) % N1 == 0;
 }
 
 cudaError_t launch_fwd_plane_col(int N3, int K3, int N2, int K2, int N1, int K1, const float* x, float2* out,

@@ -625,6 +625,7 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
       constexpr int NTW = (PCOLS / 8) / kColAccWarps;   // n-tiles of 8 real columns per warp
       constexpr int INNER = PCOLS / 2;                  // complex values per plane
       const int qN = N1 - (N1 >> 2);                    // sin x = cos(x - pi/2): index shift in the cosine table
+      const int nm = N1 - 1;                            // N1 is a power of two: indices reduce with a mask
       float accC[NTW][4], accS[NTW][4];
       float z16[4];                                     // Z_{-K1} of this lane's two complex columns
 #pragma unroll
@@ -644,9 +645,9 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int g = g8 + 8 * (e & 1), n = 8 * bc + t4 + 4 * (e >> 1);
-          const int idx = (g * n) % N1;
+          const int idx = (g * n) & nm;
           split_tf32_rna(ctab[idx], chi[e], clo[e]);
-          split_tf32_rna(ctab[(idx + qN) % N1], shi[e], slo[e]);
+          split_tf32_rna(ctab[(idx + qN) & nm], shi[e], slo[e]);
         }
         const int sw = t4 << 3;   // planes t4 and t4 + 4 carry the same permutation
 #pragma unroll
@@ -661,8 +662,8 @@ fwd_plane_kernel(const __grid_constant__ CUtensorMap in_map, float2* __restrict_
         // the unpaired mode -K1: e^{+2 pi i K1 n / N1} depends on the place in the batch only (8 K1 / N1 is whole)
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          const int idx = (K1 * k) % N1;
-          const float cs = ctab[idx], sn = ctab[(idx + qN) % N1];
+          const int idx = (K1 * k) & nm;
+          const float cs = ctab[idx], sn = ctab[(idx + qN) & nm];
           const float4 v = *reinterpret_cast<const float4*>(pb + k * PCOLS + ((2 * INNER / kColAccWarps * a + 4 * lane) ^ ((k & 3) << 3)));
           z16[0] = fmaf(v.x, cs, fmaf(-v.y, sn, z16[0]));
           z16[1] = fmaf(v.x, sn, fmaf(v.y, cs, z16[1]));
