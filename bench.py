@@ -150,8 +150,8 @@ class ClockSampler:
 NCU_TRAFFIC = {
     "cfg5_4d_128": {
         "channels": (2, 4),
-        "grid_read": (1138479500, 2277482880),      # read + write bytes per launch at 2 and at 4 channels
-        "grid_write": (1080677000, 2218299264),
+        "grid_read": (1087604500, 2178791168),      # read + write bytes per launch at 2 and at 4 channels
+        "grid_write": (1080980500, 2218048512),
         "source": "profiles/plane_kernels_cfg5_shape_c2_c4_ncu.md",
     },
 }

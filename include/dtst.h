@@ -439,6 +439,8 @@ dtst_status dtst_plan_last_cuda_error(const dtst_plan* plan, int* code, const ch
 /*
  * Diagnostics read once from the environment (for A/B measurements; not for production use):
  *   DTST_NO_PDL=1            launch every kernel without the programmatic-dependent-launch attribute
+ *   DTST_NO_COLFUSE=1        forward-type transforms: contract the third dimension in a launch of its own instead of
+ *                            inside the kernel that streams the grid (shapes for which that kernel exists)
  */
 const char* dtst_status_string(dtst_status s);
 

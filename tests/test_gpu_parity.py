@@ -301,13 +301,16 @@ def test_argument_errors_on_device():
     assert plan.launch_count() > before
 
 
-def test_bounded_wait_runs_out_and_is_reported_once():
+@pytest.mark.parametrize("which", ["plane", "plane_with_third_dimension"])
+def test_bounded_wait_runs_out_and_is_reported_once(which):
     """The failure-reporting path of the streaming kernels, made to happen on the host's request: the forward
-    plane kernel's producer stops feeding its ring after one fill, the consumers' bounded waits run out, the
+    plane kernel's producer stops feeding its ring after one fill, the consumers' bounded waits run out (and, in
+    the kernel that also contracts the third dimension, the accumulator warps' waits for their batches), the
     kernel returns normally, dtst_plan_status reports the timeout once and clears it, and the next ordinary call
     is correct.  Nothing faults and no wait is unbounded."""
     from paper_2607_14394_b200 import binding as Bn
-    w = I.WORKLOADS["cfg1_2d_64"]
+    w = I.WORKLOADS["cfg1_2d_64"] if which == "plane" else \
+        I.custom_workload("colfuse_timeout", 1, 2, 2, (32, 128, 64), (16, 16, 8), field="iid", seed=5)
     plan = _plan(w)
     assert plan.kernel_path == "fused"
     x = _dev(I.make_field(w))
