@@ -59,3 +59,43 @@ def test_pointwise_linear_argument_errors():
     with pytest.raises(Bn.DtstError) as e:       # weight gradient asked for without its scratch
         Bn.dtst_pointwise_linear_backward(out, x, W, None, torch.zeros_like(W), None, None)
     assert e.value.status == Bn.DTST_ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("B,Ci,Co,P", [
+    (2, 16, 32, 1024),      # both products on the tensor cores: weight, bias and (assigned) input gradient
+    (1, 32, 16, 128 * 37),  # an odd number of 128-point tiles, fewer tiles than CTAs
+    (3, 32, 32, 4096),
+    (2, 16, 16, 128 * 700), # more tiles than CTAs: every CTA walks several, partial sums over CTAs
+    (2, 3, 16, 1000),       # channel counts of a lifting layer: the FFMA kernels
+    (2, 16, 1, 520),        # ... and of a projection layer
+])
+def test_pointwise_linear_forward_and_backward(B, Ci, Co, P):
+    """out = W x + b and the three gradients of a point-wise linear layer (Eq. 1: the lifting and projection
+    networks; the block's bypass is the same operator without the bias) against float64 einsums."""
+    from paper_2607_14394_b200 import binding as Bn
+    rng = np.random.default_rng(1000 * Ci + Co)
+    x = rng.standard_normal((B, Ci, P)).astype(np.float32)
+    W = (rng.standard_normal((Co, Ci)) / np.sqrt(Ci)).astype(np.float32)
+    b = rng.standard_normal(Co).astype(np.float32)
+    g = rng.standard_normal((B, Co, P)).astype(np.float32)
+    dev = lambda a: torch.from_numpy(a).cuda()
+    xd, Wd, bd, gd = dev(x), dev(W), dev(b), dev(g)
+    out = torch.empty((B, Co, P), device="cuda")
+    Bn.dtst_pointwise_linear(xd, Wd, bd, out)
+    ref = O.pointwise_linear(x, W, b)
+    assert O.rel_l2(out.cpu().numpy(), ref) <= TOL
+    scratch = torch.empty(Bn.dtst_pointwise_linear_scratch_bytes(Ci, Co), dtype=torch.uint8, device="cuda")
+    gx = torch.full((B, Ci, P), float("nan"), device="cuda")
+    gW = torch.full((Co, Ci), float("nan"), device="cuda")
+    gb = torch.full((Co,), float("nan"), device="cuda")
+    Bn.dtst_pointwise_linear_backward(gd, xd, Wd, gx, gW, gb, scratch)
+    torch.cuda.synchronize()
+    x64, g64, W64 = x.astype(np.float64), g.astype(np.float64), W.astype(np.float64)
+    assert O.rel_l2(gx.cpu().numpy(), np.einsum("oi,bop->bip", W64, g64)) <= TOL
+    assert O.rel_l2(gW.cpu().numpy(), np.einsum("bop,bip->oi", g64, x64)) <= TOL
+    assert O.rel_l2(gb.cpu().numpy(), g64.sum(axis=(0, 2))) <= TOL
+    # the same bits on a second run (fixed summation order), and the weight gradient alone
+    gW2, gb2 = torch.empty_like(gW), torch.empty_like(gb)
+    Bn.dtst_pointwise_linear_backward(gd, xd, Wd, None, gW2, gb2, scratch)
+    torch.cuda.synchronize()
+    assert torch.equal(gW, gW2) and torch.equal(gb, gb2)
