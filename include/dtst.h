@@ -97,8 +97,9 @@ dtst_status dtst_plan_create_local(dtst_plan** out, int d, const int64_t N_globa
  * for a grid that lives entirely on this device.  Such a plan is used with dtst_forward_complex,
  * dtst_spectral_mul (unchanged), dtst_inverse_complex and dtst_backward_complex; the real-field entry points
  * return DTST_ERR_INVALID_ARG for it.  Virtual shards and per-rank blocks work as for real plans.  The contiguous
- * dimension of a complex plan runs on the generic kernel family (the streaming kernels read real grids); the
- * other dimensions on the folded and slab kernels.
+ * dimension of a complex plan has no streaming kernel (those read real grids and rely on the rfft fold), so it is
+ * contracted LAST, on the most reduced tensor, and expanded first; the grid itself is streamed by the folded and
+ * slab kernels of the other dimensions.
  *   F: Xhat[b,c,m] = sum_n x[b,c,n] prod_j exp(-2 pi i s_j(m) (off_j + n_j) / N_j)        (Eq. 5-6, Eq. 18)
  *   I: y[b,o,n]    = (1/prod N) sum_m Yhat[b,o,m] prod_j exp(+2 pi i s_j(m) (off_j + n_j) / N_j)   (Eq. 14)
  *      - no Hermitian doubling: nothing is implied by symmetry;

@@ -164,6 +164,28 @@ int middle_order(const dtst_plan* p, int j_top, int* out) {
   return n;
 }
 
+// The stages of a transform that starts on the grid itself, in forward order (an expansion walks it backwards).
+// Real plans contract the contiguous dimension first: it carries the rfft fold and it is the stage the streaming
+// kernels exist for.  Complex plans have no streaming kernel for it, so they contract it LAST - on the most reduced
+// tensor, where the generic kernel that serves it touches a few percent of the bytes - and the folded kernels of the
+// other dimensions stream the grid (their inner extent then contains the whole contiguous dimension: coalesced).
+// Dimension 0 still closes the list when it carries virtual shards (its slab partials are summed after it).
+int grid_order(const dtst_plan* p, int* out) {
+  const int d = p->d;
+  if (!p->complex_io) {
+    out[0] = d - 1;
+    return 1 + (d >= 2 ? middle_order(p, d - 2, out + 1) : 0);
+  }
+  int n = d >= 2 ? middle_order(p, d - 2, out) : 0;
+  if (n > 0 && p->P > 1 && out[n - 1] == 0) {
+    out[n - 1] = d - 1;
+    out[n++] = 0;
+  } else {
+    out[n++] = d - 1;
+  }
+  return n;
+}
+
 // complex elements of a tensor in which dimension i has its retained entries (contracted[i]) or its local grid extent
 long long state_elems(const dtst_plan* p, int Cn, const bool* contracted) {
   long long n = (long long)p->B * Cn;
@@ -208,9 +230,8 @@ dtst_status forward_stages(dtst_plan* p, const void* cur, int j_from, int flip, 
   char* ws = static_cast<char*>(p->ws);
   float2* buf[2] = {reinterpret_cast<float2*>(ws + L.bufA), reinterpret_cast<float2*>(ws + L.bufB)};
   float2* partial = reinterpret_cast<float2*>(ws + L.partial);
-  int list[kMaxDims + 1], n = 0;
-  if (j_from == p->d - 1) list[n++] = p->d - 1;
-  n += middle_order(p, j_from < p->d - 1 ? j_from : p->d - 2, list + n);
+  int list[kMaxDims + 1];
+  const int n = j_from == p->d - 1 ? grid_order(p, list) : middle_order(p, j_from, list);
   bool contracted[kMaxDims];
   for (int i = 0; i < p->d; ++i) contracted[i] = i > j_from;
   bool need_reduce = false;
@@ -392,15 +413,29 @@ dtst_status inverse_stages_complex(dtst_plan* p, const float2* cur_in, int j_top
   return DTST_OK;
 }
 
-// Generic expansion: [B*Cn, M] spectrum -> real grid tensor.
-dtst_status run_inverse_generic(dtst_plan* p, const float2* Yhat, float* y, int Cn, float scale, bool herm,
+// Generic expansion: [B*Cn, M] spectrum -> grid tensor (real, or complex for a complex plan): the stages of
+// grid_order walked backwards through the ping-pong buffers, the last one writing the grid.
+dtst_status run_inverse_generic(dtst_plan* p, const float2* Yhat, void* y, int Cn, float scale, bool herm,
                                 cudaStream_t st) {
-  const float2* src = Yhat;
-  const dtst_status s = inverse_stages_complex(p, Yhat, p->d - 2, -1, Cn, &src, nullptr, st);
-  if (s != DTST_OK) return s;
+  const WsLayout L = ws_layout(p);
+  char* ws = static_cast<char*>(p->ws);
+  float2* buf[2] = {reinterpret_cast<float2*>(ws + L.bufA), reinterpret_cast<float2*>(ws + L.bufB)};
+  int list[kMaxDims + 1];
+  const int n = grid_order(p, list);
   bool contracted[kMaxDims];
-  for (int i = 0; i < p->d; ++i) contracted[i] = i == p->d - 1;
-  return expand_stage(p, p->d - 1, Cn, src, y, scale, herm, contracted, st);
+  for (int i = 0; i < p->d; ++i) contracted[i] = true;
+  const void* cur = Yhat;
+  int flip = 0;
+  for (int idx = n - 1; idx >= 0; --idx) {
+    const int j = list[idx];
+    void* dst = idx == 0 ? y : static_cast<void*>(buf[flip]);
+    const dtst_status s = expand_stage(p, j, Cn, cur, dst, j == p->d - 1 ? scale : 1.0f, herm, contracted, st);
+    if (s != DTST_OK) return s;
+    contracted[j] = false;
+    cur = dst;
+    flip ^= 1;
+  }
+  return DTST_OK;
 }
 
 // The dimension in front of the plane can be expanded inside the inverse plane kernel by a helper warp
@@ -533,9 +568,8 @@ WsLayout ws_layout(const dtst_plan* p) {
     bool contracted[kMaxDims];
     // forward: the grid-side kernel (if any) leaves its result in A, the following stages alternate from B
     for (int i = 0; i < p->d; ++i) contracted[i] = i > j_from;
-    int list[kMaxDims + 1], n = 0;
-    if (j_from == p->d - 1) list[n++] = p->d - 1;
-    if (j_from >= 0 || p->d >= 2) n += middle_order(p, j_from < p->d - 1 ? j_from : p->d - 2, list + n);
+    int list[kMaxDims + 1];
+    const int n = j_from == p->d - 1 ? grid_order(p, list) : (j_from >= 0 ? middle_order(p, j_from, list) : 0);
     int flip = 0;
     if (j_from < p->d - 1) {
       put(0, state_elems(p, Cn, contracted));
@@ -546,12 +580,11 @@ WsLayout ws_layout(const dtst_plan* p) {
       if (idx != n - 1) put(flip, state_elems(p, Cn, contracted));
       flip ^= 1;
     }
-    // expansion: the same order backwards, every stage into a buffer, starting with A
+    // expansion: the same order backwards, every stage into a buffer, starting with A (a chain that starts on
+    // the grid itself ends there: its first stage writes the caller's tensor, not a buffer)
     for (int i = 0; i < p->d; ++i) contracted[i] = true;
-    const int j_top = j_from < p->d - 1 ? j_from : p->d - 2;
-    int m = j_top >= 0 ? middle_order(p, j_top, list) : 0;
     flip = 0;
-    for (int idx = m - 1; idx >= 0; --idx) {
+    for (int idx = n - 1; idx >= (j_from == p->d - 1 ? 1 : 0); --idx) {
       contracted[list[idx]] = false;
       put(flip, state_elems(p, Cn, contracted));
       flip ^= 1;
