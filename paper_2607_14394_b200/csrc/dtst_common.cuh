@@ -38,6 +38,7 @@ struct DimOp {
   long long in_outer_stride, out_outer_stride;   // in elements of the respective type
   long long in_slab_stride, out_slab_stride;
   int basis_in_smem;
+  int es_sr, es_sq;    // shared-memory basis: entry (r, q) sits at r * es_sr + q * es_sq (set by the launcher)
 };
 
 // Number of SMs of the current device (persistent kernels launch one CTA per SM, or a multiple): queried

@@ -19,7 +19,8 @@ __global__ void __launch_bounds__(256) apply_dim_kernel(DimOp p, const void* __r
   if (p.basis_in_smem) {
     const int total = p.R * p.Q;
     for (int e = threadIdx.x; e < total; e += blockDim.x) {
-      Es[e] = dimop_entry(p, e / p.Q, e % p.Q, slab);
+      const int r = e / p.Q, q = e % p.Q;
+      Es[r * p.es_sr + q * p.es_sq] = dimop_entry(p, r, q, slab);
     }
     __syncthreads();
   }
@@ -39,7 +40,7 @@ __global__ void __launch_bounds__(256) apply_dim_kernel(DimOp p, const void* __r
     const long long base = o * p.in_outer_stride + i;
     float ar = 0.f, ai = 0.f;
     for (int q = 0; q < p.Q; ++q) {
-      const float2 e = p.basis_in_smem ? Es[r * p.Q + q] : dimop_entry(p, r, q, slab);
+      const float2 e = p.basis_in_smem ? Es[r * p.es_sr + q * p.es_sq] : dimop_entry(p, r, q, slab);
       if (IN_REAL) {
         const float v = in_r[base + (long long)q * p.inner];
         ar = fmaf(e.x, v, ar);
@@ -66,7 +67,16 @@ __global__ void __launch_bounds__(256) apply_dim_kernel(DimOp p, const void* __r
 cudaError_t launch_apply_dim(const DimOp& op_in, bool in_real, bool out_real, const void* in, void* out,
                              cudaStream_t st) {
   DimOp op = op_in;
-  const size_t smem = (size_t)op.R * op.Q * sizeof(float2);
+  // Layout of the basis in shared memory.  With a wide inner extent the lanes of a warp share their output row r
+  // and read one entry (a broadcast): rows of Q entries.  With a narrow one (the contiguous dimension itself:
+  // inner = 1) neighbouring lanes own neighbouring rows and walk q together: stored [q][r] with an odd row count,
+  // their reads fall into different banks (stored [r][q] they were Q entries apart - a 32-way conflict for every
+  // multiple of 32, which made this kernel 20 times slower than it had to be).
+  const int Rp = op.R | 1;
+  const bool narrow = op.inner < 32;
+  op.es_sr = narrow ? 1 : op.Q;
+  op.es_sq = narrow ? Rp : 1;
+  const size_t smem = (size_t)(narrow ? Rp : op.R) * op.Q * sizeof(float2);
   op.basis_in_smem = smem <= 160 * 1024 ? 1 : 0;
   const size_t dyn = op.basis_in_smem ? smem : 0;
   const long long total = op.outer * op.R * op.inner;
