@@ -152,7 +152,7 @@ dtst_status dtst_plan_tune_contraction_order(dtst_plan* plan, double* bytes_befo
 /*
  * "Fast path or fail".  Shapes outside the streaming kernels' reach (odd extents, a contiguous extent that is not
  * a multiple of 32, k outside {4, 8, 12, 16} on a middle dimension, offsets on the contiguous dimension) are
- * served by a generic kernel that is an order of magnitude slower.  With required != 0 this call returns
+ * served by a generic kernel that is several times slower.  With required != 0 this call returns
  * DTST_ERR_UNSUPPORTED if ANY stage of the plan's forward- or inverse-type transforms would take that kernel,
  * and otherwise DTST_OK, after which the compute calls of this plan return DTST_ERR_UNSUPPORTED (launching
  * nothing) should a later option change (virtual shards, kernel path) make a stage fall back.  required = 0
