@@ -658,7 +658,10 @@ def main_ours(args, w):
 
     steps, warmup = max(1, args.steps), max(3, args.warmup)
     P = args.shards
-    plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out, virtual_shards=P, path=args.path)
+    # --channels is a profiler aid that runs the full workload's kernels on fewer tasks: keep the kernel choice of
+    # the full workload (with few channels the automatic choice would drop the fused third dimension)
+    plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out, virtual_shards=P, path=args.path,
+                column_contraction=1 if args.channels else 0)
 
     # the batch each rank works on is its own (weak scaling over independent samples; no collective)
     x = inputs.make_field_torch(w, dev, tag=0, rank=rank)

@@ -173,6 +173,18 @@ dtst_status dtst_plan_require_fast_path(dtst_plan* plan, int required);
  */
 dtst_status dtst_plan_set_column_expansion(dtst_plan* plan, int ring_columns);
 
+/*
+ * Forward-type transforms (dtst_forward and the first stage of dtst_backward) of plans on the fused streaming path
+ * whose shape has such a kernel contract the dimension d-3 INSIDE the kernel that streams the grid (columns of
+ * planes batched in shared memory, the column's accumulator in tensor-core fragments): the reduced tensor of the
+ * plane stage never reaches HBM and one launch disappears.  Same tolerance against the float64 statement.
+ *   mode  0 (default): whenever the kernel exists for the shape, dimension d-3 is whole on this device, first in
+ *                      the contraction order, and the plan has enough columns (batch x channels x leading extents)
+ *                      to keep every SM busy in the last round;
+ *   mode  1: whenever the kernel exists (small problems: for tests);   mode -1: never.
+ */
+dtst_status dtst_plan_set_column_contraction(dtst_plan* plan, int mode);
+
 dtst_status dtst_plan_destroy(dtst_plan* plan);
 
 /* M = number of retained modes; K[d] (host, may be NULL) = entries kept per dim. */

@@ -299,13 +299,22 @@ dtst_status run_forward_generic(dtst_plan* p, const float* x, float2* Xhat, int 
 
 // Whether the forward plane kernel also contracts the dimension in front of the plane: that dimension must be the
 // first of the middle stages in the plan's order, whole on this device, without offset and not cut into slabs.
-bool use_fwd_col(const dtst_plan* p) {
+bool use_fwd_col(const dtst_plan* p, int Cn) {
   const int d = p->d;
   if (d < 3 || !use_fused(p)) return false;
   const int c = d - 3;
   int list[kMaxDims];
   if (middle_order(p, c, list) < 1 || list[0] != c) return false;
   if (!use_mid(p, c)) return false;
+  // a CTA takes whole columns: with few columns per CTA the last round is mostly idle (a rank's thin slab), and
+  // the plain kernel, whose tasks are single planes, balances better than this one gains
+  if (p->colfuse < 0) return false;
+  if (p->colfuse == 0) {
+    long long cols = (long long)p->B * Cn;
+    for (int i = 0; i < c; ++i) cols *= p->Nl[i];
+    const long long sms = num_sms(), rounds = (cols + sms - 1) / sms;
+    if (cols * 100 < rounds * sms * 95) return false;
+  }
   return fwd_plane_col_supported((int)p->Ng[d - 1], p->kmax[d - 1], (int)p->Ng[d - 2], p->kmax[d - 2], (int)p->Ng[c],
                                  p->kmax[c]);
 }
@@ -320,7 +329,7 @@ dtst_status run_forward_fused(dtst_plan* p, const float* x, float2* Xhat, int Cn
   long long planes = (long long)p->B * Cn;
   for (int i = 0; i < b; ++i) planes *= p->Nl[i];
   float2* t1 = (d == 2) ? Xhat : reinterpret_cast<float2*>(ws + L.bufA);
-  if (use_fwd_col(p)) {
+  if (use_fwd_col(p, Cn)) {
     // the third dimension is contracted inside the plane kernel: no reduced tensor in HBM, one launch less
     const int c = d - 3;
     float2* dst = (d == 3) ? Xhat : t1;
@@ -710,6 +719,12 @@ dtst_status dtst_plan_tune_contraction_order(dtst_plan* p, double* bytes_before,
     }
   for (int i = 0; i < n; ++i) p->order_rank[list[i]] = i;
   if (bytes_after) *bytes_after = middle_stage_bytes(p);
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_set_column_contraction(dtst_plan* p, int mode) {
+  if (p == nullptr || mode < -1 || mode > 1) return DTST_ERR_INVALID_ARG;
+  p->colfuse = mode;
   return DTST_OK;
 }
 

@@ -147,6 +147,7 @@ struct dtst_plan {
   unsigned dbg_poll_limit;         // 0 = default budget of the bounded waits
   long long dbg_withhold_after;    // < 0 = off (the default)
   dtst_host_io* host_io;           // non-null after dtst_plan_enable_host_io
+  int colfuse;                     // third dimension inside the forward plane kernel: 0 auto, 1 whenever built, -1 never
   int order_rank[dtst::kMaxDims];  // contraction order of the dimensions behind the grid-side kernel: lower = earlier
   int complex_io;                  // 1: complex fields, two-sided retained set on the last dimension too
   int block_epilogue;              // DTST_BLOCK_EPILOGUE_*

@@ -23,11 +23,11 @@ def _dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def run_layer_and_check(w, path="auto", P=1, check_backward=True, tol=TOL):
+def run_layer_and_check(w, path="auto", P=1, check_backward=True, tol=TOL, **plan_kw):
     x = I.make_field(w)
     W = I.make_weights(w)
     g = I.make_upstream_grad(w)
-    plan = _plan(w, path, P)
+    plan = _plan(w, path, P, **plan_kw)
     lists = O.mode_index_lists(w.N, w.kmax)
     for j in range(w.d):
         assert plan.mode_indices(j) == lists[j].tolist()
@@ -311,7 +311,7 @@ def test_bounded_wait_runs_out_and_is_reported_once(which):
     from paper_2607_14394_b200 import binding as Bn
     w = I.WORKLOADS["cfg1_2d_64"] if which == "plane" else \
         I.custom_workload("colfuse_timeout", 1, 2, 2, (32, 128, 64), (16, 16, 8), field="iid", seed=5)
-    plan = _plan(w)
+    plan = _plan(w, column_contraction=1)
     assert plan.kernel_path == "fused"
     x = _dev(I.make_field(w))
     ref = plan.forward(x).clone()
@@ -402,15 +402,22 @@ def test_forward_with_the_third_dimension_fused(N, k, B, C, P):
     """Shapes whose forward-type transforms contract three dimensions in one kernel (columns of planes accumulated
     in the MMA fragments of extra warps): forward, inverse and backward against the oracle."""
     w = I.custom_workload("colfuse", B, C, C, N, k, field="grf", seed=47)
-    plan = _plan(w, "auto", P)
+    plan = _plan(w, "auto", P, column_contraction=1)   # these cases have too few columns for the automatic choice
     assert plan.kernel_path == "fused"
     # one launch per forward: plane kernel (+ one per remaining dimension)
     before = plan.launch_count()
     plan.forward(_dev(I.make_field(w)))
     torch.cuda.synchronize()
     assert plan.launch_count() - before <= 1 + (len(N) - 3) + (1 if P > 1 else 0)   # (+ the slab reduction)
+    # the automatic choice keeps the separate launch for so few columns (a CTA takes whole columns)
+    auto = _plan(w, "auto", P)
+    before = auto.launch_count()
+    auto.forward(_dev(I.make_field(w)))
+    torch.cuda.synchronize()
+    assert auto.launch_count() - before >= 2 + (len(N) - 3)
+    auto.close()
     plan.close()
-    run_layer_and_check(w, "auto", P=P)
+    run_layer_and_check(w, "auto", P=P, column_contraction=1)
 
 
 # ------------------------------------------------------------------ contraction order and pencils
