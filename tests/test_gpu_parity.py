@@ -420,6 +420,29 @@ def test_forward_with_the_third_dimension_fused(N, k, B, C, P):
     run_layer_and_check(w, "auto", P=P, column_contraction=1)
 
 
+def test_fused_third_dimension_many_columns_is_reproducible():
+    """More columns than SMs (some CTAs walk two columns, their batch buffers and accumulators are reused), three
+    channels, N1 = 32: two runs give the same bits (the accumulation order is fixed), a run with the separate
+    launch agrees within rounding, and the result meets the oracle."""
+    w = I.custom_workload("colfuse_many", 1, 3, 3, (50, 32, 128, 64), (4, 16, 16, 8), field="grf", seed=53)
+    x = _dev(I.make_field(w))
+    fused = _plan(w, column_contraction=1)
+    a = fused.forward(x).clone()
+    b = fused.forward(x).clone()
+    torch.cuda.synchronize()
+    assert fused.status() == 0
+    assert torch.equal(torch.view_as_real(a), torch.view_as_real(b))
+    plain = _plan(w, column_contraction=-1)
+    c = plain.forward(x)
+    torch.cuda.synchronize()
+    assert plain.launch_count() > 0 and O.rel_l2(a.cpu().numpy(), c.cpu().numpy()) <= 2e-6
+    ref = O.forward(I.make_field(w), w.kmax)
+    assert O.rel_l2(a.cpu().numpy(), ref) <= TOL
+    assert per_mode_excess(a.cpu().numpy(), ref) <= 1.0
+    fused.close()
+    plain.close()
+
+
 # ------------------------------------------------------------------ contraction order and pencils
 @pytest.mark.parametrize("N,k,order", [
     ((32, 64, 16), (4, 8, 3), (0, 1)),                 # generic/folded: dimension 0 before dimension 1
