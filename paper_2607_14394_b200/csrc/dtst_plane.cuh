@@ -1360,7 +1360,7 @@ cudaError_t plane_inv(const float2* in, float* y, long long rows, float scale, i
 // extent in front of it and its retained modes per side.  The in-kernel column expansion variant of the inverse
 // kernel is built for a leading dimension of the same shape as the second one (K1 = k2, N1 = N2).
 #define DTST_PLANE_SHAPES_A(X) X(64, 8, 128, 16) X(64, 8, 128, 8)
-#define DTST_PLANE_SHAPES_B(X) X(32, 4, 64, 8) X(64, 8, 64, 8) X(32, 8, 64, 8)
+#define DTST_PLANE_SHAPES_B(X) X(32, 4, 64, 8) X(64, 8, 64, 8) X(32, 8, 64, 8) X(32, 16, 64, 8)
 #define DTST_PLANE_SHAPES_C(X) X(32, 8, 128, 16) X(32, 8, 128, 8) X(64, 4, 64, 8)
 #define DTST_PLANE_SHAPES(X) DTST_PLANE_SHAPES_A(X) DTST_PLANE_SHAPES_B(X) DTST_PLANE_SHAPES_C(X)
 

@@ -376,6 +376,8 @@ PLANE_SHAPES = [
     ("p_32_8_128_8", 2, 1, 1, (32, 128, 32), (16, 8, 8)),
     ("p_64_4_64_8", 1, 2, 2, (32, 64, 64), (12, 8, 4)),
     ("p_64_8_64_8_d3", 1, 2, 2, (64, 64, 64), (8, 8, 8)),
+    # the paper's own layer shape in small: modes (8, 8, 8, 16) with 16 one-sided modes on a time axis of 32
+    ("p_32_16_64_8_paper", 1, 2, 2, (32, 32, 64, 32), (8, 8, 8, 16)),
 ]
 
 
