@@ -562,8 +562,8 @@ def block_summary(torch, w, x, g, W, steps, peak):
                "bytes_moved_model": {"fwd": bytes_f, "fwd_bwd": bytes_f + bytes_b},
                "fwd_gbs": bytes_f / tf / 1e6, "fwd_bwd_gbs": (bytes_f + bytes_b) / (tf + tb) / 1e6,
                "fwd_bwd_frac_of_measured_peak": (bytes_f + bytes_b) / (tf + tb) / 1e6 / peak,
-               "bypass_product": "auto: tcgen05.mma kind::tf32 (3xTF32, accumulator in TMEM) from 32 input channels "
-                                 "on, fp32 FFMA below",
+               "bypass_product": "auto: fp32 FFMA with the input channels in registers (the faster kernel at every "
+                                 "channel count measured); tcgen05.mma kind::tf32 (3xTF32, accumulator in TMEM) on request",
                "epilogue_kernel_ms": {"ffma": epi.get("ffma"), "tcgen05": epi.get("tensor")},
                "kernels": {k: {"launches": n, "avg_ms": ms / n, "bytes_per_launch": kernel_bytes[k],
                                "achieved_gbs": kernel_bytes[k] / (ms / n) / 1e6,
@@ -575,6 +575,48 @@ def block_summary(torch, w, x, g, W, steps, peak):
         return res
     except Exception as ex:
         return {"error": f"{type(ex).__name__}: {ex}"[:200]}
+
+
+def fno_summary(torch, steps=5):
+    """A whole synthetic FNO with the paper's architecture (Section "Experimental Setup": 4 Fourier blocks, modes
+    (8, 8, 8, 16), 5 fields in and out, grid 128 x 128 x 64 with a time axis of 32) forward and backward on this
+    GPU, every step in the library's kernels: at the paper's width 20 and at width 32 (the channel counts the
+    tensor-core bypass kernels serve).  Random-init weights, synthetic input; context for the paper's multi-GPU
+    figures, not a like-for-like comparison."""
+    from paper_2607_14394_b200 import FNO
+    out = {"grid": [128, 128, 64, 32], "modes": [8, 8, 8, 16], "layers": 4, "fields": 5, "steps": steps,
+           "paper_context": "the paper reports 148.3 ms forward / 246.8 ms backward for this architecture at "
+                            "128^3 on 4 V100s (its Table 5); another machine, another grid: context only"}
+    for width in (20, 32):
+        try:
+            net = FNO((128, 128, 64, 32), (8, 8, 8, 16), 1, 5, 5, width, 4, seed=11)
+            gen = torch.Generator(device="cuda").manual_seed(12)
+            a = torch.randn((1, 5, 128, 128, 64, 32), device="cuda", generator=gen)
+            gu = torch.randn((1, 5, 128, 128, 64, 32), device="cuda", generator=gen)
+            for _ in range(2):
+                net.forward(a)
+                net.backward(gu)
+            torch.cuda.synchronize()
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            fwd = bwd = 0.0
+            for _ in range(steps):
+                e[0].record()
+                net.forward(a)
+                e[1].record()
+                net.backward(gu)
+                e[2].record()
+                torch.cuda.synchronize()
+                fwd += e[0].elapsed_time(e[1])
+                bwd += e[1].elapsed_time(e[2])
+            ok = net.plan.status() == 0
+            out[f"width_{width}"] = {"fwd_ms": fwd / steps, "bwd_ms": bwd / steps, "status_ok": ok,
+                                     "kernel_path": net.plan.kernel_path}
+            net.close()
+            del net, a, gu
+            torch.cuda.empty_cache()
+        except Exception as ex:
+            out[f"width_{width}"] = {"error": f"{type(ex).__name__}: {ex}"[:200]}
+    return out
 
 
 def other_configs_summary(torch, skip_name, steps=10):
@@ -860,6 +902,7 @@ def main_ours(args, w):
             del x, g
             torch.cuda.empty_cache()
             line["other_configs"] = other_configs_summary(torch, w.name)
+            line["fno"] = fno_summary(torch)
         if not args.no_cpu_baseline:
             try:
                 # the same bounded sample, warm-up and statistics as the reference arm (--impl reference)

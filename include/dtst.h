@@ -266,8 +266,8 @@ dtst_status dtst_block_forward(dtst_plan* plan, const float* x, const void* W, c
  *   DTST_BLOCK_EPILOGUE_TENSOR  the tensor cores (tcgen05.mma kind::tf32 with the accumulator in tensor memory,
  *                               three TF32 products per fp32 product): C_in in {8, 16, 32}, C_out in {16, 32},
  *                               plans on the streaming kernel family; DTST_ERR_UNSUPPORTED otherwise;
- *   DTST_BLOCK_EPILOGUE_AUTO    (default) the tensor cores from 32 input channels on, where the product stops
- *                               fitting into the memory time of the FFMA kernel; FFMA below.
+ *   DTST_BLOCK_EPILOGUE_AUTO    (default) the faster of the two as measured on B200: the FFMA kernel, at every
+ *                               channel count the tensor-core kernel exists for.
  * Both meet the same tolerance against the float64 statement of the block.
  */
 enum { DTST_BLOCK_EPILOGUE_AUTO = 0, DTST_BLOCK_EPILOGUE_FFMA = 1, DTST_BLOCK_EPILOGUE_TENSOR = 2 };

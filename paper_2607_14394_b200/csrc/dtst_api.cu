@@ -978,15 +978,14 @@ dtst_status dtst_backward(dtst_plan* p, const float* grad_y, const void* Xhat_sa
   return DTST_OK;
 }
 
-// Which kernel forms the bypass product of dtst_block_forward: the tensor-core one (tcgen05) when asked for, or,
-// left to the library, from 32 input channels on - below that the exact-fp32 FFMA kernel is the faster one
-// (measured at 16 channels on the largest benchmark shape: 7.4 ms against 12.0 ms for 34 GB moved; the product is
-// 16 multiply-adds per output value there, which the FFMA pipe does within the memory time, while the tensor-core
-// kernel's per-tile chain of split, product and epilogue is latency-bound at four CTAs per SM).
+// Which kernel forms the bypass product of dtst_block_forward: the tensor-core one (tcgen05) only when asked for.
+// Left to the library it is the fp32 FFMA kernel, which holds a thread's input channels in registers and is the
+// faster one at every channel count measured (34 GB moved at 16 channels: 5.8 ms against 12.0 ms; 17 GB at 32
+// channels: 3.9 ms against 5.7 ms - the tensor-core kernel's per-tile chain of split, product and epilogue is
+// latency-bound at four CTAs per SM).
 static bool use_block_tensor(const dtst_plan* p) {
-  if (p->path_request != DTST_PATH_AUTO || p->block_epilogue == DTST_BLOCK_EPILOGUE_FFMA) return false;
-  if (!block_umma_supported(p->C_in, p->C_out, p->points_local, p->B)) return false;
-  return p->block_epilogue == DTST_BLOCK_EPILOGUE_TENSOR || p->C_in >= 32;
+  if (p->path_request != DTST_PATH_AUTO || p->block_epilogue != DTST_BLOCK_EPILOGUE_TENSOR) return false;
+  return block_umma_supported(p->C_in, p->C_out, p->points_local, p->B);
 }
 
 // ---- the whole block: GELU(W_bypass x + I(M(F(x), W))) and its backward pass

@@ -12,11 +12,33 @@
 namespace dtst {
 namespace {
 
-__device__ __forceinline__ float gelu_f(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f)); }
+// Phi(z) = (1 + erf(z / sqrt 2)) / 2, the standard normal distribution function of the exact (erf) form of GELU,
+// in the five-term rational form of Abramowitz & Stegun 7.1.26 / 26.2.17 (|error| <= 1.5e-7 on erf, below the
+// rounding of the fp32 arithmetic around it: 8e-8 rel-L2 on GELU against 5e-8 with a correctly rounded erf),
+// evaluated on the negative side as the tail itself, without cancellation.  The library erff costs about twice
+// the instructions, and the passes that apply the activation are bound by exactly those.  e = exp(-z^2 / 2) is
+// handed back because GELU' needs it too.
+__device__ __forceinline__ float phi_f(float z, float& e) {
+  const float t = __fdividef(1.0f, fmaf(0.2316418882f, fabsf(z), 1.0f));   // 0.3275911 / sqrt 2
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  e = __expf(-0.5f * z * z);
+  const float q = poly * t * e;            // 2 (1 - Phi(|z|))
+  return z >= 0.f ? fmaf(-0.5f, q, 1.0f) : 0.5f * q;
+}
+
+__device__ __forceinline__ float gelu_f(float v) {
+  float e;
+  return v * phi_f(v, e);
+}
 
 // d GELU / dz = Phi(z) + z phi(z)
 __device__ __forceinline__ float gelu_grad_f(float v) {
-  return 0.5f * (1.0f + erff(v * 0.70710678118654752f)) + v * __expf(-0.5f * v * v) * 0.39894228040143268f;
+  float e;
+  const float Phi = phi_f(v, e);
+  return fmaf(v * 0.39894228040143268f, e, Phi);
 }
 
 constexpr int kOC = 4;   // output channels per register tile of the FFMA kernels
@@ -70,6 +92,101 @@ __global__ void __launch_bounds__(256) block_epilogue_kernel(const float* __rest
             const float4 zv = make_float4(acc[k].x + yv.x, acc[k].y + yv.y, acc[k].z + yv.z, acc[k].w + yv.w);
             if (zb) __stcs(zb + off, zv);
             __stcs(ob + off, make_float4(gelu_f(zv.x), gelu_f(zv.y), gelu_f(zv.z), gelu_f(zv.w)));
+          }
+        }
+      }
+    }
+  }
+}
+
+// The same pass with a thread's x values held in registers: all C_in loads of a thread are in flight at once (the
+// loop above has one), and x is read exactly once instead of once per four output channels.  A thread owns V
+// consecutive points: four up to 20 input channels, two for 32 (64 registers of x either way).
+template <int V>
+struct PointVec {
+  float v[V];
+};
+template <int V>
+__device__ __forceinline__ PointVec<V> ld_points(const float* p) {
+  PointVec<V> r;
+  if constexpr (V == 4) {
+    const float4 t = __ldcs(reinterpret_cast<const float4*>(p));
+    r.v[0] = t.x; r.v[1] = t.y; r.v[2] = t.z; r.v[3] = t.w;
+  } else {
+    const float2 t = __ldcs(reinterpret_cast<const float2*>(p));
+    r.v[0] = t.x; r.v[1] = t.y;
+  }
+  return r;
+}
+template <int V>
+__device__ __forceinline__ void st_points(float* p, const PointVec<V>& r, bool streaming) {
+  if constexpr (V == 4) {
+    const float4 t = make_float4(r.v[0], r.v[1], r.v[2], r.v[3]);
+    if (streaming) __stcs(reinterpret_cast<float4*>(p), t); else *reinterpret_cast<float4*>(p) = t;
+  } else {
+    const float2 t = make_float2(r.v[0], r.v[1]);
+    if (streaming) __stcs(reinterpret_cast<float2*>(p), t); else *reinterpret_cast<float2*>(p) = t;
+  }
+}
+
+template <bool LINEAR, int CI, int V>
+__global__ void __launch_bounds__(256, 2) block_epilogue_regx_kernel(const float* __restrict__ x, float* __restrict__ out,
+                                                                    float* __restrict__ z,
+                                                                    const float* __restrict__ Wb, int B, int Co,
+                                                                    long long P) {
+  pdl_trigger();
+  extern __shared__ float wb_s[];   // [Co][CI]
+  pdl_wait();
+  for (int e = threadIdx.x; e < Co * CI; e += blockDim.x) wb_s[e] = Wb[e];
+  __syncthreads();
+  const long long groups = P / V;
+  const long long total = (long long)B * groups;
+  for (long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+       t += (long long)gridDim.x * blockDim.x) {
+    const long long b = t / groups, p0 = (t % groups) * V;
+    const float* xb = x + b * CI * P + p0;
+    float* ob = out + b * Co * P + p0;
+    float* zb = (!LINEAR && z) ? z + b * Co * P + p0 : nullptr;
+    PointVec<V> xv[CI];
+#pragma unroll
+    for (int i = 0; i < CI; ++i) xv[i] = ld_points<V>(xb + (long long)i * P);
+    for (int o0 = 0; o0 < Co; o0 += 4) {
+      PointVec<V> acc[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if constexpr (LINEAR) {
+          const float bo = (z && o0 + k < Co) ? z[o0 + k] : 0.f;
+#pragma unroll
+          for (int c = 0; c < V; ++c) acc[k].v[c] = bo;
+        } else {
+          if (o0 + k < Co) {
+            acc[k] = ld_points<V>(ob + (long long)(o0 + k) * P);   // the layer's output: requested before the products
+          } else {
+#pragma unroll
+            for (int c = 0; c < V; ++c) acc[k].v[c] = 0.f;
+          }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < CI; ++i)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float w = (o0 + k < Co) ? wb_s[(o0 + k) * CI + i] : 0.f;
+#pragma unroll
+          for (int c = 0; c < V; ++c) acc[k].v[c] = fmaf(w, xv[i].v[c], acc[k].v[c]);
+        }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (o0 + k < Co) {
+          const long long off = (long long)(o0 + k) * P;
+          if constexpr (LINEAR) {
+            st_points<V>(ob + off, acc[k], false);
+          } else {
+            if (zb) st_points<V>(zb + off, acc[k], true);
+            PointVec<V> g;
+#pragma unroll
+            for (int c = 0; c < V; ++c) g.v[c] = gelu_f(acc[k].v[c]);
+            st_points<V>(ob + off, g, true);
           }
         }
       }
@@ -281,6 +398,21 @@ static cudaError_t launch_epilogue_any(bool linear, const float* x, float* out, 
   if (blocks > cap) blocks = cap;
   const size_t smem = (size_t)Ci * Co * 4;
   cudaError_t e = cudaSuccess;
+#define DTST_REGX(ci, v)                                                                                           \
+  if (Ci == ci) {                                                                                                  \
+    auto k2 = linear ? block_epilogue_regx_kernel<true, ci, v> : block_epilogue_regx_kernel<false, ci, v>;         \
+    if (smem > 48 * 1024) e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);    \
+    if (e != cudaSuccess) return e;                                                                                \
+    long long bl = ((long long)B * (P / v) + 255) / 256;                                                           \
+    if (bl > cap) bl = cap;                                                                                        \
+    (void)launch_pdl(k2, dim3((unsigned)bl), dim3(256), smem, st, x, out, z, Wb, B, Co, P);                        \
+    return cudaGetLastError();                                                                                     \
+  }
+  DTST_REGX(8, 4)
+  DTST_REGX(16, 4)
+  DTST_REGX(20, 4)
+  DTST_REGX(32, 2)
+#undef DTST_REGX
   auto kern = linear ? block_epilogue_kernel<true> : block_epilogue_kernel<false>;
   if (smem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
