@@ -43,7 +43,9 @@ template <int CI, int CO>
 __global__ void __launch_bounds__(128, 3)
 linear_backward_mma_kernel(const float* __restrict__ gz, const float* __restrict__ x, float* __restrict__ gx,
                            const float* __restrict__ Wb, float* __restrict__ partial, int B, long long P, int mode_gx,
-                           int want_gw, int want_gb) {
+                           int want_gw, int want_gb, int ci, int co) {
+  // CI, CO: the channel counts rounded up to 16 or 32 (the MMA tiles); ci <= CI, co <= CO the real ones.  The rows
+  // of the staged tiles that belong to no channel are zero, as are the weights in front of them.
   static_assert(CI % 16 == 0 && CO % 16 == 0 && CI <= 32 && CO <= 32, "channel counts");
   constexpr int ROWS = CO + CI;
   constexpr int MTO = CO / 16, NTI = CI / 8;   // weight gradient: m-tiles over o, n-tiles over i
@@ -62,7 +64,7 @@ linear_backward_mma_kernel(const float* __restrict__ gz, const float* __restrict
       for (int e = 0; e < 4; ++e) {
         const int i = 16 * mt + g8 + 8 * (e & 1);
         const int o = 8 * ks + 2 * t4 + (e >> 1);
-        split_tf32_rna(mode_gx ? Wb[o * CI + i] : 0.f, whi[mt][ks][e], wlo[mt][ks][e]);
+        split_tf32_rna((mode_gx && o < co && i < ci) ? Wb[o * ci + i] : 0.f, whi[mt][ks][e], wlo[mt][ks][e]);
       }
   float accW[MTO][NTI][4];
   float bs[MTO][2];
@@ -74,6 +76,12 @@ linear_backward_mma_kernel(const float* __restrict__ gz, const float* __restrict
 #pragma unroll
       for (int e = 0; e < 4; ++e) accW[mt][nt][e] = 0.f;
   }
+  // rows without a channel: zero, in both buffers, once
+  for (int bufz = 0; bufz < 2; ++bufz)
+    for (int r = warp; r < ROWS; r += 4)
+      if ((r < CO && r >= co) || (r >= CO && r - CO >= ci))
+        *reinterpret_cast<float4*>(lb_s + (size_t)bufz * ROWS * kMSP + (size_t)r * kMSP + 4 * lane) =
+            make_float4(0.f, 0.f, 0.f, 0.f);
   pdl_wait();
 
   const long long tiles_per_b = P / kMTP;
@@ -82,7 +90,8 @@ linear_backward_mma_kernel(const float* __restrict__ gz, const float* __restrict
     const long long b = tile / tiles_per_b, p0 = (tile % tiles_per_b) * kMTP;
     float* dstb = lb_s + (size_t)buf * ROWS * kMSP;
     for (int r = warp; r < ROWS; r += 4) {
-      const float* src = (r < CO ? gz + ((b * CO + r) * P) : x + ((b * CI + (r - CO)) * P)) + p0 + 4 * lane;
+      if (r < CO ? r >= co : r - CO >= ci) continue;
+      const float* src = (r < CO ? gz + ((b * co + r) * P) : x + ((b * ci + (r - CO)) * P)) + p0 + 4 * lane;
       cp_async16(dstb + (size_t)r * kMSP + 4 * lane, src);
     }
     cp_async_commit();
@@ -113,9 +122,11 @@ linear_backward_mma_kernel(const float* __restrict__ gz, const float* __restrict
 #pragma unroll
         for (int mt = 0; mt < MTI; ++mt)
 #pragma unroll
-          for (int h = 0; h < 2; ++h)
-            old[nt][mt][h] = *reinterpret_cast<const float2*>(gx + ((b * CI + 16 * mt + g8 + 8 * h) * P) + p0 + pw +
-                                                               8 * nt + 2 * t4);
+          for (int h = 0; h < 2; ++h) {
+            const int i = 16 * mt + g8 + 8 * h;
+            old[nt][mt][h] = i < ci ? *reinterpret_cast<const float2*>(gx + ((b * ci + i) * P) + p0 + pw + 8 * nt + 2 * t4)
+                                    : make_float2(0.f, 0.f);
+          }
     }
 
     if (want_gw) {
@@ -185,7 +196,8 @@ linear_backward_mma_kernel(const float* __restrict__ gz, const float* __restrict
               v.x += old[nt][mt][h].x;
               v.y += old[nt][mt][h].y;
             }
-            *reinterpret_cast<float2*>(gx + ((b * CI + 16 * mt + g8 + 8 * h) * P) + p0 + pw + 8 * nt + 2 * t4) = v;
+            const int i = 16 * mt + g8 + 8 * h;
+            if (i < ci) *reinterpret_cast<float2*>(gx + ((b * ci + i) * P) + p0 + pw + 8 * nt + 2 * t4) = v;
           }
       }
     }
@@ -214,18 +226,22 @@ linear_backward_mma_kernel(const float* __restrict__ gz, const float* __restrict
       }
     }
     __syncthreads();
-    for (int e = threadIdx.x; e < PAIRS + (want_gb ? CO : 0); e += blockDim.x) {
+    // the row of `partial` has the real counts: co * ci pairs [o][i], then co bias sums
+    const int pairs = co * ci;
+    for (int e = threadIdx.x; e < pairs + (want_gb ? co : 0); e += blockDim.x) {
+      const int src = e < pairs ? (e / ci) * CI + e % ci : PAIRS + (e - pairs);
       float s = 0.f;
 #pragma unroll
-      for (int w = 0; w < 4; ++w) s += red[(size_t)w * (PAIRS + CO) + e];
-      partial[(long long)blockIdx.x * (PAIRS + CO) + e] = s;
+      for (int w = 0; w < 4; ++w) s += red[(size_t)w * (PAIRS + CO) + src];
+      partial[(long long)blockIdx.x * (pairs + co) + e] = s;
     }
   }
 }
 
 template <int CI, int CO>
 cudaError_t launch_t(const float* gz, const float* x, float* gx, int mode_gx, const float* Wb, float* partial, int B,
-                     long long P, int want_gw, int want_gb, int max_ctas, int* ctas_out, cudaStream_t st) {
+                     long long P, int want_gw, int want_gb, int max_ctas, int* ctas_out, int ci, int co,
+                     cudaStream_t st) {
   auto kern = linear_backward_mma_kernel<CI, CO>;
   size_t smem = (size_t)2 * (CO + CI) * kMSP * 4;
   const size_t red = (size_t)4 * (CO * CI + CO) * 4;
@@ -241,23 +257,26 @@ cudaError_t launch_t(const float* gz, const float* x, float* gx, int mode_gx, co
   if (ctas > max_ctas) ctas = max_ctas;
   if (ctas > tiles) ctas = tiles;
   *ctas_out = (int)ctas;
-  (void)launch_pdl(kern, dim3((unsigned)ctas), dim3(128), smem, st, gz, x, gx, Wb, partial, B, P, mode_gx, want_gw, want_gb);
+  (void)launch_pdl(kern, dim3((unsigned)ctas), dim3(128), smem, st, gz, x, gx, Wb, partial, B, P, mode_gx, want_gw, want_gb,
+                   ci, co);
   return cudaGetLastError();
 }
 
 }  // namespace
 
+// 8 to 32 channels on both sides (rounded up to 16 or 32 inside), whole tiles of points
 bool linear_backward_mma_supported(int Ci, int Co, long long P) {
-  return (Ci == 16 || Ci == 32) && (Co == 16 || Co == 32) && P % kMTP == 0 && P > 0;
+  return Ci >= 8 && Ci <= 32 && Co >= 8 && Co <= 32 && P % kMTP == 0 && P > 0;
 }
 
 // Launches the kernel above; *ctas_out = rows of `partial` that were written (the caller reduces them).
 cudaError_t launch_linear_backward_mma(const float* gz, const float* x, float* gx, int mode_gx, const float* Wb,
                                        float* partial, int B, int Ci, int Co, long long P, int want_gw, int want_gb,
                                        int max_ctas, int* ctas_out, cudaStream_t st) {
-#define DTST_CALL(ci, co) \
-  if (Ci == ci && Co == co) \
-    return launch_t<ci, co>(gz, x, gx, mode_gx, Wb, partial, B, P, want_gw, want_gb, max_ctas, ctas_out, st);
+  const int cip = Ci <= 16 ? 16 : 32, cop = Co <= 16 ? 16 : 32;
+#define DTST_CALL(c1, c2) \
+  if (cip == c1 && cop == c2) \
+    return launch_t<c1, c2>(gz, x, gx, mode_gx, Wb, partial, B, P, want_gw, want_gb, max_ctas, ctas_out, Ci, Co, st);
   DTST_CALL(16, 16)
   DTST_CALL(16, 32)
   DTST_CALL(32, 16)

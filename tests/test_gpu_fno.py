@@ -66,6 +66,9 @@ def test_pointwise_linear_argument_errors():
     (1, 32, 16, 128 * 37),  # an odd number of 128-point tiles, fewer tiles than CTAs
     (3, 32, 32, 4096),
     (2, 16, 16, 128 * 700), # more tiles than CTAs: every CTA walks several, partial sums over CTAs
+    (2, 20, 20, 1024),      # the paper's width: channel counts padded to the MMA tiles inside the kernel
+    (1, 8, 24, 128 * 5),
+    (2, 12, 9, 256),
     (2, 3, 16, 1000),       # channel counts of a lifting layer: the FFMA kernels
     (2, 16, 1, 520),        # ... and of a projection layer
 ])
