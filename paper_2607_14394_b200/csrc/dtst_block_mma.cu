@@ -39,17 +39,19 @@ __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-template <int CI, int CO>
+template <int CI, int CO, int CIN, int CON>
 __global__ void __launch_bounds__(128, 3)
 linear_backward_mma_kernel(const float* __restrict__ gz, const float* __restrict__ x, float* __restrict__ gx,
                            const float* __restrict__ Wb, float* __restrict__ partial, int B, long long P, int mode_gx,
                            int want_gw, int want_gb, int ci, int co) {
-  // CI, CO: the channel counts rounded up to 16 or 32 (the MMA tiles); ci <= CI, co <= CO the real ones.  The rows
-  // of the staged tiles that belong to no channel are zero, as are the weights in front of them.
-  static_assert(CI % 16 == 0 && CO % 16 == 0 && CI <= 32 && CO <= 32, "channel counts");
+  // CI, CO: the channel counts rounded up to 16 or 32 (the 16-row MMA operand), CIN, CON rounded up to 8, 16, 24
+  // or 32 (the 8-wide operands); ci, co the real ones.  The rows of the staged tiles that belong to no channel are
+  // zero, as are the weights in front of them.
+  static_assert(CI % 16 == 0 && CO % 16 == 0 && CI <= 32 && CO <= 32 && CIN % 8 == 0 && CON % 8 == 0 && CIN <= CI &&
+                    CON <= CO, "channel counts");
   constexpr int ROWS = CO + CI;
-  constexpr int MTO = CO / 16, NTI = CI / 8;   // weight gradient: m-tiles over o, n-tiles over i
-  constexpr int MTI = CI / 16, KSO = CO / 8;   // input gradient: m-tiles over i, k-steps over o
+  constexpr int MTO = CO / 16, NTI = CIN / 8;   // weight gradient: m-tiles over o, n-tiles over i
+  constexpr int MTI = CI / 16, KSO = CON / 8;   // input gradient: m-tiles over i, k-steps over o
   pdl_trigger();
   extern __shared__ __align__(16) float lb_s[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g8 = lane >> 2, t4 = lane & 3;
@@ -238,11 +240,11 @@ linear_backward_mma_kernel(const float* __restrict__ gz, const float* __restrict
   }
 }
 
-template <int CI, int CO>
+template <int CI, int CO, int CIN, int CON>
 cudaError_t launch_t(const float* gz, const float* x, float* gx, int mode_gx, const float* Wb, float* partial, int B,
                      long long P, int want_gw, int want_gb, int max_ctas, int* ctas_out, int ci, int co,
                      cudaStream_t st) {
-  auto kern = linear_backward_mma_kernel<CI, CO>;
+  auto kern = linear_backward_mma_kernel<CI, CO, CIN, CON>;
   size_t smem = (size_t)2 * (CO + CI) * kMSP * 4;
   const size_t red = (size_t)4 * (CO * CI + CO) * 4;
   if (smem < red) smem = red;
@@ -273,14 +275,20 @@ bool linear_backward_mma_supported(int Ci, int Co, long long P) {
 cudaError_t launch_linear_backward_mma(const float* gz, const float* x, float* gx, int mode_gx, const float* Wb,
                                        float* partial, int B, int Ci, int Co, long long P, int want_gw, int want_gb,
                                        int max_ctas, int* ctas_out, cudaStream_t st) {
-  const int cip = Ci <= 16 ? 16 : 32, cop = Co <= 16 ? 16 : 32;
-#define DTST_CALL(c1, c2) \
-  if (cip == c1 && cop == c2) \
-    return launch_t<c1, c2>(gz, x, gx, mode_gx, Wb, partial, B, P, want_gw, want_gb, max_ctas, ctas_out, Ci, Co, st);
-  DTST_CALL(16, 16)
-  DTST_CALL(16, 32)
-  DTST_CALL(32, 16)
-  DTST_CALL(32, 32)
+  // classes of a channel count: up to 16 -> tiles (16 | 16), up to 24 -> (32 | 24), up to 32 -> (32 | 32)
+  const int ki = Ci <= 16 ? 0 : (Ci <= 24 ? 1 : 2), ko = Co <= 16 ? 0 : (Co <= 24 ? 1 : 2);
+#define DTST_CALL(a, b, c16, d16, c8, d8) \
+  if (ki == a && ko == b) \
+    return launch_t<c16, d16, c8, d8>(gz, x, gx, mode_gx, Wb, partial, B, P, want_gw, want_gb, max_ctas, ctas_out, Ci, Co, st);
+  DTST_CALL(0, 0, 16, 16, 16, 16)
+  DTST_CALL(0, 1, 16, 32, 16, 24)
+  DTST_CALL(0, 2, 16, 32, 16, 32)
+  DTST_CALL(1, 0, 32, 16, 24, 16)
+  DTST_CALL(1, 1, 32, 32, 24, 24)
+  DTST_CALL(1, 2, 32, 32, 24, 32)
+  DTST_CALL(2, 0, 32, 16, 32, 16)
+  DTST_CALL(2, 1, 32, 32, 32, 24)
+  DTST_CALL(2, 2, 32, 32, 32, 32)
 #undef DTST_CALL
   return cudaErrorNotSupported;
 }
