@@ -449,7 +449,7 @@ cudaError_t launch_linear_backward(const float* gz, const float* x, float* gx, i
   const long long tiles = (long long)B * ((P + kTP - 1) / kTP);
   if (tiles <= 0) return cudaSuccess;
   if (linear_backward_mma_supported(Ci, Co, P)) {
-    // 8 to 32 channels on both sides: both products on the tensor cores (dtst_block_mma.cu)
+    // up to 32 channels per side, 20 or more together: both products on the tensor cores (dtst_block_mma.cu)
     const int want = (gWb != nullptr || gb != nullptr) ? 1 : 0;
     int rows = 0;
     cudaError_t em = launch_linear_backward_mma(gz, x, gx, gx != nullptr ? mode_gx : 0, Wb, partial, B, Ci, Co, P, want,

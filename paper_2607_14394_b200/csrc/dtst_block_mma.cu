@@ -266,29 +266,32 @@ cudaError_t launch_t(const float* gz, const float* x, float* gx, int mode_gx, co
 
 }  // namespace
 
-// 8 to 32 channels on both sides (rounded up to 16 or 32 inside), whole tiles of points
+// up to 32 channels on both sides (rounded up to the MMA tiles inside), at least 20 together (below that the products
+// are a few multiply-adds per value and the FFMA kernel serves), whole tiles of points
 bool linear_backward_mma_supported(int Ci, int Co, long long P) {
-  return Ci >= 8 && Ci <= 32 && Co >= 8 && Co <= 32 && P % kMTP == 0 && P > 0;
+  return Ci >= 1 && Ci <= 32 && Co >= 1 && Co <= 32 && Ci + Co >= 20 && P % kMTP == 0 && P > 0;
 }
 
 // Launches the kernel above; *ctas_out = rows of `partial` that were written (the caller reduces them).
 cudaError_t launch_linear_backward_mma(const float* gz, const float* x, float* gx, int mode_gx, const float* Wb,
                                        float* partial, int B, int Ci, int Co, long long P, int want_gw, int want_gb,
                                        int max_ctas, int* ctas_out, cudaStream_t st) {
-  // classes of a channel count: up to 16 -> tiles (16 | 16), up to 24 -> (32 | 24), up to 32 -> (32 | 32)
-  const int ki = Ci <= 16 ? 0 : (Ci <= 24 ? 1 : 2), ko = Co <= 16 ? 0 : (Co <= 24 ? 1 : 2);
+  // classes of a channel count: up to 8 -> tiles (16 | 8), up to 16 -> (16 | 16), up to 24 -> (32 | 24), up to 32 -> (32 | 32)
+  auto cls = [](int c) { return c <= 8 ? 0 : (c <= 16 ? 1 : (c <= 24 ? 2 : 3)); };
+  const int ki = cls(Ci), ko = cls(Co);
 #define DTST_CALL(a, b, c16, d16, c8, d8) \
   if (ki == a && ko == b) \
     return launch_t<c16, d16, c8, d8>(gz, x, gx, mode_gx, Wb, partial, B, P, want_gw, want_gb, max_ctas, ctas_out, Ci, Co, st);
-  DTST_CALL(0, 0, 16, 16, 16, 16)
-  DTST_CALL(0, 1, 16, 32, 16, 24)
-  DTST_CALL(0, 2, 16, 32, 16, 32)
-  DTST_CALL(1, 0, 32, 16, 24, 16)
-  DTST_CALL(1, 1, 32, 32, 24, 24)
-  DTST_CALL(1, 2, 32, 32, 24, 32)
-  DTST_CALL(2, 0, 32, 16, 32, 16)
-  DTST_CALL(2, 1, 32, 32, 32, 24)
-  DTST_CALL(2, 2, 32, 32, 32, 32)
+#define DTST_ROW(a, c16, c8)            \
+  DTST_CALL(a, 0, c16, 16, c8, 8)       \
+  DTST_CALL(a, 1, c16, 16, c8, 16)      \
+  DTST_CALL(a, 2, c16, 32, c8, 24)      \
+  DTST_CALL(a, 3, c16, 32, c8, 32)
+  DTST_ROW(0, 16, 8)
+  DTST_ROW(1, 16, 16)
+  DTST_ROW(2, 32, 24)
+  DTST_ROW(3, 32, 32)
+#undef DTST_ROW
 #undef DTST_CALL
   return cudaErrorNotSupported;
 }

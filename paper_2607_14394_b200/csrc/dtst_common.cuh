@@ -222,7 +222,8 @@ cudaError_t launch_linear_backward(const float* gz, const float* x, float* gx, i
                                    float* gb, float* partial, int B, int Ci, int Co, long long P, cudaStream_t st,
                                    long long* launches);
 cudaError_t launch_gelu_backward(const float* g, const float* z, float* gz, long long n, cudaStream_t st);
-// Tensor-core version of the pass below for 8 to 32 channels on both sides and points % 128 == 0 (dtst_block_mma.cu);
+// Tensor-core version of the pass below for up to 32 channels per side (at least 20 together) and points % 128 == 0
+// (dtst_block_mma.cu);
 // *ctas_out = rows of `partial` written.
 bool linear_backward_mma_supported(int Ci, int Co, long long P);
 cudaError_t launch_linear_backward_mma(const float* gz, const float* x, float* gx, int mode_gx, const float* Wb,

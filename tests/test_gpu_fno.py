@@ -69,7 +69,11 @@ def test_pointwise_linear_argument_errors():
     (2, 20, 20, 1024),      # the paper's width: channel counts padded to the MMA tiles inside the kernel
     (1, 8, 24, 128 * 5),
     (2, 12, 9, 256),
-    (2, 3, 16, 1000),       # channel counts of a lifting layer: the FFMA kernels
+    (2, 5, 20, 1024),       # a lifting layer and a projection layer of the paper's FNO on the tensor cores
+    (2, 20, 5, 1024),
+    (1, 1, 32, 256),
+    (1, 32, 1, 256),
+    (2, 3, 16, 1000),       # points not a multiple of the tile, or few channels on both sides: the FFMA kernels
     (2, 16, 1, 520),        # ... and of a projection layer
 ])
 def test_pointwise_linear_forward_and_backward(B, Ci, Co, P):
