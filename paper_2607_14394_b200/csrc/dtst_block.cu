@@ -408,6 +408,9 @@ static cudaError_t launch_epilogue_any(bool linear, const float* x, float* out, 
     (void)launch_pdl(k2, dim3((unsigned)bl), dim3(256), smem, st, x, out, z, Wb, B, Co, P);                        \
     return cudaGetLastError();                                                                                     \
   }
+  DTST_REGX(3, 4)
+  DTST_REGX(4, 4)
+  DTST_REGX(5, 4)
   DTST_REGX(8, 4)
   DTST_REGX(16, 4)
   DTST_REGX(20, 4)
