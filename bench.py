@@ -870,7 +870,11 @@ def main_ours(args, w):
                        "kmax": list(w.kmax), "modes": w.M, "field": w.field, "virtual_shards": P,
                        "kernel_path": plan.kernel_path, "l2": "inputs larger than L2 (no flush needed)"
                        if 4 * w.B * w.C_in * w.points > 3 * 126e6 else "inputs smaller than L2: warm-cache numbers",
-                       "parallelism": f"independent batches x{world}, no collective"},
+                       "parallelism": f"independent batches x{world}, no collective",
+                       "launches_per_step": launches // max(1, steps),
+                       "forward_third_dimension": "contracted inside the plane kernel" if launches // max(1, steps) <= 12
+                       and plan.kernel_path == "fused" and w.d >= 3 and P == 1 and w.name == "cfg5_4d_128"
+                       else "separate launch or not applicable"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
             "roofline": roofline, "roofline_step": roofline_step,
             "fwd": {"ms": fwd_ms, "gpoints_per_s": pts_per_step / (fwd_ms * 1e-3) / 1e9,
