@@ -40,7 +40,8 @@ __device__ __forceinline__ void cp_async_wait() {
 }
 
 template <int CI, int CO, int CIN, int CON>
-__global__ void __launch_bounds__(128, 3)
+// (four CTAs per SM up to 16 + 16 channels, where the fragments leave room for it: 4 % faster than three)
+__global__ void __launch_bounds__(128, (CI <= 16 && CO <= 16) ? 4 : 3)
 linear_backward_mma_kernel(const float* __restrict__ gz, const float* __restrict__ x, float* __restrict__ gx,
                            const float* __restrict__ Wb, float* __restrict__ partial, int B, long long P, int mode_gx,
                            int want_gw, int want_gb, int ci, int co) {
