@@ -1290,7 +1290,10 @@ inv_plane_kernel(const __grid_constant__ CUtensorMap out_map, const float2* __re
 template <int N3, int K3, int N2, int K2>
 cudaError_t plane_fwd(const float* x, float2* out, long long rows, float scale, int herm, int* status,
                                const RingDebug& dbg, cudaStream_t st) {
-  constexpr int W = 7;   // consumer warps (+ the producer warp = 2 warps per scheduler; 8 or 10 consumers measured slower)
+  // consumer warps (+ the producer warp = 2 warps per scheduler; 8 or 10 consumers measured slower on the HBM-bound
+  // shapes).  With half of the contiguous extent retained (k3 = N3 / 2) the kernel is bound by its arithmetic and
+  // 11 warps at 168 registers are 4 % faster than 7 at 232.
+  constexpr int W = (N3 == 32 && K3 == 16) ? 11 : 7;
   using Cfg = PlaneCfg<N3, K3, N2, K2>;
   const SmemPlan sp = smem_plan<Cfg, K2, K3, W>();
   if (sp.stages < 2 * Cfg::SPT) return cudaErrorInvalidConfiguration;
