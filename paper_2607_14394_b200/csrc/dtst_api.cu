@@ -130,8 +130,8 @@ bool use_row(const dtst_plan* p) {
   if (p->d == 1 && p->P > 1) return false;
   long long rows = (long long)p->B * (p->C_in > p->C_out ? p->C_in : p->C_out);
   for (int i = 0; i < a; ++i) rows *= p->Nl[i];
-  if (rows >= (1ll << 31)) return false;   // 32-bit TMA coordinates
-  return row_supported((int)p->Ng[a], p->kmax[a]);
+  if (row_supported((int)p->Ng[a], p->kmax[a])) return rows < (1ll << 31);   // 32-bit TMA coordinates
+  return rowg_supported((int)p->Ng[a], p->kmax[a]);   // any extent: the cp.async-fed kernels of dtst_rowg.cu
 }
 
 // True when no stage of any transform of this plan falls back to the generic one-thread-per-output kernel: the
@@ -509,9 +509,11 @@ dtst_status run_forward_row(dtst_plan* p, const float* x, float2* Xhat, int Cn, 
   float2* t1 = (d == 1) ? Xhat : reinterpret_cast<float2*>(ws + L.bufA);
   {
     KernelTimer kt(p, DTST_KERNEL_GRID_READ, st);
-    if (cuda_failed(p, launch_row_contract(x, t1, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0,
-                                           reinterpret_cast<int*>(ws + L.status), st)))
-      return DTST_ERR_CUDA;
+    const cudaError_t e = row_supported((int)p->Ng[a], p->kmax[a])
+                              ? launch_row_contract(x, t1, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0,
+                                                    reinterpret_cast<int*>(ws + L.status), st)
+                              : launch_rowg_contract(x, t1, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, st);
+    if (cuda_failed(p, e)) return DTST_ERR_CUDA;
   }
   ++p->launches;
   if (d == 1) return DTST_OK;
@@ -529,8 +531,10 @@ dtst_status run_inverse_row(dtst_plan* p, const float2* Yhat, float* y, int Cn, 
   long long rows = (long long)p->B * Cn;
   for (int i = 0; i < a; ++i) rows *= p->Nl[i];
   KernelTimer kt(p, DTST_KERNEL_GRID_WRITE, st);
-  if (cuda_failed(p, launch_row_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, st)))
-    return DTST_ERR_CUDA;
+  const cudaError_t e = row_supported((int)p->Ng[a], p->kmax[a])
+                            ? launch_row_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, st)
+                            : launch_rowg_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, st);
+  if (cuda_failed(p, e)) return DTST_ERR_CUDA;
   ++p->launches;
   return DTST_OK;
 }

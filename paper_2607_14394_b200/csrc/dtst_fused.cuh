@@ -51,4 +51,12 @@ cudaError_t launch_row_contract(const float* x, float2* out, long long rows, int
 cudaError_t launch_row_expand(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm,
                               cudaStream_t st);
 
+// Row kernels for any contiguous extent (dtst_rowg.cu): N3 <= 512 (odd extents included), k3 <= 32; cp.async-fed,
+// no tensor map.  Used where row_supported() says no.
+bool rowg_supported(int N3, int K3);
+cudaError_t launch_rowg_contract(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm,
+                                 cudaStream_t st);
+cudaError_t launch_rowg_expand(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm,
+                               cudaStream_t st);
+
 }  // namespace dtst

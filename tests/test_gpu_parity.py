@@ -393,6 +393,36 @@ def test_more_plane_shapes_run_fused_and_match_the_oracle(case):
     run_layer_and_check(w, "auto", P=4)
 
 
+# ------------------------------------------------------------------ contiguous extents that are no multiple of 32
+ANY_EXTENT = [
+    # name, B, Ci, Co, N, kmax, every stage streaming?
+    # the paper's own grid in small: a time axis of 30 points with all 16 one-sided modes (the Nyquist mode included)
+    ("g_paper_t30", 1, 2, 2, (16, 16, 32, 30), (4, 8, 8, 16), True),
+    ("g_100", 1, 2, 3, (32, 32, 100), (8, 8, 12), True),
+    ("g_odd_45", 2, 1, 2, (16, 32, 45), (4, 4, 12), True),           # odd extent: the middle sample has no partner
+    ("g_odd_7_ragged", 1, 3, 1, (5, 7, 7), (2, 3, 4), False),        # 105 rows: a ragged last task, k3 = N3/2 + 1
+    ("g_k3_20", 1, 2, 2, (32, 96), (8, 20), True),                   # three frequency tiles
+    ("g_k3_32_odd_rows", 1, 1, 1, (9, 330), (4, 32), False),         # four frequency tiles, 9 rows
+    ("g_k3_odd", 1, 2, 2, (32, 50), (8, 9), False),                  # odd mode count: 8-byte stores
+    ("g_1d", 2, 3, 2, (90,), (17,), True),
+    ("g_512", 1, 2, 2, (8, 512), (4, 16), True),                     # longer than the tensor-map kernels take
+]
+
+
+@pytest.mark.parametrize("case", ANY_EXTENT, ids=[c[0] for c in ANY_EXTENT])
+def test_any_contiguous_extent_runs_on_the_row_kernels(case):
+    name, B, Ci, Co, N, k, streaming = case
+    w = I.custom_workload(name, B, Ci, Co, N, k, field="grf", seed=31)
+    plan = _plan(w)
+    assert plan.kernel_path == "row"
+    if streaming:
+        plan.require_fast_path()
+    plan.close()
+    run_layer_and_check(w, "auto")
+    if N[0] % 4 == 0 and len(N) > 1:
+        run_layer_and_check(w, "auto", P=4)
+
+
 # ------------------------------------------------------------------ third dimension inside the forward plane kernel
 @pytest.mark.parametrize("N,k,B,C,P", [
     ((32, 128, 64), (16, 16, 8), 1, 3, 1),        # d = 3: the kernel writes the spectrum itself; N1 = 2 k1 (all of dim 0)
