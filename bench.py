@@ -579,20 +579,22 @@ def block_summary(torch, w, x, g, W, steps, peak):
 
 def fno_summary(torch, steps=5):
     """A whole synthetic FNO with the paper's architecture (Section "Experimental Setup": 4 Fourier blocks, modes
-    (8, 8, 8, 16), 5 fields in and out, grid 128 x 128 x 64 with a time axis of 32) forward and backward on this
-    GPU, every step in the library's kernels: at the paper's width 20 and at width 32 (the channel counts the
+    (8, 8, 8, 16), 5 fields in and out, grid 128 x 128 x 64 with a time axis of 32 or 30) forward and backward on
+    this GPU, every step in the library's kernels: at the paper's width 20 and at width 32 (the channel counts the
     tensor-core bypass kernels serve).  Random-init weights, synthetic input; context for the paper's multi-GPU
     figures, not a like-for-like comparison."""
     from paper_2607_14394_b200 import FNO
-    out = {"grid": [128, 128, 64, 32], "modes": [8, 8, 8, 16], "layers": 4, "fields": 5, "steps": steps,
+    out = {"grid": [128, 128, 64, "time_axis"], "modes": [8, 8, 8, 16], "layers": 4, "fields": 5, "steps": steps,
            "paper_context": "the paper reports 148.3 ms forward / 246.8 ms backward for this architecture at "
                             "128^3 on 4 V100s (its Table 5); another machine, another grid: context only"}
-    for width in (20, 32):
+    # (time axis, width, key): the paper's operation count is on a time axis of 30 points, which runs on the row
+    # kernels for any extent; 32 points run on the plane kernels
+    for T, width, key in ((32, 20, "width_20"), (32, 32, "width_32"), (30, 20, "t30_width_20")):
         try:
-            net = FNO((128, 128, 64, 32), (8, 8, 8, 16), 1, 5, 5, width, 4, seed=11)
+            net = FNO((128, 128, 64, T), (8, 8, 8, 16), 1, 5, 5, width, 4, seed=11)
             gen = torch.Generator(device="cuda").manual_seed(12)
-            a = torch.randn((1, 5, 128, 128, 64, 32), device="cuda", generator=gen)
-            gu = torch.randn((1, 5, 128, 128, 64, 32), device="cuda", generator=gen)
+            a = torch.randn((1, 5, 128, 128, 64, T), device="cuda", generator=gen)
+            gu = torch.randn((1, 5, 128, 128, 64, T), device="cuda", generator=gen)
             for _ in range(2):
                 net.forward(a)
                 net.backward(gu)
@@ -609,13 +611,13 @@ def fno_summary(torch, steps=5):
                 fwd += e[0].elapsed_time(e[1])
                 bwd += e[1].elapsed_time(e[2])
             ok = net.plan.status() == 0
-            out[f"width_{width}"] = {"fwd_ms": fwd / steps, "bwd_ms": bwd / steps, "status_ok": ok,
-                                     "kernel_path": net.plan.kernel_path}
+            out[key] = {"fwd_ms": fwd / steps, "bwd_ms": bwd / steps, "status_ok": ok,
+                        "kernel_path": net.plan.kernel_path, "time_axis": T}
             net.close()
             del net, a, gu
             torch.cuda.empty_cache()
         except Exception as ex:
-            out[f"width_{width}"] = {"error": f"{type(ex).__name__}: {ex}"[:200]}
+            out[key] = {"error": f"{type(ex).__name__}: {ex}"[:200]}
     return out
 
 
@@ -1143,7 +1145,7 @@ def main():
     ap.add_argument("--no-other-configs", action="store_true")
     args = ap.parse_args()
     from paper_2607_14394_b200 import inputs
-    w = inputs.WORKLOADS[args.config]
+    w = inputs.workload(args.config)
     if args.channels > 0:
         w = inputs.custom_workload(f"{w.name}_c{args.channels}", w.B, args.channels, args.channels, w.N, w.kmax,
                                    field=w.field, seed=w.seed, virtual_shards=w.virtual_shards)

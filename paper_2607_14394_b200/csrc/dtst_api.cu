@@ -134,6 +134,17 @@ bool use_row(const dtst_plan* p) {
   return rowg_supported((int)p->Ng[a], p->kmax[a]);   // any extent: the cp.async-fed kernels of dtst_rowg.cu
 }
 
+// Row path with the second-last dimension inside the grid-side kernel (dtst_rowg.cu): for contiguous extents the
+// tensor-map row kernels do not take, when that dimension is whole, carries no offset and is not cut into slabs.
+bool use_planeg(const dtst_plan* p) {
+  static const bool off = std::getenv("DTST_NO_PLANEG") != nullptr;   // diagnostic: keep the separate stage
+  if (off || !use_row(p) || p->d < 2) return false;
+  const int a = p->d - 1, b = p->d - 2;
+  if (row_supported((int)p->Ng[a], p->kmax[a])) return false;
+  if (p->Nl[b] != p->Ng[b] || p->off[b] != 0 || (b == 0 && p->P > 1)) return false;
+  return planeg_supported((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b]);
+}
+
 // True when no stage of any transform of this plan falls back to the generic one-thread-per-output kernel: the
 // grid-side stage runs on a plane or row kernel and every other dimension on a folded or slab kernel, in both
 // directions.
@@ -141,7 +152,7 @@ bool all_streaming(const dtst_plan* p) {
   if (p->complex_io) return false;   // the contiguous dimension of a complex plan runs on the generic kernel
   int first;
   if (use_fused(p)) first = p->d - 3;
-  else if (use_row(p)) first = p->d - 2;
+  else if (use_row(p)) first = use_planeg(p) ? p->d - 3 : p->d - 2;
   else return false;
   for (int j = first; j >= 0; --j) {
     if (!(use_slab(p, j) || use_mid(p, j))) return false;          // contraction
@@ -507,6 +518,19 @@ dtst_status run_forward_row(dtst_plan* p, const float* x, float2* Xhat, int Cn, 
   long long rows = (long long)p->B * Cn;
   for (int i = 0; i < a; ++i) rows *= p->Nl[i];
   float2* t1 = (d == 1) ? Xhat : reinterpret_cast<float2*>(ws + L.bufA);
+  if (use_planeg(p)) {
+    const int b = d - 2;
+    float2* dst = (d == 2) ? Xhat : t1;
+    {
+      KernelTimer kt(p, DTST_KERNEL_GRID_READ, st);
+      if (cuda_failed(p, launch_planeg_contract(x, dst, rows / p->Ng[b], (int)p->Ng[a], p->kmax[a], (int)p->Ng[b],
+                                                p->kmax[b], scale, herm ? 1 : 0, st)))
+        return DTST_ERR_CUDA;
+    }
+    ++p->launches;
+    if (d == 2) return DTST_OK;
+    return forward_stages(p, t1, d - 3, 1, Xhat, Cn, 1.0f, false, st);
+  }
   {
     KernelTimer kt(p, DTST_KERNEL_GRID_READ, st);
     const cudaError_t e = row_supported((int)p->Ng[a], p->kmax[a])
@@ -524,13 +548,22 @@ dtst_status run_inverse_row(dtst_plan* p, const float2* Yhat, float* y, int Cn, 
                             cudaStream_t st) {
   const int d = p->d, a = d - 1;
   const float2* src = Yhat;
-  if (d > 1) {
-    dtst_status s = inverse_stages_complex(p, Yhat, d - 2, -1, Cn, &src, nullptr, st);
+  const bool pg = use_planeg(p);
+  if (d > (pg ? 2 : 1)) {
+    dtst_status s = inverse_stages_complex(p, Yhat, pg ? d - 3 : d - 2, -1, Cn, &src, nullptr, st);
     if (s != DTST_OK) return s;
   }
   long long rows = (long long)p->B * Cn;
   for (int i = 0; i < a; ++i) rows *= p->Nl[i];
   KernelTimer kt(p, DTST_KERNEL_GRID_WRITE, st);
+  if (pg) {
+    const int b = d - 2;
+    if (cuda_failed(p, launch_planeg_expand(src, y, rows / p->Ng[b], (int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b],
+                                            scale, herm ? 1 : 0, st)))
+      return DTST_ERR_CUDA;
+    ++p->launches;
+    return DTST_OK;
+  }
   const cudaError_t e = row_supported((int)p->Ng[a], p->kmax[a])
                             ? launch_row_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, st)
                             : launch_rowg_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, st);

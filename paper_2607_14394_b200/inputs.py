@@ -60,6 +60,18 @@ WORKLOADS = {
                             virtual_shards=8),
 }
 
+# The paper's own layer (Section "Experimental Setup": grid 128 x 128 x 64, modes (8, 8, 8, 16), width 20), with the
+# time axis of its operation count (30 points: no multiple of 32, every one-sided mode retained) and with 32 points.
+# Not part of the benchmark definition: bench.py takes them by name, the tests do not iterate over them.
+EXTRA_WORKLOADS = {
+    "paper_4d_t30": Workload("paper_4d_t30", 1, 20, 20, (128, 128, 64, 30), (8, 8, 8, 16), "grf", 1006),
+    "paper_4d_t32": Workload("paper_4d_t32", 1, 20, 20, (128, 128, 64, 32), (8, 8, 8, 16), "grf", 1007),
+}
+
+
+def workload(name: str) -> Workload:
+    return WORKLOADS[name] if name in WORKLOADS else EXTRA_WORKLOADS[name]
+
 
 def _channel_rng(seed: int, tag: int, b: int, c: int) -> np.random.Generator:
     # One independent PCG64 stream per (tensor tag, batch, channel), so a single

@@ -406,6 +406,13 @@ ANY_EXTENT = [
     ("g_k3_odd", 1, 2, 2, (32, 50), (8, 9), False),                  # odd mode count: 8-byte stores
     ("g_1d", 2, 3, 2, (90,), (17,), True),
     ("g_512", 1, 2, 2, (8, 512), (4, 16), True),                     # longer than the tensor-map kernels take
+    # the second-last dimension inside the kernel: 24 and 32 modes (two mode tiles), 8 modes (half a tile), few
+    # frequencies (two column tiles), 16-row tasks, and more planes than warps on the GPU (the ring crosses planes)
+    ("g_plane_k2_12", 1, 2, 2, (16, 64, 60), (4, 12, 16), True),
+    ("g_plane_k2_16_k3_6", 1, 1, 2, (16, 32, 44), (8, 16, 6), False),
+    ("g_plane_k2_4", 2, 1, 1, (8, 96, 30), (4, 4, 11), False),
+    ("g_plane_200", 1, 2, 1, (8, 48, 200), (4, 8, 16), True),
+    ("g_plane_many", 2, 4, 4, (256, 32, 30), (8, 8, 16), True),
 ]
 
 
