@@ -23,7 +23,7 @@ namespace dtst {
 namespace {
 
 constexpr size_t kGSmemLimit = 227 * 1024;
-constexpr int kGMaxWarps = 12;
+constexpr int kGMaxWarps = 16;
 
 __device__ __forceinline__ void g_cp_async16(float* smem_dst, const float* gsrc) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
@@ -329,12 +329,18 @@ rowg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long lo
 // operand of the second stage's k-step over these eight rows - [modes x 8 rows] x [8 rows x real columns] - once the
 // MMA's k index is read as row 2 k (k < 4) or 2 (k - 4) + 1 and the four n-tiles as (re, im) x (f < 8, f >= 8):
 // a sum does not care how its terms or its columns are named, and the basis table is built with the same naming.
-// Nothing is transposed through shared memory; the plane's [2 K2][k3] sums live in C fragments until its last row.
+// Nothing is transposed through shared memory; the plane's sums live in C fragments until its last row.
+// The second stage is folded over the sign of the mode: cos(k phi) serves +k and -k, sin(k phi) too up to its sign, so
+// its 16-row operand holds [cos k phi, k < K2 | sin k phi, k = 1..K2] (2 K2 rows, ONE product instead of a cosine and a
+// sine product over all 2 K2 modes) and Z_{+k} = A_k - i B_k, Z_{-k} = A_k + i B_k are formed at the plane's end; the
+// one term left over, A_{K2} = sum cos(K2 phi) T of the unpaired mode -K2, runs on FFMA.
 //
 // Expansion.  The second dimension first: [16 rows x modes] x [modes x (re, im) columns] from the plane's spectrum
 // (a padded copy in shared memory, fetched one plane ahead); its C fragment (rows g8 / g8 + 8, the complex value of
 // frequency 4 nc + t4) is exactly the row operand of the contiguous stage (frequency 8 ks + t4 + 4 half <-> n-tile
-// 2 ks + half), which then runs as in rowg_expand_kernel.
+// 2 ks + half), which then runs as in rowg_expand_kernel.  The same fold: U = sum_k cos(k phi) E_k + sin(k phi) (i O_k)
+// with E_k = V_k + V_{-k}, O_k = V_k - V_{-k} formed once per plane in shared memory (the factor i is a swap of the
+// real and imaginary columns), one product over 2 K2 entries; cos(K2 phi) V_{-K2} is added on FFMA.
 // =============================================================================================
 __device__ __forceinline__ void g_cp_async8(float* smem_dst, const float2* gsrc) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
@@ -347,6 +353,16 @@ __device__ __forceinline__ float g_basis2(int part, int p, int n, int N2, int K2
   double s, c;
   sincospi(2.0 * (double)((k * n) % N2) / (double)N2, &s, &c);
   return part == 0 ? (float)c : (float)s;
+}
+
+// entry r of the folded second-stage basis at row n: cos(2 pi r n / N2) for r < K2, sin(2 pi (r - K2 + 1) n / N2) for
+// K2 <= r < 2 K2, zero beyond
+__device__ __forceinline__ float g_basis2f(int r, int n, int N2, int K2) {
+  if (r >= 2 * K2) return 0.f;
+  const long long k = r < K2 ? r : r - K2 + 1;
+  double s, c;
+  sincospi(2.0 * (double)((k * n) % N2) / (double)N2, &s, &c);
+  return r < K2 ? (float)c : (float)s;
 }
 
 __device__ __forceinline__ void g_split4(const float4& v, uint32_t (&hi)[4], uint32_t (&lo)[4]) {
@@ -365,11 +381,12 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
   constexpr int TR = 16 * MT, GPT = 2 * MT;   // rows and 8-row groups per task
   extern __shared__ float4 rg_smem[];
   const int half = N3 / 2, H = (N3 + 1) / 2, KS = (H + 7) / 8;
-  const bool odd = (N3 & 1) != 0;
   const int NG = N2 / 8, TP = N2 / TR;
   float4* atab = rg_smem;                                   // [part][ks][hi | lo][lane]: the row stage's 16-row operand
-  float4* a2tab = atab + (size_t)2 * KS * 2 * 32;           // [part][group][mtm][lane]: the second stage's, unsplit
-  float* ring = reinterpret_cast<float*>(a2tab + (size_t)2 * NG * MTM * 32);
+  float4* a2tab = atab + (size_t)2 * KS * 2 * 32;           // [group][mtm][lane]: the second stage's, folded, unsplit
+  float* cK = reinterpret_cast<float*>(a2tab + (size_t)NG * MTM * 32);   // cos(2 pi K2 n / N2)
+  float* ring = cK + ((N2 + 3) & ~3);
+  constexpr int SCW = 34, SCRF = ((16 * MTM + 1) * SCW + 3) & ~3;   // per-warp scratch of the plane's end: rows of 34 floats
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g8 = lane >> 2, t4 = lane & 3;
   const int W = blockDim.x >> 5;
 
@@ -386,20 +403,15 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
     atab[((size_t)(part * KS + ks) * 2 + 1) * 32 + l] =
         make_float4(__uint_as_float(lo[0]), __uint_as_float(lo[1]), __uint_as_float(lo[2]), __uint_as_float(lo[3]));
   }
-  for (int e = threadIdx.x; e < 2 * NG * MTM * 32; e += blockDim.x) {
-    const int l = e & 31;
-    int r = e >> 5;
-    const int mtm = r % MTM;
-    r /= MTM;
-    const int grp = r % NG, part = r / NG;
+  for (int e = threadIdx.x; e < NG * MTM * 32; e += blockDim.x) {
+    const int l = e & 31, mtm = (e >> 5) % MTM, grp = (e >> 5) / MTM;
     float v[4];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {                           // A fragment: mode l >> 2 (+8), row 2 (l & 3) (+1)
-      const int pm = 16 * mtm + (l >> 2) + 8 * (q & 1), n = 8 * grp + 2 * (l & 3) + (q >> 1);
-      v[q] = pm < 2 * K2 ? g_basis2(part, pm, n, N2, K2) : 0.f;
-    }
+    for (int q = 0; q < 4; ++q)                             // A fragment: basis row l >> 2 (+8), grid row 2 (l & 3) (+1)
+      v[q] = g_basis2f(16 * mtm + (l >> 2) + 8 * (q & 1), 8 * grp + 2 * (l & 3) + (q >> 1), N2, K2);
     a2tab[e] = make_float4(v[0], v[1], v[2], v[3]);
   }
+  for (int n = threadIdx.x; n < N2; n += blockDim.x) cK[n] = g_basis2(0, K2, n, N2, K2);   // position K2 is the mode -K2
   float2 rot[2];                                            // frequencies g8 and g8 + 8
 #pragma unroll
   for (int fh = 0; fh < 2; ++fh) {
@@ -412,7 +424,11 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
   __syncthreads();
   pdl_wait();
 
-  float* S = ring + (size_t)warp * ST * stage_floats;
+  float* S = ring + (size_t)warp * (ST * stage_floats + SCRF);
+  float* scr = S + (size_t)ST * stage_floats;
+  if (lane < 4)                                             // the zero slot behind every stage's TR x N3 floats
+    for (int q = 0; q < ST; ++q) S[(size_t)q * stage_floats + TR * N3 + lane] = 0.f;
+  __syncwarp();
   const long long stride = (long long)W * gridDim.x;
   long long pl = (long long)warp * gridDim.x + blockIdx.x;
   long long apl = pl;                                       // the task staged next: plane and place within it
@@ -433,13 +449,16 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
   for (int q = 0; q < ST - 1; ++q) load(q);
   int s = 0;
   for (; pl < planes; pl += stride) {
-    float P[MTM][NC][4], Q[MTM][NC][4];
+    float P[MTM][NC][4];
+    float lw[NC];                                           // this lane's share of the left-over sums A_{K2}
+#pragma unroll
+    for (int nc = 0; nc < NC; ++nc) lw[nc] = 0.f;
 #pragma unroll
     for (int mtm = 0; mtm < MTM; ++mtm)
 #pragma unroll
       for (int nc = 0; nc < NC; ++nc)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) P[mtm][nc][e] = Q[mtm][nc][e] = 0.f;
+        for (int e = 0; e < 4; ++e) P[mtm][nc][e] = 0.f;
     for (int j = 0; j < TP; ++j) {
       load(s == 0 ? ST - 1 : s - 1);
       g_cp_async_wait<ST - 1>();
@@ -447,80 +466,101 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
       const float* T = S + (size_t)s * stage_floats;
 #pragma unroll 1
       for (int gq = 0; gq < GPT; ++gq) {
-        const float* Trow = T + (8 * gq + g8) * N3;         // this lane's row of the group (the B operand's n index)
+        const int rowoff = (8 * gq + g8) * N3;
+        const float* Trow = T + rowoff;                     // this lane's row of the group (the B operand's n index)
+        const int zrel = TR * N3 - rowoff;                  // the stage's zero slot, as a column of this row
         float accC[4] = {0.f, 0.f, 0.f, 0.f}, accS[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 2
-        for (int ks = 0; ks < KS; ++ks) {
-          const float4 ch = atab[((size_t)(0 * KS + ks) * 2 + 0) * 32 + lane], cl = atab[((size_t)(0 * KS + ks) * 2 + 1) * 32 + lane];
-          const float4 sh = atab[((size_t)(1 * KS + ks) * 2 + 0) * 32 + lane], sl = atab[((size_t)(1 * KS + ks) * 2 + 1) * 32 + lane];
+        // one k-step: pairs jj = 8 ks + t4 (+4) from the columns (ja, jb); a pair past the end reads the zero slot twice,
+        // the middle sample of an odd extent once (its sine is exactly zero)
+        auto step = [&](int ks, int ja0, int jb0, int ja1, int jb1) {
+          const float4* at = atab + ks * 64 + lane;
+          const float4 ch = at[0], cl = at[32], sh = at[KS * 64], sl = at[KS * 64 + 32];
+          const float a0 = Trow[ja0], b0 = Trow[jb0], a1 = Trow[ja1], b1 = Trow[jb1];
           uint32_t bsh[2], bsl[2], bdh[2], bdl[2];
-#pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {                  // B fragment: pair t4 (+4)
-            const int jj = 8 * ks + t4 + 4 * hh;
-            const bool in = jj < half, mid = odd && jj == half;
-            const int ja = (in || mid) ? jj : 0, jb = in ? N3 - 1 - jj : ja;
-            const float a = Trow[ja], b = Trow[jb];
-            g_split(in ? a + b : (mid ? a : 0.f), bsh[hh], bsl[hh]);
-            g_split(in ? a - b : 0.f, bdh[hh], bdl[hh]);
-          }
+          g_split(a0 + b0, bsh[0], bsl[0]);
+          g_split(a0 - b0, bdh[0], bdl[0]);
+          g_split(a1 + b1, bsh[1], bsl[1]);
+          g_split(a1 - b1, bdh[1], bdl[1]);
           const uint32_t chv[4] = {__float_as_uint(ch.x), __float_as_uint(ch.y), __float_as_uint(ch.z), __float_as_uint(ch.w)};
           const uint32_t clv[4] = {__float_as_uint(cl.x), __float_as_uint(cl.y), __float_as_uint(cl.z), __float_as_uint(cl.w)};
           const uint32_t shv[4] = {__float_as_uint(sh.x), __float_as_uint(sh.y), __float_as_uint(sh.z), __float_as_uint(sh.w)};
           const uint32_t slv[4] = {__float_as_uint(sl.x), __float_as_uint(sl.y), __float_as_uint(sl.z), __float_as_uint(sl.w)};
           mma3_tf32(accC, chv, clv, bsh[0], bsh[1], bsl[0], bsl[1]);
           mma3_tf32(accS, shv, slv, bdh[0], bdh[1], bdl[0], bdl[1]);
+        };
+#pragma unroll 2
+        for (int ks = 0; ks < KS - 1; ++ks) {               // every pair of these k-steps exists
+          const int jj = 8 * ks + t4;
+          step(ks, jj, N3 - 1 - jj, jj + 4, N3 - 5 - jj);
+        }
+        {
+          const int jj = 8 * (KS - 1) + t4;
+          step(KS - 1, jj < H ? jj : zrel, jj < half ? N3 - 1 - jj : zrel, jj + 4 < H ? jj + 4 : zrel,
+               jj + 4 < half ? N3 - 5 - jj : zrel);
         }
         // X = rot (C - i S) of (frequency g8 + 8 fh, row 2 t4 + q): the second stage's column operand
         uint32_t bh[NC][2], bl[NC][2];
+        const int grp = j * GPT + gq;
+        const float ck0 = cK[8 * grp + 2 * t4], ck1 = cK[8 * grp + 2 * t4 + 1];
 #pragma unroll
-        for (int fh = 0; fh < NC / 2; ++fh)
+        for (int fh = 0; fh < NC / 2; ++fh) {
+          float re[2], im[2];
 #pragma unroll
           for (int q = 0; q < 2; ++q) {
             const float C = accC[2 * fh + q], Sv = accS[2 * fh + q];
-            g_split(rot[fh].x * C + rot[fh].y * Sv, bh[2 * fh][q], bl[2 * fh][q]);          // real part
-            g_split(rot[fh].y * C - rot[fh].x * Sv, bh[2 * fh + 1][q], bl[2 * fh + 1][q]);  // imaginary part
+            re[q] = rot[fh].x * C + rot[fh].y * Sv;
+            im[q] = rot[fh].y * C - rot[fh].x * Sv;
+            g_split(re[q], bh[2 * fh][q], bl[2 * fh][q]);
+            g_split(im[q], bh[2 * fh + 1][q], bl[2 * fh + 1][q]);
           }
-        const int grp = j * GPT + gq;
+          lw[2 * fh] = fmaf(ck0, re[0], fmaf(ck1, re[1], lw[2 * fh]));
+          lw[2 * fh + 1] = fmaf(ck0, im[0], fmaf(ck1, im[1], lw[2 * fh + 1]));
+        }
 #pragma unroll
         for (int mtm = 0; mtm < MTM; ++mtm) {
-          uint32_t ch2[4], cl2[4], sh2[4], sl2[4];
-          g_split4(a2tab[((size_t)(0 * NG + grp) * MTM + mtm) * 32 + lane], ch2, cl2);
-          g_split4(a2tab[((size_t)(1 * NG + grp) * MTM + mtm) * 32 + lane], sh2, sl2);
+          uint32_t ah2[4], al2[4];
+          g_split4(a2tab[(grp * MTM + mtm) * 32 + lane], ah2, al2);
 #pragma unroll
-          for (int nc = 0; nc < NC; ++nc) {
-            mma3_tf32(P[mtm][nc], ch2, cl2, bh[nc][0], bh[nc][1], bl[nc][0], bl[nc][1]);
-            mma3_tf32(Q[mtm][nc], sh2, sl2, bh[nc][0], bh[nc][1], bl[nc][0], bl[nc][1]);
-          }
+          for (int nc = 0; nc < NC; ++nc) mma3_tf32(P[mtm][nc], ah2, al2, bh[nc][0], bh[nc][1], bl[nc][0], bl[nc][1]);
         }
       }
       __syncwarp();   // every lane is done with this stage before it is filled again
       s = s == ST - 1 ? 0 : s + 1;
     }
-    // sum_n (cos - i sin)(Tr + i Ti) = (P_re + Q_im) + i (P_im - Q_re); a C fragment: modes g8 (+8), columns 2 t4 (+1)
-    float2* ob = out + pl * (2 * K2) * K3;
+    // The plane's end.  Rows of the product: A_k = sum cos(k phi) T (k < K2), then B_k = sum sin(k phi) T (k = 1..K2);
+    // a C fragment holds rows g8 (+8) and the columns 2 t4 (+1) of its tile (tile 2 fh + part: frequency 8 fh + column,
+    // real or imaginary part).  Through the warp's scratch rows, so that every output can pick up its A and its B.
 #pragma unroll
     for (int mtm = 0; mtm < MTM; ++mtm)
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int pm = 16 * mtm + g8 + 8 * h;
-        if (pm >= 2 * K2) continue;
+      for (int nc = 0; nc < NC; ++nc)
 #pragma unroll
-        for (int fh = 0; fh < NC / 2; ++fh) {
-          const int f0 = 8 * fh + 2 * t4;
-          float2 r[2];
+        for (int e = 0; e < 4; ++e)
+          scr[(16 * mtm + g8 + 8 * (e >> 1)) * SCW + 2 * (8 * (nc >> 1) + 2 * t4 + (e & 1)) + (nc & 1)] = P[mtm][nc][e];
 #pragma unroll
-          for (int q = 0; q < 2; ++q)
-            r[q] = make_float2(P[mtm][2 * fh][2 * h + q] + Q[mtm][2 * fh + 1][2 * h + q],
-                               P[mtm][2 * fh + 1][2 * h + q] - Q[mtm][2 * fh][2 * h + q]);
-          float2* dst = ob + (long long)pm * K3 + f0;
-          if (f0 + 1 < K3 && (K3 & 1) == 0) {
-            *reinterpret_cast<float4*>(dst) = make_float4(r[0].x, r[0].y, r[1].x, r[1].y);
-          } else {
-            if (f0 < K3) dst[0] = r[0];
-            if (f0 + 1 < K3) dst[1] = r[1];
-          }
-        }
+    for (int nc = 0; nc < NC; ++nc) {                       // the left-over row: add the four lanes that share a column
+      float v = lw[nc];
+      v += __shfl_xor_sync(0xffffffffu, v, 1);
+      v += __shfl_xor_sync(0xffffffffu, v, 2);
+      if (t4 == 0) scr[16 * MTM * SCW + 2 * (8 * (nc >> 1) + g8) + (nc & 1)] = v;
+    }
+    __syncwarp();
+    // Z_{+k} = A_k - i B_k at position k, Z_{-k} = A_k + i B_k at position 2 K2 - k (B_0 = 0, A_{K2} = the left-over row)
+    float2* ob = out + pl * (2 * K2) * K3;
+    for (int idx = lane; idx < 2 * K2 * K3; idx += 32) {
+      const int pm = idx / K3, f = idx - pm * K3;
+      const int k = pm < K2 ? pm : 2 * K2 - pm;
+      const float sg = pm < K2 ? -1.f : 1.f;
+      const float* ar = scr + (k < K2 ? k : 16 * MTM) * SCW + 2 * f;
+      float2 v = make_float2(ar[0], ar[1]);
+      if (k > 0) {
+        const float* br = scr + (K2 + k - 1) * SCW + 2 * f;
+        v.x -= sg * br[1];
+        v.y += sg * br[0];
       }
+      ob[idx] = v;
+    }
+    __syncwarp();   // the scratch rows are read before the next plane's end writes them
   }
 }
 
@@ -538,13 +578,15 @@ planeg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long 
   const bool odd = (N3 & 1) != 0;
   const int NM = N2 / 16, TP = N2 / TR;
   float4* btab = rg_smem;                                   // [part][ks][ntj][lane], split: the contiguous stage's basis
-  float4* a2e = btab + (size_t)2 * KSF * NTJ * 32;          // [part][16-row tile][ks2][lane], unsplit
-  float* warp_area = reinterpret_cast<float*>(a2e + (size_t)2 * NM * KS2 * 32);
+  float4* a2e = btab + (size_t)2 * KSF * NTJ * 32;          // [16-row tile][ks2][lane]: folded basis, unsplit
+  float* cK = reinterpret_cast<float*>(a2e + (size_t)NM * KS2 * 32);   // cos(2 pi K2 n / N2)
+  float* warp_area = cK + ((N2 + 3) & ~3);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g8 = lane >> 2, t4 = lane & 3;
   const int W = blockDim.x >> 5;
-  const int area_floats = stage_floats + 2 * VROWS * kGVS;
+  const int area_floats = stage_floats + (3 * VROWS + 1) * kGVS;
   float* st = warp_area + (size_t)warp * area_floats;       // output staging of a task
   float* Vs = st + stage_floats;                            // [2][VROWS][kGVS]: this plane's and the next plane's spectrum
+  float* Bm = Vs + 2 * VROWS * kGVS;                        // [VROWS + 1][kGVS]: E_k, i O_k and, last row, V_{-K2}
 
   for (int e = threadIdx.x; e < 2 * KSF * NTJ * 32; e += blockDim.x) {
     const int l = e & 31;
@@ -561,22 +603,17 @@ planeg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long 
     }
     btab[e] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(lo[0]), __uint_as_float(lo[1]));
   }
-  for (int e = threadIdx.x; e < 2 * NM * KS2 * 32; e += blockDim.x) {
-    const int l = e & 31;
-    int r = e >> 5;
-    const int ks2 = r % KS2;
-    r /= KS2;
-    const int tile = r % NM, part = r / NM;
+  for (int e = threadIdx.x; e < NM * KS2 * 32; e += blockDim.x) {
+    const int l = e & 31, ks2 = (e >> 5) % KS2, tile = (e >> 5) / KS2;
     float v[4];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {                           // A fragment: row l >> 2 (+8), mode l & 3 (+4)
-      const int n = 16 * tile + (l >> 2) + 8 * (q & 1), pm = 8 * ks2 + (l & 3) + 4 * (q >> 1);
-      v[q] = pm < 2 * K2 ? g_basis2(part, pm, n, N2, K2) : 0.f;
-    }
+    for (int q = 0; q < 4; ++q)                             // A fragment: grid row l >> 2 (+8), basis entry l & 3 (+4)
+      v[q] = g_basis2f(8 * ks2 + (l & 3) + 4 * (q >> 1), 16 * tile + (l >> 2) + 8 * (q & 1), N2, K2);
     a2e[e] = make_float4(v[0], v[1], v[2], v[3]);
   }
-  // the padding of the spectrum copies (modes past 2 K2, columns past 2 k3) meets zero basis entries: it must be finite
-  for (int e = lane; e < 2 * VROWS * kGVS; e += 32) Vs[e] = 0.f;
+  for (int n = threadIdx.x; n < N2; n += blockDim.x) cK[n] = g_basis2(0, K2, n, N2, K2);
+  // the padding of the spectrum copies (entries past 2 K2, columns past 2 k3) meets zero basis entries: it must be finite
+  for (int e = lane; e < (3 * VROWS + 1) * kGVS; e += 32) Vs[e] = 0.f;
   float2 rot[KSF][2];
 #pragma unroll
   for (int ks = 0; ks < KSF; ++ks)
@@ -608,69 +645,99 @@ planeg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long 
     fetch(pl + stride, vb ^ 1);
     g_cp_async_wait<1>();
     __syncwarp();
-    const float* V = Vs + (size_t)vb * VROWS * kGVS;
+    {
+      // E_0 = V_0, E_k = V_k + V_{-k}; i O_k with O_k = V_k - V_{-k} (k < K2), O_{K2} = -V_{-K2}; position of -k: 2 K2 - k
+      const float* V = Vs + (size_t)vb * VROWS * kGVS;
+      for (int idx = lane; idx < 2 * K2 * K3; idx += 32) {
+        const int r = idx / K3, f = idx - r * K3;
+        const int k = r < K2 ? r : r - K2 + 1;
+        const float2 vp = (k < K2) ? *reinterpret_cast<const float2*>(V + k * kGVS + 2 * f) : make_float2(0.f, 0.f);
+        const float2 vm = (k > 0) ? *reinterpret_cast<const float2*>(V + (2 * K2 - k) * kGVS + 2 * f) : make_float2(0.f, 0.f);
+        float2 o;
+        if (r < K2) o = make_float2(vp.x + vm.x, vp.y + vm.y);
+        else o = make_float2(-(vp.y - vm.y), vp.x - vm.x);
+        *reinterpret_cast<float2*>(Bm + r * kGVS + 2 * f) = o;
+      }
+      for (int c = lane; c < 2 * K3; c += 32) Bm[VROWS * kGVS + c] = V[K2 * kGVS + c];
+    }
+    __syncwarp();
+    float lv[NC][2];                                        // V_{-K2} at this lane's columns 8 nc + 2 t4 (+1)
+#pragma unroll
+    for (int nc = 0; nc < NC; ++nc)
+#pragma unroll
+      for (int q = 0; q < 2; ++q) lv[nc][q] = Bm[VROWS * kGVS + 8 * nc + 2 * t4 + q];
     for (int j = 0; j < TP; ++j) {
 #pragma unroll 1
       for (int mt = 0; mt < MT; ++mt) {
         const int tile = j * MT + mt;
-        // the second dimension: U[row][f] = sum_p e^{+i phi} V[p][f]
-        float P[NC][4], Q[NC][4];
+        // the second dimension: U[row][f] = cos(K2 phi_row) V_{-K2}[f] + sum_r basis[row][r] Bm[r][f]
+        float P[NC][4];
+        {
+          const float c0 = cK[16 * tile + g8], c1 = cK[16 * tile + g8 + 8];
 #pragma unroll
-        for (int nc = 0; nc < NC; ++nc)
+          for (int nc = 0; nc < NC; ++nc)
 #pragma unroll
-          for (int e = 0; e < 4; ++e) P[nc][e] = Q[nc][e] = 0.f;
+            for (int e = 0; e < 4; ++e) P[nc][e] = ((e >> 1) ? c1 : c0) * lv[nc][e & 1];
+        }
 #pragma unroll
         for (int ks2 = 0; ks2 < KS2; ++ks2) {
-          uint32_t ch2[4], cl2[4], sh2[4], sl2[4];
-          g_split4(a2e[((size_t)(0 * NM + tile) * KS2 + ks2) * 32 + lane], ch2, cl2);
-          g_split4(a2e[((size_t)(1 * NM + tile) * KS2 + ks2) * 32 + lane], sh2, sl2);
+          uint32_t ah2[4], al2[4];
+          g_split4(a2e[(tile * KS2 + ks2) * 32 + lane], ah2, al2);
 #pragma unroll
           for (int nc = 0; nc < NC; ++nc) {
             uint32_t b0h, b0l, b1h, b1l;
-            g_split(V[(8 * ks2 + t4) * kGVS + 8 * nc + g8], b0h, b0l);
-            g_split(V[(8 * ks2 + t4 + 4) * kGVS + 8 * nc + g8], b1h, b1l);
-            mma3_tf32(P[nc], ch2, cl2, b0h, b1h, b0l, b1l);
-            mma3_tf32(Q[nc], sh2, sl2, b0h, b1h, b0l, b1l);
+            g_split(Bm[(8 * ks2 + t4) * kGVS + 8 * nc + g8], b0h, b0l);
+            g_split(Bm[(8 * ks2 + t4 + 4) * kGVS + 8 * nc + g8], b1h, b1l);
+            mma3_tf32(P[nc], ah2, al2, b0h, b1h, b0l, b1l);
           }
         }
-        // (cos + i sin)(Vr + i Vi): U_re = P_re - Q_im, U_im = P_im + Q_re; rotated, it is the contiguous stage's row operand
+        // a C fragment holds the complex value of frequency 4 nc + t4 for the rows g8 (+8): rotated, it is the
+        // contiguous stage's row operand
         uint32_t rh[KSF][4], rl[KSF][4], ih[KSF][4], il[KSF][4];
 #pragma unroll
         for (int ks = 0; ks < KSF; ++ks)
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int nc = 2 * ks + (e >> 1), h = e & 1;
-            const float ur = P[nc][2 * h] - Q[nc][2 * h + 1], ui = P[nc][2 * h + 1] + Q[nc][2 * h];
+            const float ur = P[nc][2 * h], ui = P[nc][2 * h + 1];
             const float2 r = rot[ks][e >> 1];
             g_split(ur * r.x - ui * r.y, rh[ks][e], rl[ks][e]);
             g_split(ur * r.y + ui * r.x, ih[ks][e], il[ks][e]);
           }
-#pragma unroll 1
-        for (int ntj = 0; ntj < NTJ; ++ntj) {
+        // one tile of 8 pairs: y_j = P - Q, y_{N3-1-j} = P + Q; `last`: pairs past the end go to the dump slot behind the
+        // task's floats, the middle sample of an odd extent is P alone
+        auto tile_j = [&](int ntj, bool last) {
           float Pj[4] = {0.f, 0.f, 0.f, 0.f}, Qj[4] = {0.f, 0.f, 0.f, 0.f};
+          const float4* bt = btab + ntj * 32 + lane;
 #pragma unroll
           for (int ks = 0; ks < KSF; ++ks) {
-            const float4 bc = btab[((size_t)(0 * KSF + ks) * NTJ + ntj) * 32 + lane];
-            const float4 bs = btab[((size_t)(1 * KSF + ks) * NTJ + ntj) * 32 + lane];
+            const float4 bc = bt[ks * NTJ * 32], bs = bt[(KSF + ks) * NTJ * 32];
             mma3_tf32(Pj, rh[ks], rl[ks], __float_as_uint(bc.x), __float_as_uint(bc.y), __float_as_uint(bc.z), __float_as_uint(bc.w));
             mma3_tf32(Qj, ih[ks], il[ks], __float_as_uint(bs.x), __float_as_uint(bs.y), __float_as_uint(bs.z), __float_as_uint(bs.w));
           }
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
-            float* srow = st + (16 * mt + g8 + 8 * h) * N3;
+            const int rowoff = (16 * mt + g8 + 8 * h) * N3;
+            float* srow = st + rowoff;
+            const int dump = TR * N3 - rowoff;
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
               const int jj = 8 * ntj + 2 * t4 + q;
               const float pv = Pj[2 * h + q], qv = Qj[2 * h + q];
-              if (jj < half) {
+              if (!last) {
                 srow[jj] = pv - qv;
                 srow[N3 - 1 - jj] = pv + qv;
-              } else if (odd && jj == half) {
-                srow[jj] = pv;
+              } else {
+                const bool in = jj < half;
+                srow[in ? jj : ((odd && jj == half) ? jj : dump)] = in ? pv - qv : pv;
+                srow[in ? N3 - 1 - jj : dump] = pv + qv;
               }
             }
           }
-        }
+        };
+#pragma unroll 1
+        for (int ntj = 0; ntj < NTJ - 1; ++ntj) tile_j(ntj, false);
+        tile_j(NTJ - 1, true);
       }
       __syncwarp();
       {
@@ -680,7 +747,7 @@ planeg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long 
       }
       __syncwarp();   // the staging area is read out before the next task writes to it
     }
-    __syncwarp();     // this plane's spectrum copy is not needed any more: the plane after next may land in it
+    __syncwarp();     // this plane's operand rows are not needed any more: the next plane's are formed over them
   }
 }
 
@@ -752,18 +819,20 @@ cudaError_t launch_expand_t(const float2* in, float* y, long long rows, int N3, 
 // shared memory of the two plane kernels: tables, then per-warp areas
 size_t pg_contract_table(int N3, int N2, int MTM) {
   const int KS = ((N3 + 1) / 2 + 7) / 8;
-  return ((size_t)2 * KS * 2 + (size_t)2 * (N2 / 8) * MTM) * 32 * 16;
+  return ((size_t)2 * KS * 2 + (size_t)(N2 / 8) * MTM) * 32 * 16 + (size_t)((N2 + 3) & ~3) * 4;
 }
+size_t pg_contract_scratch(int MTM) { return (size_t)(((16 * MTM + 1) * 34 + 3) & ~3) * 4; }
 size_t pg_expand_table(int N3, int N2, int KSF, int KS2) {
   const int NTJ = ((N3 + 1) / 2 + 7) / 8;
-  return ((size_t)2 * KSF * NTJ + (size_t)2 * (N2 / 16) * KS2) * 32 * 16;
+  return ((size_t)2 * KSF * NTJ + (size_t)(N2 / 16) * KS2) * 32 * 16 + (size_t)((N2 + 3) & ~3) * 4;
 }
+size_t pg_expand_rows(int KS2) { return (size_t)(3 * 8 * KS2 + 1) * kGVS * 4; }
 
 template <int MT, int NC, int MTM, int ST>
 cudaError_t launch_pg_contract_s(const float* x, float2* out, long long planes, int N3, int K3, int N2, int K2,
                                  float scale, int herm, cudaStream_t st) {
-  const int sf = g_stage_floats(N3, MT);
-  const GCfg c = g_cfg(pg_contract_table(N3, N2, MTM), (size_t)ST * sf * 4);
+  const int sf = g_stage_floats(N3, MT) + 4;   // + the zero slot
+  const GCfg c = g_cfg(pg_contract_table(N3, N2, MTM), (size_t)ST * sf * 4 + pg_contract_scratch(MTM));
   if (c.warps < 2) return cudaErrorInvalidConfiguration;
   auto kern = planeg_contract_kernel<MT, NC, MTM, ST>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
@@ -777,8 +846,8 @@ cudaError_t launch_pg_contract_s(const float* x, float2* out, long long planes, 
 template <int MT, int NC, int MTM>
 cudaError_t launch_pg_contract_t(const float* x, float2* out, long long planes, int N3, int K3, int N2, int K2,
                                  float scale, int herm, cudaStream_t st) {
-  const size_t sb = (size_t)g_stage_floats(N3, MT) * 4;
-  return g_stages(pg_contract_table(N3, N2, MTM), sb) == 3
+  const size_t sb = (size_t)(g_stage_floats(N3, MT) + 4) * 4;
+  return g_stages(pg_contract_table(N3, N2, MTM) + kGMaxWarps * pg_contract_scratch(MTM), sb) == 3
              ? launch_pg_contract_s<MT, NC, MTM, 3>(x, out, planes, N3, K3, N2, K2, scale, herm, st)
              : launch_pg_contract_s<MT, NC, MTM, 2>(x, out, planes, N3, K3, N2, K2, scale, herm, st);
 }
@@ -786,8 +855,8 @@ cudaError_t launch_pg_contract_t(const float* x, float2* out, long long planes, 
 template <int MT, int KSF, int KS2>
 cudaError_t launch_pg_expand_t(const float2* in, float* y, long long planes, int N3, int K3, int N2, int K2,
                                float scale, int herm, cudaStream_t st) {
-  const int sf = g_stage_floats(N3, MT);
-  const GCfg c = g_cfg(pg_expand_table(N3, N2, KSF, KS2), ((size_t)sf + 2 * 8 * KS2 * kGVS) * 4);
+  const int sf = g_stage_floats(N3, MT) + 4;   // + the dump slot
+  const GCfg c = g_cfg(pg_expand_table(N3, N2, KSF, KS2), (size_t)sf * 4 + pg_expand_rows(KS2));
   if (c.warps < 2) return cudaErrorInvalidConfiguration;
   auto kern = planeg_expand_kernel<MT, KSF, KS2>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
@@ -810,8 +879,8 @@ bool planeg_supported(int N3, int K3, int N2, int K2) {
   const int MTM = (2 * K2 + 15) / 16, KS2 = (2 * K2 + 7) / 8, KSF = (K3 + 7) / 8;
   const size_t sf = (size_t)g_stage_floats(N3, mt) * 4;
   const size_t ct = pg_contract_table(N3, N2, MTM), et = pg_expand_table(N3, N2, KSF, KS2);
-  if (ct + 4 * 2 * sf > kGSmemLimit) return false;
-  return g_cfg(ct, g_stages(ct, sf) * sf).warps >= 4 && g_cfg(et, sf + (size_t)2 * 8 * KS2 * kGVS * 4).warps >= 4;
+  const size_t scr = pg_contract_scratch(MTM), sfz = sf + 16;   // contraction stages carry a zero slot
+  return g_cfg(ct, g_stages(ct + kGMaxWarps * scr, sfz) * sfz + scr).warps >= 4 && g_cfg(et, sfz + pg_expand_rows(KS2)).warps >= 4;
 }
 
 cudaError_t launch_planeg_contract(const float* x, float2* out, long long planes, int N3, int K3, int N2, int K2,
