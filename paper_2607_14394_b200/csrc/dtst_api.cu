@@ -501,6 +501,13 @@ dtst_status run_inverse_fused(dtst_plan* p, const float2* Yhat, float* y, int Cn
                                                scale, herm ? 1 : 0, reinterpret_cast<int*>(ws + L.status),
                                                p->dbg_poll_limit ? p->dbg_poll_limit : kDefaultPollLimit, st)))
       return DTST_ERR_CUDA;
+  } else if (2 * p->kmax[a] == p->Ng[a] && std::getenv("DTST_NO_PLANEG") == nullptr &&
+             planeg_supported((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b])) {
+    // half of the contiguous extent retained: the lane-per-row expansion of the tensor-map plane kernel is bound by its
+    // multiply-adds there (1.9 TB/s on the paper's layer), the tensor-core one of dtst_rowg.cu is not
+    if (cuda_failed(p, launch_planeg_expand(src, y, planes, (int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], scale,
+                                            herm ? 1 : 0, st)))
+      return DTST_ERR_CUDA;
   } else if (cuda_failed(p, launch_inv_plane((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], src, y,
                                              planes * p->Ng[b], scale, herm ? 1 : 0, nullptr, st))) {
     return DTST_ERR_CUDA;
