@@ -60,8 +60,10 @@ enum {
 enum {
   DTST_PATH_AUTO = 0,      /* fused streaming kernels where the shape allows, else generic */
   DTST_PATH_GENERIC = 1,   /* one generic contraction kernel per dimension                 */
-  DTST_PATH_ROW = 2        /* reported only: streaming kernel on the contiguous dimension,
-                              folded kernels on the others (shapes without a two-dimension kernel) */
+  DTST_PATH_ROW = 2        /* reported only: streaming kernel on the contiguous dimension (any extent up to 512,
+                              odd ones included, up to 32 one-sided modes; with the dimension in front of it inside
+                              the same kernel where its extent is a multiple of 16 - 32 for extents up to 64 - and at
+                              most 256), folded kernels on the others (shapes without a two-dimension tensor-map kernel) */
 };
 
 /*
@@ -454,6 +456,8 @@ dtst_status dtst_plan_last_cuda_error(const dtst_plan* plan, int* code, const ch
  *   DTST_NO_PDL=1            launch every kernel without the programmatic-dependent-launch attribute
  *   DTST_NO_COLFUSE=1        forward-type transforms: contract the third dimension in a launch of its own instead of
  *                            inside the kernel that streams the grid (shapes for which that kernel exists)
+ *   DTST_NO_PLANEG=1         contiguous extents that are no multiple of 32: contract / expand the dimension in front in a
+ *                            launch of its own instead of inside the row kernel
  */
 const char* dtst_status_string(dtst_status s);
 
