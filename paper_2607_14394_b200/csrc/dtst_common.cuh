@@ -242,6 +242,10 @@ cudaError_t launch_slab(bool forward, int K, const float2* in, float2* out, long
 // else the FFMA register-accumulator version (dtst_mid.cu)
 bool mid_supported(int N, int K);
 // tensor-core variant of the middle-dimension kernels (N % 32 == 0, inner % 4 == 0)
+// folded tensor-core kernels for any extent and any mode count up to 32 (dtst_midg.cu)
+bool midg_supported(int N, int K);
+cudaError_t launch_midg(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
+                        float scale, cudaStream_t st);
 bool mid_mma_supported(int N, int K, long long inner);
 cudaError_t launch_mid_mma(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
                            float scale, cudaStream_t st);

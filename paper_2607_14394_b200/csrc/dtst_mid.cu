@@ -343,18 +343,24 @@ cudaError_t launch_mid_t(bool forward, const float2* in, float2* out, long long 
 
 }  // namespace
 
-bool mid_supported(int N, int K) {
+// the double-folded FFMA kernels of this file
+static bool mid_ffma_supported(int N, int K) {
   if (N % 2 != 0 || 2 * K > N) return false;
   if (!(K == 4 || K == 8 || K == 12 || K == 16)) return false;
   const size_t smem = (size_t)(N / 2) * (((2 * K + 1 + 3) / 4) * 4) * 4 + (size_t)(K + 1) * 8;
   return smem <= 200 * 1024;
 }
 
+// some folded kernel serves this extent and mode count: the ones of this file, their tensor-core versions
+// (dtst_midmma.cu) or the ones for any extent and any mode count up to 32 (dtst_midg.cu)
+bool mid_supported(int N, int K) { return mid_ffma_supported(N, K) || midg_supported(N, K); }
+
 cudaError_t launch_mid(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
                        float scale, cudaStream_t st) {
   if (outer * inner <= 0) return cudaSuccess;
   const bool aligned16 = ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
   if (aligned16 && mid_mma_supported(N, K, inner)) return launch_mid_mma(forward, K, in, out, outer, inner, N, scale, st);
+  if (!mid_ffma_supported(N, K)) return launch_midg(forward, K, in, out, outer, inner, N, scale, st);
   // two adjacent positions per thread need an even inner extent (then every pair is 16-byte aligned and
   // never straddles two outer slices) and 16-byte aligned tensors
   const bool vec = (inner % 2 == 0) && ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;

@@ -416,6 +416,30 @@ ANY_EXTENT = [
 ]
 
 
+# ------------------------------------------------------------------ middle dimensions with any extent and mode count
+ANY_MIDDLE = [
+    # name, B, Ci, Co, N, kmax: mode counts the double-folded kernels are not built for, odd extents, odd inner extents
+    ("m_k6", 1, 2, 2, (32, 64, 64), (6, 6, 8)),
+    ("m_k10_k20", 1, 2, 1, (64, 64, 64), (10, 20, 16)),
+    ("m_k32", 1, 1, 2, (64, 96, 32), (32, 5, 8)),
+    ("m_odd_extents", 2, 1, 1, (45, 27, 64), (7, 13, 16)),
+    ("m_odd_inner", 1, 2, 2, (40, 36, 50), (9, 3, 9)),          # k3 = 9: 8-byte copies
+    ("m_2d_k24", 1, 3, 2, (100, 64), (24, 12)),
+    ("m_4d", 1, 1, 2, (20, 24, 28, 32), (5, 6, 7, 8)),
+    ("m_k1", 1, 2, 2, (6, 10, 32), (1, 2, 4)),
+]
+
+
+@pytest.mark.parametrize("case", ANY_MIDDLE, ids=[c[0] for c in ANY_MIDDLE])
+def test_any_middle_extent_and_mode_count_runs_on_folded_kernels(case):
+    name, B, Ci, Co, N, k = case
+    w = I.custom_workload(name, B, Ci, Co, N, k, field="grf", seed=37)
+    plan = _plan(w)
+    plan.require_fast_path()            # every stage on a streaming kernel, or this raises
+    plan.close()
+    run_layer_and_check(w, "auto")
+
+
 @pytest.mark.parametrize("case", ANY_EXTENT, ids=[c[0] for c in ANY_EXTENT])
 def test_any_contiguous_extent_runs_on_the_row_kernels(case):
     name, B, Ci, Co, N, k, streaming = case
@@ -559,8 +583,8 @@ def test_pencil_block_runs_on_the_tensor_core_slab_kernels():
 
 def test_fast_path_or_fail():
     from paper_2607_14394_b200 import binding as Bn
-    # an odd extent in the middle: the generic kernel would serve that dimension
-    w = I.custom_workload("slowmid", 1, 2, 2, (9, 64, 64), (3, 8, 8))
+    # 40 modes per side in the middle (the folded kernels stop at 32): the generic kernel would serve that dimension
+    w = I.custom_workload("slowmid", 1, 2, 2, (96, 64, 64), (40, 8, 8))
     plan = _plan(w)
     with pytest.raises(Bn.DtstError) as e:
         plan.require_fast_path()
