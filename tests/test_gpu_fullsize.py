@@ -184,6 +184,14 @@ def test_cfg4_3d_256_fullsize():
     _check_layer_fullsize(w, P_list=[4], rng_seed=44)
 
 
+def test_paper_layer_time_axis_30_fullsize():
+    """The paper's own layer at its width (20 channels, grid 128 x 128 x 64 x 30, modes (8, 8, 8, 16): Section
+    "Experimental Setup" and the operation count of Section "cuBLAS vs cuFFT"), which runs on the kernels for
+    contiguous extents that are no multiple of 32."""
+    w = I.EXTRA_WORKLOADS["paper_4d_t30"]
+    _check_layer_fullsize(w, P_list=[4], rng_seed=30)
+
+
 def test_cfg5_shape_iid_field_every_mode_has_equal_weight():
     """The largest shape once more with a white field: every retained mode then has the same expected
     magnitude, so no mode's error can hide behind a stronger one (the smooth fields of the benchmark put
@@ -209,13 +217,13 @@ def test_cfg5_shape_iid_field_every_mode_has_equal_weight():
         plan.close()
 
 
-@pytest.mark.parametrize("name", ["cfg5_4d_128", "cfg4_3d_256"])
+@pytest.mark.parametrize("name", ["cfg5_4d_128", "cfg4_3d_256", "paper_4d_t30"])
 def test_fullsize_properties_that_hold_at_any_size(name):
     """At the benchmark's full sizes, in its launch configuration, on every channel at once (no oracle needed):
     the adjoint identity <F x, Y> = <x, F^H Y> with F^H = dtst_backward_input, the pair
     <I Y, g> = <Y, G_Y(g)> with G_Y = dtst_backward_spectrum, and linearity of F."""
     from paper_2607_14394_b200 import Plan
-    w = I.WORKLOADS[name]
+    w = I.workload(name)
     dev = torch.device("cuda")
     plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out)
     gen = torch.Generator(device=dev).manual_seed(2024)
