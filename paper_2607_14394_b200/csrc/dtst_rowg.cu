@@ -39,6 +39,17 @@ __device__ __forceinline__ void g_split(float v, uint32_t& hi, uint32_t& lo) {
   lo = __float_as_uint(v - __uint_as_float(hi));
 }
 
+__device__ __forceinline__ void g_bits(const float4& v, uint32_t (&o)[4]) {
+  o[0] = __float_as_uint(v.x);
+  o[1] = __float_as_uint(v.y);
+  o[2] = __float_as_uint(v.z);
+  o[3] = __float_as_uint(v.w);
+}
+// one compensated product with the 8-column operand as a table entry (b0 hi, b1 hi, b0 lo, b1 lo)
+__device__ __forceinline__ void g_mma3q(float (&d)[4], const uint32_t (&ahi)[4], const uint32_t (&alo)[4], const float4& b) {
+  mma3_tf32(d, ahi, alo, __float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
+}
+
 // cos (part 0) or sin (part 1) of 2 pi f (j + 1/2) / N, the phase reduced exactly in integers
 __device__ __forceinline__ float g_basis(int part, int f, int j, int N) {
   double s, c;
@@ -148,10 +159,8 @@ rowg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long
         }
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-          mma3_tf32(accC[mt][nt], sh, sl, __float_as_uint(bc[nt].x), __float_as_uint(bc[nt].y), __float_as_uint(bc[nt].z),
-                    __float_as_uint(bc[nt].w));
-          mma3_tf32(accS[mt][nt], dh, dl, __float_as_uint(bs[nt].x), __float_as_uint(bs[nt].y), __float_as_uint(bs[nt].z),
-                    __float_as_uint(bs[nt].w));
+          g_mma3q(accC[mt][nt], sh, sl, bc[nt]);
+          g_mma3q(accS[mt][nt], dh, dl, bs[nt]);
         }
       }
     }
@@ -278,10 +287,8 @@ rowg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long lo
         float P[4] = {0.f, 0.f, 0.f, 0.f}, Q[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int ks = 0; ks < KSF; ++ks) {
-          mma3_tf32(P, rh[mt][ks], rl[mt][ks], __float_as_uint(bc[ks].x), __float_as_uint(bc[ks].y),
-                    __float_as_uint(bc[ks].z), __float_as_uint(bc[ks].w));
-          mma3_tf32(Q, ih[mt][ks], il[mt][ks], __float_as_uint(bs[ks].x), __float_as_uint(bs[ks].y),
-                    __float_as_uint(bs[ks].z), __float_as_uint(bs[ks].w));
+          g_mma3q(P, rh[mt][ks], rl[mt][ks], bc[ks]);
+          g_mma3q(Q, ih[mt][ks], il[mt][ks], bs[ks]);
         }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -481,10 +488,11 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
           g_split(a0 - b0, bdh[0], bdl[0]);
           g_split(a1 + b1, bsh[1], bsl[1]);
           g_split(a1 - b1, bdh[1], bdl[1]);
-          const uint32_t chv[4] = {__float_as_uint(ch.x), __float_as_uint(ch.y), __float_as_uint(ch.z), __float_as_uint(ch.w)};
-          const uint32_t clv[4] = {__float_as_uint(cl.x), __float_as_uint(cl.y), __float_as_uint(cl.z), __float_as_uint(cl.w)};
-          const uint32_t shv[4] = {__float_as_uint(sh.x), __float_as_uint(sh.y), __float_as_uint(sh.z), __float_as_uint(sh.w)};
-          const uint32_t slv[4] = {__float_as_uint(sl.x), __float_as_uint(sl.y), __float_as_uint(sl.z), __float_as_uint(sl.w)};
+          uint32_t chv[4], clv[4], shv[4], slv[4];
+          g_bits(ch, chv);
+          g_bits(cl, clv);
+          g_bits(sh, shv);
+          g_bits(sl, slv);
           mma3_tf32(accC, chv, clv, bsh[0], bsh[1], bsl[0], bsl[1]);
           mma3_tf32(accS, shv, slv, bdh[0], bdh[1], bdl[0], bdl[1]);
         };
@@ -712,8 +720,8 @@ planeg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long 
 #pragma unroll
           for (int ks = 0; ks < KSF; ++ks) {
             const float4 bc = bt[ks * NTJ * 32], bs = bt[(KSF + ks) * NTJ * 32];
-            mma3_tf32(Pj, rh[ks], rl[ks], __float_as_uint(bc.x), __float_as_uint(bc.y), __float_as_uint(bc.z), __float_as_uint(bc.w));
-            mma3_tf32(Qj, ih[ks], il[ks], __float_as_uint(bs.x), __float_as_uint(bs.y), __float_as_uint(bs.z), __float_as_uint(bs.w));
+            g_mma3q(Pj, rh[ks], rl[ks], bc);
+            g_mma3q(Qj, ih[ks], il[ks], bs);
           }
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
