@@ -623,10 +623,11 @@ def fno_summary(torch, steps=5):
 
 def other_configs_summary(torch, skip_name, steps=10):
     """Forward and forward+backward time of the other benchmark configurations (parity-test cases, not the
-    headline): seeded device-generated inputs of each shape, CUDA events, 3 warm-ups."""
+    headline) and of the paper's own layer on both of its time axes: seeded device-generated inputs of each shape,
+    CUDA events, 3 warm-ups."""
     from paper_2607_14394_b200 import Plan, inputs
     out = {}
-    for name, w in inputs.WORKLOADS.items():
+    for name, w in list(inputs.WORKLOADS.items()) + list(inputs.EXTRA_WORKLOADS.items()):
         if name == skip_name:
             continue
         try:
