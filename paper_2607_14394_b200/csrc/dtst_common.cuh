@@ -246,6 +246,10 @@ bool mid_supported(int N, int K);
 bool midg_supported(int N, int K);
 cudaError_t launch_midg(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
                         float scale, cudaStream_t st);
+// ... for Nl local rows that start at global index `off` of an extent Ng (a rank's block; virtual slabs taken together)
+bool midg_local_supported(int Nl, int K);
+cudaError_t launch_midg_local(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int Nl,
+                              int Ng, int off, float scale, cudaStream_t st);
 bool mid_mma_supported(int N, int K, long long inner);
 cudaError_t launch_mid_mma(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
                            float scale, cudaStream_t st);

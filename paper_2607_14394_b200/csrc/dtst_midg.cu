@@ -54,25 +54,26 @@ __device__ __forceinline__ void mg_split4(const float4& v, uint32_t (&hi)[4], ui
   mg_split(v.w, hi[3], lo[3]);
 }
 
-// entry r of the folded basis at row n: cos(2 pi r n / N) for r < K, sin(2 pi (r - K + 1) n / N) for K <= r < 2K,
-// zero beyond and for rows past the extent
-__device__ __forceinline__ float mg_basis(int r, int n, int N, int K) {
+// entry r of the folded basis at local row n (global index off + n of an extent Ng, Eq. 18): cos(k phi) for r < K
+// (k = r), sin(k phi) for K <= r < 2K (k = r - K + 1), phi = 2 pi (off + n) / Ng; zero beyond and for rows past the
+// local extent N
+__device__ __forceinline__ float mg_basis(int r, int n, int N, int Ng, int off, int K) {
   if (r >= 2 * K || n >= N) return 0.f;
   const long long k = r < K ? r : r - K + 1;
   double s, c;
-  sincospi(2.0 * (double)((k * n) % N) / (double)N, &s, &c);
+  sincospi(2.0 * (double)((k * (off + n)) % Ng) / (double)Ng, &s, &c);
   return r < K ? (float)c : (float)s;
 }
-__device__ __forceinline__ float mg_cosK(int n, int N, int K) {
+__device__ __forceinline__ float mg_cosK(int n, int N, int Ng, int off, int K) {
   if (n >= N) return 0.f;
-  return (float)cospi(2.0 * (double)(((long long)K * n) % N) / (double)N);
+  return (float)cospi(2.0 * (double)(((long long)K * (off + n)) % Ng) / (double)Ng);
 }
 
 // MTM: 16-row tiles of the folded basis (2K <= 16 MTM).  VEC: 16-byte copies (inner even, 16-byte aligned tensors).
 template <int MTM, bool VEC>
 __global__ void __launch_bounds__(kMgMaxWarps * 32, 1)
 midg_contract_kernel(const float2* __restrict__ in, float2* __restrict__ out, long long outer, long long inner, int N,
-                     int K, float scale) {
+                     int Ng, int off, int K, float scale) {
   pdl_trigger();
   extern __shared__ float4 mg_smem[];
   const int NCH = (N + kMgChunk - 1) / kMgChunk, NG = 4 * NCH;
@@ -91,10 +92,10 @@ midg_contract_kernel(const float2* __restrict__ in, float2* __restrict__ out, lo
     float v[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q)                                     // A fragment: basis row l >> 2 (+8), row 2 (l & 3) (+1)
-      v[q] = mg_basis(16 * mtm + (l >> 2) + 8 * (q & 1), 8 * grp + 2 * (l & 3) + (q >> 1), N, K);
+      v[q] = mg_basis(16 * mtm + (l >> 2) + 8 * (q & 1), 8 * grp + 2 * (l & 3) + (q >> 1), N, Ng, off, K);
     a2tab[e] = make_float4(v[0], v[1], v[2], v[3]);
   }
-  for (int n = threadIdx.x; n < NCH * kMgChunk; n += blockDim.x) cK[n] = mg_cosK(n, N, K);
+  for (int n = threadIdx.x; n < NCH * kMgChunk; n += blockDim.x) cK[n] = mg_cosK(n, N, Ng, off, K);
   // rows and columns a copy never reaches (past the extent, past a ragged block) meet zero basis entries or are not
   // stored: they must be finite
   for (int e = lane; e < kMgStages * STAGE; e += 32) S[e] = 0.f;
@@ -225,7 +226,7 @@ midg_contract_kernel(const float2* __restrict__ in, float2* __restrict__ out, lo
 template <bool VEC>
 __global__ void __launch_bounds__(kMgMaxWarps * 32, 1)
 midg_expand_kernel(const float2* __restrict__ in, float2* __restrict__ out, long long outer, long long inner, int N,
-                   int K, float scale) {
+                   int Ng, int off, int K, float scale) {
   pdl_trigger();
   extern __shared__ float4 mg_smem[];
   const int NM = (N + 15) / 16, KS2 = (2 * K + 7) / 8, VROWS = 8 * KS2;
@@ -243,10 +244,10 @@ midg_expand_kernel(const float2* __restrict__ in, float2* __restrict__ out, long
     float v[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q)                                     // A fragment: row l >> 2 (+8), basis entry l & 3 (+4)
-      v[q] = mg_basis(8 * ks2 + (l & 3) + 4 * (q >> 1), 16 * tile + (l >> 2) + 8 * (q & 1), N, K);
+      v[q] = mg_basis(8 * ks2 + (l & 3) + 4 * (q >> 1), 16 * tile + (l >> 2) + 8 * (q & 1), N, Ng, off, K);
     a2e[e] = make_float4(v[0], v[1], v[2], v[3]);
   }
-  for (int n = threadIdx.x; n < NM * 16; n += blockDim.x) cK[n] = mg_cosK(n, N, K);
+  for (int n = threadIdx.x; n < NM * 16; n += blockDim.x) cK[n] = mg_cosK(n, N, Ng, off, K);
   for (int e = lane; e < area; e += 32) Vs[e] = 0.f;                // padding meets zero basis entries: finite
   __syncthreads();
   pdl_wait();
@@ -372,8 +373,8 @@ size_t mg_expand_table(int N, int K) {
 size_t mg_expand_warp(int K) { return (size_t)(3 * 8 * ((2 * K + 7) / 8) + 1) * kMgRowE * 4; }
 
 template <int MTM, bool VEC>
-cudaError_t launch_contract_t(const float2* in, float2* out, long long outer, long long inner, int N, int K, float scale,
-                              cudaStream_t st) {
+cudaError_t launch_contract_t(const float2* in, float2* out, long long outer, long long inner, int N, int Ng, int off,
+                              int K, float scale, cudaStream_t st) {
   const MgCfg c = mg_cfg(mg_contract_table(N, MTM), mg_contract_warp(MTM));
   if (c.warps < 2) return cudaErrorInvalidConfiguration;
   auto kern = midg_contract_kernel<MTM, VEC>;
@@ -382,13 +383,13 @@ cudaError_t launch_contract_t(const float2* in, float2* out, long long outer, lo
   const long long tasks = outer * ((inner + kMgPos - 1) / kMgPos);
   const long long want = (tasks + c.warps - 1) / c.warps;
   const int grid = (int)(want < num_sms() ? want : num_sms());
-  (void)launch_pdl(kern, dim3(grid), dim3(c.warps * 32), c.smem, st, in, out, outer, inner, N, K, scale);
+  (void)launch_pdl(kern, dim3(grid), dim3(c.warps * 32), c.smem, st, in, out, outer, inner, N, Ng, off, K, scale);
   return cudaGetLastError();
 }
 
 template <bool VEC>
-cudaError_t launch_expand_t(const float2* in, float2* out, long long outer, long long inner, int N, int K, float scale,
-                            cudaStream_t st) {
+cudaError_t launch_expand_t(const float2* in, float2* out, long long outer, long long inner, int N, int Ng, int off, int K,
+                            float scale, cudaStream_t st) {
   const MgCfg c = mg_cfg(mg_expand_table(N, K), mg_expand_warp(K));
   if (c.warps < 2) return cudaErrorInvalidConfiguration;
   auto kern = midg_expand_kernel<VEC>;
@@ -397,34 +398,43 @@ cudaError_t launch_expand_t(const float2* in, float2* out, long long outer, long
   const long long tasks = outer * ((inner + kMgPos - 1) / kMgPos);
   const long long want = (tasks + c.warps - 1) / c.warps;
   const int grid = (int)(want < num_sms() ? want : num_sms());
-  (void)launch_pdl(kern, dim3(grid), dim3(c.warps * 32), c.smem, st, in, out, outer, inner, N, K, scale);
+  (void)launch_pdl(kern, dim3(grid), dim3(c.warps * 32), c.smem, st, in, out, outer, inner, N, Ng, off, K, scale);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 // Any extent with 2K <= N and any K up to 32 whose tables leave room for four warps (N up to ~1000).
-bool midg_supported(int N, int K) {
-  if (K < 1 || K > 32 || N < 2 || 2 * K > N) return false;
+bool midg_supported(int N, int K) { return N >= 2 && 2 * K <= N && midg_local_supported(N, K); }
+
+// The same for Nl local rows of a longer dimension (a rank's block, or the slabs of virtual shards taken together):
+// the rows carry their global phases, the local extent may be shorter than 2K.
+bool midg_local_supported(int Nl, int K) {
+  if (K < 1 || K > 32 || Nl < 1) return false;
   const int MTM = (2 * K + 15) / 16;
-  return mg_cfg(mg_contract_table(N, MTM), mg_contract_warp(MTM)).warps >= 4 &&
-         mg_cfg(mg_expand_table(N, K), mg_expand_warp(K)).warps >= 4;
+  return mg_cfg(mg_contract_table(Nl, MTM), mg_contract_warp(MTM)).warps >= 4 &&
+         mg_cfg(mg_expand_table(Nl, K), mg_expand_warp(K)).warps >= 4;
 }
 
-cudaError_t launch_midg(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
-                        float scale, cudaStream_t st) {
+cudaError_t launch_midg_local(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int Nl,
+                              int Ng, int off, float scale, cudaStream_t st) {
   if (outer * inner <= 0) return cudaSuccess;
   const bool vec = (inner % 2 == 0) && ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
-  if (!forward) return vec ? launch_expand_t<true>(in, out, outer, inner, N, K, scale, st)
-                           : launch_expand_t<false>(in, out, outer, inner, N, K, scale, st);
+  if (!forward) return vec ? launch_expand_t<true>(in, out, outer, inner, Nl, Ng, off, K, scale, st)
+                           : launch_expand_t<false>(in, out, outer, inner, Nl, Ng, off, K, scale, st);
   switch ((2 * K + 15) / 16) {
 #define DTST_MG(M) \
-  case M: return vec ? launch_contract_t<M, true>(in, out, outer, inner, N, K, scale, st) \
-                     : launch_contract_t<M, false>(in, out, outer, inner, N, K, scale, st);
+  case M: return vec ? launch_contract_t<M, true>(in, out, outer, inner, Nl, Ng, off, K, scale, st) \
+                     : launch_contract_t<M, false>(in, out, outer, inner, Nl, Ng, off, K, scale, st);
     DTST_MG(1) DTST_MG(2) DTST_MG(3) DTST_MG(4)
 #undef DTST_MG
     default: return cudaErrorNotSupported;
   }
+}
+
+cudaError_t launch_midg(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
+                        float scale, cudaStream_t st) {
+  return launch_midg_local(forward, K, in, out, outer, inner, N, N, 0, scale, st);
 }
 
 }  // namespace dtst

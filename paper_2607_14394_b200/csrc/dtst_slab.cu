@@ -382,14 +382,21 @@ cudaError_t launch_slab_t(bool forward, const float2* in, float2* out, long long
 
 }  // namespace
 
-bool slab_supported(int Nl, int K) {
+// the kernels of this file
+static bool slab_own_supported(int Nl, int K) {
   if (!(K == 4 || K == 8 || K == 12 || K == 16)) return false;
   return (size_t)Nl * 2 * K * sizeof(float2) <= 200 * 1024;
 }
 
+// ... or, for other mode counts, the folded kernels of dtst_midg.cu on the local rows with their global phases
+bool slab_supported(int Nl, int K) { return slab_own_supported(Nl, K) || midg_local_supported(Nl, K); }
+
 cudaError_t launch_slab(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int Nl,
                         int N, int off, int P, cudaStream_t st) {
   if (outer * inner <= 0) return cudaSuccess;
+  // Slabs of one device are consecutive rows with consecutive global indices: taken together they are ONE local
+  // block that starts at `off` (the sum over the slabs is then part of the contraction's own sum).
+  if (!slab_own_supported(Nl, K)) return launch_midg_local(forward, K, in, out, outer, inner, Nl, N, off, 1.0f, st);
   // contraction of slabs that are whole k-steps of 8 rows: tensor-core kernel
   const bool aligned16 = ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
   if (forward && aligned16 && inner % 4 == 0 && P >= 1 && Nl % P == 0 && (Nl / P) % 8 == 0) {

@@ -438,6 +438,12 @@ def test_any_middle_extent_and_mode_count_runs_on_folded_kernels(case):
     plan.require_fast_path()            # every stage on a streaming kernel, or this raises
     plan.close()
     run_layer_and_check(w, "auto")
+    if N[0] % 4 == 0:
+        # virtual shards along dimension 0: its rows carry their global phases in the same folded kernels
+        plan = _plan(w, P=4)
+        plan.require_fast_path()
+        plan.close()
+        run_layer_and_check(w, "auto", P=4)
 
 
 @pytest.mark.parametrize("case", ANY_EXTENT, ids=[c[0] for c in ANY_EXTENT])
