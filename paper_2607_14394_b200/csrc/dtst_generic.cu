@@ -162,8 +162,46 @@ __global__ void __launch_bounds__(256) mix_kernel(const float2* __restrict__ X, 
   for (int b = 0; b < NB; ++b) Y[((long long)(b0 + b) * Co + o) * M + m] = acc[b];
 }
 
+// The same sums for SMALL spectra (a 2-D layer with 12 modes has 288 of them): one thread per (m, o) and four batch
+// entries per launch leaves most of the GPU idle and every thread waiting for one load after the other (16 x 32
+// channels x 288 modes: four launches of 52 us for 3.6 MB).  Here one thread per (m, o, b), the channel loop
+// unrolled so that 16 loads are in flight per thread; W (a few MB) is re-read from L2 by every batch entry.  The
+// terms are added in the same order: the same bits as mix_kernel.
+__global__ void __launch_bounds__(128) mix_small_kernel(const float2* __restrict__ X, const float2* __restrict__ W,
+                                                       float2* __restrict__ Y, int Ci, int Co, long long M) {
+  pdl_trigger();
+  pdl_wait();
+  const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int o = blockIdx.y, b = blockIdx.z;
+  if (m >= M) return;
+  const float2* wp = W + (long long)o * M + m;
+  const float2* xp = X + (long long)b * Ci * M + m;
+  float2 acc = make_float2(0.f, 0.f);
+#pragma unroll 8
+  for (int i = 0; i < Ci; ++i) {
+    const float2 w = __ldg(wp + (long long)i * Co * M);
+    const float2 x = __ldg(xp + (long long)i * M);
+    acc.x = fmaf(x.x, w.x, acc.x);
+    acc.x = fmaf(-x.y, w.y, acc.x);
+    acc.y = fmaf(x.x, w.y, acc.y);
+    acc.y = fmaf(x.y, w.x, acc.y);
+  }
+  Y[((long long)b * Co + o) * M + m] = acc;
+}
+
+// small: few enough (m, o) pairs that mix_kernel cannot fill the GPU, and weights that stay in L2
+static bool mix_is_small(int B, int Ci, int Co, long long M) {
+  return M * Co < (long long)num_sms() * 2048 && (long long)Ci * Co * M * 8 <= (48ll << 20) && B <= 65535 && Co <= 65535;
+}
+
 cudaError_t launch_mix(const float2* X, const float2* W, float2* Y, int B, int Ci, int Co, long long M,
                        cudaStream_t st, long long* launches) {
+  if (mix_is_small(B, Ci, Co, M)) {
+    (void)launch_pdl(mix_small_kernel, dim3((unsigned)((M + 127) / 128), (unsigned)Co, (unsigned)B), dim3(128), 0, st, X, W, Y,
+                     Ci, Co, M);
+    if (launches) ++*launches;
+    return cudaGetLastError();
+  }
   dim3 grid((unsigned)((M + 255) / 256), (unsigned)Co);
   cudaError_t e = cudaSuccess;
   for (int b0 = 0; b0 < B; b0 += 4) {
@@ -246,6 +284,52 @@ __global__ void __launch_bounds__(256) mix_adjoint_kernel(const float2* __restri
   }
 }
 
+// The adjoint for small spectra, as mix_small_kernel: GX with one thread per (m, i, b) walking o, GW with one thread per
+// (m, o, i) walking b; the same order of terms, the same bits as mix_adjoint_kernel.
+__global__ void __launch_bounds__(128) mix_adjoint_gx_small_kernel(const float2* __restrict__ GY, const float2* __restrict__ W,
+                                                                  float2* __restrict__ GX, int Ci, int Co, long long M) {
+  pdl_trigger();
+  pdl_wait();
+  const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int i = blockIdx.y, b = blockIdx.z;
+  if (m >= M) return;
+  const float2* wp = W + (long long)i * Co * M + m;
+  const float2* gp = GY + (long long)b * Co * M + m;
+  float2 gx = make_float2(0.f, 0.f);
+#pragma unroll 8
+  for (int o = 0; o < Co; ++o) {   // g * conj(w)
+    const float2 w = __ldg(wp + (long long)o * M);
+    const float2 g = __ldg(gp + (long long)o * M);
+    gx.x = fmaf(g.x, w.x, gx.x);
+    gx.x = fmaf(g.y, w.y, gx.x);
+    gx.y = fmaf(g.y, w.x, gx.y);
+    gx.y = fmaf(-g.x, w.y, gx.y);
+  }
+  GX[((long long)b * Ci + i) * M + m] = gx;
+}
+
+__global__ void __launch_bounds__(128) mix_adjoint_gw_small_kernel(const float2* __restrict__ GY, const float2* __restrict__ X,
+                                                                  float2* __restrict__ GW, int B, int Ci, int Co, long long M) {
+  pdl_trigger();
+  pdl_wait();
+  const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int o = blockIdx.y, i = blockIdx.z;
+  if (m >= M) return;
+  const float2* gp = GY + (long long)o * M + m;
+  const float2* xp = X + (long long)i * M + m;
+  float2 acc = make_float2(0.f, 0.f);
+#pragma unroll 4
+  for (int b = 0; b < B; ++b) {    // conj(x) * g
+    const float2 g = __ldg(gp + (long long)b * Co * M);
+    const float2 x = __ldg(xp + (long long)b * Ci * M);
+    acc.x = fmaf(x.x, g.x, acc.x);
+    acc.x = fmaf(x.y, g.y, acc.x);
+    acc.y = fmaf(x.x, g.y, acc.y);
+    acc.y = fmaf(-x.y, g.x, acc.y);
+  }
+  GW[((long long)i * Co + o) * M + m] = acc;
+}
+
 template <int NB>
 void launch_mix_adjoint_nb(dim3 grid, cudaStream_t st, const float2* GY, const float2* X, const float2* W,
                            float2* GX, float2* GW, int b0, int B, int Ci, int Co, long long M, bool want_gw) {
@@ -261,6 +345,19 @@ void launch_mix_adjoint_nb(dim3 grid, cudaStream_t st, const float2* GY, const f
 
 cudaError_t launch_mix_adjoint(const float2* GY, const float2* X, const float2* W, float2* GX, float2* GW,
                                int B, int Ci, int Co, long long M, cudaStream_t st, long long* launches) {
+  if (mix_is_small(B, Ci, Co, M) && Ci <= 65535) {
+    const unsigned mb = (unsigned)((M + 127) / 128);
+    if (GX != nullptr) {
+      (void)launch_pdl(mix_adjoint_gx_small_kernel, dim3(mb, (unsigned)Ci, (unsigned)B), dim3(128), 0, st, GY, W, GX, Ci, Co, M);
+      if (launches) ++*launches;
+    }
+    if (GW != nullptr) {
+      (void)launch_pdl(mix_adjoint_gw_small_kernel, dim3(mb, (unsigned)Co, (unsigned)Ci), dim3(128), 0, st, GY, X, GW, B, Ci, Co,
+                       M);
+      if (launches) ++*launches;
+    }
+    return cudaGetLastError();
+  }
   dim3 grid((unsigned)((M + 255) / 256), (unsigned)Ci);
   for (int b0 = 0; b0 < B; b0 += 4) {
     const int nb = (B - b0 < 4) ? (B - b0) : 4;
