@@ -345,7 +345,9 @@ void launch_mix_adjoint_nb(dim3 grid, cudaStream_t st, const float2* GY, const f
 
 cudaError_t launch_mix_adjoint(const float2* GY, const float2* X, const float2* W, float2* GX, float2* GW,
                                int B, int Ci, int Co, long long M, cudaStream_t st, long long* launches) {
-  if (mix_is_small(B, Ci, Co, M) && Ci <= 65535) {
+  // (up to four batch entries mix_adjoint_kernel needs ONE launch that keeps x in registers and reads GY once per
+  // input channel: measured faster than the pair below, 16.7 against 22.9 us on 2 x 16 channels x 6912 modes)
+  if (mix_is_small(B, Ci, Co, M) && Ci <= 65535 && B > 4) {
     const unsigned mb = (unsigned)((M + 127) / 128);
     if (GX != nullptr) {
       (void)launch_pdl(mix_adjoint_gx_small_kernel, dim3(mb, (unsigned)Ci, (unsigned)B), dim3(128), 0, st, GY, W, GX, Ci, Co, M);
