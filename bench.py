@@ -627,12 +627,15 @@ def other_configs_summary(torch, skip_name, steps=10):
     CUDA events, 3 warm-ups."""
     from paper_2607_14394_b200 import Plan, inputs
     out = {}
-    for name, w in list(inputs.WORKLOADS.items()) + list(inputs.EXTRA_WORKLOADS.items()):
+    cases = [(name, w, "tf32x3") for name, w in list(inputs.WORKLOADS.items()) + list(inputs.EXTRA_WORKLOADS.items())]
+    # the paper's layer once more with single-pass TF32 products (a plan option with a stated error of 2e-3)
+    cases.append(("paper_4d_t30_tf32", inputs.EXTRA_WORKLOADS["paper_4d_t30"], "tf32"))
+    for name, w, arithmetic in cases:
         if name == skip_name:
             continue
         try:
             dev = torch.device("cuda", torch.cuda.current_device())
-            plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out)
+            plan = Plan(w.N, w.kmax, w.B, w.C_in, w.C_out, arithmetic=arithmetic)
             gen = torch.Generator(device=dev)
             gen.manual_seed(w.seed)
             x = torch.randn((w.B, w.C_in) + w.N, device=dev, generator=gen)
@@ -670,7 +673,7 @@ def other_configs_summary(torch, skip_name, steps=10):
             tg = graph_step_ms(torch, whole_step, steps)
             ab = algorithmic_bytes(w)
             pts = w.B * w.points
-            out[name] = {"kernel_path": plan.kernel_path, "fwd_ms": tf, "fwd_bwd_ms": tf + tb,
+            out[name] = {"kernel_path": plan.kernel_path, "arithmetic": arithmetic, "fwd_ms": tf, "fwd_bwd_ms": tf + tb,
                          "fwd_gpoints_per_s": pts / tf / 1e6, "fwd_bwd_gpoints_per_s": pts / (tf + tb) / 1e6,
                          "fwd_algorithmic_gbs": ab["fwd"] / tf / 1e6,
                          "fwd_bwd_algorithmic_gbs": ab["fwd_bwd"] / (tf + tb) / 1e6,

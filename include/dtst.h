@@ -187,6 +187,21 @@ dtst_status dtst_plan_set_column_expansion(dtst_plan* plan, int ring_columns);
  */
 dtst_status dtst_plan_set_column_contraction(dtst_plan* plan, int mode);
 
+/*
+ * Arithmetic of the tensor-core stages of the kernels for contiguous extents that are no multiple of 32 and for
+ * middle dimensions of any extent and mode count (the paper's own layer, time axis 30, runs on them; they are bound by
+ * their arithmetic, not by HBM):
+ *   DTST_ARITH_TF32X3  (default) every product as three TF32 products of hi/lo operand parts with fp32
+ *                      accumulation: rel-L2 of each output tensor against the float64 statement <= 1e-5
+ *                      (measured 1e-6..2e-6);
+ *   DTST_ARITH_TF32    one TF32 product per term (operands rounded to 11 significant bits, fp32 accumulation):
+ *                      rel-L2 <= 2e-3 (measured 2e-4..6e-4), a third of the tensor-core work.
+ * The other kernels (tensor-map plane and row kernels, double-folded middle kernels, mixing) are bound by HBM with
+ * the compensated arithmetic in place and are not affected.
+ */
+enum { DTST_ARITH_TF32X3 = 0, DTST_ARITH_TF32 = 1 };
+dtst_status dtst_plan_set_arithmetic(dtst_plan* plan, int mode);
+
 dtst_status dtst_plan_destroy(dtst_plan* plan);
 
 /* M = number of retained modes; K[d] (host, may be NULL) = entries kept per dim. */

@@ -43,7 +43,7 @@ EXPORTED = [
     "dtst_pointwise_linear_backward", "dtst_plan_create_complex", "dtst_forward_complex", "dtst_inverse_complex",
     "dtst_backward_complex", "dtst_plan_set_contraction_order", "dtst_plan_get_contraction_order",
     "dtst_plan_tune_contraction_order", "dtst_plan_host_io_bytes", "dtst_plan_enable_host_io", "dtst_step_host",
-    "dtst_host_io_wait", "dtst_plan_set_column_contraction",
+    "dtst_host_io_wait", "dtst_plan_set_column_contraction", "dtst_plan_set_arithmetic",
 ]
 
 
@@ -105,6 +105,7 @@ def lib() -> ctypes.CDLL:
     L.dtst_host_io_wait.argtypes = [vp]
     L.dtst_plan_set_column_expansion.argtypes = [vp, i32]
     L.dtst_plan_set_column_contraction.argtypes = [vp, i32]
+    L.dtst_plan_set_arithmetic.argtypes = [vp, i32]
     L.dtst_plan_require_fast_path.argtypes = [vp, i32]
     L.dtst_plan_set_block_epilogue.argtypes = [vp, i32]
     L.dtst_plan_debug_ring_fault.argtypes = [vp, ctypes.c_int64, ctypes.c_uint32]
@@ -243,6 +244,15 @@ BLOCK_EPILOGUE = {"auto": 0, "ffma": 1, "tensor": 2}
 def dtst_plan_set_block_epilogue(plan, mode) -> None:
     m = BLOCK_EPILOGUE[mode] if isinstance(mode, str) else int(mode)
     _check(lib().dtst_plan_set_block_epilogue(plan, m), "dtst_plan_set_block_epilogue")
+
+
+DTST_ARITH_TF32X3, DTST_ARITH_TF32 = 0, 1
+
+
+def dtst_plan_set_arithmetic(plan, mode) -> None:
+    if isinstance(mode, str):
+        mode = {"tf32x3": DTST_ARITH_TF32X3, "tf32": DTST_ARITH_TF32}[mode]
+    _check(lib().dtst_plan_set_arithmetic(plan, int(mode)), "dtst_plan_set_arithmetic")
 
 
 def dtst_plan_set_column_contraction(plan, mode) -> None:
@@ -449,7 +459,7 @@ class Plan:
 
     def __init__(self, N, kmax, B, C_in, C_out, N_global=None, offset=None, virtual_shards: int = 1,
                  path: str = "auto", device=None, allocate_workspace: bool = True, column_expansion: int = 0, column_contraction: int = 0,
-                 complex_fields: bool = False):
+                 complex_fields: bool = False, arithmetic: str = "tf32x3"):
         self.N = tuple(int(n) for n in N)
         self.kmax = tuple(int(k) for k in kmax)
         self.d = len(self.N)
@@ -480,6 +490,8 @@ class Plan:
             dtst_plan_set_column_expansion(self._h, column_expansion)
         if column_contraction:
             dtst_plan_set_column_contraction(self._h, column_contraction)
+        if arithmetic != "tf32x3":
+            dtst_plan_set_arithmetic(self._h, arithmetic)
         self.M, self.K = dtst_plan_num_modes(self._h, self.d)
         self.workspace = None
         if allocate_workspace:
@@ -712,6 +724,10 @@ class Plan:
     def set_column_contraction(self, mode: int) -> None:
         """0: automatic, 1: whenever the kernel exists for the shape, -1: never (forward-type transforms)."""
         dtst_plan_set_column_contraction(self._h, mode)
+
+    def set_arithmetic(self, mode) -> None:
+        """'tf32x3' (default: compensated, 1e-5) or 'tf32' (single pass, 2e-3) in the kernels for any extent."""
+        dtst_plan_set_arithmetic(self._h, mode)
 
     def require_fast_path(self, required: bool = True) -> None:
         """Raises DtstError(DTST_ERR_UNSUPPORTED) if any stage of this plan would run on the slow generic kernel."""

@@ -260,7 +260,7 @@ dtst_status forward_stages(dtst_plan* p, const void* cur, int j_from, int flip, 
       // slabs (or a rank's block) of this dimension: partial spectra formed and summed inside one kernel
       void* sdst = last ? static_cast<void*>(Xhat) : static_cast<void*>(buf[flip]);
       if (cuda_failed(p, launch_slab(true, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(sdst),
-                                     op.outer, op.inner, (int)p->Nl[j], op.N, (int)p->off[j], j == 0 ? p->P : 1, st)))
+                                     op.outer, op.inner, (int)p->Nl[j], op.N, (int)p->off[j], j == 0 ? p->P : 1, p->fast_math != 0, st)))
         return DTST_ERR_CUDA;
       ++p->launches;
       cur = sdst;
@@ -285,7 +285,7 @@ dtst_status forward_stages(dtst_plan* p, const void* cur, int j_from, int flip, 
     }
     if (!in_real && use_mid(p, j)) {
       if (cuda_failed(p, launch_mid(true, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst),
-                                    op.outer, op.inner, op.N, 1.0f, st)))
+                                    op.outer, op.inner, op.N, 1.0f, p->fast_math != 0, st)))
         return DTST_ERR_CUDA;
     } else {
       KernelTimer kt(p, DTST_KERNEL_GRID_READ, st, in_real);
@@ -391,10 +391,10 @@ dtst_status expand_stage(dtst_plan* p, int j, int Cn, const void* cur, void* dst
   cudaError_t e;
   if (!out_real && use_mid_expand(p, j)) {
     e = launch_mid(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst), outer, inner,
-                   (int)p->Ng[j], 1.0f, st);
+                   (int)p->Ng[j], 1.0f, p->fast_math != 0, st);
   } else if (!out_real && use_slab(p, j)) {
     e = launch_slab(false, p->kmax[j], static_cast<const float2*>(cur), static_cast<float2*>(dst), outer, inner,
-                    (int)p->Nl[j], (int)p->Ng[j], (int)p->off[j], j == 0 ? p->P : 1, st);
+                    (int)p->Nl[j], (int)p->Ng[j], (int)p->off[j], j == 0 ? p->P : 1, p->fast_math != 0, st);
   } else {
     KernelTimer kt(p, DTST_KERNEL_GRID_WRITE, st, out_real);
     e = launch_apply_dim(op, false, out_real, cur, dst, st);
@@ -506,7 +506,7 @@ dtst_status run_inverse_fused(dtst_plan* p, const float2* Yhat, float* y, int Cn
     // half of the contiguous extent retained: the lane-per-row expansion of the tensor-map plane kernel is bound by its
     // multiply-adds there (1.9 TB/s on the paper's layer), the tensor-core one of dtst_rowg.cu is not
     if (cuda_failed(p, launch_planeg_expand(src, y, planes, (int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], scale,
-                                            herm ? 1 : 0, st)))
+                                            herm ? 1 : 0, p->fast_math != 0, st)))
       return DTST_ERR_CUDA;
   } else if (cuda_failed(p, launch_inv_plane((int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b], src, y,
                                              planes * p->Ng[b], scale, herm ? 1 : 0, nullptr, st))) {
@@ -531,7 +531,7 @@ dtst_status run_forward_row(dtst_plan* p, const float* x, float2* Xhat, int Cn, 
     {
       KernelTimer kt(p, DTST_KERNEL_GRID_READ, st);
       if (cuda_failed(p, launch_planeg_contract(x, dst, rows / p->Ng[b], (int)p->Ng[a], p->kmax[a], (int)p->Ng[b],
-                                                p->kmax[b], scale, herm ? 1 : 0, st)))
+                                                p->kmax[b], scale, herm ? 1 : 0, p->fast_math != 0, st)))
         return DTST_ERR_CUDA;
     }
     ++p->launches;
@@ -543,7 +543,7 @@ dtst_status run_forward_row(dtst_plan* p, const float* x, float2* Xhat, int Cn, 
     const cudaError_t e = row_supported((int)p->Ng[a], p->kmax[a])
                               ? launch_row_contract(x, t1, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0,
                                                     reinterpret_cast<int*>(ws + L.status), st)
-                              : launch_rowg_contract(x, t1, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, st);
+                              : launch_rowg_contract(x, t1, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, p->fast_math != 0, st);
     if (cuda_failed(p, e)) return DTST_ERR_CUDA;
   }
   ++p->launches;
@@ -566,14 +566,14 @@ dtst_status run_inverse_row(dtst_plan* p, const float2* Yhat, float* y, int Cn, 
   if (pg) {
     const int b = d - 2;
     if (cuda_failed(p, launch_planeg_expand(src, y, rows / p->Ng[b], (int)p->Ng[a], p->kmax[a], (int)p->Ng[b], p->kmax[b],
-                                            scale, herm ? 1 : 0, st)))
+                                            scale, herm ? 1 : 0, p->fast_math != 0, st)))
       return DTST_ERR_CUDA;
     ++p->launches;
     return DTST_OK;
   }
   const cudaError_t e = row_supported((int)p->Ng[a], p->kmax[a])
                             ? launch_row_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, st)
-                            : launch_rowg_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, st);
+                            : launch_rowg_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, p->fast_math != 0, st);
   if (cuda_failed(p, e)) return DTST_ERR_CUDA;
   ++p->launches;
   return DTST_OK;
@@ -769,6 +769,12 @@ dtst_status dtst_plan_tune_contraction_order(dtst_plan* p, double* bytes_before,
 dtst_status dtst_plan_set_column_contraction(dtst_plan* p, int mode) {
   if (p == nullptr || mode < -1 || mode > 1) return DTST_ERR_INVALID_ARG;
   p->colfuse = mode;
+  return DTST_OK;
+}
+
+dtst_status dtst_plan_set_arithmetic(dtst_plan* p, int mode) {
+  if (p == nullptr || (mode != DTST_ARITH_TF32X3 && mode != DTST_ARITH_TF32)) return DTST_ERR_INVALID_ARG;
+  p->fast_math = mode == DTST_ARITH_TF32 ? 1 : 0;
   return DTST_OK;
 }
 

@@ -148,6 +148,7 @@ struct dtst_plan {
   long long dbg_withhold_after;    // < 0 = off (the default)
   dtst_host_io* host_io;           // non-null after dtst_plan_enable_host_io
   int colfuse;                     // third dimension inside the forward plane kernel: 0 auto, 1 whenever built, -1 never
+  int fast_math;                   // single-pass TF32 in the kernels for any extent (dtst_plan_set_arithmetic)
   int order_rank[dtst::kMaxDims];  // contraction order of the dimensions behind the grid-side kernel: lower = earlier
   int complex_io;                  // 1: complex fields, two-sided retained set on the last dimension too
   int block_epilogue;              // DTST_BLOCK_EPILOGUE_*
@@ -235,8 +236,9 @@ cudaError_t launch_bypass_backward(const float* gz, const float* x, float* gx, c
 
 // offset / virtual-shard kernels for a two-sided middle dimension (dtst_slab.cu)
 bool slab_supported(int Nl, int K);
+// (fast: single-pass TF32 where the stage runs on the kernels of dtst_midg.cu; the others are not affected)
 cudaError_t launch_slab(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int Nl,
-                        int N, int off, int P, cudaStream_t st);
+                        int N, int off, int P, bool fast, cudaStream_t st);
 
 // folded kernels for a two-sided middle dimension: tensor-core version (dtst_midmma.cu) where the shape allows,
 // else the FFMA register-accumulator version (dtst_mid.cu)
@@ -245,15 +247,15 @@ bool mid_supported(int N, int K);
 // folded tensor-core kernels for any extent and any mode count up to 32 (dtst_midg.cu)
 bool midg_supported(int N, int K);
 cudaError_t launch_midg(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
-                        float scale, cudaStream_t st);
+                        float scale, bool fast, cudaStream_t st);
 // ... for Nl local rows that start at global index `off` of an extent Ng (a rank's block; virtual slabs taken together)
 bool midg_local_supported(int Nl, int K);
 cudaError_t launch_midg_local(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int Nl,
-                              int Ng, int off, float scale, cudaStream_t st);
+                              int Ng, int off, float scale, bool fast, cudaStream_t st);
 bool mid_mma_supported(int N, int K, long long inner);
 cudaError_t launch_mid_mma(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
                            float scale, cudaStream_t st);
 cudaError_t launch_mid(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
-                       float scale, cudaStream_t st);
+                       float scale, bool fast, cudaStream_t st);
 
 }  // namespace dtst

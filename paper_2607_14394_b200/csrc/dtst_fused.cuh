@@ -52,18 +52,18 @@ cudaError_t launch_row_expand(const float2* in, float* y, long long rows, int N3
                               cudaStream_t st);
 
 // Row kernels for any contiguous extent (dtst_rowg.cu): N3 <= 512 (odd extents included), k3 <= 32; cp.async-fed,
-// no tensor map.  Used where row_supported() says no.
+// no tensor map.  Used where row_supported() says no.  fast: single-pass TF32 instead of the hi/lo compensated products.
 bool rowg_supported(int N3, int K3);
-cudaError_t launch_rowg_contract(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm,
+cudaError_t launch_rowg_contract(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm, bool fast,
                                  cudaStream_t st);
-cudaError_t launch_rowg_expand(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm,
+cudaError_t launch_rowg_expand(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm, bool fast,
                                cudaStream_t st);
 // The same with the dimension in front (extent N2, whole, no offset, K2 modes per side) inside the kernel:
 // x[planes][N2][N3] <-> [planes][2 K2][k3].
 bool planeg_supported(int N3, int K3, int N2, int K2);
 cudaError_t launch_planeg_contract(const float* x, float2* out, long long planes, int N3, int K3, int N2, int K2,
-                                   float scale, int herm, cudaStream_t st);
+                                   float scale, int herm, bool fast, cudaStream_t st);
 cudaError_t launch_planeg_expand(const float2* in, float* y, long long planes, int N3, int K3, int N2, int K2,
-                                 float scale, int herm, cudaStream_t st);
+                                 float scale, int herm, bool fast, cudaStream_t st);
 
 }  // namespace dtst

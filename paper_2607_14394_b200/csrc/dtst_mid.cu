@@ -356,11 +356,11 @@ static bool mid_ffma_supported(int N, int K) {
 bool mid_supported(int N, int K) { return mid_ffma_supported(N, K) || midg_supported(N, K); }
 
 cudaError_t launch_mid(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
-                       float scale, cudaStream_t st) {
+                       float scale, bool fast, cudaStream_t st) {
   if (outer * inner <= 0) return cudaSuccess;
   const bool aligned16 = ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
   if (aligned16 && mid_mma_supported(N, K, inner)) return launch_mid_mma(forward, K, in, out, outer, inner, N, scale, st);
-  if (!mid_ffma_supported(N, K)) return launch_midg(forward, K, in, out, outer, inner, N, scale, st);
+  if (!mid_ffma_supported(N, K)) return launch_midg(forward, K, in, out, outer, inner, N, scale, fast, st);
   // two adjacent positions per thread need an even inner extent (then every pair is 16-byte aligned and
   // never straddles two outer slices) and 16-byte aligned tensors
   const bool vec = (inner % 2 == 0) && ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;

@@ -43,15 +43,24 @@ __device__ __forceinline__ void mg_wait() { asm volatile("cp.async.wait_group %0
 
 // hi = v rounded to the 11 significant bits the tensor core reads, lo = the exact rest (at most 2^-12 |v|, of which the
 // hardware drops 2^-23 |v|): half the error of a truncating split, which the short sums of small extents need
+// FAST (single-pass TF32, a plan option): the rounded value alone; every use of the lo part disappears.
+template <bool FAST>
 __device__ __forceinline__ void mg_split(float v, uint32_t& hi, uint32_t& lo) {
   hi = (__float_as_uint(v) + 0x1000u) & 0xffffe000u;
-  lo = __float_as_uint(v - __uint_as_float(hi));
+  lo = FAST ? 0u : __float_as_uint(v - __uint_as_float(hi));
 }
+template <bool FAST>
 __device__ __forceinline__ void mg_split4(const float4& v, uint32_t (&hi)[4], uint32_t (&lo)[4]) {
-  mg_split(v.x, hi[0], lo[0]);
-  mg_split(v.y, hi[1], lo[1]);
-  mg_split(v.z, hi[2], lo[2]);
-  mg_split(v.w, hi[3], lo[3]);
+  mg_split<FAST>(v.x, hi[0], lo[0]);
+  mg_split<FAST>(v.y, hi[1], lo[1]);
+  mg_split<FAST>(v.z, hi[2], lo[2]);
+  mg_split<FAST>(v.w, hi[3], lo[3]);
+}
+template <bool FAST>
+__device__ __forceinline__ void mg_mma3(float (&d)[4], const uint32_t (&ahi)[4], const uint32_t (&alo)[4], uint32_t bh0,
+                                        uint32_t bh1, uint32_t bl0, uint32_t bl1) {
+  if (FAST) mma_m16n8k8_tf32(d, ahi, bh0, bh1);
+  else mma3_tf32(d, ahi, alo, bh0, bh1, bl0, bl1);
 }
 
 // entry r of the folded basis at local row n (global index off + n of an extent Ng, Eq. 18): cos(k phi) for r < K
@@ -70,7 +79,7 @@ __device__ __forceinline__ float mg_cosK(int n, int N, int Ng, int off, int K) {
 }
 
 // MTM: 16-row tiles of the folded basis (2K <= 16 MTM).  VEC: 16-byte copies (inner even, 16-byte aligned tensors).
-template <int MTM, bool VEC>
+template <int MTM, bool VEC, bool FAST>
 __global__ void __launch_bounds__(kMgMaxWarps * 32, 1)
 midg_contract_kernel(const float2* __restrict__ in, float2* __restrict__ out, long long outer, long long inner, int N,
                      int Ng, int off, int K, float scale) {
@@ -168,16 +177,16 @@ midg_contract_kernel(const float2* __restrict__ in, float2* __restrict__ out, lo
 #pragma unroll
         for (int nc = 0; nc < 4; ++nc) {
           const float v0 = r0[8 * nc], v1 = r0[kMgRow + 8 * nc];
-          mg_split(v0, bh[nc][0], bl[nc][0]);
-          mg_split(v1, bh[nc][1], bl[nc][1]);
+          mg_split<FAST>(v0, bh[nc][0], bl[nc][0]);
+          mg_split<FAST>(v1, bh[nc][1], bl[nc][1]);
           lw[nc] = fmaf(ck0, v0, fmaf(ck1, v1, lw[nc]));
         }
 #pragma unroll
         for (int mtm = 0; mtm < MTM; ++mtm) {
           uint32_t ah[4], al[4];
-          mg_split4(a2tab[(grp * MTM + mtm) * 32 + lane], ah, al);
+          mg_split4<FAST>(a2tab[(grp * MTM + mtm) * 32 + lane], ah, al);
 #pragma unroll
-          for (int nc = 0; nc < 4; ++nc) mma3_tf32(P[mtm][nc], ah, al, bh[nc][0], bh[nc][1], bl[nc][0], bl[nc][1]);
+          for (int nc = 0; nc < 4; ++nc) mg_mma3<FAST>(P[mtm][nc], ah, al, bh[nc][0], bh[nc][1], bl[nc][0], bl[nc][1]);
         }
       }
       __syncwarp();   // every lane is done with this stage before it is filled again
@@ -223,7 +232,7 @@ midg_contract_kernel(const float2* __restrict__ in, float2* __restrict__ out, lo
 }
 
 // U_n = cos(K phi_n) V_{-K} + sum_r basis[n][r] Bm[r]: Bm = E_k (k < K), then i O_k (k = 1..K).
-template <bool VEC>
+template <bool VEC, bool FAST>
 __global__ void __launch_bounds__(kMgMaxWarps * 32, 1)
 midg_expand_kernel(const float2* __restrict__ in, float2* __restrict__ out, long long outer, long long inner, int N,
                    int Ng, int off, int K, float scale) {
@@ -320,14 +329,14 @@ midg_expand_kernel(const float2* __restrict__ in, float2* __restrict__ out, long
 #pragma unroll 1
       for (int ks2 = 0; ks2 < KS2; ++ks2) {
         uint32_t ah[4], al[4];
-        mg_split4(a2e[(tile * KS2 + ks2) * 32 + lane], ah, al);
+        mg_split4<FAST>(a2e[(tile * KS2 + ks2) * 32 + lane], ah, al);
         const float* b0 = Bm + (8 * ks2 + t4) * kMgRowE + g8;
 #pragma unroll
         for (int nc = 0; nc < 4; ++nc) {
           uint32_t b0h, b0l, b1h, b1l;
-          mg_split(b0[8 * nc], b0h, b0l);
-          mg_split(b0[4 * kMgRowE + 8 * nc], b1h, b1l);
-          mma3_tf32(P[nc], ah, al, b0h, b1h, b0l, b1l);
+          mg_split<FAST>(b0[8 * nc], b0h, b0l);
+          mg_split<FAST>(b0[4 * kMgRowE + 8 * nc], b1h, b1l);
+          mg_mma3<FAST>(P[nc], ah, al, b0h, b1h, b0l, b1l);
         }
       }
       // a C fragment: rows g8 (+8), the complex position 4 nc + t4
@@ -374,10 +383,10 @@ size_t mg_expand_warp(int K) { return (size_t)(3 * 8 * ((2 * K + 7) / 8) + 1) * 
 
 template <int MTM, bool VEC>
 cudaError_t launch_contract_t(const float2* in, float2* out, long long outer, long long inner, int N, int Ng, int off,
-                              int K, float scale, cudaStream_t st) {
+                              int K, float scale, bool fast, cudaStream_t st) {
   const MgCfg c = mg_cfg(mg_contract_table(N, MTM), mg_contract_warp(MTM));
   if (c.warps < 2) return cudaErrorInvalidConfiguration;
-  auto kern = midg_contract_kernel<MTM, VEC>;
+  auto kern = fast ? midg_contract_kernel<MTM, VEC, true> : midg_contract_kernel<MTM, VEC, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
   if (e != cudaSuccess) return e;
   const long long tasks = outer * ((inner + kMgPos - 1) / kMgPos);
@@ -389,10 +398,10 @@ cudaError_t launch_contract_t(const float2* in, float2* out, long long outer, lo
 
 template <bool VEC>
 cudaError_t launch_expand_t(const float2* in, float2* out, long long outer, long long inner, int N, int Ng, int off, int K,
-                            float scale, cudaStream_t st) {
+                            float scale, bool fast, cudaStream_t st) {
   const MgCfg c = mg_cfg(mg_expand_table(N, K), mg_expand_warp(K));
   if (c.warps < 2) return cudaErrorInvalidConfiguration;
-  auto kern = midg_expand_kernel<VEC>;
+  auto kern = fast ? midg_expand_kernel<VEC, true> : midg_expand_kernel<VEC, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
   if (e != cudaSuccess) return e;
   const long long tasks = outer * ((inner + kMgPos - 1) / kMgPos);
@@ -417,15 +426,15 @@ bool midg_local_supported(int Nl, int K) {
 }
 
 cudaError_t launch_midg_local(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int Nl,
-                              int Ng, int off, float scale, cudaStream_t st) {
+                              int Ng, int off, float scale, bool fast, cudaStream_t st) {
   if (outer * inner <= 0) return cudaSuccess;
   const bool vec = (inner % 2 == 0) && ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
-  if (!forward) return vec ? launch_expand_t<true>(in, out, outer, inner, Nl, Ng, off, K, scale, st)
-                           : launch_expand_t<false>(in, out, outer, inner, Nl, Ng, off, K, scale, st);
+  if (!forward) return vec ? launch_expand_t<true>(in, out, outer, inner, Nl, Ng, off, K, scale, fast, st)
+                           : launch_expand_t<false>(in, out, outer, inner, Nl, Ng, off, K, scale, fast, st);
   switch ((2 * K + 15) / 16) {
 #define DTST_MG(M) \
-  case M: return vec ? launch_contract_t<M, true>(in, out, outer, inner, Nl, Ng, off, K, scale, st) \
-                     : launch_contract_t<M, false>(in, out, outer, inner, Nl, Ng, off, K, scale, st);
+  case M: return vec ? launch_contract_t<M, true>(in, out, outer, inner, Nl, Ng, off, K, scale, fast, st) \
+                     : launch_contract_t<M, false>(in, out, outer, inner, Nl, Ng, off, K, scale, fast, st);
     DTST_MG(1) DTST_MG(2) DTST_MG(3) DTST_MG(4)
 #undef DTST_MG
     default: return cudaErrorNotSupported;
@@ -433,8 +442,8 @@ cudaError_t launch_midg_local(bool forward, int K, const float2* in, float2* out
 }
 
 cudaError_t launch_midg(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int N,
-                        float scale, cudaStream_t st) {
-  return launch_midg_local(forward, K, in, out, outer, inner, N, N, 0, scale, st);
+                        float scale, bool fast, cudaStream_t st) {
+  return launch_midg_local(forward, K, in, out, outer, inner, N, N, 0, scale, fast, st);
 }
 
 }  // namespace dtst

@@ -33,10 +33,25 @@ __device__ __forceinline__ void g_cp_async_commit() { asm volatile("cp.async.com
 template <int N>
 __device__ __forceinline__ void g_cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// hi = the value with its low 13 mantissa bits cleared, lo = the exact rest (the tensor core drops lo's low bits)
+// hi = the value with its low 13 mantissa bits cleared, lo = the exact rest (the tensor core drops lo's low bits).
+// FAST (single-pass TF32, a plan option): the value rounded to the 11 bits the tensor core reads (it ignores the
+// low 13 bits, so adding half a unit of the last kept bit rounds); no lo part - every use of it below disappears.
+template <bool FAST>
 __device__ __forceinline__ void g_split(float v, uint32_t& hi, uint32_t& lo) {
-  hi = __float_as_uint(v) & 0xffffe000u;
-  lo = __float_as_uint(v - __uint_as_float(hi));
+  if (FAST) {
+    hi = __float_as_uint(v) + 0x1000u;
+    lo = 0u;
+  } else {
+    hi = __float_as_uint(v) & 0xffffe000u;
+    lo = __float_as_uint(v - __uint_as_float(hi));
+  }
+}
+// one product: compensated (three MMAs, d += (ahi + alo)(bhi + blo) without lo * lo) or, FAST, the hi parts alone
+template <bool FAST>
+__device__ __forceinline__ void g_mma3(float (&d)[4], const uint32_t (&ahi)[4], const uint32_t (&alo)[4], uint32_t bh0,
+                                       uint32_t bh1, uint32_t bl0, uint32_t bl1) {
+  if (FAST) mma_m16n8k8_tf32(d, ahi, bh0, bh1);
+  else mma3_tf32(d, ahi, alo, bh0, bh1, bl0, bl1);
 }
 
 __device__ __forceinline__ void g_bits(const float4& v, uint32_t (&o)[4]) {
@@ -46,8 +61,9 @@ __device__ __forceinline__ void g_bits(const float4& v, uint32_t (&o)[4]) {
   o[3] = __float_as_uint(v.w);
 }
 // one compensated product with the 8-column operand as a table entry (b0 hi, b1 hi, b0 lo, b1 lo)
+template <bool FAST>
 __device__ __forceinline__ void g_mma3q(float (&d)[4], const uint32_t (&ahi)[4], const uint32_t (&alo)[4], const float4& b) {
-  mma3_tf32(d, ahi, alo, __float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
+  g_mma3<FAST>(d, ahi, alo, __float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
 }
 
 // cos (part 0) or sin (part 1) of 2 pi f (j + 1/2) / N, the phase reduced exactly in integers
@@ -60,7 +76,7 @@ __device__ __forceinline__ float g_basis(int part, int f, int j, int N) {
 // ---------------------------------------------------------------------------------------------
 // contraction.  MT m-tiles of 16 rows per task, NT n-tiles of 8 frequencies (k3 <= 8 NT).
 // ---------------------------------------------------------------------------------------------
-template <int MT, int NT, int ST>
+template <int MT, int NT, int ST, bool FAST>
 __global__ void __launch_bounds__(kGMaxWarps * 32, 1)
 rowg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long long rows, int N3, int K3, float scale,
                      int herm, int stage_floats) {
@@ -154,13 +170,13 @@ rowg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long
           const bool in = j < half, mid = odd && j == half;
           const int ja = (in || mid) ? j : 0, jb = in ? N3 - 1 - j : ja;
           const float a = T[row * N3 + ja], b = T[row * N3 + jb];
-          g_split(in ? a + b : (mid ? a : 0.f), sh[e], sl[e]);
-          g_split(in ? a - b : 0.f, dh[e], dl[e]);
+          g_split<FAST>(in ? a + b : (mid ? a : 0.f), sh[e], sl[e]);
+          g_split<FAST>(in ? a - b : 0.f, dh[e], dl[e]);
         }
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-          g_mma3q(accC[mt][nt], sh, sl, bc[nt]);
-          g_mma3q(accS[mt][nt], dh, dl, bs[nt]);
+          g_mma3q<FAST>(accC[mt][nt], sh, sl, bc[nt]);
+          g_mma3q<FAST>(accS[mt][nt], dh, dl, bs[nt]);
         }
       }
     }
@@ -198,7 +214,7 @@ rowg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long
 // Q_j = sum_f Im z'_f sin theta_{f,j}, z'_f = scale c_f e^{-i pi f / N3} in_f.  MT m-tiles of 16 rows per task,
 // KSF k-steps of 8 frequencies (k3 <= 8 KSF).
 // ---------------------------------------------------------------------------------------------
-template <int MT, int KSF>
+template <int MT, int KSF, bool FAST>
 __global__ void __launch_bounds__(kGMaxWarps * 32, 1)
 rowg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long long rows, int N3, int K3, float scale,
                    int herm, int stage_floats) {
@@ -270,8 +286,8 @@ rowg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long lo
         for (int e = 0; e < 4; ++e) {
           const float2 v = vin[mt][ks][e];
           const float2 r = rot[ks][e >> 1];
-          g_split(v.x * r.x - v.y * r.y, rh[mt][ks][e], rl[mt][ks][e]);
-          g_split(v.x * r.y + v.y * r.x, ih[mt][ks][e], il[mt][ks][e]);
+          g_split<FAST>(v.x * r.x - v.y * r.y, rh[mt][ks][e], rl[mt][ks][e]);
+          g_split<FAST>(v.x * r.y + v.y * r.x, ih[mt][ks][e], il[mt][ks][e]);
         }
     load_inputs(t + stride);
 #pragma unroll 1
@@ -287,8 +303,8 @@ rowg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long lo
         float P[4] = {0.f, 0.f, 0.f, 0.f}, Q[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int ks = 0; ks < KSF; ++ks) {
-          g_mma3q(P, rh[mt][ks], rl[mt][ks], bc[ks]);
-          g_mma3q(Q, ih[mt][ks], il[mt][ks], bs[ks]);
+          g_mma3q<FAST>(P, rh[mt][ks], rl[mt][ks], bc[ks]);
+          g_mma3q<FAST>(Q, ih[mt][ks], il[mt][ks], bs[ks]);
         }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -372,15 +388,16 @@ __device__ __forceinline__ float g_basis2f(int r, int n, int N2, int K2) {
   return r < K2 ? (float)c : (float)s;
 }
 
+template <bool FAST>
 __device__ __forceinline__ void g_split4(const float4& v, uint32_t (&hi)[4], uint32_t (&lo)[4]) {
-  g_split(v.x, hi[0], lo[0]);
-  g_split(v.y, hi[1], lo[1]);
-  g_split(v.z, hi[2], lo[2]);
-  g_split(v.w, hi[3], lo[3]);
+  g_split<FAST>(v.x, hi[0], lo[0]);
+  g_split<FAST>(v.y, hi[1], lo[1]);
+  g_split<FAST>(v.z, hi[2], lo[2]);
+  g_split<FAST>(v.w, hi[3], lo[3]);
 }
 
 // MT: 16-row tiles per task; NC: n-tiles of the second stage (2 for k3 <= 8, else 4); MTM: 16-mode tiles (2 K2 <= 16 MTM)
-template <int MT, int NC, int MTM, int ST>
+template <int MT, int NC, int MTM, int ST, bool FAST>
 __global__ void __launch_bounds__(kGMaxWarps * 32, 1)
 planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long long planes, int N3, int K3, int N2,
                        int K2, float scale, int herm, int stage_floats) {
@@ -484,17 +501,17 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
           const float4 ch = at[0], cl = at[32], sh = at[KS * 64], sl = at[KS * 64 + 32];
           const float a0 = Trow[ja0], b0 = Trow[jb0], a1 = Trow[ja1], b1 = Trow[jb1];
           uint32_t bsh[2], bsl[2], bdh[2], bdl[2];
-          g_split(a0 + b0, bsh[0], bsl[0]);
-          g_split(a0 - b0, bdh[0], bdl[0]);
-          g_split(a1 + b1, bsh[1], bsl[1]);
-          g_split(a1 - b1, bdh[1], bdl[1]);
+          g_split<FAST>(a0 + b0, bsh[0], bsl[0]);
+          g_split<FAST>(a0 - b0, bdh[0], bdl[0]);
+          g_split<FAST>(a1 + b1, bsh[1], bsl[1]);
+          g_split<FAST>(a1 - b1, bdh[1], bdl[1]);
           uint32_t chv[4], clv[4], shv[4], slv[4];
           g_bits(ch, chv);
           g_bits(cl, clv);
           g_bits(sh, shv);
           g_bits(sl, slv);
-          mma3_tf32(accC, chv, clv, bsh[0], bsh[1], bsl[0], bsl[1]);
-          mma3_tf32(accS, shv, slv, bdh[0], bdh[1], bdl[0], bdl[1]);
+          g_mma3<FAST>(accC, chv, clv, bsh[0], bsh[1], bsl[0], bsl[1]);
+          g_mma3<FAST>(accS, shv, slv, bdh[0], bdh[1], bdl[0], bdl[1]);
         };
 #pragma unroll 2
         for (int ks = 0; ks < KS - 1; ++ks) {               // every pair of these k-steps exists
@@ -518,8 +535,8 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
             const float C = accC[2 * fh + q], Sv = accS[2 * fh + q];
             re[q] = rot[fh].x * C + rot[fh].y * Sv;
             im[q] = rot[fh].y * C - rot[fh].x * Sv;
-            g_split(re[q], bh[2 * fh][q], bl[2 * fh][q]);
-            g_split(im[q], bh[2 * fh + 1][q], bl[2 * fh + 1][q]);
+            g_split<FAST>(re[q], bh[2 * fh][q], bl[2 * fh][q]);
+            g_split<FAST>(im[q], bh[2 * fh + 1][q], bl[2 * fh + 1][q]);
           }
           lw[2 * fh] = fmaf(ck0, re[0], fmaf(ck1, re[1], lw[2 * fh]));
           lw[2 * fh + 1] = fmaf(ck0, im[0], fmaf(ck1, im[1], lw[2 * fh + 1]));
@@ -527,9 +544,9 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
 #pragma unroll
         for (int mtm = 0; mtm < MTM; ++mtm) {
           uint32_t ah2[4], al2[4];
-          g_split4(a2tab[(grp * MTM + mtm) * 32 + lane], ah2, al2);
+          g_split4<FAST>(a2tab[(grp * MTM + mtm) * 32 + lane], ah2, al2);
 #pragma unroll
-          for (int nc = 0; nc < NC; ++nc) mma3_tf32(P[mtm][nc], ah2, al2, bh[nc][0], bh[nc][1], bl[nc][0], bl[nc][1]);
+          for (int nc = 0; nc < NC; ++nc) g_mma3<FAST>(P[mtm][nc], ah2, al2, bh[nc][0], bh[nc][1], bl[nc][0], bl[nc][1]);
         }
       }
       __syncwarp();   // every lane is done with this stage before it is filled again
@@ -575,7 +592,7 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
 constexpr int kGVS = 40;   // floats per row of the padded spectrum copy: 8 mod 32, conflict-free fragment loads
 
 // MT: 16-row tiles per task; KSF: k-steps of 8 frequencies (k3 <= 8 KSF); KS2: k-steps of 8 modes (2 K2 <= 8 KS2)
-template <int MT, int KSF, int KS2>
+template <int MT, int KSF, int KS2, bool FAST>
 __global__ void __launch_bounds__(kGMaxWarps * 32, 1)
 planeg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long long planes, int N3, int K3, int N2,
                      int K2, float scale, int herm, int stage_floats) {
@@ -690,13 +707,13 @@ planeg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long 
 #pragma unroll
         for (int ks2 = 0; ks2 < KS2; ++ks2) {
           uint32_t ah2[4], al2[4];
-          g_split4(a2e[(tile * KS2 + ks2) * 32 + lane], ah2, al2);
+          g_split4<FAST>(a2e[(tile * KS2 + ks2) * 32 + lane], ah2, al2);
 #pragma unroll
           for (int nc = 0; nc < NC; ++nc) {
             uint32_t b0h, b0l, b1h, b1l;
-            g_split(Bm[(8 * ks2 + t4) * kGVS + 8 * nc + g8], b0h, b0l);
-            g_split(Bm[(8 * ks2 + t4 + 4) * kGVS + 8 * nc + g8], b1h, b1l);
-            mma3_tf32(P[nc], ah2, al2, b0h, b1h, b0l, b1l);
+            g_split<FAST>(Bm[(8 * ks2 + t4) * kGVS + 8 * nc + g8], b0h, b0l);
+            g_split<FAST>(Bm[(8 * ks2 + t4 + 4) * kGVS + 8 * nc + g8], b1h, b1l);
+            g_mma3<FAST>(P[nc], ah2, al2, b0h, b1h, b0l, b1l);
           }
         }
         // a C fragment holds the complex value of frequency 4 nc + t4 for the rows g8 (+8): rotated, it is the
@@ -709,8 +726,8 @@ planeg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long 
             const int nc = 2 * ks + (e >> 1), h = e & 1;
             const float ur = P[nc][2 * h], ui = P[nc][2 * h + 1];
             const float2 r = rot[ks][e >> 1];
-            g_split(ur * r.x - ui * r.y, rh[ks][e], rl[ks][e]);
-            g_split(ur * r.y + ui * r.x, ih[ks][e], il[ks][e]);
+            g_split<FAST>(ur * r.x - ui * r.y, rh[ks][e], rl[ks][e]);
+            g_split<FAST>(ur * r.y + ui * r.x, ih[ks][e], il[ks][e]);
           }
         // one tile of 8 pairs: y_j = P - Q, y_{N3-1-j} = P + Q; `last`: pairs past the end go to the dump slot behind the
         // task's floats, the middle sample of an odd extent is P alone
@@ -720,8 +737,8 @@ planeg_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long 
 #pragma unroll
           for (int ks = 0; ks < KSF; ++ks) {
             const float4 bc = bt[ks * NTJ * 32], bs = bt[(KSF + ks) * NTJ * 32];
-            g_mma3q(Pj, rh[ks], rl[ks], bc);
-            g_mma3q(Qj, ih[ks], il[ks], bs);
+            g_mma3q<FAST>(Pj, rh[ks], rl[ks], bc);
+            g_mma3q<FAST>(Qj, ih[ks], il[ks], bs);
           }
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
@@ -782,13 +799,13 @@ int g_stage_floats(int N3, int mt) { return (16 * mt * N3 + 3) & ~3; }
 int g_stages(size_t table_bytes, size_t stage_bytes) { return g_cfg(table_bytes, 3 * stage_bytes).warps >= 4 ? 3 : 2; }
 
 template <int MT, int NT, int ST>
-cudaError_t launch_contract_s(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm,
+cudaError_t launch_contract_s(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm, bool fast,
                               cudaStream_t st) {
   const int H = (N3 + 1) / 2, KS = (H + 7) / 8;
   const int sf = g_stage_floats(N3, MT);
   const GCfg c = g_cfg((size_t)2 * KS * NT * 32 * 16, (size_t)ST * sf * 4);
   if (c.warps < 2) return cudaErrorInvalidConfiguration;
-  auto kern = rowg_contract_kernel<MT, NT, ST>;
+  auto kern = fast ? rowg_contract_kernel<MT, NT, ST, true> : rowg_contract_kernel<MT, NT, ST, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
   if (e != cudaSuccess) return e;
   const long long tasks = (rows + 16 * MT - 1) / (16 * MT);
@@ -799,22 +816,22 @@ cudaError_t launch_contract_s(const float* x, float2* out, long long rows, int N
 }
 
 template <int MT, int NT>
-cudaError_t launch_contract_t(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm,
+cudaError_t launch_contract_t(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm, bool fast,
                               cudaStream_t st) {
   const int H = (N3 + 1) / 2, KS = (H + 7) / 8;
   const size_t sb = (size_t)g_stage_floats(N3, MT) * 4;
-  return g_stages((size_t)2 * KS * NT * 32 * 16, sb) == 3 ? launch_contract_s<MT, NT, 3>(x, out, rows, N3, K3, scale, herm, st)
-                                                          : launch_contract_s<MT, NT, 2>(x, out, rows, N3, K3, scale, herm, st);
+  return g_stages((size_t)2 * KS * NT * 32 * 16, sb) == 3 ? launch_contract_s<MT, NT, 3>(x, out, rows, N3, K3, scale, herm, fast, st)
+                                                          : launch_contract_s<MT, NT, 2>(x, out, rows, N3, K3, scale, herm, fast, st);
 }
 
 template <int MT, int KSF>
-cudaError_t launch_expand_t(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm,
+cudaError_t launch_expand_t(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm, bool fast,
                             cudaStream_t st) {
   const int H = (N3 + 1) / 2, NTJ = (H + 7) / 8;
   const int sf = g_stage_floats(N3, MT);
   const GCfg c = g_cfg((size_t)2 * KSF * NTJ * 32 * 16, (size_t)sf * 4);
   if (c.warps < 2) return cudaErrorInvalidConfiguration;
-  auto kern = rowg_expand_kernel<MT, KSF>;
+  auto kern = fast ? rowg_expand_kernel<MT, KSF, true> : rowg_expand_kernel<MT, KSF, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
   if (e != cudaSuccess) return e;
   const long long tasks = (rows + 16 * MT - 1) / (16 * MT);
@@ -838,11 +855,11 @@ size_t pg_expand_rows(int KS2) { return (size_t)(3 * 8 * KS2 + 1) * kGVS * 4; }
 
 template <int MT, int NC, int MTM, int ST>
 cudaError_t launch_pg_contract_s(const float* x, float2* out, long long planes, int N3, int K3, int N2, int K2,
-                                 float scale, int herm, cudaStream_t st) {
+                                 float scale, int herm, bool fast, cudaStream_t st) {
   const int sf = g_stage_floats(N3, MT) + 4;   // + the zero slot
   const GCfg c = g_cfg(pg_contract_table(N3, N2, MTM), (size_t)ST * sf * 4 + pg_contract_scratch(MTM));
   if (c.warps < 2) return cudaErrorInvalidConfiguration;
-  auto kern = planeg_contract_kernel<MT, NC, MTM, ST>;
+  auto kern = fast ? planeg_contract_kernel<MT, NC, MTM, ST, true> : planeg_contract_kernel<MT, NC, MTM, ST, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
   if (e != cudaSuccess) return e;
   const long long want = (planes + c.warps - 1) / c.warps;
@@ -853,20 +870,20 @@ cudaError_t launch_pg_contract_s(const float* x, float2* out, long long planes, 
 
 template <int MT, int NC, int MTM>
 cudaError_t launch_pg_contract_t(const float* x, float2* out, long long planes, int N3, int K3, int N2, int K2,
-                                 float scale, int herm, cudaStream_t st) {
+                                 float scale, int herm, bool fast, cudaStream_t st) {
   const size_t sb = (size_t)(g_stage_floats(N3, MT) + 4) * 4;
   return g_stages(pg_contract_table(N3, N2, MTM) + kGMaxWarps * pg_contract_scratch(MTM), sb) == 3
-             ? launch_pg_contract_s<MT, NC, MTM, 3>(x, out, planes, N3, K3, N2, K2, scale, herm, st)
-             : launch_pg_contract_s<MT, NC, MTM, 2>(x, out, planes, N3, K3, N2, K2, scale, herm, st);
+             ? launch_pg_contract_s<MT, NC, MTM, 3>(x, out, planes, N3, K3, N2, K2, scale, herm, fast, st)
+             : launch_pg_contract_s<MT, NC, MTM, 2>(x, out, planes, N3, K3, N2, K2, scale, herm, fast, st);
 }
 
 template <int MT, int KSF, int KS2>
 cudaError_t launch_pg_expand_t(const float2* in, float* y, long long planes, int N3, int K3, int N2, int K2,
-                               float scale, int herm, cudaStream_t st) {
+                               float scale, int herm, bool fast, cudaStream_t st) {
   const int sf = g_stage_floats(N3, MT) + 4;   // + the dump slot
   const GCfg c = g_cfg(pg_expand_table(N3, N2, KSF, KS2), (size_t)sf * 4 + pg_expand_rows(KS2));
   if (c.warps < 2) return cudaErrorInvalidConfiguration;
-  auto kern = planeg_expand_kernel<MT, KSF, KS2>;
+  auto kern = fast ? planeg_expand_kernel<MT, KSF, KS2, true> : planeg_expand_kernel<MT, KSF, KS2, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
   if (e != cudaSuccess) return e;
   const long long want = (planes + c.warps - 1) / c.warps;
@@ -892,9 +909,9 @@ bool planeg_supported(int N3, int K3, int N2, int K2) {
 }
 
 cudaError_t launch_planeg_contract(const float* x, float2* out, long long planes, int N3, int K3, int N2, int K2,
-                                   float scale, int herm, cudaStream_t st) {
+                                   float scale, int herm, bool fast, cudaStream_t st) {
   const bool two = g_mt(N3) == 2, wide = K3 > 8, tall = 2 * K2 > 16;
-#define DTST_PG(MT, NC, MTM) return launch_pg_contract_t<MT, NC, MTM>(x, out, planes, N3, K3, N2, K2, scale, herm, st)
+#define DTST_PG(MT, NC, MTM) return launch_pg_contract_t<MT, NC, MTM>(x, out, planes, N3, K3, N2, K2, scale, herm, fast, st)
   if (two) {
     if (wide) { if (tall) DTST_PG(2, 4, 2); DTST_PG(2, 4, 1); }
     if (tall) DTST_PG(2, 2, 2);
@@ -907,11 +924,11 @@ cudaError_t launch_planeg_contract(const float* x, float2* out, long long planes
 }
 
 cudaError_t launch_planeg_expand(const float2* in, float* y, long long planes, int N3, int K3, int N2, int K2,
-                                 float scale, int herm, cudaStream_t st) {
+                                 float scale, int herm, bool fast, cudaStream_t st) {
   const bool two = g_mt(N3) == 2;
   const int KSF = (K3 + 7) / 8, KS2 = (2 * K2 + 7) / 8;
 #define DTST_PG(MT, A, B) \
-  if (two == (MT == 2) && KSF == A && KS2 == B) return launch_pg_expand_t<MT, A, B>(in, y, planes, N3, K3, N2, K2, scale, herm, st);
+  if (two == (MT == 2) && KSF == A && KS2 == B) return launch_pg_expand_t<MT, A, B>(in, y, planes, N3, K3, N2, K2, scale, herm, fast, st);
   DTST_PG(2, 1, 1) DTST_PG(2, 1, 2) DTST_PG(2, 1, 3) DTST_PG(2, 1, 4)
   DTST_PG(2, 2, 1) DTST_PG(2, 2, 2) DTST_PG(2, 2, 3) DTST_PG(2, 2, 4)
   DTST_PG(1, 1, 1) DTST_PG(1, 1, 2) DTST_PG(1, 1, 3) DTST_PG(1, 1, 4)
@@ -931,31 +948,31 @@ bool rowg_supported(int N3, int K3) {
   return g_cfg(table, g_stages(table, sf) * sf).warps >= 2 && g_cfg(table, sf).warps >= 2;
 }
 
-cudaError_t launch_rowg_contract(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm,
+cudaError_t launch_rowg_contract(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm, bool fast,
                                  cudaStream_t st) {
   const int NT = (K3 + 7) / 8;
   const bool two = g_mt(N3) == 2;
   switch (NT) {
-    case 1: return two ? launch_contract_t<2, 1>(x, out, rows, N3, K3, scale, herm, st)
-                       : launch_contract_t<1, 1>(x, out, rows, N3, K3, scale, herm, st);
-    case 2: return two ? launch_contract_t<2, 2>(x, out, rows, N3, K3, scale, herm, st)
-                       : launch_contract_t<1, 2>(x, out, rows, N3, K3, scale, herm, st);
-    case 3: return launch_contract_t<1, 3>(x, out, rows, N3, K3, scale, herm, st);
-    default: return launch_contract_t<1, 4>(x, out, rows, N3, K3, scale, herm, st);
+    case 1: return two ? launch_contract_t<2, 1>(x, out, rows, N3, K3, scale, herm, fast, st)
+                       : launch_contract_t<1, 1>(x, out, rows, N3, K3, scale, herm, fast, st);
+    case 2: return two ? launch_contract_t<2, 2>(x, out, rows, N3, K3, scale, herm, fast, st)
+                       : launch_contract_t<1, 2>(x, out, rows, N3, K3, scale, herm, fast, st);
+    case 3: return launch_contract_t<1, 3>(x, out, rows, N3, K3, scale, herm, fast, st);
+    default: return launch_contract_t<1, 4>(x, out, rows, N3, K3, scale, herm, fast, st);
   }
 }
 
-cudaError_t launch_rowg_expand(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm,
+cudaError_t launch_rowg_expand(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm, bool fast,
                                cudaStream_t st) {
   const int KSF = (K3 + 7) / 8;
   const bool two = g_mt(N3) == 2;
   switch (KSF) {
-    case 1: return two ? launch_expand_t<2, 1>(in, y, rows, N3, K3, scale, herm, st)
-                       : launch_expand_t<1, 1>(in, y, rows, N3, K3, scale, herm, st);
-    case 2: return two ? launch_expand_t<2, 2>(in, y, rows, N3, K3, scale, herm, st)
-                       : launch_expand_t<1, 2>(in, y, rows, N3, K3, scale, herm, st);
-    case 3: return launch_expand_t<1, 3>(in, y, rows, N3, K3, scale, herm, st);
-    default: return launch_expand_t<1, 4>(in, y, rows, N3, K3, scale, herm, st);
+    case 1: return two ? launch_expand_t<2, 1>(in, y, rows, N3, K3, scale, herm, fast, st)
+                       : launch_expand_t<1, 1>(in, y, rows, N3, K3, scale, herm, fast, st);
+    case 2: return two ? launch_expand_t<2, 2>(in, y, rows, N3, K3, scale, herm, fast, st)
+                       : launch_expand_t<1, 2>(in, y, rows, N3, K3, scale, herm, fast, st);
+    case 3: return launch_expand_t<1, 3>(in, y, rows, N3, K3, scale, herm, fast, st);
+    default: return launch_expand_t<1, 4>(in, y, rows, N3, K3, scale, herm, fast, st);
   }
 }
 

@@ -392,11 +392,11 @@ static bool slab_own_supported(int Nl, int K) {
 bool slab_supported(int Nl, int K) { return slab_own_supported(Nl, K) || midg_local_supported(Nl, K); }
 
 cudaError_t launch_slab(bool forward, int K, const float2* in, float2* out, long long outer, long long inner, int Nl,
-                        int N, int off, int P, cudaStream_t st) {
+                        int N, int off, int P, bool fast, cudaStream_t st) {
   if (outer * inner <= 0) return cudaSuccess;
   // Slabs of one device are consecutive rows with consecutive global indices: taken together they are ONE local
   // block that starts at `off` (the sum over the slabs is then part of the contraction's own sum).
-  if (!slab_own_supported(Nl, K)) return launch_midg_local(forward, K, in, out, outer, inner, Nl, N, off, 1.0f, st);
+  if (!slab_own_supported(Nl, K)) return launch_midg_local(forward, K, in, out, outer, inner, Nl, N, off, 1.0f, fast, st);
   // contraction of slabs that are whole k-steps of 8 rows: tensor-core kernel
   const bool aligned16 = ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
   if (forward && aligned16 && inner % 4 == 0 && P >= 1 && Nl % P == 0 && (Nl / P) % 8 == 0) {

@@ -23,7 +23,7 @@ def _dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def run_layer_and_check(w, path="auto", P=1, check_backward=True, tol=TOL, **plan_kw):
+def run_layer_and_check(w, path="auto", P=1, check_backward=True, tol=TOL, fine_scale=1.0, **plan_kw):
     x = I.make_field(w)
     W = I.make_weights(w)
     g = I.make_upstream_grad(w)
@@ -63,8 +63,8 @@ def run_layer_and_check(w, path="auto", P=1, check_backward=True, tol=TOL, **pla
         fine["grad_x/plane"] = per_plane_excess(gx.cpu().numpy(), gx_ref)
     for name, e in errs.items():
         assert e <= tol, (w.name, path, P, name, e, errs)
-    for name, e in fine.items():
-        assert e <= 1.0, (w.name, path, P, name, e, fine)
+    for name, e in fine.items():     # fine_scale: the per-mode / per-plane bars scaled with a looser tolerance
+        assert e <= fine_scale, (w.name, path, P, name, e, fine)
     plan.close()
     return errs
 
@@ -458,6 +458,31 @@ def test_any_contiguous_extent_runs_on_the_row_kernels(case):
     run_layer_and_check(w, "auto")
     if N[0] % 4 == 0 and len(N) > 1:
         run_layer_and_check(w, "auto", P=4)
+
+
+# ------------------------------------------------------------------ single-pass TF32 arithmetic (a plan option)
+@pytest.mark.parametrize("N,k", [((16, 16, 32, 30), (4, 8, 8, 16)),      # the paper's layer in small: fused plane kernels
+                                 ((32, 45, 100), (6, 10, 12)),           # row kernel + middle kernels of any extent
+                                 ((40, 90), (20, 17))])
+def test_single_pass_tf32_meets_its_stated_error(N, k):
+    """DTST_ARITH_TF32: every output within 2e-3 of the float64 statement (and not by accident on the compensated path:
+    the error is well above that path's), the default arithmetic untouched."""
+    w = I.custom_workload("tf32", 1, 2, 2, N, k, field="grf", seed=41)
+    errs_fast = run_layer_and_check(w, "auto", tol=2e-3, fine_scale=200.0, arithmetic="tf32")
+    errs = run_layer_and_check(w, "auto")
+    for name in ("Xhat", "y", "grad_x", "grad_W"):
+        assert errs_fast[name] > 10.0 * errs[name], (name, errs_fast, errs)
+
+
+def test_arithmetic_option_rejects_unknown_modes():
+    from paper_2607_14394_b200 import binding as Bn
+    plan = _plan(I.WORKLOADS["cfg1_2d_64"])
+    with pytest.raises(Bn.DtstError) as e:
+        Bn.dtst_plan_set_arithmetic(plan.handle, 7)
+    assert e.value.status == Bn.DTST_ERR_INVALID_ARG
+    plan.set_arithmetic("tf32")
+    plan.set_arithmetic("tf32x3")
+    plan.close()
 
 
 # ------------------------------------------------------------------ third dimension inside the forward plane kernel
