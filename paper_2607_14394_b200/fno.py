@@ -25,8 +25,8 @@ class FNO:
     """
 
     def __init__(self, N: Sequence[int], kmax: Sequence[int], B: int, C_a: int, C_u: int, width: int, layers: int,
-                 device=None, seed: int = 0):
-        self.plan = Bn.Plan(N, kmax, B, width, width, device=device)
+                 device=None, seed: int = 0, arithmetic: str = "tf32x3"):
+        self.plan = Bn.Plan(N, kmax, B, width, width, device=device, arithmetic=arithmetic)
         dev = self.plan.device
         self.N, self.B, self.C_a, self.C_u, self.width, self.layers = tuple(N), B, C_a, C_u, width, layers
         gen = torch.Generator(device=dev).manual_seed(seed)
