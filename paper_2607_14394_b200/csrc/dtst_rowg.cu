@@ -72,6 +72,13 @@ __device__ __forceinline__ float g_basis(int part, int f, int j, int N) {
   sincospi((double)(((long long)f * (2 * j + 1)) % (2ll * N)) / (double)N, &s, &c);
   return part == 0 ? (float)c : (float)s;
 }
+// The same for the CONTRACTION tables.  The kernels form s_j = x_j + x_{N-1-j}, d_j = x_j - x_{N-1-j} for every pair
+// index without looking at it: the middle sample of an odd extent pairs with itself (s = 2 x, d = 0), so its cosine
+// carries the weight 1/2; pair indices past the end are clamped to the last pair and meet zero table entries.
+__device__ __forceinline__ float g_basis_c(int part, int f, int j, int N) {
+  const float v = g_basis(part, f, j, N);
+  return ((N & 1) && j == N / 2 && part == 0) ? 0.5f * v : v;
+}
 
 // ---------------------------------------------------------------------------------------------
 // contraction.  MT m-tiles of 16 rows per task, NT n-tiles of 8 frequencies (k3 <= 8 NT).
@@ -83,8 +90,7 @@ rowg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long
   pdl_trigger();
   constexpr int TR = 16 * MT;
   extern __shared__ float4 rg_smem[];
-  const int half = N3 / 2, H = (N3 + 1) / 2, KS = (H + 7) / 8;   // pairs (odd N3: + the middle sample), k-steps
-  const bool odd = (N3 & 1) != 0;
+  const int H = (N3 + 1) / 2, KS = (H + 7) / 8;   // pairs (odd N3: + the middle sample), k-steps
   float4* btab = rg_smem;                                          // [part][ks][nt][lane] = (b0 hi, b1 hi, b0 lo, b1 lo)
   float* ring = reinterpret_cast<float*>(btab + (size_t)2 * KS * NT * 32);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g8 = lane >> 2, t4 = lane & 3;
@@ -101,7 +107,7 @@ rowg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       const int j = 8 * ks + (l & 3) + 4 * h;
-      split_tf32_rna((f < K3 && j < H) ? g_basis(part, f, j, N3) : 0.f, hi[h], lo[h]);
+      split_tf32_rna((f < K3 && j < H) ? g_basis_c(part, f, j, N3) : 0.f, hi[h], lo[h]);
     }
     btab[e] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(lo[0]), __uint_as_float(lo[1]));
   }
@@ -166,12 +172,10 @@ rowg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long
 #pragma unroll
         for (int e = 0; e < 4; ++e) {                              // A fragment: row g8 (+8), pair t4 (+4)
           const int row = 16 * mt + g8 + 8 * (e & 1);
-          const int j = 8 * ks + t4 + 4 * (e >> 1);
-          const bool in = j < half, mid = odd && j == half;
-          const int ja = (in || mid) ? j : 0, jb = in ? N3 - 1 - j : ja;
-          const float a = T[row * N3 + ja], b = T[row * N3 + jb];
-          g_split<FAST>(in ? a + b : (mid ? a : 0.f), sh[e], sl[e]);
-          g_split<FAST>(in ? a - b : 0.f, dh[e], dl[e]);
+          const int j = min(8 * ks + t4 + 4 * (e >> 1), H - 1);   // past the end: any pair, its table entries are zero
+          const float a = T[row * N3 + j], b = T[row * N3 + N3 - 1 - j];
+          g_split<FAST>(a + b, sh[e], sl[e]);
+          g_split<FAST>(a - b, dh[e], dl[e]);
         }
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
@@ -404,7 +408,7 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
   pdl_trigger();
   constexpr int TR = 16 * MT, GPT = 2 * MT;   // rows and 8-row groups per task
   extern __shared__ float4 rg_smem[];
-  const int half = N3 / 2, H = (N3 + 1) / 2, KS = (H + 7) / 8;
+  const int H = (N3 + 1) / 2, KS = (H + 7) / 8;
   const int NG = N2 / 8, TP = N2 / TR;
   float4* atab = rg_smem;                                   // [part][ks][hi | lo][lane]: the row stage's 16-row operand
   float4* a2tab = atab + (size_t)2 * KS * 2 * 32;           // [group][mtm][lane]: the second stage's, folded, unsplit
@@ -420,7 +424,7 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
 #pragma unroll
     for (int q = 0; q < 4; ++q) {                           // A fragment: frequency l >> 2 (+8), pair l & 3 (+4)
       const int f = (l >> 2) + 8 * (q & 1), j = 8 * ks + (l & 3) + 4 * (q >> 1);
-      split_tf32_rna((f < K3 && j < H) ? g_basis(part, f, j, N3) : 0.f, hi[q], lo[q]);
+      split_tf32_rna((f < K3 && j < H) ? g_basis_c(part, f, j, N3) : 0.f, hi[q], lo[q]);
     }
     atab[((size_t)(part * KS + ks) * 2 + 0) * 32 + l] =
         make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(hi[2]), __uint_as_float(hi[3]));
@@ -450,9 +454,7 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
 
   float* S = ring + (size_t)warp * (ST * stage_floats + SCRF);
   float* scr = S + (size_t)ST * stage_floats;
-  if (lane < 4)                                             // the zero slot behind every stage's TR x N3 floats
-    for (int q = 0; q < ST; ++q) S[(size_t)q * stage_floats + TR * N3 + lane] = 0.f;
-  __syncwarp();
+  const int jl0 = min(8 * (KS - 1) + t4, H - 1), jl1 = min(8 * (KS - 1) + t4 + 4, H - 1);
   const long long stride = (long long)W * gridDim.x;
   long long pl = (long long)warp * gridDim.x + blockIdx.x;
   long long apl = pl;                                       // the task staged next: plane and place within it
@@ -490,16 +492,13 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
       const float* T = S + (size_t)s * stage_floats;
 #pragma unroll 1
       for (int gq = 0; gq < GPT; ++gq) {
-        const int rowoff = (8 * gq + g8) * N3;
-        const float* Trow = T + rowoff;                     // this lane's row of the group (the B operand's n index)
-        const int zrel = TR * N3 - rowoff;                  // the stage's zero slot, as a column of this row
+        const float* Trow = T + (8 * gq + g8) * N3;         // this lane's row of the group (the B operand's n index)
         float accC[4] = {0.f, 0.f, 0.f, 0.f}, accS[4] = {0.f, 0.f, 0.f, 0.f};
-        // one k-step: pairs jj = 8 ks + t4 (+4) from the columns (ja, jb); a pair past the end reads the zero slot twice,
-        // the middle sample of an odd extent once (its sine is exactly zero)
-        auto step = [&](int ks, int ja0, int jb0, int ja1, int jb1) {
+        // one k-step: the pairs at the columns (j0, N3-1-j0) and (j1, N3-1-j1)
+        auto step = [&](int ks, int j0, int j1) {
           const float4* at = atab + ks * 64 + lane;
           const float4 ch = at[0], cl = at[32], sh = at[KS * 64], sl = at[KS * 64 + 32];
-          const float a0 = Trow[ja0], b0 = Trow[jb0], a1 = Trow[ja1], b1 = Trow[jb1];
+          const float a0 = Trow[j0], b0 = Trow[N3 - 1 - j0], a1 = Trow[j1], b1 = Trow[N3 - 1 - j1];
           uint32_t bsh[2], bsl[2], bdh[2], bdl[2];
           g_split<FAST>(a0 + b0, bsh[0], bsl[0]);
           g_split<FAST>(a0 - b0, bdh[0], bdl[0]);
@@ -514,15 +513,8 @@ planeg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, lo
           g_mma3<FAST>(accS, shv, slv, bdh[0], bdh[1], bdl[0], bdl[1]);
         };
 #pragma unroll 2
-        for (int ks = 0; ks < KS - 1; ++ks) {               // every pair of these k-steps exists
-          const int jj = 8 * ks + t4;
-          step(ks, jj, N3 - 1 - jj, jj + 4, N3 - 5 - jj);
-        }
-        {
-          const int jj = 8 * (KS - 1) + t4;
-          step(KS - 1, jj < H ? jj : zrel, jj < half ? N3 - 1 - jj : zrel, jj + 4 < H ? jj + 4 : zrel,
-               jj + 4 < half ? N3 - 5 - jj : zrel);
-        }
+        for (int ks = 0; ks < KS - 1; ++ks) step(ks, 8 * ks + t4, 8 * ks + t4 + 4);
+        step(KS - 1, jl0, jl1);                             // the last k-step: pair indices clamped (zero table entries)
         // X = rot (C - i S) of (frequency g8 + 8 fh, row 2 t4 + q): the second stage's column operand
         uint32_t bh[NC][2], bl[NC][2];
         const int grp = j * GPT + gq;
@@ -856,7 +848,7 @@ size_t pg_expand_rows(int KS2) { return (size_t)(3 * 8 * KS2 + 1) * kGVS * 4; }
 template <int MT, int NC, int MTM, int ST>
 cudaError_t launch_pg_contract_s(const float* x, float2* out, long long planes, int N3, int K3, int N2, int K2,
                                  float scale, int herm, bool fast, cudaStream_t st) {
-  const int sf = g_stage_floats(N3, MT) + 4;   // + the zero slot
+  const int sf = g_stage_floats(N3, MT);
   const GCfg c = g_cfg(pg_contract_table(N3, N2, MTM), (size_t)ST * sf * 4 + pg_contract_scratch(MTM));
   if (c.warps < 2) return cudaErrorInvalidConfiguration;
   auto kern = fast ? planeg_contract_kernel<MT, NC, MTM, ST, true> : planeg_contract_kernel<MT, NC, MTM, ST, false>;
@@ -871,7 +863,7 @@ cudaError_t launch_pg_contract_s(const float* x, float2* out, long long planes, 
 template <int MT, int NC, int MTM>
 cudaError_t launch_pg_contract_t(const float* x, float2* out, long long planes, int N3, int K3, int N2, int K2,
                                  float scale, int herm, bool fast, cudaStream_t st) {
-  const size_t sb = (size_t)(g_stage_floats(N3, MT) + 4) * 4;
+  const size_t sb = (size_t)g_stage_floats(N3, MT) * 4;
   return g_stages(pg_contract_table(N3, N2, MTM) + kGMaxWarps * pg_contract_scratch(MTM), sb) == 3
              ? launch_pg_contract_s<MT, NC, MTM, 3>(x, out, planes, N3, K3, N2, K2, scale, herm, fast, st)
              : launch_pg_contract_s<MT, NC, MTM, 2>(x, out, planes, N3, K3, N2, K2, scale, herm, fast, st);
@@ -904,8 +896,8 @@ bool planeg_supported(int N3, int K3, int N2, int K2) {
   const int MTM = (2 * K2 + 15) / 16, KS2 = (2 * K2 + 7) / 8, KSF = (K3 + 7) / 8;
   const size_t sf = (size_t)g_stage_floats(N3, mt) * 4;
   const size_t ct = pg_contract_table(N3, N2, MTM), et = pg_expand_table(N3, N2, KSF, KS2);
-  const size_t scr = pg_contract_scratch(MTM), sfz = sf + 16;   // contraction stages carry a zero slot
-  return g_cfg(ct, g_stages(ct + kGMaxWarps * scr, sfz) * sfz + scr).warps >= 4 && g_cfg(et, sfz + pg_expand_rows(KS2)).warps >= 4;
+  const size_t scr = pg_contract_scratch(MTM), sfd = sf + 16;   // the expansion's staging carries a dump slot
+  return g_cfg(ct, g_stages(ct + kGMaxWarps * scr, sf) * sf + scr).warps >= 4 && g_cfg(et, sfd + pg_expand_rows(KS2)).warps >= 4;
 }
 
 cudaError_t launch_planeg_contract(const float* x, float2* out, long long planes, int N3, int K3, int N2, int K2,
