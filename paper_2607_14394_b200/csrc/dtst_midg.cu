@@ -69,17 +69,22 @@ __device__ __forceinline__ void mg_mma3(float (&d)[4], const uint32_t (&ahi)[4],
 __device__ __forceinline__ float mg_basis(int r, int n, int N, int Ng, int off, int K) {
   if (r >= 2 * K || n >= N) return 0.f;
   const long long k = r < K ? r : r - K + 1;
-  double s, c;
-  sincospi(2.0 * (double)((k * (off + n)) % Ng) / (double)Ng, &s, &c);
-  return r < K ? (float)c : (float)s;
+  // the phase is reduced exactly in integers to [0, 2); single precision from there on (1 ulp of the fp32 entry): in
+  // double precision the tables of a short-running launch took longer to build than its data to process
+  float s, c;
+  sincospif(2.0f * (float)((k * (off + n)) % Ng) / (float)Ng, &s, &c);
+  return r < K ? c : s;
 }
 __device__ __forceinline__ float mg_cosK(int n, int N, int Ng, int off, int K) {
   if (n >= N) return 0.f;
-  return (float)cospi(2.0 * (double)(((long long)K * (off + n)) % Ng) / (double)Ng);
+  return cospif(2.0f * (float)(((long long)K * (off + n)) % Ng) / (float)Ng);
 }
 
 // MTM: 16-row tiles of the folded basis (2K <= 16 MTM).  VEC: 16-byte copies (inner even, 16-byte aligned tensors).
-template <int MTM, bool VEC, bool FAST>
+// SPLIT: a task belongs to the whole CTA - warp w takes the row chunks w, w + W, .. and the warps' sums are added in
+// warp order at the task's end (through their scratch rows; a fixed order: the same bits on every run).  For
+// tensors with fewer tasks than the GPU has warps: a 2-D layer has batch x channels of them.
+template <int MTM, bool VEC, bool FAST, bool SPLIT>
 __global__ void __launch_bounds__(kMgMaxWarps * 32, 1)
 midg_contract_kernel(const float2* __restrict__ in, float2* __restrict__ out, long long outer, long long inner, int N,
                      int Ng, int off, int K, float scale) {
@@ -113,12 +118,14 @@ midg_contract_kernel(const float2* __restrict__ in, float2* __restrict__ out, lo
 
   const long long CB = (inner + kMgPos - 1) / kMgPos;
   const long long tasks = outer * CB;
-  const long long stride = (long long)W * gridDim.x;
-  long long t = (long long)warp * gridDim.x + blockIdx.x;
+  const long long stride = SPLIT ? (long long)gridDim.x : (long long)W * gridDim.x;
+  long long t = SPLIT ? (long long)blockIdx.x : (long long)warp * gridDim.x + blockIdx.x;
+  const int c_first = SPLIT ? warp : 0, c_step = SPLIT ? W : 1;   // this warp's chunks of a task
   // the chunk staged next: task (as outer index and block, advanced by additions) and chunk within it
   long long at = t, ao = t / CB, acb = t % CB;
   const long long sdiv = stride / CB, smod = stride % CB;
-  int ac = 0;
+  int ac = c_first;
+  if (ac >= NCH) at = tasks;                                   // a warp beyond the chunks of a task stages nothing
   auto load = [&](int s) {
     if (at < tasks) {
       const long long o = ao, cb = acb;
@@ -140,8 +147,9 @@ midg_contract_kernel(const float2* __restrict__ in, float2* __restrict__ out, lo
       }
     }
     mg_commit();
-    if (++ac == NCH) {
-      ac = 0;
+    ac += c_step;
+    if (ac >= NCH) {
+      ac = c_first;
       at += stride;
       ao += sdiv;
       acb += smod;
@@ -163,7 +171,7 @@ midg_contract_kernel(const float2* __restrict__ in, float2* __restrict__ out, lo
       for (int nc = 0; nc < 4; ++nc)
 #pragma unroll
         for (int e = 0; e < 4; ++e) P[mtm][nc][e] = 0.f;
-    for (int ch = 0; ch < NCH; ++ch) {
+    for (int ch = c_first; ch < NCH; ch += c_step) {
       load(s == 0 ? kMgStages - 1 : s - 1);
       mg_wait<kMgStages - 1>();
       __syncwarp();
@@ -207,27 +215,36 @@ midg_contract_kernel(const float2* __restrict__ in, float2* __restrict__ out, lo
       v += __shfl_xor_sync(0xffffffffu, v, 2);
       if (t4 == 0) scr[16 * MTM * kMgScw + 8 * nc + g8] = v;
     }
-    __syncwarp();
+    if (SPLIT) __syncthreads();
+    else __syncwarp();
     {
       const long long o = t / CB, cb = t - o * CB;
       const int valid = (int)(inner - cb * kMgPos < kMgPos ? inner - cb * kMgPos : kMgPos);
       float2* ob = out + o * (2 * K) * inner + cb * kMgPos;
-      for (int idx = lane; idx < 2 * K * kMgPos; idx += 32) {
+      const int nw = SPLIT ? W : 1;                                 // scratch areas to add, in warp order
+      const float* sbase = SPLIT ? areas + kMgStages * STAGE : scr;
+      const int wstride = kMgStages * STAGE + SCRF;
+      for (int idx = SPLIT ? (int)threadIdx.x : lane; idx < 2 * K * kMgPos; idx += SPLIT ? (int)blockDim.x : 32) {
         const int pm = idx >> 4, i = idx & 15;
         if (i >= valid) continue;
         const int k = pm < K ? pm : 2 * K - pm;
         const float sg = pm < K ? -1.f : 1.f;
-        const float* ar = scr + (k < K ? k : 16 * MTM) * kMgScw + 2 * i;
-        float2 v = make_float2(ar[0], ar[1]);
-        if (k > 0) {
-          const float* br = scr + (K + k - 1) * kMgScw + 2 * i;
-          v.x -= sg * br[1];
-          v.y += sg * br[0];
+        float2 a = make_float2(0.f, 0.f), bq = make_float2(0.f, 0.f);
+        for (int w = 0; w < nw; ++w) {
+          const float* ar = sbase + (size_t)w * wstride + (k < K ? k : 16 * MTM) * kMgScw + 2 * i;
+          a.x += ar[0];
+          a.y += ar[1];
+          if (k > 0) {
+            const float* br = sbase + (size_t)w * wstride + (K + k - 1) * kMgScw + 2 * i;
+            bq.x += br[0];
+            bq.y += br[1];
+          }
         }
-        ob[(long long)pm * inner + i] = make_float2(v.x * scale, v.y * scale);
+        ob[(long long)pm * inner + i] = make_float2((a.x - sg * bq.y) * scale, (a.y + sg * bq.x) * scale);
       }
     }
-    __syncwarp();   // the scratch rows are read before the next task's end writes them
+    if (SPLIT) __syncthreads();   // the scratch rows are read before the next task's end writes them
+    else __syncwarp();
   }
 }
 
@@ -235,7 +252,7 @@ midg_contract_kernel(const float2* __restrict__ in, float2* __restrict__ out, lo
 template <bool VEC, bool FAST>
 __global__ void __launch_bounds__(kMgMaxWarps * 32, 1)
 midg_expand_kernel(const float2* __restrict__ in, float2* __restrict__ out, long long outer, long long inner, int N,
-                   int Ng, int off, int K, float scale) {
+                   int Ng, int off, int K, float scale, int tpt) {
   pdl_trigger();
   extern __shared__ float4 mg_smem[];
   const int NM = (N + 15) / 16, KS2 = (2 * K + 7) / 8, VROWS = 8 * KS2;
@@ -261,12 +278,16 @@ midg_expand_kernel(const float2* __restrict__ in, float2* __restrict__ out, long
   __syncthreads();
   pdl_wait();
 
+  // a task: one outer index, one block of positions and `tpt` 16-row tiles of the output (a few tasks per column
+  // block when there are not enough blocks to fill the GPU: a 2-D layer has batch x channels of them)
   const long long CB = (inner + kMgPos - 1) / kMgPos;
-  const long long tasks = outer * CB;
+  const int NRG = (NM + tpt - 1) / tpt;
+  const long long tasks = outer * CB * NRG;
   const long long stride = (long long)W * gridDim.x;
   auto fetch = [&](long long task, int buf) {
     if (task < tasks) {
-      const long long o = task / CB, cb = task - o * CB;
+      const long long ocb = task / NRG;
+      const long long o = ocb / CB, cb = ocb - o * CB;
       const int valid = (int)(inner - cb * kMgPos < kMgPos ? inner - cb * kMgPos : kMgPos);
       const float2* src = in + o * (2 * K) * inner + cb * kMgPos;
       float* dst = Vs + (size_t)buf * VROWS * kMgRowE;
@@ -292,7 +313,9 @@ midg_expand_kernel(const float2* __restrict__ in, float2* __restrict__ out, long
     fetch(t + stride, vb ^ 1);
     mg_wait<1>();
     __syncwarp();
-    const long long o = t / CB, cb = t - o * CB;
+    const long long ocb = t / NRG;
+    const int rg = (int)(t - ocb * NRG);
+    const long long o = ocb / CB, cb = ocb - o * CB;
     const int valid = (int)(inner - cb * kMgPos < kMgPos ? inner - cb * kMgPos : kMgPos);
     {
       // E_0 = V_0, E_k = V_k + V_{-k}; i O_k with O_k = V_k - V_{-k} (k < K), O_K = -V_{-K}; position of -k: 2K - k
@@ -316,8 +339,9 @@ midg_expand_kernel(const float2* __restrict__ in, float2* __restrict__ out, long
 #pragma unroll
       for (int q = 0; q < 2; ++q) lv[nc][q] = Bm[VROWS * kMgRowE + 8 * nc + 2 * t4 + q];
     float2* ob = out + o * N * inner + cb * kMgPos;
+    const int tile_end = (rg + 1) * tpt < NM ? (rg + 1) * tpt : NM;
 #pragma unroll 1
-    for (int tile = 0; tile < NM; ++tile) {
+    for (int tile = rg * tpt; tile < tile_end; ++tile) {
       float P[4][4];
       {
         const float c0 = cK[16 * tile + g8], c1 = cK[16 * tile + g8 + 8];
@@ -386,11 +410,14 @@ cudaError_t launch_contract_t(const float2* in, float2* out, long long outer, lo
                               int K, float scale, bool fast, cudaStream_t st) {
   const MgCfg c = mg_cfg(mg_contract_table(N, MTM), mg_contract_warp(MTM));
   if (c.warps < 2) return cudaErrorInvalidConfiguration;
-  auto kern = fast ? midg_contract_kernel<MTM, VEC, true> : midg_contract_kernel<MTM, VEC, false>;
+  const long long tasks = outer * ((inner + kMgPos - 1) / kMgPos);
+  // fewer tasks than warps on the GPU (and more than one chunk of rows to share): a CTA per task
+  const bool split = tasks < (long long)c.warps * num_sms() && N > kMgChunk;
+  auto kern = split ? (fast ? midg_contract_kernel<MTM, VEC, true, true> : midg_contract_kernel<MTM, VEC, false, true>)
+                    : (fast ? midg_contract_kernel<MTM, VEC, true, false> : midg_contract_kernel<MTM, VEC, false, false>);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
   if (e != cudaSuccess) return e;
-  const long long tasks = outer * ((inner + kMgPos - 1) / kMgPos);
-  const long long want = (tasks + c.warps - 1) / c.warps;
+  const long long want = split ? tasks : (tasks + c.warps - 1) / c.warps;
   const int grid = (int)(want < num_sms() ? want : num_sms());
   (void)launch_pdl(kern, dim3(grid), dim3(c.warps * 32), c.smem, st, in, out, outer, inner, N, Ng, off, K, scale);
   return cudaGetLastError();
@@ -404,10 +431,17 @@ cudaError_t launch_expand_t(const float2* in, float2* out, long long outer, long
   auto kern = fast ? midg_expand_kernel<VEC, true> : midg_expand_kernel<VEC, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
   if (e != cudaSuccess) return e;
-  const long long tasks = outer * ((inner + kMgPos - 1) / kMgPos);
+  // 16-row tiles per task: all of them when there are column blocks enough to fill the GPU twice, else fewer
+  const long long blocks = outer * ((inner + kMgPos - 1) / kMgPos);
+  const int NM = (N + 15) / 16;
+  long long groups = (2ll * c.warps * num_sms() + blocks - 1) / blocks;
+  if (groups > NM) groups = NM;
+  if (groups < 1) groups = 1;
+  const int tpt = (int)((NM + groups - 1) / groups);
+  const long long tasks = blocks * ((NM + tpt - 1) / tpt);
   const long long want = (tasks + c.warps - 1) / c.warps;
   const int grid = (int)(want < num_sms() ? want : num_sms());
-  (void)launch_pdl(kern, dim3(grid), dim3(c.warps * 32), c.smem, st, in, out, outer, inner, N, Ng, off, K, scale);
+  (void)launch_pdl(kern, dim3(grid), dim3(c.warps * 32), c.smem, st, in, out, outer, inner, N, Ng, off, K, scale, tpt);
   return cudaGetLastError();
 }
 
