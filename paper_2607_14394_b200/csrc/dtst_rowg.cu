@@ -214,6 +214,127 @@ rowg_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long
 }
 
 // ---------------------------------------------------------------------------------------------
+// contraction of LONG rows (N3 > 256, e.g. a 421 x 421 grid): tasks of 8 rows, so that a stage is half as large and
+// twice as many warps fit an SM (with 16-row tasks three).  The product runs transposed - [16 frequencies x pairs] x
+// [pairs x 8 rows], as the first stage of planeg_contract_kernel below - and a C fragment holds the frequencies
+// g8 / g8 + 8 of the rows 2 t4, 2 t4 + 1.  MTF: 16-frequency tiles (k3 <= 16 MTF).
+// ---------------------------------------------------------------------------------------------
+template <int MTF, int ST, bool FAST>
+__global__ void __launch_bounds__(kGMaxWarps * 32, 1)
+rowg_contract8_kernel(const float* __restrict__ x, float2* __restrict__ out, long long rows, int N3, int K3, float scale,
+                      int herm, int stage_floats) {
+  pdl_trigger();
+  extern __shared__ float4 rg_smem[];
+  const int H = (N3 + 1) / 2, KS = (H + 7) / 8;
+  float4* atab = rg_smem;                                          // [part][ks][mtf][hi | lo][lane]
+  float* ring = reinterpret_cast<float*>(atab + (size_t)2 * KS * MTF * 2 * 32);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g8 = lane >> 2, t4 = lane & 3;
+  const int W = blockDim.x >> 5;
+
+  for (int e = threadIdx.x; e < 2 * KS * MTF * 32; e += blockDim.x) {
+    const int l = e & 31;
+    int r = e >> 5;
+    const int mtf = r % MTF;
+    r /= MTF;
+    const int ks = r % KS, part = r / KS;
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {                                  // A fragment: frequency l >> 2 (+8), pair l & 3 (+4)
+      const int f = 16 * mtf + (l >> 2) + 8 * (q & 1), j = 8 * ks + (l & 3) + 4 * (q >> 1);
+      split_tf32_rna((f < K3 && j < H) ? g_basis_c(part, f, j, N3) : 0.f, hi[q], lo[q]);
+    }
+    float4* dst = atab + ((size_t)((part * KS + ks) * MTF + mtf) * 2) * 32 + l;
+    dst[0] = make_float4(__uint_as_float(hi[0]), __uint_as_float(hi[1]), __uint_as_float(hi[2]), __uint_as_float(hi[3]));
+    dst[32] = make_float4(__uint_as_float(lo[0]), __uint_as_float(lo[1]), __uint_as_float(lo[2]), __uint_as_float(lo[3]));
+  }
+  float2 rot[MTF][2];                                              // frequencies 16 mtf + g8 (+8)
+#pragma unroll
+  for (int mtf = 0; mtf < MTF; ++mtf)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int f = 16 * mtf + g8 + 8 * h;
+      double sn, cs;
+      sincospi((double)f / (double)N3, &sn, &cs);
+      const float wgt = scale * (herm ? herm_weight(f, N3) : 1.0f);
+      rot[mtf][h] = make_float2((float)cs * wgt, (float)sn * wgt);
+    }
+  __syncthreads();
+  pdl_wait();
+
+  float* S = ring + (size_t)warp * ST * stage_floats;
+  const long long tasks = (rows + 7) / 8;
+  const long long stride = (long long)W * gridDim.x;
+  auto load = [&](long long t, int s) {
+    if (t < tasks) {
+      const long long r0 = t * 8;
+      const long long nr = rows - r0 < 8 ? rows - r0 : 8;
+      const int nf = (int)(nr * N3);
+      const float* src = x + r0 * N3;
+      float* dst = S + (size_t)s * stage_floats;
+      for (int i = lane; i < (nf >> 2); i += 32) g_cp_async16(dst + 4 * i, src + 4 * i);
+      const int done = nf & ~3;
+      if (lane < (nf & 3)) dst[done + lane] = __ldg(src + done + lane);
+    }
+    g_cp_async_commit();
+  };
+  const int jl0 = min(8 * (KS - 1) + t4, H - 1), jl1 = min(8 * (KS - 1) + t4 + 4, H - 1);
+  long long t = (long long)warp * gridDim.x + blockIdx.x;
+#pragma unroll
+  for (int q = 0; q < ST - 1; ++q) load(t + q * stride, q);
+  int s = 0;
+  for (; t < tasks; t += stride, s = s == ST - 1 ? 0 : s + 1) {
+    load(t + (ST - 1) * stride, s == 0 ? ST - 1 : s - 1);
+    g_cp_async_wait<ST - 1>();
+    __syncwarp();
+    const float* Trow = S + (size_t)s * stage_floats + g8 * N3;   // this lane's row (the B operand's n index)
+    float accC[MTF][4], accS[MTF][4];
+#pragma unroll
+    for (int mtf = 0; mtf < MTF; ++mtf)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) accC[mtf][e] = accS[mtf][e] = 0.f;
+    auto step = [&](int ks, int j0, int j1) {
+      const float a0 = Trow[j0], b0 = Trow[N3 - 1 - j0], a1 = Trow[j1], b1 = Trow[N3 - 1 - j1];
+      uint32_t bsh[2], bsl[2], bdh[2], bdl[2];
+      g_split<FAST>(a0 + b0, bsh[0], bsl[0]);
+      g_split<FAST>(a0 - b0, bdh[0], bdl[0]);
+      g_split<FAST>(a1 + b1, bsh[1], bsl[1]);
+      g_split<FAST>(a1 - b1, bdh[1], bdl[1]);
+#pragma unroll
+      for (int mtf = 0; mtf < MTF; ++mtf) {
+        const float4* ac = atab + ((ks * MTF + mtf) * 2) * 32 + lane;
+        const float4* as = atab + (((KS + ks) * MTF + mtf) * 2) * 32 + lane;
+        uint32_t chv[4], clv[4], shv[4], slv[4];
+        g_bits(ac[0], chv);
+        g_bits(ac[32], clv);
+        g_bits(as[0], shv);
+        g_bits(as[32], slv);
+        g_mma3<FAST>(accC[mtf], chv, clv, bsh[0], bsh[1], bsl[0], bsl[1]);
+        g_mma3<FAST>(accS[mtf], shv, slv, bdh[0], bdh[1], bdl[0], bdl[1]);
+      }
+    };
+#pragma unroll 2
+    for (int ks = 0; ks < KS - 1; ++ks) step(ks, 8 * ks + t4, 8 * ks + t4 + 4);
+    step(KS - 1, jl0, jl1);
+    // X_f = rot_f (C_f - i S_f): frequency 16 mtf + g8 + 8 h of the rows 2 t4 + q
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const long long row = t * 8 + 2 * t4 + q;
+      if (row >= rows) continue;
+#pragma unroll
+      for (int mtf = 0; mtf < MTF; ++mtf)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int f = 16 * mtf + g8 + 8 * h;
+          const float C = accC[mtf][2 * h + q], Sv = accS[mtf][2 * h + q];
+          if (f < K3)
+            out[row * K3 + f] = make_float2(rot[mtf][h].x * C + rot[mtf][h].y * Sv, rot[mtf][h].y * C - rot[mtf][h].x * Sv);
+        }
+    }
+    __syncwarp();   // every lane is done with this stage before it is filled again
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // expansion.  y_j = P_j - Q_j, y_{N3-1-j} = P_j + Q_j with P_j = sum_f Re z'_f cos theta_{f,j},
 // Q_j = sum_f Im z'_f sin theta_{f,j}, z'_f = scale c_f e^{-i pi f / N3} in_f.  MT m-tiles of 16 rows per task,
 // KSF k-steps of 8 frequencies (k3 <= 8 KSF).
@@ -816,6 +937,34 @@ cudaError_t launch_contract_t(const float* x, float2* out, long long rows, int N
                                                           : launch_contract_s<MT, NT, 2>(x, out, rows, N3, K3, scale, herm, fast, st);
 }
 
+template <int MTF, int ST>
+cudaError_t launch_contract8_s(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm, bool fast,
+                               cudaStream_t st) {
+  const int H = (N3 + 1) / 2, KS = (H + 7) / 8;
+  const int sf = (8 * N3 + 3) & ~3;
+  const GCfg c = g_cfg((size_t)2 * KS * MTF * 2 * 32 * 16, (size_t)ST * sf * 4);
+  if (c.warps < 2) return cudaErrorInvalidConfiguration;
+  auto kern = fast ? rowg_contract8_kernel<MTF, ST, true> : rowg_contract8_kernel<MTF, ST, false>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem);
+  if (e != cudaSuccess) return e;
+  const long long tasks = (rows + 7) / 8;
+  const long long want = (tasks + c.warps - 1) / c.warps;
+  const int grid = (int)(want < num_sms() ? want : num_sms());
+  (void)launch_pdl(kern, dim3(grid), dim3(c.warps * 32), c.smem, st, x, out, rows, N3, K3, scale, herm, sf);
+  return cudaGetLastError();
+}
+
+template <int MTF>
+cudaError_t launch_contract8_t(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm, bool fast,
+                               cudaStream_t st) {
+  const int H = (N3 + 1) / 2, KS = (H + 7) / 8;
+  const size_t sb = (size_t)((8 * N3 + 3) & ~3) * 4, table = (size_t)2 * KS * MTF * 2 * 32 * 16;
+  // long rows leave room for few warps: three stages only where eight warps of them fit, else two stages and more warps
+  const bool three = g_cfg(table, 3 * sb).warps >= 8 || g_cfg(table, 2 * sb).warps <= g_cfg(table, 3 * sb).warps;
+  return three ? launch_contract8_s<MTF, 3>(x, out, rows, N3, K3, scale, herm, fast, st)
+               : launch_contract8_s<MTF, 2>(x, out, rows, N3, K3, scale, herm, fast, st);
+}
+
 template <int MT, int KSF>
 cudaError_t launch_expand_t(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm, bool fast,
                             cudaStream_t st) {
@@ -944,6 +1093,9 @@ cudaError_t launch_rowg_contract(const float* x, float2* out, long long rows, in
                                  cudaStream_t st) {
   const int NT = (K3 + 7) / 8;
   const bool two = g_mt(N3) == 2;
+  if (N3 > 256)   // long rows: 8-row tasks
+    return K3 <= 16 ? launch_contract8_t<1>(x, out, rows, N3, K3, scale, herm, fast, st)
+                    : launch_contract8_t<2>(x, out, rows, N3, K3, scale, herm, fast, st);
   switch (NT) {
     case 1: return two ? launch_contract_t<2, 1>(x, out, rows, N3, K3, scale, herm, fast, st)
                        : launch_contract_t<1, 1>(x, out, rows, N3, K3, scale, herm, fast, st);

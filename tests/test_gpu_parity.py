@@ -406,6 +406,7 @@ ANY_EXTENT = [
     ("g_k3_odd", 1, 2, 2, (32, 50), (8, 9), False),                  # odd mode count: 8-byte stores
     ("g_1d", 2, 3, 2, (90,), (17,), True),
     ("g_512", 1, 2, 2, (8, 512), (4, 16), True),                     # longer than the tensor-map kernels take
+    ("g_421", 1, 3, 2, (45, 421), (12, 12), True),                   # long odd rows (8-row tasks), 135 rows: ragged
     # the second-last dimension inside the kernel: 24 and 32 modes (two mode tiles), 8 modes (half a tile), few
     # frequencies (two column tiles), 16-row tasks, and more planes than warps on the GPU (the ring crosses planes)
     ("g_plane_k2_12", 1, 2, 2, (16, 64, 60), (4, 12, 16), True),
