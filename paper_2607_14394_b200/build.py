@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdtst.so")
-SOURCES = ["dtst_api.cu", "dtst_generic.cu", "dtst_fused.cu", "dtst_plane_inst_a.cu", "dtst_plane_inst_b.cu", "dtst_plane_inst_c.cu", "dtst_plane_inst_d.cu", "dtst_row.cu", "dtst_rowg.cu", "dtst_mid.cu", "dtst_midg.cu", "dtst_midmma.cu", "dtst_slab.cu", "dtst_static.cu", "dtst_block.cu", "dtst_block_umma.cu", "dtst_block_mma.cu", "dtst_hostio.cu"]
+SOURCES = ["dtst_api.cu", "dtst_generic.cu", "dtst_fused.cu", "dtst_plane_inst_a.cu", "dtst_plane_inst_b.cu", "dtst_plane_inst_c.cu", "dtst_plane_inst_d.cu", "dtst_row.cu", "dtst_rowg.cu", "dtst_rowl.cu", "dtst_mid.cu", "dtst_midg.cu", "dtst_midmma.cu", "dtst_slab.cu", "dtst_static.cu", "dtst_block.cu", "dtst_block_umma.cu", "dtst_block_mma.cu", "dtst_hostio.cu"]
 HEADERS = ["dtst_common.cuh", "dtst_fused.cuh", "dtst_plane.cuh", "dtst_sm100.cuh", "dtst_mma.cuh", os.path.join("..", "..", "include", "dtst.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

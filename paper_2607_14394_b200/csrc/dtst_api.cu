@@ -131,7 +131,8 @@ bool use_row(const dtst_plan* p) {
   long long rows = (long long)p->B * (p->C_in > p->C_out ? p->C_in : p->C_out);
   for (int i = 0; i < a; ++i) rows *= p->Nl[i];
   if (row_supported((int)p->Ng[a], p->kmax[a])) return rows < (1ll << 31);   // 32-bit TMA coordinates
-  return rowg_supported((int)p->Ng[a], p->kmax[a]);   // any extent: the cp.async-fed kernels of dtst_rowg.cu
+  // any extent up to 512: the cp.async-fed kernels of dtst_rowg.cu; longer rows: the chunked ones of dtst_rowl.cu
+  return rowg_supported((int)p->Ng[a], p->kmax[a]) || rowl_supported((int)p->Ng[a], p->kmax[a]);
 }
 
 // Row path with the second-last dimension inside the grid-side kernel (dtst_rowg.cu): for contiguous extents the
@@ -543,7 +544,11 @@ dtst_status run_forward_row(dtst_plan* p, const float* x, float2* Xhat, int Cn, 
     const cudaError_t e = row_supported((int)p->Ng[a], p->kmax[a])
                               ? launch_row_contract(x, t1, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0,
                                                     reinterpret_cast<int*>(ws + L.status), st)
-                              : launch_rowg_contract(x, t1, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, p->fast_math != 0, st);
+                          : rowg_supported((int)p->Ng[a], p->kmax[a])
+                              ? launch_rowg_contract(x, t1, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0,
+                                                     p->fast_math != 0, st)
+                              : launch_rowl_contract(x, t1, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0,
+                                                     p->fast_math != 0, st);
     if (cuda_failed(p, e)) return DTST_ERR_CUDA;
   }
   ++p->launches;
@@ -573,7 +578,11 @@ dtst_status run_inverse_row(dtst_plan* p, const float2* Yhat, float* y, int Cn, 
   }
   const cudaError_t e = row_supported((int)p->Ng[a], p->kmax[a])
                             ? launch_row_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, st)
-                            : launch_rowg_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0, p->fast_math != 0, st);
+                        : rowg_supported((int)p->Ng[a], p->kmax[a])
+                            ? launch_rowg_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0,
+                                                 p->fast_math != 0, st)
+                            : launch_rowl_expand(src, y, rows, (int)p->Ng[a], p->kmax[a], scale, herm ? 1 : 0,
+                                                 p->fast_math != 0, st);
   if (cuda_failed(p, e)) return DTST_ERR_CUDA;
   ++p->launches;
   return DTST_OK;

@@ -58,6 +58,12 @@ cudaError_t launch_rowg_contract(const float* x, float2* out, long long rows, in
                                  cudaStream_t st);
 cudaError_t launch_rowg_expand(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm, bool fast,
                                cudaStream_t st);
+// Row kernels for long contiguous extents (dtst_rowl.cu): 512 < N3 <= 16384, N3 % 16 == 0, k3 <= 32.
+bool rowl_supported(int N3, int K3);
+cudaError_t launch_rowl_contract(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm, bool fast,
+                                 cudaStream_t st);
+cudaError_t launch_rowl_expand(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm, bool fast,
+                               cudaStream_t st);
 // The same with the dimension in front (extent N2, whole, no offset, K2 modes per side) inside the kernel:
 // x[planes][N2][N3] <-> [planes][2 K2][k3].
 bool planeg_supported(int N3, int K3, int N2, int K2);

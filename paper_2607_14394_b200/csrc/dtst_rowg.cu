@@ -287,11 +287,24 @@ rowg_contract8_kernel(const float* __restrict__ x, float2* __restrict__ out, lon
     g_cp_async_wait<ST - 1>();
     __syncwarp();
     const float* Trow = S + (size_t)s * stage_floats + g8 * N3;   // this lane's row (the B operand's n index)
-    float accC[MTF][4], accS[MTF][4];
+    // accC / accS: the running sums; cC / cS: the sums of up to eight k-steps, added to them with ordinary fp32
+    // additions (the tensor core's accumulate step truncates: one chain through all k-steps of a 512-point row cost
+    // half of the error budget)
+    float accC[MTF][4], accS[MTF][4], cC[MTF][4], cS[MTF][4];
 #pragma unroll
     for (int mtf = 0; mtf < MTF; ++mtf)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) accC[mtf][e] = accS[mtf][e] = 0.f;
+      for (int e = 0; e < 4; ++e) accC[mtf][e] = accS[mtf][e] = cC[mtf][e] = cS[mtf][e] = 0.f;
+    auto flush = [&]() {
+#pragma unroll
+      for (int mtf = 0; mtf < MTF; ++mtf)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          accC[mtf][e] += cC[mtf][e];
+          accS[mtf][e] += cS[mtf][e];
+          cC[mtf][e] = cS[mtf][e] = 0.f;
+        }
+    };
     auto step = [&](int ks, int j0, int j1) {
       const float a0 = Trow[j0], b0 = Trow[N3 - 1 - j0], a1 = Trow[j1], b1 = Trow[N3 - 1 - j1];
       uint32_t bsh[2], bsl[2], bdh[2], bdl[2];
@@ -308,13 +321,18 @@ rowg_contract8_kernel(const float* __restrict__ x, float2* __restrict__ out, lon
         g_bits(ac[32], clv);
         g_bits(as[0], shv);
         g_bits(as[32], slv);
-        g_mma3<FAST>(accC[mtf], chv, clv, bsh[0], bsh[1], bsl[0], bsl[1]);
-        g_mma3<FAST>(accS[mtf], shv, slv, bdh[0], bdh[1], bdl[0], bdl[1]);
+        g_mma3<FAST>(cC[mtf], chv, clv, bsh[0], bsh[1], bsl[0], bsl[1]);
+        g_mma3<FAST>(cS[mtf], shv, slv, bdh[0], bdh[1], bdl[0], bdl[1]);
       }
     };
+    for (int k0 = 0; k0 < KS - 1; k0 += 8) {
+      const int k1 = k0 + 8 < KS - 1 ? k0 + 8 : KS - 1;
 #pragma unroll 2
-    for (int ks = 0; ks < KS - 1; ++ks) step(ks, 8 * ks + t4, 8 * ks + t4 + 4);
+      for (int ks = k0; ks < k1; ++ks) step(ks, 8 * ks + t4, 8 * ks + t4 + 4);
+      flush();
+    }
     step(KS - 1, jl0, jl1);
+    flush();
     // X_f = rot_f (C_f - i S_f): frequency 16 mtf + g8 + 8 h of the rows 2 t4 + q
 #pragma unroll
     for (int q = 0; q < 2; ++q) {

@@ -447,6 +447,29 @@ def test_any_middle_extent_and_mode_count_runs_on_folded_kernels(case):
         run_layer_and_check(w, "auto", P=4)
 
 
+# ------------------------------------------------------------------ long contiguous extents (chunked row kernels)
+LONG_ROWS = [
+    # name, B, Ci, Co, N, kmax
+    ("l_1d_8192", 2, 3, 2, (8192,), (16,)),                 # a long 1-D signal: 64 chunks of 64 pairs
+    ("l_1d_1040_ragged", 1, 3, 1, (1040,), (32,)),          # 65 k-steps: a last chunk of one k-step; 3 rows; 32 modes
+    ("l_2d_1024", 1, 1, 2, (24, 1024), (8, 12)),            # 24 rows per channel, k3 = 12 (frequencies past k3 idle)
+    ("l_3d_528", 1, 2, 1, (6, 10, 528), (2, 4, 20)),        # three 8-frequency k-steps in the expansion
+    ("l_1d_16384_k3", 1, 2, 2, (16384,), (3,)),              # the longest row, a few frequencies of one tile
+]
+
+
+@pytest.mark.parametrize("case", LONG_ROWS, ids=[c[0] for c in LONG_ROWS])
+def test_long_rows_run_on_the_chunked_row_kernels(case):
+    name, B, Ci, Co, N, k = case
+    w = I.custom_workload(name, B, Ci, Co, N, k, field="grf", seed=43)
+    plan = _plan(w)
+    assert plan.kernel_path == "row"
+    plan.require_fast_path()
+    plan.close()
+    run_layer_and_check(w, "auto")
+    run_layer_and_check(w, "auto", tol=2e-3, fine_scale=200.0, arithmetic="tf32")
+
+
 @pytest.mark.parametrize("case", ANY_EXTENT, ids=[c[0] for c in ANY_EXTENT])
 def test_any_contiguous_extent_runs_on_the_row_kernels(case):
     name, B, Ci, Co, N, k, streaming = case
