@@ -61,7 +61,7 @@ enum {
   DTST_PATH_AUTO = 0,      /* fused streaming kernels where the shape allows, else generic */
   DTST_PATH_GENERIC = 1,   /* one generic contraction kernel per dimension                 */
   DTST_PATH_ROW = 2        /* reported only: streaming kernel on the contiguous dimension (any extent up to 512,
-                              odd ones included, and multiples of 16 up to 16384; up to 32 one-sided modes; with the
+                              odd ones included, and multiples of 8 up to 16384; up to 32 one-sided modes; with the
                               dimension in front of it inside
                               the same kernel where its extent is a multiple of 16 - 32 for extents up to 64 - and at
                               most 256), folded kernels on the others (shapes without a two-dimension tensor-map kernel) */

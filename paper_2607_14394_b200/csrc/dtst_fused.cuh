@@ -58,7 +58,7 @@ cudaError_t launch_rowg_contract(const float* x, float2* out, long long rows, in
                                  cudaStream_t st);
 cudaError_t launch_rowg_expand(const float2* in, float* y, long long rows, int N3, int K3, float scale, int herm, bool fast,
                                cudaStream_t st);
-// Row kernels for long contiguous extents (dtst_rowl.cu): 512 < N3 <= 16384, N3 % 16 == 0, k3 <= 32.
+// Row kernels for long contiguous extents (dtst_rowl.cu): 512 < N3 <= 16384, N3 % 8 == 0, k3 <= 32.
 bool rowl_supported(int N3, int K3);
 cudaError_t launch_rowl_contract(const float* x, float2* out, long long rows, int N3, int K3, float scale, int herm, bool fast,
                                  cudaStream_t st);

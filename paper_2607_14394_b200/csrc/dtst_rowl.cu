@@ -1,11 +1,12 @@
-// Row kernels for LONG contiguous extents (512 < N3 <= 16384, N3 a multiple of 16, up to 32 one-sided modes): the
+// Row kernels for LONG contiguous extents (512 < N3 <= 16384, N3 a multiple of 8, up to 32 one-sided modes): the
 // contiguous (rfft) dimension alone - a 1-D signal of 8192 points, a 1024 x 1024 grid.  Same fold and same TF32x3
 // products as dtst_rowg.cu (X_f = e^{i pi f/N3} (sum_j s_j cos theta_fj - i sum_j d_j sin theta_fj), s_j, d_j =
 // x_j +- x_{N3-1-j}, theta_fj = 2 pi f (j + 1/2) / N3), but a row no longer fits a warp's share of the shared memory
 // and its basis no table:
 //   * a task is 8 rows, streamed in CHUNKS of 64 pairs: the 64 columns from the left and the 64 mirrored columns
-//     from the right (two 256-byte segments per row, 16-byte aligned because N3 is a multiple of 4), through a
-//     per-warp cp.async ring of 4 KB stages - 16 warps per SM whatever N3 is;
+//     from the right (two 256-byte segments per row, 16-byte aligned because N3 is a multiple of 4; the last chunk
+//     may be shorter, a multiple of 4 pairs), through a per-warp cp.async ring of 4 KB stages - 16 warps per SM
+//     whatever N3 is;
 //   * the basis of chunk c is the product of two small exact tables, e^{i theta} = T1[f][j - 64 c] * T2[c][f] with
 //     T1 = e^{2 pi i f (jl + 1/2) / N3} (32 x 64 entries) and T2 = e^{2 pi i f 64 c / N3} (one row per chunk), both
 //     built once per CTA from integer-reduced phases in double precision: one complex multiplication per entry, no
@@ -82,7 +83,7 @@ rowl_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long
                      int herm) {
   pdl_trigger();
   extern __shared__ float4 rl_smem[];
-  const int KS = N3 / 16, NCK = (KS + 7) / 8;                       // k-steps of 8 pairs, chunks of 8 k-steps
+  const int H = N3 / 2, NCK = (H + kLPairs - 1) / kLPairs;          // pairs, chunks of 64 pairs (the last: H - 64 c, a multiple of 4)
   float2* T1 = reinterpret_cast<float2*>(rl_smem);
   float2* T2 = T1 + kLMaxF * kLT1;
   float* ring = reinterpret_cast<float*>(T2 + (size_t)NCK * kLMaxF);
@@ -117,15 +118,15 @@ rowl_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long
     if (at < tasks) {
       const long long r0 = at * 8;
       const int nr = (int)(rows - r0 < 8 ? rows - r0 : 8);
-      const int nk = KS - 8 * ac < 8 ? KS - 8 * ac : 8;             // k-steps of this chunk: 8 nk floats per segment
+      const int L = H - kLPairs * ac < kLPairs ? H - kLPairs * ac : kLPairs;   // pairs of this chunk = floats per segment
       const float* src = x + r0 * N3;
       float* dst = S + (size_t)s * kLStage;
-      const int ppr = 2 * nk;                                       // 16-byte pieces per segment
+      const int ppr = L >> 2;                                       // 16-byte pieces per segment
       for (int i = lane; i < nr * 2 * ppr; i += 32) {
         const int r = i / (2 * ppr), q = i - r * 2 * ppr;
         if (q < ppr) l_cp_async16(dst + r * kLRow + 4 * q, src + (long long)r * N3 + kLPairs * ac + 4 * q);
-        else l_cp_async16(dst + r * kLRow + 128 - 8 * nk + 4 * (q - ppr),
-                          src + (long long)r * N3 + N3 - kLPairs * ac - 8 * nk + 4 * (q - ppr));
+        else l_cp_async16(dst + r * kLRow + 128 - L + 4 * (q - ppr),
+                          src + (long long)r * N3 + N3 - kLPairs * ac - L + 4 * (q - ppr));
       }
     }
     l_cp_async_commit();
@@ -149,7 +150,8 @@ rowl_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long
       l_cp_async_wait<kLStages - 1>();
       __syncwarp();
       const float* Trow = S + (size_t)s * kLStage + g8 * kLRow;     // this lane's row (the 8-wide operand's n index)
-      const int nk = KS - 8 * c < 8 ? KS - 8 * c : 8;
+      const int L = H - kLPairs * c < kLPairs ? H - kLPairs * c : kLPairs;
+      const int nk = (L + 7) >> 3;                                  // k-steps; the last may hold 4 pairs only
       float2 t2[MTF][2];
 #pragma unroll
       for (int mtf = 0; mtf < MTF; ++mtf)
@@ -166,7 +168,9 @@ rowl_contract_kernel(const float* __restrict__ x, float2* __restrict__ out, long
 #pragma unroll 2
       for (int kk = 0; kk < nk; ++kk) {
         const int jl = 8 * kk + t4;
-        const float a0 = Trow[jl], b0 = Trow[127 - jl], a1 = Trow[jl + 4], b1 = Trow[123 - jl];
+        const float a0 = Trow[jl], b0 = Trow[127 - jl];
+        const bool v1 = jl + 4 < L;                                 // pairs past the chunk's end (only t4 + 4 can be) count zero
+        const float a1 = v1 ? Trow[jl + 4] : 0.f, b1 = v1 ? Trow[123 - jl] : 0.f;
         uint32_t bsh[2], bsl[2], bdh[2], bdl[2];
         l_split<FAST>(a0 + b0, bsh[0], bsl[0]);
         l_split<FAST>(a0 - b0, bdh[0], bdl[0]);
@@ -249,7 +253,7 @@ rowl_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long lo
                    int herm, int cpt) {
   pdl_trigger();
   extern __shared__ float4 rl_smem[];
-  const int KS = N3 / 16, NCK = (KS + 7) / 8;
+  const int H = N3 / 2, NCK = (H + kLPairs - 1) / kLPairs;
   float2* T1 = reinterpret_cast<float2*>(rl_smem);
   float2* T2 = T1 + kLMaxF * kLT1;
   float* stg = reinterpret_cast<float*>(T2 + (size_t)NCK * kLMaxF);
@@ -305,14 +309,14 @@ rowl_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long lo
     const int nr = (int)(rows - r0 < 8 ? rows - r0 : 8);
     const int c_end = (cg + 1) * cpt < NCK ? (cg + 1) * cpt : NCK;
     for (int c = cg * cpt; c < c_end; ++c) {
-      const int nk = KS - 8 * c < 8 ? KS - 8 * c : 8;               // 8 nk pairs in this chunk
+      const int L = H - kLPairs * c < kLPairs ? H - kLPairs * c : kLPairs;   // pairs of this chunk
       float2 t2[KSF][2];
 #pragma unroll
       for (int ks = 0; ks < KSF; ++ks)
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) t2[ks][hf] = T2[c * kLMaxF + 8 * ks + t4 + 4 * hf];
 #pragma unroll 1
-      for (int mtj = 0; 16 * mtj < 8 * nk; ++mtj) {                 // 16 pairs per product
+      for (int mtj = 0; 16 * mtj < L; ++mtj) {                      // 16 pairs per product
         float P[4] = {0.f, 0.f, 0.f, 0.f}, Q[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int ks = 0; ks < KSF; ++ks) {
@@ -342,15 +346,15 @@ rowl_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long lo
       __syncwarp();
       {
         float* dst = y + r0 * N3;
-        const int ppr = 2 * nk;
+        const int ppr = L >> 2;
         for (int i = lane; i < nr * 2 * ppr; i += 32) {
           const int r = i / (2 * ppr), q = i - r * 2 * ppr;
           if (q < ppr)
             __stcs(reinterpret_cast<float4*>(dst + (long long)r * N3 + kLPairs * c + 4 * q),
                    *reinterpret_cast<const float4*>(st + r * kLRow + 4 * q));
           else
-            __stcs(reinterpret_cast<float4*>(dst + (long long)r * N3 + N3 - kLPairs * c - 8 * nk + 4 * (q - ppr)),
-                   *reinterpret_cast<const float4*>(st + r * kLRow + 128 - 8 * nk + 4 * (q - ppr)));
+            __stcs(reinterpret_cast<float4*>(dst + (long long)r * N3 + N3 - kLPairs * c - L + 4 * (q - ppr)),
+                   *reinterpret_cast<const float4*>(st + r * kLRow + 128 - L + 4 * (q - ppr)));
         }
       }
       __syncwarp();   // the staging area is read out before the next chunk writes to it
@@ -359,7 +363,7 @@ rowl_expand_kernel(const float2* __restrict__ in, float* __restrict__ y, long lo
 }
 
 size_t l_table_bytes(int N3) {
-  const int KS = N3 / 16, NCK = (KS + 7) / 8;
+  const int NCK = (N3 / 2 + kLPairs - 1) / kLPairs;
   return ((size_t)kLMaxF * kLT1 + (size_t)NCK * kLMaxF) * sizeof(float2);
 }
 int l_warps(size_t table, size_t per_warp) {
@@ -399,7 +403,7 @@ cudaError_t launch_expand_t(const float2* in, float* y, long long rows, int N3, 
   if (e != cudaSuccess) return e;
   // chunks per task: all of them when there are row blocks enough to fill the GPU twice, else fewer
   const long long blocks = (rows + 7) / 8;
-  const int NCK = (N3 / 16 + 7) / 8;
+  const int NCK = (N3 / 2 + kLPairs - 1) / kLPairs;
   long long groups = (2ll * w * num_sms() + blocks - 1) / blocks;
   if (groups > NCK) groups = NCK;
   if (groups < 1) groups = 1;
@@ -414,7 +418,7 @@ cudaError_t launch_expand_t(const float2* in, float* y, long long rows, int N3, 
 }  // namespace
 
 bool rowl_supported(int N3, int K3) {
-  if (N3 <= 512 || N3 > 16384 || N3 % 16 != 0 || K3 < 1 || K3 > 32 || K3 > N3 / 2 + 1) return false;
+  if (N3 <= 512 || N3 > 16384 || N3 % 8 != 0 || K3 < 1 || K3 > 32 || K3 > N3 / 2 + 1) return false;
   return l_warps(l_table_bytes(N3), (size_t)kLStages * kLStage * 4 + 2 * 8 * 32 * 4) >= 4;
 }
 

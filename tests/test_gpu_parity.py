@@ -455,6 +455,8 @@ LONG_ROWS = [
     ("l_2d_1024", 1, 1, 2, (24, 1024), (8, 12)),            # 24 rows per channel, k3 = 12 (frequencies past k3 idle)
     ("l_3d_528", 1, 2, 1, (6, 10, 528), (2, 4, 20)),        # three 8-frequency k-steps in the expansion
     ("l_1d_16384_k3", 1, 2, 2, (16384,), (3,)),              # the longest row, a few frequencies of one tile
+    ("l_2d_600", 1, 2, 2, (16, 600), (4, 16)),              # 300 pairs: a last chunk of 44 (its last k-step half full)
+    ("l_1d_1000", 2, 2, 1, (1000,), (20,)),                 # 500 pairs: a last chunk of 52
 ]
 
 
