@@ -66,6 +66,11 @@ WORKLOADS = {
 EXTRA_WORKLOADS = {
     "paper_4d_t30": Workload("paper_4d_t30", 1, 20, 20, (128, 128, 64, 30), (8, 8, 8, 16), "grf", 1006),
     "paper_4d_t32": Workload("paper_4d_t32", 1, 20, 20, (128, 128, 64, 32), (8, 8, 8, 16), "grf", 1007),
+    # shapes of the usual 1-D and 2-D operator-learning problems (long rows, many batch entries, few modes): seeded
+    # synthetic fields of these shapes, as everywhere
+    "signal_1d_8192": Workload("signal_1d_8192", 20, 64, 64, (8192,), (16,), "grf", 1008),
+    "grid_2d_1024": Workload("grid_2d_1024", 4, 32, 32, (1024, 1024), (12, 12), "grf", 1009),
+    "grid_2d_421": Workload("grid_2d_421", 4, 32, 32, (421, 421), (12, 12), "grf", 1010),
 }
 
 
