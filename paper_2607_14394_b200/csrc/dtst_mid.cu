@@ -361,6 +361,10 @@ cudaError_t launch_mid(bool forward, int K, const float2* in, float2* out, long 
   const bool aligned16 = ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
   if (aligned16 && mid_mma_supported(N, K, inner)) return launch_mid_mma(forward, K, in, out, outer, inner, N, scale, st);
   if (!mid_ffma_supported(N, K)) return launch_midg(forward, K, in, out, outer, inner, N, scale, fast, st);
+  // The kernels below run one thread per two positions: a tensor with few of them (a 2-D layer: batch x channels x
+  // k3) leaves most of the GPU idle (4 x 32 x 1024 x 12: six CTAs, 147 us); the kernels for any extent split such a
+  // tensor along the contracted dimension as well.
+  if (outer * inner < 65536 && midg_supported(N, K)) return launch_midg(forward, K, in, out, outer, inner, N, scale, fast, st);
   // two adjacent positions per thread need an even inner extent (then every pair is 16-byte aligned and
   // never straddles two outer slices) and 16-byte aligned tensors
   const bool vec = (inner % 2 == 0) && ((reinterpret_cast<uintptr_t>(in) | reinterpret_cast<uintptr_t>(out)) & 15u) == 0;
