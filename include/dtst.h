@@ -189,9 +189,9 @@ dtst_status dtst_plan_set_column_expansion(dtst_plan* plan, int ring_columns);
 dtst_status dtst_plan_set_column_contraction(dtst_plan* plan, int mode);
 
 /*
- * Arithmetic of the tensor-core stages of the kernels for contiguous extents that are no multiple of 32 and for
- * middle dimensions of any extent and mode count (the paper's own layer, time axis 30, runs on them; they are bound by
- * their arithmetic, not by HBM):
+ * Arithmetic of the tensor-core stages of the kernels for contiguous extents that are no multiple of 32 or longer than
+ * 256 points and for middle dimensions of any extent and mode count (the paper's own layer, time axis 30, runs on
+ * them; they are bound by their arithmetic, not by HBM):
  *   DTST_ARITH_TF32X3  (default) every product as three TF32 products of hi/lo operand parts with fp32
  *                      accumulation: rel-L2 of each output tensor against the float64 statement <= 1e-5
  *                      (measured 1e-6..2e-6);
